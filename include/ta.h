@@ -1,0 +1,343 @@
+/*
+ * ta.h - C ABI of the trace-window analyzer (single NVIDIA B200, sm_100a).
+ *
+ * The library rebuilds operator executions and cross-process dependencies from
+ * one or more bounded profiling windows of host-operator, host-API, launch,
+ * kernel, memcpy and collective events.  It implements the reconstruction
+ * stage of the paper's Analyzer (Sec. 6.1 "Deriving Performance Observations",
+ * Fig. "Key performance observations" (a) and (e)), fed by the record model of
+ * Sec. 5.2 "Cross-Layer Profiling Collection".  The paper states the problem;
+ * it gives no algorithm, so every rule below that is not followed by a
+ * citation is this library's own reading and is stated in full.
+ *
+ * General conventions
+ *   - All times are int64 nanoseconds, all ids are integers; nothing on the
+ *     path is floating point.
+ *   - Every entry point returns a ta_status; nothing throws, aborts or traps.
+ *     After any error the handle stays valid for ta_free().
+ *   - "device" pointers live in the memory of env.device, "host" pointers are
+ *     ordinary host memory.  Result structs are filled with device pointers
+ *     OWNED BY THE HANDLE (valid until ta_free) and host scalars.  Host-side
+ *     per-window summary arrays are CALLER-OWNED, W entries, and are filled
+ *     after one stream synchronisation at the end of the call.
+ *   - Every kernel is enqueued on env.cuda_stream.
+ *   - "Sorted position" p in [0, n) always means a position in the canonical
+ *     order produced by ta_sort_timeline; every per-event output of the later
+ *     calls is indexed by sorted position.
+ *   - Call order: load -> sort -> { correlate -> attribute ; gaps ;
+ *     aggregate(value_sel 0) ; collectives }.  aggregate(value_sel 1) needs
+ *     attribute.  A call made too early returns TA_ERR_ORDER.
+ */
+#ifndef TA_H
+#define TA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- record model (Sec. 5.2: call function / thread / entry+return times;
+ * host API intervals; device activity; correlation id; device and stream ids)
+ * 40-byte little-endian record.                                             */
+typedef struct ta_event {
+  int64_t ts_start; /* entry / start time, ns                                */
+  int64_t ts_end;   /* return / completion time, ns, >= ts_start             */
+  int64_t corr_id;  /* LAUNCH,KERNEL,MEMCPY: correlation id (per process);
+                       COLL: communicator id; otherwise ignored              */
+  int32_t pid;      /* process id (signed compare)                           */
+  int32_t name_id;  /* symbol id of the function / kernel                    */
+  int32_t seq;      /* COLL: sequence number inside the communicator         */
+  int16_t stream;   /* host kinds: host thread index; device kinds: stream   */
+  int16_t kind;     /* TA_KIND_*                                             */
+} ta_event;
+
+enum {
+  TA_KIND_OP = 0,     /* host: operator / Python call range                  */
+  TA_KIND_API = 1,    /* host: accelerator API call other than a launch      */
+  TA_KIND_LAUNCH = 2, /* host: submission API call                           */
+  TA_KIND_KERNEL = 3, /* device: kernel execution                            */
+  TA_KIND_MEMCPY = 4, /* device: memory operation                            */
+  TA_KIND_COLL = 5    /* device: collective                                  */
+};
+#define TA_N_KINDS 6
+#define TA_NBINS 40     /* log2 histogram bins; bin 39 collects >= 2^39 ns   */
+#define TA_MAX_DEPTH 8  /* deepest legal nesting of OP ranges                */
+
+typedef enum ta_status {
+  TA_OK = 0,
+  TA_ERR_INVALID_ARG = 1,
+  TA_ERR_OOM = 2,        /* env.alloc returned NULL                          */
+  TA_ERR_CUDA = 3,       /* a CUDA runtime call failed                       */
+  TA_ERR_ORDER = 4,      /* entry point called before its prerequisites      */
+  TA_ERR_TOO_LARGE = 5,  /* a documented size limit was exceeded             */
+  TA_ERR_OVERFLOW = 6,   /* an internal bounded table filled up              */
+  TA_ERR_TIMEOUT = 7,    /* a bounded device-side wait gave up               */
+  TA_ERR_DEPTH = 8,      /* some host event has more than TA_MAX_DEPTH enclosing OPs */
+  TA_ERR_BAD_NESTING = 9 /* two ranges of one host thread overlap partially  */
+} ta_status;
+
+/* Caller-supplied device memory and stream.  alloc returns device memory on
+ * `device` aligned to at least 256 bytes, or NULL; release takes it back.  If
+ * alloc is NULL the library uses the device's stream-ordered pool. */
+typedef struct ta_env {
+  void *(*alloc)(size_t bytes, void *ctx);
+  void (*release)(void *ptr, void *ctx);
+  void *ctx;
+  void *cuda_stream; /* cudaStream_t */
+  int32_t device;
+} ta_env;
+
+typedef struct ta_window ta_window; /* opaque handle; owns every result buffer */
+
+/* ------------------------------------------------------------------------
+ * ta_load_window - ingest and validate (start-time filtering separates
+ * successive windows, Sec. 5.2 "Session transitions").
+ *
+ * events   n records, device memory if events_on_device else host memory
+ *          (then copied to the device first).  BORROWED: must stay alive and
+ *          unmodified until ta_sort_timeline has returned; never freed here.
+ * win_off  host, W+1 ascending offsets, win_off[0]=0, win_off[W]=n.  Record k
+ *          belongs to window w iff win_off[w] <= k < win_off[w+1].
+ * win_t0/1 host, W entries, t0 < t1, t1 - t0 < 2^40.
+ * A record is DROPPED by the first rule that applies:
+ *   kind outside [0,5]            -> n_bad_kind
+ *   ts_end < ts_start             -> n_bad_interval
+ *   ts_start < t0 or >= t1        -> n_out_of_window
+ * (ts_end > t1 is legal.)  Dropped records take part in nothing but `perm`.
+ * Limits: n < 2^31; at most 4096 distinct (pid, domain, stream) triples; the
+ * sort key (window, triple, ts_start - t0) must fit 63 bits.
+ * out_summary: host, W entries, caller-owned.
+ * Errors: INVALID_ARG (null pointers, bad offsets, t0 >= t1), TOO_LARGE, OOM, CUDA.
+ */
+typedef struct ta_load_summary {
+  int64_t n_events, n_valid, n_bad_kind, n_bad_interval, n_out_of_window;
+} ta_load_summary;
+
+ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
+                         int32_t events_on_device, const int64_t *win_off,
+                         const int64_t *win_t0, const int64_t *win_t1, int32_t W,
+                         ta_load_summary *out_summary, ta_window **handle);
+
+/* ------------------------------------------------------------------------
+ * ta_sort_timeline - canonical order (device and stream identifiers locate
+ * device work, thread identifiers locate calls: Sec. 5.2).
+ *
+ * domain d = 0 for kinds 0..2 (host), 1 for kinds 3..5 (device).
+ * Canonical order = ascending by the tuple
+ *   (dropped, window, pid, d, stream, ts_start, -ts_end, input index),
+ * pid and stream compared as signed integers.  For a dropped record
+ * d = (kind >= 3).  perm[p] = input index of the record at sorted position p;
+ * kept records occupy [0, n_valid), dropped ones [n_valid, n).
+ * A LANE is a maximal run of kept records with equal (window, pid, d, stream);
+ * lanes are listed in sorted order, lane l covers [lane_off[l], lane_off[l+1]).
+ * The eight columns hold the records in sorted order (all n of them).
+ */
+typedef struct ta_sort_result {
+  int64_t n, n_valid;
+  int32_t n_lanes;
+  int32_t n_windows;
+  const int32_t *perm;                         /* device, n                  */
+  const int64_t *ts_start, *ts_end, *corr_id;  /* device, n each             */
+  const int32_t *pid, *name_id, *seq;          /* device, n each             */
+  const int16_t *stream, *kind;                /* device, n each             */
+  const int32_t *lane_window, *lane_pid;       /* device, n_lanes each       */
+  const int16_t *lane_stream, *lane_domain;    /* device, n_lanes each       */
+  const int32_t *lane_off;                     /* device, n_lanes + 1        */
+} ta_sort_result;
+
+ta_status ta_sort_timeline(ta_window *h, ta_sort_result *out);
+
+/* ------------------------------------------------------------------------
+ * ta_correlate_launches - correlation id associates submissions with device
+ * activity (Sec. 5.2; Fig. "Key performance observations" (a)).
+ *
+ * Build side: kept LAUNCH records.  Probe side: kept KERNEL and MEMCPY
+ * records.  Key = (window, pid, corr_id), all 64 bits of corr_id significant.
+ * For a probe at sorted position i, launch_of[i] = the SMALLEST sorted
+ * position of a LAUNCH with an equal key, or -1.  If matched to l:
+ *   launch_latency[i] = ts_start[i] - ts_start[l]          (signed)
+ *   queue_delay[i]    = max(0, ts_start[i] - ts_end[l])
+ * Elsewhere launch_of = -1 and both times are 0.  kernels_of_launch[l] = number
+ * of probes with launch_of == l (0 at non-launch positions); several probes
+ * per launch are legal (graph replay, Sec. 6.1).
+ * Per-window summary: n_dup_launch counts LAUNCH records whose key already
+ * belongs to a smaller sorted position; n_orphan_launch counts LAUNCH records
+ * that are not such duplicates and have no probe; min/max are 0 when
+ * n_matched == 0.
+ */
+typedef struct ta_join_summary {
+  int64_t n_probe, n_matched, n_unmatched, n_launch, n_dup_launch, n_orphan_launch;
+  int64_t sum_latency, min_latency, max_latency, sum_queue, max_queue;
+} ta_join_summary;
+
+typedef struct ta_join_result {
+  const int32_t *launch_of;         /* device, n */
+  const int64_t *launch_latency;    /* device, n */
+  const int64_t *queue_delay;       /* device, n */
+  const int32_t *kernels_of_launch; /* device, n */
+} ta_join_result;
+
+ta_status ta_correlate_launches(ta_window *h, ta_join_result *out,
+                                ta_join_summary *out_summary);
+
+/* ------------------------------------------------------------------------
+ * ta_attribute_operators - thread id plus call intervals link host API calls
+ * to the enclosing calls (Sec. 9.1); T_op spans the first kernel start to the
+ * last completion (Sec. 6.1).  Device work can outlive the enclosing call
+ * (Sec. 5.2), so containment is tested on the LAUNCH interval.
+ *
+ * Inside one host lane, OP j ENCLOSES host record i (i != j) iff
+ * ts_start[j] <= ts_start[i] and ts_end[i] <= ts_end[j] and, when both
+ * intervals are identical, j precedes i in canonical order.
+ *   parent[i] = the encloser with the largest ts_start, then the smallest
+ *               ts_end, then the largest sorted position; -1 if none.
+ *   depth[i]  = number of enclosers.
+ * Device records: op_of[i] = parent[launch_of[i]] for KERNEL/MEMCPY with a
+ * launch, else -1.  For every OP r, over device records with op_of == r:
+ *   op_n_kernels[r], op_first_start[r] = min ts_start, op_last_end[r] =
+ *   max ts_end, op_kernel_ns[r] = sum of durations;
+ *   T_op[r] = op_last_end[r] - op_first_start[r].
+ * All four are 0 when op_n_kernels[r] == 0 and at non-OP positions.
+ * Returns TA_ERR_BAD_NESTING if some OP j and host record i of one lane have
+ * ts_start[j] < ts_start[i] < ts_end[j] < ts_end[i], else TA_ERR_DEPTH if some
+ * depth exceeds TA_MAX_DEPTH; in both cases the summaries' max_depth /
+ * bad_nesting fields are filled and the other outputs are unspecified.
+ */
+typedef struct ta_attr_summary {
+  int64_t n_attributed, n_no_launch, n_no_op;
+  int32_t max_depth, bad_nesting;
+} ta_attr_summary;
+
+typedef struct ta_attr_result {
+  const int32_t *parent;         /* device, n */
+  const uint8_t *depth;          /* device, n */
+  const int32_t *op_of;          /* device, n */
+  const int64_t *op_first_start; /* device, n */
+  const int64_t *op_last_end;    /* device, n */
+  const int64_t *op_kernel_ns;   /* device, n */
+  const int32_t *op_n_kernels;   /* device, n */
+} ta_attr_result;
+
+ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out,
+                                 ta_attr_summary *out_summary);
+
+/* ------------------------------------------------------------------------
+ * ta_stream_gaps - device activity records reveal idle intervals (Sec. 9.1).
+ *
+ * For a device lane of a window [W0, W1) with records 0..m-1 in canonical
+ * order and clipped ends c_i = min(ts_end_i, W1):
+ *   P_0 = W0, P_{i+1} = max(P_i, c_i)
+ *   gap_before[i] = max(0, ts_start_i - P_i)
+ *   busy_i        = max(0, c_i - max(ts_start_i, P_i))
+ *   tail_gap      = W1 - P_m
+ * so that busy + idle == W1 - W0 for every lane.  Each positive gap g (head,
+ * interior, tail) adds one to histogram bin min(39, floor(log2 g)).
+ * lane_gaps / lane_hist have one row per lane of the lane table; rows of host
+ * lanes are zero.  win_hist[w] sums the window's lanes.  The long-gap list
+ * holds every gap with g > 0 and g >= min_gap_ns, ordered by lane, then time,
+ * a lane's tail gap last.
+ */
+typedef struct ta_lane_gaps {
+  int64_t busy, idle, n_events, n_gaps, max_gap, first_start, last_end;
+} ta_lane_gaps;
+
+typedef struct ta_long_gap {
+  int32_t lane;       /* index into the lane table                           */
+  int32_t next_event; /* sorted position of the record after the gap, -1 = tail */
+  int64_t gap_start;  /* = P_i                                               */
+  int64_t gap_len;
+} ta_long_gap;
+
+typedef struct ta_gap_result {
+  const int64_t *gap_before;      /* device, n (0 at host and dropped positions) */
+  const ta_lane_gaps *lane_gaps;  /* device, n_lanes                         */
+  const uint32_t *lane_hist;      /* device, n_lanes x TA_NBINS              */
+  const uint32_t *win_hist;       /* device, n_windows x TA_NBINS            */
+  const ta_long_gap *long_gaps;   /* device, n_long_gaps                     */
+  int64_t n_long_gaps;
+} ta_gap_result;
+
+ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out);
+
+/* ------------------------------------------------------------------------
+ * ta_aggregate_ops - per-symbol call counts and duration statistics (the
+ * fidelity measures of Sec. 8.1 are per-symbol counts and kernel durations).
+ *
+ * Population: kept records with (1 << kind) & kind_mask.  value_sel 0: value =
+ * ts_end - ts_start.  value_sel 1: kind_mask must be exactly 1 << TA_KIND_OP
+ * (else INVALID_ARG); the population is further restricted to OPs with
+ * op_n_kernels > 0 and value = T_op.  Group key (window, pid, name_id); one
+ * output row per non-empty group in ascending signed key order with count,
+ * sum, min, max and a histogram whose bin is min(39, floor(log2 v)) for
+ * v >= 1 and 0 for v <= 0.
+ * Limit: (#windows x #pids x (max name_id - min name_id + 1)) <= 2^27, else
+ * TA_ERR_TOO_LARGE.  The result buffers of an earlier ta_aggregate_ops call on
+ * the same handle stay valid.
+ */
+typedef struct ta_agg_result {
+  int64_t n_groups;
+  const int32_t *g_window, *g_pid, *g_name;       /* device, n_groups each   */
+  const int64_t *g_count, *g_sum, *g_min, *g_max; /* device, n_groups each   */
+  const uint32_t *g_hist;                         /* device, n_groups x TA_NBINS */
+} ta_agg_result;
+
+ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel,
+                           ta_agg_result *out);
+
+/* ------------------------------------------------------------------------
+ * ta_match_collectives - cross-process links by shared identifiers; ranks
+ * meet in collectives and a late rank leaves the others waiting (Sec. 6.1
+ * "Execution progress and state", Sec. 9.2).
+ *
+ * Population: kept COLL records; comm_id = corr_id.  Group key
+ * (window, comm_id, seq), groups output in ascending signed key order.
+ * Per group: n_members, min_start, max_start, skew = max_start - min_start,
+ * max_end, straggler_pid = pid of the member with the largest ts_start (ties:
+ * smallest pid), flags bit0 INCOMPLETE (n_members != the size given for that
+ * comm_id in `sizes`; for a comm_id not listed: n_members < 2), bit1 DUP_PID
+ * (some pid occurs twice).  wait_ns[i] = max_start - ts_start[i] for every
+ * member of every group, 0 at non-COLL positions.  Rank table: one row per
+ * (window, pid) that has COLL records, ascending; its four counters cover only
+ * members of groups with flags == 0 (n_coll = number of such members,
+ * n_straggler = number of those groups whose straggler_pid is this pid).
+ * sizes: host, n_comms entries (may be NULL when n_comms == 0).
+ */
+typedef struct ta_comm_size {
+  int64_t comm_id;
+  int32_t n_ranks;
+  int32_t reserved;
+} ta_comm_size;
+
+#define TA_COLL_INCOMPLETE 1
+#define TA_COLL_DUP_PID 2
+
+typedef struct ta_coll_result {
+  int64_t n_groups, n_ranks;
+  const int32_t *g_window;      /* device, n_groups */
+  const int64_t *g_comm;        /* device, n_groups */
+  const int32_t *g_seq;         /* device, n_groups */
+  const int32_t *g_n_members;   /* device, n_groups */
+  const int64_t *g_min_start, *g_max_start, *g_skew, *g_max_end; /* device, n_groups */
+  const int32_t *g_straggler_pid, *g_flags;                      /* device, n_groups */
+  const int64_t *wait_ns;       /* device, n */
+  const int32_t *r_window, *r_pid;                               /* device, n_ranks */
+  const int64_t *r_n_coll, *r_sum_wait, *r_max_wait, *r_n_straggler; /* device, n_ranks */
+} ta_coll_result;
+
+ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes,
+                               int32_t n_comms, ta_coll_result *out);
+
+/* ta_free - releases every buffer of the handle through env.release.
+ * NULL-safe.  Synchronises the handle's stream first. */
+void ta_free(ta_window *h);
+
+/* Helpers that carry no work. */
+const char *ta_strerror(ta_status s);
+int32_t ta_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TA_H */

@@ -1,0 +1,193 @@
+"""Brute-force twins of the analyzer's definitions, in plain Python.
+
+Written independently of both analyzers, straight from the definitions in
+include/ta.h, with quadratic scans and tick bitmaps.  Only for tiny windows.
+"""
+import numpy as np
+
+
+def log2_bin(v):
+    if v <= 1:
+        return 0
+    return min(39, int(v).bit_length() - 1)
+
+
+def load(ev, win_off, t0, t1):
+    n = len(ev)
+    W = len(t0)
+    win = np.zeros(n, dtype=np.int64)
+    dropped = np.zeros(n, dtype=bool)
+    summ = [dict(n_events=0, n_valid=0, n_bad_kind=0, n_bad_interval=0, n_out_of_window=0)
+            for _ in range(W)]
+    for w in range(W):
+        for k in range(win_off[w], win_off[w + 1]):
+            win[k] = w
+            s = summ[w]
+            s["n_events"] += 1
+            e = ev[k]
+            if not (0 <= e["kind"] <= 5):
+                dropped[k] = True
+                s["n_bad_kind"] += 1
+            elif e["ts_end"] < e["ts_start"]:
+                dropped[k] = True
+                s["n_bad_interval"] += 1
+            elif e["ts_start"] < t0[w] or e["ts_start"] >= t1[w]:
+                dropped[k] = True
+                s["n_out_of_window"] += 1
+            else:
+                s["n_valid"] += 1
+    return win, dropped, summ
+
+
+def canonical_perm(ev, win, dropped):
+    def key(k):
+        e = ev[k]
+        return (bool(dropped[k]), int(win[k]), int(e["pid"]), 1 if e["kind"] >= 3 else 0,
+                int(e["stream"]), int(e["ts_start"]), -int(e["ts_end"]), k)
+    return sorted(range(len(ev)), key=key)
+
+
+def lanes(sv, wins, n_valid):
+    """sv: records in sorted order; returns list of (window, pid, domain, stream, begin, end)."""
+    out = []
+    for p in range(n_valid):
+        k = (int(wins[p]), int(sv[p]["pid"]), 1 if sv[p]["kind"] >= 3 else 0, int(sv[p]["stream"]))
+        if not out or out[-1][:4] != k:
+            if out:
+                out[-1] = out[-1][:5] + (p,)
+            out.append(k + (p, None))
+    if out:
+        out[-1] = out[-1][:5] + (n_valid,)
+    return out
+
+
+def join(sv, wins, n_valid):
+    n = len(sv)
+    launch_of = [-1] * n
+    lat = [0] * n
+    qd = [0] * n
+    kol = [0] * n
+    for i in range(n_valid):
+        if sv[i]["kind"] not in (3, 4):
+            continue
+        for l in range(n_valid):
+            if (sv[l]["kind"] == 2 and wins[l] == wins[i] and sv[l]["pid"] == sv[i]["pid"]
+                    and sv[l]["corr_id"] == sv[i]["corr_id"]):
+                launch_of[i] = l
+                lat[i] = int(sv[i]["ts_start"]) - int(sv[l]["ts_start"])
+                qd[i] = max(0, int(sv[i]["ts_start"]) - int(sv[l]["ts_end"]))
+                kol[l] += 1
+                break
+    return launch_of, lat, qd, kol
+
+
+def attribution(sv, wins, n_valid, lane_list):
+    """O(n^2) scan of the enclosure definition.  Returns parent, depth, bad_nesting."""
+    n = len(sv)
+    parent = [-1] * n
+    depth = [0] * n
+    bad = False
+    for (w, pid, dom, st, b, e) in lane_list:
+        if dom != 0:
+            continue
+        for i in range(b, e):
+            si, ei = int(sv[i]["ts_start"]), int(sv[i]["ts_end"])
+            enc = []
+            for j in range(b, e):
+                if j == i or sv[j]["kind"] != 0:
+                    continue
+                sj, ej = int(sv[j]["ts_start"]), int(sv[j]["ts_end"])
+                if sj < si < ej < ei:
+                    bad = True
+                if sj <= si and ei <= ej and ((sj, ej) != (si, ei) or j < i):
+                    enc.append(j)
+            depth[i] = len(enc)
+            if enc:
+                parent[i] = max(enc, key=lambda j: (int(sv[j]["ts_start"]), -int(sv[j]["ts_end"]), j))
+    return parent, depth, bad
+
+
+def gaps_bitmap(sv, lane, W0, W1):
+    """Marks every tick of [W0, W1) covered by a record of the lane; returns busy, idle,
+    list of (start, len) of idle runs.  A zero-length record covers no tick but is still an
+    observation of the stream, so an idle run is cut at the start time of such a record."""
+    (_, _, _, _, b, e) = lane
+    cov = np.zeros(W1 - W0, dtype=bool)
+    for i in range(b, e):
+        s, t = int(sv[i]["ts_start"]), min(int(sv[i]["ts_end"]), W1)
+        if t > s:
+            cov[s - W0:t - W0] = True
+    busy = int(cov.sum())
+    runs = []
+    t = 0
+    L = len(cov)
+    while t < L:
+        if not cov[t]:
+            u = t
+            while u < L and not cov[u]:
+                u += 1
+            cuts = sorted({int(sv[i]["ts_start"]) - W0 for i in range(b, e)
+                           if t < int(sv[i]["ts_start"]) - W0 < u})
+            a = t
+            for c in cuts + [u]:
+                runs.append((W0 + a, c - a))
+                a = c
+            t = u
+        else:
+            t += 1
+    return busy, L - busy, runs
+
+
+def aggregate(sv, wins, n_valid, kind_mask, values):
+    """values: per sorted position value or None (not in the population)."""
+    rows = {}
+    for p in range(n_valid):
+        if not ((1 << int(sv[p]["kind"])) & kind_mask) or values[p] is None:
+            continue
+        key = (int(wins[p]), int(sv[p]["pid"]), int(sv[p]["name_id"]))
+        v = int(values[p])
+        r = rows.setdefault(key, dict(count=0, sum=0, min=v, max=v, hist=[0] * 40))
+        r["count"] += 1
+        r["sum"] += v
+        r["min"] = min(r["min"], v)
+        r["max"] = max(r["max"], v)
+        r["hist"][log2_bin(v)] += 1
+    return [(k, rows[k]) for k in sorted(rows)]
+
+
+def collectives(sv, wins, n_valid, sizes):
+    exp = dict(sizes)
+    groups = {}
+    for p in range(n_valid):
+        if sv[p]["kind"] == 5:
+            groups.setdefault((int(wins[p]), int(sv[p]["corr_id"]), int(sv[p]["seq"])), []).append(p)
+    out = []
+    wait = {}
+    ranks = {}
+    for key in sorted(groups):
+        m = groups[key]
+        starts = [int(sv[p]["ts_start"]) for p in m]
+        mx = max(starts)
+        strag = min(int(sv[p]["pid"]) for p in m if int(sv[p]["ts_start"]) == mx)
+        flags = 0
+        if key[1] in exp:
+            if len(m) != exp[key[1]]:
+                flags |= 1
+        elif len(m) < 2:
+            flags |= 1
+        pids = [int(sv[p]["pid"]) for p in m]
+        if len(set(pids)) != len(pids):
+            flags |= 2
+        for p in m:
+            wait[p] = mx - int(sv[p]["ts_start"])
+            r = ranks.setdefault((key[0], int(sv[p]["pid"])), [0, 0, 0, 0])
+            if flags == 0:
+                r[0] += 1
+                r[1] += wait[p]
+                r[2] = max(r[2], wait[p])
+        if flags == 0:
+            ranks[(key[0], strag)][3] += 1
+        out.append((key, dict(n=len(m), min_start=min(starts), max_start=mx, skew=mx - min(starts),
+                              max_end=max(int(sv[p]["ts_end"]) for p in m), straggler=strag,
+                              flags=flags)))
+    return out, wait, [(k, ranks[k]) for k in sorted(ranks)]

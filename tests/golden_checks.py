@@ -1,0 +1,126 @@
+"""Checks of a result dict (see runners.py) against the hand-worked fixtures
+under tests/golden/.  Used for the oracle (CPU) and for the CUDA library."""
+import numpy as np
+
+from helpers import bins_of, ints, kv, load_golden
+
+
+def _device_lane(r):
+    d = np.nonzero(r["lane_domain"] == 1)[0]
+    assert len(d) == 1
+    return int(d[0])
+
+
+def check_H1(run):
+    g = load_golden("H1_gaps.txt")
+    r = run(g["events"], [0, len(g["events"])], [g["t0"]], [g["t1"]], min_gap=g["min_gap"])
+    e = g["expect"]
+    assert r["gap_before"].tolist() == ints(e["gap_before"])
+    l = _device_lane(r)
+    lg = r["lane_gaps"][l]
+    assert lg["busy"] == int(e["lane_busy"][0]) and lg["idle"] == int(e["lane_idle"][0])
+    assert lg["busy"] + lg["idle"] == g["t1"] - g["t0"]
+    assert lg["n_gaps"] == int(e["lane_n_gaps"][0]) and lg["max_gap"] == int(e["lane_max_gap"][0])
+    assert lg["first_start"] == int(e["lane_first_start"][0])
+    assert lg["last_end"] == int(e["lane_last_end"][0]) and lg["n_events"] == 6
+    hist = np.zeros(40, dtype=np.int64)
+    for t in e["hist_bins"]:
+        hist += bins_of(t)
+    assert r["lane_hist"][l].tolist() == hist.tolist()
+    assert r["win_hist"][0].tolist() == hist.tolist()
+    want = [tuple(int(x) for x in t.split(",")) for t in e["long_gaps"]]
+    got = [(int(x["next_event"]), int(x["gap_start"]), int(x["gap_len"])) for x in r["long_gaps"]]
+    assert got == want
+    assert all(int(x["lane"]) == l for x in r["long_gaps"])
+
+
+def check_H2(run):
+    g = load_golden("H2_join_attribution.txt")
+    n = len(g["events"])
+    r = run(g["events"], [0, n], [g["t0"]], [g["t1"]], agg_masks=(1 << 3,))
+    e = g["expect"]
+    assert r["perm"].tolist() == list(range(n))
+    for k in ("parent", "depth", "launch_of", "launch_latency", "queue_delay", "kernels_of_launch",
+              "op_of"):
+        assert r[k].tolist() == ints(e[k]), k
+    for k, v in kv(e["join"]).items():
+        assert int(r["join_sum"][0][k]) == v, k
+    for k, v in kv(e["attr"]).items():
+        assert int(r["attr_sum"][0][k]) == v, k
+    assert r["attr_status"] == 0
+    seen = set()
+    for t in e["op"]:
+        pos, rest = t.split(":")
+        pos = int(pos)
+        nk, first, last, kns = (int(x) for x in rest.split(","))
+        assert (int(r["op_n_kernels"][pos]), int(r["op_first_start"][pos]),
+                int(r["op_last_end"][pos]), int(r["op_kernel_ns"][pos])) == (nk, first, last, kns)
+        seen.add(pos)
+    for p in range(n):
+        if p not in seen:
+            assert r["op_n_kernels"][p] == 0 and r["op_first_start"][p] == 0
+            assert r["op_last_end"][p] == 0 and r["op_kernel_ns"][p] == 0
+    for pref, key in (("agg0_", "agg_kernel"), ("aggT_", "agg_top")):
+        rows = e[key]
+        assert len(r[pref + "g_name"]) == len(rows)
+        for i, t in enumerate(rows):
+            name, rest = t.split(":", 1)
+            cnt, sm, mn, mx, bins = rest.split(",", 4)
+            assert int(r[pref + "g_window"][i]) == 0 and int(r[pref + "g_pid"][i]) == 1
+            assert int(r[pref + "g_name"][i]) == int(name)
+            assert (int(r[pref + "g_count"][i]), int(r[pref + "g_sum"][i]),
+                    int(r[pref + "g_min"][i]), int(r[pref + "g_max"][i])) == \
+                (int(cnt), int(sm), int(mn), int(mx))
+            assert r[pref + "g_hist"][i].tolist() == bins_of(bins).tolist()
+
+
+def check_H3(run):
+    g = load_golden("H3_collectives.txt")
+    n = len(g["events"])
+    r = run(g["events"], [0, n], [g["t0"]], [g["t1"]], comm_sizes=g["comm_sizes"])
+    e = g["expect"]
+    assert r["c_seq"].tolist() == [0, 1, 2] and r["c_comm"].tolist() == [5, 5, 5]
+    for i, t in enumerate(e["groups"]):
+        nm, mn, mx, sk, me, st, fl = (int(x) for x in t.split(","))
+        got = (int(r["c_n_members"][i]), int(r["c_min_start"][i]), int(r["c_max_start"][i]),
+               int(r["c_skew"][i]), int(r["c_max_end"][i]), int(r["c_straggler_pid"][i]),
+               int(r["c_flags"][i]))
+        assert got == (nm, mn, mx, sk, me, st, fl), i
+    waits = {}
+    for p in range(n):
+        waits[(int(r["pid"][p]), int(r["seq"][p]))] = int(r["wait_ns"][p])
+    for t in e["waits"]:
+        k, v = t.split(":")
+        assert waits[tuple(int(x) for x in k.split(","))] == int(v), t
+    assert r["r_pid"].tolist() == [0, 1, 2, 3]
+    for t in e["ranks"]:
+        pid, rest = t.split(":")
+        i = int(pid)
+        assert (int(r["r_n_coll"][i]), int(r["r_sum_wait"][i]), int(r["r_max_wait"][i]),
+                int(r["r_n_straggler"][i])) == tuple(int(x) for x in rest.split(","))
+
+
+def check_H4(run):
+    g = load_golden("H4_idle_figure.txt")
+    n = len(g["events"])
+    r = run(g["events"], [0, n], [g["t0"]], [g["t1"]])
+    e = g["expect"]
+    lg = r["lane_gaps"][0]
+    assert lg["busy"] == int(e["lane_busy"][0]) and lg["idle"] == int(e["lane_idle"][0])
+    assert lg["n_gaps"] == int(e["lane_n_gaps"][0]) and lg["max_gap"] == int(e["lane_max_gap"][0])
+    assert r["gap_before"].sum() == 0
+    assert len(r["long_gaps"]) == 1 and r["long_gaps"][0]["next_event"] == -1
+
+
+def check_H5(run):
+    g = load_golden("H5_ties.txt")
+    n = len(g["events"])
+    r = run(g["events"], [0, n], [g["t0"]], [g["t1"]])
+    e = g["expect"]
+    assert r["perm"].tolist() == ints(e["perm"])
+    assert r["parent"].tolist() == ints(e["parent"])
+    assert r["depth"].tolist() == ints(e["depth"])
+    assert r["attr_status"] == 0
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5]

@@ -1,0 +1,258 @@
+"""Pins the CPU oracle to brute-force twins of the definitions (tests/brute.py)
+on random tiny adversarial windows: quadratic scans and tick bitmaps."""
+import numpy as np
+import pytest
+
+import brute
+from runners import DEVICE_MASK, run_oracle
+from tiny import random_window
+
+SEEDS = list(range(12))
+
+
+def _sorted_view(ev, r):
+    return ev[r["perm"]]
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_load_and_canonical_order(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1, min_gap=5, comm_sizes=sizes)
+    win, dropped, summ = brute.load(ev, off, t0, t1)
+    for w, s in enumerate(summ):
+        for k, v in s.items():
+            assert int(r["load_sum"][w][k]) == v
+    perm = brute.canonical_perm(ev, win, dropped)
+    assert r["perm"].tolist() == perm
+    assert r["n_valid"] == int((~dropped).sum())
+    sv = ev[perm]
+    for k in ("ts_start", "ts_end", "corr_id", "pid", "name_id", "seq", "stream", "kind"):
+        assert np.array_equal(r[k], sv[k])
+    ll = brute.lanes(sv, win[perm], r["n_valid"])
+    assert r["lane_off"].tolist() == [l[4] for l in ll] + [r["n_valid"]]
+    assert r["lane_window"].tolist() == [l[0] for l in ll]
+    assert r["lane_pid"].tolist() == [l[1] for l in ll]
+    assert r["lane_domain"].tolist() == [l[2] for l in ll]
+    assert r["lane_stream"].tolist() == [l[3] for l in ll]
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_join_against_quadratic_scan(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    lo, lat, qd, kol = brute.join(sv, wins, r["n_valid"])
+    assert r["launch_of"].tolist() == lo
+    assert r["launch_latency"].tolist() == lat
+    assert r["queue_delay"].tolist() == qd
+    assert r["kernels_of_launch"].tolist() == kol
+    # every probe is matched to exactly one launch or counted unmatched
+    js = r["join_sum"]
+    assert (js["n_matched"] + js["n_unmatched"] == js["n_probe"]).all()
+    for w in range(len(t0)):
+        sel = [i for i in range(r["n_valid"]) if wins[i] == w and sv[i]["kind"] in (3, 4)]
+        assert js[w]["n_probe"] == len(sel)
+        assert js[w]["n_matched"] == sum(1 for i in sel if lo[i] >= 0)
+        assert js[w]["sum_latency"] == sum(lat[i] for i in sel)
+        assert js[w]["sum_queue"] == sum(qd[i] for i in sel)
+        m = [lat[i] for i in sel if lo[i] >= 0]
+        assert js[w]["min_latency"] == (min(m) if m else 0)
+        assert js[w]["max_latency"] == (max(m) if m else 0)
+        launches = [i for i in range(r["n_valid"]) if wins[i] == w and sv[i]["kind"] == 2]
+        assert js[w]["n_launch"] == len(launches)
+        dup = 0
+        orphan = 0
+        for i in launches:
+            first = min(j for j in launches if sv[j]["pid"] == sv[i]["pid"]
+                        and sv[j]["corr_id"] == sv[i]["corr_id"])
+            if first != i:
+                dup += 1
+            elif kol[i] == 0:
+                orphan += 1
+        assert js[w]["n_dup_launch"] == dup and js[w]["n_orphan_launch"] == orphan
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_attribution_against_quadratic_scan(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    ll = brute.lanes(sv, wins, r["n_valid"])
+    parent, depth, bad = brute.attribution(sv, wins, r["n_valid"], ll)
+    assert not bad and r["attr_status"] in (0, 8)
+    assert r["parent"].tolist() == parent
+    assert r["depth"].tolist() == depth
+    assert (r["attr_status"] == 8) == (max(depth) > 8)
+    # for properly nested lanes the parent is the nearest earlier OP that ends no earlier
+    for (w, pid, dom, st, b, e) in ll:
+        if dom:
+            continue
+        for i in range(b, e):
+            near = -1
+            for j in range(i - 1, b - 1, -1):
+                if sv[j]["kind"] == 0 and sv[j]["ts_end"] >= sv[i]["ts_end"]:
+                    near = j
+                    break
+            assert parent[i] == near
+    # device records inherit the parent of their launch; per-OP sums are direct
+    n = len(ev)
+    op_of = [-1] * n
+    for i in range(r["n_valid"]):
+        if sv[i]["kind"] in (3, 4) and r["launch_of"][i] >= 0:
+            op_of[i] = parent[r["launch_of"][i]]
+    assert r["op_of"].tolist() == op_of
+    for p in range(n):
+        mem = [i for i in range(n) if op_of[i] == p]
+        assert r["op_n_kernels"][p] == len(mem)
+        if mem:
+            assert r["op_first_start"][p] == min(int(sv[i]["ts_start"]) for i in mem)
+            assert r["op_last_end"][p] == max(int(sv[i]["ts_end"]) for i in mem)
+            assert r["op_kernel_ns"][p] == sum(int(sv[i]["ts_end"] - sv[i]["ts_start"]) for i in mem)
+        else:
+            assert r["op_first_start"][p] == r["op_last_end"][p] == r["op_kernel_ns"][p] == 0
+    a = r["attr_sum"]
+    assert (a["n_attributed"] + a["n_no_launch"] + a["n_no_op"] == r["join_sum"]["n_probe"]).all()
+    assert r["op_n_kernels"].sum() == a["n_attributed"].sum()
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_bad_nesting_flag(seed):
+    ev, off, t0, t1, sizes = random_window(100 + seed, nested=False, defects=False)
+    r = run_oracle(ev, off, t0, t1)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    ll = brute.lanes(sv, wins, r["n_valid"])
+    parent, depth, bad = brute.attribution(sv, wins, r["n_valid"], ll)
+    assert (r["attr_status"] == 9) == bad
+    assert bool(r["attr_sum"]["bad_nesting"].any()) == bad
+    # the oracle evaluates the definition even then
+    assert r["parent"].tolist() == parent and r["depth"].tolist() == depth
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_gaps_against_tick_bitmap(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    min_gap = 7
+    r = run_oracle(ev, off, t0, t1, min_gap=min_gap)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    ll = brute.lanes(sv, wins, r["n_valid"])
+    want_long = []
+    win_hist = np.zeros((len(t0), 40), dtype=np.int64)
+    for li, lane in enumerate(ll):
+        lg = r["lane_gaps"][li]
+        if lane[2] == 0:
+            assert all(int(lg[k]) == 0 for k in lg.dtype.names)
+            assert r["lane_hist"][li].sum() == 0
+            continue
+        W0, W1 = t0[lane[0]], t1[lane[0]]
+        busy, idle, runs = brute.gaps_bitmap(sv, lane, W0, W1)
+        assert lg["busy"] == busy and lg["idle"] == idle
+        assert lg["busy"] + lg["idle"] == W1 - W0
+        assert lg["n_gaps"] == len(runs)
+        assert lg["max_gap"] == max([x[1] for x in runs], default=0)
+        assert lg["n_events"] == lane[5] - lane[4]
+        hist = np.zeros(40, dtype=np.int64)
+        for (_, ln) in runs:
+            hist[brute.log2_bin(ln)] += 1
+        assert r["lane_hist"][li].tolist() == hist.tolist()
+        assert r["lane_hist"][li].sum() == lg["n_gaps"]
+        win_hist[lane[0]] += hist
+        # each idle run ends where a record starts (or at the window end)
+        for (st, ln) in runs:
+            if ln >= min_gap:
+                end = st + ln
+                nxt = -1
+                if end < W1:
+                    nxt = min(i for i in range(lane[4], lane[5]) if sv[i]["ts_start"] == end)
+                want_long.append((li, nxt, st, ln))
+        # gap_before of a record = length of the idle run that ends at its start, for the first
+        # record (in canonical order) that starts there
+        ends = {st + ln: ln for (st, ln) in runs}
+        seen = set()
+        for i in range(lane[4], lane[5]):
+            s = int(sv[i]["ts_start"])
+            g = ends.get(s, 0) if s not in seen else 0
+            seen.add(s)
+            assert r["gap_before"][i] == g
+    assert r["win_hist"].tolist() == win_hist.tolist()
+    got = [(int(x["lane"]), int(x["next_event"]), int(x["gap_start"]), int(x["gap_len"]))
+           for x in r["long_gaps"]]
+    assert got == want_long
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_aggregates_against_dict(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    masks = (DEVICE_MASK, 1 << 2, 0b111111)
+    r = run_oracle(ev, off, t0, t1, agg_masks=masks)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    n = len(ev)
+    dur = [int(sv[p]["ts_end"]) - int(sv[p]["ts_start"]) for p in range(n)]
+    top = [int(r["op_last_end"][p] - r["op_first_start"][p]) if r["op_n_kernels"][p] > 0 else None
+           for p in range(n)]
+    cases = [(f"agg{i}_", m, dur) for i, m in enumerate(masks)] + [("aggT_", 1, top)]
+    for pref, mask, vals in cases:
+        rows = brute.aggregate(sv, wins, r["n_valid"], mask, vals)
+        assert len(rows) == len(r[pref + "g_count"])
+        for i, (key, row) in enumerate(rows):
+            assert (int(r[pref + "g_window"][i]), int(r[pref + "g_pid"][i]),
+                    int(r[pref + "g_name"][i])) == key
+            assert int(r[pref + "g_count"][i]) == row["count"]
+            assert int(r[pref + "g_sum"][i]) == row["sum"]
+            assert int(r[pref + "g_min"][i]) == row["min"]
+            assert int(r[pref + "g_max"][i]) == row["max"]
+            assert r[pref + "g_hist"][i].tolist() == row["hist"]
+            assert r[pref + "g_hist"][i].sum() == row["count"]
+        pop = sum(1 for p in range(r["n_valid"])
+                  if ((1 << int(sv[p]["kind"])) & mask) and vals[p] is not None)
+        assert int(r[pref + "g_count"].sum()) == pop
+
+
+def test_log2_bins_bracket_values():
+    from helpers import make_events
+    vals = [0, 1, 2, 3, 4, 7, 8, 1023, 1024, 2**38, 2**39 - 1, 2**39, 2**45]
+    ev = make_events([("KERNEL", 1, 0, 10, 10 + v, 0, i, 0) for i, v in enumerate(vals)])
+    r = run_oracle(ev, [0, len(ev)], [0], [100], agg_masks=(1 << 3,))
+    for i, v in enumerate(vals):
+        b = int(np.nonzero(r["agg0_g_hist"][i])[0][0])
+        if v <= 1:
+            assert b == 0
+        elif b < 39:
+            assert 2**b <= v < 2**(b + 1)
+        else:
+            assert v >= 2**39
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_collectives_against_dict(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1, comm_sizes=sizes)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    groups, wait, ranks = brute.collectives(sv, wins, r["n_valid"], sizes)
+    assert len(groups) == len(r["c_seq"])
+    for i, (key, g) in enumerate(groups):
+        assert (int(r["c_window"][i]), int(r["c_comm"][i]), int(r["c_seq"][i])) == key
+        assert (int(r["c_n_members"][i]), int(r["c_min_start"][i]), int(r["c_max_start"][i]),
+                int(r["c_skew"][i]), int(r["c_max_end"][i]), int(r["c_straggler_pid"][i]),
+                int(r["c_flags"][i])) == (g["n"], g["min_start"], g["max_start"], g["skew"],
+                                          g["max_end"], g["straggler"], g["flags"])
+    want = np.zeros(len(ev), dtype=np.int64)
+    for p, v in wait.items():
+        want[p] = v
+    assert r["wait_ns"].tolist() == want.tolist()
+    assert len(ranks) == len(r["r_pid"])
+    for i, (key, row) in enumerate(ranks):
+        assert (int(r["r_window"][i]), int(r["r_pid"][i])) == key
+        assert [int(r["r_n_coll"][i]), int(r["r_sum_wait"][i]), int(r["r_max_wait"][i]),
+                int(r["r_n_straggler"][i])] == row
+    # in every unflagged group somebody waits 0 and somebody waits the whole skew
+    for i, (key, g) in enumerate(groups):
+        if g["flags"] == 0:
+            ws = [wait[p] for p in range(r["n_valid"]) if sv[p]["kind"] == 5
+                  and (int(wins[p]), int(sv[p]["corr_id"]), int(sv[p]["seq"])) == key]
+            assert min(ws) == 0 and max(ws) == g["skew"]
