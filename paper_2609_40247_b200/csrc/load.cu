@@ -1,0 +1,228 @@
+// ta_load_window kernels: validity (start-time filtering separates windows,
+// Sec. 5.2), discovery and dense ranking of the (pid, domain, stream) triples
+// that name a lane, and the 64-bit sort key (window | triple rank | ts_start -
+// t0) together with the digit histograms of every radix pass.
+// HBM-bound: each kernel streams the 40-byte records once.
+#include "ta_internal.cuh"
+#include "records.cuh"
+
+#define TRIPLE_EMPTY (~0ull)
+
+__device__ __forceinline__ i64 warp_min_i64(i64 v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = min(v, (i64)__shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ i64 warp_max_i64(i64 v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, (i64)__shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Pass 1 over the records: defect counters, the set of lane triples, the range
+// of name ids and the longest duration.
+__global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n, const int64_t *off,
+                                                  const int64_t *t0, const int64_t *t1, int W,
+                                                  TripleTable *tt, ta_load_summary *sum,
+                                                  int64_t *misc, int32_t *status) {
+  __shared__ u64 cache[256];
+  cache[threadIdx.x] = TRIPLE_EMPTY;
+  __syncthreads();
+  i64 mn = INT64_MAX, mx = INT64_MIN, md = 0;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    Rec r = load_rec(ev, i);
+    int w = window_of(off, W, i);
+    int def = defect_of(r, t0[w], t1[w]);
+    if (def) {
+      int64_t *f = def == 1 ? &sum[w].n_bad_kind
+                            : def == 2 ? &sum[w].n_bad_interval : &sum[w].n_out_of_window;
+      atomicAdd((u64 *)f, 1ull);
+      continue;
+    }
+    mn = min(mn, (i64)r.name);
+    mx = max(mx, (i64)r.name);
+    md = max(md, r.ts_end - r.ts_start);
+    u64 code = triple_code(r.pid, r.kind, r.stream);
+    u32 hsh = hash_code(code);
+    if (cache[hsh & 255] == code) continue;  // a stale miss only costs a probe
+    u32 slot = hsh & (TA_TRIPLE_SLOTS - 1);
+    bool done = false;
+    for (int probe = 0; probe < TA_TRIPLE_SLOTS; probe++) {
+      u64 cur = ld_relaxed(&tt->slots[slot]);
+      if (cur == code) { done = true; break; }
+      if (cur == TRIPLE_EMPTY) {
+        u64 old = atomicCAS(&tt->slots[slot], TRIPLE_EMPTY, code);
+        if (old == TRIPLE_EMPTY || old == code) { done = true; break; }
+      }
+      slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
+    }
+    if (!done) ta_set_err(status, TA_ERR_TOO_LARGE);
+    cache[hsh & 255] = code;
+  }
+  mn = warp_min_i64(mn);
+  mx = warp_max_i64(mx);
+  md = warp_max_i64(md);
+  if ((threadIdx.x & 31) == 0) {
+    if (mn != INT64_MAX) {
+      atomicMin((i64 *)&misc[0], mn);
+      atomicMax((i64 *)&misc[1], mx);
+    }
+    if (md > 0) atomicMax((i64 *)&misc[2], md);
+  }
+}
+
+// One CTA: sorts the discovered triples, ranks them and the pids they contain.
+__global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t *status) {
+  extern __shared__ u64 buf[];  // TA_TRIPLE_SLOTS
+  const int tid = threadIdx.x;
+  for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x) buf[i] = tt->slots[i];
+  __syncthreads();
+  for (int k = 2; k <= TA_TRIPLE_SLOTS; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x) {
+        int ixj = i ^ j;
+        if (ixj > i) {
+          u64 a = buf[i], b = buf[ixj];
+          bool up = (i & k) == 0;
+          if ((a > b) == up) { buf[i] = b; buf[ixj] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  __shared__ int n_tr;
+  if (tid == 0) n_tr = 0;
+  __syncthreads();
+  for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x)
+    if (buf[i] != TRIPLE_EMPTY && (i + 1 == TA_TRIPLE_SLOTS || buf[i + 1] == TRIPLE_EMPTY)) n_tr = i + 1;
+  __syncthreads();
+  int n = n_tr;
+  if (n > TA_MAX_TRIPLES) {
+    if (tid == 0) ta_set_err(status, TA_ERR_TOO_LARGE);
+    n = TA_MAX_TRIPLES;
+  }
+  for (int i = tid; i < n; i += blockDim.x) tt->sorted_code[i] = buf[i];
+  if (tid == 0) {
+    int pr = -1;
+    u64 prev = ~0ull;
+    for (int i = 0; i < n; i++) {
+      u64 pidb = buf[i] >> 17;
+      if (pidb != prev) { pr++; prev = pidb; tt->pid_value[pr] = (int32_t)((u32)pidb ^ 0x80000000u); }
+      tt->pid_rank[i] = pr;
+    }
+    status[ST_N_TRIPLES] = n;
+    status[ST_N_PIDS] = pr + 1;
+  }
+  for (int s = tid; s < TA_TRIPLE_SLOTS; s += blockDim.x) {
+    u64 c = tt->slots[s];
+    int r = -1;
+    if (c != TRIPLE_EMPTY) {
+      int lo = 0, hi = n - 1;
+      while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (buf[mid] < c) lo = mid + 1;
+        else hi = mid;
+      }
+      r = lo;
+    }
+    tt->rank_of_slot[s] = r;
+  }
+}
+
+struct LoadArgs {
+  const ta_event *ev;
+  int64_t n;
+  const int64_t *off, *t0, *t1;
+  int W;
+  const TripleTable *tt;
+  u64 *keys;
+  u32 *hist;
+  int sbits, tbits, wbits;
+  SortPlan plan;
+};
+
+// Pass 2 over the records: sort key and the digit histograms of all passes.
+__global__ void __launch_bounds__(256) k_load(LoadArgs a) {
+  __shared__ u32 sh[10 * 256];
+  for (int i = threadIdx.x; i < a.plan.n_pass * 256; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  const u64 dropped_key = 1ull << (a.sbits + a.tbits + a.wbits);
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t n_round = ((a.n + 31) / 32) * 32;  // keep warps converged for match_any
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += stride) {
+    bool in = i < a.n;
+    u64 key = 0;
+    if (in) {
+      Rec r = load_rec(a.ev, i);
+      int w = window_of(a.off, a.W, i);
+      if (defect_of(r, a.t0[w], a.t1[w])) {
+        key = dropped_key;
+      } else {
+        u64 code = triple_code(r.pid, r.kind, r.stream);
+        u32 slot = hash_code(code) & (TA_TRIPLE_SLOTS - 1);
+        while (__ldg(&a.tt->slots[slot]) != code) slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
+        u64 rank = (u64)__ldg(&a.tt->rank_of_slot[slot]);
+        key = ((u64)w << (a.tbits + a.sbits)) | (rank << a.sbits) | (u64)(r.ts_start - a.t0[w]);
+      }
+      a.keys[i] = key;
+    }
+    u32 active = __ballot_sync(0xffffffffu, in);
+    if (!in) continue;
+    const int lane = threadIdx.x & 31;
+    for (int p = 0; p < a.plan.n_pass; p++) {
+      u32 d = (u32)(key >> a.plan.shift[p]) & ((1u << a.plan.bits[p]) - 1u);
+      u32 m = __match_any_sync(active, d);
+      if (lane == __ffs(m) - 1) atomicAdd(&sh[p * 256 + d], (u32)__popc(m));
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < a.plan.n_pass * 256; i += blockDim.x)
+    if (sh[i]) atomicAdd(&a.hist[i], sh[i]);
+}
+
+// ------------------------------------------------------------------ host
+static int bit_length(uint64_t v) {
+  int b = 0;
+  while (v) { b++; v >>= 1; }
+  return b;
+}
+
+static int grid_for(int64_t n, int threads, int per_sm) {
+  int64_t g = (n + threads - 1) / threads;
+  int64_t cap = 148ll * per_sm;
+  return (int)(g < 1 ? 1 : (g > cap ? cap : g));
+}
+
+ta_status ta_launch_discover(ta_window *h) {
+  if (h->n > 0) {
+    k_discover<<<grid_for(h->n, 256, 8), 256, 0, h->stream>>>(
+        h->events, h->n, h->d_off, h->d_t0, h->d_t1, h->W, h->d_triples, h->d_load_sum, h->d_misc,
+        h->d_status);
+  }
+  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank_triples, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        TA_TRIPLE_SLOTS * (int)sizeof(u64)));
+  k_rank_triples<<<1, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_status);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  return TA_OK;
+}
+
+ta_status ta_launch_load(ta_window *h) {
+  // key layout: [dropped][window][triple rank][ts_start - t0]
+  int64_t max_span = 1;
+  for (int w = 0; w < h->W; w++) max_span = max_span > h->h_t1[w] - h->h_t0[w] ? max_span : h->h_t1[w] - h->h_t0[w];
+  h->sbits = bit_length((uint64_t)(max_span - 1));
+  h->tbits = bit_length((uint64_t)(h->n_triples > 0 ? h->n_triples - 1 : 0));
+  h->wbits = bit_length((uint64_t)(h->W - 1));
+  int total = h->sbits + h->tbits + h->wbits + (h->has_dropped ? 1 : 0);
+  if (total > 63) return TA_ERR_TOO_LARGE;
+  if (((int64_t)h->W << h->tbits) > (1ll << 24)) return TA_ERR_TOO_LARGE;
+  h->plan = ta_make_plan(0, total);
+  if (h->n == 0) return TA_OK;
+  LoadArgs a;
+  a.ev = h->events; a.n = h->n; a.off = h->d_off; a.t0 = h->d_t0; a.t1 = h->d_t1; a.W = h->W;
+  a.tt = h->d_triples; a.keys = h->d_keys; a.hist = h->d_hist;
+  a.sbits = h->sbits; a.tbits = h->tbits; a.wbits = h->wbits; a.plan = h->plan;
+  k_load<<<grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  return TA_OK;
+}

@@ -1,0 +1,255 @@
+// Stable LSD radix sort of (64-bit key, 32-bit value) pairs: one scatter pass
+// per digit with a chained-scan ("one sweep") over tiles, so each pass reads and
+// writes every pair exactly once.  Digits are at most 8 bits wide; the digit
+// histograms of all passes are taken up front (by the load kernel for the
+// timeline sort, by k_radix_hist otherwise).
+//
+// Tile layout: RS_THREADS x RS_ITEMS pairs per CTA, keys staged through shared
+// memory so that both the global loads (warp-striped) and the scattered stores
+// (runs of equal digits) are coalesced.  HBM-bound: 12 B read + 12 B written
+// per pair and pass.
+#include "ta_internal.cuh"
+
+#define RS_THREADS 384
+#define RS_ITEMS 12
+#define RS_TILE (RS_THREADS * RS_ITEMS)
+#define RS_WARPS (RS_THREADS / 32)
+#define RS_BINS 256
+
+struct RadixArgs {
+  const u64 *keys_in;
+  u64 *keys_out;
+  const u32 *vals_in;  // may be null: value = global index
+  u32 *vals_out;
+  int64_t n;
+  int shift, bits;
+  const u32 *bin_offset;  // exclusive global digit offsets of this pass
+  u64 *tile_state;        // [tile][RS_BINS]
+  u32 *tile_counter;
+  int32_t *status;
+};
+
+struct RadixSmem {
+  u64 keys[RS_TILE];  // aliased by u32 values after the keys are written out
+  u32 warp_hist[RS_WARPS][RS_BINS];
+  u32 bin_start[RS_BINS];
+  i64 adj[RS_BINS];
+  u64 scan_tmp[33];
+  int tile;
+  int fail;
+};
+
+__global__ void __launch_bounds__(RS_THREADS) k_radix_pass(RadixArgs a) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  RadixSmem &s = *reinterpret_cast<RadixSmem *>(smem_raw);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    s.tile = (int)atomicAdd(a.tile_counter, 1u);
+    s.fail = 0;
+  }
+  for (int i = tid; i < RS_WARPS * RS_BINS; i += RS_THREADS) (&s.warp_hist[0][0])[i] = 0;
+  __syncthreads();
+  const int tile = s.tile;
+  const int64_t base = (int64_t)tile * RS_TILE;
+  const int count = (int)min((int64_t)RS_TILE, a.n - base);
+  const u32 mask = (1u << a.bits) - 1u;
+
+  u64 key[RS_ITEMS];
+  int lrank[RS_ITEMS];
+  const int wbase = warp * 32 * RS_ITEMS;
+#pragma unroll
+  for (int j = 0; j < RS_ITEMS; j++) {
+    int li = wbase + j * 32 + lane;
+    key[j] = li < count ? a.keys_in[base + li] : ~0ull;
+  }
+  // rank inside the warp, item row by item row (stable: row-major, then lane)
+#pragma unroll
+  for (int j = 0; j < RS_ITEMS; j++) {
+    int li = wbase + j * 32 + lane;
+    bool valid = li < count;
+    u32 d = valid ? ((u32)(key[j] >> a.shift) & mask) : 0xFFFFFFFFu;
+    u32 m = __match_any_sync(0xffffffffu, d);
+    int leader = __ffs(m) - 1;
+    u32 pre = 0;
+    if (valid && lane == leader) {
+      pre = s.warp_hist[warp][d];
+      s.warp_hist[warp][d] = pre + __popc(m);
+    }
+    pre = __shfl_sync(0xffffffffu, pre, leader);
+    lrank[j] = (int)(pre + __popc(m & ((1u << lane) - 1u)));
+    __syncwarp();
+  }
+  __syncthreads();
+  // per digit: exclusive offsets of the warps, then the CTA's digit count
+  u32 cnt = 0;
+  if (tid < RS_BINS) {
+    u32 run = 0;
+#pragma unroll
+    for (int w = 0; w < RS_WARPS; w++) {
+      u32 t = s.warp_hist[w][tid];
+      s.warp_hist[w][tid] = run;
+      run += t;
+    }
+    cnt = run;
+  }
+  u64 total;
+  u64 ex = block_scan_exclusive<OpAdd>((u64)cnt, OpAdd(), s.scan_tmp, &total);
+  if (tid < RS_BINS) s.bin_start[tid] = (u32)ex;
+  // chained scan over tiles, one digit per thread
+  if (tid < (1 << a.bits)) {
+    u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
+    u64 excl;
+    if (tile == 0) {
+      excl = a.bin_offset[tid];
+      st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
+    } else {
+      st_relaxed(st, td_pack(TD_AGG, cnt));
+      excl = 0;
+      bool timed_out = false;
+      for (int t = tile - 1;; --t) {
+        u64 w = td_wait(a.tile_state + (size_t)t * RS_BINS + tid, a.status, &timed_out);
+        excl += w & TD_MASK;
+        if ((w >> 62) == TD_PREFIX) break;
+      }
+      st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
+      if (timed_out) s.fail = 1;
+    }
+    s.adj[tid] = (i64)excl - (i64)ex;
+  }
+  __syncthreads();
+  if (s.fail) return;
+  // stage keys in shared memory in digit order
+#pragma unroll
+  for (int j = 0; j < RS_ITEMS; j++) {
+    int li = wbase + j * 32 + lane;
+    if (li < count) {
+      u32 d = (u32)(key[j] >> a.shift) & mask;
+      lrank[j] += (int)(s.bin_start[d] + s.warp_hist[warp][d]);
+      s.keys[lrank[j]] = key[j];
+    }
+  }
+  __syncthreads();
+  u32 gpos[RS_ITEMS];
+#pragma unroll
+  for (int k = 0; k < RS_ITEMS; k++) {
+    int sl = tid + k * RS_THREADS;
+    gpos[k] = 0xFFFFFFFFu;
+    if (sl < count) {
+      u64 kk = s.keys[sl];
+      u32 d = (u32)(kk >> a.shift) & mask;
+      i64 p = s.adj[d] + sl;
+      gpos[k] = (u32)p;
+      a.keys_out[p] = kk;
+    }
+  }
+  __syncthreads();
+  u32 *svals = reinterpret_cast<u32 *>(s.keys);
+#pragma unroll
+  for (int j = 0; j < RS_ITEMS; j++) {
+    int li = wbase + j * 32 + lane;
+    if (li < count) svals[lrank[j]] = a.vals_in ? a.vals_in[base + li] : (u32)(base + li);
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < RS_ITEMS; k++) {
+    int sl = tid + k * RS_THREADS;
+    if (sl < count) a.vals_out[gpos[k]] = svals[sl];
+  }
+}
+
+// digit histograms of every pass (used when the caller has none)
+__global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, int64_t n, SortPlan plan,
+                                                    u32 *hist) {
+  __shared__ u32 sh[10 * RS_BINS];
+  for (int i = threadIdx.x; i < plan.n_pass * RS_BINS; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x) {
+    u64 k = keys[i];
+    for (int p = 0; p < plan.n_pass; p++)
+      atomicAdd(&sh[p * RS_BINS + ((u32)(k >> plan.shift[p]) & ((1u << plan.bits[p]) - 1u))], 1u);
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < plan.n_pass * RS_BINS; i += blockDim.x)
+    if (sh[i]) atomicAdd(&hist[i], sh[i]);
+}
+
+// exclusive scan of each pass's histogram: one CTA of 256 threads per pass
+__global__ void __launch_bounds__(256) k_radix_scan_hist(const u32 *hist, u32 *bin_offset) {
+  __shared__ u64 tmp[33];
+  u64 total;
+  u32 v = hist[blockIdx.x * RS_BINS + threadIdx.x];
+  u64 ex = block_scan_exclusive<OpAdd>((u64)v, OpAdd(), tmp, &total);
+  bin_offset[blockIdx.x * RS_BINS + threadIdx.x] = (u32)ex;
+}
+
+SortPlan ta_make_plan(int lo_bit, int hi_bit) {
+  SortPlan p;
+  int total = hi_bit - lo_bit;
+  if (total < 1) total = 1;
+  p.n_pass = (total + 7) / 8;
+  int b = lo_bit;
+  for (int i = 0; i < p.n_pass; i++) {
+    int w = (total - (b - lo_bit) + (p.n_pass - i) - 1) / (p.n_pass - i);  // spread bits evenly
+    p.shift[i] = b;
+    p.bits[i] = w;
+    b += w;
+  }
+  return p;
+}
+
+static size_t n_tiles_of(int64_t n) { return (size_t)((n + RS_TILE - 1) / RS_TILE); }
+
+size_t ta_sort_temp_bytes(int64_t n) {
+  size_t tiles = n_tiles_of(n);
+  if (tiles == 0) tiles = 1;
+  return Carver::pad(tiles * RS_BINS * sizeof(u64)) + Carver::pad(16 * sizeof(u32)) +
+         2 * Carver::pad(10 * RS_BINS * sizeof(u32));
+}
+
+// Sorts n pairs by the key bits the plan covers.  Pass outputs alternate between
+// (keys_scratch, vals_scratch) and (keys_final, vals_final) such that the last
+// pass writes the final buffers; keys_in / vals_in are only read (vals_in null =
+// the value of pair i is i).  keys_in must not alias scratch or final.
+// `hist` = precomputed [pass][256] digit histograms, or null.
+ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_in,
+                              u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
+                              u32 *vals_final, int64_t n, const SortPlan &plan, const u32 *hist,
+                              void *temp) {
+  if (n <= 0) return TA_OK;
+  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_radix_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(RadixSmem)));
+  size_t tiles = n_tiles_of(n);
+  Carver c(temp);
+  u64 *state = c.take<u64>(tiles * RS_BINS);
+  u32 *counter = c.take<u32>(16);
+  u32 *bin_offset = c.take<u32>(10 * RS_BINS);
+  u32 *own_hist = c.take<u32>(10 * RS_BINS);
+  cudaStream_t st = h->stream;
+  if (!hist) {
+    TA_CHECK_CUDA(h, cudaMemsetAsync(own_hist, 0, 10 * RS_BINS * sizeof(u32), st));
+    int64_t want = (n + 255) / 256;
+    int grid = (int)(want < 148 * 8 ? want : 148 * 8);
+    k_radix_hist<<<grid, 256, 0, st>>>(keys_in, n, plan, own_hist);
+    hist = own_hist;
+  }
+  k_radix_scan_hist<<<plan.n_pass, 256, 0, st>>>(hist, bin_offset);
+  const u64 *kin = keys_in;
+  const u32 *vin = vals_in;
+  for (int p = 0; p < plan.n_pass; p++) {
+    bool to_final = ((plan.n_pass - 1 - p) & 1) == 0;
+    TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * RS_BINS * sizeof(u64), st));
+    TA_CHECK_CUDA(h, cudaMemsetAsync(counter, 0, sizeof(u32), st));
+    RadixArgs a;
+    a.keys_in = kin; a.keys_out = to_final ? keys_final : keys_scratch;
+    a.vals_in = vin; a.vals_out = to_final ? vals_final : vals_scratch;
+    a.n = n; a.shift = plan.shift[p]; a.bits = plan.bits[p];
+    a.bin_offset = bin_offset + p * RS_BINS;
+    a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
+    k_radix_pass<<<(unsigned)tiles, RS_THREADS, sizeof(RadixSmem), st>>>(a);
+    kin = a.keys_out;
+    vin = a.vals_out;
+  }
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  return TA_OK;
+}

@@ -1,0 +1,244 @@
+// C-ABI entry points (include/ta.h): argument checks, the handle, memory
+// through the caller's allocator, call-order bookkeeping.  All arithmetic lives
+// in the kernels of the other translation units.
+#include <cstring>
+#include <new>
+
+#include "ta_internal.cuh"
+
+void *ta_dalloc(ta_window *h, size_t bytes) {
+  if (bytes == 0) bytes = 256;
+  void *p = nullptr;
+  if (h->env.alloc) {
+    p = h->env.alloc(bytes, h->env.ctx);
+  } else {
+    if (cudaMallocAsync(&p, bytes, h->stream) != cudaSuccess) {
+      cudaGetLastError();
+      p = nullptr;
+    }
+  }
+  if (p) h->allocs.push_back(p);
+  return p;
+}
+
+static void release_one(ta_window *h, void *p) {
+  if (h->env.alloc) {
+    if (h->env.release) h->env.release(p, h->env.ctx);
+  } else {
+    cudaFreeAsync(p, h->stream);
+  }
+}
+
+void ta_dfree(ta_window *h, void *p) {
+  if (!p) return;
+  for (size_t i = 0; i < h->allocs.size(); i++)
+    if (h->allocs[i] == p) {
+      h->allocs[i] = h->allocs.back();
+      h->allocs.pop_back();
+      release_one(h, p);
+      return;
+    }
+}
+
+ta_status ta_read_status(ta_window *h, int32_t *w) {
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(w, h->d_status, ST_WORDS * sizeof(int32_t),
+                                   cudaMemcpyDeviceToHost, h->stream));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(h->stream));
+  return TA_OK;
+}
+
+extern "C" {
+
+const char *ta_strerror(ta_status s) {
+  switch (s) {
+    case TA_OK: return "ok";
+    case TA_ERR_INVALID_ARG: return "invalid argument";
+    case TA_ERR_OOM: return "device allocation failed";
+    case TA_ERR_CUDA: return "CUDA runtime error";
+    case TA_ERR_ORDER: return "entry point called before its prerequisites";
+    case TA_ERR_TOO_LARGE: return "size limit exceeded";
+    case TA_ERR_OVERFLOW: return "internal table overflow";
+    case TA_ERR_TIMEOUT: return "bounded device-side wait gave up";
+    case TA_ERR_DEPTH: return "operator nesting deeper than TA_MAX_DEPTH";
+    case TA_ERR_BAD_NESTING: return "partially overlapping ranges on one host thread";
+  }
+  return "unknown status";
+}
+
+int32_t ta_version(void) { return 1; }
+
+static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_device,
+                           ta_load_summary *out_summary) {
+  const int64_t n = h->n;
+  const int W = h->W;
+  cudaStream_t st = h->stream;
+  size_t bytes = 3 * Carver::pad((W + 1) * 8) + Carver::pad(ST_WORDS * 4) +
+                 Carver::pad(sizeof(TripleTable)) + Carver::pad(16 * 8) +
+                 Carver::pad(W * sizeof(ta_load_summary)) + Carver::pad(10 * 256 * 4) + 256;
+  void *b = ta_dalloc(h, bytes);
+  if (!b) return TA_ERR_OOM;
+  Carver c(b);
+  h->d_off = c.take<int64_t>(W + 1);
+  h->d_t0 = c.take<int64_t>(W + 1);
+  h->d_t1 = c.take<int64_t>(W + 1);
+  h->d_status = c.take<int32_t>(ST_WORDS);
+  h->d_triples = c.take<TripleTable>(1);
+  h->d_misc = c.take<int64_t>(16);
+  h->d_load_sum = c.take<ta_load_summary>(W);
+  h->d_hist = c.take<u32>(10 * 256);
+  h->d_keys = (u64 *)ta_dalloc(h, (size_t)(n > 0 ? n : 1) * 8);
+  if (!h->d_keys) return TA_ERR_OOM;
+
+  if (!on_device) {
+    h->events_copy = ta_dalloc(h, (size_t)(n > 0 ? n : 1) * sizeof(ta_event));
+    if (!h->events_copy) return TA_ERR_OOM;
+    if (n > 0)
+      TA_CHECK_CUDA(h, cudaMemcpyAsync(h->events_copy, events, (size_t)n * sizeof(ta_event),
+                                       cudaMemcpyHostToDevice, st));
+    h->events = (const ta_event *)h->events_copy;
+  } else {
+    h->events = events;
+  }
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_off, h->h_off.data(), (W + 1) * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t0, h->h_t0.data(), W * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t1, h->h_t1.data(), W * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status, 0, ST_WORDS * 4, st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_triples->slots, 0xFF, sizeof(h->d_triples->slots), st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_load_sum, 0, W * sizeof(ta_load_summary), st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_hist, 0, 10 * 256 * 4, st));
+  int64_t misc_init[16] = {0};
+  misc_init[0] = INT64_MAX;
+  misc_init[1] = INT64_MIN;
+  misc_init[2] = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_misc, misc_init, sizeof(misc_init), cudaMemcpyHostToDevice, st));
+
+  TA_TRY(ta_launch_discover(h));
+
+  int32_t words[ST_WORDS];
+  int64_t misc[16];
+  std::vector<ta_load_summary> sums(W);
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(misc, h->d_misc, sizeof(misc), cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(sums.data(), h->d_load_sum, W * sizeof(ta_load_summary),
+                                   cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_read_status(h, words));
+  if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+  h->n_triples = words[ST_N_TRIPLES];
+  h->n_pids = words[ST_N_PIDS];
+  h->min_name = misc[0];
+  h->max_name = misc[1];
+  h->max_dur = misc[2];
+  h->n_valid = 0;
+  for (int w = 0; w < W; w++) {
+    ta_load_summary &s = sums[w];
+    s.n_events = h->h_off[w + 1] - h->h_off[w];
+    s.n_valid = s.n_events - s.n_bad_kind - s.n_bad_interval - s.n_out_of_window;
+    h->n_valid += s.n_valid;
+    if (out_summary) out_summary[w] = s;
+  }
+  h->has_dropped = h->n_valid < n ? 1 : 0;
+  TA_TRY(ta_launch_load(h));
+  h->stage |= 1;
+  return TA_OK;
+}
+
+ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
+                         int32_t events_on_device, const int64_t *win_off, const int64_t *win_t0,
+                         const int64_t *win_t1, int32_t W, ta_load_summary *out_summary,
+                         ta_window **handle) {
+  if (!handle) return TA_ERR_INVALID_ARG;
+  *handle = nullptr;
+  if (!env || n < 0 || W < 1 || !win_off || !win_t0 || !win_t1 || (n > 0 && !events))
+    return TA_ERR_INVALID_ARG;
+  if (n >= (1ll << 31)) return TA_ERR_TOO_LARGE;
+  if ((env->alloc == nullptr) != (env->release == nullptr)) return TA_ERR_INVALID_ARG;
+  if (win_off[0] != 0 || win_off[W] != n) return TA_ERR_INVALID_ARG;
+  for (int w = 0; w < W; w++) {
+    if (win_off[w + 1] < win_off[w]) return TA_ERR_INVALID_ARG;
+    if (win_t0[w] >= win_t1[w]) return TA_ERR_INVALID_ARG;
+    if ((uint64_t)win_t1[w] - (uint64_t)win_t0[w] >= (1ull << 40)) return TA_ERR_TOO_LARGE;
+  }
+  ta_window *h = new (std::nothrow) ta_window();
+  if (!h) return TA_ERR_OOM;
+  h->env = *env;
+  h->stream = (cudaStream_t)env->cuda_stream;
+  h->device = env->device;
+  h->last_cuda = cudaSuccess;
+  h->n = n;
+  h->W = W;
+  h->stage = 0;
+  h->events = nullptr;
+  h->events_copy = nullptr;
+  h->d_keys = nullptr;
+  h->attr_status = 0;
+  h->h_off.assign(win_off, win_off + W + 1);
+  h->h_t0.assign(win_t0, win_t0 + W);
+  h->h_t1.assign(win_t1, win_t1 + W);
+  *handle = h;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
+  return load_impl(h, events, events_on_device, out_summary);
+}
+
+ta_status ta_sort_timeline(ta_window *h, ta_sort_result *out) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 1) || (h->stage & 2)) return TA_ERR_ORDER;
+  TA_TRY(ta_run_sort_timeline(h));
+  h->stage |= 2;
+  *out = h->sorted;
+  return TA_OK;
+}
+
+ta_status ta_correlate_launches(ta_window *h, ta_join_result *out, ta_join_summary *out_summary) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 2) || (h->stage & 4)) return TA_ERR_ORDER;
+  TA_TRY(ta_run_correlate(h, out_summary));
+  h->stage |= 4;
+  *out = h->join;
+  return TA_OK;
+}
+
+ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out, ta_attr_summary *out_summary) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 4) || (h->stage & 8)) return TA_ERR_ORDER;
+  ta_status s = ta_run_attribute(h, out_summary);
+  if (s != TA_OK && s != TA_ERR_DEPTH && s != TA_ERR_BAD_NESTING) return s;
+  h->stage |= 8;
+  h->attr_status = (int)s;
+  *out = h->attr;
+  return s;
+}
+
+ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 2)) return TA_ERR_ORDER;
+  return ta_run_gaps(h, min_gap_ns, out);
+}
+
+ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel, ta_agg_result *out) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (value_sel != 0 && value_sel != 1) return TA_ERR_INVALID_ARG;
+  if (value_sel == 1 && kind_mask != (1u << TA_KIND_OP)) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 2)) return TA_ERR_ORDER;
+  if (value_sel == 1 && (!(h->stage & 8) || h->attr_status != 0)) return TA_ERR_ORDER;
+  return ta_run_aggregate(h, kind_mask, value_sel, out);
+}
+
+ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_comms,
+                               ta_coll_result *out) {
+  if (!h || !out || n_comms < 0 || (n_comms > 0 && !sizes)) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 2)) return TA_ERR_ORDER;
+  return ta_run_collectives(h, sizes, n_comms, out);
+}
+
+void ta_free(ta_window *h) {
+  if (!h) return;
+  cudaSetDevice(h->device);
+  cudaStreamSynchronize(h->stream);
+  for (void *p : h->allocs) release_one(h, p);
+  h->allocs.clear();
+  delete h;
+}
+
+}  // extern "C"

@@ -1,0 +1,287 @@
+// Internal declarations of the trace-window analyzer CUDA library (sm_100a).
+// Host-side handle, memory helpers, and the device primitives every step
+// shares: relaxed loads/stores for tile descriptors, a bounded decoupled
+// look-back, warp/block scans.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "../../include/ta.h"
+
+typedef unsigned long long u64;
+typedef long long i64;
+typedef unsigned int u32;
+
+// ---------------------------------------------------------------- limits
+#define TA_MAX_TRIPLES 4096       // distinct (pid, domain, stream)
+#define TA_TRIPLE_SLOTS 8192      // open-addressing slots for them
+#define TA_MAX_COMMS 1024         // distinct communicator ids
+#define TA_COMM_SLOTS 2048
+#define TA_SPIN_LIMIT (1 << 22)   // polls of a tile descriptor before giving up
+#define TA_TIE_RUN_MAX 48         // equal-key runs up to this length are fixed in place
+#define TA_AGG_DENSE_LIMIT (1ll << 27)
+
+// device status word indices (h->d_status)
+enum { ST_ERR = 0, ST_LONG_RUN = 1, ST_N_TRIPLES = 2, ST_N_PIDS = 3, ST_N_COMMS = 4, ST_WORDS = 16 };
+
+struct TripleTable {       // device-resident, filled by the discovery kernel
+  u64 slots[TA_TRIPLE_SLOTS];          // biased code or EMPTY
+  int32_t rank_of_slot[TA_TRIPLE_SLOTS];
+  u64 sorted_code[TA_MAX_TRIPLES];     // ascending
+  int32_t pid_rank[TA_MAX_TRIPLES];    // per triple rank
+  int32_t pid_value[TA_MAX_TRIPLES];   // per pid rank
+};
+
+struct SortPlan {
+  int n_pass;
+  int shift[10];
+  int bits[10];
+};
+
+// --------------------------------------------------------------- handle
+struct ta_window {
+  ta_env env;
+  cudaStream_t stream;
+  int device;
+  cudaError_t last_cuda;
+  int64_t n;
+  int32_t W;
+  int stage;  // bit flags: 1 loaded, 2 sorted, 4 correlated, 8 attributed
+
+  const ta_event *events;  // device, borrowed (or events_copy)
+  void *events_copy;
+  std::vector<int64_t> h_off, h_t0, h_t1;
+  int64_t *d_off, *d_t0, *d_t1;
+
+  std::vector<void *> allocs;  // everything obtained from env.alloc
+
+  // load products
+  int32_t *d_status;
+  TripleTable *d_triples;
+  int64_t *d_misc;           // [0]=min name,[1]=max name,[2]=max duration (atomics)
+  ta_load_summary *d_load_sum;
+  u64 *d_keys;
+  u32 *d_hist;               // [pass][256]
+  int64_t n_valid;
+  int n_triples, n_pids;
+  int sbits, tbits, wbits, has_dropped;
+  int64_t min_name, max_name, max_dur;
+  SortPlan plan;
+
+  // sort products
+  ta_sort_result sorted;
+  u64 *d_sorted_keys;        // (window, triple, ts_rel) of each sorted position
+  int32_t *d_lane_code;      // per lane: window << tbits | triple rank
+  int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
+  std::vector<int32_t> h_lane_off;
+
+  // join / attribution products
+  ta_join_result join;
+  ta_attr_result attr;
+  int attr_status;
+};
+
+// -------------------------------------------------------------- memory
+void *ta_dalloc(ta_window *h, size_t bytes);            // NULL on failure
+void ta_dfree(ta_window *h, void *p);                   // early release of one allocation
+// carve sub-buffers out of one allocation
+struct Carver {
+  char *base;
+  size_t off;
+  explicit Carver(void *b = nullptr) : base((char *)b), off(0) {}
+  static size_t pad(size_t b) { return (b + 255) & ~(size_t)255; }
+  template <class T>
+  T *take(size_t count) {
+    T *p = (T *)(base + off);
+    off += pad(count * sizeof(T));
+    return p;
+  }
+};
+
+#define TA_CHECK_CUDA(h, x)                                  \
+  do {                                                       \
+    cudaError_t e__ = (x);                                   \
+    if (e__ != cudaSuccess) {                                \
+      (h)->last_cuda = e__;                                  \
+      return TA_ERR_CUDA;                                    \
+    }                                                        \
+  } while (0)
+#define TA_TRY(x)                      \
+  do {                                 \
+    ta_status s__ = (x);               \
+    if (s__ != TA_OK) return s__;      \
+  } while (0)
+
+// ----------------------------------------------- launchers (one per .cu)
+// sort.cu
+size_t ta_sort_temp_bytes(int64_t n);
+ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_in,
+                              u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
+                              u32 *vals_final, int64_t n, const SortPlan &plan,
+                              const u32 *hist /*nullable*/, void *temp);
+SortPlan ta_make_plan(int lo_bit, int hi_bit);
+// load.cu
+ta_status ta_launch_discover(ta_window *h);
+ta_status ta_launch_rank_triples(ta_window *h);
+ta_status ta_launch_load(ta_window *h);
+// timeline.cu
+ta_status ta_run_sort_timeline(ta_window *h);
+// join.cu
+ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary);
+// attr.cu
+ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary);
+// gaps.cu
+ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out);
+// agg.cu
+ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_agg_result *out);
+// coll.cu
+ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_comms,
+                             ta_coll_result *out);
+
+ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
+
+// =================================================================== device
+#ifdef __CUDACC__
+
+__device__ __forceinline__ u64 ld_relaxed(const u64 *p) {
+  u64 v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed(u64 *p, u64 v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ int32_t ld_relaxed_i32(const int32_t *p) {
+  int32_t v;
+  asm volatile("ld.relaxed.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+__device__ __forceinline__ void ta_set_err(int32_t *status, int code) {
+  atomicCAS(&status[ST_ERR], 0, code);
+}
+
+// Tile descriptor: bits 63..62 = flag, low 62 bits = value.
+#define TD_EMPTY 0ull
+#define TD_AGG 1ull
+#define TD_PREFIX 2ull
+#define TD_MASK ((1ull << 62) - 1)
+__device__ __forceinline__ u64 td_pack(u64 flag, u64 v) { return (flag << 62) | (v & TD_MASK); }
+
+// Polls a descriptor until it is published; gives up after TA_SPIN_LIMIT polls
+// (sets *timed_out and returns a PREFIX of 0 so that the caller terminates).
+__device__ __forceinline__ u64 td_wait(const u64 *p, int32_t *status, bool *timed_out) {
+  u64 w = ld_relaxed(p);
+  int spins = 0;
+  while ((w >> 62) == TD_EMPTY) {
+    if (++spins > TA_SPIN_LIMIT || ld_relaxed_i32(&status[ST_ERR]) != 0) {
+      *timed_out = true;
+      ta_set_err(status, TA_ERR_TIMEOUT);
+      return td_pack(TD_PREFIX, 0);
+    }
+    __nanosleep(40);
+    w = ld_relaxed(p);
+  }
+  return w;
+}
+
+struct OpAdd {
+  __device__ __forceinline__ u64 operator()(u64 a, u64 b) const { return a + b; }
+  __device__ __forceinline__ u64 identity() const { return 0; }
+};
+struct OpMax {
+  __device__ __forceinline__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; }
+  __device__ __forceinline__ u64 identity() const { return 0; }
+};
+
+template <class Op>
+__device__ __forceinline__ u64 warp_reduce(u64 v, Op op) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = op(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+template <class Op>
+__device__ __forceinline__ u64 warp_scan_inclusive(u64 v, Op op) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    u64 t = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v = op(t, v);
+  }
+  return v;
+}
+
+// Decoupled look-back for one value per tile; called by all 32 lanes of ONE
+// warp.  Publishes this tile's aggregate, combines the predecessors' values
+// (commutative op) and publishes the inclusive prefix.  Returns the exclusive
+// prefix in every lane.
+template <class Op>
+__device__ __forceinline__ u64 tile_lookback(u64 *state, int tile, u64 aggregate, Op op,
+                                             int32_t *status) {
+  const int lane = threadIdx.x & 31;
+  if (tile == 0) {
+    if (lane == 0) st_relaxed(&state[0], td_pack(TD_PREFIX, aggregate));
+    return op.identity();
+  }
+  if (lane == 0) st_relaxed(&state[tile], td_pack(TD_AGG, aggregate));
+  u64 excl = op.identity();
+  bool timed_out = false;
+  for (int base = tile - 1;; base -= 32) {
+    int idx = base - lane;
+    u64 w = idx >= 0 ? td_wait(&state[idx], status, &timed_out) : td_pack(TD_PREFIX, op.identity());
+    u32 pm = __ballot_sync(0xffffffffu, (w >> 62) == TD_PREFIX);
+    int first = pm ? (__ffs(pm) - 1) : 31;
+    u64 c = lane <= first ? (w & TD_MASK) : op.identity();
+    c = warp_reduce(c, op);
+    excl = op(c, excl);
+    if (pm) break;
+  }
+  if (lane == 0) st_relaxed(&state[tile], td_pack(TD_PREFIX, op(excl, aggregate)));
+  return excl;
+}
+
+// Block-wide exclusive scan of one value per thread (blockDim.x multiple of 32,
+// <= 1024).  `smem` needs 33 u64.  Returns the exclusive prefix; *total gets the
+// block aggregate in every thread.
+template <class Op>
+__device__ __forceinline__ u64 block_scan_exclusive(u64 v, Op op, u64 *smem, u64 *total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  u64 inc = warp_scan_inclusive(v, op);
+  if (lane == 31) smem[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    u64 w = lane < nw ? smem[lane] : op.identity();
+    u64 wi = warp_scan_inclusive(w, op);
+    if (lane < nw) smem[lane] = wi;
+    if (lane == nw - 1) smem[32] = wi;
+  }
+  __syncthreads();
+  u64 prev_lane = __shfl_up_sync(0xffffffffu, inc, 1);
+  u64 ex = lane == 0 ? op.identity() : prev_lane;
+  if (warp > 0) ex = op(smem[warp - 1], ex);
+  *total = smem[32];
+  __syncthreads();
+  return ex;
+}
+
+// Lane of a sorted position: binary search in lane_off (n_lanes + 1 entries).
+__device__ __forceinline__ int lane_of_pos(const int32_t *lane_off, int n_lanes, int64_t p) {
+  int lo = 0, hi = n_lanes - 1;
+  while (lo < hi) {
+    int mid = (lo + hi + 1) >> 1;
+    if ((int64_t)lane_off[mid] <= p) lo = mid;
+    else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ int log2_bin(int64_t v) {
+  if (v <= 1) return 0;
+  int b = 63 - __clzll(v);
+  return b > TA_NBINS - 1 ? TA_NBINS - 1 : b;
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,286 @@
+// ta_sort_timeline: canonical order of the timeline.
+//
+//   1. stable radix sort of (key, input index) by the key built at load time
+//      (window | lane triple rank | ts_start - t0); stability gives the input
+//      index tie-break for free;
+//   2. runs of equal keys are reordered by ts_end descending (short runs in
+//      place; if a longer run exists the sort is redone with the duration as a
+//      least-significant key);
+//   3. dropped records (tail) are ordered by the full tuple with a chain of
+//      stable sorts;
+//   4. whole 40-byte records are gathered once into eight sorted columns and
+//      lane boundaries are recorded.
+#include "records.cuh"
+#include "ta_internal.cuh"
+
+// ---- step 2: equal-key runs --------------------------------------------
+__global__ void __launch_bounds__(256) k_fix_ties(const u64 *keys, u32 *perm, int64_t n_valid,
+                                                  const ta_event *ev, int32_t *status) {
+  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n_valid || p + 1 >= n_valid) return;
+  u64 k = keys[p];
+  if (keys[p + 1] != k) return;
+  if (p > 0 && keys[p - 1] == k) return;
+  int len = 2;
+  while (p + len < n_valid && len <= TA_TIE_RUN_MAX && keys[p + len] == k) len++;
+  if (len > TA_TIE_RUN_MAX) {
+    status[ST_LONG_RUN] = 1;
+    return;
+  }
+  u32 idx[TA_TIE_RUN_MAX];
+  i64 end[TA_TIE_RUN_MAX];
+  for (int i = 0; i < len; i++) {
+    idx[i] = perm[p + i];
+    end[i] = reinterpret_cast<const i64 *>(ev)[(int64_t)idx[i] * 5 + 1];
+  }
+  for (int i = 1; i < len; i++) {  // stable insertion sort, ts_end descending
+    u32 xi = idx[i];
+    i64 xe = end[i];
+    int j = i - 1;
+    while (j >= 0 && end[j] < xe) {
+      idx[j + 1] = idx[j];
+      end[j + 1] = end[j];
+      j--;
+    }
+    idx[j + 1] = xi;
+    end[j + 1] = xe;
+  }
+  for (int i = 0; i < len; i++) perm[p + i] = idx[i];
+}
+
+// ---- fallback: duration as a least-significant key ------------------------
+__global__ void __launch_bounds__(256) k_duration_key(const ta_event *ev, int64_t n, const u64 *keys,
+                                                      u64 dropped_bit, i64 max_dur, u64 *out) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  if (keys[i] & dropped_bit) { out[i] = 0; return; }
+  const i64 *p = reinterpret_cast<const i64 *>(ev) + i * 5;
+  out[i] = (u64)(max_dur - (p[1] - p[0]));  // longer first
+}
+__global__ void __launch_bounds__(256) k_gather_u64(const u64 *src, const u32 *idx, int64_t n, u64 *dst) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[idx[i]];
+}
+
+// ---- step 3: full-tuple keys for the dropped tail -------------------------
+// stage 0: ~ts_end, 1: ts_start, 2: (pid, domain, stream), 3: window
+__global__ void __launch_bounds__(256) k_tail_key(const ta_event *ev, const u32 *idx, int64_t m,
+                                                  int stage, const int64_t *off, int W, u64 *out) {
+  int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= m) return;
+  Rec r = load_rec(ev, idx[j]);
+  u64 k;
+  if (stage == 0) k = ~((u64)r.ts_end ^ (1ull << 63));
+  else if (stage == 1) k = (u64)r.ts_start ^ (1ull << 63);
+  else if (stage == 2) k = triple_code(r.pid, r.kind, r.stream);
+  else k = (u64)window_of(off, W, idx[j]);
+  out[j] = k;
+}
+
+// ---- step 4: gather records into sorted columns + lane heads ---------------
+struct GatherArgs {
+  const ta_event *ev;
+  const u32 *perm;
+  const u64 *keys;
+  int64_t n, n_valid;
+  int sbits;
+  i64 *ts_start, *ts_end, *corr;
+  int32_t *pid, *name, *seq;
+  int16_t *stream, *kind;
+  int32_t *lane_start;  // per lane code, -1 = empty
+};
+
+__global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
+  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= a.n) return;
+  Rec r = load_rec(a.ev, a.perm[p]);
+  a.ts_start[p] = r.ts_start;
+  a.ts_end[p] = r.ts_end;
+  a.corr[p] = r.corr;
+  a.pid[p] = r.pid;
+  a.name[p] = r.name;
+  a.seq[p] = r.seq;
+  a.stream[p] = r.stream;
+  a.kind[p] = r.kind;
+  if (p < a.n_valid) {
+    u64 code = a.keys[p] >> a.sbits;
+    if (p == 0 || (a.keys[p - 1] >> a.sbits) != code) a.lane_start[code] = (int32_t)p;
+  }
+}
+
+// One CTA: compacts the non-empty lane codes into the lane table (code order is
+// canonical order).
+__global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, int64_t n_codes,
+                                                     int tbits, int n_pids, const TripleTable *tt,
+                                                     int64_t n_valid, int32_t *lane_window,
+                                                     int32_t *lane_pid, int16_t *lane_stream,
+                                                     int16_t *lane_domain, int32_t *lane_off,
+                                                     int32_t *lane_code, int32_t *lane_slot,
+                                                     int32_t *n_lanes_out, int64_t cap) {
+  __shared__ u64 tmp[33];
+  __shared__ u64 base;
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int64_t c0 = 0; c0 < n_codes; c0 += blockDim.x) {
+    int64_t c = c0 + threadIdx.x;
+    int32_t st = c < n_codes ? lane_start[c] : -1;
+    u64 total;
+    u64 ex = block_scan_exclusive<OpAdd>(st >= 0 ? 1ull : 0ull, OpAdd(), tmp, &total);
+    if (st >= 0) {
+      int64_t l = (int64_t)(base + ex);
+      if (l < cap) {
+        int w = (int)(c >> tbits), t = (int)(c & ((1ll << tbits) - 1));
+        u64 code = tt->sorted_code[t];
+        lane_window[l] = w;
+        lane_pid[l] = code_pid(code);
+        lane_stream[l] = code_stream(code);
+        lane_domain[l] = code_domain(code);
+        lane_off[l] = st;
+        lane_code[l] = (int32_t)c;
+        lane_slot[l] = w * n_pids + tt->pid_rank[t];
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) base += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    int64_t L = (int64_t)base;
+    if (L < cap + 1) lane_off[L] = (int32_t)n_valid;
+    *n_lanes_out = (int32_t)L;
+  }
+}
+
+static inline int nblk(int64_t n, int t) { return (int)((n + t - 1) / t); }
+
+ta_status ta_run_sort_timeline(ta_window *h) {
+  const int64_t n = h->n;
+  cudaStream_t st = h->stream;
+  const int64_t n_codes = (int64_t)h->W << h->tbits;  // lane code = window << tbits | triple rank
+  const int64_t lane_cap = (n_codes < n ? n_codes : n) + 1;  // lanes <= min(codes, records)
+
+  // result buffers (kept until ta_free)
+  size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
+                2 * Carver::pad(n * 2) + Carver::pad(n * 8) /*sorted keys*/ +
+                4 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
+                Carver::pad((lane_cap + 1) * 4) + 512;
+  void *kb = ta_dalloc(h, keep);
+  if (!kb) return TA_ERR_OOM;
+  Carver ck(kb);
+  u32 *perm = ck.take<u32>(n);
+  i64 *c_ts = ck.take<i64>(n), *c_te = ck.take<i64>(n), *c_corr = ck.take<i64>(n);
+  int32_t *c_pid = ck.take<int32_t>(n), *c_name = ck.take<int32_t>(n), *c_seq = ck.take<int32_t>(n);
+  int16_t *c_stream = ck.take<int16_t>(n), *c_kind = ck.take<int16_t>(n);
+  u64 *skeys = ck.take<u64>(n);
+  int32_t *lane_window = ck.take<int32_t>(lane_cap), *lane_pid = ck.take<int32_t>(lane_cap);
+  int32_t *lane_code = ck.take<int32_t>(lane_cap), *lane_slot = ck.take<int32_t>(lane_cap);
+  int16_t *lane_stream = ck.take<int16_t>(lane_cap), *lane_domain = ck.take<int16_t>(lane_cap);
+  int32_t *lane_off = ck.take<int32_t>(lane_cap + 1);
+  int32_t *n_lanes_dev = ck.take<int32_t>(1);
+
+  // temporaries (released at the end of the call)
+  size_t tmp_bytes = Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
+                     Carver::pad(n_codes * 4) + 512;
+  void *tb = ta_dalloc(h, tmp_bytes);
+  if (!tb) return TA_ERR_OOM;
+  Carver ct(tb);
+  u64 *kscr = ct.take<u64>(n);
+  u32 *vscr = ct.take<u32>(n);
+  int32_t *lane_start = ct.take<int32_t>(n_codes);
+  void *sort_tmp = ct.base + ct.off;
+
+  TA_CHECK_CUDA(h, cudaMemsetAsync(lane_start, 0xFF, n_codes * sizeof(int32_t), st));
+  if (n > 0) {
+    // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
+    TA_TRY(ta_radix_sort_pairs(h, h->d_keys, nullptr, kscr, vscr, skeys, perm, n, h->plan,
+                               h->d_hist, sort_tmp));
+    // step 2: equal-key runs
+    if (h->n_valid > 1)
+      k_fix_ties<<<nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
+                                                        h->d_status);
+    int32_t words[ST_WORDS];
+    TA_TRY(ta_read_status(h, words));
+    if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+    if (words[ST_LONG_RUN]) {
+      // redo with the duration as a least-significant key: first a stable sort by
+      // (max_dur - duration), then the timeline key on top of that order
+      void *xb = ta_dalloc(h, Carver::pad(n * 8) + Carver::pad(n * 4));
+      if (!xb) return TA_ERR_OOM;
+      Carver cx(xb);
+      u64 *dkeys = cx.take<u64>(n);
+      u32 *dorder = cx.take<u32>(n);
+      const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
+      k_duration_key<<<nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit, h->max_dur,
+                                                   dkeys);
+      int dbits = 1;
+      while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
+      SortPlan dplan = ta_make_plan(0, dbits);
+      TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
+                                 sort_tmp));
+      k_gather_u64<<<nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
+      TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
+                                 sort_tmp));
+      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+      ta_dfree(h, xb);
+    }
+    // step 3: dropped tail, chain of stable sorts over the full tuple (least
+    // significant field first)
+    const int64_t m = n - h->n_valid;
+    if (m > 1) {
+      void *xb = ta_dalloc(h, 2 * Carver::pad(m * 8) + Carver::pad(m * 4));
+      if (!xb) return TA_ERR_OOM;
+      Carver cx(xb);
+      u64 *tk = cx.take<u64>(m), *tk2 = cx.take<u64>(m);
+      u32 *alt = cx.take<u32>(m);
+      u32 *cur = perm + h->n_valid, *nxt = alt;
+      for (int stage = 0; stage < 4; stage++) {
+        if (stage == 3 && h->W == 1) break;
+        k_tail_key<<<nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
+        int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : 64;
+        SortPlan tp = ta_make_plan(0, bits);
+        TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
+        u32 *t = cur; cur = nxt; nxt = t;
+      }
+      if (cur != perm + h->n_valid)
+        TA_CHECK_CUDA(h, cudaMemcpyAsync(perm + h->n_valid, cur, m * sizeof(u32),
+                                         cudaMemcpyDeviceToDevice, st));
+      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+      ta_dfree(h, xb);
+    }
+    // step 4
+    GatherArgs g;
+    g.ev = h->events; g.perm = perm; g.keys = skeys; g.n = n; g.n_valid = h->n_valid;
+    g.sbits = h->sbits;
+    g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
+    g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
+    k_gather<<<nblk(n, 256), 256, 0, st>>>(g);
+  }
+  k_lane_table<<<1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
+                                   h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
+                                   lane_window, lane_pid, lane_stream, lane_domain, lane_off,
+                                   lane_code, lane_slot, n_lanes_dev, lane_cap);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  int32_t n_lanes = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  h->h_lane_off.assign((size_t)n_lanes + 1, 0);
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_lane_off.data(), lane_off, ((size_t)n_lanes + 1) * 4,
+                                   cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  ta_dfree(h, tb);
+  ta_dfree(h, h->d_keys);
+  h->d_keys = nullptr;
+
+  ta_sort_result &r = h->sorted;
+  r.n = n; r.n_valid = h->n_valid; r.n_lanes = n_lanes; r.n_windows = h->W;
+  r.perm = (const int32_t *)perm;
+  r.ts_start = (const int64_t *)c_ts; r.ts_end = (const int64_t *)c_te;
+  r.corr_id = (const int64_t *)c_corr;
+  r.pid = c_pid; r.name_id = c_name; r.seq = c_seq; r.stream = c_stream; r.kind = c_kind;
+  r.lane_window = lane_window; r.lane_pid = lane_pid; r.lane_stream = lane_stream;
+  r.lane_domain = lane_domain; r.lane_off = lane_off;
+  h->d_sorted_keys = skeys;
+  h->d_lane_code = lane_code;
+  h->d_lane_slot = lane_slot;
+  return TA_OK;
+}

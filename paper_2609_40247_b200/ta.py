@@ -1,0 +1,383 @@
+"""Python binding of the C ABI in include/ta.h (argument marshalling only).
+
+Every step runs in the CUDA library (libta.so, built by
+`python -m paper_2609_40247_b200.build`); PyTorch supplies device memory (its
+caching allocator, through the ta_env callbacks) and the stream.  There is no
+CPU fallback: if the library is missing, loading fails with an error.
+
+    with ta.Window(events_u8_cuda, win_off, t0, t1) as w:
+        s = w.sort_timeline();  j = w.correlate_launches();  a = w.attribute_operators()
+        g = w.stream_gaps(500_000);  k = w.aggregate_ops(ta.DEVICE_KINDS, 0)
+        c = w.match_collectives([(comm_id, n_ranks), ...])
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libta.so")
+
+KIND_OP, KIND_API, KIND_LAUNCH, KIND_KERNEL, KIND_MEMCPY, KIND_COLL = range(6)
+DEVICE_KINDS = (1 << KIND_KERNEL) | (1 << KIND_MEMCPY) | (1 << KIND_COLL)
+NBINS = 40
+
+STATUS_NAMES = ["TA_OK", "TA_ERR_INVALID_ARG", "TA_ERR_OOM", "TA_ERR_CUDA", "TA_ERR_ORDER",
+                "TA_ERR_TOO_LARGE", "TA_ERR_OVERFLOW", "TA_ERR_TIMEOUT", "TA_ERR_DEPTH",
+                "TA_ERR_BAD_NESTING"]
+TA_ERR_DEPTH, TA_ERR_BAD_NESTING = 8, 9
+
+EVENT_DTYPE = np.dtype([("ts_start", "<i8"), ("ts_end", "<i8"), ("corr_id", "<i8"), ("pid", "<i4"),
+                        ("name_id", "<i4"), ("seq", "<i4"), ("stream", "<i2"), ("kind", "<i2")])
+LOAD_SUM = np.dtype([(k, "<i8") for k in
+                     ("n_events", "n_valid", "n_bad_kind", "n_bad_interval", "n_out_of_window")])
+JOIN_SUM = np.dtype([(k, "<i8") for k in
+                     ("n_probe", "n_matched", "n_unmatched", "n_launch", "n_dup_launch",
+                      "n_orphan_launch", "sum_latency", "min_latency", "max_latency", "sum_queue",
+                      "max_queue")])
+ATTR_SUM = np.dtype([("n_attributed", "<i8"), ("n_no_launch", "<i8"), ("n_no_op", "<i8"),
+                     ("max_depth", "<i4"), ("bad_nesting", "<i4")])
+LANE_GAPS = np.dtype([(k, "<i8") for k in
+                      ("busy", "idle", "n_events", "n_gaps", "max_gap", "first_start", "last_end")])
+LONG_GAP = np.dtype([("lane", "<i4"), ("next_event", "<i4"), ("gap_start", "<i8"), ("gap_len", "<i8")])
+COMM_SIZE = np.dtype([("comm_id", "<i8"), ("n_ranks", "<i4"), ("reserved", "<i4")])
+
+_vp = ctypes.c_void_p
+_ALLOC_T = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p)
+_RELEASE_T = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_void_p)
+
+
+class _Env(ctypes.Structure):
+    _fields_ = [("alloc", _ALLOC_T), ("release", _RELEASE_T), ("ctx", _vp), ("cuda_stream", _vp),
+                ("device", ctypes.c_int32)]
+
+
+def _ptr_struct(name, fields):
+    return type(name, (ctypes.Structure,), {"_fields_": fields})
+
+
+_SortResult = _ptr_struct("_SortResult", [
+    ("n", ctypes.c_int64), ("n_valid", ctypes.c_int64), ("n_lanes", ctypes.c_int32),
+    ("n_windows", ctypes.c_int32), ("perm", _vp), ("ts_start", _vp), ("ts_end", _vp),
+    ("corr_id", _vp), ("pid", _vp), ("name_id", _vp), ("seq", _vp), ("stream", _vp), ("kind", _vp),
+    ("lane_window", _vp), ("lane_pid", _vp), ("lane_stream", _vp), ("lane_domain", _vp),
+    ("lane_off", _vp)])
+_JoinResult = _ptr_struct("_JoinResult", [
+    ("launch_of", _vp), ("launch_latency", _vp), ("queue_delay", _vp), ("kernels_of_launch", _vp)])
+_AttrResult = _ptr_struct("_AttrResult", [
+    ("parent", _vp), ("depth", _vp), ("op_of", _vp), ("op_first_start", _vp), ("op_last_end", _vp),
+    ("op_kernel_ns", _vp), ("op_n_kernels", _vp)])
+_GapResult = _ptr_struct("_GapResult", [
+    ("gap_before", _vp), ("lane_gaps", _vp), ("lane_hist", _vp), ("win_hist", _vp),
+    ("long_gaps", _vp), ("n_long_gaps", ctypes.c_int64)])
+_AggResult = _ptr_struct("_AggResult", [
+    ("n_groups", ctypes.c_int64), ("g_window", _vp), ("g_pid", _vp), ("g_name", _vp),
+    ("g_count", _vp), ("g_sum", _vp), ("g_min", _vp), ("g_max", _vp), ("g_hist", _vp)])
+_CollResult = _ptr_struct("_CollResult", [
+    ("n_groups", ctypes.c_int64), ("n_ranks", ctypes.c_int64), ("g_window", _vp), ("g_comm", _vp),
+    ("g_seq", _vp), ("g_n_members", _vp), ("g_min_start", _vp), ("g_max_start", _vp),
+    ("g_skew", _vp), ("g_max_end", _vp), ("g_straggler_pid", _vp), ("g_flags", _vp),
+    ("wait_ns", _vp), ("r_window", _vp), ("r_pid", _vp), ("r_n_coll", _vp), ("r_sum_wait", _vp),
+    ("r_max_wait", _vp), ("r_n_straggler", _vp)])
+
+EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
+           "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
+           "ta_version"]
+
+_lib = None
+
+
+class TaError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = status
+        name = STATUS_NAMES[status] if 0 <= status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{where}: {name}")
+
+
+def lib():
+    """Loads libta.so; raises if it has not been built (no fallback exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(
+                f"{_LIB_PATH} is missing: build it with `python -m paper_2609_40247_b200.build` "
+                "(nvcc, sm_100a). The analyzer has no CPU fallback.")
+        L = ctypes.CDLL(_LIB_PATH)
+        L.ta_load_window.restype = ctypes.c_int
+        L.ta_load_window.argtypes = [ctypes.POINTER(_Env), _vp, ctypes.c_int64, ctypes.c_int32, _vp,
+                                     _vp, _vp, ctypes.c_int32, _vp, ctypes.POINTER(_vp)]
+        L.ta_sort_timeline.restype = ctypes.c_int
+        L.ta_sort_timeline.argtypes = [_vp, ctypes.POINTER(_SortResult)]
+        L.ta_correlate_launches.restype = ctypes.c_int
+        L.ta_correlate_launches.argtypes = [_vp, ctypes.POINTER(_JoinResult), _vp]
+        L.ta_attribute_operators.restype = ctypes.c_int
+        L.ta_attribute_operators.argtypes = [_vp, ctypes.POINTER(_AttrResult), _vp]
+        L.ta_stream_gaps.restype = ctypes.c_int
+        L.ta_stream_gaps.argtypes = [_vp, ctypes.c_int64, ctypes.POINTER(_GapResult)]
+        L.ta_aggregate_ops.restype = ctypes.c_int
+        L.ta_aggregate_ops.argtypes = [_vp, ctypes.c_uint32, ctypes.c_int32, ctypes.POINTER(_AggResult)]
+        L.ta_match_collectives.restype = ctypes.c_int
+        L.ta_match_collectives.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(_CollResult)]
+        L.ta_free.restype = None
+        L.ta_free.argtypes = [_vp]
+        L.ta_strerror.restype = ctypes.c_char_p
+        L.ta_strerror.argtypes = [ctypes.c_int]
+        L.ta_version.restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+class _DevView:
+    """Exposes a raw device range to torch through __cuda_array_interface__."""
+
+    def __init__(self, ptr, nbytes, owner):
+        self.owner = owner
+        self.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1",
+                                         "data": (int(ptr), False), "version": 2}
+
+
+class _Result:
+    """Device pointers owned by the window handle, with typed access."""
+    _layout: dict = {}
+
+    def __init__(self, window, raw, extra=None):
+        self._w = window
+        self._raw = raw
+        self.__dict__.update(extra or {})
+
+    def _spec(self, name):
+        dt, count = self._layout[name]
+        cnt = count(self) if callable(count) else count
+        return np.dtype(dt), int(cnt)
+
+    def tensor(self, name):
+        """Zero-copy torch view (uint8 for struct arrays) of a device result; valid while
+        the window is open."""
+        import torch
+        dt, cnt = self._spec(name)
+        ptr = getattr(self._raw, name)
+        nbytes = cnt * dt.itemsize
+        if nbytes == 0 or not ptr:
+            return torch.empty(0, dtype=torch.uint8, device=f"cuda:{self._w.device}")
+        return torch.as_tensor(_DevView(ptr, nbytes, self._w), device=f"cuda:{self._w.device}")
+
+    def numpy(self, name):
+        if name in self.__dict__ and isinstance(self.__dict__[name], np.ndarray):
+            return self.__dict__[name]
+        dt, cnt = self._spec(name)
+        if cnt == 0:
+            out = np.empty(0, dtype=dt)
+        else:
+            import torch
+            with torch.cuda.stream(self._w.torch_stream):
+                out = self.tensor(name).cpu().numpy().view(dt).copy()
+        if name.endswith("_hist"):
+            out = out.reshape(-1, NBINS)
+        return out
+
+
+class SortResult(_Result):
+    _layout = {
+        "perm": ("<i4", lambda r: r.n), "ts_start": ("<i8", lambda r: r.n),
+        "ts_end": ("<i8", lambda r: r.n), "corr_id": ("<i8", lambda r: r.n),
+        "pid": ("<i4", lambda r: r.n), "name_id": ("<i4", lambda r: r.n),
+        "seq": ("<i4", lambda r: r.n), "stream": ("<i2", lambda r: r.n),
+        "kind": ("<i2", lambda r: r.n),
+        "lane_window": ("<i4", lambda r: r.n_lanes), "lane_pid": ("<i4", lambda r: r.n_lanes),
+        "lane_stream": ("<i2", lambda r: r.n_lanes), "lane_domain": ("<i2", lambda r: r.n_lanes),
+        "lane_off": ("<i4", lambda r: r.n_lanes + 1),
+    }
+
+
+class JoinResult(_Result):
+    _layout = {"launch_of": ("<i4", lambda r: r.n), "launch_latency": ("<i8", lambda r: r.n),
+               "queue_delay": ("<i8", lambda r: r.n), "kernels_of_launch": ("<i4", lambda r: r.n)}
+
+
+class AttrResult(_Result):
+    _layout = {"parent": ("<i4", lambda r: r.n), "depth": ("|u1", lambda r: r.n),
+               "op_of": ("<i4", lambda r: r.n), "op_first_start": ("<i8", lambda r: r.n),
+               "op_last_end": ("<i8", lambda r: r.n), "op_kernel_ns": ("<i8", lambda r: r.n),
+               "op_n_kernels": ("<i4", lambda r: r.n)}
+
+
+class GapResult(_Result):
+    _layout = {"gap_before": ("<i8", lambda r: r.n), "lane_gaps": (LANE_GAPS, lambda r: r.n_lanes),
+               "lane_hist": ("<u4", lambda r: r.n_lanes * NBINS),
+               "win_hist": ("<u4", lambda r: r.n_windows * NBINS),
+               "long_gaps": (LONG_GAP, lambda r: r.n_long_gaps)}
+
+
+class AggResult(_Result):
+    _layout = {"g_window": ("<i4", lambda r: r.n_groups), "g_pid": ("<i4", lambda r: r.n_groups),
+               "g_name": ("<i4", lambda r: r.n_groups), "g_count": ("<i8", lambda r: r.n_groups),
+               "g_sum": ("<i8", lambda r: r.n_groups), "g_min": ("<i8", lambda r: r.n_groups),
+               "g_max": ("<i8", lambda r: r.n_groups),
+               "g_hist": ("<u4", lambda r: r.n_groups * NBINS)}
+
+
+class CollResult(_Result):
+    _names = {"c_window": "g_window", "c_comm": "g_comm", "c_seq": "g_seq",
+              "c_n_members": "g_n_members", "c_min_start": "g_min_start",
+              "c_max_start": "g_max_start", "c_skew": "g_skew", "c_max_end": "g_max_end",
+              "c_straggler_pid": "g_straggler_pid", "c_flags": "g_flags"}
+    _layout = {"g_window": ("<i4", lambda r: r.n_groups), "g_comm": ("<i8", lambda r: r.n_groups),
+               "g_seq": ("<i4", lambda r: r.n_groups), "g_n_members": ("<i4", lambda r: r.n_groups),
+               "g_min_start": ("<i8", lambda r: r.n_groups),
+               "g_max_start": ("<i8", lambda r: r.n_groups), "g_skew": ("<i8", lambda r: r.n_groups),
+               "g_max_end": ("<i8", lambda r: r.n_groups),
+               "g_straggler_pid": ("<i4", lambda r: r.n_groups),
+               "g_flags": ("<i4", lambda r: r.n_groups), "wait_ns": ("<i8", lambda r: r.n),
+               "r_window": ("<i4", lambda r: r.n_ranks), "r_pid": ("<i4", lambda r: r.n_ranks),
+               "r_n_coll": ("<i8", lambda r: r.n_ranks), "r_sum_wait": ("<i8", lambda r: r.n_ranks),
+               "r_max_wait": ("<i8", lambda r: r.n_ranks),
+               "r_n_straggler": ("<i8", lambda r: r.n_ranks)}
+
+    def numpy(self, name):
+        return super().numpy(self._names.get(name, name))
+
+    def tensor(self, name):
+        return super().tensor(self._names.get(name, name))
+
+
+class Window:
+    """One analysis handle (ta_window).  `events`: a CUDA tensor holding n 40-byte
+    records (any dtype, contiguous) - borrowed until sort_timeline() returns - or a
+    host numpy array of EVENT_DTYPE (copied to the device by the library)."""
+
+    def __init__(self, events, win_off, win_t0, win_t1, device=None, stream=None,
+                 use_torch_allocator=True):
+        import torch
+        L = lib()
+        self._lib = L
+        self._h = _vp()
+        on_device = hasattr(events, "is_cuda")
+        if on_device:
+            if not events.is_cuda or not events.is_contiguous():
+                raise ValueError("events tensor must be a contiguous CUDA tensor")
+            nbytes = events.numel() * events.element_size()
+            ev_ptr = events.data_ptr()
+            device = events.device.index if device is None else device
+        else:
+            events = np.ascontiguousarray(events)
+            nbytes = events.nbytes
+            ev_ptr = events.ctypes.data
+            device = torch.cuda.current_device() if device is None else device
+        if nbytes % 40:
+            raise ValueError("events must hold whole 40-byte records")
+        self.n = nbytes // 40
+        self.device = int(device)
+        self._events = events  # keep the borrowed buffer alive
+        self.torch_stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+        self._off = np.ascontiguousarray(win_off, dtype=np.int64)
+        self._t0 = np.ascontiguousarray(win_t0, dtype=np.int64)
+        self._t1 = np.ascontiguousarray(win_t1, dtype=np.int64)
+        self.W = len(self._t0)
+        if len(self._off) != self.W + 1 or len(self._t1) != self.W:
+            raise ValueError("win_off needs W+1 entries, win_t0 / win_t1 W entries")
+        dev, sptr = self.device, self.torch_stream.cuda_stream
+
+        def _alloc(size, ctx):
+            try:
+                return torch.cuda.caching_allocator_alloc(int(size), dev, sptr)
+            except Exception:
+                return None
+
+        def _release(ptr, ctx):
+            torch.cuda.caching_allocator_delete(ptr)
+
+        self._alloc_cb = _ALLOC_T(_alloc)
+        self._release_cb = _RELEASE_T(_release)
+        env = _Env()
+        if use_torch_allocator:
+            env.alloc, env.release = self._alloc_cb, self._release_cb
+        env.ctx = None
+        env.cuda_stream = sptr
+        env.device = dev
+        self._env = env
+        self.load_summary = np.zeros(self.W, dtype=LOAD_SUM)
+        st = L.ta_load_window(ctypes.byref(env), ev_ptr, self.n, 1 if on_device else 0,
+                              self._off.ctypes.data, self._t0.ctypes.data, self._t1.ctypes.data,
+                              self.W, self.load_summary.ctypes.data, ctypes.byref(self._h))
+        if st != 0:
+            self.close()
+            raise TaError(st, "ta_load_window")
+        self._sorted = None
+
+    # -- context manager / lifetime
+    def close(self):
+        if self._h:
+            self._lib.ta_free(self._h)
+            self._h = _vp()
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _dims(self):
+        s = self._sorted
+        return {"n": self.n, "n_lanes": s.n_lanes if s else 0, "n_windows": self.W}
+
+    # -- the seven calls
+    def sort_timeline(self) -> SortResult:
+        raw = _SortResult()
+        st = self._lib.ta_sort_timeline(self._h, ctypes.byref(raw))
+        if st != 0:
+            raise TaError(st, "ta_sort_timeline")
+        self._sorted = SortResult(self, raw, {"n": raw.n, "n_valid": raw.n_valid,
+                                              "n_lanes": raw.n_lanes, "n_windows": raw.n_windows})
+        self._events = None  # the borrow ends here
+        return self._sorted
+
+    def correlate_launches(self) -> JoinResult:
+        raw = _JoinResult()
+        summ = np.zeros(self.W, dtype=JOIN_SUM)
+        st = self._lib.ta_correlate_launches(self._h, ctypes.byref(raw), summ.ctypes.data)
+        if st != 0:
+            raise TaError(st, "ta_correlate_launches")
+        return JoinResult(self, raw, dict(self._dims(), join_sum=summ))
+
+    def attribute_operators(self, check=True) -> AttrResult:
+        """check=False returns the result even for TA_ERR_DEPTH / TA_ERR_BAD_NESTING
+        (see .status); the summaries are valid, the other outputs unspecified."""
+        raw = _AttrResult()
+        summ = np.zeros(self.W, dtype=ATTR_SUM)
+        st = self._lib.ta_attribute_operators(self._h, ctypes.byref(raw), summ.ctypes.data)
+        if st != 0 and (check or st not in (TA_ERR_DEPTH, TA_ERR_BAD_NESTING)):
+            raise TaError(st, "ta_attribute_operators")
+        return AttrResult(self, raw, dict(self._dims(), attr_sum=summ, status=st))
+
+    def stream_gaps(self, min_gap_ns: int) -> GapResult:
+        raw = _GapResult()
+        st = self._lib.ta_stream_gaps(self._h, int(min_gap_ns), ctypes.byref(raw))
+        if st != 0:
+            raise TaError(st, "ta_stream_gaps")
+        return GapResult(self, raw, dict(self._dims(), n_long_gaps=raw.n_long_gaps))
+
+    def aggregate_ops(self, kind_mask: int, value_sel: int) -> AggResult:
+        raw = _AggResult()
+        st = self._lib.ta_aggregate_ops(self._h, kind_mask, value_sel, ctypes.byref(raw))
+        if st != 0:
+            raise TaError(st, "ta_aggregate_ops")
+        return AggResult(self, raw, dict(self._dims(), n_groups=raw.n_groups))
+
+    def match_collectives(self, comm_sizes=()) -> CollResult:
+        arr = np.zeros(len(comm_sizes), dtype=COMM_SIZE)
+        for i, (cid, nr) in enumerate(comm_sizes):
+            arr[i] = (cid, nr, 0)
+        raw = _CollResult()
+        st = self._lib.ta_match_collectives(self._h, arr.ctypes.data if len(arr) else None, len(arr),
+                                            ctypes.byref(raw))
+        if st != 0:
+            raise TaError(st, "ta_match_collectives")
+        return CollResult(self, raw, dict(self._dims(), n_groups=raw.n_groups, n_ranks=raw.n_ranks))
