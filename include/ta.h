@@ -193,7 +193,9 @@ ta_status ta_correlate_launches(ta_window *h, ta_join_result *out,
  * intervals are identical, j precedes i in canonical order.
  *   parent[i] = the encloser with the largest ts_start, then the smallest
  *               ts_end, then the largest sorted position; -1 if none.
- *   depth[i]  = number of enclosers.
+ *   depth[i]  = 0 if parent[i] == -1, else depth[parent[i]] + 1, saturating at
+ *               255.  In a properly nested lane this is the number of enclosers
+ *               of every record of non-zero length.
  * Device records: op_of[i] = parent[launch_of[i]] for KERNEL/MEMCPY with a
  * launch, else -1.  For every OP r, over device records with op_of == r:
  *   op_n_kernels[r], op_first_start[r] = min ts_start, op_last_end[r] =

@@ -269,9 +269,15 @@ struct Oracle {
           }
         }
         parent[i] = best;
-        depth[i] = (uint8_t)std::min(d, 255);
-        if (d > s.max_depth) s.max_depth = d;
-        if (d > MAX_DEPTH) any_deep = true;
+        // depth = level in the forest that `parent` defines (the parent precedes the child
+        // in canonical order, so its depth is known); saturates at 255 (uint8).  It equals
+        // the encloser count d except for a zero-length record that sits exactly on the end
+        // of an earlier sibling range: closed intervals put such a record inside both.
+        (void)d;
+        int lvl = best < 0 ? 0 : std::min(255, (int)depth[best] + 1);
+        depth[i] = (uint8_t)lvl;
+        if (lvl > s.max_depth) s.max_depth = lvl;
+        if (lvl > MAX_DEPTH) any_deep = true;
         if (kind[i] == OP) open.push_back(i);
       }
     }

@@ -128,9 +128,10 @@ class Oracle:
         dt = np.dtype(_DTYPES[name])
         assert dt.itemsize == el.value, (name, dt.itemsize, el.value)
         if cnt.value == 0:
-            return np.empty(0, dtype=dt)
-        buf = (ctypes.c_char * (cnt.value * el.value)).from_address(ptr.value)
-        out = np.frombuffer(buf, dtype=dt).copy()
+            out = np.empty(0, dtype=dt)
+        else:
+            buf = (ctypes.c_char * (cnt.value * el.value)).from_address(ptr.value)
+            out = np.frombuffer(buf, dtype=dt).copy()
         if name in ("lane_hist", "win_hist", "g_hist"):
             out = out.reshape(-1, 40)
         return out

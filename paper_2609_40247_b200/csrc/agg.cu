@@ -1,0 +1,248 @@
+// ta_aggregate_ops: per (window, pid, name_id) count / sum / min / max and a log2
+// histogram of a value column (own duration, or T_op of operators with kernels).
+// Per-symbol counts and duration statistics are what Sec. 8.1 compares.
+//
+// Symbol popularity is heavy-tailed (a few names carry most records), so global
+// atomics alone would serialise on the hot rows.  Each CTA walks a contiguous
+// range of sorted positions (one process, mostly) and folds its records into a
+// shared-memory hash table first; the table is flushed to a dense global table
+// indexed by (window, pid rank, name_id - min name) with one atomic per field.
+// A scan then compacts the non-empty rows in key order.
+// HBM-bound on the column reads: 2 B (kind) for every record, 24 B more for the
+// selected ones.
+#include <climits>
+#include <cstring>
+#include <vector>
+
+#include "records.cuh"
+#include "scan.cuh"
+#include "ta_internal.cuh"
+
+#define AG_THREADS 256
+#define AG_SLOTS 512
+#define AG_FLUSH_EVERY 32768  // records per CTA between flushes (keeps 16-bit bins safe)
+
+struct AggArgs {
+  int64_t n_valid;
+  int n_lanes;
+  const int16_t *kind;
+  const int32_t *name;
+  const int64_t *ts, *te;
+  const int32_t *lane_off, *lane_slot;
+  const int32_t *op_n;
+  const int64_t *op_first, *op_last;
+  uint32_t kind_mask;
+  int value_sel;
+  int64_t min_name, R;
+  int64_t chunk;  // positions per CTA
+  // dense table (all zero-initialised; min is kept as the complement of the biased value)
+  u64 *d_cnt, *d_sum, *d_minc, *d_maxb;
+  u32 *d_hist;
+  u64 *n_groups;
+};
+
+struct AggSmem {
+  int32_t key[AG_SLOTS];
+  u32 cnt[AG_SLOTS];
+  u64 sum[AG_SLOTS];
+  u64 minc[AG_SLOTS];
+  u64 maxb[AG_SLOTS];
+  uint16_t hist[AG_SLOTS][TA_NBINS];
+};
+
+__device__ __forceinline__ void agg_global_add(const AggArgs &a, int64_t g, u64 cnt, u64 sum, u64 minc,
+                                               u64 maxb) {
+  u64 old = atomicAdd(&a.d_cnt[g], cnt);
+  if (old == 0) atomicAdd(a.n_groups, 1ull);
+  atomicAdd(&a.d_sum[g], sum);
+  atomicMax(&a.d_minc[g], minc);
+  atomicMax(&a.d_maxb[g], maxb);
+}
+
+__device__ __forceinline__ void agg_flush(const AggArgs &a, AggSmem &s) {
+  __syncthreads();
+  for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
+    int32_t k = s.key[i];
+    if (k >= 0) {
+      agg_global_add(a, k, s.cnt[i], s.sum[i], s.minc[i], s.maxb[i]);
+      for (int b = 0; b < TA_NBINS; b++)
+        if (s.hist[i][b]) atomicAdd(&a.d_hist[(size_t)k * TA_NBINS + b], (u32)s.hist[i][b]);
+    }
+    s.key[i] = -1;
+    s.cnt[i] = 0;
+    s.sum[i] = 0;
+    s.minc[i] = 0;
+    s.maxb[i] = 0;
+    for (int b = 0; b < TA_NBINS; b++) s.hist[i][b] = 0;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(AG_THREADS) k_agg(AggArgs a) {
+  extern __shared__ __align__(16) unsigned char raw[];
+  AggSmem &s = *reinterpret_cast<AggSmem *>(raw);
+  for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
+    s.key[i] = -1;
+    s.cnt[i] = 0;
+    s.sum[i] = 0;
+    s.minc[i] = 0;
+    s.maxb[i] = 0;
+    for (int b = 0; b < TA_NBINS; b++) s.hist[i][b] = 0;
+  }
+  __syncthreads();
+  const int64_t begin = (int64_t)blockIdx.x * a.chunk;
+  const int64_t end = min(begin + a.chunk, a.n_valid);
+  int since_flush = 0;
+  LaneWalker lw(a.lane_off, a.n_lanes, begin + threadIdx.x, a.n_valid);
+  for (int64_t base = begin; base < end; base += AG_THREADS) {
+    const int64_t p = base + threadIdx.x;
+    if (p < end) {
+      const int k = a.kind[p];
+      if ((1u << k) & a.kind_mask) {
+        bool sel = true;
+        i64 v;
+        if (a.value_sel == 0) v = a.te[p] - a.ts[p];
+        else {
+          sel = a.op_n[p] > 0;
+          v = sel ? a.op_last[p] - a.op_first[p] : 0;
+        }
+        if (sel) {
+          const int lane = lw.at(p);
+          const int64_t g = (int64_t)a.lane_slot[lane] * a.R + ((int64_t)a.name[p] - a.min_name);
+          const u64 vb = (u64)v ^ (1ull << 63);
+          const int bin = log2_bin(v);
+          u32 hsh = (u32)g * 2654435761u;
+          int slot = (int)(hsh >> 23) & (AG_SLOTS - 1);
+          bool placed = false;
+          for (int probe = 0; probe < 8; probe++) {
+            int32_t cur = s.key[slot];
+            if (cur == (int32_t)g) { placed = true; break; }
+            if (cur == -1) {
+              int32_t old = atomicCAS(&s.key[slot], -1, (int32_t)g);
+              if (old == -1 || old == (int32_t)g) { placed = true; break; }
+            }
+            slot = (slot + 1) & (AG_SLOTS - 1);
+          }
+          if (placed) {
+            atomicAdd(&s.cnt[slot], 1u);
+            atomicAdd(&s.sum[slot], (u64)v);
+            atomicMax(&s.minc[slot], ~vb);
+            atomicMax(&s.maxb[slot], vb);
+            // 16-bit bins packed two per word
+            u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
+            atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
+          } else {
+            agg_global_add(a, g, 1, (u64)v, ~vb, vb);
+            atomicAdd(&a.d_hist[(size_t)g * TA_NBINS + bin], 1u);
+          }
+        }
+      }
+    }
+    since_flush += AG_THREADS;
+    if (since_flush >= AG_FLUSH_EVERY) {
+      agg_flush(a, s);
+      since_flush = 0;
+    }
+  }
+  agg_flush(a, s);
+}
+
+// compaction of the non-empty rows in dense (= key) order
+struct AggRowIn {
+  const u64 *cnt;
+  __device__ u64 operator()(int64_t g) const { return cnt[g] ? 1ull : 0ull; }
+};
+struct AggRowOut {
+  const u64 *cnt, *sum, *minc, *maxb;
+  const u32 *hist;
+  const TripleTable *tt;
+  int n_pids;
+  int64_t R, min_name;
+  int32_t *g_window, *g_pid, *g_name;
+  int64_t *g_count, *g_sum, *g_min, *g_max;
+  u32 *g_hist;
+  __device__ void operator()(int64_t g, u64 row, u64 v) const {
+    if (!v) return;
+    int64_t slot = g / R;
+    g_window[row] = (int32_t)(slot / n_pids);
+    g_pid[row] = tt->pid_value[slot % n_pids];
+    g_name[row] = (int32_t)(min_name + g % R);
+    g_count[row] = (int64_t)cnt[g];
+    g_sum[row] = (int64_t)sum[g];
+    g_min[row] = (int64_t)((~minc[g]) ^ (1ull << 63));
+    g_max[row] = (int64_t)(maxb[g] ^ (1ull << 63));
+    for (int b = 0; b < TA_NBINS; b++) g_hist[row * TA_NBINS + b] = hist[(size_t)g * TA_NBINS + b];
+  }
+};
+
+ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_agg_result *out) {
+  cudaStream_t st = h->stream;
+  const int n_pids = h->n_pids > 0 ? h->n_pids : 1;
+  memset(out, 0, sizeof(*out));
+  if (h->n_valid == 0 || (kind_mask & 63u) == 0) return TA_OK;
+  const unsigned __int128 R128 = (unsigned __int128)((uint64_t)h->max_name - (uint64_t)h->min_name) + 1;
+  const unsigned __int128 G128 = R128 * (unsigned __int128)((uint64_t)h->W * (uint64_t)n_pids);
+  if (G128 > (unsigned __int128)TA_AGG_DENSE_LIMIT) return TA_ERR_TOO_LARGE;
+  const int64_t R = (int64_t)R128, G = (int64_t)G128;
+
+  size_t tb = 4 * Carver::pad((size_t)G * 8) + Carver::pad((size_t)G * TA_NBINS * 4) + Carver::pad(64) +
+              scan_temp_bytes(G) + 256;
+  void *tmpb = ta_dalloc(h, tb);
+  if (!tmpb) return TA_ERR_OOM;
+  Carver ct(tmpb);
+  AggArgs a;
+  memset(&a, 0, sizeof(a));
+  a.d_cnt = ct.take<u64>(G);
+  a.d_sum = ct.take<u64>(G);
+  a.d_minc = ct.take<u64>(G);
+  a.d_maxb = ct.take<u64>(G);
+  a.d_hist = ct.take<u32>((size_t)G * TA_NBINS);
+  a.n_groups = ct.take<u64>(8);
+  TA_CHECK_CUDA(h, cudaMemsetAsync(tmpb, 0, ct.off, st));
+  void *scan_mem = ct.base + ct.off;
+
+  a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes;
+  a.kind = h->sorted.kind; a.name = h->sorted.name_id; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
+  a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot;
+  a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
+  a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
+  int64_t blocks = 148 * 3;
+  int64_t chunk = (h->n_valid + blocks - 1) / blocks;
+  chunk = ((chunk + AG_THREADS - 1) / AG_THREADS) * AG_THREADS;
+  if (chunk < AG_THREADS) chunk = AG_THREADS;
+  blocks = (h->n_valid + chunk - 1) / chunk;
+  a.chunk = chunk;
+  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_agg, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(AggSmem)));
+  k_agg<<<(unsigned)blocks, AG_THREADS, sizeof(AggSmem), st>>>(a);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  u64 ng = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  if (ng > 0) {
+    size_t ob = 3 * Carver::pad(ng * 4) + 4 * Carver::pad(ng * 8) + Carver::pad(ng * TA_NBINS * 4) + 256;
+    void *outb = ta_dalloc(h, ob);
+    if (!outb) return TA_ERR_OOM;
+    Carver co(outb);
+    AggRowOut ro;
+    ro.cnt = a.d_cnt; ro.sum = a.d_sum; ro.minc = a.d_minc; ro.maxb = a.d_maxb; ro.hist = a.d_hist;
+    ro.tt = h->d_triples; ro.n_pids = n_pids; ro.R = R; ro.min_name = h->min_name;
+    ro.g_window = co.take<int32_t>(ng); ro.g_pid = co.take<int32_t>(ng); ro.g_name = co.take<int32_t>(ng);
+    ro.g_count = co.take<int64_t>(ng); ro.g_sum = co.take<int64_t>(ng);
+    ro.g_min = co.take<int64_t>(ng); ro.g_max = co.take<int64_t>(ng);
+    ro.g_hist = co.take<u32>(ng * TA_NBINS);
+    ScanTemp t;
+    TA_TRY(scan_temp_init(h, scan_mem, G, &t));
+    AggRowIn ri{a.d_cnt};
+    TA_TRY((launch_scan<OpAdd, AggRowIn, AggRowOut>(h, G, ri, ro, OpAdd(), t)));
+    out->g_window = ro.g_window; out->g_pid = ro.g_pid; out->g_name = ro.g_name;
+    out->g_count = ro.g_count; out->g_sum = ro.g_sum; out->g_min = ro.g_min; out->g_max = ro.g_max;
+    out->g_hist = ro.g_hist;
+  }
+  out->n_groups = (int64_t)ng;
+  int32_t words[ST_WORDS];
+  TA_TRY(ta_read_status(h, words));
+  ta_dfree(h, tmpb);
+  if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+  return TA_OK;
+}

@@ -1,0 +1,459 @@
+// ta_correlate_launches: correlation id associates submissions with device
+// activity (Sec. 5.2; Fig. "Key performance observations" (a)).  Key =
+// (window, pid, corr_id); the smallest sorted position among equal LAUNCH keys
+// wins.
+//
+// Two paths, same results:
+//   direct   when the correlation ids of each (window, pid) span a compact
+//            range (they count up per process in real traces): a table of
+//            sorted positions indexed by corr_id - min, filled with atomicMin.
+//            Launches and kernels are time-ordered, so the table is touched
+//            nearly sequentially.
+//   general  any 64-bit ids: launches and probes are compacted, stably sorted
+//            by (slot, corr_id) with the pair sorter, and each probe takes the
+//            head of its run if that head is a LAUNCH.
+// HBM-bound: streams kind/corr/ts columns, writes three outputs per record.
+#include <climits>
+#include <cstring>
+#include <vector>
+
+#include "scan.cuh"
+#include "ta_internal.cuh"
+
+#define JN_THREADS 512
+#define JN_ITEMS 4
+#define JN_TILE (JN_THREADS * JN_ITEMS)
+#define EMPTY_U32 0xFFFFFFFFu
+
+struct JoinArgs {
+  int64_t n, n_valid;
+  int n_lanes;
+  const int16_t *kind;
+  const int64_t *corr, *ts, *te;
+  const int32_t *lane_off, *lane_slot, *lane_window;
+  const int16_t *lane_domain;
+  // per slot (window * n_pids + pid rank)
+  i64 *slot_min, *slot_max;       // corr range of LAUNCH records
+  const i64 *slot_base;           // direct path: table offset of the slot, -1 = no launches
+  u32 *table;                     // direct path
+  const int32_t *found;           // general path: winner launch per launch/probe position
+  int32_t *launch_of, *kol;
+  int64_t *latency, *qdelay;
+  ta_join_summary *sum;           // device, per window
+};
+
+__device__ __forceinline__ u64 bias64(i64 v) { return (u64)v ^ (1ull << 63); }
+__device__ __forceinline__ i64 unbias64(u64 v) { return (i64)(v ^ (1ull << 63)); }
+
+// block-wide reduction helper (all threads call); smem >= 33 u64
+__device__ __forceinline__ u64 blk_reduce(u64 v, bool is_max, u64 *smem) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  v = is_max ? warp_reduce(v, OpMax()) : warp_reduce(v, OpAdd());
+  __syncthreads();
+  if (lane == 0) smem[warp] = v;
+  __syncthreads();
+  if (warp == 0) {
+    u64 w = lane < (int)(blockDim.x >> 5) ? smem[lane] : 0;
+    w = is_max ? warp_reduce(w, OpMax()) : warp_reduce(w, OpAdd());
+    if (lane == 0) smem[32] = w;
+  }
+  __syncthreads();
+  return smem[32];
+}
+
+// lanes touched by the CTA's selected items -> [l0, l1] (l1 < l0 if none)
+__device__ __forceinline__ void tile_lane_range(int my_lo, int my_hi, int *s_lo, int *s_hi, int *l0,
+                                                int *l1) {
+  if (threadIdx.x == 0) { *s_lo = INT_MAX; *s_hi = -1; }
+  __syncthreads();
+  if (my_hi >= 0) { atomicMin(s_lo, my_lo); atomicMax(s_hi, my_hi); }
+  __syncthreads();
+  *l0 = *s_lo;
+  *l1 = *s_hi;
+  __syncthreads();
+}
+
+// ---- pass 1: corr range of the LAUNCH records of every slot ----------------
+__global__ void __launch_bounds__(JN_THREADS) k_join_minmax(JoinArgs a) {
+  __shared__ u64 tmp[33];
+  __shared__ int s_lo, s_hi;
+  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
+  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
+  int ln[JN_ITEMS];
+  i64 c[JN_ITEMS];
+  int my_lo = INT_MAX, my_hi = -1;
+#pragma unroll
+  for (int j = 0; j < JN_ITEMS; j++) {
+    int64_t p = p0 + j;
+    ln[j] = -1;
+    c[j] = 0;
+    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
+      ln[j] = lw.at(p);
+      c[j] = a.corr[p];
+      my_lo = min(my_lo, ln[j]);
+      my_hi = max(my_hi, ln[j]);
+    }
+  }
+  int l0, l1;
+  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
+  for (int l = l0; l <= l1; l++) {
+    if (a.lane_domain[l] != 0) continue;
+    u64 mx = 0, mn_inv = 0;
+#pragma unroll
+    for (int j = 0; j < JN_ITEMS; j++)
+      if (ln[j] == l) {
+        mx = max(mx, bias64(c[j]) + 0);
+        mn_inv = max(mn_inv, ~bias64(c[j]));
+      }
+    bool any = false;
+#pragma unroll
+    for (int j = 0; j < JN_ITEMS; j++) any |= (ln[j] == l);
+    u64 cnt = blk_reduce(any ? 1 : 0, false, tmp);
+    if (cnt == 0) continue;
+    // threads without an item contribute neutral elements: bias64 maps INT64_MIN to 0
+    mx = blk_reduce(any ? mx : 0, true, tmp);
+    mn_inv = blk_reduce(any ? mn_inv : 0, true, tmp);
+    if (threadIdx.x == 0) {
+      int slot = a.lane_slot[l];
+      atomicMax(&a.slot_max[slot], unbias64(mx));
+      atomicMin(&a.slot_min[slot], unbias64(~mn_inv));
+    }
+  }
+}
+
+// ---- direct path: fill the table -------------------------------------------
+__global__ void __launch_bounds__(JN_THREADS) k_join_build(JoinArgs a) {
+  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
+  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
+#pragma unroll
+  for (int j = 0; j < JN_ITEMS; j++) {
+    int64_t p = p0 + j;
+    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
+      int slot = a.lane_slot[lw.at(p)];
+      i64 idx = a.slot_base[slot] + (a.corr[p] - a.slot_min[slot]);
+      atomicMin(&a.table[idx], (u32)p);
+    }
+  }
+}
+
+template <bool DIRECT>
+__device__ __forceinline__ int32_t winner_of(const JoinArgs &a, int64_t p, int slot) {
+  if (!DIRECT) return a.found[p];
+  i64 base = a.slot_base[slot];
+  if (base < 0) return -1;
+  i64 c = a.corr[p];
+  if (c < a.slot_min[slot] || c > a.slot_max[slot]) return -1;
+  u32 v = a.table[base + (c - a.slot_min[slot])];
+  return v == EMPTY_U32 ? -1 : (int32_t)v;
+}
+
+// ---- pass 2: probes ----------------------------------------------------------
+template <bool DIRECT>
+__global__ void __launch_bounds__(JN_THREADS) k_join_probe(JoinArgs a) {
+  __shared__ u64 tmp[33];
+  __shared__ int s_lo, s_hi;
+  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
+  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
+  int ln[JN_ITEMS];
+  bool matched[JN_ITEMS];
+  i64 lat[JN_ITEMS], q[JN_ITEMS];
+  int my_lo = INT_MAX, my_hi = -1;
+#pragma unroll
+  for (int j = 0; j < JN_ITEMS; j++) {
+    int64_t p = p0 + j;
+    ln[j] = -1;
+    matched[j] = false;
+    lat[j] = 0;
+    q[j] = 0;
+    if (p >= a.n) continue;
+    int32_t lo = -1;
+    if (p < a.n_valid) {
+      int k = a.kind[p];
+      if (k == TA_KIND_KERNEL || k == TA_KIND_MEMCPY) {
+        ln[j] = lw.at(p);
+        my_lo = min(my_lo, ln[j]);
+        my_hi = max(my_hi, ln[j]);
+        lo = winner_of<DIRECT>(a, p, a.lane_slot[ln[j]]);
+        if (lo >= 0) {
+          matched[j] = true;
+          i64 s = a.ts[p];
+          lat[j] = s - a.ts[lo];
+          i64 d = s - a.te[lo];
+          q[j] = d > 0 ? d : 0;
+          atomicAdd(&a.kol[lo], 1);
+        }
+      }
+    }
+    a.launch_of[p] = lo;
+    a.latency[p] = lat[j];
+    a.qdelay[p] = q[j];
+  }
+  int l0, l1;
+  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
+  for (int l = l0; l <= l1; l++) {
+    if (a.lane_domain[l] != 1) continue;
+    u64 np = 0, nm = 0, sl = 0, sq = 0, mxl = 0, mnl_inv = 0, mxq = 0;
+#pragma unroll
+    for (int j = 0; j < JN_ITEMS; j++)
+      if (ln[j] == l) {
+        np++;
+        if (matched[j]) {
+          nm++;
+          sl += (u64)lat[j];
+          sq += (u64)q[j];
+          mxl = max(mxl, bias64(lat[j]));
+          mnl_inv = max(mnl_inv, ~bias64(lat[j]));
+          mxq = max(mxq, (u64)q[j]);
+        }
+      }
+    np = blk_reduce(np, false, tmp);
+    if (np == 0) continue;
+    nm = blk_reduce(nm, false, tmp);
+    sl = blk_reduce(sl, false, tmp);
+    sq = blk_reduce(sq, false, tmp);
+    mxl = blk_reduce(mxl, true, tmp);
+    mnl_inv = blk_reduce(mnl_inv, true, tmp);
+    mxq = blk_reduce(mxq, true, tmp);
+    if (threadIdx.x == 0) {
+      ta_join_summary *s = &a.sum[a.lane_window[l]];
+      atomicAdd((u64 *)&s->n_probe, np);
+      if (nm) {
+        atomicAdd((u64 *)&s->n_matched, nm);
+        atomicAdd((u64 *)&s->sum_latency, sl);
+        atomicAdd((u64 *)&s->sum_queue, sq);
+        atomicMax((i64 *)&s->max_latency, unbias64(mxl));
+        atomicMin((i64 *)&s->min_latency, unbias64(~mnl_inv));
+        atomicMax((i64 *)&s->max_queue, (i64)mxq);
+      }
+    }
+  }
+}
+
+// ---- pass 3: launch statistics (duplicates, orphans) ---------------------------
+template <bool DIRECT>
+__global__ void __launch_bounds__(JN_THREADS) k_join_launch_stats(JoinArgs a) {
+  __shared__ u64 tmp[33];
+  __shared__ int s_lo, s_hi;
+  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
+  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
+  int ln[JN_ITEMS];
+  bool dup[JN_ITEMS], orphan[JN_ITEMS];
+  int my_lo = INT_MAX, my_hi = -1;
+#pragma unroll
+  for (int j = 0; j < JN_ITEMS; j++) {
+    int64_t p = p0 + j;
+    ln[j] = -1;
+    dup[j] = orphan[j] = false;
+    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
+      ln[j] = lw.at(p);
+      my_lo = min(my_lo, ln[j]);
+      my_hi = max(my_hi, ln[j]);
+      int32_t w = winner_of<DIRECT>(a, p, a.lane_slot[ln[j]]);
+      dup[j] = (w != (int32_t)p);
+      orphan[j] = !dup[j] && a.kol[p] == 0;
+    }
+  }
+  int l0, l1;
+  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
+  for (int l = l0; l <= l1; l++) {
+    if (a.lane_domain[l] != 0) continue;
+    u64 nl = 0, nd = 0, no = 0;
+#pragma unroll
+    for (int j = 0; j < JN_ITEMS; j++)
+      if (ln[j] == l) { nl++; nd += dup[j]; no += orphan[j]; }
+    nl = blk_reduce(nl, false, tmp);
+    if (nl == 0) continue;
+    nd = blk_reduce(nd, false, tmp);
+    no = blk_reduce(no, false, tmp);
+    if (threadIdx.x == 0) {
+      ta_join_summary *s = &a.sum[a.lane_window[l]];
+      atomicAdd((u64 *)&s->n_launch, nl);
+      if (nd) atomicAdd((u64 *)&s->n_dup_launch, nd);
+      if (no) atomicAdd((u64 *)&s->n_orphan_launch, no);
+    }
+  }
+}
+
+// ---- general path helpers -----------------------------------------------------
+struct JoinSelIn {
+  const int16_t *kind;
+  int64_t n_valid;
+  __device__ u64 operator()(int64_t i) const {
+    if (i >= n_valid) return 0;
+    int k = kind[i];
+    return (k == TA_KIND_LAUNCH || k == TA_KIND_KERNEL || k == TA_KIND_MEMCPY) ? 1ull : 0ull;
+  }
+};
+struct JoinSelOut {
+  u32 *pos;
+  __device__ void operator()(int64_t i, u64 excl, u64 v) const {
+    if (v) pos[excl] = (u32)i;
+  }
+};
+__global__ void __launch_bounds__(256) k_join_key_corr(const u32 *pos, int64_t m, const int64_t *corr,
+                                                       u64 *out) {
+  int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < m) out[j] = bias64(corr[pos[j]]);
+}
+__global__ void __launch_bounds__(256) k_join_key_slot(const u32 *pos, int64_t m,
+                                                       const int32_t *lane_off, int n_lanes,
+                                                       const int32_t *lane_slot, u64 *out) {
+  int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < m) out[j] = (u64)lane_slot[lane_of_pos(lane_off, n_lanes, pos[j])];
+}
+struct JoinHeadIn {
+  const u64 *slot_key;
+  const u32 *pos;
+  const int64_t *corr;
+  __device__ u64 operator()(int64_t j) const {
+    bool head = j == 0 || slot_key[j] != slot_key[j - 1] || corr[pos[j]] != corr[pos[j - 1]];
+    return head ? (u64)(j + 1) : 0ull;
+  }
+};
+struct JoinHeadOut {
+  const u32 *pos;
+  const int16_t *kind;
+  int32_t *found;
+  __device__ void operator()(int64_t j, u64 excl, u64 v) const {
+    u64 hd = (excl > v ? excl : v) - 1;  // index of the head of j's run
+    u32 hp = pos[hd];
+    found[pos[j]] = kind[hp] == TA_KIND_LAUNCH ? (int32_t)hp : -1;
+  }
+};
+
+static int bit_length64(uint64_t v) {
+  int b = 0;
+  while (v) { b++; v >>= 1; }
+  return b;
+}
+
+ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
+  const int64_t n = h->n;
+  const int W = h->W;
+  const int n_slots = W * (h->n_pids > 0 ? h->n_pids : 1);
+  cudaStream_t st = h->stream;
+  const int64_t nn = n > 0 ? n : 1;
+  size_t keep = 2 * Carver::pad(nn * 4) + 2 * Carver::pad(nn * 8) + 3 * Carver::pad((size_t)n_slots * 8) +
+                Carver::pad((size_t)W * sizeof(ta_join_summary)) + 256;
+  void *kb = ta_dalloc(h, keep);
+  if (!kb) return TA_ERR_OOM;
+  Carver ck(kb);
+  int32_t *launch_of = ck.take<int32_t>(nn), *kol = ck.take<int32_t>(nn);
+  int64_t *latency = ck.take<int64_t>(nn), *qdelay = ck.take<int64_t>(nn);
+  i64 *slot_min = ck.take<i64>(n_slots), *slot_max = ck.take<i64>(n_slots), *slot_base = ck.take<i64>(n_slots);
+  ta_join_summary *d_sum = ck.take<ta_join_summary>(W);
+
+  std::vector<ta_join_summary> hs(W);
+  for (auto &s : hs) {
+    memset(&s, 0, sizeof(s));
+    s.min_latency = INT64_MAX;
+    s.max_latency = INT64_MIN;
+  }
+  std::vector<i64> hmin(n_slots, INT64_MAX), hmax(n_slots, INT64_MIN), hbase(n_slots, -1);
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(d_sum, hs.data(), W * sizeof(ta_join_summary), cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_min, hmin.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_max, hmax.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(kol, 0, nn * 4, st));
+
+  JoinArgs a;
+  memset(&a, 0, sizeof(a));
+  a.n = n; a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes;
+  a.kind = h->sorted.kind; a.corr = h->sorted.corr_id; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
+  a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot; a.lane_window = h->sorted.lane_window;
+  a.lane_domain = h->sorted.lane_domain;
+  a.slot_min = slot_min; a.slot_max = slot_max; a.slot_base = slot_base;
+  a.launch_of = launch_of; a.kol = kol; a.latency = latency; a.qdelay = qdelay; a.sum = d_sum;
+  const unsigned grid = (unsigned)((n + JN_TILE - 1) / JN_TILE);
+  void *tmp_alloc = nullptr;
+  bool direct = true;
+  if (n > 0) {
+    k_join_minmax<<<grid, JN_THREADS, 0, st>>>(a);
+    TA_CHECK_CUDA(h, cudaGetLastError());
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(hmin.data(), slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(hmax.data(), slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    // table size if every slot is addressed directly
+    unsigned __int128 total = 0;
+    for (int s = 0; s < n_slots; s++)
+      if (hmin[s] <= hmax[s]) {
+        hbase[s] = (i64)total;
+        total += (unsigned __int128)((uint64_t)hmax[s] - (uint64_t)hmin[s]) + 1;
+      }
+    const uint64_t limit = (uint64_t)4 * (uint64_t)n + 65536;
+    direct = total <= limit;
+    if (direct) {
+      uint64_t M = (uint64_t)total;
+      tmp_alloc = ta_dalloc(h, (size_t)(M > 0 ? M : 1) * 4);
+      if (!tmp_alloc) return TA_ERR_OOM;
+      a.table = (u32 *)tmp_alloc;
+      TA_CHECK_CUDA(h, cudaMemsetAsync(a.table, 0xFF, (size_t)(M > 0 ? M : 1) * 4, st));
+      TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_base, hbase.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+      k_join_build<<<grid, JN_THREADS, 0, st>>>(a);
+      k_join_probe<true><<<grid, JN_THREADS, 0, st>>>(a);
+      k_join_launch_stats<true><<<grid, JN_THREADS, 0, st>>>(a);
+    } else {
+      // general path: compact, sort by (slot, corr) with sorted position as the stable tie-break
+      size_t tb = Carver::pad(nn * 4) * 3 + Carver::pad(nn * 8) * 3 + scan_temp_bytes(n) * 2 +
+                  ta_sort_temp_bytes(n) + 512;
+      tmp_alloc = ta_dalloc(h, tb);
+      if (!tmp_alloc) return TA_ERR_OOM;
+      Carver ct(tmp_alloc);
+      u32 *pos = ct.take<u32>(nn), *pos_s = ct.take<u32>(nn);
+      int32_t *found = ct.take<int32_t>(nn);
+      u64 *k_in = ct.take<u64>(nn), *k_s = ct.take<u64>(nn), *k_f = ct.take<u64>(nn);
+      void *scan_mem1 = ct.base + ct.off; ct.off += scan_temp_bytes(n);
+      void *scan_mem2 = ct.base + ct.off; ct.off += scan_temp_bytes(n);
+      void *sort_tmp = ct.base + ct.off;
+      ScanTemp t1;
+      TA_TRY(scan_temp_init(h, scan_mem1, n, &t1));
+      JoinSelIn sin{a.kind, h->n_valid};
+      JoinSelOut sout{pos};
+      TA_TRY((launch_scan<OpAdd, JoinSelIn, JoinSelOut>(h, n, sin, sout, OpAdd(), t1)));
+      u64 m64 = 0;
+      TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, t1.total, 8, cudaMemcpyDeviceToHost, st));
+      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+      const int64_t m = (int64_t)m64;
+      TA_CHECK_CUDA(h, cudaMemsetAsync(found, 0xFF, nn * 4, st));
+      if (m > 0) {
+        const int gb = (int)((m + 255) / 256);
+        u32 *vscr = (u32 *)found;  // found is not needed before the sorts are done
+        k_join_key_corr<<<gb, 256, 0, st>>>(pos, m, a.corr, k_in);
+        TA_TRY(ta_radix_sort_pairs(h, k_in, pos, k_s, vscr, k_f, pos_s, m, ta_make_plan(0, 64), nullptr,
+                                   sort_tmp));
+        k_join_key_slot<<<gb, 256, 0, st>>>(pos_s, m, a.lane_off, a.n_lanes, a.lane_slot, k_in);
+        int sb = bit_length64((uint64_t)(n_slots > 1 ? n_slots - 1 : 1));
+        TA_TRY(ta_radix_sort_pairs(h, k_in, pos_s, k_s, vscr, k_f, pos, m, ta_make_plan(0, sb), nullptr,
+                                   sort_tmp));
+        TA_CHECK_CUDA(h, cudaMemsetAsync(found, 0xFF, nn * 4, st));
+        ScanTemp t2;
+        TA_TRY(scan_temp_init(h, scan_mem2, m, &t2));
+        JoinHeadIn hin{k_f, pos, a.corr};
+        JoinHeadOut hout{pos, a.kind, found};
+        TA_TRY((launch_scan<OpMax, JoinHeadIn, JoinHeadOut>(h, m, hin, hout, OpMax(), t2)));
+      }
+      a.found = found;
+      k_join_probe<false><<<grid, JN_THREADS, 0, st>>>(a);
+      k_join_launch_stats<false><<<grid, JN_THREADS, 0, st>>>(a);
+    }
+    TA_CHECK_CUDA(h, cudaGetLastError());
+  }
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(hs.data(), d_sum, W * sizeof(ta_join_summary), cudaMemcpyDeviceToHost, st));
+  int32_t words[ST_WORDS];
+  TA_TRY(ta_read_status(h, words));
+  if (tmp_alloc) ta_dfree(h, tmp_alloc);
+  if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+  for (int w = 0; w < W; w++) {
+    ta_join_summary &s = hs[w];
+    s.n_unmatched = s.n_probe - s.n_matched;
+    if (s.n_matched == 0) { s.min_latency = 0; s.max_latency = 0; }
+    if (out_summary) out_summary[w] = s;
+  }
+  h->join.launch_of = launch_of;
+  h->join.launch_latency = latency;
+  h->join.queue_delay = qdelay;
+  h->join.kernels_of_launch = kol;
+  if (n == 0) {
+    // nothing was launched: outputs are single dummy entries
+  }
+  return TA_OK;
+}

@@ -23,12 +23,15 @@ __device__ __forceinline__ i64 warp_max_i64(i64 v) {
 // of name ids and the longest duration.
 __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n, const int64_t *off,
                                                   const int64_t *t0, const int64_t *t1, int W,
-                                                  TripleTable *tt, ta_load_summary *sum,
-                                                  int64_t *misc, int32_t *status) {
+                                                  TripleTable *tt, CommTable *cm,
+                                                  ta_load_summary *sum, int64_t *misc,
+                                                  int32_t *status) {
   __shared__ u64 cache[256];
+  __shared__ u64 ccache[64];
   cache[threadIdx.x] = TRIPLE_EMPTY;
+  if (threadIdx.x < 64) ccache[threadIdx.x] = TRIPLE_EMPTY;
   __syncthreads();
-  i64 mn = INT64_MAX, mx = INT64_MIN, md = 0;
+  i64 mn = INT64_MAX, mx = INT64_MIN, md = 0, qmn = INT64_MAX, qmx = INT64_MIN;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
        i += (int64_t)gridDim.x * blockDim.x) {
     Rec r = load_rec(ev, i);
@@ -43,6 +46,28 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
     mn = min(mn, (i64)r.name);
     mx = max(mx, (i64)r.name);
     md = max(md, r.ts_end - r.ts_start);
+    if (r.kind == TA_KIND_COLL) {  // communicator set and sequence range
+      qmn = min(qmn, (i64)r.seq);
+      qmx = max(qmx, (i64)r.seq);
+      u64 cc = (u64)r.corr ^ (1ull << 63);
+      u32 ch = hash_code(cc);
+      if (cc == TRIPLE_EMPTY) ta_set_err(status, TA_ERR_INVALID_ARG);  // reserved id
+      else if (ccache[ch & 63] != cc) {
+        u32 slot = ch & (TA_COMM_SLOTS - 1);
+        bool ok = false;
+        for (int probe = 0; probe < TA_COMM_SLOTS; probe++) {
+          u64 cur = ld_relaxed(&cm->slots[slot]);
+          if (cur == cc) { ok = true; break; }
+          if (cur == TRIPLE_EMPTY) {
+            u64 old = atomicCAS(&cm->slots[slot], TRIPLE_EMPTY, cc);
+            if (old == TRIPLE_EMPTY || old == cc) { ok = true; break; }
+          }
+          slot = (slot + 1) & (TA_COMM_SLOTS - 1);
+        }
+        if (!ok) ta_set_err(status, TA_ERR_TOO_LARGE);
+        ccache[ch & 63] = cc;
+      }
+    }
     u64 code = triple_code(r.pid, r.kind, r.stream);
     u32 hsh = hash_code(code);
     if (cache[hsh & 255] == code) continue;  // a stale miss only costs a probe
@@ -63,6 +88,12 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
   mn = warp_min_i64(mn);
   mx = warp_max_i64(mx);
   md = warp_max_i64(md);
+  qmn = warp_min_i64(qmn);
+  qmx = warp_max_i64(qmx);
+  if ((threadIdx.x & 31) == 0 && qmn != INT64_MAX) {
+    atomicMin((i64 *)&misc[3], qmn);
+    atomicMax((i64 *)&misc[4], qmx);
+  }
   if ((threadIdx.x & 31) == 0) {
     if (mn != INT64_MAX) {
       atomicMin((i64 *)&misc[0], mn);
@@ -126,6 +157,52 @@ __global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t 
       r = lo;
     }
     tt->rank_of_slot[s] = r;
+  }
+}
+
+// One CTA: sorts and ranks the communicator ids.
+__global__ void __launch_bounds__(1024) k_rank_comms(CommTable *cm, int32_t *status) {
+  __shared__ u64 buf[TA_COMM_SLOTS];
+  __shared__ int n_c;
+  const int tid = threadIdx.x;
+  for (int i = tid; i < TA_COMM_SLOTS; i += blockDim.x) buf[i] = cm->slots[i];
+  if (tid == 0) n_c = 0;
+  __syncthreads();
+  for (int k = 2; k <= TA_COMM_SLOTS; k <<= 1)
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = tid; i < TA_COMM_SLOTS; i += blockDim.x) {
+        int ixj = i ^ j;
+        if (ixj > i) {
+          u64 a = buf[i], b = buf[ixj];
+          bool up = (i & k) == 0;
+          if ((a > b) == up) { buf[i] = b; buf[ixj] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  for (int i = tid; i < TA_COMM_SLOTS; i += blockDim.x)
+    if (buf[i] != TRIPLE_EMPTY && (i + 1 == TA_COMM_SLOTS || buf[i + 1] == TRIPLE_EMPTY)) n_c = i + 1;
+  __syncthreads();
+  int n = n_c;
+  if (n > TA_MAX_COMMS) {
+    if (tid == 0) ta_set_err(status, TA_ERR_TOO_LARGE);
+    n = TA_MAX_COMMS;
+  }
+  for (int i = tid; i < n; i += blockDim.x) cm->sorted_id[i] = buf[i];
+  if (tid == 0) status[ST_N_COMMS] = n;
+  for (int s = tid; s < TA_COMM_SLOTS; s += blockDim.x) {
+    u64 c = cm->slots[s];
+    int r = -1;
+    if (c != TRIPLE_EMPTY) {
+      int lo = 0, hi = n - 1;
+      while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (buf[mid] < c) lo = mid + 1;
+        else hi = mid;
+      }
+      r = lo;
+    }
+    cm->rank_of_slot[s] = r;
   }
 }
 
@@ -196,9 +273,10 @@ static int grid_for(int64_t n, int threads, int per_sm) {
 ta_status ta_launch_discover(ta_window *h) {
   if (h->n > 0) {
     k_discover<<<grid_for(h->n, 256, 8), 256, 0, h->stream>>>(
-        h->events, h->n, h->d_off, h->d_t0, h->d_t1, h->W, h->d_triples, h->d_load_sum, h->d_misc,
-        h->d_status);
+        h->events, h->n, h->d_off, h->d_t0, h->d_t1, h->W, h->d_triples, h->d_comms, h->d_load_sum,
+        h->d_misc, h->d_status);
   }
+  k_rank_comms<<<1, 1024, 0, h->stream>>>(h->d_comms, h->d_status);
   TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank_triples, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         TA_TRIPLE_SLOTS * (int)sizeof(u64)));
   k_rank_triples<<<1, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_status);

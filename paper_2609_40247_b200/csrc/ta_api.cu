@@ -73,7 +73,7 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   const int W = h->W;
   cudaStream_t st = h->stream;
   size_t bytes = 3 * Carver::pad((W + 1) * 8) + Carver::pad(ST_WORDS * 4) +
-                 Carver::pad(sizeof(TripleTable)) + Carver::pad(16 * 8) +
+                 Carver::pad(sizeof(TripleTable)) + Carver::pad(sizeof(CommTable)) + Carver::pad(16 * 8) +
                  Carver::pad(W * sizeof(ta_load_summary)) + Carver::pad(10 * 256 * 4) + 256;
   void *b = ta_dalloc(h, bytes);
   if (!b) return TA_ERR_OOM;
@@ -83,6 +83,7 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   h->d_t1 = c.take<int64_t>(W + 1);
   h->d_status = c.take<int32_t>(ST_WORDS);
   h->d_triples = c.take<TripleTable>(1);
+  h->d_comms = c.take<CommTable>(1);
   h->d_misc = c.take<int64_t>(16);
   h->d_load_sum = c.take<ta_load_summary>(W);
   h->d_hist = c.take<u32>(10 * 256);
@@ -104,12 +105,15 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t1, h->h_t1.data(), W * 8, cudaMemcpyHostToDevice, st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status, 0, ST_WORDS * 4, st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_triples->slots, 0xFF, sizeof(h->d_triples->slots), st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_comms->slots, 0xFF, sizeof(h->d_comms->slots), st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_load_sum, 0, W * sizeof(ta_load_summary), st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_hist, 0, 10 * 256 * 4, st));
   int64_t misc_init[16] = {0};
   misc_init[0] = INT64_MAX;
   misc_init[1] = INT64_MIN;
   misc_init[2] = 0;
+  misc_init[3] = INT64_MAX;
+  misc_init[4] = INT64_MIN;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_misc, misc_init, sizeof(misc_init), cudaMemcpyHostToDevice, st));
 
   TA_TRY(ta_launch_discover(h));
@@ -127,6 +131,9 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   h->min_name = misc[0];
   h->max_name = misc[1];
   h->max_dur = misc[2];
+  h->min_seq = misc[3];
+  h->max_seq = misc[4];
+  h->n_comms = words[ST_N_COMMS];
   h->n_valid = 0;
   for (int w = 0; w < W; w++) {
     ta_load_summary &s = sums[w];

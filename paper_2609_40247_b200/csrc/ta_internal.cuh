@@ -35,6 +35,12 @@ struct TripleTable {       // device-resident, filled by the discovery kernel
   int32_t pid_value[TA_MAX_TRIPLES];   // per pid rank
 };
 
+struct CommTable {         // communicator ids seen on COLL records (biased; all-ones = empty)
+  u64 slots[TA_COMM_SLOTS];
+  int32_t rank_of_slot[TA_COMM_SLOTS];
+  u64 sorted_id[TA_MAX_COMMS];         // ascending (biased)
+};
+
 struct SortPlan {
   int n_pass;
   int shift[10];
@@ -61,7 +67,10 @@ struct ta_window {
   // load products
   int32_t *d_status;
   TripleTable *d_triples;
-  int64_t *d_misc;           // [0]=min name,[1]=max name,[2]=max duration (atomics)
+  int64_t *d_misc;           // [0]=min name,[1]=max name,[2]=max duration,[3]=min seq,[4]=max seq
+  CommTable *d_comms;
+  int n_comms;
+  int64_t min_seq, max_seq;
   ta_load_summary *d_load_sum;
   u64 *d_keys;
   u32 *d_hist;               // [pass][256]

@@ -86,6 +86,7 @@ def attribution(sv, wins, n_valid, lane_list):
     n = len(sv)
     parent = [-1] * n
     depth = [0] * n
+    n_enc = [0] * n
     bad = False
     for (w, pid, dom, st, b, e) in lane_list:
         if dom != 0:
@@ -101,10 +102,17 @@ def attribution(sv, wins, n_valid, lane_list):
                     bad = True
                 if sj <= si and ei <= ej and ((sj, ej) != (si, ei) or j < i):
                     enc.append(j)
-            depth[i] = len(enc)
+            n_enc[i] = len(enc)
             if enc:
                 parent[i] = max(enc, key=lambda j: (int(sv[j]["ts_start"]), -int(sv[j]["ts_end"]), j))
-    return parent, depth, bad
+    # depth = level in the forest the parents define
+    for i in range(n):
+        d, c = 0, parent[i]
+        while c >= 0:
+            d += 1
+            c = parent[c]
+        depth[i] = min(d, 255)
+    return parent, depth, bad, n_enc
 
 
 def gaps_bitmap(sv, lane, W0, W1):

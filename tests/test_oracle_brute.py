@@ -80,10 +80,15 @@ def test_attribution_against_quadratic_scan(seed):
     sv = _sorted_view(ev, r)
     wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
     ll = brute.lanes(sv, wins, r["n_valid"])
-    parent, depth, bad = brute.attribution(sv, wins, r["n_valid"], ll)
+    parent, depth, bad, n_enc = brute.attribution(sv, wins, r["n_valid"], ll)
     assert not bad and r["attr_status"] in (0, 8)
     assert r["parent"].tolist() == parent
     assert r["depth"].tolist() == depth
+    # the forest level equals the number of enclosers for every record of non-zero length
+    for i in range(r["n_valid"]):
+        if sv[i]["kind"] <= 2 and sv[i]["ts_end"] > sv[i]["ts_start"]:
+            assert depth[i] == min(n_enc[i], 255)
+        assert depth[i] <= n_enc[i]
     assert (r["attr_status"] == 8) == (max(depth) > 8)
     # for properly nested lanes the parent is the nearest earlier OP that ends no earlier
     for (w, pid, dom, st, b, e) in ll:
@@ -124,7 +129,7 @@ def test_bad_nesting_flag(seed):
     sv = _sorted_view(ev, r)
     wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
     ll = brute.lanes(sv, wins, r["n_valid"])
-    parent, depth, bad = brute.attribution(sv, wins, r["n_valid"], ll)
+    parent, depth, bad, _ = brute.attribution(sv, wins, r["n_valid"], ll)
     assert (r["attr_status"] == 9) == bad
     assert bool(r["attr_sum"]["bad_nesting"].any()) == bad
     # the oracle evaluates the definition even then
