@@ -339,6 +339,18 @@ void ta_free(ta_window *h);
 const char *ta_strerror(ta_status s);
 int32_t ta_version(void);
 
+/* Instrumentation (process-wide, not thread-safe; meant for benchmarks).
+ * ta_launch_count: number of kernels this library has launched since it was
+ * loaded.  ta_profile_enable(1): from now on record a CUDA event pair around
+ * every radix-sort pass (the dominant kernel) on the launching stream, and
+ * forget the pairs recorded so far; ta_profile_enable(0) stops recording.
+ * ta_profile_radix: synchronises the recorded events and returns the number of
+ * passes timed and the sum of their durations in milliseconds (0 on success,
+ * -1 on a CUDA error). */
+int64_t ta_launch_count(void);
+void ta_profile_enable(int32_t on);
+int32_t ta_profile_radix(int64_t *n_passes, double *total_ms);
+
 #ifdef __cplusplus
 }
 #endif

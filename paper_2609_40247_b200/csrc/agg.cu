@@ -214,7 +214,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.chunk = chunk;
   TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_agg, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)sizeof(AggSmem)));
-  k_agg<<<(unsigned)blocks, AG_THREADS, sizeof(AggSmem), st>>>(a);
+  k_agg<<<TA_N (unsigned)blocks, AG_THREADS, sizeof(AggSmem), st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   u64 ng = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));

@@ -470,9 +470,9 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   a.launch_of = h->join.launch_of; a.op_of = op_of; a.op_n = op_n; a.op_first = op_first;
   a.op_last = op_last; a.op_ns = op_ns;
   if (n > 0) {
-    k_attr<<<(unsigned)tiles, AT_THREADS, 0, st>>>(a);
-    k_attr_ops<<<(unsigned)((n + 2047) / 2048), 512, 0, st>>>(a);
-    k_attr_finalize<<<(unsigned)((h->n_valid + 255) / 256 > 0 ? (h->n_valid + 255) / 256 : 1), 256, 0, st>>>(a);
+    k_attr<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
+    k_attr_ops<<<TA_N (unsigned)((n + 2047) / 2048), 512, 0, st>>>(a);
+    k_attr_finalize<<<TA_N (unsigned)((h->n_valid + 255) / 256 > 0 ? (h->n_valid + 255) / 256 : 1), 256, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
   }
   std::vector<ta_attr_summary> hs(W);

@@ -288,7 +288,7 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   TA_CHECK_CUDA(h, cudaMemcpyAsync(d_expected, expected.data(), h->n_comms * 4, cudaMemcpyHostToDevice, st));
 
   const int gb = (int)((m + 255) / 256);
-  k_coll_keys<<<gb, 256, 0, st>>>(cx, k_in, slot_of);
+  k_coll_keys<<<TA_N gb, 256, 0, st>>>(cx, k_in, slot_of);
   TA_TRY(ta_radix_sort_pairs(h, k_in, nullptr, k_s, v_s, ks, cs, m,
                              ta_make_plan(0, cx.qbits + cx.cbits + wbits), nullptr, sort_tmp));
   ScanTemp s2;
@@ -314,13 +314,13 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   ga.g_comm = co.take<int64_t>(ng); ga.g_min = co.take<int64_t>(ng); ga.g_max = co.take<int64_t>(ng);
   ga.g_skew = co.take<int64_t>(ng); ga.g_end = co.take<int64_t>(ng);
   ga.r_nstrag = r_nstrag;
-  k_coll_groups<<<(unsigned)((ng + 255) / 256), 256, 0, st>>>(ga);
+  k_coll_groups<<<TA_N (unsigned)((ng + 255) / 256), 256, 0, st>>>(ga);
 
   // 5. members
   CollMemberArgs ma;
   ma.c = cx; ma.gid_of_c = gid_of_c; ma.slot_of = slot_of; ma.g_max = ga.g_max; ma.g_flags = ga.g_flags;
   ma.wait_ns = wait_ns; ma.r_seen = r_seen; ma.r_ncoll = r_ncoll; ma.r_sum = r_sum; ma.r_maxw = r_maxw;
-  k_coll_members<<<gb, 256, 0, st>>>(ma);
+  k_coll_members<<<TA_N gb, 256, 0, st>>>(ma);
   TA_CHECK_CUDA(h, cudaGetLastError());
 
   // rank table: compact the (window, pid) slots that saw a COLL record

@@ -244,7 +244,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   a.gap_before = gap_before; a.lane_gaps = lane_gaps; a.lane_hist = lane_hist; a.win_hist = win_hist;
   a.long_gaps = list; a.list_cap = cap; a.st_max = st_max; a.st_cnt = st_cnt;
   a.counter = (u32 *)(scal + 1); a.status = h->d_status; a.n_long_out = scal;
-  if (tiles > 0) k_gaps<<<(unsigned)tiles, GP_THREADS, 0, st>>>(a);
+  if (tiles > 0) k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   u64 n_long = 0;
   int32_t words[ST_WORDS];
@@ -257,7 +257,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
     if (!b2) return TA_ERR_OOM;
     TA_CHECK_CUDA(h, cudaMemsetAsync(st_max, 0, (char *)zero_end - (char *)st_max, st));
     a.long_gaps = (ta_long_gap *)b2; a.list_cap = (i64)n_long; a.list_only = 1;
-    k_gaps<<<(unsigned)tiles, GP_THREADS, 0, st>>>(a);
+    k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_TRY(ta_read_status(h, words));
     if (words[ST_ERR]) return (ta_status)words[ST_ERR];

@@ -367,7 +367,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   void *tmp_alloc = nullptr;
   bool direct = true;
   if (n > 0) {
-    k_join_minmax<<<grid, JN_THREADS, 0, st>>>(a);
+    k_join_minmax<<<TA_N grid, JN_THREADS, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_CHECK_CUDA(h, cudaMemcpyAsync(hmin.data(), slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaMemcpyAsync(hmax.data(), slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
@@ -388,9 +388,9 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       a.table = (u32 *)tmp_alloc;
       TA_CHECK_CUDA(h, cudaMemsetAsync(a.table, 0xFF, (size_t)(M > 0 ? M : 1) * 4, st));
       TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_base, hbase.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
-      k_join_build<<<grid, JN_THREADS, 0, st>>>(a);
-      k_join_probe<true><<<grid, JN_THREADS, 0, st>>>(a);
-      k_join_launch_stats<true><<<grid, JN_THREADS, 0, st>>>(a);
+      k_join_build<<<TA_N grid, JN_THREADS, 0, st>>>(a);
+      k_join_probe<true><<<TA_N grid, JN_THREADS, 0, st>>>(a);
+      k_join_launch_stats<true><<<TA_N grid, JN_THREADS, 0, st>>>(a);
     } else {
       // general path: compact, sort by (slot, corr) with sorted position as the stable tie-break
       size_t tb = Carver::pad(nn * 4) * 3 + Carver::pad(nn * 8) * 3 + scan_temp_bytes(n) * 2 +
@@ -417,10 +417,10 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       if (m > 0) {
         const int gb = (int)((m + 255) / 256);
         u32 *vscr = (u32 *)found;  // found is not needed before the sorts are done
-        k_join_key_corr<<<gb, 256, 0, st>>>(pos, m, a.corr, k_in);
+        k_join_key_corr<<<TA_N gb, 256, 0, st>>>(pos, m, a.corr, k_in);
         TA_TRY(ta_radix_sort_pairs(h, k_in, pos, k_s, vscr, k_f, pos_s, m, ta_make_plan(0, 64), nullptr,
                                    sort_tmp));
-        k_join_key_slot<<<gb, 256, 0, st>>>(pos_s, m, a.lane_off, a.n_lanes, a.lane_slot, k_in);
+        k_join_key_slot<<<TA_N gb, 256, 0, st>>>(pos_s, m, a.lane_off, a.n_lanes, a.lane_slot, k_in);
         int sb = bit_length64((uint64_t)(n_slots > 1 ? n_slots - 1 : 1));
         TA_TRY(ta_radix_sort_pairs(h, k_in, pos_s, k_s, vscr, k_f, pos, m, ta_make_plan(0, sb), nullptr,
                                    sort_tmp));
@@ -432,8 +432,8 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
         TA_TRY((launch_scan<OpMax, JoinHeadIn, JoinHeadOut>(h, m, hin, hout, OpMax(), t2)));
       }
       a.found = found;
-      k_join_probe<false><<<grid, JN_THREADS, 0, st>>>(a);
-      k_join_launch_stats<false><<<grid, JN_THREADS, 0, st>>>(a);
+      k_join_probe<false><<<TA_N grid, JN_THREADS, 0, st>>>(a);
+      k_join_launch_stats<false><<<TA_N grid, JN_THREADS, 0, st>>>(a);
     }
     TA_CHECK_CUDA(h, cudaGetLastError());
   }

@@ -272,14 +272,14 @@ static int grid_for(int64_t n, int threads, int per_sm) {
 
 ta_status ta_launch_discover(ta_window *h) {
   if (h->n > 0) {
-    k_discover<<<grid_for(h->n, 256, 8), 256, 0, h->stream>>>(
+    k_discover<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(
         h->events, h->n, h->d_off, h->d_t0, h->d_t1, h->W, h->d_triples, h->d_comms, h->d_load_sum,
         h->d_misc, h->d_status);
   }
-  k_rank_comms<<<1, 1024, 0, h->stream>>>(h->d_comms, h->d_status);
+  k_rank_comms<<<TA_N 1, 1024, 0, h->stream>>>(h->d_comms, h->d_status);
   TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank_triples, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         TA_TRIPLE_SLOTS * (int)sizeof(u64)));
-  k_rank_triples<<<1, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_status);
+  k_rank_triples<<<TA_N 1, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_status);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }
@@ -300,7 +300,7 @@ ta_status ta_launch_load(ta_window *h) {
   a.ev = h->events; a.n = h->n; a.off = h->d_off; a.t0 = h->d_t0; a.t1 = h->d_t1; a.W = h->W;
   a.tt = h->d_triples; a.keys = h->d_keys; a.hist = h->d_hist;
   a.sbits = h->sbits; a.tbits = h->tbits; a.wbits = h->wbits; a.plan = h->plan;
-  k_load<<<grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
+  k_load<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }

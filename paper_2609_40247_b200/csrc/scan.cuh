@@ -72,7 +72,7 @@ template <class Op, class In, class Out>
 static inline ta_status launch_scan(ta_window *h, int64_t n, In in, Out out, Op op, ScanTemp t) {
   if (n <= 0) return TA_OK;
   int64_t tiles = (n + SC_TILE - 1) / SC_TILE;
-  k_scan<Op, In, Out><<<(unsigned)tiles, SC_THREADS, 0, h->stream>>>(n, in, out, op, t, h->d_status);
+  k_scan<Op, In, Out><<<TA_N (unsigned)tiles, SC_THREADS, 0, h->stream>>>(n, in, out, op, t, h->d_status);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }

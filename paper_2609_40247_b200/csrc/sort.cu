@@ -230,10 +230,10 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
     TA_CHECK_CUDA(h, cudaMemsetAsync(own_hist, 0, 10 * RS_BINS * sizeof(u32), st));
     int64_t want = (n + 255) / 256;
     int grid = (int)(want < 148 * 8 ? want : 148 * 8);
-    k_radix_hist<<<grid, 256, 0, st>>>(keys_in, n, plan, own_hist);
+    k_radix_hist<<<TA_N grid, 256, 0, st>>>(keys_in, n, plan, own_hist);
     hist = own_hist;
   }
-  k_radix_scan_hist<<<plan.n_pass, 256, 0, st>>>(hist, bin_offset);
+  k_radix_scan_hist<<<TA_N plan.n_pass, 256, 0, st>>>(hist, bin_offset);
   const u64 *kin = keys_in;
   const u32 *vin = vals_in;
   for (int p = 0; p < plan.n_pass; p++) {
@@ -246,7 +246,10 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
     a.n = n; a.shift = plan.shift[p]; a.bits = plan.bits[p];
     a.bin_offset = bin_offset + p * RS_BINS;
     a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
-    k_radix_pass<<<(unsigned)tiles, RS_THREADS, sizeof(RadixSmem), st>>>(a);
+    const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
+    if (timed) ta_profile_mark(st, 1);
+    k_radix_pass<<<TA_N (unsigned)tiles, RS_THREADS, sizeof(RadixSmem), st>>>(a);
+    if (timed) ta_profile_mark(st, 0);
     kin = a.keys_out;
     vin = a.vals_out;
   }

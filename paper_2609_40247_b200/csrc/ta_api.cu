@@ -47,7 +47,47 @@ ta_status ta_read_status(ta_window *h, int32_t *w) {
   return TA_OK;
 }
 
+// ---- instrumentation: launch counter and event pairs around the radix passes ----
+long long g_ta_launches = 0;
+int g_ta_profile = 0;
+static std::vector<cudaEvent_t> g_prof_events;  // begin, end, begin, end, ...
+static size_t g_prof_used = 0;
+
+void ta_profile_mark(cudaStream_t st, int begin) {
+  (void)begin;
+  if (g_prof_used == g_prof_events.size()) {
+    cudaEvent_t e;
+    if (cudaEventCreate(&e) != cudaSuccess) return;
+    g_prof_events.push_back(e);
+  }
+  cudaEventRecord(g_prof_events[g_prof_used++], st);
+}
+
 extern "C" {
+
+// Instrumentation helpers (they carry no work).  ta_profile_enable(1) makes the
+// library record a CUDA event pair around every radix-sort pass and forgets the
+// pairs recorded so far; ta_profile_radix reads them back (synchronises the
+// events): number of passes timed and their summed duration in milliseconds.
+void ta_profile_enable(int32_t on) {
+  g_ta_profile = on;
+  g_prof_used = 0;
+}
+int32_t ta_profile_radix(int64_t *n_passes, double *total_ms) {
+  int64_t n = 0;
+  double ms = 0;
+  for (size_t i = 0; i + 1 < g_prof_used; i += 2) {
+    if (cudaEventSynchronize(g_prof_events[i + 1]) != cudaSuccess) return -1;
+    float t = 0;
+    if (cudaEventElapsedTime(&t, g_prof_events[i], g_prof_events[i + 1]) != cudaSuccess) return -1;
+    ms += t;
+    n++;
+  }
+  if (n_passes) *n_passes = n;
+  if (total_ms) *total_ms = ms;
+  return 0;
+}
+int64_t ta_launch_count(void) { return g_ta_launches; }
 
 const char *ta_strerror(ta_status s) {
   switch (s) {

@@ -152,6 +152,13 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
 
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 
+// ---- instrumentation (no work: a launch counter and optional event pairs) ----
+extern long long g_ta_launches;   // kernels launched by this library since load
+extern int g_ta_profile;          // 1 = record a CUDA event pair around each radix pass
+static inline unsigned ta_one() { ++g_ta_launches; return 1u; }
+#define TA_N ta_one() *           // used as kernel<<<TA_N grid, ...>>>: counts the launch
+void ta_profile_mark(cudaStream_t st, int begin);  // called around k_radix_pass when profiling
+
 // =================================================================== device
 #ifdef __CUDACC__
 

@@ -196,7 +196,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
                                h->d_hist, sort_tmp));
     // step 2: equal-key runs
     if (h->n_valid > 1)
-      k_fix_ties<<<nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
+      k_fix_ties<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
                                                         h->d_status);
     int32_t words[ST_WORDS];
     TA_TRY(ta_read_status(h, words));
@@ -210,14 +210,14 @@ ta_status ta_run_sort_timeline(ta_window *h) {
       u64 *dkeys = cx.take<u64>(n);
       u32 *dorder = cx.take<u32>(n);
       const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
-      k_duration_key<<<nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit, h->max_dur,
+      k_duration_key<<<TA_N nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit, h->max_dur,
                                                    dkeys);
       int dbits = 1;
       while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
       SortPlan dplan = ta_make_plan(0, dbits);
       TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
                                  sort_tmp));
-      k_gather_u64<<<nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
+      k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
       TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
                                  sort_tmp));
       TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
@@ -235,7 +235,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
       u32 *cur = perm + h->n_valid, *nxt = alt;
       for (int stage = 0; stage < 4; stage++) {
         if (stage == 3 && h->W == 1) break;
-        k_tail_key<<<nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
+        k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
         int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : 64;
         SortPlan tp = ta_make_plan(0, bits);
         TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
@@ -253,9 +253,9 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     g.sbits = h->sbits;
     g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
     g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
-    k_gather<<<nblk(n, 256), 256, 0, st>>>(g);
+    k_gather<<<TA_N nblk(n, 256), 256, 0, st>>>(g);
   }
-  k_lane_table<<<1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
+  k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
                                    h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
                                    lane_window, lane_pid, lane_stream, lane_domain, lane_off,
                                    lane_code, lane_slot, n_lanes_dev, lane_cap);

@@ -84,7 +84,7 @@ _CollResult = _ptr_struct("_CollResult", [
 
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
-           "ta_version"]
+           "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix"]
 
 _lib = None
 
@@ -125,8 +125,32 @@ def lib():
         L.ta_strerror.restype = ctypes.c_char_p
         L.ta_strerror.argtypes = [ctypes.c_int]
         L.ta_version.restype = ctypes.c_int32
+        L.ta_launch_count.restype = ctypes.c_int64
+        L.ta_profile_enable.restype = None
+        L.ta_profile_enable.argtypes = [ctypes.c_int32]
+        L.ta_profile_radix.restype = ctypes.c_int32
+        L.ta_profile_radix.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
         _lib = L
     return _lib
+
+
+def launch_count() -> int:
+    """Kernels launched by the library since it was loaded."""
+    return int(lib().ta_launch_count())
+
+
+def profile_enable(on: bool) -> None:
+    """Start (and reset) / stop the CUDA-event timing of the radix-sort passes."""
+    lib().ta_profile_enable(1 if on else 0)
+
+
+def profile_radix():
+    """(number of radix passes timed, their summed duration in ms)."""
+    n = ctypes.c_int64()
+    ms = ctypes.c_double()
+    if lib().ta_profile_radix(ctypes.byref(n), ctypes.byref(ms)) != 0:
+        raise RuntimeError("ta_profile_radix: CUDA error")
+    return n.value, ms.value
 
 
 class _DevView:
