@@ -335,6 +335,43 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes,
  * NULL-safe.  Synchronises the handle's stream first. */
 void ta_free(ta_window *h);
 
+/* ------------------------------------------------------------------------
+ * ta_lane_gaps_noalloc - the stream-gap scan of ONE device lane, for callers
+ * that cannot allocate device memory.  (The paper has no counterpart for this
+ * entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: a monitoring agent that lives inside a serving process whose
+ * device heap is fully reserved at start-up, a plug-in whose host forbids
+ * cudaMalloc / cudaFree inside its callbacks, or a latency-critical loop that
+ * cannot afford the device-wide synchronisation an allocation or a free may
+ * imply.  Every other entry point obtains its buffers through ta_env; this one
+ * obtains nothing: it calls no cudaMalloc, cudaFree or any allocating routine.
+ * Its scratch (tile descriptors of the scan, a counter, a status word: about
+ * 16 KB) is a fixed array inside the library image, which every GPU that loads
+ * the library holds until the process exits.
+ *
+ * Input: the records of one device lane of one window [win_t0, win_t1), already
+ * in canonical order (ts_start ascending), as two device columns of n entries;
+ * every ts_start lies in the window.  Output, both caller-owned device memory:
+ * gap_before[n] and one ta_lane_gaps row, with exactly the values ta_stream_gaps
+ * gives for that lane (gap_before, busy, idle, n_events, n_gaps, max_gap,
+ * first_start, last_end).  No histogram and no long-gap list.
+ *
+ * Limits and rules: n <= TA_NOALLOC_MAX_RECORDS, else TA_ERR_TOO_LARGE (the
+ * fixed scratch covers no more).  The first call on a device looks up the
+ * address of the scratch array (with that device current) and should therefore
+ * be made before any stream capture begins.  All calls on a device share the
+ * one scratch array, which keeps the previous call's contents; each call clears
+ * it first, so two calls that overlap on the GPU (different streams or threads)
+ * race and must be serialised by the caller.  The call enqueues its work on
+ * cuda_stream, waits for it and returns TA_OK, TA_ERR_INVALID_ARG,
+ * TA_ERR_TOO_LARGE, TA_ERR_CUDA or TA_ERR_TIMEOUT.
+ */
+#define TA_NOALLOC_MAX_RECORDS (1 << 22)
+ta_status ta_lane_gaps_noalloc(const int64_t *ts_start, const int64_t *ts_end, int64_t n,
+                               int64_t win_t0, int64_t win_t1, int64_t *gap_before,
+                               ta_lane_gaps *lane_out, void *cuda_stream);
+
 /* Helpers that carry no work. */
 const char *ta_strerror(ta_status s);
 int32_t ta_version(void);

@@ -84,7 +84,9 @@ _CollResult = _ptr_struct("_CollResult", [
 
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
-           "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix"]
+           "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
+           "ta_lane_gaps_noalloc"]
+NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
 
@@ -125,6 +127,9 @@ def lib():
         L.ta_strerror.restype = ctypes.c_char_p
         L.ta_strerror.argtypes = [ctypes.c_int]
         L.ta_version.restype = ctypes.c_int32
+        L.ta_lane_gaps_noalloc.restype = ctypes.c_int
+        L.ta_lane_gaps_noalloc.argtypes = [_vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                           _vp, _vp, _vp]
         L.ta_launch_count.restype = ctypes.c_int64
         L.ta_profile_enable.restype = None
         L.ta_profile_enable.argtypes = [ctypes.c_int32]
@@ -132,6 +137,38 @@ def lib():
         L.ta_profile_radix.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
         _lib = L
     return _lib
+
+
+def lane_gaps_noalloc(ts_start, ts_end, win_t0: int, win_t1: int, gap_before=None, lane_out=None,
+                      stream=None):
+    """Gap scan of one device lane through ta_lane_gaps_noalloc, the entry point for
+    callers that may not allocate device memory: the library call itself allocates
+    nothing (its scratch is a fixed array inside libta.so).  The output buffers are
+    the caller's; pass `gap_before` (int64, n) and `lane_out` (uint8, 56 bytes) to
+    reuse buffers you already own, otherwise this wrapper creates them with torch.
+    Inputs: int64 CUDA tensors of one lane in canonical order.  Calls must not
+    overlap on the GPU (they share the scratch array); at most NOALLOC_MAX_RECORDS
+    records.  Returns (gap_before tensor, lane summary as a LANE_GAPS numpy record)."""
+    import torch
+    L = lib()
+    if not (ts_start.is_cuda and ts_end.is_cuda and ts_start.dtype == torch.int64
+            and ts_end.dtype == torch.int64 and ts_start.is_contiguous() and ts_end.is_contiguous()):
+        raise ValueError("ts_start / ts_end must be contiguous int64 CUDA tensors")
+    n = ts_start.numel()
+    if ts_end.numel() != n:
+        raise ValueError("ts_start and ts_end differ in length")
+    dev = ts_start.device
+    if gap_before is None:
+        gap_before = torch.empty(max(n, 1), dtype=torch.int64, device=dev)
+    if lane_out is None:
+        lane_out = torch.empty(LANE_GAPS.itemsize, dtype=torch.uint8, device=dev)
+    s = stream if stream is not None else torch.cuda.current_stream(dev)
+    with torch.cuda.device(dev):
+        st = L.ta_lane_gaps_noalloc(ts_start.data_ptr(), ts_end.data_ptr(), n, int(win_t0), int(win_t1),
+                                    gap_before.data_ptr(), lane_out.data_ptr(), s.cuda_stream)
+    if st != 0:
+        raise TaError(st, "ta_lane_gaps_noalloc")
+    return gap_before[:n], lane_out.cpu().numpy().view(LANE_GAPS)[0]
 
 
 def launch_count() -> int:
