@@ -6,16 +6,16 @@
 // One pass over the sorted ts_start / ts_end / kind columns.  The scan is made
 // lane-aware without segment flags: the scanned value is (lane + 1) << 40 |
 // (clipped end - window start), which grows from lane to lane, so a prefix
-// that belongs to an earlier lane is recognised by its upper bits.  Two chained
-// tile scans run in the same kernel: the maximum, then the number of long-gap
-// list entries (so the list is written in order, without a sort).
+// that belongs to an earlier lane is recognised by its upper bits.  Long gaps
+// are rare: they are appended to a list with an atomic cursor and the list is
+// put in (lane, time) order afterwards with the pair sorter.
 // HBM-bound: 18 B read + 8 B written per device record.
 #include <climits>
 
 #include "ta_internal.cuh"
 
-#define GP_THREADS 512
-#define GP_ITEMS 4
+#define GP_THREADS 256
+#define GP_ITEMS 8
 #define GP_TILE (GP_THREADS * GP_ITEMS)
 #define GP_LOW ((1ull << 40) - 1)
 
@@ -32,180 +32,247 @@ struct GapArgs {
   int64_t *gap_before;
   ta_lane_gaps *lane_gaps;
   u32 *lane_hist, *win_hist;
-  ta_long_gap *long_gaps;
+  ta_long_gap *list;  // unordered
+  u64 *list_key;      // lane << 32 | next_event (0xFFFFFFFF for a tail gap)
   i64 list_cap;
-  u64 *st_max, *st_cnt;
+  u64 *st_max;
   u32 *counter;
   int32_t *status;
-  u64 *n_long_out;
+  u64 *n_long;        // append cursor
 };
 
-__device__ __forceinline__ u64 block_reduce(u64 v, bool is_max, u64 *smem) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  v = is_max ? warp_reduce(v, OpMax()) : warp_reduce(v, OpAdd());
-  __syncthreads();
-  if (lane == 0) smem[warp] = v;
-  __syncthreads();
-  if (warp == 0) {
-    u64 w = lane < (int)(blockDim.x >> 5) ? smem[lane] : 0;
-    w = is_max ? warp_reduce(w, OpMax()) : warp_reduce(w, OpAdd());
-    if (lane == 0) smem[32] = w;
+// largest l with lane_off[l] <= p, found by the 32 lanes of one warp together
+__device__ __forceinline__ int warp_lane_search(const int32_t *lane_off, int n_lanes, int64_t p) {
+  const int lane = threadIdx.x & 31;
+  int lo = 0, hi = n_lanes;
+  while (hi - lo > 1) {
+    int step = (hi - lo + 31) >> 5;
+    int idx = lo + lane * step;
+    bool ok = idx < hi && (int64_t)lane_off[idx] <= p;
+    u32 m = __ballot_sync(0xffffffffu, ok);
+    int k = 31 - __clz((int)m);  // lane 0 always qualifies (lane_off[lo] <= p)
+    lo = lo + k * step;
+    hi = min(hi, lo + step);
   }
-  __syncthreads();
-  return smem[32];
+  return lo;
 }
 
-__global__ void __launch_bounds__(GP_THREADS) k_gaps(GapArgs a) {
+__global__ void __launch_bounds__(GP_THREADS, 3) k_gaps(GapArgs a) {
   __shared__ u64 tmp[33];
-  __shared__ u64 s_excl_max, s_excl_cnt;
-  __shared__ u32 s_hist[TA_NBINS];
-  __shared__ int s_tile;
+  __shared__ u64 red[4][GP_THREADS / 32];
+  __shared__ u64 s_excl_max;
+  __shared__ u32 s_hist[2][TA_NBINS];  // the tile's first two lanes; further lanes go straight to global
+  __shared__ int s_tile, s_lane0, s_lane1;
   const int tid = threadIdx.x;
-  if (tid == 0) s_tile = (int)atomicAdd(a.counter, 1u);
+  if (tid == 0) { s_tile = (int)atomicAdd(a.counter, 1u); s_lane1 = -1; }
+  if (tid < 2 * TA_NBINS) (&s_hist[0][0])[tid] = 0;
   __syncthreads();
   const int tile = s_tile;
-  const int64_t p0 = (int64_t)tile * GP_TILE + (int64_t)tid * GP_ITEMS;
-
-  // lane of the first item, then walk
-  int lane_id = -1;
-  if (p0 < a.n_valid && a.n_lanes > 0) lane_id = lane_of_pos(a.lane_off, a.n_lanes, p0);
-  i64 s[GP_ITEMS], ce[GP_ITEMS], W0[GP_ITEMS], W1[GP_ITEMS];
-  int ln[GP_ITEMS];
-  bool dev[GP_ITEMS];
-  u64 v[GP_ITEMS];
-  u64 run = 0;
+  const int64_t tile_start = (int64_t)tile * GP_TILE;
+  const int64_t p0 = tile_start + (int64_t)tid * GP_ITEMS;
+  if (tid < 32) {
+    int l = -1;
+    if (tile_start < a.n_valid && a.n_lanes > 0) l = warp_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (tid == 0) s_lane0 = l;
+  }
+  // kinds of the thread's eight records (0 = not a device record of the window)
+  int16_t kd[GP_ITEMS];
+  const bool full = p0 + GP_ITEMS <= a.n;
+  if (full) {
+    uint4 q = *reinterpret_cast<const uint4 *>(a.kind + p0);
+    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS; j++) kd[j] = hq[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS; j++) kd[j] = p0 + j < a.n ? a.kind[p0 + j] : (int16_t)0;
+  }
+  bool any_dev = false;
 #pragma unroll
   for (int j = 0; j < GP_ITEMS; j++) {
-    int64_t p = p0 + j;
-    dev[j] = false;
-    ln[j] = -1;
-    v[j] = 0;
-    s[j] = ce[j] = W0[j] = W1[j] = 0;
-    if (p < a.n_valid) {
-      while (lane_id + 1 < a.n_lanes && (int64_t)a.lane_off[lane_id + 1] <= p) lane_id++;
-      if (a.kind[p] >= 3) {
-        dev[j] = true;
-        ln[j] = lane_id;
-        int w = a.lane_window[lane_id];
-        W0[j] = a.t0[w];
-        W1[j] = a.t1[w];
-        s[j] = a.ts[p];
-        i64 e = a.te[p];
-        ce[j] = e < W1[j] ? e : W1[j];
-        v[j] = ((u64)(lane_id + 1) << 40) | (u64)(ce[j] - W0[j]);
+    if (p0 + j >= a.n_valid) kd[j] = 0;
+    any_dev |= kd[j] >= 3;
+  }
+  i64 s[GP_ITEMS], ce[GP_ITEMS];  // ce: ts_end, clipped below
+#pragma unroll
+  for (int j = 0; j < GP_ITEMS; j++) s[j] = ce[j] = 0;
+  if (any_dev) {
+    if (full) {
+      const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
+      const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
+#pragma unroll
+      for (int j = 0; j < GP_ITEMS / 2; j++) {
+        longlong2 x = ps[j], y = pe[j];
+        s[2 * j] = x.x; s[2 * j + 1] = x.y;
+        ce[2 * j] = y.x; ce[2 * j + 1] = y.y;
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < GP_ITEMS; j++)
+        if (p0 + j < a.n) { s[j] = a.ts[p0 + j]; ce[j] = a.te[p0 + j]; }
+    }
+  }
+  __syncthreads();
+  const int l0 = s_lane0;
+  // lanes of the items: walk forward from the tile's first lane
+  int ln[GP_ITEMS];
+  u64 run = 0;
+  {
+    int l = l0;
+    int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+    i64 w0 = 0, w1 = 0;
+    int wl = -1;
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS; j++) {
+      const int64_t p = p0 + j;
+      ln[j] = -1;
+      if (kd[j] >= 3) {
+        while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+        if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
+        ln[j] = l;
+        ce[j] = ce[j] < w1 ? ce[j] : w1;
+        u64 v = ((u64)(l + 1) << 40) | (u64)(ce[j] - w0);
+        run = run > v ? run : v;
       }
     }
-    run = run > v[j] ? run : v[j];
+    const int64_t plast = min(tile_start + GP_TILE, a.n_valid) - 1;
+    if (plast >= p0 && plast < p0 + GP_ITEMS) {  // this thread owns the tile's last kept record
+      while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      s_lane1 = l;
+    }
   }
   u64 tile_max;
   u64 thread_excl = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &tile_max);
   if (tid < 32) {
-    u64 e = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status);
-    if (tid == 0) s_excl_max = e;
+    u64 ex = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status);
+    if (tid == 0) s_excl_max = ex;
   }
   __syncthreads();
   u64 pre = s_excl_max > thread_excl ? s_excl_max : thread_excl;
 
-  // gaps, busy, list flags
-  i64 gap[GP_ITEMS], P[GP_ITEMS], tail[GP_ITEMS];
-  i64 busy[GP_ITEMS];
-  bool last[GP_ITEMS];
-  int cnt = 0;
-#pragma unroll
-  for (int j = 0; j < GP_ITEMS; j++) {
-    int64_t p = p0 + j;
-    gap[j] = 0; busy[j] = 0; tail[j] = 0; last[j] = false; P[j] = 0;
-    if (dev[j]) {
-      i64 Pi = ((pre >> 40) == (u64)(ln[j] + 1)) ? W0[j] + (i64)(pre & GP_LOW) : W0[j];
-      P[j] = Pi;
-      gap[j] = s[j] > Pi ? s[j] - Pi : 0;
-      i64 from = s[j] > Pi ? s[j] : Pi;
-      busy[j] = ce[j] > from ? ce[j] - from : 0;
-      last[j] = (p + 1 == (int64_t)a.lane_off[ln[j] + 1]);
-      if (last[j]) {
-        i64 Pm = Pi > ce[j] ? Pi : ce[j];
-        tail[j] = W1[j] - Pm;
-      }
-      if (gap[j] > 0 && gap[j] >= a.min_gap) cnt++;
-      if (last[j] && tail[j] > 0 && tail[j] >= a.min_gap) cnt++;
-      pre = pre > v[j] ? pre : v[j];
-    }
-    if (p < a.n && !a.list_only) a.gap_before[p] = gap[j];
-  }
-  // ordered long-gap list
-  u64 tile_cnt;
-  u64 cnt_excl = block_scan_exclusive<OpAdd>((u64)cnt, OpAdd(), tmp, &tile_cnt);
-  if (tid < 32) {
-    u64 e = tile_lookback<OpAdd>(a.st_cnt, tile, tile_cnt, OpAdd(), a.status);
-    if (tid == 0) {
-      s_excl_cnt = e;
-      if ((int64_t)(tile + 1) * GP_TILE >= a.n) *a.n_long_out = e + tile_cnt;  // last tile
-    }
-  }
-  __syncthreads();
-  if (cnt) {
-    i64 o = (i64)(s_excl_cnt + cnt_excl);
+  // gaps; statistics of the thread's first lane stay in registers, anything else is rare
+  i64 gap[GP_ITEMS];
+  u64 sb = 0, si = 0, ng = 0, mg = 0;
+  int lm = -1;
+  {
+    i64 w0 = 0, w1 = 0;
+    int wl = -1;
 #pragma unroll
     for (int j = 0; j < GP_ITEMS; j++) {
-      if (!dev[j]) continue;
-      if (gap[j] > 0 && gap[j] >= a.min_gap) {
-        if (o < a.list_cap) a.long_gaps[o] = ta_long_gap{ln[j], (int32_t)(p0 + j), P[j], gap[j]};
-        o++;
+      gap[j] = 0;
+      const int l = ln[j];
+      if (l < 0) continue;
+      if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
+      const i64 Pi = ((pre >> 40) == (u64)(l + 1)) ? w0 + (i64)(pre & GP_LOW) : w0;
+      const i64 g = s[j] > Pi ? s[j] - Pi : 0;
+      const i64 from = s[j] > Pi ? s[j] : Pi;
+      const i64 bz = ce[j] > from ? ce[j] - from : 0;
+      const bool last = (p0 + j + 1 == (int64_t)a.lane_off[l + 1]);
+      i64 tl = 0;
+      if (last) tl = w1 - (Pi > ce[j] ? Pi : ce[j]);
+      gap[j] = g;
+      pre = max(pre, ((u64)(l + 1) << 40) | (u64)(ce[j] - w0));
+      // long-gap list (rare)
+      const bool lg = g > 0 && g >= a.min_gap, lt = last && tl > 0 && tl >= a.min_gap;
+      if (lg || lt) {
+        i64 o = (i64)atomicAdd(a.n_long, (u64)((lg ? 1 : 0) + (lt ? 1 : 0)));
+        if (lg) {
+          if (o < a.list_cap) {
+            a.list[o] = ta_long_gap{l, (int32_t)(p0 + j), Pi, g};
+            a.list_key[o] = ((u64)l << 32) | (u64)(u32)(p0 + j);
+          }
+          o++;
+        }
+        if (lt && o < a.list_cap) {
+          a.list[o] = ta_long_gap{l, -1, w1 - tl, tl};
+          a.list_key[o] = ((u64)l << 32) | 0xFFFFFFFFull;
+        }
       }
-      if (last[j] && tail[j] > 0 && tail[j] >= a.min_gap) {
-        if (o < a.list_cap) a.long_gaps[o] = ta_long_gap{ln[j], -1, W1[j] - tail[j], tail[j]};
-        o++;
+      if (a.list_only) continue;
+      if (lm < 0) lm = l;
+      const int li = l - l0;
+      if (l == lm && li <= 1) {
+        sb += (u64)bz;
+        si += (u64)(g + tl);
+        if (g > 0) { ng++; mg = max(mg, (u64)g); atomicAdd(&s_hist[li][log2_bin(g)], 1u); }
+        if (tl > 0) { ng++; mg = max(mg, (u64)tl); atomicAdd(&s_hist[li][log2_bin(tl)], 1u); }
+      } else {  // a thread that straddles a lane boundary, or a third lane in the tile
+        ta_lane_gaps *gl = &a.lane_gaps[l];
+        const int w = a.lane_window[l];
+        if (bz) atomicAdd((u64 *)&gl->busy, (u64)bz);
+        if (g + tl) atomicAdd((u64 *)&gl->idle, (u64)(g + tl));
+        if (g > 0) {
+          atomicAdd((u64 *)&gl->n_gaps, 1ull);
+          atomicMax((i64 *)&gl->max_gap, g);
+          atomicAdd(&a.lane_hist[(size_t)l * TA_NBINS + log2_bin(g)], 1u);
+          atomicAdd(&a.win_hist[(size_t)w * TA_NBINS + log2_bin(g)], 1u);
+        }
+        if (tl > 0) {
+          atomicAdd((u64 *)&gl->n_gaps, 1ull);
+          atomicMax((i64 *)&gl->max_gap, tl);
+          atomicAdd(&a.lane_hist[(size_t)l * TA_NBINS + log2_bin(tl)], 1u);
+          atomicAdd(&a.win_hist[(size_t)w * TA_NBINS + log2_bin(tl)], 1u);
+        }
       }
-    }
-  }
-  if (a.list_only) return;
-
-  // per-lane statistics: one masked block reduction per lane that meets the tile
-  __shared__ int s_l0, s_l1;
-  if (tid == 0) { s_l0 = INT_MAX; s_l1 = -1; }
-  __syncthreads();
-  int my_lo = INT_MAX, my_hi = -1;
-#pragma unroll
-  for (int j = 0; j < GP_ITEMS; j++)
-    if (dev[j]) { my_lo = min(my_lo, ln[j]); my_hi = max(my_hi, ln[j]); }
-  if (my_hi >= 0) { atomicMin(&s_l0, my_lo); atomicMax(&s_l1, my_hi); }
-  __syncthreads();
-  const int l0 = s_l0, l1 = s_l1;
-  for (int l = l0; l <= l1; l++) {
-    if (a.lane_domain[l] != 1) continue;  // uniform over the CTA
-    if (tid < TA_NBINS) s_hist[tid] = 0;
-    __syncthreads();
-    u64 sb = 0, si = 0, ng = 0, mg = 0;
-#pragma unroll
-    for (int j = 0; j < GP_ITEMS; j++) {
-      if (!dev[j] || ln[j] != l) continue;
-      sb += (u64)busy[j];
-      si += (u64)gap[j];
-      if (gap[j] > 0) { ng++; mg = max(mg, (u64)gap[j]); atomicAdd(&s_hist[log2_bin(gap[j])], 1u); }
-      if (last[j]) {
-        si += (u64)tail[j];
-        if (tail[j] > 0) { ng++; mg = max(mg, (u64)tail[j]); atomicAdd(&s_hist[log2_bin(tail[j])], 1u); }
-        a.lane_gaps[l].last_end = W1[j] - tail[j];
+      if (last) {
+        a.lane_gaps[l].last_end = w1 - tl;
         a.lane_gaps[l].n_events = (i64)a.lane_off[l + 1] - (i64)a.lane_off[l];
       }
       if (p0 + j == (int64_t)a.lane_off[l]) a.lane_gaps[l].first_start = s[j];
     }
-    sb = block_reduce(sb, false, tmp);
-    si = block_reduce(si, false, tmp);
-    ng = block_reduce(ng, false, tmp);
-    mg = block_reduce(mg, true, tmp);
-    if (tid == 0) {
-      if (sb) atomicAdd((u64 *)&a.lane_gaps[l].busy, sb);
-      if (si) atomicAdd((u64 *)&a.lane_gaps[l].idle, si);
-      if (ng) atomicAdd((u64 *)&a.lane_gaps[l].n_gaps, ng);
-      if (mg) atomicMax((i64 *)&a.lane_gaps[l].max_gap, (i64)mg);
-    }
-    if (tid < TA_NBINS && s_hist[tid]) {
-      atomicAdd(&a.lane_hist[(size_t)l * TA_NBINS + tid], s_hist[tid]);
-      atomicAdd(&a.win_hist[(size_t)a.lane_window[l] * TA_NBINS + tid], s_hist[tid]);
-    }
-    __syncthreads();
   }
+  if (a.list_only) return;
+  if (full) {
+    longlong2 *pg = reinterpret_cast<longlong2 *>(a.gap_before + p0);
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS / 2; j++) pg[j] = make_longlong2(gap[2 * j], gap[2 * j + 1]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS; j++)
+      if (p0 + j < a.n) a.gap_before[p0 + j] = gap[j];
+  }
+  // fold the register statistics of the tile's first two lanes
+  const int l1 = s_lane1;
+  for (int li = 0; li < 2; li++) {
+    const int l = l0 + li;
+    if (l0 < 0 || l > l1) break;
+    if (a.lane_domain[l] != 1) continue;  // uniform over the CTA
+    const bool mine = lm == l;
+    u64 r0 = warp_reduce(mine ? sb : 0, OpAdd());
+    u64 r1 = warp_reduce(mine ? si : 0, OpAdd());
+    u64 r2 = warp_reduce(mine ? ng : 0, OpAdd());
+    u64 r3 = warp_reduce(mine ? mg : 0, OpMax());
+    __syncthreads();
+    if ((tid & 31) == 0) { red[0][tid >> 5] = r0; red[1][tid >> 5] = r1; red[2][tid >> 5] = r2; red[3][tid >> 5] = r3; }
+    __syncthreads();
+    if (tid < 4) {
+      u64 t = 0;
+      for (int w = 0; w < GP_THREADS / 32; w++) t = tid == 3 ? max(t, red[3][w]) : t + red[tid][w];
+      if (t) {
+        ta_lane_gaps *gl = &a.lane_gaps[l];
+        if (tid == 0) atomicAdd((u64 *)&gl->busy, t);
+        else if (tid == 1) atomicAdd((u64 *)&gl->idle, t);
+        else if (tid == 2) atomicAdd((u64 *)&gl->n_gaps, t);
+        else atomicMax((i64 *)&gl->max_gap, (i64)t);
+      }
+    }
+    if (tid < TA_NBINS && s_hist[li][tid]) {
+      atomicAdd(&a.lane_hist[(size_t)l * TA_NBINS + tid], s_hist[li][tid]);
+      atomicAdd(&a.win_hist[(size_t)a.lane_window[l] * TA_NBINS + tid], s_hist[li][tid]);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(256) k_gap_list_gather(const ta_long_gap *src, const u32 *order,
+                                                         int64_t m, ta_long_gap *dst) {
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < m) dst[i] = src[order[i]];
+}
+
+static int bit_len_g(uint64_t v) {
+  int b = 0;
+  while (v) { b++; v >>= 1; }
+  return b;
 }
 
 ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
@@ -215,11 +282,10 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   cudaStream_t st = h->stream;
   if (L >= (1 << 22) - 1) return TA_ERR_TOO_LARGE;
   const int64_t tiles = (n + GP_TILE - 1) / GP_TILE;
-  int64_t cap = n / 8 > 65536 ? n / 8 : 65536;
+  int64_t cap = n / 16 > 65536 ? n / 16 : 65536;
   size_t bytes = Carver::pad((size_t)(n > 0 ? n : 1) * 8) + Carver::pad((size_t)(L + 1) * sizeof(ta_lane_gaps)) +
                  Carver::pad((size_t)(L + 1) * TA_NBINS * 4) + Carver::pad((size_t)W * TA_NBINS * 4) +
-                 Carver::pad((size_t)cap * sizeof(ta_long_gap)) + 2 * Carver::pad((size_t)(tiles + 1) * 8) +
-                 Carver::pad(64) + 512;
+                 Carver::pad((size_t)(tiles + 1) * 8) + Carver::pad(64) + 512;
   void *b = ta_dalloc(h, bytes);
   if (!b) return TA_ERR_OOM;
   Carver c(b);
@@ -229,11 +295,16 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   ta_lane_gaps *lane_gaps = c.take<ta_lane_gaps>(L + 1);
   u32 *lane_hist = c.take<u32>((size_t)(L + 1) * TA_NBINS);
   u32 *win_hist = c.take<u32>((size_t)W * TA_NBINS);
-  u64 *st_max = c.take<u64>(tiles + 1), *st_cnt = c.take<u64>(tiles + 1);
-  u64 *scal = c.take<u64>(8);  // [0] n_long, [1] tile counter
+  u64 *st_max = c.take<u64>(tiles + 1);
+  u64 *scal = c.take<u64>(8);  // [0] list cursor, [1] tile counter
   char *zero_end = c.base + c.off;
-  ta_long_gap *list = c.take<ta_long_gap>(cap);
   TA_CHECK_CUDA(h, cudaMemsetAsync(zero_begin, 0, zero_end - zero_begin, st));
+  // unordered list + keys (temporary)
+  void *lt = ta_dalloc(h, Carver::pad((size_t)cap * sizeof(ta_long_gap)) + Carver::pad((size_t)cap * 8) + 256);
+  if (!lt) return TA_ERR_OOM;
+  Carver cl(lt);
+  ta_long_gap *ulist = cl.take<ta_long_gap>(cap);
+  u64 *ukeys = cl.take<u64>(cap);
 
   GapArgs a;
   a.n = n; a.n_valid = h->n_valid; a.n_lanes = L;
@@ -242,8 +313,8 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   a.lane_domain = h->sorted.lane_domain; a.t0 = h->d_t0; a.t1 = h->d_t1;
   a.min_gap = min_gap; a.list_only = 0;
   a.gap_before = gap_before; a.lane_gaps = lane_gaps; a.lane_hist = lane_hist; a.win_hist = win_hist;
-  a.long_gaps = list; a.list_cap = cap; a.st_max = st_max; a.st_cnt = st_cnt;
-  a.counter = (u32 *)(scal + 1); a.status = h->d_status; a.n_long_out = scal;
+  a.list = ulist; a.list_key = ukeys; a.list_cap = cap; a.st_max = st_max;
+  a.counter = (u32 *)(scal + 1); a.status = h->d_status; a.n_long = scal;
   if (tiles > 0) k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   u64 n_long = 0;
@@ -253,21 +324,46 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
   if ((int64_t)n_long > cap) {
     // rare: a tiny min_gap made the list longer than the first guess; rebuild it
-    void *b2 = ta_dalloc(h, (size_t)n_long * sizeof(ta_long_gap));
-    if (!b2) return TA_ERR_OOM;
+    ta_dfree(h, lt);
+    cap = (int64_t)n_long;
+    lt = ta_dalloc(h, Carver::pad((size_t)cap * sizeof(ta_long_gap)) + Carver::pad((size_t)cap * 8) + 256);
+    if (!lt) return TA_ERR_OOM;
+    Carver cl2(lt);
+    ulist = cl2.take<ta_long_gap>(cap);
+    ukeys = cl2.take<u64>(cap);
     TA_CHECK_CUDA(h, cudaMemsetAsync(st_max, 0, (char *)zero_end - (char *)st_max, st));
-    a.long_gaps = (ta_long_gap *)b2; a.list_cap = (i64)n_long; a.list_only = 1;
+    a.list = ulist; a.list_key = ukeys; a.list_cap = cap; a.list_only = 1;
     k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_TRY(ta_read_status(h, words));
     if (words[ST_ERR]) return (ta_status)words[ST_ERR];
-    list = (ta_long_gap *)b2;
   }
+  // order the list by (lane, position; tail last)
+  ta_long_gap *list = nullptr;
+  const int64_t m = (int64_t)n_long;
+  if (m > 0) {
+    list = (ta_long_gap *)ta_dalloc(h, (size_t)m * sizeof(ta_long_gap));
+    if (!list) return TA_ERR_OOM;
+    void *stb = ta_dalloc(h, 2 * Carver::pad((size_t)m * 8) + 2 * Carver::pad((size_t)m * 4) +
+                                 ta_sort_temp_bytes(m) + 256);
+    if (!stb) return TA_ERR_OOM;
+    Carver cs(stb);
+    u64 *ks = cs.take<u64>(m), *kf = cs.take<u64>(m);
+    u32 *vs = cs.take<u32>(m), *order = cs.take<u32>(m);
+    TA_TRY(ta_radix_sort_pairs(h, ukeys, nullptr, ks, vs, kf, order, m,
+                               ta_make_plan(0, 32 + bit_len_g((uint64_t)(L > 1 ? L - 1 : 1))), nullptr,
+                               cs.base + cs.off));
+    k_gap_list_gather<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(ulist, order, m, list);
+    TA_CHECK_CUDA(h, cudaGetLastError());
+    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    ta_dfree(h, stb);
+  }
+  ta_dfree(h, lt);
   out->gap_before = gap_before;
   out->lane_gaps = lane_gaps;
   out->lane_hist = lane_hist;
   out->win_hist = win_hist;
   out->long_gaps = list;
-  out->n_long_gaps = (int64_t)n_long;
+  out->n_long_gaps = m;
   return TA_OK;
 }
