@@ -19,7 +19,9 @@
 #include "ta_internal.cuh"
 
 #define AG_THREADS 256
-#define AG_SLOTS 512
+#define AG_ITEMS 4
+#define AG_STEP (AG_THREADS * AG_ITEMS)
+#define AG_SLOTS 256
 #define AG_FLUSH_EVERY 32768  // records per CTA between flushes (keeps 16-bit bins safe)
 
 struct AggArgs {
@@ -34,7 +36,7 @@ struct AggArgs {
   uint32_t kind_mask;
   int value_sel;
   int64_t min_name, R;
-  int64_t chunk;  // positions per CTA
+  int64_t chunk;  // positions per CTA, a multiple of AG_STEP
   // dense table (all zero-initialised; min is kept as the complement of the biased value)
   u64 *d_cnt, *d_sum, *d_minc, *d_maxb;
   u32 *d_hist;
@@ -59,86 +61,110 @@ __device__ __forceinline__ void agg_global_add(const AggArgs &a, int64_t g, u64 
   atomicMax(&a.d_maxb[g], maxb);
 }
 
+__device__ __forceinline__ void agg_clear(AggSmem &s) {
+  for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
+    s.key[i] = -1;
+    s.cnt[i] = 0;
+    s.sum[i] = 0;
+    s.minc[i] = 0;
+    s.maxb[i] = 0;
+  }
+  u32 *hw = reinterpret_cast<u32 *>(&s.hist[0][0]);
+  for (int i = threadIdx.x; i < AG_SLOTS * TA_NBINS / 2; i += AG_THREADS) hw[i] = 0;
+}
+
 __device__ __forceinline__ void agg_flush(const AggArgs &a, AggSmem &s) {
   __syncthreads();
   for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
     int32_t k = s.key[i];
-    if (k >= 0) {
-      agg_global_add(a, k, s.cnt[i], s.sum[i], s.minc[i], s.maxb[i]);
-      for (int b = 0; b < TA_NBINS; b++)
-        if (s.hist[i][b]) atomicAdd(&a.d_hist[(size_t)k * TA_NBINS + b], (u32)s.hist[i][b]);
-    }
-    s.key[i] = -1;
-    s.cnt[i] = 0;
-    s.sum[i] = 0;
-    s.minc[i] = 0;
-    s.maxb[i] = 0;
-    for (int b = 0; b < TA_NBINS; b++) s.hist[i][b] = 0;
+    if (k >= 0) agg_global_add(a, k, s.cnt[i], s.sum[i], s.minc[i], s.maxb[i]);
   }
+  // histogram bins: one thread per (slot, bin)
+  for (int i = threadIdx.x; i < AG_SLOTS * TA_NBINS; i += AG_THREADS) {
+    const int sl = i / TA_NBINS, b = i - sl * TA_NBINS;
+    const u32 c = s.hist[sl][b];
+    if (c) atomicAdd(&a.d_hist[(size_t)s.key[sl] * TA_NBINS + b], c);
+  }
+  __syncthreads();
+  agg_clear(s);
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(AG_THREADS) k_agg(AggArgs a) {
-  extern __shared__ __align__(16) unsigned char raw[];
-  AggSmem &s = *reinterpret_cast<AggSmem *>(raw);
-  for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
-    s.key[i] = -1;
-    s.cnt[i] = 0;
-    s.sum[i] = 0;
-    s.minc[i] = 0;
-    s.maxb[i] = 0;
-    for (int b = 0; b < TA_NBINS; b++) s.hist[i][b] = 0;
-  }
+__global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
+  __shared__ AggSmem s;
+  agg_clear(s);
   __syncthreads();
   const int64_t begin = (int64_t)blockIdx.x * a.chunk;
   const int64_t end = min(begin + a.chunk, a.n_valid);
   int since_flush = 0;
-  LaneWalker lw(a.lane_off, a.n_lanes, begin + threadIdx.x, a.n_valid);
-  for (int64_t base = begin; base < end; base += AG_THREADS) {
-    const int64_t p = base + threadIdx.x;
-    if (p < end) {
-      const int k = a.kind[p];
-      if ((1u << k) & a.kind_mask) {
-        bool sel = true;
-        i64 v;
-        if (a.value_sel == 0) v = a.te[p] - a.ts[p];
-        else {
-          sel = a.op_n[p] > 0;
-          v = sel ? a.op_last[p] - a.op_first[p] : 0;
+  LaneWalker lw(a.lane_off, a.n_lanes, begin + (int64_t)threadIdx.x * AG_ITEMS, a.n_valid);
+  for (int64_t base = begin; base < end; base += AG_STEP) {
+    const int64_t p0 = base + (int64_t)threadIdx.x * AG_ITEMS;
+    // all loads of the thread's four records are issued before any of them is used
+    int16_t kd[AG_ITEMS];
+    if (p0 + AG_ITEMS <= end) {
+      uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
+      const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++) kd[j] = hq[j];
+    } else {
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++) kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
+    }
+    bool sel[AG_ITEMS];
+    i64 v[AG_ITEMS];
+    int32_t nm[AG_ITEMS];
+#pragma unroll
+    for (int j = 0; j < AG_ITEMS; j++) {
+      sel[j] = kd[j] >= 0 && ((a.kind_mask >> kd[j]) & 1u);
+      v[j] = 0;
+      nm[j] = 0;
+    }
+    if (a.value_sel == 0) {
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++)
+        if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
+    } else {
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++)
+        if (sel[j]) sel[j] = a.op_n[p0 + j] > 0;
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++)
+        if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
+    }
+#pragma unroll
+    for (int j = 0; j < AG_ITEMS; j++) {
+      if (!sel[j]) continue;
+      const int lane = lw.at(p0 + j);
+      const int64_t g = (int64_t)a.lane_slot[lane] * a.R + ((int64_t)nm[j] - a.min_name);
+      const u64 vb = (u64)v[j] ^ (1ull << 63);
+      const int bin = log2_bin(v[j]);
+      u32 hsh = (u32)g * 2654435761u;
+      int slot = (int)(hsh >> 24) & (AG_SLOTS - 1);
+      bool placed = false;
+      for (int probe = 0; probe < 8; probe++) {
+        int32_t cur = s.key[slot];
+        if (cur == (int32_t)g) { placed = true; break; }
+        if (cur == -1) {
+          int32_t old = atomicCAS(&s.key[slot], -1, (int32_t)g);
+          if (old == -1 || old == (int32_t)g) { placed = true; break; }
         }
-        if (sel) {
-          const int lane = lw.at(p);
-          const int64_t g = (int64_t)a.lane_slot[lane] * a.R + ((int64_t)a.name[p] - a.min_name);
-          const u64 vb = (u64)v ^ (1ull << 63);
-          const int bin = log2_bin(v);
-          u32 hsh = (u32)g * 2654435761u;
-          int slot = (int)(hsh >> 23) & (AG_SLOTS - 1);
-          bool placed = false;
-          for (int probe = 0; probe < 8; probe++) {
-            int32_t cur = s.key[slot];
-            if (cur == (int32_t)g) { placed = true; break; }
-            if (cur == -1) {
-              int32_t old = atomicCAS(&s.key[slot], -1, (int32_t)g);
-              if (old == -1 || old == (int32_t)g) { placed = true; break; }
-            }
-            slot = (slot + 1) & (AG_SLOTS - 1);
-          }
-          if (placed) {
-            atomicAdd(&s.cnt[slot], 1u);
-            atomicAdd(&s.sum[slot], (u64)v);
-            atomicMax(&s.minc[slot], ~vb);
-            atomicMax(&s.maxb[slot], vb);
-            // 16-bit bins packed two per word
-            u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
-            atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
-          } else {
-            agg_global_add(a, g, 1, (u64)v, ~vb, vb);
-            atomicAdd(&a.d_hist[(size_t)g * TA_NBINS + bin], 1u);
-          }
-        }
+        slot = (slot + 1) & (AG_SLOTS - 1);
+      }
+      if (placed) {
+        atomicAdd(&s.cnt[slot], 1u);
+        atomicAdd(&s.sum[slot], (u64)v[j]);
+        atomicMax(&s.minc[slot], ~vb);
+        atomicMax(&s.maxb[slot], vb);
+        // 16-bit bins packed two per word
+        u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
+        atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
+      } else {
+        agg_global_add(a, g, 1, (u64)v[j], ~vb, vb);
+        atomicAdd(&a.d_hist[(size_t)g * TA_NBINS + bin], 1u);
       }
     }
-    since_flush += AG_THREADS;
+    since_flush += AG_STEP;
     if (since_flush >= AG_FLUSH_EVERY) {
       agg_flush(a, s);
       since_flush = 0;
@@ -206,15 +232,13 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot;
   a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
   a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
-  int64_t blocks = 148 * 3;
+  int64_t blocks = 148 * 6;
   int64_t chunk = (h->n_valid + blocks - 1) / blocks;
-  chunk = ((chunk + AG_THREADS - 1) / AG_THREADS) * AG_THREADS;
-  if (chunk < AG_THREADS) chunk = AG_THREADS;
+  chunk = ((chunk + AG_STEP - 1) / AG_STEP) * AG_STEP;
+  if (chunk < AG_STEP) chunk = AG_STEP;
   blocks = (h->n_valid + chunk - 1) / chunk;
   a.chunk = chunk;
-  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_agg, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(AggSmem)));
-  k_agg<<<TA_N (unsigned)blocks, AG_THREADS, sizeof(AggSmem), st>>>(a);
+  k_agg<<<TA_N (unsigned)blocks, AG_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   u64 ng = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
