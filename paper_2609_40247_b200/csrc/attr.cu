@@ -4,16 +4,19 @@
 //
 // In canonical order (ts_start ascending, ts_end descending) a properly nested
 // host lane has a simple structure: the innermost encloser of record i is the
-// nearest earlier OP that is still running when i starts.  That is answered
-//   - inside a tile of 2048 records (256 threads x 8 consecutive records) by a
-//     backward look over the thread's own records and, failing that, one descent
-//     of a max-tree over the threads' largest OP end times in shared memory;
-//   - across tiles by carrying the stack of still-open OPs (at most
-//     TA_MAX_DEPTH + 1 entries when nesting is legal) through a bounded
-//     decoupled look-back that one warp performs with one stack entry per lane.
-//     Combining a carried stack with a tile's stack is associative: entries that
-//     end no later than the tile's outermost surviving OP can never be chosen
-//     again and are dropped.
+// nearest earlier OP that is still running when i starts.  Tiles of 2048
+// records (256 threads x 8 consecutive records), three kernels, no kernel ever
+// waits for another CTA:
+//   k_attr_agg     per tile, the stack of OPs that are still undominated at the
+//                  tile's end (at most TA_MAX_DEPTH + 1 entries when nesting is
+//                  legal);
+//   k_attr_carry   one warp per host lane folds those stacks along the lane's
+//                  tiles (one stack entry per warp lane; entries that end no
+//                  later than a later tile's outermost surviving OP are dropped)
+//                  and leaves every tile the stack that is open at its start;
+//   k_attr_resolve per record: a backward look over the thread's own records,
+//                  else one descent of a max-tree over the threads' largest OP
+//                  end times in shared memory, else the carried stack.
 // Partial overlap is detected on the way: that nearest running OP must also
 // cover i's end.
 // HBM-bound: 18 B read per host record + 5 B written per record, plus the
@@ -35,6 +38,7 @@
 struct AttrArgs {
   int64_t n, n_valid;
   int n_lanes;
+  int64_t n_tiles;
   const int16_t *kind;
   const int64_t *ts, *te;
   const int32_t *lane_off, *lane_window;
@@ -42,29 +46,16 @@ struct AttrArgs {
   int32_t *parent;
   uint8_t *depth;
   ta_attr_summary *sum;
-  // tile descriptors
-  u64 *flag;
-  int32_t *agg_meta, *pre_meta;  // count | reset << 8
-  i64 *agg_e, *pre_e;            // [tile][AT_CAP]
-  int32_t *agg_pos, *pre_pos;
-  u32 *counter;
+  // per tile: stack at the tile's end (agg) and stack open at its start (carry)
+  int32_t *agg_meta, *carry_cnt;  // agg_meta = count | reset << 8
+  i64 *agg_e, *carry_e;           // [tile][AT_CAP]
+  int32_t *agg_pos, *carry_pos;
   int32_t *status;
-  // second kernel
+  // k_attr_ops
   const int32_t *launch_of;
   int32_t *op_of, *op_n;
   u64 *op_first, *op_last;
   int64_t *op_ns;
-};
-
-struct AttrSmem {
-  i64 leaf[AT_TILE];              // OP end time, INT64_MIN elsewhere
-  i64 T[2 * AT_THREADS];          // max-tree over the threads' maxima, leaves at [AT_THREADS, 2*AT_THREADS)
-  int16_t parent_local[AT_TILE];
-  uint8_t kcarry[AT_TILE];
-  i64 agg_e[AT_CAP], carry_e[AT_CAP];
-  int32_t agg_pos[AT_CAP], carry_pos[AT_CAP];
-  int agg_raw, carry_cnt;
-  int tile, lane0, lane1, dmax;
 };
 
 // A stack of open operators, one entry per lane of a warp (bottom = lane 0).
@@ -111,61 +102,216 @@ __device__ __forceinline__ int warp_lane_search_a(const int32_t *lane_off, int n
   return lo;
 }
 
-__device__ __forceinline__ void publish_stack(i64 *pe, int32_t *pp, int32_t *pmeta, u64 *flag, int tile,
-                                              const WStack &s, u64 kind) {
-  const int lane = threadIdx.x & 31;
-  if (lane < s.cnt) {
-    pe[(size_t)tile * AT_CAP + lane] = s.e;
-    pp[(size_t)tile * AT_CAP + lane] = s.pos;
-  }
-  if (lane == 0) pmeta[tile] = s.cnt | (s.reset << 8);
-  __threadfence();
-  __syncwarp();
-  if (lane == 0) st_relaxed(&flag[tile], td_pack(kind, 0));
-}
-
-__global__ void __launch_bounds__(AT_THREADS, 3) k_attr(AttrArgs a) {
-  __shared__ AttrSmem s;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) {
-    s.tile = (int)atomicAdd(a.counter, 1u);
-    s.lane1 = -1;
-    s.agg_raw = 0;
-    s.dmax = 0;
-    s.lane0 = -1;
-  }
-  __syncthreads();
-  const int tile = s.tile;
-  const int64_t tile_start = (int64_t)tile * AT_TILE;
-  const int x0 = tid * AT_ITEMS;
-  const int64_t p0 = tile_start + x0;
-  const bool full = p0 + AT_ITEMS <= a.n;
-  if (warp == 0 && tile_start < a.n_valid && a.n_lanes > 0) {
-    int l = warp_lane_search_a(a.lane_off, a.n_lanes, tile_start);
-    if (lane == 0) s.lane0 = l;
-  }
-  int16_t kd[AT_ITEMS];
-  if (full) {
-    uint4 q = *reinterpret_cast<const uint4 *>(a.kind + p0);
+__device__ __forceinline__ void load_kinds8(const int16_t *kind, int64_t p0, int64_t n, int16_t *kd) {
+  if (p0 + AT_ITEMS <= n) {
+    uint4 q = *reinterpret_cast<const uint4 *>(kind + p0);
     const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
 #pragma unroll
     for (int j = 0; j < AT_ITEMS; j++) kd[j] = hq[j];
   } else {
 #pragma unroll
-    for (int j = 0; j < AT_ITEMS; j++) kd[j] = p0 + j < a.n ? a.kind[p0 + j] : (int16_t)9;
+    for (int j = 0; j < AT_ITEMS; j++) kd[j] = p0 + j < n ? kind[p0 + j] : (int16_t)9;
   }
+}
+__device__ __forceinline__ void load_i64x8(const int64_t *col, int64_t p0, int64_t n, i64 *v) {
+  if (p0 + AT_ITEMS <= n) {
+    const longlong2 *ps = reinterpret_cast<const longlong2 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS / 2; j++) {
+      longlong2 x = ps[j];
+      v[2 * j] = x.x;
+      v[2 * j + 1] = x.y;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++) v[j] = p0 + j < n ? col[p0 + j] : 0;
+  }
+}
+
+// ---- kernel 1: the stack each tile leaves behind --------------------------------
+__global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
+  __shared__ i64 wmax[AT_THREADS / 32];
+  __shared__ i64 s_e[AT_CAP];
+  __shared__ int32_t s_pos[AT_CAP];
+  __shared__ int s_raw, s_lane1;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile = blockIdx.x;
+  const int64_t tile_start = (int64_t)tile * AT_TILE;
+  const int64_t p0 = tile_start + (int64_t)tid * AT_ITEMS;
+  const int64_t plast = min(tile_start + AT_TILE, a.n_valid) - 1;
+  if (tid == 0) s_raw = 0;
+  if (warp == 0) {
+    int l = -1;
+    if (plast >= tile_start) l = warp_lane_search_a(a.lane_off, a.n_lanes, plast);
+    if (lane == 0) s_lane1 = l;
+  }
+  int16_t kd[AT_ITEMS];
+  load_kinds8(a.kind, p0, a.n, kd);
+  __syncthreads();
+  const int lane1 = s_lane1;
+  if (lane1 < 0 || a.lane_domain[lane1] != 0) {
+    if (tid == 0) a.agg_meta[tile] = 1 << 8;  // nothing carried past a device lane
+    return;
+  }
+  const int64_t seg_begin = a.lane_off[lane1];  // first record of the tile's last lane
+  unsigned opmask = 0;
+#pragma unroll
+  for (int j = 0; j < AT_ITEMS; j++)
+    if (kd[j] == TA_KIND_OP && p0 + j <= plast && p0 + j >= seg_begin) opmask |= 1u << j;
+  i64 en[AT_ITEMS];
+#pragma unroll
+  for (int j = 0; j < AT_ITEMS; j++) en[j] = INT64_MIN;
+  i64 m8 = INT64_MIN;
+  if (opmask) {
+    i64 t[AT_ITEMS];
+    load_i64x8(a.te, p0, a.n, t);
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++)
+      if (opmask & (1u << j)) { en[j] = t[j]; m8 = m8 > t[j] ? m8 : t[j]; }
+  }
+  // largest OP end among the threads after this one
+  i64 after = INT64_MIN;
+  {
+    i64 v = m8;  // inclusive suffix max inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      i64 t = __shfl_down_sync(0xffffffffu, v, o);
+      if (lane + o < 32) v = v > t ? v : t;
+    }
+    if (lane == 0) wmax[warp] = v;
+    i64 nxt = __shfl_down_sync(0xffffffffu, v, 1);
+    after = lane < 31 ? nxt : INT64_MIN;
+    __syncthreads();
+    for (int w = warp + 1; w < AT_THREADS / 32; w++) after = after > wmax[w] ? after : wmax[w];
+  }
+  i64 sfx = after;
+#pragma unroll
+  for (int j = AT_ITEMS - 1; j >= 0; j--) {
+    if (opmask & (1u << j)) {
+      if (en[j] > sfx) {
+        int o = atomicAdd(&s_raw, 1);
+        if (o < AT_CAP) { s_e[o] = en[j]; s_pos[o] = (int32_t)(p0 + j); }
+      }
+      sfx = sfx > en[j] ? sfx : en[j];
+    }
+  }
+  __syncthreads();
+  if (warp == 0) {
+    const int raw = s_raw;
+    const int cnt = raw > AT_CAP ? AT_CAP : raw;
+    if (raw > AT_CAP && lane == 0) ta_set_err(a.status, TA_ERR_DEPTH);
+    // survivors were appended in arbitrary order: rank them by position
+    const i64 me = lane < cnt ? s_e[lane] : 0;
+    const int32_t mp = lane < cnt ? s_pos[lane] : INT_MAX;
+    int rank = 0;
+    for (int k = 0; k < cnt; k++) rank += __shfl_sync(0xffffffffu, mp, k) < mp ? 1 : 0;
+    if (lane < cnt) {
+      a.agg_e[(size_t)tile * AT_CAP + rank] = me;
+      a.agg_pos[(size_t)tile * AT_CAP + rank] = mp;
+    }
+    if (lane == 0) a.agg_meta[tile] = cnt | ((seg_begin >= tile_start ? 1 : 0) << 8);
+  }
+}
+
+// ---- kernel 2: one warp per host lane folds the tile stacks along the lane -----
+__global__ void __launch_bounds__(128) k_attr_carry(AttrArgs a) {
+  __shared__ i64 st_e[4][32][AT_CAP];
+  __shared__ int32_t st_pos[4][32][AT_CAP];
+  __shared__ int st_meta[4][32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int l = blockIdx.x * 4 + warp;
+  if (l >= a.n_lanes || a.lane_domain[l] != 0) return;
+  const int64_t b = a.lane_off[l], e = a.lane_off[l + 1];
+  if (e <= b) return;
+  const int64_t ta = b / AT_TILE, tb = (e - 1) / AT_TILE;
+  if (tb == ta) return;
+  bool overflow = false;
+  WStack acc;  // stack at the end of the tiles folded so far
+  {
+    const int m = a.agg_meta[ta];
+    acc.cnt = m & 0xFF;
+    acc.reset = 0;
+    acc.e = lane < acc.cnt ? a.agg_e[(size_t)ta * AT_CAP + lane] : 0;
+    acc.pos = lane < acc.cnt ? a.agg_pos[(size_t)ta * AT_CAP + lane] : 0;
+  }
+  for (int64_t t0 = ta + 1; t0 <= tb; t0 += 32) {
+    // stage up to 32 tile stacks: one tile per lane
+    const int64_t t = t0 + lane;
+    int m = 0;
+    if (t < tb) {  // the lane's last tile leaves nothing that is needed
+      m = a.agg_meta[t];
+      const int c = m & 0xFF;
+#pragma unroll
+      for (int k = 0; k < AT_CAP; k++)
+        if (k < c) {
+          st_e[warp][lane][k] = a.agg_e[(size_t)t * AT_CAP + k];
+          st_pos[warp][lane][k] = a.agg_pos[(size_t)t * AT_CAP + k];
+        }
+    }
+    st_meta[warp][lane] = m;
+    __syncwarp();
+    const int cntb = (int)min((int64_t)32, tb - t0 + 1);
+    for (int i = 0; i < cntb; i++) {
+      const int64_t ti = t0 + i;
+      if (lane < acc.cnt) {
+        a.carry_e[(size_t)ti * AT_CAP + lane] = acc.e;
+        a.carry_pos[(size_t)ti * AT_CAP + lane] = acc.pos;
+      }
+      if (lane == 0) a.carry_cnt[ti] = acc.cnt;
+      if (ti < tb) {
+        const int mi = st_meta[warp][i];
+        WStack nxt;
+        nxt.cnt = mi & 0xFF;
+        nxt.reset = 0;
+        nxt.e = lane < nxt.cnt ? st_e[warp][i][lane] : 0;
+        nxt.pos = lane < nxt.cnt ? st_pos[warp][i][lane] : 0;
+        wstack_combine(acc, nxt, &overflow);
+        acc = nxt;
+      }
+    }
+    __syncwarp();
+  }
+  if (overflow && lane == 0) ta_set_err(a.status, TA_ERR_DEPTH);
+}
+
+// ---- kernel 3: parent and depth of every host record -----------------------------
+struct AttrSmem {
+  i64 leaf[AT_TILE];              // OP end time, INT64_MIN elsewhere
+  i64 T[2 * AT_THREADS];          // max-tree over the threads' maxima, leaves at [AT_THREADS, 2*AT_THREADS)
+  int16_t parent_local[AT_TILE];
+  uint8_t kcarry[AT_TILE];
+  i64 carry_e[AT_CAP];
+  int32_t carry_pos[AT_CAP];
+  int lane0, lane1, dmax;
+};
+
+__global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
+  __shared__ AttrSmem s;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tile = blockIdx.x;
+  const int64_t tile_start = (int64_t)tile * AT_TILE;
+  const int x0 = tid * AT_ITEMS;
+  const int64_t p0 = tile_start + x0;
+  const bool full = p0 + AT_ITEMS <= a.n;
+  if (tid == 0) { s.lane1 = -1; s.dmax = 0; s.lane0 = -1; }
+  __syncthreads();
+  if (warp == 0 && tile_start < a.n_valid && a.n_lanes > 0) {
+    int l = warp_lane_search_a(a.lane_off, a.n_lanes, tile_start);
+    if (lane == 0) s.lane0 = l;
+  }
+  const int ccnt = a.carry_cnt[tile];
+  if (tid < ccnt) {
+    s.carry_e[tid] = a.carry_e[(size_t)tile * AT_CAP + tid];
+    s.carry_pos[tid] = a.carry_pos[(size_t)tile * AT_CAP + tid];
+  }
+  int16_t kd[AT_ITEMS];
+  load_kinds8(a.kind, p0, a.n, kd);
   unsigned hostmask = 0;
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++)
     if (p0 + j < a.n_valid && kd[j] <= TA_KIND_LAUNCH) hostmask |= 1u << j;
   const int any_host = __syncthreads_or(hostmask != 0);
   if (!any_host) {
-    // no host record here: the tile ends in a device lane (or beyond the kept records)
-    if (tid == 0) {
-      a.pre_meta[tile] = 1 << 8;
-      __threadfence();
-      st_relaxed(&a.flag[tile], td_pack(TD_PREFIX, 0));
-    }
     if (full) {
       *reinterpret_cast<int4 *>(a.parent + p0) = make_int4(-1, -1, -1, -1);
       *reinterpret_cast<int4 *>(a.parent + p0 + 4) = make_int4(-1, -1, -1, -1);
@@ -180,20 +326,8 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr(AttrArgs a) {
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) st[j] = en[j] = 0;
   if (hostmask) {
-    if (full) {
-      const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
-      const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
-#pragma unroll
-      for (int j = 0; j < AT_ITEMS / 2; j++) {
-        longlong2 x = ps[j], y = pe[j];
-        st[2 * j] = x.x; st[2 * j + 1] = x.y;
-        en[2 * j] = y.x; en[2 * j + 1] = y.y;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < AT_ITEMS; j++)
-        if (p0 + j < a.n) { st[j] = a.ts[p0 + j]; en[j] = a.te[p0 + j]; }
-    }
+    load_i64x8(a.ts, p0, a.n, st);
+    load_i64x8(a.te, p0, a.n, en);
   }
   // lanes, leaves, the thread's maximum
   const int l0 = s.lane0;
@@ -254,17 +388,16 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr(AttrArgs a) {
   }
   __syncthreads();
 
-  // nearest earlier OP of the tile that is still running when the record starts
+  // nearest earlier OP that is still running when the record starts
   unsigned bad = 0;
-  i64 thr[AT_ITEMS];
+  int32_t par_abs[AT_ITEMS];
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) {
     const int x = x0 + j;
     int pl = AT_NONE;
-    thr[j] = 0;
+    par_abs[j] = -1;
     if (hostmask & (1u << j)) {
       const i64 t = en[j] > st[j] ? st[j] + 1 : en[j];
-      thr[j] = t;
       int y = -1;
       for (int k = x - 1; k >= x0; k--)
         if (s.leaf[k] >= t) { y = k; break; }
@@ -285,121 +418,22 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr(AttrArgs a) {
       const int lo = lo_local[j];
       if (y >= 0 && y >= lo) {
         pl = y;
+        par_abs[j] = (int32_t)(tile_start + y);
         if (s.leaf[y] < en[j]) bad |= 1u << j;
-      } else {
-        pl = lo >= 0 ? AT_NONE : AT_UNRESOLVED;
+      } else if (lo >= 0) {
+        pl = AT_NONE;
+      } else {  // the encloser, if any, lies before the tile: the carried stack has it
+        pl = AT_UNRESOLVED;
+        int k = 0;
+        while (k < ccnt && s.carry_e[k] >= t) k++;
+        s.kcarry[x] = (uint8_t)k;
+        if (k > 0) {
+          par_abs[j] = s.carry_pos[k - 1];
+          if (s.carry_e[k - 1] < en[j]) bad |= 1u << j;
+        }
       }
     }
     s.parent_local[x] = (int16_t)pl;
-  }
-
-  // stack of the tile's last lane segment: OPs that no later OP of the tile dominates
-  const int lane_last = s.lane1;
-  const bool last_is_host = lane_last >= 0 && a.lane_domain[lane_last] == 0;
-  if (last_is_host) {
-    i64 sfx = INT64_MIN;
-    int l = tid + 1 + AT_THREADS, r = 2 * AT_THREADS;
-    while (l < r) {
-      if (l & 1) { sfx = sfx > s.T[l] ? sfx : s.T[l]; l++; }
-      if (r & 1) { --r; sfx = sfx > s.T[r] ? sfx : s.T[r]; }
-      l >>= 1;
-      r >>= 1;
-    }
-#pragma unroll
-    for (int j = AT_ITEMS - 1; j >= 0; j--) {
-      if ((hostmask & (1u << j)) && kd[j] == TA_KIND_OP) {
-        if (ln[j] == lane_last && en[j] > sfx) {
-          int o = atomicAdd(&s.agg_raw, 1);
-          if (o < AT_CAP) { s.agg_e[o] = en[j]; s.agg_pos[o] = (int32_t)(p0 + j); }
-        }
-        sfx = sfx > en[j] ? sfx : en[j];
-      }
-    }
-  }
-  __syncthreads();
-
-  if (warp == 0) {
-    bool overflow = s.agg_raw > AT_CAP;
-    WStack agg;
-    agg.cnt = overflow ? AT_CAP : s.agg_raw;
-    agg.reset = (!last_is_host || (int64_t)a.lane_off[lane_last] >= tile_start) ? 1 : 0;
-    // order the surviving OPs by position (they were appended in arbitrary order)
-    {
-      const i64 me = lane < agg.cnt ? s.agg_e[lane] : 0;
-      const int32_t mp = lane < agg.cnt ? s.agg_pos[lane] : INT_MAX;
-      int rank = 0;
-      for (int k = 0; k < agg.cnt; k++) rank += __shfl_sync(0xffffffffu, mp, k) < mp ? 1 : 0;
-      __syncwarp();
-      if (lane < agg.cnt) { s.agg_e[rank] = me; s.agg_pos[rank] = mp; }
-      __syncwarp();
-      agg.e = lane < agg.cnt ? s.agg_e[lane] : 0;
-      agg.pos = lane < agg.cnt ? s.agg_pos[lane] : 0;
-    }
-    bool need_carry = false;
-    if (tile > 0 && l0 >= 0) need_carry = a.lane_domain[l0] == 0 && (int64_t)a.lane_off[l0] < tile_start;
-    if (agg.reset) publish_stack(a.pre_e, a.pre_pos, a.pre_meta, a.flag, tile, agg, TD_PREFIX);
-    else publish_stack(a.agg_e, a.agg_pos, a.agg_meta, a.flag, tile, agg, TD_AGG);
-    WStack acc;
-    acc.cnt = 0; acc.reset = 0; acc.e = 0; acc.pos = 0;
-    if (need_carry) {
-      for (int t = tile - 1; t >= 0; --t) {
-        u64 w = 0;
-        int to = 0;
-        if (lane == 0) {
-          bool timed_out = false;
-          w = td_wait(&a.flag[t], a.status, &timed_out);
-          to = timed_out ? 1 : 0;
-        }
-        w = __shfl_sync(0xffffffffu, w, 0);
-        to = __shfl_sync(0xffffffffu, to, 0);
-        if (to) break;
-        __threadfence();
-        const bool is_prefix = (w >> 62) == TD_PREFIX;
-        const int32_t meta = ld_relaxed_i32(is_prefix ? &a.pre_meta[t] : &a.agg_meta[t]);
-        WStack ear;
-        ear.cnt = meta & 0xFF;
-        ear.reset = (meta >> 8) & 1;
-        ear.e = 0; ear.pos = 0;
-        if (lane < ear.cnt) {
-          const i64 *pe = (is_prefix ? a.pre_e : a.agg_e) + (size_t)t * AT_CAP;
-          const int32_t *pp = (is_prefix ? a.pre_pos : a.agg_pos) + (size_t)t * AT_CAP;
-          ear.e = (i64)ld_relaxed((const u64 *)&pe[lane]);
-          ear.pos = ld_relaxed_i32(&pp[lane]);
-        }
-        wstack_combine(ear, acc, &overflow);
-        if (is_prefix || ear.reset) break;
-      }
-    }
-    if (lane < acc.cnt) { s.carry_e[lane] = acc.e; s.carry_pos[lane] = acc.pos; }
-    if (lane == 0) s.carry_cnt = acc.cnt;
-    if (!agg.reset) {
-      WStack incl = agg;
-      wstack_combine(acc, incl, &overflow);
-      publish_stack(a.pre_e, a.pre_pos, a.pre_meta, a.flag, tile, incl, TD_PREFIX);
-    }
-    if (overflow && lane == 0) ta_set_err(a.status, TA_ERR_DEPTH);
-  }
-  __syncthreads();
-
-  // records whose encloser lies before the tile: look it up in the carried stack
-  int32_t par_abs[AT_ITEMS];
-  const int ccnt = s.carry_cnt;
-#pragma unroll
-  for (int j = 0; j < AT_ITEMS; j++) {
-    const int x = x0 + j;
-    par_abs[j] = -1;
-    if (!(hostmask & (1u << j))) continue;
-    const int pl = s.parent_local[x];
-    if (pl >= 0) par_abs[j] = (int32_t)(tile_start + pl);
-    else if (pl == AT_UNRESOLVED) {
-      int k = 0;
-      while (k < ccnt && s.carry_e[k] >= thr[j]) k++;
-      s.kcarry[x] = (uint8_t)k;
-      if (k > 0) {
-        par_abs[j] = s.carry_pos[k - 1];
-        if (s.carry_e[k - 1] < en[j]) bad |= 1u << j;
-      }
-    }
   }
   __syncthreads();
   int dmax = 0;
@@ -435,6 +469,7 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr(AttrArgs a) {
       if (p0 + j < a.n) { a.parent[p0 + j] = par_abs[j]; a.depth[p0 + j] = dep[j]; }
   }
   // per-window maximum depth (a tile rarely meets more than one window)
+  const int lane_last = s.lane1;
   const int w_first = l0 >= 0 ? a.lane_window[l0] : 0;
   const int w_last = lane_last >= 0 ? a.lane_window[lane_last] : w_first;
   if (w_first == w_last) {
@@ -528,6 +563,7 @@ __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
   }
 }
 
+
 ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   const int64_t n = h->n, nn = n > 0 ? n : 1;
   const int W = h->W;
@@ -549,25 +585,22 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   TA_CHECK_CUDA(h, cudaMemsetAsync(zero_begin, 0, zero_end - zero_begin, st));
 
   const int64_t tt = tiles > 0 ? tiles : 1;
-  size_t tb = Carver::pad(tt * 8) + 2 * Carver::pad(tt * 4) + 2 * Carver::pad(tt * AT_CAP * 8) +
-              2 * Carver::pad(tt * AT_CAP * 4) + Carver::pad(64) + 256;
+  size_t tb = 2 * Carver::pad(tt * 4) + 2 * Carver::pad(tt * AT_CAP * 8) + 2 * Carver::pad(tt * AT_CAP * 4) + 256;
   void *tmpb = ta_dalloc(h, tb);
   if (!tmpb) return TA_ERR_OOM;
   Carver ct(tmpb);
   AttrArgs a;
   memset(&a, 0, sizeof(a));
-  a.flag = ct.take<u64>(tt);
   a.agg_meta = ct.take<int32_t>(tt);
-  a.pre_meta = ct.take<int32_t>(tt);
-  a.counter = ct.take<u32>(16);
-  const size_t zero_bytes = ct.off;  // flags, metas and the counter start at zero; payloads need not
+  a.carry_cnt = ct.take<int32_t>(tt);
+  const size_t zero_bytes = ct.off;  // metas and carry counts start at zero; payloads need not
   a.agg_e = ct.take<i64>(tt * AT_CAP);
-  a.pre_e = ct.take<i64>(tt * AT_CAP);
+  a.carry_e = ct.take<i64>(tt * AT_CAP);
   a.agg_pos = ct.take<int32_t>(tt * AT_CAP);
-  a.pre_pos = ct.take<int32_t>(tt * AT_CAP);
+  a.carry_pos = ct.take<int32_t>(tt * AT_CAP);
   TA_CHECK_CUDA(h, cudaMemsetAsync(tmpb, 0, zero_bytes, st));
 
-  a.n = n; a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes;
+  a.n = n; a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes; a.n_tiles = tiles;
   a.kind = h->sorted.kind; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window;
   a.lane_domain = h->sorted.lane_domain;
@@ -575,7 +608,9 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   a.launch_of = h->join.launch_of; a.op_of = op_of; a.op_n = op_n; a.op_first = op_first;
   a.op_last = op_last; a.op_ns = op_ns;
   if (n > 0) {
-    k_attr<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
+    k_attr_agg<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
+    if (a.n_lanes > 0) k_attr_carry<<<TA_N (unsigned)((a.n_lanes + 3) / 4), 128, 0, st>>>(a);
+    k_attr_resolve<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
     k_attr_ops<<<TA_N (unsigned)((n + 2047) / 2048), 512, 0, st>>>(a);
     const int64_t fb = (h->n_valid + 255) / 256;
     k_attr_finalize<<<TA_N (unsigned)(fb > 0 ? fb : 1), 256, 0, st>>>(a);
