@@ -245,7 +245,7 @@ def main():
     barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
     launches = ta.launch_count() - launches0
-    n_pass, radix_ms = ta.profile_radix()
+    n_pass, radix_ms, radix_bytes = ta.profile_radix()
     ta.profile_enable(False)
     clocks = sampler.stop()
 
@@ -282,8 +282,8 @@ def main():
         value = total_events * args.steps / (elapsed_ms * 1e-3)
         roof = None
         if n_pass > 0 and radix_ms > 0:
-            per_launch_bytes = 24.0 * n  # 12 B read + 12 B written per (key, index) pair
-            ach = per_launch_bytes * n_pass / (radix_ms * 1e-3) / 1e9
+            per_launch_bytes = radix_bytes / n_pass  # 8 B read + 8 B written per packed key
+            ach = radix_bytes / (radix_ms * 1e-3) / 1e9
             roof = {"bound": "hbm", "kernel": "k_radix_pass", "achieved": ach, "peak": peak,
                     "peak_source": f"of {peak_kind}", "unit": "GB/s", "frac": ach / peak,
                     "launches_timed": n_pass, "avg_launch_ms": radix_ms / n_pass,

@@ -382,11 +382,13 @@ int32_t ta_version(void);
  * every radix-sort pass (the dominant kernel) on the launching stream, and
  * forget the pairs recorded so far; ta_profile_enable(0) stops recording.
  * ta_profile_radix: synchronises the recorded events and returns the number of
- * passes timed and the sum of their durations in milliseconds (0 on success,
- * -1 on a CUDA error). */
+ * passes timed, the sum of their durations in milliseconds and the algorithmic
+ * bytes they moved (16 B per record and pass when the sort key carries the
+ * record index, 24 B when (key, index) pairs are sorted); 0 on success, -1 on a
+ * CUDA error. */
 int64_t ta_launch_count(void);
 void ta_profile_enable(int32_t on);
-int32_t ta_profile_radix(int64_t *n_passes, double *total_ms);
+int32_t ta_profile_radix(int64_t *n_passes, double *total_ms, double *total_bytes);
 
 #ifdef __cplusplus
 }

@@ -215,6 +215,7 @@ struct LoadArgs {
   u64 *keys;
   u32 *hist;
   int sbits, tbits, wbits;
+  int packed, dshift, ibits;  // packed: key also carries the index inside the window (low ibits)
   SortPlan plan;
 };
 
@@ -223,33 +224,42 @@ __global__ void __launch_bounds__(256) k_load(LoadArgs a) {
   __shared__ u32 sh[10 * 256];
   for (int i = threadIdx.x; i < a.plan.n_pass * 256; i += blockDim.x) sh[i] = 0;
   __syncthreads();
-  const u64 dropped_key = 1ull << (a.sbits + a.tbits + a.wbits);
+  const int tsb = a.sbits - a.dshift;  // time bits kept in the key
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-  const int64_t n_round = ((a.n + 31) / 32) * 32;  // keep warps converged for match_any
+  const int64_t n_round = ((a.n + 31) / 32) * 32;  // keep warps converged for the votes
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += stride) {
     bool in = i < a.n;
     u64 key = 0;
     if (in) {
       Rec r = load_rec(a.ev, i);
       int w = window_of(a.off, a.W, i);
+      u64 hi;  // [dropped][window][triple rank][time]
       if (defect_of(r, a.t0[w], a.t1[w])) {
-        key = dropped_key;
+        hi = (1ull << (a.wbits + a.tbits + tsb)) | ((u64)w << (a.tbits + tsb));
+        if (!a.packed) hi = 1ull << (a.wbits + a.tbits + tsb);
       } else {
         u64 code = triple_code(r.pid, r.kind, r.stream);
         u32 slot = hash_code(code) & (TA_TRIPLE_SLOTS - 1);
         while (__ldg(&a.tt->slots[slot]) != code) slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
         u64 rank = (u64)__ldg(&a.tt->rank_of_slot[slot]);
-        key = ((u64)w << (a.tbits + a.sbits)) | (rank << a.sbits) | (u64)(r.ts_start - a.t0[w]);
+        hi = ((u64)w << (a.tbits + tsb)) | (rank << tsb) | ((u64)(r.ts_start - a.t0[w]) >> a.dshift);
       }
+      key = a.packed ? (hi << a.ibits) | (u64)(i - a.off[w]) : hi;
       a.keys[i] = key;
     }
     u32 active = __ballot_sync(0xffffffffu, in);
     if (!in) continue;
     const int lane = threadIdx.x & 31;
+    const int leader = __ffs(active) - 1;
     for (int p = 0; p < a.plan.n_pass; p++) {
+      // high digits are the same across a warp most of the time: one vote, one add
       u32 d = (u32)(key >> a.plan.shift[p]) & ((1u << a.plan.bits[p]) - 1u);
-      u32 m = __match_any_sync(active, d);
-      if (lane == __ffs(m) - 1) atomicAdd(&sh[p * 256 + d], (u32)__popc(m));
+      u32 d0 = __shfl_sync(active, d, leader);
+      if (__all_sync(active, d == d0)) {
+        if (lane == leader) atomicAdd(&sh[p * 256 + d0], (u32)__popc(active));
+      } else {
+        atomicAdd(&sh[p * 256 + d], 1u);
+      }
     }
   }
   __syncthreads();
@@ -284,22 +294,40 @@ ta_status ta_launch_discover(ta_window *h) {
   return TA_OK;
 }
 
-ta_status ta_launch_load(ta_window *h) {
-  // key layout: [dropped][window][triple rank][ts_start - t0]
-  int64_t max_span = 1;
-  for (int w = 0; w < h->W; w++) max_span = max_span > h->h_t1[w] - h->h_t0[w] ? max_span : h->h_t1[w] - h->h_t0[w];
+// Chooses the key layout and launches k_load.  allow_packed: try the layout that also
+// carries the record's index inside its window in the low bits, so that the sort
+// moves 8-byte keys only; it needs (window + triple + time + index) bits to fit 64
+// after giving up at most TA_PACK_MAX_DROP low time bits (records that collide in
+// the coarser time are put right by the equal-key fix-up).
+ta_status ta_launch_load(ta_window *h, bool allow_packed) {
+  // key layout: [dropped][window][triple rank][(ts_start - t0) >> dshift]{[index in window]}
+  int64_t max_span = 1, max_win = 1;
+  for (int w = 0; w < h->W; w++) {
+    max_span = max_span > h->h_t1[w] - h->h_t0[w] ? max_span : h->h_t1[w] - h->h_t0[w];
+    max_win = max_win > h->h_off[w + 1] - h->h_off[w] ? max_win : h->h_off[w + 1] - h->h_off[w];
+  }
   h->sbits = bit_length((uint64_t)(max_span - 1));
   h->tbits = bit_length((uint64_t)(h->n_triples > 0 ? h->n_triples - 1 : 0));
   h->wbits = bit_length((uint64_t)(h->W - 1));
-  int total = h->sbits + h->tbits + h->wbits + (h->has_dropped ? 1 : 0);
+  const int hd = h->has_dropped ? 1 : 0;
+  int total = h->sbits + h->tbits + h->wbits + hd;
   if (total > 63) return TA_ERR_TOO_LARGE;
   if (((int64_t)h->W << h->tbits) > (1ll << 24)) return TA_ERR_TOO_LARGE;
-  h->plan = ta_make_plan(0, total);
+  h->ibits = bit_length((uint64_t)(max_win - 1));
+  if (h->ibits < 1) h->ibits = 1;
+  int drop = total + h->ibits - 64;
+  if (drop < 0) drop = 0;
+  h->packed = allow_packed && drop <= TA_PACK_MAX_DROP && drop < h->sbits;
+  h->dshift = h->packed ? drop : 0;
+  if (h->packed) h->plan = ta_make_plan(h->ibits, h->ibits + total - h->dshift);
+  else h->plan = ta_make_plan(0, total);
   if (h->n == 0) return TA_OK;
+  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_hist, 0, 10 * 256 * 4, h->stream));
   LoadArgs a;
   a.ev = h->events; a.n = h->n; a.off = h->d_off; a.t0 = h->d_t0; a.t1 = h->d_t1; a.W = h->W;
   a.tt = h->d_triples; a.keys = h->d_keys; a.hist = h->d_hist;
   a.sbits = h->sbits; a.tbits = h->tbits; a.wbits = h->wbits; a.plan = h->plan;
+  a.packed = h->packed; a.dshift = h->dshift; a.ibits = h->ibits;
   k_load<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;

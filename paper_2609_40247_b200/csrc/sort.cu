@@ -1,19 +1,15 @@
-// Stable LSD radix sort of (64-bit key, 32-bit value) pairs: one scatter pass
-// per digit with a chained-scan ("one sweep") over tiles, so each pass reads and
-// writes every pair exactly once.  Digits are at most 8 bits wide; the digit
-// histograms of all passes are taken up front (by the load kernel for the
-// timeline sort, by k_radix_hist otherwise).
+// Stable LSD radix sort of 64-bit keys, with or without a 32-bit value: one
+// scatter pass per digit with a chained scan over tiles ("one sweep"), so each
+// pass reads and writes every element exactly once.  Digits are at most 8 bits
+// wide; the digit histograms of all passes are taken up front (by the load kernel
+// for the timeline sort, by k_radix_hist otherwise).
 //
-// Tile layout: RS_THREADS x RS_ITEMS pairs per CTA, keys staged through shared
+// Tile layout: THREADS x ITEMS elements per CTA, keys staged through shared
 // memory so that both the global loads (warp-striped) and the scattered stores
-// (runs of equal digits) are coalesced.  HBM-bound: 12 B read + 12 B written
-// per pair and pass.
+// (runs of equal digits) are coalesced.  HBM-bound: per element and pass 8 B read
+// + 8 B written (keys only) or 12 B + 12 B (pairs).
 #include "ta_internal.cuh"
 
-#define RS_THREADS 384
-#define RS_ITEMS 12
-#define RS_TILE (RS_THREADS * RS_ITEMS)
-#define RS_WARPS (RS_THREADS / 32)
 #define RS_BINS 256
 
 struct RadixArgs {
@@ -29,9 +25,10 @@ struct RadixArgs {
   int32_t *status;
 };
 
+template <int THREADS, int ITEMS>
 struct RadixSmem {
-  u64 keys[RS_TILE];  // aliased by u32 values after the keys are written out
-  u32 warp_hist[RS_WARPS][RS_BINS];
+  u64 keys[THREADS * ITEMS];  // aliased by u32 values after the keys are written out
+  u32 warp_hist[THREADS / 32][RS_BINS];
   u32 bin_start[RS_BINS];
   i64 adj[RS_BINS];
   u64 scan_tmp[33];
@@ -39,32 +36,35 @@ struct RadixSmem {
   int fail;
 };
 
-__global__ void __launch_bounds__(RS_THREADS) k_radix_pass(RadixArgs a) {
+template <int THREADS, int ITEMS, bool VALS>
+__global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
+  constexpr int TILE = THREADS * ITEMS;
+  constexpr int WARPS = THREADS / 32;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  RadixSmem &s = *reinterpret_cast<RadixSmem *>(smem_raw);
+  RadixSmem<THREADS, ITEMS> &s = *reinterpret_cast<RadixSmem<THREADS, ITEMS> *>(smem_raw);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     s.tile = (int)atomicAdd(a.tile_counter, 1u);
     s.fail = 0;
   }
-  for (int i = tid; i < RS_WARPS * RS_BINS; i += RS_THREADS) (&s.warp_hist[0][0])[i] = 0;
+  for (int i = tid; i < WARPS * RS_BINS; i += THREADS) (&s.warp_hist[0][0])[i] = 0;
   __syncthreads();
   const int tile = s.tile;
-  const int64_t base = (int64_t)tile * RS_TILE;
-  const int count = (int)min((int64_t)RS_TILE, a.n - base);
+  const int64_t base = (int64_t)tile * TILE;
+  const int count = (int)min((int64_t)TILE, a.n - base);
   const u32 mask = (1u << a.bits) - 1u;
 
-  u64 key[RS_ITEMS];
-  int lrank[RS_ITEMS];
-  const int wbase = warp * 32 * RS_ITEMS;
+  u64 key[ITEMS];
+  int lrank[ITEMS];
+  const int wbase = warp * 32 * ITEMS;
 #pragma unroll
-  for (int j = 0; j < RS_ITEMS; j++) {
+  for (int j = 0; j < ITEMS; j++) {
     int li = wbase + j * 32 + lane;
     key[j] = li < count ? a.keys_in[base + li] : ~0ull;
   }
   // rank inside the warp, item row by item row (stable: row-major, then lane)
 #pragma unroll
-  for (int j = 0; j < RS_ITEMS; j++) {
+  for (int j = 0; j < ITEMS; j++) {
     int li = wbase + j * 32 + lane;
     bool valid = li < count;
     u32 d = valid ? ((u32)(key[j] >> a.shift) & mask) : 0xFFFFFFFFu;
@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(RS_THREADS) k_radix_pass(RadixArgs a) {
   if (tid < RS_BINS) {
     u32 run = 0;
 #pragma unroll
-    for (int w = 0; w < RS_WARPS; w++) {
+    for (int w = 0; w < WARPS; w++) {
       u32 t = s.warp_hist[w][tid];
       s.warp_hist[w][tid] = run;
       run += t;
@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(RS_THREADS) k_radix_pass(RadixArgs a) {
   if (s.fail) return;
   // stage keys in shared memory in digit order
 #pragma unroll
-  for (int j = 0; j < RS_ITEMS; j++) {
+  for (int j = 0; j < ITEMS; j++) {
     int li = wbase + j * 32 + lane;
     if (li < count) {
       u32 d = (u32)(key[j] >> a.shift) & mask;
@@ -129,33 +129,40 @@ __global__ void __launch_bounds__(RS_THREADS) k_radix_pass(RadixArgs a) {
     }
   }
   __syncthreads();
-  u32 gpos[RS_ITEMS];
+  u32 gpos[VALS ? ITEMS : 1];
 #pragma unroll
-  for (int k = 0; k < RS_ITEMS; k++) {
-    int sl = tid + k * RS_THREADS;
-    gpos[k] = 0xFFFFFFFFu;
+  for (int k = 0; k < ITEMS; k++) {
+    int sl = tid + k * THREADS;
+    if (VALS) gpos[k] = 0xFFFFFFFFu;
     if (sl < count) {
       u64 kk = s.keys[sl];
       u32 d = (u32)(kk >> a.shift) & mask;
       i64 p = s.adj[d] + sl;
-      gpos[k] = (u32)p;
+      if (VALS) gpos[k] = (u32)p;
       a.keys_out[p] = kk;
     }
   }
+  if (!VALS) return;
   __syncthreads();
   u32 *svals = reinterpret_cast<u32 *>(s.keys);
 #pragma unroll
-  for (int j = 0; j < RS_ITEMS; j++) {
+  for (int j = 0; j < ITEMS; j++) {
     int li = wbase + j * 32 + lane;
     if (li < count) svals[lrank[j]] = a.vals_in ? a.vals_in[base + li] : (u32)(base + li);
   }
   __syncthreads();
 #pragma unroll
-  for (int k = 0; k < RS_ITEMS; k++) {
-    int sl = tid + k * RS_THREADS;
-    if (sl < count) a.vals_out[gpos[k]] = svals[sl];
+  for (int k = 0; k < ITEMS; k++) {
+    int sl = tid + k * THREADS;
+    if (sl < count) a.vals_out[gpos[VALS ? k : 0]] = svals[sl];
   }
 }
+
+// tile shapes
+#define RSP_THREADS 384  // pairs
+#define RSP_ITEMS 12
+#define RSK_THREADS 384  // keys only
+#define RSK_ITEMS 16
 
 // digit histograms of every pass (used when the caller has none)
 __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, int64_t n, SortPlan plan,
@@ -198,30 +205,39 @@ SortPlan ta_make_plan(int lo_bit, int hi_bit) {
   return p;
 }
 
-static size_t n_tiles_of(int64_t n) { return (size_t)((n + RS_TILE - 1) / RS_TILE); }
+static size_t min_tile() {
+  size_t a = (size_t)RSP_THREADS * RSP_ITEMS, b = (size_t)RSK_THREADS * RSK_ITEMS;
+  return a < b ? a : b;
+}
 
 size_t ta_sort_temp_bytes(int64_t n) {
-  size_t tiles = n_tiles_of(n);
+  size_t tiles = (size_t)((n + (int64_t)min_tile() - 1) / (int64_t)min_tile());
   if (tiles == 0) tiles = 1;
   return Carver::pad(tiles * RS_BINS * sizeof(u64)) + Carver::pad(16 * sizeof(u32)) +
          2 * Carver::pad(10 * RS_BINS * sizeof(u32));
 }
 
-// Sorts n pairs by the key bits the plan covers.  Pass outputs alternate between
-// (keys_scratch, vals_scratch) and (keys_final, vals_final) such that the last
-// pass writes the final buffers; keys_in / vals_in are only read (vals_in null =
-// the value of pair i is i).  keys_in must not alias scratch or final.
+// Sorts n keys (vals: pairs) by the key bits the plan covers.  Pass outputs
+// alternate between the scratch and the final buffers such that the last pass
+// writes the final ones; keys_in / vals_in are only read (pairs with vals_in null:
+// the value of element i is i).  keys_in must not alias scratch or final.
 // `hist` = precomputed [pass][256] digit histograms, or null.
-ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_in,
-                              u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
-                              u32 *vals_final, int64_t n, const SortPlan &plan, const u32 *hist,
-                              void *temp) {
+template <bool VALS>
+static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in, u64 *keys_scratch,
+                            u32 *vals_scratch, u64 *keys_final, u32 *vals_final, int64_t n,
+                            const SortPlan &plan, const u32 *hist, void *temp) {
   if (n <= 0) return TA_OK;
-  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_radix_pass, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(RadixSmem)));
-  size_t tiles = n_tiles_of(n);
+  constexpr int THREADS = VALS ? RSP_THREADS : RSK_THREADS;
+  constexpr int ITEMS = VALS ? RSP_ITEMS : RSK_ITEMS;
+  constexpr int TILE = THREADS * ITEMS;
+  typedef RadixSmem<THREADS, ITEMS> Smem;
+  auto kern = k_radix_pass<THREADS, ITEMS, VALS>;
+  TA_CHECK_CUDA(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)sizeof(Smem)));
+  size_t tiles = (size_t)((n + TILE - 1) / TILE);
   Carver c(temp);
-  u64 *state = c.take<u64>(tiles * RS_BINS);
+  size_t max_tiles = (size_t)((n + (int64_t)min_tile() - 1) / (int64_t)min_tile());
+  u64 *state = c.take<u64>(max_tiles * RS_BINS);
   u32 *counter = c.take<u32>(16);
   u32 *bin_offset = c.take<u32>(10 * RS_BINS);
   u32 *own_hist = c.take<u32>(10 * RS_BINS);
@@ -247,12 +263,26 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
     a.bin_offset = bin_offset + p * RS_BINS;
     a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
-    if (timed) ta_profile_mark(st, 1);
-    k_radix_pass<<<TA_N (unsigned)tiles, RS_THREADS, sizeof(RadixSmem), st>>>(a);
-    if (timed) ta_profile_mark(st, 0);
+    if (timed) ta_profile_mark(st, 1, (VALS ? 24.0 : 16.0) * (double)n);
+    kern<<<TA_N (unsigned)tiles, THREADS, sizeof(Smem), st>>>(a);
+    if (timed) ta_profile_mark(st, 0, 0.0);
     kin = a.keys_out;
     vin = a.vals_out;
   }
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
+}
+
+ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_in,
+                              u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
+                              u32 *vals_final, int64_t n, const SortPlan &plan, const u32 *hist,
+                              void *temp) {
+  return radix_sort<true>(h, keys_in, vals_in, keys_scratch, vals_scratch, keys_final, vals_final, n,
+                          plan, hist, temp);
+}
+
+ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
+                             int64_t n, const SortPlan &plan, const u32 *hist, void *temp) {
+  return radix_sort<false>(h, keys_in, nullptr, keys_scratch, nullptr, keys_final, nullptr, n, plan,
+                           hist, temp);
 }

@@ -52,9 +52,10 @@ long long g_ta_launches = 0;
 int g_ta_profile = 0;
 static std::vector<cudaEvent_t> g_prof_events;  // begin, end, begin, end, ...
 static size_t g_prof_used = 0;
+static double g_prof_bytes = 0;  // algorithmic bytes of the timed passes
 
-void ta_profile_mark(cudaStream_t st, int begin) {
-  (void)begin;
+void ta_profile_mark(cudaStream_t st, int begin, double bytes) {
+  if (begin) g_prof_bytes += bytes;
   if (g_prof_used == g_prof_events.size()) {
     cudaEvent_t e;
     if (cudaEventCreate(&e) != cudaSuccess) return;
@@ -72,8 +73,9 @@ extern "C" {
 void ta_profile_enable(int32_t on) {
   g_ta_profile = on;
   g_prof_used = 0;
+  g_prof_bytes = 0;
 }
-int32_t ta_profile_radix(int64_t *n_passes, double *total_ms) {
+int32_t ta_profile_radix(int64_t *n_passes, double *total_ms, double *total_bytes) {
   int64_t n = 0;
   double ms = 0;
   for (size_t i = 0; i + 1 < g_prof_used; i += 2) {
@@ -85,6 +87,7 @@ int32_t ta_profile_radix(int64_t *n_passes, double *total_ms) {
   }
   if (n_passes) *n_passes = n;
   if (total_ms) *total_ms = ms;
+  if (total_bytes) *total_bytes = g_prof_bytes;
   return 0;
 }
 int64_t ta_launch_count(void) { return g_ta_launches; }
@@ -183,7 +186,7 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
     if (out_summary) out_summary[w] = s;
   }
   h->has_dropped = h->n_valid < n ? 1 : 0;
-  TA_TRY(ta_launch_load(h));
+  TA_TRY(ta_launch_load(h, true));
   h->stage |= 1;
   return TA_OK;
 }

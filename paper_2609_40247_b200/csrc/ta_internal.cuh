@@ -22,6 +22,7 @@ typedef unsigned int u32;
 #define TA_COMM_SLOTS 2048
 #define TA_SPIN_LIMIT (1 << 22)   // polls of a tile descriptor before giving up
 #define TA_TIE_RUN_MAX 48         // equal-key runs up to this length are fixed in place
+#define TA_PACK_MAX_DROP 8         // low time bits a packed key may give up
 #define TA_AGG_DENSE_LIMIT (1ll << 27)
 
 // device status word indices (h->d_status)
@@ -77,15 +78,14 @@ struct ta_window {
   int64_t n_valid;
   int n_triples, n_pids;
   int sbits, tbits, wbits, has_dropped;
+  int packed, dshift, ibits;   // packed keys: low ibits = index inside the window, dshift low time bits dropped
   int64_t min_name, max_name, max_dur;
   SortPlan plan;
 
   // sort products
   ta_sort_result sorted;
-  u64 *d_sorted_keys;        // (window, triple, ts_rel) of each sorted position
   int32_t *d_lane_code;      // per lane: window << tbits | triple rank
   int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
-  std::vector<int32_t> h_lane_off;
 
   // join / attribution products
   ta_join_result join;
@@ -131,11 +131,14 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
                               u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
                               u32 *vals_final, int64_t n, const SortPlan &plan,
                               const u32 *hist /*nullable*/, void *temp);
+ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
+                             int64_t n, const SortPlan &plan, const u32 *hist /*nullable*/,
+                             void *temp);
 SortPlan ta_make_plan(int lo_bit, int hi_bit);
 // load.cu
 ta_status ta_launch_discover(ta_window *h);
 ta_status ta_launch_rank_triples(ta_window *h);
-ta_status ta_launch_load(ta_window *h);
+ta_status ta_launch_load(ta_window *h, bool allow_packed);
 // timeline.cu
 ta_status ta_run_sort_timeline(ta_window *h);
 // join.cu
@@ -157,7 +160,7 @@ extern long long g_ta_launches;   // kernels launched by this library since load
 extern int g_ta_profile;          // 1 = record a CUDA event pair around each radix pass
 static inline unsigned ta_one() { ++g_ta_launches; return 1u; }
 #define TA_N ta_one() *           // used as kernel<<<TA_N grid, ...>>>: counts the launch
-void ta_profile_mark(cudaStream_t st, int begin);  // called around k_radix_pass when profiling
+void ta_profile_mark(cudaStream_t st, int begin, double bytes);  // called around k_radix_pass when profiling
 
 // =================================================================== device
 #ifdef __CUDACC__

@@ -80,10 +80,12 @@ __global__ void __launch_bounds__(256) k_tail_key(const ta_event *ev, const u32 
 // ---- step 4: gather records into sorted columns + lane heads ---------------
 struct GatherArgs {
   const ta_event *ev;
-  const u32 *perm;
+  u32 *perm;          // pairs: input; packed keys: written here for the kept records
   const u64 *keys;
   int64_t n, n_valid;
-  int sbits;
+  int sbits;          // key bits below the lane code (time bits kept [+ index bits])
+  int packed, ibits, wshift, wbits;
+  const int64_t *off;
   i64 *ts_start, *ts_end, *corr;
   int32_t *pid, *name, *seq;
   int16_t *stream, *kind;
@@ -93,7 +95,16 @@ struct GatherArgs {
 __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= a.n) return;
-  Rec r = load_rec(a.ev, a.perm[p]);
+  u32 idx;
+  if (a.packed && p < a.n_valid) {
+    const u64 k = a.keys[p];
+    const int w = a.wbits ? (int)((k >> a.wshift) & ((1ull << a.wbits) - 1)) : 0;
+    idx = (u32)(a.off[w] + (int64_t)(k & ((1ull << a.ibits) - 1)));
+    a.perm[p] = idx;
+  } else {
+    idx = a.perm[p];
+  }
+  Rec r = load_rec(a.ev, idx);
   a.ts_start[p] = r.ts_start;
   a.ts_end[p] = r.ts_end;
   a.corr[p] = r.corr;
@@ -151,6 +162,55 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
   }
 }
 
+// ---- packed keys: equal (lane, coarse time) runs, ordered by (ts_start, -ts_end, index) --
+struct PackInfo {
+  int ibits, wshift, wbits;
+  const int64_t *off;
+};
+__device__ __forceinline__ u32 packed_index(u64 k, const PackInfo &pi) {
+  const int w = pi.wbits ? (int)((k >> pi.wshift) & ((1ull << pi.wbits) - 1)) : 0;
+  return (u32)(pi.off[w] + (int64_t)(k & ((1ull << pi.ibits) - 1)));
+}
+__global__ void __launch_bounds__(256) k_fix_ties_packed(u64 *keys, int64_t n_valid, const ta_event *ev,
+                                                         PackInfo pi, int32_t *status) {
+  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= n_valid || p + 1 >= n_valid) return;
+  const u64 k = keys[p];
+  const u64 hk = k >> pi.ibits;
+  if ((keys[p + 1] >> pi.ibits) != hk) return;
+  if (p > 0 && (keys[p - 1] >> pi.ibits) == hk) return;
+  int len = 2;
+  while (p + len < n_valid && len <= TA_TIE_RUN_MAX && (keys[p + len] >> pi.ibits) == hk) len++;
+  if (len > TA_TIE_RUN_MAX) {
+    status[ST_LONG_RUN] = 1;
+    return;
+  }
+  u64 kk[TA_TIE_RUN_MAX];
+  i64 st[TA_TIE_RUN_MAX], en[TA_TIE_RUN_MAX];
+  for (int i = 0; i < len; i++) {
+    kk[i] = keys[p + i];
+    const i64 *r = reinterpret_cast<const i64 *>(ev) + (int64_t)packed_index(kk[i], pi) * 5;
+    st[i] = r[0];
+    en[i] = r[1];
+  }
+  for (int i = 1; i < len; i++) {  // stable insertion sort: ts_start ascending, ts_end descending
+    u64 xk = kk[i];
+    i64 xs = st[i], xe = en[i];
+    int j = i - 1;
+    while (j >= 0 && (st[j] > xs || (st[j] == xs && en[j] < xe))) {
+      kk[j + 1] = kk[j]; st[j + 1] = st[j]; en[j + 1] = en[j];
+      j--;
+    }
+    kk[j + 1] = xk; st[j + 1] = xs; en[j + 1] = xe;
+  }
+  for (int i = 0; i < len; i++) keys[p + i] = kk[i];
+}
+__global__ void __launch_bounds__(256) k_unpack_tail(const u64 *keys, int64_t n_valid, int64_t n,
+                                                     PackInfo pi, u32 *perm) {
+  int64_t p = n_valid + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p < n) perm[p] = packed_index(keys[p], pi);
+}
+
 static inline int nblk(int64_t n, int t) { return (int)((n + t - 1) / t); }
 
 ta_status ta_run_sort_timeline(ta_window *h) {
@@ -161,8 +221,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
 
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
-                2 * Carver::pad(n * 2) + Carver::pad(n * 8) /*sorted keys*/ +
-                4 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
+                2 * Carver::pad(n * 2) + 4 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
                 Carver::pad((lane_cap + 1) * 4) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
@@ -171,7 +230,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   i64 *c_ts = ck.take<i64>(n), *c_te = ck.take<i64>(n), *c_corr = ck.take<i64>(n);
   int32_t *c_pid = ck.take<int32_t>(n), *c_name = ck.take<int32_t>(n), *c_seq = ck.take<int32_t>(n);
   int16_t *c_stream = ck.take<int16_t>(n), *c_kind = ck.take<int16_t>(n);
-  u64 *skeys = ck.take<u64>(n);
   int32_t *lane_window = ck.take<int32_t>(lane_cap), *lane_pid = ck.take<int32_t>(lane_cap);
   int32_t *lane_code = ck.take<int32_t>(lane_cap), *lane_slot = ck.take<int32_t>(lane_cap);
   int16_t *lane_stream = ck.take<int16_t>(lane_cap), *lane_domain = ck.take<int16_t>(lane_cap);
@@ -179,52 +237,71 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *n_lanes_dev = ck.take<int32_t>(1);
 
   // temporaries (released at the end of the call)
-  size_t tmp_bytes = Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
+  size_t tmp_bytes = 2 * Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
                      Carver::pad(n_codes * 4) + 512;
   void *tb = ta_dalloc(h, tmp_bytes);
   if (!tb) return TA_ERR_OOM;
   Carver ct(tb);
-  u64 *kscr = ct.take<u64>(n);
+  u64 *kscr = ct.take<u64>(n), *skeys = ct.take<u64>(n);
   u32 *vscr = ct.take<u32>(n);
   int32_t *lane_start = ct.take<int32_t>(n_codes);
   void *sort_tmp = ct.base + ct.off;
 
   TA_CHECK_CUDA(h, cudaMemsetAsync(lane_start, 0xFF, n_codes * sizeof(int32_t), st));
   if (n > 0) {
-    // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
-    TA_TRY(ta_radix_sort_pairs(h, h->d_keys, nullptr, kscr, vscr, skeys, perm, n, h->plan,
-                               h->d_hist, sort_tmp));
-    // step 2: equal-key runs
-    if (h->n_valid > 1)
-      k_fix_ties<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
-                                                        h->d_status);
     int32_t words[ST_WORDS];
-    TA_TRY(ta_read_status(h, words));
-    if (words[ST_ERR]) return (ta_status)words[ST_ERR];
-    if (words[ST_LONG_RUN]) {
-      // redo with the duration as a least-significant key: first a stable sort by
-      // (max_dur - duration), then the timeline key on top of that order
-      void *xb = ta_dalloc(h, Carver::pad(n * 8) + Carver::pad(n * 4));
-      if (!xb) return TA_ERR_OOM;
-      Carver cx(xb);
-      u64 *dkeys = cx.take<u64>(n);
-      u32 *dorder = cx.take<u32>(n);
-      const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
-      k_duration_key<<<TA_N nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit, h->max_dur,
-                                                   dkeys);
-      int dbits = 1;
-      while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
-      SortPlan dplan = ta_make_plan(0, dbits);
-      TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
-                                 sort_tmp));
-      k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
-      TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
-                                 sort_tmp));
-      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-      ta_dfree(h, xb);
+    if (h->packed) {
+      // keys carry the index: 8-byte elements, fewer bytes per pass
+      PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
+      TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp));
+      if (h->n_valid > 1)
+        k_fix_ties_packed<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, h->events, pi,
+                                                                 h->d_status);
+      TA_TRY(ta_read_status(h, words));
+      if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+      if (words[ST_LONG_RUN]) {
+        // a long run of equal coarse keys: start over with (key, index) pairs at full resolution
+        TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status + ST_LONG_RUN, 0, sizeof(int32_t), st));
+        TA_TRY(ta_launch_load(h, false));
+      } else if (n > h->n_valid) {
+        k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm);
+      }
+    }
+    if (!h->packed) {
+      // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
+      TA_TRY(ta_radix_sort_pairs(h, h->d_keys, nullptr, kscr, vscr, skeys, perm, n, h->plan,
+                                 h->d_hist, sort_tmp));
+      // step 2: equal-key runs
+      if (h->n_valid > 1)
+        k_fix_ties<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
+                                                          h->d_status);
+      TA_TRY(ta_read_status(h, words));
+      if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+      if (words[ST_LONG_RUN]) {
+        // redo with the duration as a least-significant key: first a stable sort by
+        // (max_dur - duration), then the timeline key on top of that order
+        void *xb = ta_dalloc(h, Carver::pad(n * 8) + Carver::pad(n * 4));
+        if (!xb) return TA_ERR_OOM;
+        Carver cx(xb);
+        u64 *dkeys = cx.take<u64>(n);
+        u32 *dorder = cx.take<u32>(n);
+        const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
+        k_duration_key<<<TA_N nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit,
+                                                     h->max_dur, dkeys);
+        int dbits = 1;
+        while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
+        SortPlan dplan = ta_make_plan(0, dbits);
+        TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
+                                   sort_tmp));
+        k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
+        TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
+                                   sort_tmp));
+        TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+        ta_dfree(h, xb);
+      }
     }
     // step 3: dropped tail, chain of stable sorts over the full tuple (least
-    // significant field first)
+    // significant field first); perm[n_valid..n) holds the tail in input order
     const int64_t m = n - h->n_valid;
     if (m > 1) {
       void *xb = ta_dalloc(h, 2 * Carver::pad(m * 8) + Carver::pad(m * 4));
@@ -250,7 +327,9 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     // step 4
     GatherArgs g;
     g.ev = h->events; g.perm = perm; g.keys = skeys; g.n = n; g.n_valid = h->n_valid;
-    g.sbits = h->sbits;
+    g.packed = h->packed; g.ibits = h->ibits; g.wbits = h->wbits; g.off = h->d_off;
+    g.wshift = h->ibits + h->tbits + (h->sbits - h->dshift);
+    g.sbits = h->packed ? h->ibits + (h->sbits - h->dshift) : h->sbits;
     g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
     g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
     k_gather<<<TA_N nblk(n, 256), 256, 0, st>>>(g);
@@ -262,10 +341,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   TA_CHECK_CUDA(h, cudaGetLastError());
   int32_t n_lanes = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-  h->h_lane_off.assign((size_t)n_lanes + 1, 0);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_lane_off.data(), lane_off, ((size_t)n_lanes + 1) * 4,
-                                   cudaMemcpyDeviceToHost, st));
   TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
   ta_dfree(h, tb);
   ta_dfree(h, h->d_keys);
@@ -279,7 +354,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   r.pid = c_pid; r.name_id = c_name; r.seq = c_seq; r.stream = c_stream; r.kind = c_kind;
   r.lane_window = lane_window; r.lane_pid = lane_pid; r.lane_stream = lane_stream;
   r.lane_domain = lane_domain; r.lane_off = lane_off;
-  h->d_sorted_keys = skeys;
   h->d_lane_code = lane_code;
   h->d_lane_slot = lane_slot;
   return TA_OK;

@@ -134,7 +134,8 @@ def lib():
         L.ta_profile_enable.restype = None
         L.ta_profile_enable.argtypes = [ctypes.c_int32]
         L.ta_profile_radix.restype = ctypes.c_int32
-        L.ta_profile_radix.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double)]
+        L.ta_profile_radix.argtypes = [ctypes.POINTER(ctypes.c_int64), ctypes.POINTER(ctypes.c_double),
+                                       ctypes.POINTER(ctypes.c_double)]
         _lib = L
     return _lib
 
@@ -182,12 +183,13 @@ def profile_enable(on: bool) -> None:
 
 
 def profile_radix():
-    """(number of radix passes timed, their summed duration in ms)."""
+    """(number of radix passes timed, their summed duration in ms, algorithmic bytes moved)."""
     n = ctypes.c_int64()
     ms = ctypes.c_double()
-    if lib().ta_profile_radix(ctypes.byref(n), ctypes.byref(ms)) != 0:
+    nb = ctypes.c_double()
+    if lib().ta_profile_radix(ctypes.byref(n), ctypes.byref(ms), ctypes.byref(nb)) != 0:
         raise RuntimeError("ta_profile_radix: CUDA error")
-    return n.value, ms.value
+    return n.value, ms.value, nb.value
 
 
 class _DevView:
