@@ -318,6 +318,20 @@ ta_status ta_launch_load(ta_window *h, bool allow_packed) {
   int drop = total + h->ibits - 64;
   if (drop < 0) drop = 0;
   h->packed = allow_packed && drop <= TA_PACK_MAX_DROP && drop < h->sbits;
+  if (h->packed) {
+    // Coarser time saves whole passes as long as records of one lane rarely share a time
+    // bucket (the equal-key fix-up restores the exact order).  Allow a coarsening whose
+    // expected bucket occupancy stays below 1/4, assuming lanes up to 4x the average size.
+    const double per_lane = 4.0 * (double)(h->n_valid > 0 ? h->n_valid : 1) /
+                            ((double)h->W * (double)(h->n_triples > 0 ? h->n_triples : 1));
+    int best = drop, best_pass = (total - drop + 7) / 8;
+    for (int d = drop + 1; d <= TA_PACK_MAX_DROP && d < h->sbits; d++) {
+      if (per_lane * (double)(1ull << d) / (double)max_span > 0.25) break;
+      const int np = (total - d + 7) / 8;
+      if (np < best_pass) { best = d; best_pass = np; }
+    }
+    drop = best;
+  }
   h->dshift = h->packed ? drop : 0;
   if (h->packed) h->plan = ta_make_plan(h->ibits, h->ibits + total - h->dshift);
   else h->plan = ta_make_plan(0, total);

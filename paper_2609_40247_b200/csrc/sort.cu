@@ -68,16 +68,25 @@ __global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
     int li = wbase + j * 32 + lane;
     bool valid = li < count;
     u32 d = valid ? ((u32)(key[j] >> a.shift) & mask) : 0xFFFFFFFFu;
+#ifdef RS_USE_MATCH
     u32 m = __match_any_sync(0xffffffffu, d);
-    int leader = __ffs(m) - 1;
-    u32 pre = 0;
-    if (valid && lane == leader) {
-      pre = s.warp_hist[warp][d];
-      s.warp_hist[warp][d] = pre + __popc(m);
+#else
+    // lanes with the same digit: one ballot per digit bit (cheaper than match.any here)
+    u32 m = __ballot_sync(0xffffffffu, valid);
+    if (!valid) m = ~m;
+#pragma unroll
+    for (int b = 0; b < 8; b++) {
+      if (b < a.bits) {
+        const u32 bal = __ballot_sync(0xffffffffu, (d >> b) & 1u);
+        m &= ((d >> b) & 1u) ? bal : ~bal;
+      }
     }
+#endif
+    const int leader = __ffs(m) - 1;
+    u32 pre = 0;
+    if (valid && lane == leader) pre = atomicAdd(&s.warp_hist[warp][d], (u32)__popc(m));
     pre = __shfl_sync(0xffffffffu, pre, leader);
     lrank[j] = (int)(pre + __popc(m & ((1u << lane) - 1u)));
-    __syncwarp();
   }
   __syncthreads();
   // per digit: exclusive offsets of the warps, then the CTA's digit count
@@ -161,8 +170,12 @@ __global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
 // tile shapes
 #define RSP_THREADS 384  // pairs
 #define RSP_ITEMS 12
+#ifndef RSK_THREADS
 #define RSK_THREADS 384  // keys only
+#endif
+#ifndef RSK_ITEMS
 #define RSK_ITEMS 16
+#endif
 
 // digit histograms of every pass (used when the caller has none)
 __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, int64_t n, SortPlan plan,

@@ -22,7 +22,7 @@ typedef unsigned int u32;
 #define TA_COMM_SLOTS 2048
 #define TA_SPIN_LIMIT (1 << 22)   // polls of a tile descriptor before giving up
 #define TA_TIE_RUN_MAX 48         // equal-key runs up to this length are fixed in place
-#define TA_PACK_MAX_DROP 8         // low time bits a packed key may give up
+#define TA_PACK_MAX_DROP 12        // low time bits a packed key may give up
 #define TA_AGG_DENSE_LIMIT (1ll << 27)
 
 // device status word indices (h->d_status)

@@ -10,6 +10,8 @@
 //      stable sorts;
 //   4. whole 40-byte records are gathered once into eight sorted columns and
 //      lane boundaries are recorded.
+#include <climits>
+
 #include "records.cuh"
 #include "ta_internal.cuh"
 
@@ -185,10 +187,43 @@ __global__ void __launch_bounds__(256) k_fix_ties_packed(u64 *keys, int64_t n_va
     status[ST_LONG_RUN] = 1;
     return;
   }
+  if (len <= 4) {
+    // short runs (the common case) stay in registers: all loads first, then a tiny network
+    u64 kk[4];
+    i64 st[4], en[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) kk[i] = i < len ? keys[p + i] : 0;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+      st[i] = LLONG_MAX;  // padding sorts last and is never written back
+      en[i] = LLONG_MIN;
+      if (i < len) {
+        const i64 *r = reinterpret_cast<const i64 *>(ev) + (int64_t)packed_index(kk[i], pi) * 5;
+        st[i] = r[0];
+        en[i] = r[1];
+      }
+    }
+    // stable: bubble passes that only swap strictly out-of-order neighbours
+#pragma unroll
+    for (int pass = 0; pass < 3; pass++)
+#pragma unroll
+      for (int i = 0; i < 3 - pass; i++) {
+        const bool sw = st[i] > st[i + 1] || (st[i] == st[i + 1] && en[i] < en[i + 1]);
+        if (sw) {
+          u64 tk = kk[i]; kk[i] = kk[i + 1]; kk[i + 1] = tk;
+          i64 ts = st[i]; st[i] = st[i + 1]; st[i + 1] = ts;
+          i64 te = en[i]; en[i] = en[i + 1]; en[i + 1] = te;
+        }
+      }
+#pragma unroll
+    for (int i = 0; i < 4; i++)
+      if (i < len) keys[p + i] = kk[i];
+    return;
+  }
   u64 kk[TA_TIE_RUN_MAX];
   i64 st[TA_TIE_RUN_MAX], en[TA_TIE_RUN_MAX];
+  for (int i = 0; i < len; i++) kk[i] = keys[p + i];
   for (int i = 0; i < len; i++) {
-    kk[i] = keys[p + i];
     const i64 *r = reinterpret_cast<const i64 *>(ev) + (int64_t)packed_index(kk[i], pi) * 5;
     st[i] = r[0];
     en[i] = r[1];
