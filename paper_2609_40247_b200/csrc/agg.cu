@@ -46,7 +46,7 @@ struct AggArgs {
 struct AggSmem {
   int32_t key[AG_SLOTS];
   u32 cnt[AG_SLOTS];
-  u64 sum[AG_SLOTS];
+  u32 sum16[3][AG_SLOTS];  // the sum in 16-bit limbs: native 32-bit shared-memory atomics only
   u64 minc[AG_SLOTS];
   u64 maxb[AG_SLOTS];
   uint16_t hist[AG_SLOTS][TA_NBINS];
@@ -65,7 +65,7 @@ __device__ __forceinline__ void agg_clear(AggSmem &s) {
   for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
     s.key[i] = -1;
     s.cnt[i] = 0;
-    s.sum[i] = 0;
+    s.sum16[0][i] = s.sum16[1][i] = s.sum16[2][i] = 0;
     s.minc[i] = 0;
     s.maxb[i] = 0;
   }
@@ -77,7 +77,10 @@ __device__ __forceinline__ void agg_flush(const AggArgs &a, AggSmem &s) {
   __syncthreads();
   for (int i = threadIdx.x; i < AG_SLOTS; i += AG_THREADS) {
     int32_t k = s.key[i];
-    if (k >= 0) agg_global_add(a, k, s.cnt[i], s.sum[i], s.minc[i], s.maxb[i]);
+    if (k >= 0)
+      agg_global_add(a, k, s.cnt[i],
+                     (u64)s.sum16[0][i] + ((u64)s.sum16[1][i] << 16) + ((u64)s.sum16[2][i] << 32),
+                     s.minc[i], s.maxb[i]);
   }
   // histogram bins: one thread per (slot, bin)
   for (int i = threadIdx.x; i < AG_SLOTS * TA_NBINS; i += AG_THREADS) {
@@ -153,9 +156,16 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
       }
       if (placed) {
         atomicAdd(&s.cnt[slot], 1u);
-        atomicAdd(&s.sum[slot], (u64)v[j]);
-        atomicMax(&s.minc[slot], ~vb);
-        atomicMax(&s.maxb[slot], vb);
+        {  // values are durations (>= 0): 16 + 16 + 32 bit limbs, at most 32768 adds per flush
+          const u64 uv = (u64)v[j];
+          atomicAdd(&s.sum16[0][slot], (u32)(uv & 0xFFFF));
+          if (uv >> 16) atomicAdd(&s.sum16[1][slot], (u32)((uv >> 16) & 0xFFFF));
+          if (uv >> 32) atomicAdd(&s.sum16[2][slot], (u32)(uv >> 32));
+        }
+        // 64-bit min/max in shared memory are compare-and-swap loops: skip them unless the
+        // value would actually move the extreme (rare once a slot has seen a few records)
+        if (~vb > s.minc[slot]) atomicMax(&s.minc[slot], ~vb);
+        if (vb > s.maxb[slot]) atomicMax(&s.maxb[slot], vb);
         // 16-bit bins packed two per word
         u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
         atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
