@@ -148,82 +148,152 @@ __device__ __forceinline__ int32_t winner_of(const JoinArgs &a, int64_t p, int s
 }
 
 // ---- pass 2: probes ----------------------------------------------------------
+// 256 threads x 8 consecutive positions; every output column is written once.
+#define JP_THREADS 256
+#define JP_TILE (JP_THREADS * 8)
+
 template <bool DIRECT>
-__global__ void __launch_bounds__(JN_THREADS) k_join_probe(JoinArgs a) {
-  __shared__ u64 tmp[33];
-  __shared__ int s_lo, s_hi;
-  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
-  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
-  int ln[JN_ITEMS];
-  bool matched[JN_ITEMS];
-  i64 lat[JN_ITEMS], q[JN_ITEMS];
-  int my_lo = INT_MAX, my_hi = -1;
+__global__ void __launch_bounds__(JP_THREADS, 3) k_join_probe(JoinArgs a) {
+  __shared__ u64 red[7][JP_THREADS / 32];
+  __shared__ int s_lane0, s_lane1;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t tile_start = (int64_t)blockIdx.x * JP_TILE;
+  const int64_t p0 = tile_start + (int64_t)tid * 8;
+  if (tid == 0) { s_lane0 = -1; s_lane1 = -1; }
+  __syncthreads();
+  if (tid < 32 && tile_start < a.n_valid && a.n_lanes > 0) {
+    int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (lane == 0) s_lane0 = l;
+  }
+  int16_t kd[8];
+  load8_i16(a.kind, p0, a.n, 0, kd);
+  unsigned pm = 0;  // probes among the thread's records
 #pragma unroll
-  for (int j = 0; j < JN_ITEMS; j++) {
-    int64_t p = p0 + j;
-    ln[j] = -1;
-    matched[j] = false;
-    lat[j] = 0;
-    q[j] = 0;
-    if (p >= a.n) continue;
-    int32_t lo = -1;
-    if (p < a.n_valid) {
-      int k = a.kind[p];
-      if (k == TA_KIND_KERNEL || k == TA_KIND_MEMCPY) {
-        ln[j] = lw.at(p);
-        my_lo = min(my_lo, ln[j]);
-        my_hi = max(my_hi, ln[j]);
-        lo = winner_of<DIRECT>(a, p, a.lane_slot[ln[j]]);
-        if (lo >= 0) {
-          matched[j] = true;
-          i64 s = a.ts[p];
-          lat[j] = s - a.ts[lo];
-          i64 d = s - a.te[lo];
-          q[j] = d > 0 ? d : 0;
-          atomicAdd(&a.kol[lo], 1);
+  for (int j = 0; j < 8; j++)
+    if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
+  i64 c[8], s[8];
+#pragma unroll
+  for (int j = 0; j < 8; j++) c[j] = s[j] = 0;
+  if (pm) {
+    load8_i64(a.corr, p0, a.n, c);
+    load8_i64(a.ts, p0, a.n, s);
+  }
+  __syncthreads();
+  const int l0 = s_lane0;
+  int32_t lo[8];
+  int ln[8];
+  {
+    int l = l0;
+    int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+    int slot = l >= 0 ? a.lane_slot[l] : 0;
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      lo[j] = -1;
+      ln[j] = -1;
+      if (pm & (1u << j)) {
+        const int64_t p = p0 + j;
+        while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; slot = a.lane_slot[l]; }
+        ln[j] = l;
+        if (DIRECT) {
+          const i64 base = a.slot_base[slot];
+          if (base >= 0 && c[j] >= a.slot_min[slot] && c[j] <= a.slot_max[slot]) {
+            const u32 v = a.table[base + (c[j] - a.slot_min[slot])];
+            lo[j] = v == EMPTY_U32 ? -1 : (int32_t)v;
+          }
+        } else {
+          lo[j] = a.found[p];
         }
       }
     }
-    a.launch_of[p] = lo;
-    a.latency[p] = lat[j];
-    a.qdelay[p] = q[j];
+    const int64_t plast = min(tile_start + JP_TILE, a.n_valid) - 1;
+    if (plast >= p0 && plast < p0 + 8) {
+      while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      s_lane1 = l;
+    }
   }
-  int l0, l1;
-  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
-  for (int l = l0; l <= l1; l++) {
-    if (a.lane_domain[l] != 1) continue;
-    u64 np = 0, nm = 0, sl = 0, sq = 0, mxl = 0, mnl_inv = 0, mxq = 0;
+  // launch times of the matched probes (independent gathers, issued together)
+  i64 ls[8], le[8];
 #pragma unroll
-    for (int j = 0; j < JN_ITEMS; j++)
-      if (ln[j] == l) {
-        np++;
-        if (matched[j]) {
-          nm++;
-          sl += (u64)lat[j];
-          sq += (u64)q[j];
-          mxl = max(mxl, bias64(lat[j]));
-          mnl_inv = max(mnl_inv, ~bias64(lat[j]));
-          mxq = max(mxq, (u64)q[j]);
-        }
+  for (int j = 0; j < 8; j++) {
+    ls[j] = le[j] = 0;
+    if (lo[j] >= 0) { ls[j] = a.ts[lo[j]]; le[j] = a.te[lo[j]]; }
+  }
+  i64 lat[8], q[8];
+  u64 np = 0, nm = 0, sl = 0, sq = 0, mxl = 0, mnl_inv = 0, mxq = 0;
+  int lm = -1;
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    lat[j] = q[j] = 0;
+    if (!(pm & (1u << j))) continue;
+    const bool matched = lo[j] >= 0;
+    if (matched) {
+      lat[j] = s[j] - ls[j];
+      const i64 d = s[j] - le[j];
+      q[j] = d > 0 ? d : 0;
+      atomicAdd(&a.kol[lo[j]], 1);
+    }
+    if (lm < 0) lm = ln[j];
+    if (ln[j] == lm && ln[j] - l0 <= 1) {
+      np++;
+      if (matched) {
+        nm++;
+        sl += (u64)lat[j];
+        sq += (u64)q[j];
+        mxl = max(mxl, bias64(lat[j]));
+        mnl_inv = max(mnl_inv, ~bias64(lat[j]));
+        mxq = max(mxq, (u64)q[j]);
       }
-    np = blk_reduce(np, false, tmp);
-    if (np == 0) continue;
-    nm = blk_reduce(nm, false, tmp);
-    sl = blk_reduce(sl, false, tmp);
-    sq = blk_reduce(sq, false, tmp);
-    mxl = blk_reduce(mxl, true, tmp);
-    mnl_inv = blk_reduce(mnl_inv, true, tmp);
-    mxq = blk_reduce(mxq, true, tmp);
-    if (threadIdx.x == 0) {
-      ta_join_summary *s = &a.sum[a.lane_window[l]];
-      atomicAdd((u64 *)&s->n_probe, np);
-      if (nm) {
-        atomicAdd((u64 *)&s->n_matched, nm);
-        atomicAdd((u64 *)&s->sum_latency, sl);
-        atomicAdd((u64 *)&s->sum_queue, sq);
-        atomicMax((i64 *)&s->max_latency, unbias64(mxl));
-        atomicMin((i64 *)&s->min_latency, unbias64(~mnl_inv));
-        atomicMax((i64 *)&s->max_queue, (i64)mxq);
+    } else {  // a thread that straddles a lane boundary, or a third lane in the tile
+      ta_join_summary *sm = &a.sum[a.lane_window[ln[j]]];
+      atomicAdd((u64 *)&sm->n_probe, 1ull);
+      if (matched) {
+        atomicAdd((u64 *)&sm->n_matched, 1ull);
+        atomicAdd((u64 *)&sm->sum_latency, (u64)lat[j]);
+        atomicAdd((u64 *)&sm->sum_queue, (u64)q[j]);
+        atomicMax((i64 *)&sm->max_latency, lat[j]);
+        atomicMin((i64 *)&sm->min_latency, lat[j]);
+        atomicMax((i64 *)&sm->max_queue, q[j]);
+      }
+    }
+  }
+  store8_i32(a.launch_of, p0, a.n, lo);
+  store8_i64(a.latency, p0, a.n, lat);
+  store8_i64(a.qdelay, p0, a.n, q);
+  __syncthreads();
+  const int l1 = s_lane1;
+  for (int li = 0; li < 2; li++) {
+    const int l = l0 + li;
+    if (l0 < 0 || l > l1) break;
+    if (a.lane_domain[l] != 1) continue;  // uniform over the CTA
+    const bool mine = lm == l;
+    u64 r[7] = {mine ? np : 0, mine ? nm : 0, mine ? sl : 0, mine ? sq : 0,
+                mine ? mxl : 0, mine ? mnl_inv : 0, mine ? mxq : 0};
+#pragma unroll
+    for (int k = 0; k < 4; k++) r[k] = warp_reduce(r[k], OpAdd());
+#pragma unroll
+    for (int k = 4; k < 7; k++) r[k] = warp_reduce(r[k], OpMax());
+    __syncthreads();
+    if (lane == 0)
+#pragma unroll
+      for (int k = 0; k < 7; k++) red[k][tid >> 5] = r[k];
+    __syncthreads();
+    if (tid == 0) {
+      u64 t[7] = {0, 0, 0, 0, 0, 0, 0};
+      for (int w = 0; w < JP_THREADS / 32; w++) {
+        for (int k = 0; k < 4; k++) t[k] += red[k][w];
+        for (int k = 4; k < 7; k++) t[k] = max(t[k], red[k][w]);
+      }
+      if (t[0]) {
+        ta_join_summary *sm = &a.sum[a.lane_window[l]];
+        atomicAdd((u64 *)&sm->n_probe, t[0]);
+        if (t[1]) {
+          atomicAdd((u64 *)&sm->n_matched, t[1]);
+          atomicAdd((u64 *)&sm->sum_latency, t[2]);
+          atomicAdd((u64 *)&sm->sum_queue, t[3]);
+          atomicMax((i64 *)&sm->max_latency, unbias64(t[4]));
+          atomicMin((i64 *)&sm->min_latency, unbias64(~t[5]));
+          atomicMax((i64 *)&sm->max_queue, (i64)t[6]);
+        }
       }
     }
   }
@@ -231,45 +301,73 @@ __global__ void __launch_bounds__(JN_THREADS) k_join_probe(JoinArgs a) {
 
 // ---- pass 3: launch statistics (duplicates, orphans) ---------------------------
 template <bool DIRECT>
-__global__ void __launch_bounds__(JN_THREADS) k_join_launch_stats(JoinArgs a) {
-  __shared__ u64 tmp[33];
-  __shared__ int s_lo, s_hi;
-  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
-  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
-  int ln[JN_ITEMS];
-  bool dup[JN_ITEMS], orphan[JN_ITEMS];
-  int my_lo = INT_MAX, my_hi = -1;
+__global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
+  __shared__ u64 red[JP_THREADS / 32];
+  __shared__ int s_lane0, s_lane1;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t tile_start = (int64_t)blockIdx.x * JP_TILE;
+  const int64_t p0 = tile_start + (int64_t)tid * 8;
+  if (tid == 0) { s_lane0 = -1; s_lane1 = -1; }
+  __syncthreads();
+  if (tid < 32 && tile_start < a.n_valid && a.n_lanes > 0) {
+    int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (lane == 0) s_lane0 = l;
+  }
+  int16_t kd[8];
+  load8_i16(a.kind, p0, a.n, 0, kd);
+  unsigned lmask = 0;
 #pragma unroll
-  for (int j = 0; j < JN_ITEMS; j++) {
-    int64_t p = p0 + j;
-    ln[j] = -1;
-    dup[j] = orphan[j] = false;
-    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
-      ln[j] = lw.at(p);
-      my_lo = min(my_lo, ln[j]);
-      my_hi = max(my_hi, ln[j]);
-      int32_t w = winner_of<DIRECT>(a, p, a.lane_slot[ln[j]]);
-      dup[j] = (w != (int32_t)p);
-      orphan[j] = !dup[j] && a.kol[p] == 0;
+  for (int j = 0; j < 8; j++)
+    if (p0 + j < a.n_valid && kd[j] == TA_KIND_LAUNCH) lmask |= 1u << j;
+  __syncthreads();
+  const int l0 = s_lane0;
+  u64 packed = 0;  // n_launch | n_dup << 20 | n_orphan << 40 for the thread's first lane
+  int lm = -1;
+  {
+    int l = l0;
+    int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      if (!(lmask & (1u << j))) continue;
+      const int64_t p = p0 + j;
+      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      const int32_t w = winner_of<DIRECT>(a, p, a.lane_slot[l]);
+      const bool dup = w != (int32_t)p;
+      const bool orphan = !dup && a.kol[p] == 0;
+      if (lm < 0) lm = l;
+      if (l == lm && l - l0 <= 1) {
+        packed += 1ull + ((u64)dup << 20) + ((u64)orphan << 40);
+      } else {
+        ta_join_summary *sm = &a.sum[a.lane_window[l]];
+        atomicAdd((u64 *)&sm->n_launch, 1ull);
+        if (dup) atomicAdd((u64 *)&sm->n_dup_launch, 1ull);
+        if (orphan) atomicAdd((u64 *)&sm->n_orphan_launch, 1ull);
+      }
+    }
+    const int64_t plast = min(tile_start + JP_TILE, a.n_valid) - 1;
+    if (plast >= p0 && plast < p0 + 8) {
+      while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      s_lane1 = l;
     }
   }
-  int l0, l1;
-  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
-  for (int l = l0; l <= l1; l++) {
+  __syncthreads();
+  const int l1 = s_lane1;
+  for (int li = 0; li < 2; li++) {
+    const int l = l0 + li;
+    if (l0 < 0 || l > l1) break;
     if (a.lane_domain[l] != 0) continue;
-    u64 nl = 0, nd = 0, no = 0;
-#pragma unroll
-    for (int j = 0; j < JN_ITEMS; j++)
-      if (ln[j] == l) { nl++; nd += dup[j]; no += orphan[j]; }
-    nl = blk_reduce(nl, false, tmp);
-    if (nl == 0) continue;
-    nd = blk_reduce(nd, false, tmp);
-    no = blk_reduce(no, false, tmp);
-    if (threadIdx.x == 0) {
-      ta_join_summary *s = &a.sum[a.lane_window[l]];
-      atomicAdd((u64 *)&s->n_launch, nl);
-      if (nd) atomicAdd((u64 *)&s->n_dup_launch, nd);
-      if (no) atomicAdd((u64 *)&s->n_orphan_launch, no);
+    u64 v = warp_reduce(lm == l ? packed : 0, OpAdd());
+    __syncthreads();
+    if (lane == 0) red[tid >> 5] = v;
+    __syncthreads();
+    if (tid == 0) {
+      u64 t = 0;
+      for (int w = 0; w < JP_THREADS / 32; w++) t += red[w];
+      const u64 m = (1ull << 20) - 1;
+      ta_join_summary *sm = &a.sum[a.lane_window[l]];
+      if (t & m) atomicAdd((u64 *)&sm->n_launch, t & m);
+      if ((t >> 20) & m) atomicAdd((u64 *)&sm->n_dup_launch, (t >> 20) & m);
+      if ((t >> 40) & m) atomicAdd((u64 *)&sm->n_orphan_launch, (t >> 40) & m);
     }
   }
 }
@@ -364,6 +462,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   a.slot_min = slot_min; a.slot_max = slot_max; a.slot_base = slot_base;
   a.launch_of = launch_of; a.kol = kol; a.latency = latency; a.qdelay = qdelay; a.sum = d_sum;
   const unsigned grid = (unsigned)((n + JN_TILE - 1) / JN_TILE);
+  const unsigned grid8 = (unsigned)((n + JP_TILE - 1) / JP_TILE);
   void *tmp_alloc = nullptr;
   bool direct = true;
   if (n > 0) {
@@ -389,8 +488,8 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       TA_CHECK_CUDA(h, cudaMemsetAsync(a.table, 0xFF, (size_t)(M > 0 ? M : 1) * 4, st));
       TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_base, hbase.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
       k_join_build<<<TA_N grid, JN_THREADS, 0, st>>>(a);
-      k_join_probe<true><<<TA_N grid, JN_THREADS, 0, st>>>(a);
-      k_join_launch_stats<true><<<TA_N grid, JN_THREADS, 0, st>>>(a);
+      k_join_probe<true><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
+      k_join_launch_stats<true><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
     } else {
       // general path: compact, sort by (slot, corr) with sorted position as the stable tie-break
       size_t tb = Carver::pad(nn * 4) * 3 + Carver::pad(nn * 8) * 3 + scan_temp_bytes(n) * 2 +
@@ -432,8 +531,8 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
         TA_TRY((launch_scan<OpMax, JoinHeadIn, JoinHeadOut>(h, m, hin, hout, OpMax(), t2)));
       }
       a.found = found;
-      k_join_probe<false><<<TA_N grid, JN_THREADS, 0, st>>>(a);
-      k_join_launch_stats<false><<<TA_N grid, JN_THREADS, 0, st>>>(a);
+      k_join_probe<false><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
+      k_join_launch_stats<false><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
     }
     TA_CHECK_CUDA(h, cudaGetLastError());
   }

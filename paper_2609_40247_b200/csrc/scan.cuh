@@ -77,6 +77,71 @@ static inline ta_status launch_scan(ta_window *h, int64_t n, In in, Out out, Op 
   return TA_OK;
 }
 
+// ---- helpers for kernels that give every thread eight consecutive sorted positions ----
+// largest l with lane_off[l] <= p, found by the 32 lanes of one warp together
+__device__ __forceinline__ int tile_lane_search(const int32_t *lane_off, int n_lanes, int64_t p) {
+  const int lane = threadIdx.x & 31;
+  int lo = 0, hi = n_lanes;
+  while (hi - lo > 1) {
+    int step = (hi - lo + 31) >> 5;
+    int idx = lo + lane * step;
+    bool ok = idx < hi && (int64_t)lane_off[idx] <= p;
+    u32 m = __ballot_sync(0xffffffffu, ok);
+    int k = 31 - __clz((int)m);  // lane 0 always qualifies
+    lo = lo + k * step;
+    hi = min(hi, lo + step);
+  }
+  return lo;
+}
+__device__ __forceinline__ void load8_i16(const int16_t *col, int64_t p0, int64_t n, int16_t fill,
+                                          int16_t *v) {
+  if (p0 + 8 <= n) {
+    uint4 q = *reinterpret_cast<const uint4 *>(col + p0);
+    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] = hq[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] = p0 + j < n ? col[p0 + j] : fill;
+  }
+}
+__device__ __forceinline__ void load8_i64(const int64_t *col, int64_t p0, int64_t n, i64 *v) {
+  if (p0 + 8 <= n) {
+    const longlong2 *ps = reinterpret_cast<const longlong2 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      longlong2 x = ps[j];
+      v[2 * j] = x.x;
+      v[2 * j + 1] = x.y;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++) v[j] = p0 + j < n ? col[p0 + j] : 0;
+  }
+}
+__device__ __forceinline__ void store8_i64(int64_t *col, int64_t p0, int64_t n, const i64 *v) {
+  if (p0 + 8 <= n) {
+    longlong2 *ps = reinterpret_cast<longlong2 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < 4; j++) ps[j] = make_longlong2(v[2 * j], v[2 * j + 1]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+      if (p0 + j < n) col[p0 + j] = v[j];
+  }
+}
+__device__ __forceinline__ void store8_i32(int32_t *col, int64_t p0, int64_t n, const int32_t *v) {
+  if (p0 + 8 <= n) {
+    int4 *ps = reinterpret_cast<int4 *>(col + p0);
+    ps[0] = make_int4(v[0], v[1], v[2], v[3]);
+    ps[1] = make_int4(v[4], v[5], v[6], v[7]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++)
+      if (p0 + j < n) col[p0 + j] = v[j];
+  }
+}
+
 // Walks the lane table along ascending sorted positions.
 struct LaneWalker {
   const int32_t *lane_off;
