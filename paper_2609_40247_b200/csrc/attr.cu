@@ -485,84 +485,122 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
 }
 
 // ---- device records inherit the operator of their launch ------------------------
-__global__ void __launch_bounds__(512) k_attr_ops(AttrArgs a) {
-  __shared__ u64 tmp[33];
-  __shared__ int s_lo, s_hi;
-  const int64_t p0 = ((int64_t)blockIdx.x * 512 + threadIdx.x) * 4;
-  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
-  int ln[4];
-  int cls[4];  // 0 none, 1 attributed, 2 no launch, 3 no op
-  int my_lo = INT_MAX, my_hi = -1;
+__global__ void __launch_bounds__(AT_THREADS, 3) k_attr_ops(AttrArgs a) {
+  __shared__ u64 red[AT_THREADS / 32];
+  __shared__ int s_lane0, s_lane1;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int64_t tile_start = (int64_t)blockIdx.x * AT_TILE;
+  const int64_t p0 = tile_start + (int64_t)tid * AT_ITEMS;
+  if (tid == 0) { s_lane0 = -1; s_lane1 = -1; }
+  __syncthreads();
+  if (tid < 32 && tile_start < a.n_valid && a.n_lanes > 0) {
+    int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (lane == 0) s_lane0 = l;
+  }
+  int16_t kd[AT_ITEMS];
+  load8_i16(a.kind, p0, a.n, 0, kd);
+  unsigned pm = 0;
 #pragma unroll
-  for (int j = 0; j < 4; j++) {
-    int64_t p = p0 + j;
-    ln[j] = -1;
-    cls[j] = 0;
-    if (p >= a.n) continue;
-    int32_t op = -1;
-    if (p < a.n_valid) {
-      int k = a.kind[p];
-      if (k == TA_KIND_KERNEL || k == TA_KIND_MEMCPY) {
-        ln[j] = lw.at(p);
-        my_lo = min(my_lo, ln[j]);
-        my_hi = max(my_hi, ln[j]);
-        int32_t l = a.launch_of[p];
-        if (l < 0) cls[j] = 2;
-        else {
-          op = a.parent[l];
-          if (op < 0) cls[j] = 3;
-          else {
-            cls[j] = 1;
-            i64 s = a.ts[p], e = a.te[p];
-            atomicAdd(&a.op_n[op], 1);
-            atomicAdd((u64 *)&a.op_ns[op], (u64)(e - s));
-            atomicMax(&a.op_first[op], ~((u64)s ^ (1ull << 63)));
-            atomicMax(&a.op_last[op], (u64)e ^ (1ull << 63));
-          }
-        }
+  for (int j = 0; j < AT_ITEMS; j++)
+    if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
+  int32_t lo[AT_ITEMS], op[AT_ITEMS];
+  i64 st[AT_ITEMS], en[AT_ITEMS];
+#pragma unroll
+  for (int j = 0; j < AT_ITEMS; j++) { lo[j] = -1; op[j] = -1; st[j] = en[j] = 0; }
+  if (pm) {
+    if (p0 + AT_ITEMS <= a.n) {
+      const int4 x = *reinterpret_cast<const int4 *>(a.launch_of + p0);
+      const int4 y = *reinterpret_cast<const int4 *>(a.launch_of + p0 + 4);
+      lo[0] = x.x; lo[1] = x.y; lo[2] = x.z; lo[3] = x.w;
+      lo[4] = y.x; lo[5] = y.y; lo[6] = y.z; lo[7] = y.w;
+    } else {
+#pragma unroll
+      for (int j = 0; j < AT_ITEMS; j++)
+        if (p0 + j < a.n) lo[j] = a.launch_of[p0 + j];
+    }
+    load8_i64(a.ts, p0, a.n, st);
+    load8_i64(a.te, p0, a.n, en);
+    // parents of the launches: independent gathers, issued together
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++)
+      if ((pm & (1u << j)) && lo[j] >= 0) op[j] = a.parent[lo[j]];
+  }
+  __syncthreads();
+  const int l0 = s_lane0;
+  u64 packed = 0;  // attributed | no launch << 20 | no op << 40, for the thread's first lane
+  int lm = -1;
+  {
+    int l = l0;
+    int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++) {
+      if (!(pm & (1u << j))) { op[j] = -1; continue; }
+      const int64_t p = p0 + j;
+      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      u64 add;
+      if (lo[j] < 0) add = 1ull << 20;
+      else if (op[j] < 0) add = 1ull << 40;
+      else {
+        add = 1ull;
+        const int32_t r = op[j];
+        atomicAdd(&a.op_n[r], 1);
+        atomicAdd((u64 *)&a.op_ns[r], (u64)(en[j] - st[j]));
+        atomicMax(&a.op_first[r], ~((u64)st[j] ^ (1ull << 63)));
+        atomicMax(&a.op_last[r], (u64)en[j] ^ (1ull << 63));
+      }
+      if (lm < 0) lm = l;
+      if (l == lm && l - l0 <= 1) packed += add;
+      else {
+        ta_attr_summary *sm = &a.sum[a.lane_window[l]];
+        if (add == 1ull) atomicAdd((u64 *)&sm->n_attributed, 1ull);
+        else if (add == (1ull << 20)) atomicAdd((u64 *)&sm->n_no_launch, 1ull);
+        else atomicAdd((u64 *)&sm->n_no_op, 1ull);
       }
     }
-    a.op_of[p] = op;
-  }
-  if (threadIdx.x == 0) { s_lo = INT_MAX; s_hi = -1; }
-  __syncthreads();
-  if (my_hi >= 0) { atomicMin(&s_lo, my_lo); atomicMax(&s_hi, my_hi); }
-  __syncthreads();
-  const int l0 = s_lo, l1 = s_hi;
-  for (int l = l0; l <= l1; l++) {
-    if (a.lane_domain[l] != 1) continue;
-    u64 c1 = 0, c2 = 0, c3 = 0;
-#pragma unroll
-    for (int j = 0; j < 4; j++)
-      if (ln[j] == l) { c1 += cls[j] == 1; c2 += cls[j] == 2; c3 += cls[j] == 3; }
-    u64 packed = c1 | (c2 << 20) | (c3 << 40);  // each < 2^20 per tile
-    u64 v = warp_reduce(packed, OpAdd());
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0) tmp[threadIdx.x >> 5] = v;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      u64 t = 0;
-      for (int w = 0; w < 16; w++) t += tmp[w];
-      ta_attr_summary *s = &a.sum[a.lane_window[l]];
-      u64 m = (1ull << 20) - 1;
-      if (t & m) atomicAdd((u64 *)&s->n_attributed, t & m);
-      if ((t >> 20) & m) atomicAdd((u64 *)&s->n_no_launch, (t >> 20) & m);
-      if ((t >> 40) & m) atomicAdd((u64 *)&s->n_no_op, (t >> 40) & m);
+    const int64_t plast = min(tile_start + AT_TILE, a.n_valid) - 1;
+    if (plast >= p0 && plast < p0 + AT_ITEMS) {
+      while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      s_lane1 = l;
     }
+  }
+  store8_i32(a.op_of, p0, a.n, op);
+  __syncthreads();
+  const int l1 = s_lane1;
+  for (int li = 0; li < 2; li++) {
+    const int l = l0 + li;
+    if (l0 < 0 || l > l1) break;
+    if (a.lane_domain[l] != 1) continue;
+    u64 v = warp_reduce(lm == l ? packed : 0, OpAdd());
     __syncthreads();
+    if (lane == 0) red[tid >> 5] = v;
+    __syncthreads();
+    if (tid == 0) {
+      u64 t = 0;
+      for (int w = 0; w < AT_THREADS / 32; w++) t += red[w];
+      const u64 m = (1ull << 20) - 1;
+      ta_attr_summary *sm = &a.sum[a.lane_window[l]];
+      if (t & m) atomicAdd((u64 *)&sm->n_attributed, t & m);
+      if ((t >> 20) & m) atomicAdd((u64 *)&sm->n_no_launch, (t >> 20) & m);
+      if ((t >> 40) & m) atomicAdd((u64 *)&sm->n_no_op, (t >> 40) & m);
+    }
   }
 }
 
 // first/last were accumulated in an order-preserving unsigned encoding (0 = untouched)
 __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
-  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (p >= a.n_valid || a.kind[p] != TA_KIND_OP) return;
-  if (a.op_n[p] > 0) {
-    a.op_first[p] = (~a.op_first[p]) ^ (1ull << 63);
-    a.op_last[p] = a.op_last[p] ^ (1ull << 63);
+  const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (p0 >= a.n_valid) return;
+  int16_t kd[8];
+  load8_i16(a.kind, p0, a.n, 9, kd);
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    const int64_t p = p0 + j;
+    if (p < a.n_valid && kd[j] == TA_KIND_OP && a.op_n[p] > 0) {
+      a.op_first[p] = (~a.op_first[p]) ^ (1ull << 63);
+      a.op_last[p] = a.op_last[p] ^ (1ull << 63);
+    }
   }
 }
-
 
 ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   const int64_t n = h->n, nn = n > 0 ? n : 1;
@@ -611,8 +649,8 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
     k_attr_agg<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
     if (a.n_lanes > 0) k_attr_carry<<<TA_N (unsigned)((a.n_lanes + 3) / 4), 128, 0, st>>>(a);
     k_attr_resolve<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
-    k_attr_ops<<<TA_N (unsigned)((n + 2047) / 2048), 512, 0, st>>>(a);
-    const int64_t fb = (h->n_valid + 255) / 256;
+    k_attr_ops<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
+    const int64_t fb = (h->n_valid + 2047) / 2048;
     k_attr_finalize<<<TA_N (unsigned)(fb > 0 ? fb : 1), 256, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
   }
