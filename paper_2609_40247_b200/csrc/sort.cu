@@ -82,11 +82,15 @@ __global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
       }
     }
 #endif
-    const int leader = __ffs(m) - 1;
-    u32 pre = 0;
-    if (valid && lane == leader) pre = atomicAdd(&s.warp_hist[warp][d], (u32)__popc(m));
-    pre = __shfl_sync(0xffffffffu, pre, leader);
-    lrank[j] = (int)(pre + __popc(m & ((1u << lane) - 1u)));
+    // one population count per key (they run on the slow special-function pipe): the number of
+    // peers at or above the lane.  The lowest peer adds the group size to the warp's digit
+    // counter; every peer then reads the counter back and steps down from its new value.
+    const u32 above1 = (u32)__popc(m >> lane);
+    if (valid && (m & ((1u << lane) - 1u)) == 0) atomicAdd(&s.warp_hist[warp][d], above1);
+    __syncwarp();
+    const u32 after = valid ? s.warp_hist[warp][d] : 0u;
+    lrank[j] = (int)(after - above1);
+    __syncwarp();
   }
   __syncthreads();
   // per digit: exclusive offsets of the warps, then the CTA's digit count
