@@ -234,9 +234,7 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   u32 *pos_all = c1.take<u32>(nn);
   ScanTemp s1;
   TA_TRY(scan_temp_init(h, c1.base + c1.off, n, &s1));
-  CollSelIn sin{h->sorted.kind, h->n_valid};
-  CollSelOut sout{pos_all};
-  TA_TRY((launch_scan<OpAdd, CollSelIn, CollSelOut>(h, n, sin, sout, OpAdd(), s1)));
+  TA_TRY(launch_compact_kind(h, h->sorted.kind, h->n_valid, 1u << TA_KIND_COLL, pos_all, s1));
   u64 m64 = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, s1.total, 8, cudaMemcpyDeviceToHost, st));
   std::vector<u64> comm_sorted(h->n_comms);

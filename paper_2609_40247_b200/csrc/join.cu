@@ -505,9 +505,9 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       void *sort_tmp = ct.base + ct.off;
       ScanTemp t1;
       TA_TRY(scan_temp_init(h, scan_mem1, n, &t1));
-      JoinSelIn sin{a.kind, h->n_valid};
-      JoinSelOut sout{pos};
-      TA_TRY((launch_scan<OpAdd, JoinSelIn, JoinSelOut>(h, n, sin, sout, OpAdd(), t1)));
+      TA_TRY(launch_compact_kind(h, a.kind, h->n_valid,
+                                 (1u << TA_KIND_LAUNCH) | (1u << TA_KIND_KERNEL) | (1u << TA_KIND_MEMCPY),
+                                 pos, t1));
       u64 m64 = 0;
       TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, t1.total, 8, cudaMemcpyDeviceToHost, st));
       TA_CHECK_CUDA(h, cudaStreamSynchronize(st));

@@ -142,6 +142,54 @@ __device__ __forceinline__ void store8_i32(int32_t *col, int64_t p0, int64_t n, 
   }
 }
 
+// Ordered compaction of the sorted positions whose kind is in `kind_mask`: 256 threads x 16
+// positions per tile, vector loads of the kind column, one tile scan.
+#define CK_THREADS 256
+#define CK_ITEMS 16
+#define CK_TILE (CK_THREADS * CK_ITEMS)
+static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_t *kind, int64_t n_valid,
+                                                             u32 kind_mask, u32 *pos_out, ScanTemp t,
+                                                             int32_t *status) {
+  __shared__ u64 tmp[33];
+  __shared__ u64 s_excl;
+  __shared__ int s_tile;
+  const int tid = threadIdx.x;
+  if (tid == 0) s_tile = (int)atomicAdd(t.counter, 1u);
+  __syncthreads();
+  const int tile = s_tile;
+  const int64_t p0 = (int64_t)tile * CK_TILE + (int64_t)tid * CK_ITEMS;
+  int16_t kd[CK_ITEMS];
+  load8_i16(kind, p0, n_valid, -1, kd);
+  load8_i16(kind, p0 + 8, n_valid, -1, kd + 8);
+  u32 sel = 0;
+#pragma unroll
+  for (int j = 0; j < CK_ITEMS; j++)
+    if (kd[j] >= 0 && ((kind_mask >> kd[j]) & 1u)) sel |= 1u << j;
+  u64 total;
+  u64 ex = block_scan_exclusive<OpAdd>((u64)__popc(sel), OpAdd(), tmp, &total);
+  if (tid < 32) {
+    u64 e = tile_lookback<OpAdd>(t.state, tile, total, OpAdd(), status);
+    if (tid == 0) {
+      s_excl = e;
+      if ((int64_t)(tile + 1) * CK_TILE >= n_valid) *t.total = e + total;
+    }
+  }
+  __syncthreads();
+  u64 o = s_excl + ex;
+#pragma unroll
+  for (int j = 0; j < CK_ITEMS; j++)
+    if (sel & (1u << j)) pos_out[o++] = (u32)(p0 + j);
+}
+static inline ta_status launch_compact_kind(ta_window *h, const int16_t *kind, int64_t n_valid,
+                                            u32 kind_mask, u32 *pos_out, ScanTemp t) {
+  if (n_valid <= 0) return TA_OK;
+  int64_t tiles = (n_valid + CK_TILE - 1) / CK_TILE;
+  k_compact_kind<<<TA_N (unsigned)tiles, CK_THREADS, 0, h->stream>>>(kind, n_valid, kind_mask, pos_out, t,
+                                                                   h->d_status);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  return TA_OK;
+}
+
 // Walks the lane table along ascending sorted positions.
 struct LaneWalker {
   const int32_t *lane_off;
