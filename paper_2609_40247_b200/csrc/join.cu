@@ -431,14 +431,15 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   const int n_slots = W * (h->n_pids > 0 ? h->n_pids : 1);
   cudaStream_t st = h->stream;
   const int64_t nn = n > 0 ? n : 1;
-  size_t keep = 2 * Carver::pad(nn * 4) + 2 * Carver::pad(nn * 8) + 3 * Carver::pad((size_t)n_slots * 8) +
+  size_t keep = 2 * Carver::pad(nn * 4) + 2 * Carver::pad(nn * 8) + Carver::pad((size_t)n_slots * 8) +
                 Carver::pad((size_t)W * sizeof(ta_join_summary)) + 256;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
   Carver ck(kb);
   int32_t *launch_of = ck.take<int32_t>(nn), *kol = ck.take<int32_t>(nn);
   int64_t *latency = ck.take<int64_t>(nn), *qdelay = ck.take<int64_t>(nn);
-  i64 *slot_min = ck.take<i64>(n_slots), *slot_max = ck.take<i64>(n_slots), *slot_base = ck.take<i64>(n_slots);
+  i64 *slot_min = h->d_slot_min, *slot_max = h->d_slot_max;  // filled while the records were gathered
+  i64 *slot_base = ck.take<i64>(n_slots);
   ta_join_summary *d_sum = ck.take<ta_join_summary>(W);
 
   std::vector<ta_join_summary> hs(W);
@@ -447,10 +448,9 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
     s.min_latency = INT64_MAX;
     s.max_latency = INT64_MIN;
   }
-  std::vector<i64> hmin(n_slots, INT64_MAX), hmax(n_slots, INT64_MIN), hbase(n_slots, -1);
+  std::vector<i64> hmin(h->h_slot_min.begin(), h->h_slot_min.end());
+  std::vector<i64> hmax(h->h_slot_max.begin(), h->h_slot_max.end()), hbase(n_slots, -1);
   TA_CHECK_CUDA(h, cudaMemcpyAsync(d_sum, hs.data(), W * sizeof(ta_join_summary), cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_min, hmin.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_max, hmax.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(kol, 0, nn * 4, st));
 
   JoinArgs a;
@@ -466,11 +466,6 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   void *tmp_alloc = nullptr;
   bool direct = true;
   if (n > 0) {
-    k_join_minmax<<<TA_N grid, JN_THREADS, 0, st>>>(a);
-    TA_CHECK_CUDA(h, cudaGetLastError());
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(hmin.data(), slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(hmax.data(), slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
     // table size if every slot is addressed directly
     unsigned __int128 total = 0;
     for (int s = 0; s < n_slots; s++)

@@ -86,6 +86,8 @@ struct ta_window {
   ta_sort_result sorted;
   int32_t *d_lane_code;      // per lane: window << tbits | triple rank
   int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
+  i64 *d_slot_min, *d_slot_max;               // per slot: corr_id range of its LAUNCH records
+  std::vector<int64_t> h_slot_min, h_slot_max;  // host copies (INT64_MAX / INT64_MIN when none)
 
   // join / attribution products
   ta_join_result join;

@@ -88,6 +88,10 @@ struct GatherArgs {
   int sbits;          // key bits below the lane code (time bits kept [+ index bits])
   int packed, ibits, wshift, wbits;
   const int64_t *off;
+  // corr_id range of the LAUNCH records per (window, pid) slot, for the join
+  const TripleTable *tt;
+  int tbits, n_pids;
+  i64 *slot_min, *slot_max;
   i64 *ts_start, *ts_end, *corr;
   int32_t *pid, *name, *seq;
   int16_t *stream, *kind;
@@ -95,8 +99,12 @@ struct GatherArgs {
 };
 
 __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
+  __shared__ int s_slot[8];
+  __shared__ u64 s_mx[8], s_mn[8];
   int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (p >= a.n) return;
+  int slot = -1;
+  u64 mx = 0, mn_inv = 0;
+  if (p < a.n) {
   u32 idx;
   if (a.packed && p < a.n_valid) {
     const u64 k = a.keys[p];
@@ -118,6 +126,50 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   if (p < a.n_valid) {
     u64 code = a.keys[p] >> a.sbits;
     if (p == 0 || (a.keys[p - 1] >> a.sbits) != code) a.lane_start[code] = (int32_t)p;
+    if (r.kind == TA_KIND_LAUNCH) {
+      slot = (int)(code >> a.tbits) * a.n_pids + a.tt->pid_rank[code & ((1ull << a.tbits) - 1)];
+      mx = (u64)r.corr ^ (1ull << 63);
+      mn_inv = ~mx;
+    }
+  }
+  }  // p < n
+  // fold the range per CTA (a CTA almost always sits inside one lane)
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const u32 has = __ballot_sync(0xffffffffu, slot >= 0);
+  int wslot = -1;
+  if (has) {
+    wslot = __shfl_sync(0xffffffffu, slot, __ffs(has) - 1);
+    if (__all_sync(0xffffffffu, slot < 0 || slot == wslot)) {
+      mx = warp_reduce(mx, OpMax());
+      mn_inv = warp_reduce(mn_inv, OpMax());
+    } else {  // mixed warp (lane boundary): every thread for itself
+      if (slot >= 0) {
+        atomicMax(&a.slot_max[slot], (i64)(mx ^ (1ull << 63)));
+        atomicMin(&a.slot_min[slot], (i64)((~mn_inv) ^ (1ull << 63)));
+      }
+      wslot = -1;
+    }
+  }
+  if (lane == 0) { s_slot[warp] = wslot; s_mx[warp] = mx; s_mn[warp] = mn_inv; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int cur = -1;
+    u64 cmx = 0, cmn = 0;
+    for (int w = 0; w <= 8; w++) {
+      const int sl = w < 8 ? s_slot[w] : -2;
+      if (sl == -1) continue;
+      if (sl != cur) {
+        if (cur >= 0) {
+          const i64 hi = (i64)(cmx ^ (1ull << 63)), lo = (i64)((~cmn) ^ (1ull << 63));
+          if (hi > a.slot_max[cur]) atomicMax(&a.slot_max[cur], hi);
+          if (lo < a.slot_min[cur]) atomicMin(&a.slot_min[cur], lo);
+        }
+        cur = sl;
+        cmx = 0;
+        cmn = 0;
+      }
+      if (w < 8) { cmx = max(cmx, s_mx[w]); cmn = max(cmn, s_mn[w]); }
+    }
   }
 }
 
@@ -253,11 +305,12 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   cudaStream_t st = h->stream;
   const int64_t n_codes = (int64_t)h->W << h->tbits;  // lane code = window << tbits | triple rank
   const int64_t lane_cap = (n_codes < n ? n_codes : n) + 1;  // lanes <= min(codes, records)
+  const int64_t n_slots = (int64_t)h->W * (h->n_pids > 0 ? h->n_pids : 1);
 
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
                 2 * Carver::pad(n * 2) + 4 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
-                Carver::pad((lane_cap + 1) * 4) + 512;
+                Carver::pad((lane_cap + 1) * 4) + 2 * Carver::pad((size_t)n_slots * 8) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
   Carver ck(kb);
@@ -270,6 +323,12 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int16_t *lane_stream = ck.take<int16_t>(lane_cap), *lane_domain = ck.take<int16_t>(lane_cap);
   int32_t *lane_off = ck.take<int32_t>(lane_cap + 1);
   int32_t *n_lanes_dev = ck.take<int32_t>(1);
+  h->d_slot_min = ck.take<i64>(n_slots);
+  h->d_slot_max = ck.take<i64>(n_slots);
+  h->h_slot_min.assign((size_t)n_slots, INT64_MAX);
+  h->h_slot_max.assign((size_t)n_slots, INT64_MIN);
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_min, h->h_slot_min.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_max, h->h_slot_max.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
 
   // temporaries (released at the end of the call)
   size_t tmp_bytes = 2 * Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
@@ -367,6 +426,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     g.sbits = h->packed ? h->ibits + (h->sbits - h->dshift) : h->sbits;
     g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
     g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
+    g.tt = h->d_triples; g.tbits = h->tbits; g.n_pids = h->n_pids > 0 ? h->n_pids : 1;
+    g.slot_min = h->d_slot_min; g.slot_max = h->d_slot_max;
     k_gather<<<TA_N nblk(n, 256), 256, 0, st>>>(g);
   }
   k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
@@ -376,6 +437,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   TA_CHECK_CUDA(h, cudaGetLastError());
   int32_t n_lanes = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_max.data(), h->d_slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
   TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
   ta_dfree(h, tb);
   ta_dfree(h, h->d_keys);
