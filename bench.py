@@ -18,9 +18,7 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 import numpy as np
@@ -65,55 +63,54 @@ def measured_peak():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons (NVML, read-only) while the timed region runs."""
 
     def __init__(self, device_index):
         self.idx = device_index
-        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
-        self.p = None
+        self.sm, self.reasons, self.max_mhz = [], set(), None
+        self._stop = False
+        self._thread = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            # LOCAL_RANK indexes the visible devices; map through CUDA_VISIBLE_DEVICES if it is set
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.idx
+            if vis:
+                ids = [x for x in vis.split(",") if x != ""]
+                if self.idx < len(ids) and ids[self.idx].isdigit():
+                    idx = int(ids[self.idx])
+            hnd = nv.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = float(nv.nvmlDeviceGetMaxClockInfo(hnd, nv.NVML_CLOCK_SM))
+            names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                     "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                     "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                     "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+            while not self._stop:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(hnd, nv.NVML_CLOCK_SM)))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(hnd)
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+                time.sleep(0.01)
+        except Exception as e:  # no NVML: report that no samples were taken
+            self.error = str(e)
 
     def start(self):
-        try:
-            self.p = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
-                 "-i", str(self.idx)], stdout=self.f, stderr=subprocess.DEVNULL)
-        except Exception:
-            self.p = None
+        import threading
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
 
     def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.p is not None:
-            self.p.terminate()
-            try:
-                self.p.wait(timeout=5)
-            except Exception:
-                self.p.kill()
-        self.f.flush()
-        self.f.seek(0)
-        sm, mx, reasons = [], [], set()
-        for line in self.f.read().splitlines():
-            t = [x.strip() for x in line.split(",")]
-            if len(t) < 9:
-                continue
-            try:
-                sm.append(float(t[1]))
-                mx.append(float(t[2]))
-            except ValueError:
-                continue
-            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
-                                "sw_power_cap"), t[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        self.f.close()
-        os.unlink(self.f.name)
-        if sm:
-            out["sm_mhz"] = statistics.median(sm)
-            out["sm_max_mhz"] = max(mx)
-            out["samples"] = len(sm)
-        out["reasons"] = sorted(reasons)
+        self._stop = True
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+        out = {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
+        if self.sm:
+            out["sm_mhz"] = statistics.median(self.sm)
+            out["samples"] = len(self.sm)
         return out
 
 
@@ -228,11 +225,12 @@ def main():
         torch.cuda.synchronize()
 
     # ---- device-resident timing ----
-    sampler = ClockSampler(local_rank)  # started before the warm-up: nvidia-smi needs a moment
-    sampler.start()
     for _ in range(max(args.warmup, 0)):
         run_pipeline(ta, dev_buf, wl)
     barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.05)
     ta.profile_enable(True)
     launches0 = ta.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

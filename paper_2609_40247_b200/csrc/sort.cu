@@ -6,11 +6,17 @@
 //
 // Tile layout: THREADS x ITEMS elements per CTA, keys staged through shared
 // memory so that both the global loads (warp-striped) and the scattered stores
-// (runs of equal digits) are coalesced.  HBM-bound: per element and pass 8 B read
-// + 8 B written (keys only) or 12 B + 12 B (pairs).
+// (runs of equal digits) are coalesced.  HBM-bound by design (per element and
+// pass 8 B read + 8 B written for keys, 12 B + 12 B for pairs); in practice the
+// pass is instruction-bound on B200, so the kernel is specialised on the digit
+// width and on full tiles, and every key costs one population count, one
+// shared-memory atomic and as many warp votes as the digit has bits.
 #include "ta_internal.cuh"
 
 #define RS_BINS 256
+#ifndef RS_MINB
+#define RS_MINB 2  // resident CTAs per SM the register budget is sized for
+#endif
 
 struct RadixArgs {
   const u64 *keys_in;
@@ -18,7 +24,7 @@ struct RadixArgs {
   const u32 *vals_in;  // may be null: value = global index
   u32 *vals_out;
   int64_t n;
-  int shift, bits;
+  int shift;
   const u32 *bin_offset;  // exclusive global digit offsets of this pass
   u64 *tile_state;        // [tile][RS_BINS]
   u32 *tile_counter;
@@ -28,88 +34,78 @@ struct RadixArgs {
 template <int THREADS, int ITEMS>
 struct RadixSmem {
   u64 keys[THREADS * ITEMS];  // aliased by u32 values after the keys are written out
-  u32 warp_hist[THREADS / 32][RS_BINS];
-  u32 bin_start[RS_BINS];
-  i64 adj[RS_BINS];
+  u32 warp_hist[THREADS / 32][RS_BINS];  // per warp: digit counts, later tile-local start of the warp's run
+  u32 adj[RS_BINS];           // global position of a digit's run minus its tile-local start (mod 2^32)
   u64 scan_tmp[33];
   int tile;
   int fail;
 };
 
-template <int THREADS, int ITEMS, bool VALS>
-__global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
+template <int THREADS, int ITEMS, bool VALS, int BITS, bool FULL>
+__device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS, ITEMS> &s, int tile,
+                                           int count) {
   constexpr int TILE = THREADS * ITEMS;
   constexpr int WARPS = THREADS / 32;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  RadixSmem<THREADS, ITEMS> &s = *reinterpret_cast<RadixSmem<THREADS, ITEMS> *>(smem_raw);
+  constexpr u32 MASK = (1u << BITS) - 1u;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) {
-    s.tile = (int)atomicAdd(a.tile_counter, 1u);
-    s.fail = 0;
-  }
-  for (int i = tid; i < WARPS * RS_BINS; i += THREADS) (&s.warp_hist[0][0])[i] = 0;
-  __syncthreads();
-  const int tile = s.tile;
   const int64_t base = (int64_t)tile * TILE;
-  const int count = (int)min((int64_t)TILE, a.n - base);
-  const u32 mask = (1u << a.bits) - 1u;
+  const u32 lt = (1u << lane) - 1u;
 
   u64 key[ITEMS];
-  int lrank[ITEMS];
+  int rd[ITEMS];  // (tile-local rank << 8) | digit
   const int wbase = warp * 32 * ITEMS;
 #pragma unroll
   for (int j = 0; j < ITEMS; j++) {
-    int li = wbase + j * 32 + lane;
-    key[j] = li < count ? a.keys_in[base + li] : ~0ull;
+    const int li = wbase + j * 32 + lane;
+    key[j] = (FULL || li < count) ? a.keys_in[base + li] : ~0ull;
   }
   // rank inside the warp, item row by item row (stable: row-major, then lane)
+  u32 *wh = s.warp_hist[warp];
 #pragma unroll
   for (int j = 0; j < ITEMS; j++) {
-    int li = wbase + j * 32 + lane;
-    bool valid = li < count;
-    u32 d = valid ? ((u32)(key[j] >> a.shift) & mask) : 0xFFFFFFFFu;
-#ifdef RS_USE_MATCH
-    u32 m = __match_any_sync(0xffffffffu, d);
-#else
-    // lanes with the same digit: one ballot per digit bit (cheaper than match.any here)
-    u32 m = __ballot_sync(0xffffffffu, valid);
-    if (!valid) m = ~m;
+    const bool valid = FULL || (wbase + j * 32 + lane) < count;
+    const u32 d = (u32)(key[j] >> a.shift) & MASK;
+    // lanes with the same digit: one vote per digit bit
+    u32 m = FULL ? 0xffffffffu : __ballot_sync(0xffffffffu, valid);
+    if (!FULL && !valid) m = ~m;
 #pragma unroll
-    for (int b = 0; b < 8; b++) {
-      if (b < a.bits) {
-        const u32 bal = __ballot_sync(0xffffffffu, (d >> b) & 1u);
-        m &= ((d >> b) & 1u) ? bal : ~bal;
-      }
+    for (int b = 0; b < BITS; b++) {
+      const u32 bit = (d >> b) & 1u;
+      const u32 bal = __ballot_sync(0xffffffffu, valid && bit);
+      m &= bal ^ (bit - 1u);  // bit set: keep bal; bit clear: keep ~bal
     }
-#endif
-    // one population count per key (they run on the slow special-function pipe): the number of
-    // peers at or above the lane.  The lowest peer adds the group size to the warp's digit
-    // counter; every peer then reads the counter back and steps down from its new value.
+    if (!FULL && !valid) m = 0;
+    // one population count per key: the number of peers at or above the lane.  The lowest
+    // peer adds the group size to the warp's digit counter; every peer then reads the counter
+    // back and steps down from its new value.
     const u32 above1 = (u32)__popc(m >> lane);
-    if (valid && (m & ((1u << lane) - 1u)) == 0) atomicAdd(&s.warp_hist[warp][d], above1);
+    if (valid && (m & lt) == 0) atomicAdd(&wh[d], above1);
     __syncwarp();
-    const u32 after = valid ? s.warp_hist[warp][d] : 0u;
-    lrank[j] = (int)(after - above1);
+    const u32 after = valid ? wh[d] : 0u;
+    rd[j] = (int)(((after - above1) << 8) | d);
     __syncwarp();
   }
   __syncthreads();
-  // per digit: exclusive offsets of the warps, then the CTA's digit count
+  // per digit: the CTA's count, exclusive starts of the digits, and per warp the tile-local
+  // start of its run (so the scatter needs one shared load per key)
   u32 cnt = 0;
   if (tid < RS_BINS) {
-    u32 run = 0;
+#pragma unroll
+    for (int w = 0; w < WARPS; w++) cnt += s.warp_hist[w][tid];
+  }
+  u64 total;
+  const u64 ex = block_scan_exclusive<OpAdd>((u64)cnt, OpAdd(), s.scan_tmp, &total);
+  if (tid < RS_BINS) {
+    u32 run = (u32)ex;
 #pragma unroll
     for (int w = 0; w < WARPS; w++) {
-      u32 t = s.warp_hist[w][tid];
+      const u32 t = s.warp_hist[w][tid];
       s.warp_hist[w][tid] = run;
       run += t;
     }
-    cnt = run;
   }
-  u64 total;
-  u64 ex = block_scan_exclusive<OpAdd>((u64)cnt, OpAdd(), s.scan_tmp, &total);
-  if (tid < RS_BINS) s.bin_start[tid] = (u32)ex;
   // chained scan over tiles, one digit per thread
-  if (tid < (1 << a.bits)) {
+  if (tid < (1 << BITS)) {
     u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
     u64 excl;
     if (tile == 0) {
@@ -120,38 +116,37 @@ __global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
       excl = 0;
       bool timed_out = false;
       for (int t = tile - 1;; --t) {
-        u64 w = td_wait(a.tile_state + (size_t)t * RS_BINS + tid, a.status, &timed_out);
+        const u64 w = td_wait(a.tile_state + (size_t)t * RS_BINS + tid, a.status, &timed_out);
         excl += w & TD_MASK;
         if ((w >> 62) == TD_PREFIX) break;
       }
       st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
       if (timed_out) s.fail = 1;
     }
-    s.adj[tid] = (i64)excl - (i64)ex;
+    s.adj[tid] = (u32)excl - (u32)ex;
   }
   __syncthreads();
   if (s.fail) return;
   // stage keys in shared memory in digit order
 #pragma unroll
   for (int j = 0; j < ITEMS; j++) {
-    int li = wbase + j * 32 + lane;
-    if (li < count) {
-      u32 d = (u32)(key[j] >> a.shift) & mask;
-      lrank[j] += (int)(s.bin_start[d] + s.warp_hist[warp][d]);
-      s.keys[lrank[j]] = key[j];
+    if (FULL || (wbase + j * 32 + lane) < count) {
+      const u32 d = (u32)rd[j] & 0xFFu;
+      const int r = (rd[j] >> 8) + (int)wh[d];
+      rd[j] = r;
+      s.keys[r] = key[j];
     }
   }
   __syncthreads();
   u32 gpos[VALS ? ITEMS : 1];
 #pragma unroll
   for (int k = 0; k < ITEMS; k++) {
-    int sl = tid + k * THREADS;
+    const int sl = tid + k * THREADS;
     if (VALS) gpos[k] = 0xFFFFFFFFu;
-    if (sl < count) {
-      u64 kk = s.keys[sl];
-      u32 d = (u32)(kk >> a.shift) & mask;
-      i64 p = s.adj[d] + sl;
-      if (VALS) gpos[k] = (u32)p;
+    if (FULL || sl < count) {
+      const u64 kk = s.keys[sl];
+      const u32 p = s.adj[(u32)(kk >> a.shift) & MASK] + (u32)sl;
+      if (VALS) gpos[k] = p;
       a.keys_out[p] = kk;
     }
   }
@@ -160,15 +155,33 @@ __global__ void __launch_bounds__(THREADS) k_radix_pass(RadixArgs a) {
   u32 *svals = reinterpret_cast<u32 *>(s.keys);
 #pragma unroll
   for (int j = 0; j < ITEMS; j++) {
-    int li = wbase + j * 32 + lane;
-    if (li < count) svals[lrank[j]] = a.vals_in ? a.vals_in[base + li] : (u32)(base + li);
+    const int li = wbase + j * 32 + lane;
+    if (FULL || li < count) svals[rd[j]] = a.vals_in ? a.vals_in[base + li] : (u32)(base + li);
   }
   __syncthreads();
 #pragma unroll
   for (int k = 0; k < ITEMS; k++) {
-    int sl = tid + k * THREADS;
-    if (sl < count) a.vals_out[gpos[VALS ? k : 0]] = svals[sl];
+    const int sl = tid + k * THREADS;
+    if (FULL || sl < count) a.vals_out[gpos[VALS ? k : 0]] = svals[sl];
   }
+}
+
+template <int THREADS, int ITEMS, bool VALS, int BITS>
+__global__ void __launch_bounds__(THREADS, RS_MINB) k_radix_pass(RadixArgs a) {
+  constexpr int TILE = THREADS * ITEMS;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  RadixSmem<THREADS, ITEMS> &s = *reinterpret_cast<RadixSmem<THREADS, ITEMS> *>(smem_raw);
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    s.tile = (int)atomicAdd(a.tile_counter, 1u);
+    s.fail = 0;
+  }
+  for (int i = tid; i < (THREADS / 32) * RS_BINS; i += THREADS) (&s.warp_hist[0][0])[i] = 0;
+  __syncthreads();
+  const int tile = s.tile;
+  const int count = (int)min((int64_t)TILE, a.n - (int64_t)tile * TILE);
+  if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true>(a, s, tile, count);
+  else radix_tile<THREADS, ITEMS, VALS, BITS, false>(a, s, tile, count);
 }
 
 // tile shapes
@@ -234,6 +247,25 @@ size_t ta_sort_temp_bytes(int64_t n) {
          2 * Carver::pad(10 * RS_BINS * sizeof(u32));
 }
 
+template <int THREADS, int ITEMS, bool VALS>
+static cudaError_t launch_pass(const RadixArgs &a, int bits, unsigned tiles, cudaStream_t st) {
+  typedef RadixSmem<THREADS, ITEMS> Smem;
+#define RS_CASE(B)                                                                                  \
+  case B: {                                                                                         \
+    auto kern = k_radix_pass<THREADS, ITEMS, VALS, B>;                                              \
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
+                                         (int)sizeof(Smem));                                        \
+    if (e != cudaSuccess) return e;                                                                 \
+    kern<<<TA_N tiles, THREADS, sizeof(Smem), st>>>(a);                                             \
+    return cudaGetLastError();                                                                      \
+  }
+  switch (bits) {
+    RS_CASE(1) RS_CASE(2) RS_CASE(3) RS_CASE(4) RS_CASE(5) RS_CASE(6) RS_CASE(7) RS_CASE(8)
+  }
+#undef RS_CASE
+  return cudaErrorInvalidValue;
+}
+
 // Sorts n keys (vals: pairs) by the key bits the plan covers.  Pass outputs
 // alternate between the scratch and the final buffers such that the last pass
 // writes the final ones; keys_in / vals_in are only read (pairs with vals_in null:
@@ -247,10 +279,6 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
   constexpr int THREADS = VALS ? RSP_THREADS : RSK_THREADS;
   constexpr int ITEMS = VALS ? RSP_ITEMS : RSK_ITEMS;
   constexpr int TILE = THREADS * ITEMS;
-  typedef RadixSmem<THREADS, ITEMS> Smem;
-  auto kern = k_radix_pass<THREADS, ITEMS, VALS>;
-  TA_CHECK_CUDA(h, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)sizeof(Smem)));
   size_t tiles = (size_t)((n + TILE - 1) / TILE);
   Carver c(temp);
   size_t max_tiles = (size_t)((n + (int64_t)min_tile() - 1) / (int64_t)min_tile());
@@ -276,12 +304,12 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     RadixArgs a;
     a.keys_in = kin; a.keys_out = to_final ? keys_final : keys_scratch;
     a.vals_in = vin; a.vals_out = to_final ? vals_final : vals_scratch;
-    a.n = n; a.shift = plan.shift[p]; a.bits = plan.bits[p];
+    a.n = n; a.shift = plan.shift[p];
     a.bin_offset = bin_offset + p * RS_BINS;
     a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
     if (timed) ta_profile_mark(st, 1, (VALS ? 24.0 : 16.0) * (double)n);
-    kern<<<TA_N (unsigned)tiles, THREADS, sizeof(Smem), st>>>(a);
+    TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, VALS>(a, plan.bits[p], (unsigned)tiles, st)));
     if (timed) ta_profile_mark(st, 0, 0.0);
     kin = a.keys_out;
     vin = a.vals_out;
