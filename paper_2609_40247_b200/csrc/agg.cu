@@ -3,8 +3,9 @@
 // Per-symbol counts and duration statistics are what Sec. 8.1 compares.
 //
 // Symbol popularity is heavy-tailed (a few names carry most records), so global
-// atomics alone would serialise on the hot rows.  Each CTA walks a contiguous
-// range of sorted positions (one process, mostly) and folds its records into a
+// atomics alone would serialise on the hot rows.  Each CTA takes 16384
+// consecutive sorted positions (one process, mostly; CTAs whose lanes cannot
+// hold a selected kind return at once) and folds its records into a
 // shared-memory hash table first; the table is flushed to a dense global table
 // indexed by (window, pid rank, name_id - min name) with one atomic per field.
 // A scan then compacts the non-empty rows in key order.
@@ -22,6 +23,7 @@
 #define AG_ITEMS 4
 #define AG_STEP (AG_THREADS * AG_ITEMS)
 #define AG_SLOTS 256
+#define AG_ITEM (16 * AG_STEP)   // positions per CTA
 #define AG_FLUSH_EVERY 32768  // records per CTA between flushes (keeps 16-bit bins safe)
 
 struct AggArgs {
@@ -36,7 +38,11 @@ struct AggArgs {
   uint32_t kind_mask;
   int value_sel;
   int64_t min_name, R;
-  int64_t chunk;  // positions per CTA, a multiple of AG_STEP
+  const int16_t *lane_domain;
+  const int32_t *lane_dom_end;
+  int want_domain;  // 0 / 1: the selected kinds all live in lanes of this domain; -1: both
+  int64_t chunk;    // positions per CTA, a multiple of AG_STEP
+  unsigned n_items, spread, per;
   // dense table (all zero-initialised; min is kept as the complement of the biased value)
   u64 *d_cnt, *d_sum, *d_minc, *d_maxb;
   u32 *d_hist;
@@ -95,89 +101,105 @@ __device__ __forceinline__ void agg_flush(const AggArgs &a, AggSmem &s) {
 
 __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
   __shared__ AggSmem s;
-  agg_clear(s);
-  __syncthreads();
-  const int64_t begin = (int64_t)blockIdx.x * a.chunk;
-  const int64_t end = min(begin + a.chunk, a.n_valid);
   int since_flush = 0;
-  LaneWalker lw(a.lane_off, a.n_lanes, begin + (int64_t)threadIdx.x * AG_ITEMS, a.n_valid);
-  for (int64_t base = begin; base < end; base += AG_STEP) {
-    const int64_t p0 = base + (int64_t)threadIdx.x * AG_ITEMS;
-    // all loads of the thread's four records are issued before any of them is used
-    int16_t kd[AG_ITEMS];
-    if (p0 + AG_ITEMS <= end) {
-      uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
-      const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
-#pragma unroll
-      for (int j = 0; j < AG_ITEMS; j++) kd[j] = hq[j];
-    } else {
-#pragma unroll
-      for (int j = 0; j < AG_ITEMS; j++) kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
-    }
-    bool sel[AG_ITEMS];
-    i64 v[AG_ITEMS];
-    int32_t nm[AG_ITEMS];
-#pragma unroll
-    for (int j = 0; j < AG_ITEMS; j++) {
-      sel[j] = kd[j] >= 0 && ((a.kind_mask >> kd[j]) & 1u);
-      v[j] = 0;
-      nm[j] = 0;
-    }
-    if (a.value_sel == 0) {
-#pragma unroll
-      for (int j = 0; j < AG_ITEMS; j++)
-        if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
-    } else {
-#pragma unroll
-      for (int j = 0; j < AG_ITEMS; j++)
-        if (sel[j]) sel[j] = a.op_n[p0 + j] > 0;
-#pragma unroll
-      for (int j = 0; j < AG_ITEMS; j++)
-        if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
-    }
-#pragma unroll
-    for (int j = 0; j < AG_ITEMS; j++) {
-      if (!sel[j]) continue;
-      const int lane = lw.at(p0 + j);
-      const int64_t g = (int64_t)a.lane_slot[lane] * a.R + ((int64_t)nm[j] - a.min_name);
-      const u64 vb = (u64)v[j] ^ (1ull << 63);
-      const int bin = log2_bin(v[j]);
-      u32 hsh = (u32)g * 2654435761u;
-      int slot = (int)(hsh >> 24) & (AG_SLOTS - 1);
-      bool placed = false;
-      for (int probe = 0; probe < 8; probe++) {
-        int32_t cur = s.key[slot];
-        if (cur == (int32_t)g) { placed = true; break; }
-        if (cur == -1) {
-          int32_t old = atomicCAS(&s.key[slot], -1, (int32_t)g);
-          if (old == -1 || old == (int32_t)g) { placed = true; break; }
-        }
-        slot = (slot + 1) & (AG_SLOTS - 1);
-      }
-      if (placed) {
-        atomicAdd(&s.cnt[slot], 1u);
-        {  // values are durations (>= 0): 16 + 16 + 32 bit limbs, at most 32768 adds per flush
-          const u64 uv = (u64)v[j];
-          atomicAdd(&s.sum16[0][slot], (u32)(uv & 0xFFFF));
-          if (uv >> 16) atomicAdd(&s.sum16[1][slot], (u32)((uv >> 16) & 0xFFFF));
-          if (uv >> 32) atomicAdd(&s.sum16[2][slot], (u32)(uv >> 32));
-        }
-        // 64-bit min/max in shared memory are compare-and-swap loops: skip them unless the
-        // value would actually move the extreme (rare once a slot has seen a few records)
-        if (~vb > s.minc[slot]) atomicMax(&s.minc[slot], ~vb);
-        if (vb > s.maxb[slot]) atomicMax(&s.maxb[slot], vb);
-        // 16-bit bins packed two per word
-        u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
-        atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
+  LaneWalker lw(a.lane_off, a.n_lanes, a.n_valid, a.n_valid);
+  {
+    // CTA b -> chunk (b mod G) * S + b / G: CTAs that run together work far apart in the
+    // timeline (different processes), so their flushes rarely meet on the same global rows;
+    // chunks whose lanes cannot hold a selected kind return at once and make room
+    const unsigned item = (blockIdx.x % a.spread) * a.per + blockIdx.x / a.spread;
+    if (item >= a.n_items) return;
+    const int64_t begin = (int64_t)item * a.chunk;
+    const int64_t end = min(begin + a.chunk, a.n_valid);
+    int bl = lane_of_pos(a.lane_off, a.n_lanes, begin);  // lane of `base`, the same in every thread
+    if (a.want_domain >= 0 &&
+        span_outside_domain(a.lane_domain, a.lane_dom_end, bl, end, a.want_domain))
+      return;
+    agg_clear(s);
+    __syncthreads();
+    for (int64_t base = begin; base < end; base += AG_STEP) {
+      while (bl + 1 < a.n_lanes && (int64_t)a.lane_off[bl + 1] <= base) bl++;
+      if (a.want_domain >= 0 && span_outside_domain(a.lane_domain, a.lane_dom_end, bl,
+                                                    min(base + AG_STEP, end), a.want_domain))
+        continue;
+      lw.lane = bl;
+      const int64_t p0 = base + (int64_t)threadIdx.x * AG_ITEMS;
+      // all loads of the thread's four records are issued before any of them is used
+      int16_t kd[AG_ITEMS];
+      if (p0 + AG_ITEMS <= end) {
+        uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
+        const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+  #pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++) kd[j] = hq[j];
       } else {
-        agg_global_add(a, g, 1, (u64)v[j], ~vb, vb);
-        atomicAdd(&a.d_hist[(size_t)g * TA_NBINS + bin], 1u);
+  #pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++) kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
       }
-    }
-    since_flush += AG_STEP;
-    if (since_flush >= AG_FLUSH_EVERY) {
-      agg_flush(a, s);
-      since_flush = 0;
+      bool sel[AG_ITEMS];
+      i64 v[AG_ITEMS];
+      int32_t nm[AG_ITEMS];
+  #pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++) {
+        sel[j] = kd[j] >= 0 && ((a.kind_mask >> kd[j]) & 1u);
+        v[j] = 0;
+        nm[j] = 0;
+      }
+      if (a.value_sel == 0) {
+  #pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
+      } else {
+  #pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) sel[j] = a.op_n[p0 + j] > 0;
+  #pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
+      }
+  #pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++) {
+        if (!sel[j]) continue;
+        const int lane = lw.at(p0 + j);
+        const int64_t g = (int64_t)a.lane_slot[lane] * a.R + ((int64_t)nm[j] - a.min_name);
+        const u64 vb = (u64)v[j] ^ (1ull << 63);
+        const int bin = log2_bin(v[j]);
+        u32 hsh = (u32)g * 2654435761u;
+        int slot = (int)(hsh >> 24) & (AG_SLOTS - 1);
+        bool placed = false;
+        for (int probe = 0; probe < 8; probe++) {
+          int32_t cur = s.key[slot];
+          if (cur == (int32_t)g) { placed = true; break; }
+          if (cur == -1) {
+            int32_t old = atomicCAS(&s.key[slot], -1, (int32_t)g);
+            if (old == -1 || old == (int32_t)g) { placed = true; break; }
+          }
+          slot = (slot + 1) & (AG_SLOTS - 1);
+        }
+        if (placed) {
+          atomicAdd(&s.cnt[slot], 1u);
+          {  // values are durations (>= 0): 16 + 16 + 32 bit limbs, at most 32768 adds per flush
+            const u64 uv = (u64)v[j];
+            atomicAdd(&s.sum16[0][slot], (u32)(uv & 0xFFFF));
+            if (uv >> 16) atomicAdd(&s.sum16[1][slot], (u32)((uv >> 16) & 0xFFFF));
+            if (uv >> 32) atomicAdd(&s.sum16[2][slot], (u32)(uv >> 32));
+          }
+          // 64-bit min/max in shared memory are compare-and-swap loops: skip them unless the
+          // value would actually move the extreme (rare once a slot has seen a few records)
+          if (~vb > s.minc[slot]) atomicMax(&s.minc[slot], ~vb);
+          if (vb > s.maxb[slot]) atomicMax(&s.maxb[slot], vb);
+          // 16-bit bins packed two per word
+          u32 *hw = reinterpret_cast<u32 *>(&s.hist[slot][0]) + (bin >> 1);
+          atomicAdd(hw, (bin & 1) ? 0x10000u : 1u);
+        } else {
+          agg_global_add(a, g, 1, (u64)v[j], ~vb, vb);
+          atomicAdd(&a.d_hist[(size_t)g * TA_NBINS + bin], 1u);
+        }
+      }
+      since_flush += AG_STEP;
+      if (since_flush >= AG_FLUSH_EVERY) {
+        agg_flush(a, s);
+        since_flush = 0;
+      }
     }
   }
   agg_flush(a, s);
@@ -242,12 +264,14 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot;
   a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
   a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
-  int64_t blocks = 148 * 6;
-  int64_t chunk = (h->n_valid + blocks - 1) / blocks;
-  chunk = ((chunk + AG_STEP - 1) / AG_STEP) * AG_STEP;
-  if (chunk < AG_STEP) chunk = AG_STEP;
-  blocks = (h->n_valid + chunk - 1) / chunk;
-  a.chunk = chunk;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
+  const bool host_kinds = (a.kind_mask & 7u) != 0, dev_kinds = (a.kind_mask & 56u) != 0;
+  a.want_domain = host_kinds && dev_kinds ? -1 : (dev_kinds ? 1 : 0);
+  a.chunk = AG_ITEM;
+  a.n_items = (unsigned)((h->n_valid + a.chunk - 1) / a.chunk);
+  a.spread = a.n_items < 148u * 6u ? a.n_items : 148u * 6u;
+  a.per = (a.n_items + a.spread - 1) / a.spread;
+  const int64_t blocks = (int64_t)a.spread * a.per;
   k_agg<<<TA_N (unsigned)blocks, AG_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   u64 ng = 0;

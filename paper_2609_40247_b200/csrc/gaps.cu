@@ -26,6 +26,7 @@ struct GapArgs {
   const int16_t *kind;
   const int32_t *lane_off, *lane_window;
   const int16_t *lane_domain;
+  const int32_t *lane_dom_end;
   const int64_t *t0, *t1;
   i64 min_gap;
   int list_only;  // second run: only (re)write the long-gap list
@@ -75,9 +76,26 @@ __global__ void __launch_bounds__(GP_THREADS, 3) k_gaps(GapArgs a) {
     if (tile_start < a.n_valid && a.n_lanes > 0) l = warp_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (tid == 0) s_lane0 = l;
   }
+  __syncthreads();
+  const int l0 = s_lane0;
+  const bool full = p0 + GP_ITEMS <= a.n;
+  if (l0 >= 0 && span_outside_domain(a.lane_domain, a.lane_dom_end, l0,
+                                     min(tile_start + GP_TILE, a.n_valid), 1)) {
+    // host lanes only: no gaps here, and no later device lane can use anything scanned so far
+    if (tid == 0) st_relaxed(&a.st_max[tile], td_pack(TD_PREFIX, 0));
+    if (a.list_only) return;
+    if (full) {
+      longlong2 *pg = reinterpret_cast<longlong2 *>(a.gap_before + p0);
+#pragma unroll
+      for (int j = 0; j < GP_ITEMS / 2; j++) pg[j] = make_longlong2(0, 0);
+    } else {
+      for (int j = 0; j < GP_ITEMS; j++)
+        if (p0 + j < a.n) a.gap_before[p0 + j] = 0;
+    }
+    return;
+  }
   // kinds of the thread's eight records (0 = not a device record of the window)
   int16_t kd[GP_ITEMS];
-  const bool full = p0 + GP_ITEMS <= a.n;
   if (full) {
     uint4 q = *reinterpret_cast<const uint4 *>(a.kind + p0);
     const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
@@ -112,8 +130,6 @@ __global__ void __launch_bounds__(GP_THREADS, 3) k_gaps(GapArgs a) {
         if (p0 + j < a.n) { s[j] = a.ts[p0 + j]; ce[j] = a.te[p0 + j]; }
     }
   }
-  __syncthreads();
-  const int l0 = s_lane0;
   // lanes of the items: walk forward from the tile's first lane
   int ln[GP_ITEMS];
   u64 run = 0;
@@ -310,7 +326,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   a.n = n; a.n_valid = h->n_valid; a.n_lanes = L;
   a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end; a.kind = h->sorted.kind;
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window;
-  a.lane_domain = h->sorted.lane_domain; a.t0 = h->d_t0; a.t1 = h->d_t1;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end; a.t0 = h->d_t0; a.t1 = h->d_t1;
   a.min_gap = min_gap; a.list_only = 0;
   a.gap_before = gap_before; a.lane_gaps = lane_gaps; a.lane_hist = lane_hist; a.win_hist = win_hist;
   a.list = ulist; a.list_key = ukeys; a.list_cap = cap; a.st_max = st_max;

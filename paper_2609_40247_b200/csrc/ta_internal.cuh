@@ -86,6 +86,7 @@ struct ta_window {
   ta_sort_result sorted;
   int32_t *d_lane_code;      // per lane: window << tbits | triple rank
   int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
+  int32_t *d_lane_dom_end;   // per lane: first position behind the run of lanes of the same domain
   i64 *d_slot_min, *d_slot_max;               // per slot: corr_id range of its LAUNCH records
   std::vector<int64_t> h_slot_min, h_slot_max;  // host copies (INT64_MAX / INT64_MIN when none)
 
@@ -288,6 +289,12 @@ __device__ __forceinline__ u64 block_scan_exclusive(u64 v, Op op, u64 *smem, u64
   return ex;
 }
 
+// True when no record of [p, p_end) lies in a lane of domain `want`; l = lane of p.
+__device__ __forceinline__ bool span_outside_domain(const int16_t *lane_domain,
+                                                    const int32_t *lane_dom_end, int l,
+                                                    int64_t p_end, int want) {
+  return lane_domain[l] != want && (int64_t)lane_dom_end[l] >= p_end;
+}
 // Lane of a sorted position: binary search in lane_off (n_lanes + 1 entries).
 __device__ __forceinline__ int lane_of_pos(const int32_t *lane_off, int n_lanes, int64_t p) {
   int lo = 0, hi = n_lanes - 1;

@@ -181,7 +181,8 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
                                                      int32_t *lane_pid, int16_t *lane_stream,
                                                      int16_t *lane_domain, int32_t *lane_off,
                                                      int32_t *lane_code, int32_t *lane_slot,
-                                                     int32_t *n_lanes_out, int64_t cap) {
+                                                     int32_t *lane_dom_end, int32_t *n_lanes_out,
+                                                     int64_t cap) {
   __shared__ u64 tmp[33];
   __shared__ u64 base;
   if (threadIdx.x == 0) base = 0;
@@ -213,6 +214,15 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
     int64_t L = (int64_t)base;
     if (L < cap + 1) lane_off[L] = (int32_t)n_valid;
     *n_lanes_out = (int32_t)L;
+  }
+  __syncthreads();
+  // per lane: the first position behind the run of lanes of its domain (host and device lanes
+  // alternate per (window, pid), so the runs are a few lanes long)
+  const int64_t L = (int64_t)base < cap ? (int64_t)base : cap;
+  for (int64_t l = threadIdx.x; l < L; l += blockDim.x) {
+    int64_t m = l + 1;
+    while (m < L && lane_domain[m] == lane_domain[l]) m++;
+    lane_dom_end[l] = m < L ? lane_off[m] : (int32_t)n_valid;
   }
 }
 
@@ -309,7 +319,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
 
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
-                2 * Carver::pad(n * 2) + 4 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
+                2 * Carver::pad(n * 2) + 5 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
                 Carver::pad((lane_cap + 1) * 4) + 2 * Carver::pad((size_t)n_slots * 8) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
@@ -322,6 +332,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *lane_code = ck.take<int32_t>(lane_cap), *lane_slot = ck.take<int32_t>(lane_cap);
   int16_t *lane_stream = ck.take<int16_t>(lane_cap), *lane_domain = ck.take<int16_t>(lane_cap);
   int32_t *lane_off = ck.take<int32_t>(lane_cap + 1);
+  int32_t *lane_dom_end = ck.take<int32_t>(lane_cap);
   int32_t *n_lanes_dev = ck.take<int32_t>(1);
   h->d_slot_min = ck.take<i64>(n_slots);
   h->d_slot_max = ck.take<i64>(n_slots);
@@ -433,7 +444,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
                                    h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
                                    lane_window, lane_pid, lane_stream, lane_domain, lane_off,
-                                   lane_code, lane_slot, n_lanes_dev, lane_cap);
+                                   lane_code, lane_slot, lane_dom_end, n_lanes_dev, lane_cap);
   TA_CHECK_CUDA(h, cudaGetLastError());
   int32_t n_lanes = 0;
   TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
@@ -454,5 +465,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   r.lane_domain = lane_domain; r.lane_off = lane_off;
   h->d_lane_code = lane_code;
   h->d_lane_slot = lane_slot;
+  h->d_lane_dom_end = lane_dom_end;
   return TA_OK;
 }
