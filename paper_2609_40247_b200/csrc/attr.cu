@@ -32,6 +32,12 @@
 #define AT_ITEMS 8
 #define AT_TILE (AT_THREADS * AT_ITEMS)
 #define AT_CAP 16
+#ifndef AT_RES_MINB
+#define AT_RES_MINB 3
+#endif
+#ifndef AT_OPS_MINB
+#define AT_OPS_MINB 3
+#endif
 #define AT_NONE (-1)
 #define AT_UNRESOLVED (-2)
 
@@ -275,8 +281,11 @@ __global__ void __launch_bounds__(128) k_attr_carry(AttrArgs a) {
 }
 
 // ---- kernel 3: parent and depth of every host record -----------------------------
-struct AttrSmem {
-  i64 leaf[AT_TILE];              // OP end time, INT64_MIN elsewhere
+// a thread's eight leaves are followed by one pad entry: the threads of a warp then touch
+// distinct banks when each walks its own records
+#define AT_LX(x) ((x) + ((x) >> 3))
+struct __align__(16) AttrSmem {
+  i64 leaf[AT_TILE + AT_TILE / 8];  // OP end time, INT64_MIN elsewhere; index through AT_LX
   i64 T[2 * AT_THREADS];          // max-tree over the threads' maxima, leaves at [AT_THREADS, 2*AT_THREADS)
   int16_t parent_local[AT_TILE];
   uint8_t kcarry[AT_TILE];
@@ -285,7 +294,7 @@ struct AttrSmem {
   int lane0, lane1, dmax;
 };
 
-__global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
+__global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrArgs a) {
   __shared__ AttrSmem s;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x;
@@ -334,6 +343,7 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
   int ln[AT_ITEMS];
   int lo_local[AT_ITEMS];  // first tile-local index of the record's lane (-1: the lane began earlier)
   i64 m8 = INT64_MIN;
+  unsigned opmask = 0;  // the thread's own OP records (its leaves are their en[])
   {
     int l = l0;
     int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
@@ -348,9 +358,9 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
         while (p >= next_off) { l++; cur_off = next_off; next_off = a.lane_off[l + 1]; }
         ln[j] = l;
         lo_local[j] = cur_off < tile_start ? -1 : (int)(cur_off - tile_start);
-        if (kd[j] == TA_KIND_OP) leaf = en[j];
+        if (kd[j] == TA_KIND_OP) { leaf = en[j]; opmask |= 1u << j; }
       }
-      s.leaf[x0 + j] = leaf;
+      s.leaf[AT_LX(x0 + j)] = leaf;
       m8 = leaf > m8 ? leaf : m8;
     }
     const int64_t plast = min(tile_start + AT_TILE, a.n_valid) - 1;
@@ -388,38 +398,60 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
   }
   __syncthreads();
 
-  // nearest earlier OP that is still running when the record starts
+  // nearest earlier OP that is still running when the record starts.  Consecutive records
+  // mostly share it: when the threshold t did not go down since the previous record, nothing
+  // between the previous answer and that record can qualify, so the previous answer (or the
+  // fact that the tile holds none) is reused and the tree is only walked when it has ended.
   unsigned bad = 0;
   int32_t par_abs[AT_ITEMS];
+  int16_t plv[AT_ITEMS];
+  uint8_t kc[AT_ITEMS];
+  bool have = false;  // (tq, yq, yeq): threshold and answer of the previous search outside the thread
+  i64 tq = 0, yeq = 0;
+  int yq = -1;
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) {
     const int x = x0 + j;
     int pl = AT_NONE;
     par_abs[j] = -1;
+    kc[j] = 0;
     if (hostmask & (1u << j)) {
       const i64 t = en[j] > st[j] ? st[j] + 1 : en[j];
       int y = -1;
-      for (int k = x - 1; k >= x0; k--)
-        if (s.leaf[k] >= t) { y = k; break; }
+      i64 ye = 0;  // end time of y
+#pragma unroll
+      for (int jj = AT_ITEMS - 1; jj >= 0; jj--)
+        if (jj < j && y < 0 && (opmask & (1u << jj)) && en[jj] >= t) { y = x0 + jj; ye = en[jj]; }
       if (y < 0) {
-        int pos = AT_THREADS + tid;
-        while (pos > 1) {
-          if ((pos & 1) && s.T[pos - 1] >= t) {
-            pos = pos - 1;
-            while (pos < AT_THREADS) pos = s.T[2 * pos + 1] >= t ? 2 * pos + 1 : 2 * pos;
-            const int tb = (pos - AT_THREADS) * AT_ITEMS;
-            for (int k = tb + AT_ITEMS - 1; k >= tb; k--)
-              if (s.leaf[k] >= t) { y = k; break; }
-            break;
+        if (have && t >= tq && (yq < 0 || yeq >= t)) {
+          y = yq;
+          ye = yeq;
+        } else {
+          int pos = AT_THREADS + tid;
+          while (pos > 1) {
+            if ((pos & 1) && s.T[pos - 1] >= t) {
+              pos = pos - 1;
+              while (pos < AT_THREADS) pos = s.T[2 * pos + 1] >= t ? 2 * pos + 1 : 2 * pos;
+              const int tb = (pos - AT_THREADS) * AT_ITEMS;
+              for (int k = tb + AT_ITEMS - 1; k >= tb; k--) {
+                ye = s.leaf[AT_LX(k)];
+                if (ye >= t) { y = k; break; }
+              }
+              break;
+            }
+            pos >>= 1;
           }
-          pos >>= 1;
+          have = true;
+          yq = y;
+          yeq = ye;
         }
+        tq = t;
       }
       const int lo = lo_local[j];
       if (y >= 0 && y >= lo) {
         pl = y;
         par_abs[j] = (int32_t)(tile_start + y);
-        if (s.leaf[y] < en[j]) bad |= 1u << j;
+        if (ye < en[j]) bad |= 1u << j;
       } else if (lo >= 0) {
         pl = AT_NONE;
       } else {  // the encloser, if any, lies before the tile: the carried stack has it
@@ -427,28 +459,53 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
         int k = 0;
         while (k < ccnt && s.carry_e[k] >= t) k++;
         s.kcarry[x] = (uint8_t)k;
+        kc[j] = (uint8_t)k;
         if (k > 0) {
           par_abs[j] = s.carry_pos[k - 1];
           if (s.carry_e[k - 1] < en[j]) bad |= 1u << j;
         }
       }
     }
-    s.parent_local[x] = (int16_t)pl;
+    plv[j] = (int16_t)pl;
+  }
+  {
+    uint4 q;
+    q.x = (u32)(uint16_t)plv[0] | ((u32)(uint16_t)plv[1] << 16);
+    q.y = (u32)(uint16_t)plv[2] | ((u32)(uint16_t)plv[3] << 16);
+    q.z = (u32)(uint16_t)plv[4] | ((u32)(uint16_t)plv[5] << 16);
+    q.w = (u32)(uint16_t)plv[6] | ((u32)(uint16_t)plv[7] << 16);
+    *reinterpret_cast<uint4 *>(&s.parent_local[x0]) = q;
   }
   __syncthreads();
+  // depth = level in the parent forest; the chain is only followed through shared memory when
+  // the parent is another thread's record and differs from the previous record's parent
   int dmax = 0;
   uint8_t dep[AT_ITEMS];
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) {
     int d = 0;
     if (hostmask & (1u << j)) {
-      int c = x0 + j;
-      for (int it = 0; it < 300; it++) {
-        const int pl = s.parent_local[c];
-        if (pl == AT_NONE) break;
-        if (pl == AT_UNRESOLVED) { d += s.kcarry[c]; break; }
-        d++;
-        c = pl;
+      const int pl = plv[j];
+      if (pl == AT_UNRESOLVED) {
+        d = kc[j];
+      } else if (pl >= x0) {  // one of the thread's own earlier records
+#pragma unroll
+        for (int jj = 0; jj < AT_ITEMS; jj++)
+          if (jj < j && pl == x0 + jj) d = dep[jj] + 1;
+      } else if (pl >= 0) {
+        if (j > 0 && (hostmask & (1u << (j > 0 ? j - 1 : 0))) && plv[j > 0 ? j - 1 : 0] == pl) {
+          d = dep[j > 0 ? j - 1 : 0];
+        } else {
+          d = 1;
+          int c = pl;
+          for (int it = 0; it < 300; it++) {
+            const int q = s.parent_local[c];
+            if (q == AT_NONE) break;
+            if (q == AT_UNRESOLVED) { d += s.kcarry[c]; break; }
+            d++;
+            c = q;
+          }
+        }
       }
       if (d > 255) d = 255;
       dmax = max(dmax, d);
@@ -485,7 +542,7 @@ __global__ void __launch_bounds__(AT_THREADS, 3) k_attr_resolve(AttrArgs a) {
 }
 
 // ---- device records inherit the operator of their launch ------------------------
-__global__ void __launch_bounds__(AT_THREADS, 3) k_attr_ops(AttrArgs a) {
+__global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a) {
   __shared__ u64 red[AT_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
   const int tid = threadIdx.x, lane = tid & 31;

@@ -16,6 +16,9 @@
 
 #define GP_THREADS 256
 #define GP_ITEMS 8
+#ifndef GP_MINB
+#define GP_MINB 4
+#endif
 #define GP_TILE (GP_THREADS * GP_ITEMS)
 #define GP_LOW ((1ull << 40) - 1)
 
@@ -58,7 +61,7 @@ __device__ __forceinline__ int warp_lane_search(const int32_t *lane_off, int n_l
   return lo;
 }
 
-__global__ void __launch_bounds__(GP_THREADS, 3) k_gaps(GapArgs a) {
+__global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   __shared__ u64 tmp[33];
   __shared__ u64 red[4][GP_THREADS / 32];
   __shared__ u64 s_excl_max;

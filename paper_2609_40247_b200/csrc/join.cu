@@ -150,10 +150,13 @@ __device__ __forceinline__ int32_t winner_of(const JoinArgs &a, int64_t p, int s
 // ---- pass 2: probes ----------------------------------------------------------
 // 256 threads x 8 consecutive positions; every output column is written once.
 #define JP_THREADS 256
+#ifndef JP_MINB
+#define JP_MINB 3
+#endif
 #define JP_TILE (JP_THREADS * 8)
 
 template <bool DIRECT>
-__global__ void __launch_bounds__(JP_THREADS, 3) k_join_probe(JoinArgs a) {
+__global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) {
   __shared__ u64 red[7][JP_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
   const int tid = threadIdx.x, lane = tid & 31;

@@ -14,8 +14,12 @@
 #include "ta_internal.cuh"
 
 #define RS_BINS 256
-#ifndef RS_MINB
-#define RS_MINB 2  // resident CTAs per SM the register budget is sized for
+// resident CTAs per SM the register budget is sized for (pairs, keys only)
+#ifndef RSP_MINB
+#define RSP_MINB 2
+#endif
+#ifndef RSK_MINB
+#define RSK_MINB 4
 #endif
 
 struct RadixArgs {
@@ -104,15 +108,29 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
       run += t;
     }
   }
-  // chained scan over tiles, one digit per thread
+  // chained scan over tiles, one digit per thread: the tile's own count is published first,
+  // the keys are staged in shared memory in digit order (which needs tile-local offsets only),
+  // and the look back over the earlier tiles comes last, when they have had time to publish
+  u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
   if (tid < (1 << BITS)) {
-    u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
+    if (tile == 0) st_relaxed(st, td_pack(TD_PREFIX, (u64)a.bin_offset[tid] + cnt));
+    else st_relaxed(st, td_pack(TD_AGG, cnt));
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < ITEMS; j++) {
+    if (FULL || (wbase + j * 32 + lane) < count) {
+      const u32 d = (u32)rd[j] & 0xFFu;
+      const int r = (rd[j] >> 8) + (int)wh[d];
+      rd[j] = r;
+      s.keys[r] = key[j];
+    }
+  }
+  if (tid < (1 << BITS)) {
     u64 excl;
     if (tile == 0) {
       excl = a.bin_offset[tid];
-      st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
     } else {
-      st_relaxed(st, td_pack(TD_AGG, cnt));
       excl = 0;
       bool timed_out = false;
       for (int t = tile - 1;; --t) {
@@ -127,17 +145,6 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   }
   __syncthreads();
   if (s.fail) return;
-  // stage keys in shared memory in digit order
-#pragma unroll
-  for (int j = 0; j < ITEMS; j++) {
-    if (FULL || (wbase + j * 32 + lane) < count) {
-      const u32 d = (u32)rd[j] & 0xFFu;
-      const int r = (rd[j] >> 8) + (int)wh[d];
-      rd[j] = r;
-      s.keys[r] = key[j];
-    }
-  }
-  __syncthreads();
   u32 gpos[VALS ? ITEMS : 1];
 #pragma unroll
   for (int k = 0; k < ITEMS; k++) {
@@ -167,7 +174,7 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
 }
 
 template <int THREADS, int ITEMS, bool VALS, int BITS>
-__global__ void __launch_bounds__(THREADS, RS_MINB) k_radix_pass(RadixArgs a) {
+__global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_pass(RadixArgs a) {
   constexpr int TILE = THREADS * ITEMS;
   extern __shared__ __align__(16) unsigned char smem_raw[];
   RadixSmem<THREADS, ITEMS> &s = *reinterpret_cast<RadixSmem<THREADS, ITEMS> *>(smem_raw);
@@ -188,7 +195,7 @@ __global__ void __launch_bounds__(THREADS, RS_MINB) k_radix_pass(RadixArgs a) {
 #define RSP_THREADS 384  // pairs
 #define RSP_ITEMS 12
 #ifndef RSK_THREADS
-#define RSK_THREADS 384  // keys only
+#define RSK_THREADS 256  // keys only
 #endif
 #ifndef RSK_ITEMS
 #define RSK_ITEMS 16
