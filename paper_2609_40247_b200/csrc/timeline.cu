@@ -96,33 +96,62 @@ struct GatherArgs {
   int32_t *pid, *name, *seq;
   int16_t *stream, *kind;
   int32_t *lane_start;  // per lane code, -1 = empty
+  int32_t *status;
 };
+__device__ __forceinline__ u32 gather_index(u64 k, const GatherArgs &a) {
+  const int w = a.wbits ? (int)((k >> a.wshift) & ((1ull << a.wbits) - 1)) : 0;
+  return (u32)(a.off[w] + (int64_t)(k & ((1ull << a.ibits) - 1)));
+}
 
 __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   __shared__ int s_slot[8];
   __shared__ u64 s_mx[8], s_mn[8];
-  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   int slot = -1;
   u64 mx = 0, mn_inv = 0;
   if (p < a.n) {
   u32 idx;
+  int64_t dst = p;  // where the record goes: p, or its place inside a run of equal coarse keys
+  int before = 0, after = 0;
   if (a.packed && p < a.n_valid) {
     const u64 k = a.keys[p];
-    const int w = a.wbits ? (int)((k >> a.wshift) & ((1ull << a.wbits) - 1)) : 0;
-    idx = (u32)(a.off[w] + (int64_t)(k & ((1ull << a.ibits) - 1)));
-    a.perm[p] = idx;
+    idx = gather_index(k, a);
+    // packed keys order the records down to a coarse time only: members of a run of equal
+    // (lane, coarse time) sit in input order and are ranked here by (ts_start, -ts_end)
+    const u64 hk = k >> a.ibits;
+    while (before <= TA_TIE_RUN_MAX && p - before > 0 && (a.keys[p - before - 1] >> a.ibits) == hk)
+      before++;
+    while (after <= TA_TIE_RUN_MAX && p + after + 1 < a.n_valid &&
+           (a.keys[p + after + 1] >> a.ibits) == hk)
+      after++;
+    if (before + after + 1 > TA_TIE_RUN_MAX) {
+      a.status[ST_LONG_RUN] = 1;  // the caller starts over with full-resolution keys
+      before = after = 0;
+    }
   } else {
     idx = a.perm[p];
   }
   Rec r = load_rec(a.ev, idx);
-  a.ts_start[p] = r.ts_start;
-  a.ts_end[p] = r.ts_end;
-  a.corr[p] = r.corr;
-  a.pid[p] = r.pid;
-  a.name[p] = r.name;
-  a.seq[p] = r.seq;
-  a.stream[p] = r.stream;
-  a.kind[p] = r.kind;
+  if (before + after > 0) {
+    int rank = 0;
+    for (int q = -before; q <= after; q++) {
+      if (q == 0) continue;
+      const i64 *o = reinterpret_cast<const i64 *>(a.ev) + (int64_t)gather_index(a.keys[p + q], a) * 5;
+      const i64 os = o[0], oe = o[1];
+      const bool first = os < r.ts_start || (os == r.ts_start && (oe > r.ts_end || (oe == r.ts_end && q < 0)));
+      rank += first ? 1 : 0;
+    }
+    dst = p - before + rank;
+  }
+  if (a.packed && p < a.n_valid) a.perm[dst] = idx;
+  a.ts_start[dst] = r.ts_start;
+  a.ts_end[dst] = r.ts_end;
+  a.corr[dst] = r.corr;
+  a.pid[dst] = r.pid;
+  a.name[dst] = r.name;
+  a.seq[dst] = r.seq;
+  a.stream[dst] = r.stream;
+  a.kind[dst] = r.kind;
   if (p < a.n_valid) {
     u64 code = a.keys[p] >> a.sbits;
     if (p == 0 || (a.keys[p - 1] >> a.sbits) != code) a.lane_start[code] = (int32_t)p;
@@ -226,7 +255,7 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
   }
 }
 
-// ---- packed keys: equal (lane, coarse time) runs, ordered by (ts_start, -ts_end, index) --
+// ---- packed keys: index of the record a key stands for -------------------------
 struct PackInfo {
   int ibits, wshift, wbits;
   const int64_t *off;
@@ -234,73 +263,6 @@ struct PackInfo {
 __device__ __forceinline__ u32 packed_index(u64 k, const PackInfo &pi) {
   const int w = pi.wbits ? (int)((k >> pi.wshift) & ((1ull << pi.wbits) - 1)) : 0;
   return (u32)(pi.off[w] + (int64_t)(k & ((1ull << pi.ibits) - 1)));
-}
-__global__ void __launch_bounds__(256) k_fix_ties_packed(u64 *keys, int64_t n_valid, const ta_event *ev,
-                                                         PackInfo pi, int32_t *status) {
-  int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (p >= n_valid || p + 1 >= n_valid) return;
-  const u64 k = keys[p];
-  const u64 hk = k >> pi.ibits;
-  if ((keys[p + 1] >> pi.ibits) != hk) return;
-  if (p > 0 && (keys[p - 1] >> pi.ibits) == hk) return;
-  int len = 2;
-  while (p + len < n_valid && len <= TA_TIE_RUN_MAX && (keys[p + len] >> pi.ibits) == hk) len++;
-  if (len > TA_TIE_RUN_MAX) {
-    status[ST_LONG_RUN] = 1;
-    return;
-  }
-  if (len <= 4) {
-    // short runs (the common case) stay in registers: all loads first, then a tiny network
-    u64 kk[4];
-    i64 st[4], en[4];
-#pragma unroll
-    for (int i = 0; i < 4; i++) kk[i] = i < len ? keys[p + i] : 0;
-#pragma unroll
-    for (int i = 0; i < 4; i++) {
-      st[i] = LLONG_MAX;  // padding sorts last and is never written back
-      en[i] = LLONG_MIN;
-      if (i < len) {
-        const i64 *r = reinterpret_cast<const i64 *>(ev) + (int64_t)packed_index(kk[i], pi) * 5;
-        st[i] = r[0];
-        en[i] = r[1];
-      }
-    }
-    // stable: bubble passes that only swap strictly out-of-order neighbours
-#pragma unroll
-    for (int pass = 0; pass < 3; pass++)
-#pragma unroll
-      for (int i = 0; i < 3 - pass; i++) {
-        const bool sw = st[i] > st[i + 1] || (st[i] == st[i + 1] && en[i] < en[i + 1]);
-        if (sw) {
-          u64 tk = kk[i]; kk[i] = kk[i + 1]; kk[i + 1] = tk;
-          i64 ts = st[i]; st[i] = st[i + 1]; st[i + 1] = ts;
-          i64 te = en[i]; en[i] = en[i + 1]; en[i + 1] = te;
-        }
-      }
-#pragma unroll
-    for (int i = 0; i < 4; i++)
-      if (i < len) keys[p + i] = kk[i];
-    return;
-  }
-  u64 kk[TA_TIE_RUN_MAX];
-  i64 st[TA_TIE_RUN_MAX], en[TA_TIE_RUN_MAX];
-  for (int i = 0; i < len; i++) kk[i] = keys[p + i];
-  for (int i = 0; i < len; i++) {
-    const i64 *r = reinterpret_cast<const i64 *>(ev) + (int64_t)packed_index(kk[i], pi) * 5;
-    st[i] = r[0];
-    en[i] = r[1];
-  }
-  for (int i = 1; i < len; i++) {  // stable insertion sort: ts_start ascending, ts_end descending
-    u64 xk = kk[i];
-    i64 xs = st[i], xe = en[i];
-    int j = i - 1;
-    while (j >= 0 && (st[j] > xs || (st[j] == xs && en[j] < xe))) {
-      kk[j + 1] = kk[j]; st[j + 1] = st[j]; en[j + 1] = en[j];
-      j--;
-    }
-    kk[j + 1] = xk; st[j + 1] = xs; en[j + 1] = xe;
-  }
-  for (int i = 0; i < len; i++) keys[p + i] = kk[i];
 }
 __global__ void __launch_bounds__(256) k_unpack_tail(const u64 *keys, int64_t n_valid, int64_t n,
                                                      PackInfo pi, u32 *perm) {
@@ -336,10 +298,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *n_lanes_dev = ck.take<int32_t>(1);
   h->d_slot_min = ck.take<i64>(n_slots);
   h->d_slot_max = ck.take<i64>(n_slots);
-  h->h_slot_min.assign((size_t)n_slots, INT64_MAX);
-  h->h_slot_max.assign((size_t)n_slots, INT64_MIN);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_min, h->h_slot_min.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_max, h->h_slot_max.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
 
   // temporaries (released at the end of the call)
   size_t tmp_bytes = 2 * Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
@@ -352,105 +310,110 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *lane_start = ct.take<int32_t>(n_codes);
   void *sort_tmp = ct.base + ct.off;
 
-  TA_CHECK_CUDA(h, cudaMemsetAsync(lane_start, 0xFF, n_codes * sizeof(int32_t), st));
-  if (n > 0) {
+  int32_t n_lanes = 0;
+  // Packed keys settle the order down to a coarse time; the gather ranks the members of a run
+  // of equal coarse keys itself.  A run too long for that is reported at the end, and the
+  // second attempt sorts (key, index) pairs at full time resolution.
+  for (int attempt = 0; attempt < 2; attempt++) {
     int32_t words[ST_WORDS];
-    if (h->packed) {
-      // keys carry the index: 8-byte elements, fewer bytes per pass
-      PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
-      TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp));
-      if (h->n_valid > 1)
-        k_fix_ties_packed<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, h->events, pi,
-                                                                 h->d_status);
-      TA_TRY(ta_read_status(h, words));
-      if (words[ST_ERR]) return (ta_status)words[ST_ERR];
-      if (words[ST_LONG_RUN]) {
-        // a long run of equal coarse keys: start over with (key, index) pairs at full resolution
-        TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status + ST_LONG_RUN, 0, sizeof(int32_t), st));
-        TA_TRY(ta_launch_load(h, false));
-      } else if (n > h->n_valid) {
-        k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm);
+    h->h_slot_min.assign((size_t)n_slots, INT64_MAX);
+    h->h_slot_max.assign((size_t)n_slots, INT64_MIN);
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_min, h->h_slot_min.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_max, h->h_slot_max.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+    TA_CHECK_CUDA(h, cudaMemsetAsync(lane_start, 0xFF, n_codes * sizeof(int32_t), st));
+    if (n > 0) {
+      if (h->packed) {
+        // keys carry the index: 8-byte elements, fewer bytes per pass
+        PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
+        TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp));
+        if (n > h->n_valid)
+          k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm);
       }
-    }
-    if (!h->packed) {
-      // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
-      TA_TRY(ta_radix_sort_pairs(h, h->d_keys, nullptr, kscr, vscr, skeys, perm, n, h->plan,
-                                 h->d_hist, sort_tmp));
-      // step 2: equal-key runs
-      if (h->n_valid > 1)
-        k_fix_ties<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
-                                                          h->d_status);
-      TA_TRY(ta_read_status(h, words));
-      if (words[ST_ERR]) return (ta_status)words[ST_ERR];
-      if (words[ST_LONG_RUN]) {
-        // redo with the duration as a least-significant key: first a stable sort by
-        // (max_dur - duration), then the timeline key on top of that order
-        void *xb = ta_dalloc(h, Carver::pad(n * 8) + Carver::pad(n * 4));
+      if (!h->packed) {
+        // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
+        TA_TRY(ta_radix_sort_pairs(h, h->d_keys, nullptr, kscr, vscr, skeys, perm, n, h->plan,
+                                   h->d_hist, sort_tmp));
+        // step 2: equal-key runs
+        if (h->n_valid > 1)
+          k_fix_ties<<<TA_N nblk(h->n_valid, 256), 256, 0, st>>>(skeys, perm, h->n_valid, h->events,
+                                                            h->d_status);
+        TA_TRY(ta_read_status(h, words));
+        if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+        if (words[ST_LONG_RUN]) {
+          TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status + ST_LONG_RUN, 0, sizeof(int32_t), st));
+          // redo with the duration as a least-significant key: first a stable sort by
+          // (max_dur - duration), then the timeline key on top of that order
+          void *xb = ta_dalloc(h, Carver::pad(n * 8) + Carver::pad(n * 4));
+          if (!xb) return TA_ERR_OOM;
+          Carver cx(xb);
+          u64 *dkeys = cx.take<u64>(n);
+          u32 *dorder = cx.take<u32>(n);
+          const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
+          k_duration_key<<<TA_N nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit,
+                                                       h->max_dur, dkeys);
+          int dbits = 1;
+          while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
+          SortPlan dplan = ta_make_plan(0, dbits);
+          TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
+                                     sort_tmp));
+          k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
+          TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
+                                     sort_tmp));
+          TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+          ta_dfree(h, xb);
+        }
+      }
+      // step 3: dropped tail, chain of stable sorts over the full tuple (least
+      // significant field first); perm[n_valid..n) holds the tail in input order
+      const int64_t m = n - h->n_valid;
+      if (m > 1) {
+        void *xb = ta_dalloc(h, 2 * Carver::pad(m * 8) + Carver::pad(m * 4));
         if (!xb) return TA_ERR_OOM;
         Carver cx(xb);
-        u64 *dkeys = cx.take<u64>(n);
-        u32 *dorder = cx.take<u32>(n);
-        const u64 dropped_bit = h->has_dropped ? 1ull << (h->sbits + h->tbits + h->wbits) : 0ull;
-        k_duration_key<<<TA_N nblk(n, 256), 256, 0, st>>>(h->events, n, h->d_keys, dropped_bit,
-                                                     h->max_dur, dkeys);
-        int dbits = 1;
-        while (dbits < 63 && (h->max_dur >> dbits) != 0) dbits++;
-        SortPlan dplan = ta_make_plan(0, dbits);
-        TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
-                                   sort_tmp));
-        k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
-        TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
-                                   sort_tmp));
+        u64 *tk = cx.take<u64>(m), *tk2 = cx.take<u64>(m);
+        u32 *alt = cx.take<u32>(m);
+        u32 *cur = perm + h->n_valid, *nxt = alt;
+        for (int stage = 0; stage < 4; stage++) {
+          if (stage == 3 && h->W == 1) break;
+          k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
+          int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : 64;
+          SortPlan tp = ta_make_plan(0, bits);
+          TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
+          u32 *t = cur; cur = nxt; nxt = t;
+        }
+        if (cur != perm + h->n_valid)
+          TA_CHECK_CUDA(h, cudaMemcpyAsync(perm + h->n_valid, cur, m * sizeof(u32),
+                                           cudaMemcpyDeviceToDevice, st));
         TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
         ta_dfree(h, xb);
       }
+      // step 4
+      GatherArgs g;
+      g.ev = h->events; g.perm = perm; g.keys = skeys; g.n = n; g.n_valid = h->n_valid;
+      g.packed = h->packed; g.ibits = h->ibits; g.wbits = h->wbits; g.off = h->d_off;
+      g.wshift = h->ibits + h->tbits + (h->sbits - h->dshift);
+      g.sbits = h->packed ? h->ibits + (h->sbits - h->dshift) : h->sbits;
+      g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
+      g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
+      g.tt = h->d_triples; g.tbits = h->tbits; g.n_pids = h->n_pids > 0 ? h->n_pids : 1;
+      g.slot_min = h->d_slot_min; g.slot_max = h->d_slot_max; g.status = h->d_status;
+      k_gather<<<TA_N nblk(n, 256), 256, 0, st>>>(g);
     }
-    // step 3: dropped tail, chain of stable sorts over the full tuple (least
-    // significant field first); perm[n_valid..n) holds the tail in input order
-    const int64_t m = n - h->n_valid;
-    if (m > 1) {
-      void *xb = ta_dalloc(h, 2 * Carver::pad(m * 8) + Carver::pad(m * 4));
-      if (!xb) return TA_ERR_OOM;
-      Carver cx(xb);
-      u64 *tk = cx.take<u64>(m), *tk2 = cx.take<u64>(m);
-      u32 *alt = cx.take<u32>(m);
-      u32 *cur = perm + h->n_valid, *nxt = alt;
-      for (int stage = 0; stage < 4; stage++) {
-        if (stage == 3 && h->W == 1) break;
-        k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
-        int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : 64;
-        SortPlan tp = ta_make_plan(0, bits);
-        TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
-        u32 *t = cur; cur = nxt; nxt = t;
-      }
-      if (cur != perm + h->n_valid)
-        TA_CHECK_CUDA(h, cudaMemcpyAsync(perm + h->n_valid, cur, m * sizeof(u32),
-                                         cudaMemcpyDeviceToDevice, st));
-      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-      ta_dfree(h, xb);
-    }
-    // step 4
-    GatherArgs g;
-    g.ev = h->events; g.perm = perm; g.keys = skeys; g.n = n; g.n_valid = h->n_valid;
-    g.packed = h->packed; g.ibits = h->ibits; g.wbits = h->wbits; g.off = h->d_off;
-    g.wshift = h->ibits + h->tbits + (h->sbits - h->dshift);
-    g.sbits = h->packed ? h->ibits + (h->sbits - h->dshift) : h->sbits;
-    g.ts_start = c_ts; g.ts_end = c_te; g.corr = c_corr; g.pid = c_pid; g.name = c_name; g.seq = c_seq;
-    g.stream = c_stream; g.kind = c_kind; g.lane_start = lane_start;
-    g.tt = h->d_triples; g.tbits = h->tbits; g.n_pids = h->n_pids > 0 ? h->n_pids : 1;
-    g.slot_min = h->d_slot_min; g.slot_max = h->d_slot_max;
-    k_gather<<<TA_N nblk(n, 256), 256, 0, st>>>(g);
+    k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
+                                     h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
+                                     lane_window, lane_pid, lane_stream, lane_domain, lane_off,
+                                     lane_code, lane_slot, lane_dom_end, n_lanes_dev, lane_cap);
+    TA_CHECK_CUDA(h, cudaGetLastError());
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_max.data(), h->d_slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
+    TA_TRY(ta_read_status(h, words));
+    if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+    if (!words[ST_LONG_RUN]) break;
+    if (!h->packed) return TA_ERR_OVERFLOW;  // cannot happen: the pair path resolves long runs itself
+    TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status + ST_LONG_RUN, 0, sizeof(int32_t), st));
+    TA_TRY(ta_launch_load(h, false));
   }
-  k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
-                                   h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
-                                   lane_window, lane_pid, lane_stream, lane_domain, lane_off,
-                                   lane_code, lane_slot, lane_dom_end, n_lanes_dev, lane_cap);
-  TA_CHECK_CUDA(h, cudaGetLastError());
-  int32_t n_lanes = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_max.data(), h->d_slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
   ta_dfree(h, tb);
   ta_dfree(h, h->d_keys);
   h->d_keys = nullptr;

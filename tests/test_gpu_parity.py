@@ -52,6 +52,28 @@ def test_larger_random_window_spans_tiles():
     both(ev, off, t0, t1, min_gap=1, comm_sizes=sizes)
 
 
+@pytest.mark.parametrize("run_len", [2, 5, 31, 48, 49, 400])
+def test_runs_of_equal_start_times(run_len):
+    """Many records of one stream start at the same time: their order (longer first, then
+    input order) comes from the run ranking of the gather up to 48 members, and from the
+    full-resolution pair sort with its duration key beyond that."""
+    rng = np.random.default_rng(run_len)
+    rows = []
+    for pid in (4, 9):
+        for s0 in (100, 5000, 5001):
+            for i in range(run_len):
+                dur = int(rng.integers(0, 6))  # few distinct durations: equal intervals too
+                rows.append(("KERNEL", pid, 1, s0, s0 + dur, int(rng.integers(0, 50)), i % 3, 0))
+        for i in range(300):  # ordinary traffic around the runs
+            s = int(rng.integers(0, 9000))
+            rows.append(("KERNEL", pid, int(rng.integers(0, 2)), s, s + int(rng.integers(0, 40)),
+                         int(rng.integers(0, 50)), int(rng.integers(0, 4)), 0))
+            rows.append(("LAUNCH", pid, 0, s // 2, s // 2 + 1, int(rng.integers(0, 50)), 0, 0))
+    order = rng.permutation(len(rows))
+    ev = make_events([rows[i] for i in order])
+    both(ev, [0, len(ev)], [0], [10000], min_gap=5)
+
+
 def test_deep_nesting_is_reported():
     rows = [("OP", 1, 0, 10 + i, 1000 - i, 0, i, 0) for i in range(12)]
     rows.append(("LAUNCH", 1, 0, 100, 110, 1, 0, 0))
