@@ -1,0 +1,109 @@
+"""Parity at the benchmark's full sizes.  The oracle cannot redo 2^26 or 2^28 records in
+seconds, so the whole analysis runs once on the GPU and is compared with the oracle on
+sub-problems the analysis decomposes into (one process of the window; the collective
+records of all processes; whole windows of the multi-window batch), plus properties that
+hold at any size."""
+from functools import partial
+
+import numpy as np
+import pytest
+
+from paper_2609_40247_b200 import synth
+from restrict import Subset, _typed, run_gpu_restricted, subset_input
+from runners import assert_same, run_oracle
+
+pytestmark = pytest.mark.gpu
+MIN_GAP = 500_000
+
+
+def _properties(t0, t1, full):
+    import torch
+    s, j, a, g, c = full["sort"], full["join"], full["attr"], full["gaps"], full["coll"]
+    n, nv = s.n, s.n_valid
+    perm = _typed(s, "perm")[0].long()
+    seen = torch.zeros(n, dtype=torch.bool, device=perm.device)
+    seen[perm] = True
+    assert bool(seen.all()), "perm is not a permutation"
+    del seen
+    # canonical order inside every lane: ts_start ascending, ts_end descending on ties
+    ts, te = _typed(s, "ts_start")[0][:nv], _typed(s, "ts_end")[0][:nv]
+    lane_off = _typed(s, "lane_off")[0].long()
+    out_of_order = (ts[1:] < ts[:-1]) | ((ts[1:] == ts[:-1]) & (te[1:] > te[:-1]))
+    bad = out_of_order.nonzero().squeeze(1) + 1
+    is_lane_start = torch.zeros(nv + 1, dtype=torch.bool, device=perm.device)
+    is_lane_start[lane_off] = True
+    assert bool(is_lane_start[bad].all()), "order violated inside a lane"
+    # the join: every match points at a LAUNCH of the same process with the same correlation id
+    kind, corr, pid = _typed(s, "kind")[0], _typed(s, "corr_id")[0], _typed(s, "pid")[0]
+    lof = _typed(j, "launch_of")[0].long()
+    m = (lof >= 0).nonzero().squeeze(1)
+    tgt = lof[m]
+    assert bool((kind[tgt] == 2).all()) and bool((corr[tgt] == corr[m]).all())
+    assert bool((pid[tgt] == pid[m]).all())
+    assert bool(((kind[m] == 3) | (kind[m] == 4)).all())
+    js, asum = j.numpy("join_sum"), a.numpy("attr_sum")
+    assert np.array_equal(js["n_matched"] + js["n_unmatched"], js["n_probe"])
+    assert int(js["n_matched"].sum()) == len(m)
+    assert int(_typed(j, "kernels_of_launch")[0].sum()) == len(m)
+    assert np.array_equal(asum["n_attributed"] + asum["n_no_launch"] + asum["n_no_op"], js["n_probe"])
+    assert int(_typed(a, "op_n_kernels")[0].sum()) == int(asum["n_attributed"].sum())
+    # gaps: busy + idle is the window length for every device lane; window histograms add up
+    lg = g.numpy("lane_gaps")
+    lw = s.numpy("lane_window")
+    dev = s.numpy("lane_domain") == 1
+    span = (np.asarray(t1, dtype=np.int64) - np.asarray(t0, dtype=np.int64))[lw]
+    assert np.array_equal((lg["busy"] + lg["idle"])[dev], span[dev])
+    lh, wh = g.numpy("lane_hist").astype(np.int64), g.numpy("win_hist").astype(np.int64)
+    acc = np.zeros_like(wh)
+    np.add.at(acc, lw[dev], lh[dev])
+    assert np.array_equal(acc, wh)
+    # aggregates count every kept device record once
+    n_dev = int((kind[:nv] >= 3).sum())
+    assert int(full["agg_dev"].numpy("g_count").sum()) == n_dev
+
+
+def _compare(events, win_off, t0, t1, comm_sizes, subsets, restricted):
+    t0, t1 = np.asarray(t0), np.asarray(t1)
+    for sub in subsets:
+        ev_s, off_s, wkeep = subset_input(events, win_off, sub.sel, sub.windows)
+        o = run_oracle(ev_s, off_s, t0[wkeep], t1[wkeep], min_gap=MIN_GAP, comm_sizes=comm_sizes)
+        g = restricted[sub.name]
+        skip = set(k for k in o if k not in g)
+        assert len(skip) < len(o) and o["n_valid"] > 100_000
+        if "coll" in sub.groups:
+            assert len(o["c_window"]) > 1000
+        if "join" in sub.groups:
+            assert int((o["launch_of"] >= 0).sum()) > 10_000 and int((o["parent"] >= 0).sum()) > 10_000
+        assert_same(o, g, skip=tuple(skip))
+
+
+def test_c3_full_size_one_process_and_collectives():
+    wl = synth.make_workload("c3", 1.0, truth=False)
+    ev = wl.events
+    assert len(ev) > 2**25
+    pids = np.unique(ev["pid"])
+    per_pid = ("sort", "join", "attr", "gaps", "agg")
+    subsets = [Subset(f"pid{p}", ev["pid"] == p, per_pid, pid=int(p)) for p in (pids[0], pids[-1])]
+    subsets.append(Subset("coll", ev["kind"] == 5, ("sort", "coll")))
+    r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
+                           comm_sizes=wl.comm_sizes,
+                           checks=partial(_properties, wl.win_t0, wl.win_t1))
+    _compare(ev, wl.win_off, wl.win_t0, wl.win_t1, wl.comm_sizes, subsets, r)
+
+
+def test_c4_full_size_whole_windows():
+    wl = synth.make_workload("c4", 1.0, truth=False)
+    ev = wl.events
+    assert len(ev) > 2**27
+    off = np.asarray(wl.win_off)
+    W = len(off) - 1
+    keep = sorted({0, 1, 2, W // 2, W - 1})
+    sel = np.zeros(len(ev), dtype=bool)
+    for w in keep:
+        sel[off[w]:off[w + 1]] = True
+    every = ("sort", "join", "attr", "gaps", "agg", "coll")
+    subsets = [Subset("windows", sel, every, windows=keep)]
+    r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
+                           comm_sizes=wl.comm_sizes,
+                           checks=partial(_properties, wl.win_t0, wl.win_t1))
+    _compare(ev, wl.win_off, wl.win_t0, wl.win_t1, wl.comm_sizes, subsets, r)
