@@ -36,8 +36,8 @@ WORKLOAD_TEXT = {
     "c4": "c4: fleet batch of 512 independent 30 s windows",
 }
 # ncu: dram__bytes_read.sum + dram__bytes_write.sum of one k_radix_pass launch divided by the
-# records it sorted (profiles/radix_pass_c3_scaled.txt); None until a capture exists
-RADIX_TRAFFIC_BYTES_PER_RECORD = None
+# records it sorted, on the quarter-size case (profiles/radix_pass_c3_quarter.txt)
+RADIX_TRAFFIC_BYTES_PER_RECORD = 14.1
 
 
 def parse_args():
@@ -114,16 +114,32 @@ class ClockSampler:
         return out
 
 
-def run_pipeline(ta, buf, wl, read_back=False):
-    """The whole hot path once.  Returns (n_valid, bytes read back from the device)."""
+def run_pipeline(ta, buf, wl, read_back=False, per_call=None):
+    """The whole hot path once.  Returns (n_valid, bytes read back from the device).
+    per_call: dict that collects the wall time of each call (every call ends synchronised)."""
+    marks = [time.perf_counter()]
+
+    def mark(name):
+        if per_call is not None:
+            marks.append(time.perf_counter())
+            per_call.setdefault(name, []).append(1e3 * (marks[-1] - marks[-2]))
+
     with ta.Window(buf, wl.win_off, wl.win_t0, wl.win_t1) as w:
+        mark("load_window")
         s = w.sort_timeline()
+        mark("sort_timeline")
         j = w.correlate_launches()
+        mark("correlate_launches")
         a = w.attribute_operators()
+        mark("attribute_operators")
         g = w.stream_gaps(500_000)
+        mark("stream_gaps")
         k1 = w.aggregate_ops(ta.DEVICE_KINDS, 0)
+        mark("aggregate_ops(device kinds, duration)")
         k2 = w.aggregate_ops(1 << ta.KIND_OP, 1)
+        mark("aggregate_ops(OP, T_op)")
         c = w.match_collectives(wl.comm_sizes)
+        mark("match_collectives")
         nbytes = w.load_summary.nbytes + j.join_sum.nbytes + a.attr_sum.nbytes
         if read_back:
             for res, names in ((g, ("lane_gaps", "win_hist", "long_gaps")),
@@ -133,6 +149,37 @@ def run_pipeline(ta, buf, wl, read_back=False):
                 for nm in names:
                     nbytes += res.numpy(nm).nbytes
         return s.n_valid, nbytes
+
+
+def lsd_model_bytes_per_event(wl):
+    """Algorithmic bytes per record of the whole path when the sort is modelled as an LSD radix
+    sort of (key, index) pairs with one pass per key byte: the numerator of the headline
+    roofline fraction, recomputed from the workload's own event mix and key width."""
+    ev = wl.events
+    n = max(len(ev), 1)
+    kinds = np.bincount(np.clip(ev["kind"].astype(np.int64), 0, 6), minlength=7)[:6] / n
+    f_o, f_api, f_l, f_k, f_m, f_c = (float(x) for x in kinds)
+    f_K = f_k + f_m
+    f_h, f_d = f_o + f_api + f_l, f_K + f_c
+
+    def bits(x):
+        return int(np.ceil(np.log2(max(int(x), 1)))) if x > 1 else 0
+
+    n_streams = len(np.unique(ev["stream"])) if len(ev) else 1
+    span = int(np.max(np.asarray(wl.win_t1) - np.asarray(wl.win_t0))) if len(wl.win_t0) else 1
+    key_bits = bits(len(wl.win_t0)) + bits(len(np.unique(ev["pid"]))) + 1 + bits(n_streams) + bits(span)
+    passes = (key_bits + 7) // 8
+    parts = {
+        "load": 52.0,
+        "sort": 8.0 + passes * 24.0,
+        "gather": 84.0,
+        "join": f_l * 44.0 + f_K * 64.0,
+        "attribute": f_h * 23.0 + f_K * 40.0 + f_o * 28.0,
+        "gaps": f_d * 26.0,
+        "aggregate": (2.0 + f_d * 24.0) + (2.0 + f_o * 32.0),
+        "collectives": f_c * 100.0,
+    }
+    return sum(parts.values()), key_bits, passes, parts
 
 
 def time_oracle(wl):
@@ -247,6 +294,12 @@ def main():
     ta.profile_enable(False)
     clocks = sampler.stop()
 
+    # ---- per-call breakdown (outside the timed region) ----
+    per_call = {}
+    for _ in range(3):
+        run_pipeline(ta, dev_buf, wl, per_call=per_call)
+    per_call_ms = {k: round(min(v), 4) for k, v in per_call.items()}
+
     # ---- end to end: pinned host input, host<->device copies inside the timed region ----
     e2e = None
     if args.e2e_steps > 0:
@@ -310,8 +363,18 @@ def main():
                              "no L2 flush needed above 126 MB"},
             "clocks": clocks, "gpu_launches": int(launches),
             "roofline": roof, "cpu_baseline": cpu,
-            "hbm_model": {"events_per_s_at_peak_108B": peak * 1e9 / 108.0,
-                          "frac_of_compulsory_model": value / world * 108.0 / (peak * 1e9)},
+            "per_call_ms": per_call_ms,
+        }
+        lsd_bytes, key_bits, passes, parts = lsd_model_bytes_per_event(wl)
+        per_gpu = value / world
+        line["hbm_model"] = {
+            "lsd_bytes_per_event": round(lsd_bytes, 2), "lsd_key_bits": key_bits, "lsd_passes": passes,
+            "lsd_parts": {k: round(v, 2) for k, v in parts.items()},
+            "frac_of_measured_peak": per_gpu * lsd_bytes / (peak * 1e9),
+            "frac_of_nominal_8TBs": per_gpu * lsd_bytes / 8.0e12,
+            "target_ms_for_half_of_measured_peak": 2e3 * n * lsd_bytes / (peak * 1e9),
+            "compulsory_bytes_per_event": 108.0,
+            "frac_of_measured_peak_compulsory": per_gpu * 108.0 / (peak * 1e9),
         }
         if e2e:
             line["e2e"] = {"value": total_events * args.e2e_steps / (e2e["ms"] * 1e-3), "unit": UNIT,
