@@ -80,7 +80,9 @@ typedef enum ta_status {
 
 /* Caller-supplied device memory and stream.  alloc returns device memory on
  * `device` aligned to at least 256 bytes, or NULL; release takes it back.  If
- * alloc is NULL the library uses the device's stream-ordered pool. */
+ * alloc is NULL the library allocates stream-ordered from a pool of its own (one
+ * per device, created on first use) that keeps freed memory for later calls
+ * until the process ends. */
 typedef struct ta_env {
   void *(*alloc)(size_t bytes, void *ctx);
   void (*release)(void *ptr, void *ctx);

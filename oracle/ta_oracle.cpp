@@ -111,6 +111,10 @@ struct Oracle {
   std::vector<int32_t> r_window, r_pid;
   std::vector<int64_t> r_n_coll, r_sum_wait, r_max_wait, r_n_straggler;
 
+  // device-level coverage
+  std::vector<int32_t> d_window, d_pid;
+  std::vector<int64_t> d_n_events, d_busy, d_idle, d_compute, d_comm, d_overlap, d_exposed;
+
   bool is_kept(int64_t p) const { return p < n_valid; }
 
   // ---- step 1: validity.  Start-time filtering separates successive windows
@@ -434,6 +438,54 @@ struct Oracle {
       r_max_wait.push_back(kv.second.max_wait); r_n_straggler.push_back(kv.second.n_straggler);
     }
   }
+
+  // ---- device-level coverage: from GPU activity, communication hidden by computation is
+  // told apart from exposed time; exposed time is interval coverage (Sec. 6.1, "Execution
+  // progress and state"; Fig. "Overlap and exposed work": a compute lane, a communication / IO
+  // lane, their overlap, the exposed remainder).  Readings: per (window, process), over all
+  // device streams; compute = KERNEL records, communication / IO = MEMCPY and COLL records;
+  // every interval is [ts_start, min(ts_end, t1)); busy = measure of the union of all of them,
+  // compute / comm = measure of each class's union, overlap = measure of the intersection of
+  // the two unions, exposed = comm - overlap, idle = window length - busy.
+  // Written out as a sweep over interval boundaries with one open-interval counter per class.
+  void device_overlap() {
+    d_window.clear(); d_pid.clear(); d_n_events.clear(); d_busy.clear(); d_idle.clear();
+    d_compute.clear(); d_comm.clear(); d_overlap.clear(); d_exposed.clear();
+    std::map<std::pair<int32_t, int32_t>, std::vector<int32_t>> groups;
+    for (int64_t p = 0; p < n_valid; p++)
+      if (kind[p] >= KERNEL) groups[std::make_pair(win_sorted[p], pid[p])].push_back((int32_t)p);
+    for (auto& kv : groups) {
+      const int32_t w = kv.first.first;
+      struct Edge { int64_t t; int cls; int delta; };
+      std::vector<Edge> edges;
+      for (int32_t p : kv.second) {
+        const int64_t s = ts_start[p], e = std::min(ts_end[p], t1[w]);
+        if (e <= s) continue;  // an empty interval covers nothing
+        const int cls = kind[p] == KERNEL ? 0 : 1;
+        edges.push_back(Edge{s, cls, +1});
+        edges.push_back(Edge{e, cls, -1});
+      }
+      std::sort(edges.begin(), edges.end(), [](const Edge& a, const Edge& b) { return a.t < b.t; });
+      int64_t open[2] = {0, 0}, busy = 0, comp = 0, comm = 0, both = 0;
+      for (size_t i = 0; i < edges.size();) {
+        size_t j = i;
+        while (j < edges.size() && edges[j].t == edges[i].t) { open[edges[j].cls] += edges[j].delta; j++; }
+        if (j < edges.size()) {
+          const int64_t dt = edges[j].t - edges[i].t;
+          if (open[0] > 0 || open[1] > 0) busy += dt;
+          if (open[0] > 0) comp += dt;
+          if (open[1] > 0) comm += dt;
+          if (open[0] > 0 && open[1] > 0) both += dt;
+        }
+        i = j;
+      }
+      d_window.push_back(w); d_pid.push_back(kv.first.second);
+      d_n_events.push_back((int64_t)kv.second.size());
+      d_busy.push_back(busy); d_idle.push_back((t1[w] - t0[w]) - busy);
+      d_compute.push_back(comp); d_comm.push_back(comm); d_overlap.push_back(both);
+      d_exposed.push_back(comm - both);
+    }
+  }
 };
 
 template <class T>
@@ -466,6 +518,7 @@ int32_t orc_aggregate(void* h, uint32_t mask, int32_t sel) { return ((Oracle*)h)
 void orc_collectives(void* h, const void* sizes, int32_t n_comms) {
   ((Oracle*)h)->collectives((const CommSize*)sizes, n_comms);
 }
+void orc_device_overlap(void* h) { ((Oracle*)h)->device_overlap(); }
 int64_t orc_n_valid(void* h) { return ((Oracle*)h)->n_valid; }
 
 // Exposes a result array by name: pointer into the oracle's storage, element
@@ -484,6 +537,7 @@ int32_t orc_get(void* h, const char* name, const void** ptr, int64_t* count, int
   G(c_window) G(c_comm) G(c_seq) G(c_n_members) G(c_min_start) G(c_max_start) G(c_skew) G(c_max_end)
   G(c_straggler_pid) G(c_flags) G(wait_ns)
   G(r_window) G(r_pid) G(r_n_coll) G(r_sum_wait) G(r_max_wait) G(r_n_straggler)
+  G(d_window) G(d_pid) G(d_n_events) G(d_busy) G(d_idle) G(d_compute) G(d_comm) G(d_overlap) G(d_exposed)
 #undef G
   return -1;
 }

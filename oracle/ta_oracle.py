@@ -50,6 +50,9 @@ _DTYPES = {
     "c_straggler_pid": np.int32, "c_flags": np.int32, "wait_ns": np.int64,
     "r_window": np.int32, "r_pid": np.int32, "r_n_coll": np.int64, "r_sum_wait": np.int64,
     "r_max_wait": np.int64, "r_n_straggler": np.int64,
+    "d_window": np.int32, "d_pid": np.int32, "d_n_events": np.int64, "d_busy": np.int64,
+    "d_idle": np.int64, "d_compute": np.int64, "d_comm": np.int64, "d_overlap": np.int64,
+    "d_exposed": np.int64,
 }
 
 _lib = None
@@ -84,6 +87,8 @@ def _load():
         lib.orc_aggregate.restype = ctypes.c_int32
         lib.orc_collectives.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32]
         lib.orc_collectives.restype = None
+        lib.orc_device_overlap.argtypes = [ctypes.c_void_p]
+        lib.orc_device_overlap.restype = None
         lib.orc_n_valid.argtypes = [ctypes.c_void_p]
         lib.orc_n_valid.restype = ctypes.c_int64
         lib.orc_get.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_void_p),
@@ -167,6 +172,11 @@ class Oracle:
             arr[i] = (cid, nr, 0)
         self._sizes = arr
         self._lib.orc_collectives(self._h, arr.ctypes.data if len(arr) else None, len(arr))
+
+    def device_overlap(self):
+        """Per (window, process): busy / idle over all device streams, compute and
+        communication coverage, their overlap and the exposed communication (needs sort())."""
+        self._lib.orc_device_overlap(self._h)
 
     def run_all(self, min_gap_ns: int = 500_000, comm_sizes=()):
         """load, sort, correlate, attribute, gaps, collectives; returns attribute's status."""

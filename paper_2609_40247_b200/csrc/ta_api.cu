@@ -6,13 +6,41 @@
 
 #include "ta_internal.cuh"
 
+// Without caller callbacks memory comes from a private stream-ordered pool per device that
+// keeps what it has been given (release threshold = everything): the default pool hands its
+// memory back at every synchronisation, which makes each call pay for fresh gigabytes.
+static cudaMemPool_t own_pool(int device) {
+  static cudaMemPool_t pools[64] = {};
+  if (device < 0 || device >= 64) return nullptr;
+  if (!pools[device]) {
+    cudaMemPoolProps props;
+    memset(&props, 0, sizeof(props));
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = device;
+    cudaMemPool_t pool = nullptr;
+    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    unsigned long long keep = ~0ull;
+    cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    pools[device] = pool;
+  }
+  return pools[device];
+}
+
 void *ta_dalloc(ta_window *h, size_t bytes) {
   if (bytes == 0) bytes = 256;
   void *p = nullptr;
   if (h->env.alloc) {
     p = h->env.alloc(bytes, h->env.ctx);
   } else {
-    if (cudaMallocAsync(&p, bytes, h->stream) != cudaSuccess) {
+    cudaMemPool_t pool = own_pool(h->device);
+    cudaError_t e = pool ? cudaMallocFromPoolAsync(&p, bytes, pool, h->stream)
+                         : cudaMallocAsync(&p, bytes, h->stream);
+    if (e != cudaSuccess) {
       cudaGetLastError();
       p = nullptr;
     }

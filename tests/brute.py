@@ -199,3 +199,30 @@ def collectives(sv, wins, n_valid, sizes):
                               max_end=max(int(sv[p]["ts_end"]) for p in m), straggler=strag,
                               flags=flags)))
     return out, wait, [(k, ranks[k]) for k in sorted(ranks)]
+
+
+def device_overlap(sv, wins, n_valid, t0, t1):
+    """Per (window, pid): marks every tick of the window covered by a KERNEL record and every
+    tick covered by a MEMCPY or COLL record; returns {(w, pid): (n, busy, idle, compute, comm,
+    overlap, exposed)} counted tick by tick."""
+    rows = {}
+    for p in range(n_valid):
+        k = int(sv[p]["kind"])
+        if k < 3:
+            continue
+        w = int(wins[p])
+        key = (w, int(sv[p]["pid"]))
+        L = int(t1[w] - t0[w])
+        if key not in rows:
+            rows[key] = [0, np.zeros(L, dtype=bool), np.zeros(L, dtype=bool)]
+        rows[key][0] += 1
+        s, e = int(sv[p]["ts_start"]) - int(t0[w]), min(int(sv[p]["ts_end"]), int(t1[w])) - int(t0[w])
+        if e > s:
+            rows[key][1 if k == 3 else 2][s:e] = True
+    out = {}
+    for key, (cnt, comp, comm) in rows.items():
+        busy = int((comp | comm).sum())
+        both = int((comp & comm).sum())
+        out[key] = (cnt, busy, len(comp) - busy, int(comp.sum()), int(comm.sum()), both,
+                    int(comm.sum()) - both)
+    return out

@@ -123,4 +123,14 @@ def check_H5(run):
     assert r["attr_status"] == 0
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5]
+def check_H6(run):
+    g = load_golden("H6_overlap.txt")
+    r = run(g["events"], [0, len(g["events"])], [g["t0"]], [g["t1"]])
+    want = [tuple(int(x) for x in t.split(":")) for t in g["expect"]["overlap_rows"]]
+    got = list(zip(*(r[k].tolist() for k in ("d_pid", "d_n_events", "d_busy", "d_idle", "d_compute",
+                                            "d_comm", "d_overlap", "d_exposed"))))
+    assert got == want
+    assert r["d_window"].tolist() == [0] * len(want)
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6]

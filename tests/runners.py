@@ -14,6 +14,9 @@ COLL_KEYS = ["c_window", "c_comm", "c_seq", "c_n_members", "c_min_start", "c_max
              "c_max_end", "c_straggler_pid", "c_flags", "wait_ns", "r_window", "r_pid", "r_n_coll",
              "r_sum_wait", "r_max_wait", "r_n_straggler"]
 
+OVERLAP_KEYS = ["d_window", "d_pid", "d_n_events", "d_busy", "d_idle", "d_compute", "d_comm",
+                "d_overlap", "d_exposed"]
+
 DEVICE_MASK = (1 << 3) | (1 << 4) | (1 << 5)
 OP_MASK = 1
 
@@ -45,6 +48,9 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
         r[f"aggT_{k}"] = o.get(k)
     o.collectives(comm_sizes)
     for k in COLL_KEYS:
+        r[k] = o.get(k)
+    o.device_overlap()
+    for k in OVERLAP_KEYS:
         r[k] = o.get(k)
     o.close()
     return r
@@ -87,6 +93,9 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
         c = w.match_collectives(comm_sizes)
         for k in COLL_KEYS:
             r[k] = c.numpy(k)
+        d = w.device_overlap()
+        for k in OVERLAP_KEYS:
+            r[k] = d.numpy(k)
     return r
 
 

@@ -261,3 +261,18 @@ def test_collectives_against_dict(seed):
             ws = [wait[p] for p in range(r["n_valid"]) if sv[p]["kind"] == 5
                   and (int(wins[p]), int(sv[p]["corr_id"]), int(sv[p]["seq"])) == key]
             assert min(ws) == 0 and max(ws) == g["skew"]
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_device_overlap_against_tick_bitmaps(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1, min_gap=5, comm_sizes=sizes)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    rows = brute.device_overlap(sv, wins, r["n_valid"], t0, t1)
+    got = {(int(w), int(p)): tuple(int(r[k][i]) for k in ("d_n_events", "d_busy", "d_idle", "d_compute",
+                                                          "d_comm", "d_overlap", "d_exposed"))
+           for i, (w, p) in enumerate(zip(r["d_window"], r["d_pid"]))}
+    assert got == rows
+    assert list(got) == sorted(got)  # rows come in (window, pid) order
+    assert len(rows) > 0

@@ -73,6 +73,25 @@ def check_against_truth(wl, r):
     assert np.array_equal(r["agg0_g_hist"].sum(axis=1), r["agg0_g_count"])
     assert (r["agg0_g_min"] <= r["agg0_g_max"]).all()
     assert int(r["aggT_g_count"].sum()) == int((r["op_n_kernels"] > 0).sum())
+    # device-level coverage: set identities, and bounds from the per-stream figures
+    span = (np.asarray(wl.win_t1) - np.asarray(wl.win_t0))[r["d_window"]]
+    assert np.array_equal(r["d_busy"] + r["d_idle"], span)
+    assert np.array_equal(r["d_busy"], r["d_compute"] + r["d_comm"] - r["d_overlap"])
+    assert np.array_equal(r["d_exposed"], r["d_comm"] - r["d_overlap"])
+    assert (r["d_overlap"] <= np.minimum(r["d_compute"], r["d_comm"])).all()
+    assert int(r["d_n_events"].sum()) == len(dev)
+    devl = np.nonzero(r["lane_domain"] == 1)[0]
+    key = {(int(w), int(p)): i for i, (w, p) in enumerate(zip(r["d_window"], r["d_pid"]))}
+    lane_max = np.zeros(len(key), dtype=np.int64)
+    lane_sum = np.zeros(len(key), dtype=np.int64)
+    for l in devl:
+        i = key[(int(r["lane_window"][l]), int(r["lane_pid"][l]))]
+        b = int(r["lane_gaps"]["busy"][l])
+        lane_max[i] = max(lane_max[i], b)
+        lane_sum[i] += b
+    assert (r["d_busy"] >= lane_max).all() and (r["d_busy"] <= lane_sum).all()
+    if not (kind == 5).any() and not (kind == 4).any():
+        assert not r["d_comm"].any()
 
 
 @pytest.mark.parametrize("name,scale,shuffle", CASES)
