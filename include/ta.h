@@ -333,6 +333,37 @@ typedef struct ta_coll_result {
 ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes,
                                int32_t n_comms, ta_coll_result *out);
 
+/* ------------------------------------------------------------------------
+ * ta_device_overlap - device-level coverage per (window, process): from GPU
+ * activity, communication hidden by computation is told apart from exposed
+ * time, and exposed time is interval coverage (Sec. 6.1, "Execution progress
+ * and state"; Fig. "Overlap and exposed work").  Beyond the seven calls above:
+ * the first of the analyses that build on them.  Needs ta_sort_timeline only.
+ *
+ * For every (window, pid) that has at least one kept device record, over ALL of
+ * its device streams, with every record's interval taken as
+ * [ts_start, min(ts_end, t1)) (an empty interval covers nothing):
+ *   d_n_events  number of kept device records
+ *   d_busy      measure of the union of all intervals; d_idle = (t1 - t0) - d_busy
+ *   d_compute   measure of the union of the KERNEL intervals
+ *   d_comm      measure of the union of the MEMCPY and COLL intervals
+ *   d_overlap   measure of the intersection of those two unions
+ *   d_exposed   d_comm - d_overlap
+ * Rows are ordered by (window, pid ascending).  Readings (the paper names the
+ * two lanes "Compute" and "Comm. / IO" and gives no rule): memory copies count
+ * as communication / IO; ends are clipped to the window as in ta_stream_gaps.
+ * All arrays are device memory owned by the handle, n_rows entries each.
+ * Limits: as ta_load_window, and windows x pids < 2^22 (TA_ERR_TOO_LARGE).
+ * Errors: TA_ERR_ORDER before ta_sort_timeline; TA_ERR_OOM; TA_ERR_CUDA;
+ * TA_ERR_TIMEOUT.  One stream synchronisation at the end. */
+typedef struct ta_overlap_result {
+  int64_t n_rows;
+  const int32_t *d_window, *d_pid;
+  const int64_t *d_n_events, *d_busy, *d_idle, *d_compute, *d_comm, *d_overlap, *d_exposed;
+} ta_overlap_result;
+
+ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out);
+
 /* ta_free - releases every buffer of the handle through env.release.
  * NULL-safe.  Synchronises the handle's stream first. */
 void ta_free(ta_window *h);

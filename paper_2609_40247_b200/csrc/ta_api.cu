@@ -310,6 +310,16 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes, int32_t 
   return ta_run_collectives(h, sizes, n_comms, out);
 }
 
+ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out) {
+  if (!h || !out) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 2)) return TA_ERR_ORDER;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
+  return ta_run_overlap(h, out);
+}
+
 void ta_free(ta_window *h) {
   if (!h) return;
   cudaSetDevice(h->device);

@@ -87,6 +87,8 @@ struct ta_window {
   int32_t *d_lane_code;      // per lane: window << tbits | triple rank
   int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
   int32_t *d_lane_dom_end;   // per lane: first position behind the run of lanes of the same domain
+  int32_t *d_lane_dev_base;  // per device lane: number of device records in earlier lanes
+  int64_t n_device;          // kept device records
   i64 *d_slot_min, *d_slot_max;               // per slot: corr_id range of its LAUNCH records
   std::vector<int64_t> h_slot_min, h_slot_max;  // host copies (INT64_MAX / INT64_MIN when none)
 
@@ -155,6 +157,9 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
 // coll.cu
 ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_comms,
                              ta_coll_result *out);
+
+// overlap.cu
+ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out);
 
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 

@@ -210,8 +210,8 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
                                                      int32_t *lane_pid, int16_t *lane_stream,
                                                      int16_t *lane_domain, int32_t *lane_off,
                                                      int32_t *lane_code, int32_t *lane_slot,
-                                                     int32_t *lane_dom_end, int32_t *n_lanes_out,
-                                                     int64_t cap) {
+                                                     int32_t *lane_dom_end, int32_t *lane_dev_base,
+                                                     int32_t *n_lanes_out, int64_t cap) {
   __shared__ u64 tmp[33];
   __shared__ u64 base;
   if (threadIdx.x == 0) base = 0;
@@ -253,6 +253,22 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
     while (m < L && lane_domain[m] == lane_domain[l]) m++;
     lane_dom_end[l] = m < L ? lane_off[m] : (int32_t)n_valid;
   }
+  // per device lane: how many device records sit in earlier lanes (their index once the device
+  // records are taken out in order); n_lanes_out[1] = the number of device records
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int64_t l0 = 0; l0 < L; l0 += blockDim.x) {
+    const int64_t l = l0 + threadIdx.x;
+    u64 sz = 0;
+    if (l < L && lane_domain[l] == 1) sz = (u64)((l + 1 < L ? lane_off[l + 1] : (int32_t)n_valid) - lane_off[l]);
+    u64 total;
+    const u64 ex = block_scan_exclusive<OpAdd>(sz, OpAdd(), tmp, &total);
+    if (l < L) lane_dev_base[l] = (int32_t)(base + ex);
+    __syncthreads();
+    if (threadIdx.x == 0) base += total;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) n_lanes_out[1] = (int32_t)base;
 }
 
 // ---- packed keys: index of the record a key stands for -------------------------
@@ -281,7 +297,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
 
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
-                2 * Carver::pad(n * 2) + 5 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
+                2 * Carver::pad(n * 2) + 6 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
                 Carver::pad((lane_cap + 1) * 4) + 2 * Carver::pad((size_t)n_slots * 8) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
@@ -295,7 +311,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int16_t *lane_stream = ck.take<int16_t>(lane_cap), *lane_domain = ck.take<int16_t>(lane_cap);
   int32_t *lane_off = ck.take<int32_t>(lane_cap + 1);
   int32_t *lane_dom_end = ck.take<int32_t>(lane_cap);
-  int32_t *n_lanes_dev = ck.take<int32_t>(1);
+  int32_t *lane_dev_base = ck.take<int32_t>(lane_cap);
+  int32_t *n_lanes_dev = ck.take<int32_t>(2);  // [0] lanes, [1] device records
   h->d_slot_min = ck.take<i64>(n_slots);
   h->d_slot_max = ck.take<i64>(n_slots);
 
@@ -310,7 +327,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *lane_start = ct.take<int32_t>(n_codes);
   void *sort_tmp = ct.base + ct.off;
 
-  int32_t n_lanes = 0;
+  int32_t n_lanes_host[2] = {0, 0};
   // Packed keys settle the order down to a coarse time; the gather ranks the members of a run
   // of equal coarse keys itself.  A run too long for that is reported at the end, and the
   // second attempt sorts (key, index) pairs at full time resolution.
@@ -402,9 +419,9 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
                                      h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
                                      lane_window, lane_pid, lane_stream, lane_domain, lane_off,
-                                     lane_code, lane_slot, lane_dom_end, n_lanes_dev, lane_cap);
+                                     lane_code, lane_slot, lane_dom_end, lane_dev_base, n_lanes_dev, lane_cap);
     TA_CHECK_CUDA(h, cudaGetLastError());
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_lanes, n_lanes_dev, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(n_lanes_host, n_lanes_dev, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_max.data(), h->d_slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
     TA_TRY(ta_read_status(h, words));
@@ -418,6 +435,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   ta_dfree(h, h->d_keys);
   h->d_keys = nullptr;
 
+  const int32_t n_lanes = n_lanes_host[0];
+  h->n_device = n_lanes_host[1];
   ta_sort_result &r = h->sorted;
   r.n = n; r.n_valid = h->n_valid; r.n_lanes = n_lanes; r.n_windows = h->W;
   r.perm = (const int32_t *)perm;
@@ -429,5 +448,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   h->d_lane_code = lane_code;
   h->d_lane_slot = lane_slot;
   h->d_lane_dom_end = lane_dom_end;
+  h->d_lane_dev_base = lane_dev_base;
   return TA_OK;
 }

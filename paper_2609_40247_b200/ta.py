@@ -81,11 +81,15 @@ _CollResult = _ptr_struct("_CollResult", [
     ("g_skew", _vp), ("g_max_end", _vp), ("g_straggler_pid", _vp), ("g_flags", _vp),
     ("wait_ns", _vp), ("r_window", _vp), ("r_pid", _vp), ("r_n_coll", _vp), ("r_sum_wait", _vp),
     ("r_max_wait", _vp), ("r_n_straggler", _vp)])
+_OverlapResult = _ptr_struct("_OverlapResult", [
+    ("n_rows", ctypes.c_int64), ("d_window", _vp), ("d_pid", _vp), ("d_n_events", _vp),
+    ("d_busy", _vp), ("d_idle", _vp), ("d_compute", _vp), ("d_comm", _vp), ("d_overlap", _vp),
+    ("d_exposed", _vp)])
 
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
-           "ta_lane_gaps_noalloc"]
+           "ta_lane_gaps_noalloc", "ta_device_overlap"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -122,6 +126,8 @@ def lib():
         L.ta_aggregate_ops.argtypes = [_vp, ctypes.c_uint32, ctypes.c_int32, ctypes.POINTER(_AggResult)]
         L.ta_match_collectives.restype = ctypes.c_int
         L.ta_match_collectives.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(_CollResult)]
+        L.ta_device_overlap.restype = ctypes.c_int
+        L.ta_device_overlap.argtypes = [_vp, ctypes.POINTER(_OverlapResult)]
         L.ta_free.restype = None
         L.ta_free.argtypes = [_vp]
         L.ta_strerror.restype = ctypes.c_char_p
@@ -305,6 +311,12 @@ class CollResult(_Result):
         return super().tensor(self._names.get(name, name))
 
 
+class OverlapResult(_Result):
+    _layout = dict([("d_window", ("<i4", lambda r: r.n_rows)), ("d_pid", ("<i4", lambda r: r.n_rows))] +
+                   [(k, ("<i8", lambda r: r.n_rows)) for k in
+                    ("d_n_events", "d_busy", "d_idle", "d_compute", "d_comm", "d_overlap", "d_exposed")])
+
+
 class Window:
     """One analysis handle (ta_window).  `events`: a CUDA tensor holding n 40-byte
     records (any dtype, contiguous) - borrowed until sort_timeline() returns - or a
@@ -433,6 +445,13 @@ class Window:
         if st != 0:
             raise TaError(st, "ta_aggregate_ops")
         return AggResult(self, raw, dict(self._dims(), n_groups=raw.n_groups))
+
+    def device_overlap(self) -> OverlapResult:
+        raw = _OverlapResult()
+        st = self._lib.ta_device_overlap(self._h, ctypes.byref(raw))
+        if st != 0:
+            raise TaError(st, "ta_device_overlap")
+        return OverlapResult(self, raw, dict(self._dims(), n_rows=raw.n_rows))
 
     def match_collectives(self, comm_sizes=()) -> CollResult:
         arr = np.zeros(len(comm_sizes), dtype=COMM_SIZE)

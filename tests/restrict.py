@@ -12,7 +12,8 @@ host, where they are compared with the oracle run on the subset.
 import numpy as np
 
 from paper_2609_40247_b200.ta import NBINS
-from runners import AGG_KEYS, ATTR_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS, OP_MASK
+from runners import (AGG_KEYS, ATTR_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS, OP_MASK,
+                     OVERLAP_KEYS)
 
 _POSITIONAL = {"launch_of", "parent", "op_of"}  # values are sorted positions (or -1)
 _PER_RECORD_SORT = ["ts_start", "ts_end", "corr_id", "pid", "name_id", "seq", "stream", "kind"]
@@ -22,7 +23,8 @@ _LANE_COLS = ["lane_window", "lane_pid", "lane_stream", "lane_domain"]
 class Subset:
     """sel: bool mask over the input records; windows: kept window indices (None = all);
     pid: restrict aggregate rows to this pid (None = all); groups: which result groups
-    are meaningful for the subset (any of "sort", "join", "attr", "gaps", "agg", "coll")."""
+    are meaningful for the subset (any of "sort", "join", "attr", "gaps", "agg", "coll",
+    "overlap")."""
 
     def __init__(self, name, sel, groups, windows=None, pid=None):
         self.name, self.sel, self.groups, self.windows, self.pid = name, sel, groups, windows, pid
@@ -64,10 +66,11 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
         ag_dev = w.aggregate_ops(DEVICE_MASK, 0)
         ag_op = w.aggregate_ops(OP_MASK, 1) if a.status == 0 else None
         c = w.match_collectives(comm_sizes)
+        ov = w.device_overlap()
         del buf
         if checks is not None:
             checks(dict(window=w, sort=s, join=j, attr=a, gaps=g, agg_dev=ag_dev, agg_op=ag_op,
-                        coll=c))
+                        coll=c, overlap=ov))
         n, n_valid = s.n, s.n_valid
         perm = _typed(s, "perm")[0].long()
         lane_off = _typed(s, "lane_off")[0].long()
@@ -175,6 +178,16 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
                         continue
                     v = t[crow] if k.startswith("c_") else t[rrow]
                     if k in ("c_window", "r_window"):
+                        v = wmap[v.long()]
+                    r[k] = _host(v, dt)
+            if "overlap" in sub.groups:
+                rows = wmap[_typed(ov, "d_window")[0].long()] >= 0
+                if sub.pid is not None:
+                    rows &= _typed(ov, "d_pid")[0] == sub.pid
+                for k in OVERLAP_KEYS:
+                    t, dt = _typed(ov, k)
+                    v = t[rows]
+                    if k == "d_window":
                         v = wmap[v.long()]
                     r[k] = _host(v, dt)
             out[sub.name] = r

@@ -57,6 +57,14 @@ def _properties(t0, t1, full):
     acc = np.zeros_like(wh)
     np.add.at(acc, lw[dev], lh[dev])
     assert np.array_equal(acc, wh)
+    # device-level coverage: set identities, every device record counted once
+    ov = {k: full["overlap"].numpy(k) for k in ("d_window", "d_busy", "d_idle", "d_compute", "d_comm",
+                                                 "d_overlap", "d_exposed", "d_n_events")}
+    ospan = (np.asarray(t1, dtype=np.int64) - np.asarray(t0, dtype=np.int64))[ov["d_window"]]
+    assert np.array_equal(ov["d_busy"] + ov["d_idle"], ospan)
+    assert np.array_equal(ov["d_busy"], ov["d_compute"] + ov["d_comm"] - ov["d_overlap"])
+    assert (ov["d_overlap"] >= 0).all() and (ov["d_exposed"] >= 0).all()
+    assert int(ov["d_n_events"].sum()) == int((kind[:nv] >= 3).sum())
     # aggregates count every kept device record once
     n_dev = int((kind[:nv] >= 3).sum())
     assert int(full["agg_dev"].numpy("g_count").sum()) == n_dev
@@ -82,7 +90,7 @@ def test_c3_full_size_one_process_and_collectives():
     ev = wl.events
     assert len(ev) > 2**25
     pids = np.unique(ev["pid"])
-    per_pid = ("sort", "join", "attr", "gaps", "agg")
+    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap")
     subsets = [Subset(f"pid{p}", ev["pid"] == p, per_pid, pid=int(p)) for p in (pids[0], pids[-1])]
     subsets.append(Subset("coll", ev["kind"] == 5, ("sort", "coll")))
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
@@ -101,7 +109,7 @@ def test_c4_full_size_whole_windows():
     sel = np.zeros(len(ev), dtype=bool)
     for w in keep:
         sel[off[w]:off[w + 1]] = True
-    every = ("sort", "join", "attr", "gaps", "agg", "coll")
+    every = ("sort", "join", "attr", "gaps", "agg", "coll", "overlap")
     subsets = [Subset("windows", sel, every, windows=keep)]
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
                            comm_sizes=wl.comm_sizes,
