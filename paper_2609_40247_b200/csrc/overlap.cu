@@ -8,12 +8,13 @@
 //   sum_i max(0, e_i - max(s_i, P_i)),   P_i = max of the ends seen before i,
 // the same recurrence as the per-stream gap scan, so the step is: take the device
 // records of every process out of their stream lanes, sort them by (window, process,
-// ts_start) with the pair sorter, and run ONE chained max-scan with three channels
+// ts_start) - keys that carry the record's index in their low bits when (process slot, time,
+// index) fit 64 bits, (key, index) pairs otherwise - and run ONE chained max-scan with three channels
 // (all records, computation, communication).  The measure of the intersection follows
 // from the three unions: |A n B| = |A| + |B| - |A u B|.  Scanned values are tagged with
 // the (window, process) slot in their upper bits, as in the gap scan, so a prefix that
 // belongs to an earlier process is recognised and ignored.
-// HBM-bound on the sort: 12 B + 12 B per device record and pass.
+// HBM-bound on the sort: 8 B + 8 B (keys) or 12 B + 12 B (pairs) per device record and pass.
 #include <climits>
 #include <cstring>
 
@@ -32,8 +33,8 @@ struct OvKeyArgs {
   const int32_t *lane_off, *lane_slot, *lane_window, *lane_dom_end, *lane_dev_base;
   const int16_t *lane_domain;
   const int64_t *t0;
-  int tsbits;
-  u64 *keys;  // [device record index] (slot << tsbits) | (ts_start - t0)
+  int tsbits, idxbits;
+  u64 *keys;  // [device record index] ((slot << tsbits) | (ts_start - t0)) << idxbits | index
   u32 *pos;   // [device record index] sorted position
 };
 
@@ -76,7 +77,8 @@ __global__ void __launch_bounds__(OV_THREADS) k_ov_keys(OvKeyArgs a) {
     }
     if (!dev) continue;
     const int64_t c = cbase + (p - cur_off);
-    a.keys[c] = ((u64)slot << a.tsbits) | (u64)(s[j] - w0);
+    a.keys[c] = ((((u64)slot << a.tsbits) | (u64)(s[j] - w0)) << a.idxbits) |
+                (a.idxbits ? (u64)c : 0ull);
     a.pos[c] = (u32)p;
   }
 }
@@ -84,7 +86,8 @@ __global__ void __launch_bounds__(OV_THREADS) k_ov_keys(OvKeyArgs a) {
 struct OvScanArgs {
   int64_t m;          // device records
   const u64 *keys;    // sorted
-  const u32 *pos;     // sorted position of each
+  const u32 *pos;     // sorted position: of element i (pairs), or of device record index c (packed keys)
+  int idxbits;        // packed keys: low bits hold the device record index; 0 = pairs
   const int64_t *te;
   const int16_t *kind;
   const int64_t *t0, *t1;
@@ -113,7 +116,12 @@ __global__ void __launch_bounds__(OV_THREADS, 3) k_ov_scan(OvScanArgs a) {
   for (int j = 0; j < OV_ITEMS; j++) {
     const bool in = i0 + j < a.m;
     key[j] = in ? a.keys[i0 + j] : ~0ull;
-    pp[j] = in ? a.pos[i0 + j] : 0u;
+    if (a.idxbits) {
+      pp[j] = in ? a.pos[key[j] & ((1ull << a.idxbits) - 1)] : 0u;
+      key[j] >>= a.idxbits;
+    } else {
+      pp[j] = in ? a.pos[i0 + j] : 0u;
+    }
   }
 #pragma unroll
   for (int j = 0; j < OV_ITEMS; j++) {
@@ -253,6 +261,11 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   const int tsbits = ov_bit_len((uint64_t)max_span);
   const int slot_bits = ov_bit_len((uint64_t)(n_slots - 1));
   if (tsbits > 40 || tsbits + slot_bits > 63 || n_slots >= (1ll << 22)) return TA_ERR_TOO_LARGE;
+  // when (slot, time, index) fit one 64-bit word the index travels inside the key and the
+  // passes move keys only (8 B + 8 B per record instead of 12 B + 12 B)
+  int idxbits = ov_bit_len((uint64_t)(m - 1));
+  if (idxbits < 1) idxbits = 1;
+  if (tsbits + slot_bits + idxbits > 64) idxbits = 0;
 
   // results (kept): at most one row per slot
   size_t kb = 2 * Carver::pad((size_t)n_slots * 4) + 7 * Carver::pad((size_t)n_slots * 8) + 256;
@@ -289,14 +302,21 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   ka.ts = h->sorted.ts_start;
   ka.lane_off = h->sorted.lane_off; ka.lane_slot = h->d_lane_slot; ka.lane_window = h->sorted.lane_window;
   ka.lane_dom_end = h->d_lane_dom_end; ka.lane_dev_base = h->d_lane_dev_base;
-  ka.lane_domain = h->sorted.lane_domain; ka.t0 = h->d_t0; ka.tsbits = tsbits;
+  ka.lane_domain = h->sorted.lane_domain; ka.t0 = h->d_t0; ka.tsbits = tsbits; ka.idxbits = idxbits;
   ka.keys = k_in; ka.pos = v_in;
   const int64_t key_tiles = (h->n_valid + OV_TILE - 1) / OV_TILE;
   k_ov_keys<<<TA_N (unsigned)key_tiles, OV_THREADS, 0, st>>>(ka);
   TA_CHECK_CUDA(h, cudaGetLastError());
-  TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, k_fin, v_fin, m,
-                             ta_make_plan(0, tsbits + slot_bits), nullptr, sort_tmp));
-  sa.m = m; sa.keys = k_fin; sa.pos = v_fin;
+  if (idxbits) {
+    TA_TRY(ta_radix_sort_keys(h, k_in, k_scr, k_fin, m,
+                              ta_make_plan(idxbits, idxbits + tsbits + slot_bits), nullptr, sort_tmp));
+    sa.pos = v_in;
+  } else {
+    TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, k_fin, v_fin, m,
+                               ta_make_plan(0, tsbits + slot_bits), nullptr, sort_tmp));
+    sa.pos = v_fin;
+  }
+  sa.m = m; sa.keys = k_fin; sa.idxbits = idxbits;
   sa.te = h->sorted.ts_end; sa.kind = h->sorted.kind; sa.t0 = h->d_t0; sa.t1 = h->d_t1;
   sa.tsbits = tsbits; sa.n_pids = n_pids; sa.status = h->d_status;
   k_ov_scan<<<TA_N (unsigned)tiles, OV_THREADS, 0, st>>>(sa);
