@@ -10,10 +10,11 @@
 //   k_attr_agg     per tile, the stack of OPs that are still undominated at the
 //                  tile's end (at most TA_MAX_DEPTH + 1 entries when nesting is
 //                  legal);
-//   k_attr_carry   one warp per host lane folds those stacks along the lane's
-//                  tiles (one stack entry per warp lane; entries that end no
-//                  later than a later tile's outermost surviving OP are dropped)
-//                  and leaves every tile the stack that is open at its start;
+//   k_attr_fold_*  an exclusive scan of those stacks under the stack monoid (one
+//                  stack entry per warp lane; entries that end no later than a
+//                  later tile's outermost surviving OP are dropped; a tile whose
+//                  last lane starts inside it cuts off what came before), as a
+//                  fan-out-32 tree, leaves every tile the stack open at its start;
 //   k_attr_resolve per record: a backward look over the thread's own records,
 //                  else one descent of a max-tree over the threads' largest OP
 //                  end times in shared memory, else the carried stack.
@@ -219,65 +220,125 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
   }
 }
 
-// ---- kernel 2: one warp per host lane folds the tile stacks along the lane -----
-__global__ void __launch_bounds__(128) k_attr_carry(AttrArgs a) {
-  __shared__ i64 st_e[4][32][AT_CAP];
-  __shared__ int32_t st_pos[4][32][AT_CAP];
-  __shared__ int st_meta[4][32];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int l = blockIdx.x * 4 + warp;
-  if (l >= a.n_lanes || a.lane_domain[l] != 0) return;
-  const int64_t b = a.lane_off[l], e = a.lane_off[l + 1];
-  if (e <= b) return;
-  const int64_t ta = b / AT_TILE, tb = (e - 1) / AT_TILE;
-  if (tb == ta) return;
-  bool overflow = false;
-  WStack acc;  // stack at the end of the tiles folded so far
-  {
-    const int m = a.agg_meta[ta];
-    acc.cnt = m & 0xFF;
-    acc.reset = 0;
-    acc.e = lane < acc.cnt ? a.agg_e[(size_t)ta * AT_CAP + lane] : 0;
-    acc.pos = lane < acc.cnt ? a.agg_pos[(size_t)ta * AT_CAP + lane] : 0;
-  }
-  for (int64_t t0 = ta + 1; t0 <= tb; t0 += 32) {
-    // stage up to 32 tile stacks: one tile per lane
-    const int64_t t = t0 + lane;
-    int m = 0;
-    if (t < tb) {  // the lane's last tile leaves nothing that is needed
-      m = a.agg_meta[t];
-      const int c = m & 0xFF;
+// ---- kernel 2: the stack open at the start of every tile --------------------------
+// An exclusive scan of the tile stacks under the stack monoid (wstack_combine; a stack whose
+// reset flag is set cuts off everything before it, which is how lanes stay apart).  One fold
+// over all tiles would be a serial chain as long as the longest host lane, so it is done as a
+// tree with fan-out 32: fold groups of 32 stacks upwards until at most 32 remain, scan those
+// with one warp, then unfold downwards.  Every step is one warp working through 32 staged
+// stacks; no kernel waits for another.
+struct StackArr {
+  int32_t *meta;  // count | reset << 8
+  i64 *e;
+  int32_t *pos;
+};
+#define AT_FAN 32
+struct StackStage {
+  i64 e[4][AT_FAN][AT_CAP];
+  int32_t pos[4][AT_FAN][AT_CAP];
+  int meta[4][AT_FAN];
+};
+// lane i of the warp copies stack first + i into the stage (count 0 beyond n)
+__device__ __forceinline__ void stack_stage(const StackArr &src, int64_t first, int64_t n, StackStage &st,
+                                            int warp, int lane) {
+  const int64_t t = first + lane;
+  int m = 0;
+  if (t < n) {
+    m = src.meta[t];
+    const int c = m & 0xFF;
 #pragma unroll
-      for (int k = 0; k < AT_CAP; k++)
-        if (k < c) {
-          st_e[warp][lane][k] = a.agg_e[(size_t)t * AT_CAP + k];
-          st_pos[warp][lane][k] = a.agg_pos[(size_t)t * AT_CAP + k];
-        }
-    }
-    st_meta[warp][lane] = m;
-    __syncwarp();
-    const int cntb = (int)min((int64_t)32, tb - t0 + 1);
-    for (int i = 0; i < cntb; i++) {
-      const int64_t ti = t0 + i;
-      if (lane < acc.cnt) {
-        a.carry_e[(size_t)ti * AT_CAP + lane] = acc.e;
-        a.carry_pos[(size_t)ti * AT_CAP + lane] = acc.pos;
+    for (int k = 0; k < AT_CAP; k++)
+      if (k < c) {
+        st.e[warp][lane][k] = src.e[(size_t)t * AT_CAP + k];
+        st.pos[warp][lane][k] = src.pos[(size_t)t * AT_CAP + k];
       }
-      if (lane == 0) a.carry_cnt[ti] = acc.cnt;
-      if (ti < tb) {
-        const int mi = st_meta[warp][i];
-        WStack nxt;
-        nxt.cnt = mi & 0xFF;
-        nxt.reset = 0;
-        nxt.e = lane < nxt.cnt ? st_e[warp][i][lane] : 0;
-        nxt.pos = lane < nxt.cnt ? st_pos[warp][i][lane] : 0;
-        wstack_combine(acc, nxt, &overflow);
-        acc = nxt;
-      }
-    }
-    __syncwarp();
   }
-  if (overflow && lane == 0) ta_set_err(a.status, TA_ERR_DEPTH);
+  st.meta[warp][lane] = m;
+  __syncwarp();
+}
+__device__ __forceinline__ WStack stack_staged(const StackStage &st, int warp, int i, int lane) {
+  WStack x;
+  const int m = st.meta[warp][i];
+  x.cnt = m & 0xFF;
+  x.reset = (m >> 8) & 1;
+  x.e = lane < x.cnt ? st.e[warp][i][lane] : 0;
+  x.pos = lane < x.cnt ? st.pos[warp][i][lane] : 0;
+  return x;
+}
+__device__ __forceinline__ WStack stack_load(const StackArr &src, int64_t t, int lane) {
+  WStack x;
+  const int m = src.meta[t];
+  x.cnt = m & 0xFF;
+  x.reset = (m >> 8) & 1;
+  x.e = lane < x.cnt ? src.e[(size_t)t * AT_CAP + lane] : 0;
+  x.pos = lane < x.cnt ? src.pos[(size_t)t * AT_CAP + lane] : 0;
+  return x;
+}
+__device__ __forceinline__ void stack_store(const StackArr &dst, int64_t t, const WStack &x, int lane,
+                                            bool count_only) {
+  if (lane < x.cnt) {
+    dst.e[(size_t)t * AT_CAP + lane] = x.e;
+    dst.pos[(size_t)t * AT_CAP + lane] = x.pos;
+  }
+  if (lane == 0) dst.meta[t] = count_only ? x.cnt : (x.cnt | (x.reset << 8));
+}
+
+// parent[j] = child[32j] (+) ... (+) child[32j + 31]
+__global__ void __launch_bounds__(128) k_attr_fold_up(StackArr child, int64_t n_child, StackArr parent,
+                                                      int64_t n_parent, int32_t *status) {
+  __shared__ StackStage st;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t j = (int64_t)blockIdx.x * 4 + warp;
+  if (j >= n_parent) return;
+  stack_stage(child, j * AT_FAN, n_child, st, warp, lane);
+  bool overflow = false;
+  WStack acc;
+  acc.cnt = 0; acc.reset = 0; acc.e = 0; acc.pos = 0;
+  const int cnt = (int)min((int64_t)AT_FAN, n_child - j * AT_FAN);
+  for (int i = 0; i < cnt; i++) {
+    WStack nxt = stack_staged(st, warp, i, lane);
+    wstack_combine(acc, nxt, &overflow);
+    acc = nxt;
+  }
+  stack_store(parent, j, acc, lane, false);
+  if (overflow && lane == 0) ta_set_err(status, TA_ERR_DEPTH);
+}
+
+// one warp: start[i] = node[0] (+) ... (+) node[i - 1] for the few nodes of the top level
+__global__ void __launch_bounds__(32) k_attr_fold_top(StackArr node, int64_t n, StackArr start,
+                                                      int leaf, int32_t *status) {
+  const int lane = threadIdx.x & 31;
+  bool overflow = false;
+  WStack acc;
+  acc.cnt = 0; acc.reset = 0; acc.e = 0; acc.pos = 0;
+  for (int64_t i = 0; i < n; i++) {
+    stack_store(start, i, acc, lane, leaf != 0);
+    WStack nxt = stack_load(node, i, lane);
+    wstack_combine(acc, nxt, &overflow);
+    acc = nxt;
+  }
+  if (overflow && lane == 0) ta_set_err(status, TA_ERR_DEPTH);
+}
+
+// child_start[32j + i] = parent_start[j] (+) child[32j] (+) ... (+) child[32j + i - 1]
+__global__ void __launch_bounds__(128) k_attr_fold_down(StackArr child, int64_t n_child,
+                                                        StackArr parent_start, int64_t n_parent,
+                                                        StackArr child_start, int leaf, int32_t *status) {
+  __shared__ StackStage st;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t j = (int64_t)blockIdx.x * 4 + warp;
+  if (j >= n_parent) return;
+  stack_stage(child, j * AT_FAN, n_child, st, warp, lane);
+  bool overflow = false;
+  WStack acc = stack_load(parent_start, j, lane);
+  const int cnt = (int)min((int64_t)AT_FAN, n_child - j * AT_FAN);
+  for (int i = 0; i < cnt; i++) {
+    stack_store(child_start, j * AT_FAN + i, acc, lane, leaf != 0);
+    WStack nxt = stack_staged(st, warp, i, lane);
+    wstack_combine(acc, nxt, &overflow);
+    acc = nxt;
+  }
+  if (overflow && lane == 0) ta_set_err(status, TA_ERR_DEPTH);
 }
 
 // ---- kernel 3: parent and depth of every host record -----------------------------
@@ -681,6 +742,12 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
 
   const int64_t tt = tiles > 0 ? tiles : 1;
   size_t tb = 2 * Carver::pad(tt * 4) + 2 * Carver::pad(tt * AT_CAP * 8) + 2 * Carver::pad(tt * AT_CAP * 4) + 256;
+  // upper levels of the stack scan: node and start stacks per level
+  std::vector<int64_t> level_n(1, tt);
+  while (level_n.back() > AT_FAN) level_n.push_back((level_n.back() + AT_FAN - 1) / AT_FAN);
+  for (size_t k = 1; k < level_n.size(); k++)
+    tb += 2 * (Carver::pad(level_n[k] * 4) + Carver::pad(level_n[k] * AT_CAP * 8) +
+               Carver::pad(level_n[k] * AT_CAP * 4));
   void *tmpb = ta_dalloc(h, tb);
   if (!tmpb) return TA_ERR_OOM;
   Carver ct(tmpb);
@@ -704,7 +771,27 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   a.op_last = op_last; a.op_ns = op_ns;
   if (n > 0) {
     k_attr_agg<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
-    if (a.n_lanes > 0) k_attr_carry<<<TA_N (unsigned)((a.n_lanes + 3) / 4), 128, 0, st>>>(a);
+    {
+      // level 0 = tiles; fold upwards until at most AT_FAN stacks remain, scan those, unfold
+      std::vector<StackArr> node(level_n.size()), start(level_n.size());
+      node[0] = StackArr{a.agg_meta, a.agg_e, a.agg_pos};
+      start[0] = StackArr{a.carry_cnt, a.carry_e, a.carry_pos};
+      for (size_t k = 1; k < level_n.size(); k++) {
+        const int64_t c = level_n[k];
+        node[k] = StackArr{ct.take<int32_t>(c), ct.take<i64>(c * AT_CAP), ct.take<int32_t>(c * AT_CAP)};
+        start[k] = StackArr{ct.take<int32_t>(c), ct.take<i64>(c * AT_CAP), ct.take<int32_t>(c * AT_CAP)};
+      }
+      const size_t top = level_n.size() - 1;
+      for (size_t k = 1; k <= top; k++)
+        k_attr_fold_up<<<TA_N (unsigned)((level_n[k] + 3) / 4), 128, 0, st>>>(
+            node[k - 1], level_n[k - 1], node[k], level_n[k], h->d_status);
+      k_attr_fold_top<<<TA_N 1, 32, 0, st>>>(node[top], level_n[top], start[top], top == 0 ? 1 : 0,
+                                            h->d_status);
+      for (size_t k = top; k >= 1; k--)
+        k_attr_fold_down<<<TA_N (unsigned)((level_n[k] + 3) / 4), 128, 0, st>>>(
+            node[k - 1], level_n[k - 1], start[k], level_n[k], start[k - 1], k == 1 ? 1 : 0,
+            h->d_status);
+    }
     k_attr_resolve<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
     k_attr_ops<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
     const int64_t fb = (h->n_valid + 2047) / 2048;
