@@ -274,21 +274,28 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   const int64_t blocks = (int64_t)a.spread * a.per;
   k_agg<<<TA_N (unsigned)blocks, AG_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
+  // Rows are compacted without waiting for their count when a bound on it (dense rows, selected
+  // records) keeps the output small; otherwise the count is fetched first.
   u64 ng = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-  if (ng > 0) {
-    size_t ob = 3 * Carver::pad(ng * 4) + 4 * Carver::pad(ng * 8) + Carver::pad(ng * TA_NBINS * 4) + 256;
+  u64 cap = (u64)G < (u64)h->n_valid ? (u64)G : (u64)h->n_valid;
+  const bool bounded = cap * (28 + 32 + TA_NBINS * 4) <= (256ull << 20);
+  if (!bounded) {
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    cap = ng;
+  }
+  if (cap > 0) {
+    size_t ob = 3 * Carver::pad(cap * 4) + 4 * Carver::pad(cap * 8) + Carver::pad(cap * TA_NBINS * 4) + 256;
     void *outb = ta_dalloc(h, ob);
     if (!outb) return TA_ERR_OOM;
     Carver co(outb);
     AggRowOut ro;
     ro.cnt = a.d_cnt; ro.sum = a.d_sum; ro.minc = a.d_minc; ro.maxb = a.d_maxb; ro.hist = a.d_hist;
     ro.tt = h->d_triples; ro.n_pids = n_pids; ro.R = R; ro.min_name = h->min_name;
-    ro.g_window = co.take<int32_t>(ng); ro.g_pid = co.take<int32_t>(ng); ro.g_name = co.take<int32_t>(ng);
-    ro.g_count = co.take<int64_t>(ng); ro.g_sum = co.take<int64_t>(ng);
-    ro.g_min = co.take<int64_t>(ng); ro.g_max = co.take<int64_t>(ng);
-    ro.g_hist = co.take<u32>(ng * TA_NBINS);
+    ro.g_window = co.take<int32_t>(cap); ro.g_pid = co.take<int32_t>(cap); ro.g_name = co.take<int32_t>(cap);
+    ro.g_count = co.take<int64_t>(cap); ro.g_sum = co.take<int64_t>(cap);
+    ro.g_min = co.take<int64_t>(cap); ro.g_max = co.take<int64_t>(cap);
+    ro.g_hist = co.take<u32>(cap * TA_NBINS);
     ScanTemp t;
     TA_TRY(scan_temp_init(h, scan_mem, G, &t));
     AggRowIn ri{a.d_cnt};
@@ -297,9 +304,10 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
     out->g_count = ro.g_count; out->g_sum = ro.g_sum; out->g_min = ro.g_min; out->g_max = ro.g_max;
     out->g_hist = ro.g_hist;
   }
-  out->n_groups = (int64_t)ng;
+  if (bounded) TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
+  out->n_groups = (int64_t)ng;
   ta_dfree(h, tmpb);
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
   return TA_OK;
