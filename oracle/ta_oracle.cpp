@@ -111,6 +111,11 @@ struct Oracle {
   std::vector<int32_t> r_window, r_pid;
   std::vector<int64_t> r_n_coll, r_sum_wait, r_max_wait, r_n_straggler;
 
+  // gap blame
+  std::vector<int32_t> b_class, b_launch;      // per long gap
+  std::vector<int64_t> b_win_count, b_win_ns;  // [window][class]
+  std::vector<int64_t> op_gap_ns;              // per sorted position
+
   // device-level coverage
   std::vector<int32_t> d_window, d_pid;
   std::vector<int64_t> d_n_events, d_busy, d_idle, d_compute, d_comm, d_overlap, d_exposed;
@@ -352,17 +357,20 @@ struct Oracle {
   // ---- step 6: per-symbol counts and duration statistics (Sec. 8.1 compares
   // per-symbol call counts and kernel durations).
   int aggregate(uint32_t kind_mask, int value_sel) {
-    if (value_sel != 0 && value_sel != 1) return 1;
-    if (value_sel == 1 && kind_mask != (1u << OP)) return 1;
+    if (value_sel < 0 || value_sel > 2) return 1;
+    if (value_sel != 0 && kind_mask != (1u << OP)) return 1;
     struct Row { int64_t count, sum, mn, mx; uint32_t hist[NBINS]; };
     std::map<std::tuple<int32_t, int32_t, int32_t>, Row> rows;
     for (int64_t p = 0; p < n_valid; p++) {
       if (!((1u << kind[p]) & kind_mask)) continue;
       int64_t v;
       if (value_sel == 0) v = ts_end[p] - ts_start[p];
-      else {
+      else if (value_sel == 1) {
         if (op_n_kernels[p] <= 0) continue;
         v = op_last_end[p] - op_first_start[p];
+      } else {  // idle time of the process's device streams that coincides with the operator
+        if (op_gap_ns[p] <= 0) continue;
+        v = op_gap_ns[p];
       }
       auto key = std::make_tuple(win_sorted[p], pid[p], name_id[p]);
       auto it = rows.find(key);
@@ -436,6 +444,56 @@ struct Oracle {
       r_window.push_back(kv.first.first); r_pid.push_back(kv.first.second);
       r_n_coll.push_back(kv.second.n_coll); r_sum_wait.push_back(kv.second.sum_wait);
       r_max_wait.push_back(kv.second.max_wait); r_n_straggler.push_back(kv.second.n_straggler);
+    }
+  }
+
+  // ---- gap blame (needs correlate() and gaps()).  For waits, readiness, dispatch and first
+  // use are compared: ready work dispatched late implicates submission (Sec. 6.2, engine
+  // patterns; "submission gaps", Sec. 8.2), and waits in a host call are matched with the
+  // device idle time they coincide with (Sec. 9.1: waits in one call coincide with 13.8 s of
+  // GPU idle).  Readings, per long gap of the list gaps() made:
+  //   class 3 TAIL        the gap runs to the end of the window (no next record);
+  //   class 0 NO_LAUNCH   the next record has no launch (a COLL record, or launch_of = -1);
+  //   class 1 SUBMISSION  its launch started at or after the gap began (the stream was already
+  //                       idle when the host submitted the work);
+  //   class 2 QUEUED      its launch started before the gap began (submitted in time, started late).
+  // And per OP record: op_gap_ns = sum over the long gaps of ALL device streams of the OP's
+  // (window, process) of the length of [gap_start, gap_start + gap_len) n [ts_start, ts_end).
+  void blame() {
+    const size_t G = long_gaps.size();
+    b_class.assign(G, 0); b_launch.assign(G, -1);
+    b_win_count.assign((size_t)W * 4, 0); b_win_ns.assign((size_t)W * 4, 0);
+    for (size_t k = 0; k < G; k++) {
+      const LongGap& g = long_gaps[k];
+      int cls;
+      if (g.next_event < 0) cls = 3;
+      else {
+        const int32_t l = launch_of[g.next_event];
+        b_launch[k] = l;
+        if (l < 0) cls = 0;
+        else cls = ts_start[l] >= g.gap_start ? 1 : 2;
+      }
+      b_class[k] = cls;
+      const int32_t w = lane_window[g.lane];
+      b_win_count[(size_t)w * 4 + cls]++;
+      b_win_ns[(size_t)w * 4 + cls] += g.gap_len;
+    }
+    // the long gaps of each (window, process), all device streams together
+    std::map<std::pair<int32_t, int32_t>, std::vector<std::pair<int64_t, int64_t>>> idle;
+    for (const LongGap& g : long_gaps)
+      idle[std::make_pair(lane_window[g.lane], lane_pid[g.lane])].push_back(
+          std::make_pair(g.gap_start, g.gap_start + g.gap_len));
+    op_gap_ns.assign(n, 0);
+    for (int64_t p = 0; p < n_valid; p++) {
+      if (kind[p] != OP) continue;
+      auto it = idle.find(std::make_pair(win_sorted[p], pid[p]));
+      if (it == idle.end()) continue;
+      int64_t sum = 0;
+      for (const auto& iv : it->second) {
+        const int64_t lo = std::max(iv.first, ts_start[p]), hi = std::min(iv.second, ts_end[p]);
+        if (hi > lo) sum += hi - lo;
+      }
+      op_gap_ns[p] = sum;
     }
   }
 
@@ -519,6 +577,7 @@ void orc_collectives(void* h, const void* sizes, int32_t n_comms) {
   ((Oracle*)h)->collectives((const CommSize*)sizes, n_comms);
 }
 void orc_device_overlap(void* h) { ((Oracle*)h)->device_overlap(); }
+void orc_blame(void* h) { ((Oracle*)h)->blame(); }
 int64_t orc_n_valid(void* h) { return ((Oracle*)h)->n_valid; }
 
 // Exposes a result array by name: pointer into the oracle's storage, element
@@ -537,6 +596,7 @@ int32_t orc_get(void* h, const char* name, const void** ptr, int64_t* count, int
   G(c_window) G(c_comm) G(c_seq) G(c_n_members) G(c_min_start) G(c_max_start) G(c_skew) G(c_max_end)
   G(c_straggler_pid) G(c_flags) G(wait_ns)
   G(r_window) G(r_pid) G(r_n_coll) G(r_sum_wait) G(r_max_wait) G(r_n_straggler)
+  G(b_class) G(b_launch) G(b_win_count) G(b_win_ns) G(op_gap_ns)
   G(d_window) G(d_pid) G(d_n_events) G(d_busy) G(d_idle) G(d_compute) G(d_comm) G(d_overlap) G(d_exposed)
 #undef G
   return -1;

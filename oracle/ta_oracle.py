@@ -50,6 +50,8 @@ _DTYPES = {
     "c_straggler_pid": np.int32, "c_flags": np.int32, "wait_ns": np.int64,
     "r_window": np.int32, "r_pid": np.int32, "r_n_coll": np.int64, "r_sum_wait": np.int64,
     "r_max_wait": np.int64, "r_n_straggler": np.int64,
+    "b_class": np.int32, "b_launch": np.int32, "b_win_count": np.int64, "b_win_ns": np.int64,
+    "op_gap_ns": np.int64,
     "d_window": np.int32, "d_pid": np.int32, "d_n_events": np.int64, "d_busy": np.int64,
     "d_idle": np.int64, "d_compute": np.int64, "d_comm": np.int64, "d_overlap": np.int64,
     "d_exposed": np.int64,
@@ -89,6 +91,8 @@ def _load():
         lib.orc_collectives.restype = None
         lib.orc_device_overlap.argtypes = [ctypes.c_void_p]
         lib.orc_device_overlap.restype = None
+        lib.orc_blame.argtypes = [ctypes.c_void_p]
+        lib.orc_blame.restype = None
         lib.orc_n_valid.argtypes = [ctypes.c_void_p]
         lib.orc_n_valid.restype = ctypes.c_int64
         lib.orc_get.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_void_p),
@@ -139,6 +143,8 @@ class Oracle:
             out = np.frombuffer(buf, dtype=dt).copy()
         if name in ("lane_hist", "win_hist", "g_hist"):
             out = out.reshape(-1, 40)
+        if name in ("b_win_count", "b_win_ns"):
+            out = out.reshape(-1, 4)
         return out
 
     @property
@@ -172,6 +178,11 @@ class Oracle:
             arr[i] = (cid, nr, 0)
         self._sizes = arr
         self._lib.orc_collectives(self._h, arr.ctypes.data if len(arr) else None, len(arr))
+
+    def blame(self):
+        """Classifies the long gaps of the last gaps() call and charges them to the operators
+        they coincide with (needs correlate() and gaps())."""
+        self._lib.orc_blame(self._h)
 
     def device_overlap(self):
         """Per (window, process): busy / idle over all device streams, compute and

@@ -226,3 +226,36 @@ def device_overlap(sv, wins, n_valid, t0, t1):
         out[key] = (cnt, busy, len(comp) - busy, int(comp.sum()), int(comm.sum()), both,
                     int(comm.sum()) - both)
     return out
+
+
+def blame(sv, wins, n_valid, lane_list, long_gaps, launch_of, t0, t1):
+    """Classes of the long gaps (3 tail, 0 no launch, 1 submission, 2 queued) and, tick by tick,
+    how many device streams of the operator's (window, pid) sit in a long gap while it runs."""
+    cls = []
+    for g in long_gaps:
+        nxt = int(g["next_event"])
+        if nxt < 0:
+            cls.append(3)
+        elif int(launch_of[nxt]) < 0:
+            cls.append(0)
+        else:
+            cls.append(1 if int(sv[int(launch_of[nxt])]["ts_start"]) >= int(g["gap_start"]) else 2)
+    idle = {}
+    for g in long_gaps:
+        w, pid = lane_list[int(g["lane"])][0], lane_list[int(g["lane"])][1]
+        arr = idle.setdefault((w, pid), np.zeros(int(t1[w] - t0[w]), dtype=np.int64))
+        a = int(g["gap_start"]) - int(t0[w])
+        arr[a:a + int(g["gap_len"])] += 1
+    op_gap = np.zeros(len(sv), dtype=np.int64)
+    for p in range(n_valid):
+        if int(sv[p]["kind"]) != 0:
+            continue
+        w = int(wins[p])
+        arr = idle.get((w, int(sv[p]["pid"])))
+        if arr is None:
+            continue
+        a = max(int(sv[p]["ts_start"]) - int(t0[w]), 0)
+        b = min(int(sv[p]["ts_end"]) - int(t0[w]), len(arr))
+        if b > a:
+            op_gap[p] = int(arr[a:b].sum())
+    return cls, op_gap

@@ -133,4 +133,17 @@ def check_H6(run):
     assert r["d_window"].tolist() == [0] * len(want)
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6]
+def check_H7(run):
+    g = load_golden("H7_gap_blame.txt")
+    r = run(g["events"], [0, len(g["events"])], [g["t0"]], [g["t1"]], min_gap=g["min_gap"])
+    e = g["expect"]
+    assert r["b_class"].tolist() == ints(e["classes"])
+    want = [tuple(int(x) for x in t.split(":")) for t in e["class_totals"]]
+    assert [(int(c), int(n)) for c, n in zip(r["b_win_count"][0], r["b_win_ns"][0])] == want
+    charged = [tuple(int(x) for x in t.split(":")) for t in e["charged"]]
+    got = list(zip(r["aggG_g_name"].tolist(), r["aggG_g_count"].tolist(), r["aggG_g_sum"].tolist()))
+    assert got == charged and r["aggG_g_pid"].tolist() == [1, 1]
+    assert int(r["op_gap_ns"].sum()) == sum(c[2] for c in charged)
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7]

@@ -14,6 +14,7 @@ COLL_KEYS = ["c_window", "c_comm", "c_seq", "c_n_members", "c_min_start", "c_max
              "c_max_end", "c_straggler_pid", "c_flags", "wait_ns", "r_window", "r_pid", "r_n_coll",
              "r_sum_wait", "r_max_wait", "r_n_straggler"]
 
+BLAME_KEYS = ["b_class", "b_launch", "b_win_count", "b_win_ns", "op_gap_ns"]
 OVERLAP_KEYS = ["d_window", "d_pid", "d_n_events", "d_busy", "d_idle", "d_compute", "d_comm",
                 "d_overlap", "d_exposed"]
 
@@ -49,6 +50,12 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
     o.collectives(comm_sizes)
     for k in COLL_KEYS:
         r[k] = o.get(k)
+    o.blame()
+    for k in BLAME_KEYS:
+        r[k] = o.get(k)
+    assert o.aggregate(OP_MASK, 2) == 0
+    for k in AGG_KEYS:
+        r[f"aggG_{k}"] = o.get(k)
     o.device_overlap()
     for k in OVERLAP_KEYS:
         r[k] = o.get(k)
@@ -93,6 +100,12 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
         c = w.match_collectives(comm_sizes)
         for k in COLL_KEYS:
             r[k] = c.numpy(k)
+        b = w.blame_gaps(g)
+        for k in BLAME_KEYS:
+            r[k] = b.numpy(k)
+        ag = w.aggregate_ops(OP_MASK, 2)
+        for k in AGG_KEYS:
+            r[f"aggG_{k}"] = ag.numpy(k)
         d = w.device_overlap()
         for k in OVERLAP_KEYS:
             r[k] = d.numpy(k)

@@ -276,3 +276,30 @@ def test_device_overlap_against_tick_bitmaps(seed):
     assert got == rows
     assert list(got) == sorted(got)  # rows come in (window, pid) order
     assert len(rows) > 0
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_gap_blame_against_ticks(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1, min_gap=5, comm_sizes=sizes)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    ll = brute.lanes(sv, wins, r["n_valid"])
+    cls, op_gap = brute.blame(sv, wins, r["n_valid"], ll, r["long_gaps"], r["launch_of"], t0, t1)
+    assert r["b_class"].tolist() == cls
+    assert np.array_equal(r["op_gap_ns"], op_gap)
+    assert len(cls) > 0 and len(set(cls)) >= 2
+    cnt = np.zeros((len(t0), 4), dtype=np.int64)
+    ns = np.zeros((len(t0), 4), dtype=np.int64)
+    for g, c in zip(r["long_gaps"], cls):
+        w = ll[int(g["lane"])][0]
+        cnt[w, c] += 1
+        ns[w, c] += int(g["gap_len"])
+    assert np.array_equal(r["b_win_count"], cnt) and np.array_equal(r["b_win_ns"], ns)
+    # the per-name table is the plain aggregate of the per-operator figures
+    rows = brute.aggregate(sv, wins, r["n_valid"], 1, [int(v) if v > 0 else None for v in op_gap])
+    assert len(rows) == len(r["aggG_g_count"])
+    for i, (key, row) in enumerate(rows):
+        assert (int(r["aggG_g_window"][i]), int(r["aggG_g_pid"][i]), int(r["aggG_g_name"][i])) == key
+        assert int(r["aggG_g_count"][i]) == row["count"] and int(r["aggG_g_sum"][i]) == row["sum"]
+        assert int(r["aggG_g_min"][i]) == row["min"] and int(r["aggG_g_max"][i]) == row["max"]

@@ -112,3 +112,9 @@ def test_injected_stalls_show_up_as_long_gaps():
     interior = r["long_gaps"][r["long_gaps"]["next_event"] >= 0]
     assert len(interior) == n_long_truth
     assert np.array_equal(np.sort(r["gap_before"][interior["next_event"]]), np.sort(val[dev & (val >= 500_000)]))
+    # a host stall right before a launch leaves the stream idle until the host submits: every
+    # such gap is submission-bound
+    cls = r["b_class"][r["long_gaps"]["next_event"] >= 0]
+    assert (cls == 1).mean() > 0.95 and not (cls == 3).any()
+    assert int(r["b_win_count"].sum()) == len(r["long_gaps"])
+    assert int(r["b_win_ns"].sum()) == int(r["long_gaps"]["gap_len"].sum())
