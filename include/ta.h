@@ -272,7 +272,9 @@ ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out);
  * Population: kept records with (1 << kind) & kind_mask.  value_sel 0: value =
  * ts_end - ts_start.  value_sel 1: kind_mask must be exactly 1 << TA_KIND_OP
  * (else INVALID_ARG); the population is further restricted to OPs with
- * op_n_kernels > 0 and value = T_op.  Group key (window, pid, name_id); one
+ * op_n_kernels > 0 and value = T_op.  value_sel 2 (after ta_blame_gaps, else
+ * TA_ERR_ORDER; kind_mask again exactly 1 << TA_KIND_OP): OPs with
+ * op_gap_ns > 0, value = op_gap_ns.  Group key (window, pid, name_id); one
  * output row per non-empty group in ascending signed key order with count,
  * sum, min, max and a histogram whose bin is min(39, floor(log2 v)) for
  * v >= 1 and 0 for v <= 0.
@@ -363,6 +365,50 @@ typedef struct ta_overlap_result {
 } ta_overlap_result;
 
 ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out);
+
+/* ------------------------------------------------------------------------
+ * ta_blame_gaps - why a device stream sat idle, and which host calls the idle
+ * time coincides with.  For waits, readiness, dispatch and first use are
+ * compared: ready work dispatched late implicates submission (Sec. 6.2, engine
+ * patterns; "submission gaps", Sec. 8.2); waits in one host call are found to
+ * coincide with the GPU idle time (Sec. 9.1).  Beyond the seven calls above.
+ * Needs ta_correlate_launches and the result of a ta_stream_gaps call on the
+ * same handle (`gaps`, borrowed for the duration of the call).
+ *
+ * Readings (the paper gives no rule).  Per long gap k of gaps->long_gaps:
+ *   g_class[k] = TA_BLAME_TAIL        the gap runs to the window end (next_event = -1)
+ *                TA_BLAME_NO_LAUNCH   the record that ends it has launch_of = -1
+ *                                     (COLL records, kernels whose launch is missing)
+ *                TA_BLAME_SUBMISSION  ts_start[launch] >= gap_start: the stream was
+ *                                     already idle when the host submitted the work
+ *                TA_BLAME_QUEUED      ts_start[launch] <  gap_start: submitted in
+ *                                     time, started late (queue, dependency)
+ *   g_launch[k] = that launch's sorted position, or -1.
+ * out_summary[w].count[c] / .ns[c]: number and total length of the long gaps of
+ * window w per class c.
+ * Per OP record r: op_gap_ns[r] = sum, over the long gaps of ALL device streams
+ * of r's (window, pid), of the length of [gap_start, gap_start + gap_len) n
+ * [ts_start[r], ts_end[r]); 0 at every other position.  With one stream per
+ * device this is the GPU idle time that coincides with the call; with several
+ * streams it is stream-idle time (each stream counts).  The per-symbol table is
+ * ta_aggregate_ops(h, 1 << TA_KIND_OP, 2, ...): operators with op_gap_ns > 0.
+ * All arrays are device memory owned by the handle.
+ * Errors: TA_ERR_ORDER before ta_correlate_launches; TA_ERR_INVALID_ARG;
+ * TA_ERR_OOM; TA_ERR_CUDA; TA_ERR_TIMEOUT.  One stream synchronisation. */
+enum { TA_BLAME_NO_LAUNCH = 0, TA_BLAME_SUBMISSION = 1, TA_BLAME_QUEUED = 2, TA_BLAME_TAIL = 3 };
+
+typedef struct ta_blame_summary {
+  int64_t count[4], ns[4]; /* indexed by TA_BLAME_* */
+} ta_blame_summary;
+
+typedef struct ta_blame_result {
+  int64_t n_long_gaps;
+  const int32_t *g_class, *g_launch; /* device, n_long_gaps */
+  const int64_t *op_gap_ns;          /* device, n           */
+} ta_blame_result;
+
+ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
+                        ta_blame_summary *out_summary /* host, n_windows entries */);
 
 /* ta_free - releases every buffer of the handle through env.release.
  * NULL-safe.  Synchronises the handle's stream first. */

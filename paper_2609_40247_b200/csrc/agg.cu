@@ -35,6 +35,7 @@ struct AggArgs {
   const int32_t *lane_off, *lane_slot;
   const int32_t *op_n;
   const int64_t *op_first, *op_last;
+  const int64_t *op_gap;  // value_sel 2
   uint32_t kind_mask;
   int value_sel;
   int64_t min_name, R;
@@ -129,34 +130,41 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
       if (p0 + AG_ITEMS <= end) {
         uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
         const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
-  #pragma unroll
+#pragma unroll
         for (int j = 0; j < AG_ITEMS; j++) kd[j] = hq[j];
       } else {
-  #pragma unroll
+#pragma unroll
         for (int j = 0; j < AG_ITEMS; j++) kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
       }
       bool sel[AG_ITEMS];
       i64 v[AG_ITEMS];
       int32_t nm[AG_ITEMS];
-  #pragma unroll
+#pragma unroll
       for (int j = 0; j < AG_ITEMS; j++) {
         sel[j] = kd[j] >= 0 && ((a.kind_mask >> kd[j]) & 1u);
         v[j] = 0;
         nm[j] = 0;
       }
       if (a.value_sel == 0) {
-  #pragma unroll
+#pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
-      } else {
-  #pragma unroll
+      } else if (a.value_sel == 1) {
+#pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) sel[j] = a.op_n[p0 + j] > 0;
-  #pragma unroll
+#pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
+      } else {
+#pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) { v[j] = a.op_gap[p0 + j]; sel[j] = v[j] > 0; }
+#pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) nm[j] = a.name[p0 + j];
       }
-  #pragma unroll
+#pragma unroll
       for (int j = 0; j < AG_ITEMS; j++) {
         if (!sel[j]) continue;
         const int lane = lw.at(p0 + j);
@@ -263,6 +271,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.kind = h->sorted.kind; a.name = h->sorted.name_id; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot;
   a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
+  a.op_gap = h->d_op_gap_ns;
   a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
   a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   const bool host_kinds = (a.kind_mask & 7u) != 0, dev_kinds = (a.kind_mask & 56u) != 0;

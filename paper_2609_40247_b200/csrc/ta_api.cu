@@ -248,6 +248,7 @@ ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
   h->events_copy = nullptr;
   h->d_keys = nullptr;
   h->attr_status = 0;
+  h->d_op_gap_ns = nullptr;
   h->h_off.assign(win_off, win_off + W + 1);
   h->h_t0.assign(win_t0, win_t0 + W);
   h->h_t1.assign(win_t1, win_t1 + W);
@@ -296,10 +297,11 @@ ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out) {
 
 ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel, ta_agg_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
-  if (value_sel != 0 && value_sel != 1) return TA_ERR_INVALID_ARG;
-  if (value_sel == 1 && kind_mask != (1u << TA_KIND_OP)) return TA_ERR_INVALID_ARG;
+  if (value_sel < 0 || value_sel > 2) return TA_ERR_INVALID_ARG;
+  if (value_sel != 0 && kind_mask != (1u << TA_KIND_OP)) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
   if (value_sel == 1 && (!(h->stage & 8) || h->attr_status != 0)) return TA_ERR_ORDER;
+  if (value_sel == 2 && !h->d_op_gap_ns) return TA_ERR_ORDER;
   return ta_run_aggregate(h, kind_mask, value_sel, out);
 }
 
@@ -308,6 +310,18 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes, int32_t 
   if (!h || !out || n_comms < 0 || (n_comms > 0 && !sizes)) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
   return ta_run_collectives(h, sizes, n_comms, out);
+}
+
+ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
+                        ta_blame_summary *out_summary) {
+  if (!h || !gaps || !out || !out_summary) return TA_ERR_INVALID_ARG;
+  if (gaps->n_long_gaps < 0 || (gaps->n_long_gaps > 0 && !gaps->long_gaps)) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 4)) return TA_ERR_ORDER;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
+  return ta_run_blame(h, gaps, out, out_summary);
 }
 
 ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out) {

@@ -88,6 +88,7 @@ struct ta_window {
   int32_t *d_lane_slot;      // per lane: window * n_pids + pid rank
   int32_t *d_lane_dom_end;   // per lane: first position behind the run of lanes of the same domain
   int32_t *d_lane_dev_base;  // per device lane: number of device records in earlier lanes
+  int32_t *d_lane_dom_next;  // per lane: index of the first later lane of the other domain
   int64_t n_device;          // kept device records
   i64 *d_slot_min, *d_slot_max;               // per slot: corr_id range of its LAUNCH records
   std::vector<int64_t> h_slot_min, h_slot_max;  // host copies (INT64_MAX / INT64_MIN when none)
@@ -95,6 +96,7 @@ struct ta_window {
   // join / attribution products
   ta_join_result join;
   ta_attr_result attr;
+  const int64_t *d_op_gap_ns;  // per sorted position, set by the gap blame (null before)
   int attr_status;
 };
 
@@ -160,6 +162,9 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
 
 // overlap.cu
 ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out);
+// blame.cu
+ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
+                       ta_blame_summary *out_summary);
 
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 

@@ -210,8 +210,9 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
                                                      int32_t *lane_pid, int16_t *lane_stream,
                                                      int16_t *lane_domain, int32_t *lane_off,
                                                      int32_t *lane_code, int32_t *lane_slot,
-                                                     int32_t *lane_dom_end, int32_t *lane_dev_base,
-                                                     int32_t *n_lanes_out, int64_t cap) {
+                                                     int32_t *lane_dom_end, int32_t *lane_dom_next,
+                                                     int32_t *lane_dev_base, int32_t *n_lanes_out,
+                                                     int64_t cap) {
   __shared__ u64 tmp[33];
   __shared__ u64 base;
   if (threadIdx.x == 0) base = 0;
@@ -252,6 +253,7 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
     int64_t m = l + 1;
     while (m < L && lane_domain[m] == lane_domain[l]) m++;
     lane_dom_end[l] = m < L ? lane_off[m] : (int32_t)n_valid;
+    lane_dom_next[l] = (int32_t)m;  // index of the first later lane of the other domain (L if none)
   }
   // per device lane: how many device records sit in earlier lanes (their index once the device
   // records are taken out in order); n_lanes_out[1] = the number of device records
@@ -297,7 +299,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
 
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
-                2 * Carver::pad(n * 2) + 6 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
+                2 * Carver::pad(n * 2) + 7 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
                 Carver::pad((lane_cap + 1) * 4) + 2 * Carver::pad((size_t)n_slots * 8) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
@@ -312,6 +314,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *lane_off = ck.take<int32_t>(lane_cap + 1);
   int32_t *lane_dom_end = ck.take<int32_t>(lane_cap);
   int32_t *lane_dev_base = ck.take<int32_t>(lane_cap);
+  int32_t *lane_dom_next = ck.take<int32_t>(lane_cap);
   int32_t *n_lanes_dev = ck.take<int32_t>(2);  // [0] lanes, [1] device records
   h->d_slot_min = ck.take<i64>(n_slots);
   h->d_slot_max = ck.take<i64>(n_slots);
@@ -419,7 +422,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     k_lane_table<<<TA_N 1, 1024, 0, st>>>(lane_start, n_codes, h->tbits,
                                      h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
                                      lane_window, lane_pid, lane_stream, lane_domain, lane_off,
-                                     lane_code, lane_slot, lane_dom_end, lane_dev_base, n_lanes_dev, lane_cap);
+                                     lane_code, lane_slot, lane_dom_end, lane_dom_next, lane_dev_base, n_lanes_dev,
+                                     lane_cap);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_CHECK_CUDA(h, cudaMemcpyAsync(n_lanes_host, n_lanes_dev, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
@@ -449,5 +453,6 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   h->d_lane_slot = lane_slot;
   h->d_lane_dom_end = lane_dom_end;
   h->d_lane_dev_base = lane_dev_base;
+  h->d_lane_dom_next = lane_dom_next;
   return TA_OK;
 }

@@ -81,6 +81,8 @@ _CollResult = _ptr_struct("_CollResult", [
     ("g_skew", _vp), ("g_max_end", _vp), ("g_straggler_pid", _vp), ("g_flags", _vp),
     ("wait_ns", _vp), ("r_window", _vp), ("r_pid", _vp), ("r_n_coll", _vp), ("r_sum_wait", _vp),
     ("r_max_wait", _vp), ("r_n_straggler", _vp)])
+_BlameResult = _ptr_struct("_BlameResult", [
+    ("n_long_gaps", ctypes.c_int64), ("g_class", _vp), ("g_launch", _vp), ("op_gap_ns", _vp)])
 _OverlapResult = _ptr_struct("_OverlapResult", [
     ("n_rows", ctypes.c_int64), ("d_window", _vp), ("d_pid", _vp), ("d_n_events", _vp),
     ("d_busy", _vp), ("d_idle", _vp), ("d_compute", _vp), ("d_comm", _vp), ("d_overlap", _vp),
@@ -89,7 +91,7 @@ _OverlapResult = _ptr_struct("_OverlapResult", [
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
-           "ta_lane_gaps_noalloc", "ta_device_overlap"]
+           "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -126,6 +128,8 @@ def lib():
         L.ta_aggregate_ops.argtypes = [_vp, ctypes.c_uint32, ctypes.c_int32, ctypes.POINTER(_AggResult)]
         L.ta_match_collectives.restype = ctypes.c_int
         L.ta_match_collectives.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(_CollResult)]
+        L.ta_blame_gaps.restype = ctypes.c_int
+        L.ta_blame_gaps.argtypes = [_vp, _vp, ctypes.POINTER(_BlameResult), _vp]
         L.ta_device_overlap.restype = ctypes.c_int
         L.ta_device_overlap.argtypes = [_vp, ctypes.POINTER(_OverlapResult)]
         L.ta_free.restype = None
@@ -311,6 +315,25 @@ class CollResult(_Result):
         return super().tensor(self._names.get(name, name))
 
 
+BLAME_SUM = np.dtype([("count", "<i8", (4,)), ("ns", "<i8", (4,))])
+
+
+class BlameResult(_Result):
+    _names = {"b_class": "g_class", "b_launch": "g_launch"}
+    _layout = {"g_class": ("<i4", lambda r: r.n_long_gaps), "g_launch": ("<i4", lambda r: r.n_long_gaps),
+               "op_gap_ns": ("<i8", lambda r: r.n)}
+
+    def numpy(self, name):
+        if name == "b_win_count":
+            return self.blame_sum["count"].astype(np.int64).reshape(-1, 4)
+        if name == "b_win_ns":
+            return self.blame_sum["ns"].astype(np.int64).reshape(-1, 4)
+        return super().numpy(self._names.get(name, name))
+
+    def tensor(self, name):
+        return super().tensor(self._names.get(name, name))
+
+
 class OverlapResult(_Result):
     _layout = dict([("d_window", ("<i4", lambda r: r.n_rows)), ("d_pid", ("<i4", lambda r: r.n_rows))] +
                    [(k, ("<i8", lambda r: r.n_rows)) for k in
@@ -445,6 +468,15 @@ class Window:
         if st != 0:
             raise TaError(st, "ta_aggregate_ops")
         return AggResult(self, raw, dict(self._dims(), n_groups=raw.n_groups))
+
+    def blame_gaps(self, gaps) -> BlameResult:
+        """gaps: the GapResult of an earlier stream_gaps() call on this window."""
+        raw = _BlameResult()
+        summ = np.zeros(self.W, dtype=BLAME_SUM)
+        st = self._lib.ta_blame_gaps(self._h, ctypes.byref(gaps._raw), ctypes.byref(raw), summ.ctypes.data)
+        if st != 0:
+            raise TaError(st, "ta_blame_gaps")
+        return BlameResult(self, raw, dict(self._dims(), n_long_gaps=raw.n_long_gaps, blame_sum=summ))
 
     def device_overlap(self) -> OverlapResult:
         raw = _OverlapResult()

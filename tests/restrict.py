@@ -12,8 +12,8 @@ host, where they are compared with the oracle run on the subset.
 import numpy as np
 
 from paper_2609_40247_b200.ta import NBINS
-from runners import (AGG_KEYS, ATTR_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS, OP_MASK,
-                     OVERLAP_KEYS)
+from runners import (AGG_KEYS, ATTR_KEYS, BLAME_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS,
+                     OP_MASK, OVERLAP_KEYS)
 
 _POSITIONAL = {"launch_of", "parent", "op_of"}  # values are sorted positions (or -1)
 _PER_RECORD_SORT = ["ts_start", "ts_end", "corr_id", "pid", "name_id", "seq", "stream", "kind"]
@@ -67,10 +67,12 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
         ag_op = w.aggregate_ops(OP_MASK, 1) if a.status == 0 else None
         c = w.match_collectives(comm_sizes)
         ov = w.device_overlap()
+        bl = w.blame_gaps(g)
+        ag_gap = w.aggregate_ops(OP_MASK, 2)
         del buf
         if checks is not None:
             checks(dict(window=w, sort=s, join=j, attr=a, gaps=g, agg_dev=ag_dev, agg_op=ag_op,
-                        coll=c, overlap=ov))
+                        coll=c, overlap=ov, blame=bl))
         n, n_valid = s.n, s.n_valid
         perm = _typed(s, "perm")[0].long()
         lane_off = _typed(s, "lane_off")[0].long()
@@ -148,8 +150,26 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
                     r["long_gaps"] = cols.contiguous().cpu().numpy().reshape(-1).view(dt).copy()
                 else:
                     r["long_gaps"] = np.empty(0, dtype=dt)
+            if "blame" in sub.groups:
+                r["op_gap_ns"] = per_record(bl, "op_gap_ns")
+                t, dt = _typed(g, "long_gaps")
+                if t.shape[0]:
+                    lanes_of = t.reshape(-1).view(torch.int32).reshape(-1, dt.itemsize // 4)[:, 0]
+                    rows = lkeep[lanes_of.long()]
+                    r["b_class"] = _host(_typed(bl, "b_class")[0][rows], np.dtype("<i4"))
+                    v = _typed(bl, "b_launch")[0][rows]
+                    r["b_launch"] = _host(torch.where(v >= 0, pos_map[v.clamp(min=0).long()], v),
+                                          np.dtype("<i4"))
+                else:
+                    r["b_class"] = np.empty(0, dtype=np.int32)
+                    r["b_launch"] = np.empty(0, dtype=np.int32)
+                if sub.windows is not None:
+                    r["b_win_count"] = bl.numpy("b_win_count")[wkeep]
+                    r["b_win_ns"] = bl.numpy("b_win_ns")[wkeep]
             if "agg" in sub.groups:
-                for tag, res in (("agg0", ag_dev), ("aggT", ag_op)):
+                for tag, res in (("agg0", ag_dev), ("aggT", ag_op), ("aggG", ag_gap)):
+                    if tag == "aggG" and "blame" not in sub.groups:
+                        continue
                     if res is None:
                         continue
                     gw = _typed(res, "g_window")[0]
