@@ -140,9 +140,12 @@ def run_pipeline(ta, buf, wl, read_back=False, per_call=None):
         mark("aggregate_ops(OP, T_op)")
         c = w.match_collectives(wl.comm_sizes)
         mark("match_collectives")
-        if per_call is not None:  # the first analysis built on top of the hot path: not part of a step
+        if per_call is not None:  # analyses built on top of the hot path: not part of a step
             w.device_overlap()
             mark("device_overlap (outside the timed step)")
+            w.blame_gaps(g)
+            w.aggregate_ops(1 << ta.KIND_OP, 2)
+            mark("blame_gaps + aggregate_ops(OP, idle charged) (outside the timed step)")
         nbytes = w.load_summary.nbytes + j.join_sum.nbytes + a.attr_sum.nbytes
         if read_back:
             for res, names in ((g, ("lane_gaps", "win_hist", "long_gaps")),

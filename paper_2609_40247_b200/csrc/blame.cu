@@ -102,18 +102,33 @@ __global__ void __launch_bounds__(256) k_blame_lanes(BlameArgs a) {
   a.lane_first[l] = (int32_t)lo;
 }
 
-// total long-gap length of list range [first, last) that lies before time t
-__device__ __forceinline__ i64 gap_time_before(const BlameArgs &a, int64_t first, int64_t last, i64 t) {
-  int64_t lo = first, hi = last;  // number of gaps that start before t
+// number of gaps of list range [first, last) that start before time t
+__device__ __forceinline__ int64_t gaps_started_before(const BlameArgs &a, int64_t first, int64_t last,
+                                                       i64 t) {
+  int64_t lo = first, hi = last;
   while (lo < hi) {
     const int64_t mid = (lo + hi) >> 1;
     if (a.list[mid].gap_start < t) lo = mid + 1;
     else hi = mid;
   }
-  if (lo == first) return 0;
-  const int64_t k = lo - 1;
+  return lo;
+}
+// total long-gap length of the range that lies before time t, given i = gaps_started_before(t)
+__device__ __forceinline__ i64 gap_time_before(const BlameArgs &a, int64_t first, int64_t i, i64 t) {
+  if (i == first) return 0;
+  const int64_t k = i - 1;
   const i64 part = t - a.list[k].gap_start, len = a.list[k].gap_len;
   return (i64)(a.pre[k] - a.pre[first]) + (part < len ? part : len);
+}
+// length of [s, e) that lies inside the gaps of the range
+__device__ __forceinline__ i64 gap_time_within(const BlameArgs &a, int64_t first, int64_t last, i64 s,
+                                               i64 e) {
+  const int64_t ie = gaps_started_before(a, first, last, e);
+  if (ie == first) return 0;  // every gap starts at or after e
+  const ta_long_gap g = a.list[ie - 1];
+  if (g.gap_start < s && g.gap_start + g.gap_len <= s) return 0;  // the last gap before e ends before s
+  const int64_t is = g.gap_start < s ? ie : gaps_started_before(a, first, ie, s);
+  return gap_time_before(a, first, ie, e) - gap_time_before(a, first, is, s);
 }
 
 __global__ void __launch_bounds__(BL_THREADS) k_blame_ops(BlameArgs a) {
@@ -161,7 +176,7 @@ __global__ void __launch_bounds__(BL_THREADS) k_blame_ops(BlameArgs a) {
     for (int d = dlo; d < dhi; d++) {
       const int64_t first = a.lane_first[d], last = a.lane_first[d + 1];
       if (first == last) continue;
-      sum += gap_time_before(a, first, last, e[j]) - gap_time_before(a, first, last, s[j]);
+      sum += gap_time_within(a, first, last, s[j], e[j]);
     }
     if (sum) a.op_gap_ns[p] = sum;
   }
