@@ -17,17 +17,6 @@
 #include "scan.cuh"
 #include "ta_internal.cuh"
 
-struct CollSelIn {
-  const int16_t *kind;
-  int64_t n_valid;
-  __device__ u64 operator()(int64_t i) const { return (i < n_valid && kind[i] == TA_KIND_COLL) ? 1ull : 0ull; }
-};
-struct CollSelOut {
-  u32 *pos;
-  __device__ void operator()(int64_t i, u64 excl, u64 v) const {
-    if (v) pos[excl] = (u32)i;
-  }
-};
 
 struct CollCtx {
   int64_t m;

@@ -73,53 +73,6 @@ __device__ __forceinline__ void tile_lane_range(int my_lo, int my_hi, int *s_lo,
   __syncthreads();
 }
 
-// ---- pass 1: corr range of the LAUNCH records of every slot ----------------
-__global__ void __launch_bounds__(JN_THREADS) k_join_minmax(JoinArgs a) {
-  __shared__ u64 tmp[33];
-  __shared__ int s_lo, s_hi;
-  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
-  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
-  int ln[JN_ITEMS];
-  i64 c[JN_ITEMS];
-  int my_lo = INT_MAX, my_hi = -1;
-#pragma unroll
-  for (int j = 0; j < JN_ITEMS; j++) {
-    int64_t p = p0 + j;
-    ln[j] = -1;
-    c[j] = 0;
-    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
-      ln[j] = lw.at(p);
-      c[j] = a.corr[p];
-      my_lo = min(my_lo, ln[j]);
-      my_hi = max(my_hi, ln[j]);
-    }
-  }
-  int l0, l1;
-  tile_lane_range(my_lo, my_hi, &s_lo, &s_hi, &l0, &l1);
-  for (int l = l0; l <= l1; l++) {
-    if (a.lane_domain[l] != 0) continue;
-    u64 mx = 0, mn_inv = 0;
-#pragma unroll
-    for (int j = 0; j < JN_ITEMS; j++)
-      if (ln[j] == l) {
-        mx = max(mx, bias64(c[j]) + 0);
-        mn_inv = max(mn_inv, ~bias64(c[j]));
-      }
-    bool any = false;
-#pragma unroll
-    for (int j = 0; j < JN_ITEMS; j++) any |= (ln[j] == l);
-    u64 cnt = blk_reduce(any ? 1 : 0, false, tmp);
-    if (cnt == 0) continue;
-    // threads without an item contribute neutral elements: bias64 maps INT64_MIN to 0
-    mx = blk_reduce(any ? mx : 0, true, tmp);
-    mn_inv = blk_reduce(any ? mn_inv : 0, true, tmp);
-    if (threadIdx.x == 0) {
-      int slot = a.lane_slot[l];
-      atomicMax(&a.slot_max[slot], unbias64(mx));
-      atomicMin(&a.slot_min[slot], unbias64(~mn_inv));
-    }
-  }
-}
 
 // ---- direct path: fill the table -------------------------------------------
 __global__ void __launch_bounds__(JN_THREADS) k_join_build(JoinArgs a) {
@@ -376,21 +329,6 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
 }
 
 // ---- general path helpers -----------------------------------------------------
-struct JoinSelIn {
-  const int16_t *kind;
-  int64_t n_valid;
-  __device__ u64 operator()(int64_t i) const {
-    if (i >= n_valid) return 0;
-    int k = kind[i];
-    return (k == TA_KIND_LAUNCH || k == TA_KIND_KERNEL || k == TA_KIND_MEMCPY) ? 1ull : 0ull;
-  }
-};
-struct JoinSelOut {
-  u32 *pos;
-  __device__ void operator()(int64_t i, u64 excl, u64 v) const {
-    if (v) pos[excl] = (u32)i;
-  }
-};
 __global__ void __launch_bounds__(256) k_join_key_corr(const u32 *pos, int64_t m, const int64_t *corr,
                                                        u64 *out) {
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;

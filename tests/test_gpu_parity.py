@@ -52,19 +52,31 @@ def test_larger_random_window_spans_tiles():
     both(ev, off, t0, t1, min_gap=1, comm_sizes=sizes)
 
 
-@pytest.mark.parametrize("run_len", [2, 5, 31, 48, 49, 400])
-def test_runs_of_equal_start_times(run_len):
+def test_sparse_correlation_ids_take_the_sort_merge_join():
+    """Correlation ids spread over a range far wider than the record count: the direct-address
+    table is not used, launches and probes are matched by sorting (several tiles of each)."""
+    wl = synth.make_workload("c1", 0.02, truth=False)
+    ev = wl.events.copy()
+    dev_or_launch = ev["kind"] != 5
+    ev["corr_id"][dev_or_launch] = ev["corr_id"][dev_or_launch] * 1_000_003 - 2**45
+    o, g = both(ev, wl.win_off, wl.win_t0, wl.win_t1, comm_sizes=wl.comm_sizes)
+    assert int(o["join_sum"]["n_matched"].sum()) > 20_000
+
+
+@pytest.mark.parametrize("run_len,ordinary", [(2, 300), (5, 300), (31, 300), (48, 300), (49, 300),
+                                              (400, 300), (60, 12000)])
+def test_runs_of_equal_start_times(run_len, ordinary):
     """Many records of one stream start at the same time: their order (longer first, then
     input order) comes from the run ranking of the gather up to 48 members, and from the
     full-resolution pair sort with its duration key beyond that."""
-    rng = np.random.default_rng(run_len)
+    rng = np.random.default_rng(run_len + ordinary)
     rows = []
     for pid in (4, 9):
         for s0 in (100, 5000, 5001):
             for i in range(run_len):
                 dur = int(rng.integers(0, 6))  # few distinct durations: equal intervals too
                 rows.append(("KERNEL", pid, 1, s0, s0 + dur, int(rng.integers(0, 50)), i % 3, 0))
-        for i in range(300):  # ordinary traffic around the runs
+        for i in range(ordinary):  # ordinary traffic around the runs
             s = int(rng.integers(0, 9000))
             rows.append(("KERNEL", pid, int(rng.integers(0, 2)), s, s + int(rng.integers(0, 40)),
                          int(rng.integers(0, 50)), int(rng.integers(0, 4)), 0))
