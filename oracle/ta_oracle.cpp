@@ -111,6 +111,12 @@ struct Oracle {
   std::vector<int32_t> r_window, r_pid;
   std::vector<int64_t> r_n_coll, r_sum_wait, r_max_wait, r_n_straggler;
 
+  // inclusive roll-up and graph replays
+  std::vector<int32_t> incl_n_kernels;
+  std::vector<int64_t> incl_first_start, incl_last_end, incl_kernel_ns;
+  std::vector<int64_t> replay_first_start, replay_last_end, replay_kernel_ns;
+  std::vector<int64_t> roll_sum;  // [window][3]: graph launches, their kernels, most kernels of one launch
+
   // gap blame
   std::vector<int32_t> b_class, b_launch;      // per long gap
   std::vector<int64_t> b_win_count, b_win_ns;  // [window][class]
@@ -447,6 +453,55 @@ struct Oracle {
     }
   }
 
+  // ---- inclusive operator figures and graph replays (needs attribute() without error).
+  // An invocation's kernel composition comes from the call-to-kernel links, and T_op spans the
+  // first kernel start to the last completion (Sec. 6.1, "Operator execution and efficiency").
+  // Readings: the inclusive figures of an OP are those of the OP itself plus those of every OP
+  // below it in the parent forest (count and nanoseconds add; first start is the minimum and
+  // last end the maximum over the OPs that own kernels; all zero when the subtree owns none).
+  // CUDA Graph replay hides the operator calls and launch correlations separate the replays:
+  // a LAUNCH that owns two or more device records is one replay, spanning the first start to
+  // the last end of those records, with the sum of their durations; all zero for other launches.
+  void rollup() {
+    incl_n_kernels.assign(n, 0); incl_kernel_ns.assign(n, 0);
+    incl_first_start.assign(n, 0); incl_last_end.assign(n, 0);
+    for (int64_t p = 0; p < n_valid; p++) {
+      if (kind[p] != OP || op_n_kernels[p] <= 0) continue;
+      incl_n_kernels[p] = op_n_kernels[p]; incl_kernel_ns[p] = op_kernel_ns[p];
+      incl_first_start[p] = op_first_start[p]; incl_last_end[p] = op_last_end[p];
+    }
+    // a child always follows its parent in canonical order: going backwards, every OP is
+    // complete before it is added to its parent
+    for (int64_t p = n_valid - 1; p >= 0; p--) {
+      if (kind[p] != OP || incl_n_kernels[p] <= 0 || parent[p] < 0) continue;
+      const int32_t q = parent[p];
+      if (incl_n_kernels[q] == 0) { incl_first_start[q] = incl_first_start[p]; incl_last_end[q] = incl_last_end[p]; }
+      else {
+        incl_first_start[q] = std::min(incl_first_start[q], incl_first_start[p]);
+        incl_last_end[q] = std::max(incl_last_end[q], incl_last_end[p]);
+      }
+      incl_n_kernels[q] += incl_n_kernels[p]; incl_kernel_ns[q] += incl_kernel_ns[p];
+    }
+    replay_first_start.assign(n, 0); replay_last_end.assign(n, 0); replay_kernel_ns.assign(n, 0);
+    roll_sum.assign((size_t)W * 3, 0);
+    std::vector<uint8_t> seen(n, 0);
+    for (int64_t p = 0; p < n_valid; p++) {
+      const int32_t l = (kind[p] == KERNEL || kind[p] == MEMCPY) ? launch_of[p] : -1;
+      if (l < 0 || kernels_of_launch[l] < 2) continue;
+      if (!seen[l]) { seen[l] = 1; replay_first_start[l] = ts_start[p]; replay_last_end[l] = ts_end[p]; }
+      else {
+        replay_first_start[l] = std::min(replay_first_start[l], ts_start[p]);
+        replay_last_end[l] = std::max(replay_last_end[l], ts_end[p]);
+      }
+      replay_kernel_ns[l] += ts_end[p] - ts_start[p];
+    }
+    for (int64_t p = 0; p < n_valid; p++) {
+      if (kind[p] != LAUNCH || kernels_of_launch[p] < 2) continue;
+      int64_t* r = &roll_sum[(size_t)win_sorted[p] * 3];
+      r[0]++; r[1] += kernels_of_launch[p]; r[2] = std::max<int64_t>(r[2], kernels_of_launch[p]);
+    }
+  }
+
   // ---- gap blame (needs correlate() and gaps()).  For waits, readiness, dispatch and first
   // use are compared: ready work dispatched late implicates submission (Sec. 6.2, engine
   // patterns; "submission gaps", Sec. 8.2), and waits in a host call are matched with the
@@ -578,6 +633,7 @@ void orc_collectives(void* h, const void* sizes, int32_t n_comms) {
 }
 void orc_device_overlap(void* h) { ((Oracle*)h)->device_overlap(); }
 void orc_blame(void* h) { ((Oracle*)h)->blame(); }
+void orc_rollup(void* h) { ((Oracle*)h)->rollup(); }
 int64_t orc_n_valid(void* h) { return ((Oracle*)h)->n_valid; }
 
 // Exposes a result array by name: pointer into the oracle's storage, element
@@ -596,6 +652,8 @@ int32_t orc_get(void* h, const char* name, const void** ptr, int64_t* count, int
   G(c_window) G(c_comm) G(c_seq) G(c_n_members) G(c_min_start) G(c_max_start) G(c_skew) G(c_max_end)
   G(c_straggler_pid) G(c_flags) G(wait_ns)
   G(r_window) G(r_pid) G(r_n_coll) G(r_sum_wait) G(r_max_wait) G(r_n_straggler)
+  G(incl_n_kernels) G(incl_first_start) G(incl_last_end) G(incl_kernel_ns)
+  G(replay_first_start) G(replay_last_end) G(replay_kernel_ns) G(roll_sum)
   G(b_class) G(b_launch) G(b_win_count) G(b_win_ns) G(op_gap_ns)
   G(d_window) G(d_pid) G(d_n_events) G(d_busy) G(d_idle) G(d_compute) G(d_comm) G(d_overlap) G(d_exposed)
 #undef G

@@ -50,6 +50,9 @@ _DTYPES = {
     "c_straggler_pid": np.int32, "c_flags": np.int32, "wait_ns": np.int64,
     "r_window": np.int32, "r_pid": np.int32, "r_n_coll": np.int64, "r_sum_wait": np.int64,
     "r_max_wait": np.int64, "r_n_straggler": np.int64,
+    "incl_n_kernels": np.int32, "incl_first_start": np.int64, "incl_last_end": np.int64,
+    "incl_kernel_ns": np.int64, "replay_first_start": np.int64, "replay_last_end": np.int64,
+    "replay_kernel_ns": np.int64, "roll_sum": np.int64,
     "b_class": np.int32, "b_launch": np.int32, "b_win_count": np.int64, "b_win_ns": np.int64,
     "op_gap_ns": np.int64,
     "d_window": np.int32, "d_pid": np.int32, "d_n_events": np.int64, "d_busy": np.int64,
@@ -93,6 +96,8 @@ def _load():
         lib.orc_device_overlap.restype = None
         lib.orc_blame.argtypes = [ctypes.c_void_p]
         lib.orc_blame.restype = None
+        lib.orc_rollup.argtypes = [ctypes.c_void_p]
+        lib.orc_rollup.restype = None
         lib.orc_n_valid.argtypes = [ctypes.c_void_p]
         lib.orc_n_valid.restype = ctypes.c_int64
         lib.orc_get.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_void_p),
@@ -145,6 +150,8 @@ class Oracle:
             out = out.reshape(-1, 40)
         if name in ("b_win_count", "b_win_ns"):
             out = out.reshape(-1, 4)
+        if name == "roll_sum":
+            out = out.reshape(-1, 3)
         return out
 
     @property
@@ -178,6 +185,10 @@ class Oracle:
             arr[i] = (cid, nr, 0)
         self._sizes = arr
         self._lib.orc_collectives(self._h, arr.ctypes.data if len(arr) else None, len(arr))
+
+    def rollup(self):
+        """Inclusive per-operator kernel figures and graph replays (needs attribute() == 0)."""
+        self._lib.orc_rollup(self._h)
 
     def blame(self):
         """Classifies the long gaps of the last gaps() call and charges them to the operators

@@ -259,3 +259,39 @@ def blame(sv, wins, n_valid, lane_list, long_gaps, launch_of, t0, t1):
         if b > a:
             op_gap[p] = int(arr[a:b].sum())
     return cls, op_gap
+
+
+def rollup(sv, n_valid, parent, op_n, op_first, op_last, op_ns, launch_of, kol):
+    """Inclusive figures: every OP that owns kernels is added to itself and to each OP on its
+    parent chain.  Replays: the probes of every launch that owns two or more, collected in a
+    dict.  Returns (incl_n, incl_first, incl_last, incl_ns, replays{launch: (first, last, ns)})."""
+    n = len(sv)
+    acc = {}
+    for p in range(n_valid):
+        if int(sv[p]["kind"]) != 0 or int(op_n[p]) <= 0:
+            continue
+        q = p
+        hops = 0
+        while q >= 0:
+            a = acc.setdefault(q, [0, None, None, 0])
+            a[0] += int(op_n[p])
+            a[3] += int(op_ns[p])
+            a[1] = int(op_first[p]) if a[1] is None else min(a[1], int(op_first[p]))
+            a[2] = int(op_last[p]) if a[2] is None else max(a[2], int(op_last[p]))
+            q = int(parent[q])
+            hops += 1
+            assert hops < 1000
+    incl = [np.zeros(n, dtype=np.int64) for _ in range(4)]
+    for q, a in acc.items():
+        incl[0][q], incl[1][q], incl[2][q], incl[3][q] = a[0], a[1], a[2], a[3]
+    replays = {}
+    for p in range(n_valid):
+        if int(sv[p]["kind"]) not in (3, 4):
+            continue
+        l = int(launch_of[p])
+        if l < 0 or int(kol[l]) < 2:
+            continue
+        s, e = int(sv[p]["ts_start"]), int(sv[p]["ts_end"])
+        r = replays.setdefault(l, [s, e, 0])
+        r[0], r[1], r[2] = min(r[0], s), max(r[1], e), r[2] + (e - s)
+    return incl[0], incl[1], incl[2], incl[3], replays

@@ -146,4 +146,17 @@ def check_H7(run):
     assert int(r["op_gap_ns"].sum()) == sum(c[2] for c in charged)
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7]
+def check_H8(run):
+    g = load_golden("H8_rollup.txt")
+    r = run(g["events"], [0, len(g["events"])], [g["t0"]], [g["t1"]])
+    e = g["expect"]
+    assert r["attr_status"] == 0
+    for key, name in (("incl_n_kernels", "incl_n"), ("incl_kernel_ns", "incl_ns"),
+                      ("incl_first_start", "incl_first"), ("incl_last_end", "incl_last"),
+                      ("replay_first_start", "replay_first"), ("replay_last_end", "replay_last"),
+                      ("replay_kernel_ns", "replay_ns")):
+        assert r[key].tolist() == ints(e[name]), key
+    assert r["roll_sum"][0].tolist() == ints(e["roll_sum"])
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8]

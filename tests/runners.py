@@ -14,6 +14,8 @@ COLL_KEYS = ["c_window", "c_comm", "c_seq", "c_n_members", "c_min_start", "c_max
              "c_max_end", "c_straggler_pid", "c_flags", "wait_ns", "r_window", "r_pid", "r_n_coll",
              "r_sum_wait", "r_max_wait", "r_n_straggler"]
 
+ROLLUP_KEYS = ["incl_n_kernels", "incl_first_start", "incl_last_end", "incl_kernel_ns",
+               "replay_first_start", "replay_last_end", "replay_kernel_ns", "roll_sum"]
 BLAME_KEYS = ["b_class", "b_launch", "b_win_count", "b_win_ns", "op_gap_ns"]
 OVERLAP_KEYS = ["d_window", "d_pid", "d_n_events", "d_busy", "d_idle", "d_compute", "d_comm",
                 "d_overlap", "d_exposed"]
@@ -50,6 +52,10 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
     o.collectives(comm_sizes)
     for k in COLL_KEYS:
         r[k] = o.get(k)
+    if r["attr_status"] == 0:
+        o.rollup()
+        for k in ROLLUP_KEYS:
+            r[k] = o.get(k)
     o.blame()
     for k in BLAME_KEYS:
         r[k] = o.get(k)
@@ -100,6 +106,10 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
         c = w.match_collectives(comm_sizes)
         for k in COLL_KEYS:
             r[k] = c.numpy(k)
+        if a.status == 0:
+            ru = w.rollup_operators()
+            for k in ROLLUP_KEYS:
+                r[k] = ru.numpy(k)
         b = w.blame_gaps(g)
         for k in BLAME_KEYS:
             r[k] = b.numpy(k)

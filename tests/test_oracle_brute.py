@@ -303,3 +303,32 @@ def test_gap_blame_against_ticks(seed):
         assert (int(r["aggG_g_window"][i]), int(r["aggG_g_pid"][i]), int(r["aggG_g_name"][i])) == key
         assert int(r["aggG_g_count"][i]) == row["count"] and int(r["aggG_g_sum"][i]) == row["sum"]
         assert int(r["aggG_g_min"][i]) == row["min"] and int(r["aggG_g_max"][i]) == row["max"]
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_rollup_against_parent_chains(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    r = run_oracle(ev, off, t0, t1, min_gap=5, comm_sizes=sizes)
+    if r["attr_status"] != 0:
+        pytest.skip("window with a nesting error: no roll-up")
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    n, first, last, ns, replays = brute.rollup(sv, r["n_valid"], r["parent"], r["op_n_kernels"],
+                                               r["op_first_start"], r["op_last_end"], r["op_kernel_ns"],
+                                               r["launch_of"], r["kernels_of_launch"])
+    assert np.array_equal(r["incl_n_kernels"], n) and np.array_equal(r["incl_kernel_ns"], ns)
+    assert np.array_equal(r["incl_first_start"], first) and np.array_equal(r["incl_last_end"], last)
+    want = np.zeros((3, len(sv)), dtype=np.int64)
+    for l, (a, b, c) in replays.items():
+        want[:, l] = (a, b, c)
+    assert np.array_equal(r["replay_first_start"], want[0]) and np.array_equal(r["replay_last_end"], want[1])
+    assert np.array_equal(r["replay_kernel_ns"], want[2])
+    summ = np.zeros((len(t0), 3), dtype=np.int64)
+    for l in replays:
+        w = wins[l]
+        k = int(r["kernels_of_launch"][l])
+        summ[w] = (summ[w][0] + 1, summ[w][1] + k, max(summ[w][2], k))
+    assert np.array_equal(r["roll_sum"], summ)
+    # roots of the forest hold everything that was attributed below them
+    roots = (sv["kind"][:r["n_valid"]] == 0) & (r["parent"][:r["n_valid"]] < 0)
+    assert int(r["incl_n_kernels"][:r["n_valid"]][roots].sum()) == int(r["attr_sum"]["n_attributed"].sum())

@@ -73,6 +73,19 @@ def check_against_truth(wl, r):
     assert np.array_equal(r["agg0_g_hist"].sum(axis=1), r["agg0_g_count"])
     assert (r["agg0_g_min"] <= r["agg0_g_max"]).all()
     assert int(r["aggT_g_count"].sum()) == int((r["op_n_kernels"] > 0).sum())
+    # inclusive figures: the roots hold every attributed kernel; a subtree covers its own kernels
+    if r["attr_status"] == 0:
+        nv = r["n_valid"]
+        roots = (r["kind"][:nv] == 0) & (r["parent"][:nv] < 0)
+        assert int(r["incl_n_kernels"][:nv][roots].sum()) == int(r["attr_sum"]["n_attributed"].sum())
+        assert int(r["incl_kernel_ns"][:nv][roots].sum()) == int(r["op_kernel_ns"].sum())
+        own = r["op_n_kernels"] > 0
+        assert (r["incl_n_kernels"] >= r["op_n_kernels"]).all()
+        assert (r["incl_first_start"][own] <= r["op_first_start"][own]).all()
+        assert (r["incl_last_end"][own] >= r["op_last_end"][own]).all()
+        many = r["kernels_of_launch"] >= 2
+        assert int(many.sum()) == int(r["roll_sum"][:, 0].sum())
+        assert int(r["kernels_of_launch"][many].sum()) == int(r["roll_sum"][:, 1].sum())
     # device-level coverage: set identities, and bounds from the per-stream figures
     span = (np.asarray(wl.win_t1) - np.asarray(wl.win_t0))[r["d_window"]]
     assert np.array_equal(r["d_busy"] + r["d_idle"], span)
