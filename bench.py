@@ -146,6 +146,8 @@ def run_pipeline(ta, buf, wl, read_back=False, per_call=None):
             w.blame_gaps(g)
             w.aggregate_ops(1 << ta.KIND_OP, 2)
             mark("blame_gaps + aggregate_ops(OP, idle charged) (outside the timed step)")
+            w.rollup_operators()
+            mark("rollup_operators (outside the timed step)")
         nbytes = w.load_summary.nbytes + j.join_sum.nbytes + a.attr_sum.nbytes
         if read_back:
             for res, names in ((g, ("lane_gaps", "win_hist", "long_gaps")),

@@ -367,6 +367,43 @@ typedef struct ta_overlap_result {
 ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out);
 
 /* ------------------------------------------------------------------------
+ * ta_rollup_operators - inclusive per-operator kernel figures and graph
+ * replays.  An invocation's kernel composition comes from the call-to-kernel
+ * links and T_op spans the first kernel start to the last completion; CUDA
+ * Graph replay hides the operator calls and launch correlations separate the
+ * replays (Sec. 6.1, "Operator execution and efficiency").  Beyond the seven
+ * calls above.  Needs ta_attribute_operators to have returned TA_OK.
+ *
+ * Readings.  For an OP at sorted position r, over r itself and every OP below it
+ * in the forest `parent` defines:
+ *   incl_n_kernels[r] = sum of op_n_kernels, incl_kernel_ns[r] = sum of op_kernel_ns,
+ *   incl_first_start[r] = min of op_first_start, incl_last_end[r] = max of
+ *   op_last_end over those of them that own kernels; all four 0 when none does.
+ * For a LAUNCH at position l with kernels_of_launch[l] >= 2 (one graph replay):
+ *   replay_first_start[l] / replay_last_end[l] = min ts_start / max ts_end
+ *   (unclipped) of the device records with launch_of == l, replay_kernel_ns[l] =
+ *   sum of their durations; 0 for every other position.
+ * out_summary[w]: number of such launches in window w, the device records they
+ * own, and the most owned by one launch.
+ * MFU, MBU and SOL_op of the same section need per-invocation operation counts
+ * and device peaks that a 40-byte record does not carry; they are not computed.
+ * All arrays are device memory owned by the handle, n entries each.
+ * Errors: TA_ERR_ORDER unless ta_attribute_operators returned TA_OK;
+ * TA_ERR_OOM; TA_ERR_CUDA.  One stream synchronisation at the end. */
+typedef struct ta_rollup_summary {
+  int64_t n_graph_launches, n_graph_kernels, max_kernels_per_launch;
+} ta_rollup_summary;
+
+typedef struct ta_rollup_result {
+  const int32_t *incl_n_kernels;
+  const int64_t *incl_first_start, *incl_last_end, *incl_kernel_ns;
+  const int64_t *replay_first_start, *replay_last_end, *replay_kernel_ns;
+} ta_rollup_result;
+
+ta_status ta_rollup_operators(ta_window *h, ta_rollup_result *out,
+                              ta_rollup_summary *out_summary /* host, n_windows entries */);
+
+/* ------------------------------------------------------------------------
  * ta_blame_gaps - why a device stream sat idle, and which host calls the idle
  * time coincides with.  For waits, readiness, dispatch and first use are
  * compared: ready work dispatched late implicates submission (Sec. 6.2, engine

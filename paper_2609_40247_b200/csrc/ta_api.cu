@@ -312,6 +312,16 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes, int32_t 
   return ta_run_collectives(h, sizes, n_comms, out);
 }
 
+ta_status ta_rollup_operators(ta_window *h, ta_rollup_result *out, ta_rollup_summary *out_summary) {
+  if (!h || !out || !out_summary) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 8) || h->attr_status != 0) return TA_ERR_ORDER;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
+  return ta_run_rollup(h, out, out_summary);
+}
+
 ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
                         ta_blame_summary *out_summary) {
   if (!h || !gaps || !out || !out_summary) return TA_ERR_INVALID_ARG;

@@ -162,6 +162,8 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
 
 // overlap.cu
 ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out);
+// rollup.cu
+ta_status ta_run_rollup(ta_window *h, ta_rollup_result *out, ta_rollup_summary *out_summary);
 // blame.cu
 ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
                        ta_blame_summary *out_summary);

@@ -81,6 +81,9 @@ _CollResult = _ptr_struct("_CollResult", [
     ("g_skew", _vp), ("g_max_end", _vp), ("g_straggler_pid", _vp), ("g_flags", _vp),
     ("wait_ns", _vp), ("r_window", _vp), ("r_pid", _vp), ("r_n_coll", _vp), ("r_sum_wait", _vp),
     ("r_max_wait", _vp), ("r_n_straggler", _vp)])
+_RollupResult = _ptr_struct("_RollupResult", [
+    ("incl_n_kernels", _vp), ("incl_first_start", _vp), ("incl_last_end", _vp), ("incl_kernel_ns", _vp),
+    ("replay_first_start", _vp), ("replay_last_end", _vp), ("replay_kernel_ns", _vp)])
 _BlameResult = _ptr_struct("_BlameResult", [
     ("n_long_gaps", ctypes.c_int64), ("g_class", _vp), ("g_launch", _vp), ("op_gap_ns", _vp)])
 _OverlapResult = _ptr_struct("_OverlapResult", [
@@ -91,7 +94,8 @@ _OverlapResult = _ptr_struct("_OverlapResult", [
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
-           "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps"]
+           "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps",
+           "ta_rollup_operators"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -128,6 +132,8 @@ def lib():
         L.ta_aggregate_ops.argtypes = [_vp, ctypes.c_uint32, ctypes.c_int32, ctypes.POINTER(_AggResult)]
         L.ta_match_collectives.restype = ctypes.c_int
         L.ta_match_collectives.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(_CollResult)]
+        L.ta_rollup_operators.restype = ctypes.c_int
+        L.ta_rollup_operators.argtypes = [_vp, ctypes.POINTER(_RollupResult), _vp]
         L.ta_blame_gaps.restype = ctypes.c_int
         L.ta_blame_gaps.argtypes = [_vp, _vp, ctypes.POINTER(_BlameResult), _vp]
         L.ta_device_overlap.restype = ctypes.c_int
@@ -315,6 +321,24 @@ class CollResult(_Result):
         return super().tensor(self._names.get(name, name))
 
 
+ROLLUP_SUM = np.dtype([(k, "<i8") for k in ("n_graph_launches", "n_graph_kernels",
+                                            "max_kernels_per_launch")])
+
+
+class RollupResult(_Result):
+    _layout = dict([("incl_n_kernels", ("<i4", lambda r: r.n))] +
+                   [(k, ("<i8", lambda r: r.n)) for k in
+                    ("incl_first_start", "incl_last_end", "incl_kernel_ns", "replay_first_start",
+                     "replay_last_end", "replay_kernel_ns")])
+
+    def numpy(self, name):
+        if name == "roll_sum":
+            s = self.rollup_sum
+            return np.stack([s["n_graph_launches"], s["n_graph_kernels"], s["max_kernels_per_launch"]],
+                            axis=1).astype(np.int64)
+        return super().numpy(name)
+
+
 BLAME_SUM = np.dtype([("count", "<i8", (4,)), ("ns", "<i8", (4,))])
 
 
@@ -468,6 +492,14 @@ class Window:
         if st != 0:
             raise TaError(st, "ta_aggregate_ops")
         return AggResult(self, raw, dict(self._dims(), n_groups=raw.n_groups))
+
+    def rollup_operators(self) -> RollupResult:
+        raw = _RollupResult()
+        summ = np.zeros(self.W, dtype=ROLLUP_SUM)
+        st = self._lib.ta_rollup_operators(self._h, ctypes.byref(raw), summ.ctypes.data)
+        if st != 0:
+            raise TaError(st, "ta_rollup_operators")
+        return RollupResult(self, raw, dict(self._dims(), rollup_sum=summ))
 
     def blame_gaps(self, gaps) -> BlameResult:
         """gaps: the GapResult of an earlier stream_gaps() call on this window."""

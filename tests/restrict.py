@@ -13,7 +13,7 @@ import numpy as np
 
 from paper_2609_40247_b200.ta import NBINS
 from runners import (AGG_KEYS, ATTR_KEYS, BLAME_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS,
-                     OP_MASK, OVERLAP_KEYS)
+                     OP_MASK, OVERLAP_KEYS, ROLLUP_KEYS)
 
 _POSITIONAL = {"launch_of", "parent", "op_of"}  # values are sorted positions (or -1)
 _PER_RECORD_SORT = ["ts_start", "ts_end", "corr_id", "pid", "name_id", "seq", "stream", "kind"]
@@ -67,6 +67,7 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
         ag_op = w.aggregate_ops(OP_MASK, 1) if a.status == 0 else None
         c = w.match_collectives(comm_sizes)
         ov = w.device_overlap()
+        ru = w.rollup_operators() if a.status == 0 else None
         bl = w.blame_gaps(g)
         ag_gap = w.aggregate_ops(OP_MASK, 2)
         del buf
@@ -150,6 +151,11 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
                     r["long_gaps"] = cols.contiguous().cpu().numpy().reshape(-1).view(dt).copy()
                 else:
                     r["long_gaps"] = np.empty(0, dtype=dt)
+            if "rollup" in sub.groups and ru is not None:
+                for k in ROLLUP_KEYS[:-1]:
+                    r[k] = per_record(ru, k)
+                if sub.windows is not None:
+                    r["roll_sum"] = ru.numpy("roll_sum")[wkeep]
             if "blame" in sub.groups:
                 r["op_gap_ns"] = per_record(bl, "op_gap_ns")
                 t, dt = _typed(g, "long_gaps")

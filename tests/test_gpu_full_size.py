@@ -90,7 +90,7 @@ def test_c3_full_size_one_process_and_collectives():
     ev = wl.events
     assert len(ev) > 2**25
     pids = np.unique(ev["pid"])
-    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap", "blame")
+    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap", "blame", "rollup")
     subsets = [Subset(f"pid{p}", ev["pid"] == p, per_pid, pid=int(p)) for p in (pids[0], pids[-1])]
     subsets.append(Subset("coll", ev["kind"] == 5, ("sort", "coll")))
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
@@ -109,7 +109,7 @@ def test_c4_full_size_whole_windows():
     sel = np.zeros(len(ev), dtype=bool)
     for w in keep:
         sel[off[w]:off[w + 1]] = True
-    every = ("sort", "join", "attr", "gaps", "agg", "coll", "overlap", "blame")
+    every = ("sort", "join", "attr", "gaps", "agg", "coll", "overlap", "blame", "rollup")
     subsets = [Subset("windows", sel, every, windows=keep)]
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
                            comm_sizes=wl.comm_sizes,
