@@ -106,12 +106,28 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
 // One CTA: sorts the discovered triples, ranks them and the pids they contain.
 __global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t *status) {
   extern __shared__ u64 buf[];  // TA_TRIPLE_SLOTS
+  __shared__ u64 tmp[33];
+  __shared__ int n_tr;
   const int tid = threadIdx.x;
-  for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x) buf[i] = tt->slots[i];
+  // the occupied slots, packed to the front (a window has tens of triples, not thousands)
+  if (tid == 0) n_tr = 0;
   __syncthreads();
-  for (int k = 2; k <= TA_TRIPLE_SLOTS; k <<= 1)
+  for (int c0 = 0; c0 < TA_TRIPLE_SLOTS; c0 += blockDim.x) {
+    const u64 v = tt->slots[c0 + tid];
+    u64 total;
+    const u64 ex = block_scan_exclusive<OpAdd>(v != TRIPLE_EMPTY ? 1ull : 0ull, OpAdd(), tmp, &total);
+    if (v != TRIPLE_EMPTY) buf[n_tr + (int)ex] = v;
+    __syncthreads();
+    if (tid == 0) n_tr += (int)total;
+    __syncthreads();
+  }
+  int padded = 32;
+  while (padded < n_tr) padded <<= 1;
+  for (int i = n_tr + tid; i < padded; i += blockDim.x) buf[i] = TRIPLE_EMPTY;  // sorts last
+  __syncthreads();
+  for (int k = 2; k <= padded; k <<= 1)
     for (int j = k >> 1; j > 0; j >>= 1) {
-      for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x) {
+      for (int i = tid; i < padded; i += blockDim.x) {
         int ixj = i ^ j;
         if (ixj > i) {
           u64 a = buf[i], b = buf[ixj];
@@ -121,12 +137,6 @@ __global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t 
       }
       __syncthreads();
     }
-  __shared__ int n_tr;
-  if (tid == 0) n_tr = 0;
-  __syncthreads();
-  for (int i = tid; i < TA_TRIPLE_SLOTS; i += blockDim.x)
-    if (buf[i] != TRIPLE_EMPTY && (i + 1 == TA_TRIPLE_SLOTS || buf[i + 1] == TRIPLE_EMPTY)) n_tr = i + 1;
-  __syncthreads();
   int n = n_tr;
   if (n > TA_MAX_TRIPLES) {
     if (tid == 0) ta_set_err(status, TA_ERR_TOO_LARGE);
