@@ -710,14 +710,38 @@ __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
   if (p0 >= a.n_valid) return;
   int16_t kd[8];
   load8_i16(a.kind, p0, a.n, 9, kd);
+  unsigned ops = 0;
 #pragma unroll
-  for (int j = 0; j < 8; j++) {
-    const int64_t p = p0 + j;
-    if (p < a.n_valid && kd[j] == TA_KIND_OP && a.op_n[p] > 0) {
-      a.op_first[p] = (~a.op_first[p]) ^ (1ull << 63);
-      a.op_last[p] = a.op_last[p] ^ (1ull << 63);
-    }
+  for (int j = 0; j < 8; j++)
+    if (p0 + j < a.n_valid && kd[j] == TA_KIND_OP) ops |= 1u << j;
+  if (!ops) return;
+  // counts of all eight positions in two vector loads, then both times of the operators that
+  // own kernels: the thread's misses overlap instead of following one another
+  int32_t cnt[8];
+  if (p0 + 8 <= a.n) {
+    const int4 x = *reinterpret_cast<const int4 *>(a.op_n + p0);
+    const int4 y = *reinterpret_cast<const int4 *>(a.op_n + p0 + 4);
+    cnt[0] = x.x; cnt[1] = x.y; cnt[2] = x.z; cnt[3] = x.w;
+    cnt[4] = y.x; cnt[5] = y.y; cnt[6] = y.z; cnt[7] = y.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++) cnt[j] = p0 + j < a.n ? a.op_n[p0 + j] : 0;
   }
+  unsigned m = 0;
+#pragma unroll
+  for (int j = 0; j < 8; j++)
+    if ((ops & (1u << j)) && cnt[j] > 0) m |= 1u << j;
+  if (!m) return;
+  u64 f[8], l[8];
+#pragma unroll
+  for (int j = 0; j < 8; j++)
+    if (m & (1u << j)) { f[j] = a.op_first[p0 + j]; l[j] = a.op_last[p0 + j]; }
+#pragma unroll
+  for (int j = 0; j < 8; j++)
+    if (m & (1u << j)) {
+      a.op_first[p0 + j] = (~f[j]) ^ (1ull << 63);
+      a.op_last[p0 + j] = l[j] ^ (1ull << 63);
+    }
 }
 
 ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
