@@ -309,7 +309,8 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   TA_CHECK_CUDA(h, cudaGetLastError());
   if (idxbits) {
     TA_TRY(ta_radix_sort_keys(h, k_in, k_scr, k_fin, m,
-                              ta_make_plan(idxbits, idxbits + tsbits + slot_bits), nullptr, sort_tmp));
+                              ta_make_plan(idxbits, idxbits + tsbits + slot_bits), nullptr, sort_tmp,
+                              true));  // coverage sums do not depend on the order of equal starts
     sa.pos = v_in;
   } else {
     TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, k_fin, v_fin, m,

@@ -45,7 +45,10 @@ struct RadixSmem {
   int fail;
 };
 
-template <int THREADS, int ITEMS, bool VALS, int BITS, bool FULL>
+// STABLE = false: equal digits may leave the pass in any order (one shared-memory atomic per
+// key instead of the vote ranking).  Only legal for the FIRST pass of a sort whose caller
+// does not rely on the input order of keys that are equal in all sorted bits.
+template <int THREADS, int ITEMS, bool VALS, int BITS, bool FULL, bool STABLE>
 __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS, ITEMS> &s, int tile,
                                            int count) {
   constexpr int TILE = THREADS * ITEMS;
@@ -69,6 +72,11 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   for (int j = 0; j < ITEMS; j++) {
     const bool valid = FULL || (wbase + j * 32 + lane) < count;
     const u32 d = (u32)(key[j] >> a.shift) & MASK;
+    if (!STABLE) {
+      const u32 old = valid ? atomicAdd(&wh[d], 1u) : 0u;
+      rd[j] = (int)((old << 8) | d);
+      continue;
+    }
     // lanes with the same digit: one vote per digit bit
     u32 m = FULL ? 0xffffffffu : __ballot_sync(0xffffffffu, valid);
     if (!FULL && !valid) m = ~m;
@@ -173,7 +181,7 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   }
 }
 
-template <int THREADS, int ITEMS, bool VALS, int BITS>
+template <int THREADS, int ITEMS, bool VALS, int BITS, bool STABLE>
 __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_pass(RadixArgs a) {
   constexpr int TILE = THREADS * ITEMS;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -187,8 +195,8 @@ __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_p
   __syncthreads();
   const int tile = s.tile;
   const int count = (int)min((int64_t)TILE, a.n - (int64_t)tile * TILE);
-  if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true>(a, s, tile, count);
-  else radix_tile<THREADS, ITEMS, VALS, BITS, false>(a, s, tile, count);
+  if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true, STABLE>(a, s, tile, count);
+  else radix_tile<THREADS, ITEMS, VALS, BITS, false, STABLE>(a, s, tile, count);
 }
 
 // tile shapes
@@ -254,12 +262,12 @@ size_t ta_sort_temp_bytes(int64_t n) {
          2 * Carver::pad(10 * RS_BINS * sizeof(u32));
 }
 
-template <int THREADS, int ITEMS, bool VALS>
+template <int THREADS, int ITEMS, bool VALS, bool STABLE>
 static cudaError_t launch_pass(const RadixArgs &a, int bits, unsigned tiles, cudaStream_t st) {
   typedef RadixSmem<THREADS, ITEMS> Smem;
 #define RS_CASE(B)                                                                                  \
   case B: {                                                                                         \
-    auto kern = k_radix_pass<THREADS, ITEMS, VALS, B>;                                              \
+    auto kern = k_radix_pass<THREADS, ITEMS, VALS, B, STABLE>;                                      \
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
                                          (int)sizeof(Smem));                                        \
     if (e != cudaSuccess) return e;                                                                 \
@@ -281,7 +289,8 @@ static cudaError_t launch_pass(const RadixArgs &a, int bits, unsigned tiles, cud
 template <bool VALS>
 static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in, u64 *keys_scratch,
                             u32 *vals_scratch, u64 *keys_final, u32 *vals_final, int64_t n,
-                            const SortPlan &plan, const u32 *hist, void *temp) {
+                            const SortPlan &plan, const u32 *hist, void *temp,
+                            bool first_pass_unstable) {
   if (n <= 0) return TA_OK;
   constexpr int THREADS = VALS ? RSP_THREADS : RSK_THREADS;
   constexpr int ITEMS = VALS ? RSP_ITEMS : RSK_ITEMS;
@@ -316,7 +325,10 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
     if (timed) ta_profile_mark(st, 1, (VALS ? 24.0 : 16.0) * (double)n);
-    TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, VALS>(a, plan.bits[p], (unsigned)tiles, st)));
+    if (!VALS && p == 0 && first_pass_unstable)
+      TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, false, false>(a, plan.bits[p], (unsigned)tiles, st)));
+    else
+      TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, VALS, true>(a, plan.bits[p], (unsigned)tiles, st)));
     if (timed) ta_profile_mark(st, 0, 0.0);
     kin = a.keys_out;
     vin = a.vals_out;
@@ -330,11 +342,12 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
                               u32 *vals_final, int64_t n, const SortPlan &plan, const u32 *hist,
                               void *temp) {
   return radix_sort<true>(h, keys_in, vals_in, keys_scratch, vals_scratch, keys_final, vals_final, n,
-                          plan, hist, temp);
+                          plan, hist, temp, false);
 }
 
 ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
-                             int64_t n, const SortPlan &plan, const u32 *hist, void *temp) {
+                             int64_t n, const SortPlan &plan, const u32 *hist, void *temp,
+                             bool first_pass_unstable) {
   return radix_sort<false>(h, keys_in, nullptr, keys_scratch, nullptr, keys_final, nullptr, n, plan,
-                           hist, temp);
+                           hist, temp, first_pass_unstable);
 }

@@ -140,7 +140,8 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
                               const u32 *hist /*nullable*/, void *temp);
 ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
                              int64_t n, const SortPlan &plan, const u32 *hist /*nullable*/,
-                             void *temp);
+                             void *temp,
+                             bool first_pass_unstable);
 SortPlan ta_make_plan(int lo_bit, int hi_bit);
 // load.cu
 ta_status ta_launch_discover(ta_window *h);

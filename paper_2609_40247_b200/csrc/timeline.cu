@@ -117,7 +117,8 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
     const u64 k = a.keys[p];
     idx = gather_index(k, a);
     // packed keys order the records down to a coarse time only: members of a run of equal
-    // (lane, coarse time) sit in input order and are ranked here by (ts_start, -ts_end)
+    // (lane, coarse time) sit in no particular order (the first radix pass is not stable) and
+    // are ranked here by (ts_start, -ts_end, input index)
     const u64 hk = k >> a.ibits;
     while (before <= TA_TIE_RUN_MAX && p - before > 0 && (a.keys[p - before - 1] >> a.ibits) == hk)
       before++;
@@ -136,9 +137,10 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
     int rank = 0;
     for (int q = -before; q <= after; q++) {
       if (q == 0) continue;
-      const i64 *o = reinterpret_cast<const i64 *>(a.ev) + (int64_t)gather_index(a.keys[p + q], a) * 5;
+      const u32 oi = gather_index(a.keys[p + q], a);
+      const i64 *o = reinterpret_cast<const i64 *>(a.ev) + (int64_t)oi * 5;
       const i64 os = o[0], oe = o[1];
-      const bool first = os < r.ts_start || (os == r.ts_start && (oe > r.ts_end || (oe == r.ts_end && q < 0)));
+      const bool first = os < r.ts_start || (os == r.ts_start && (oe > r.ts_end || (oe == r.ts_end && oi < idx)));
       rank += first ? 1 : 0;
     }
     dst = p - before + rank;
@@ -345,7 +347,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
       if (h->packed) {
         // keys carry the index: 8-byte elements, fewer bytes per pass
         PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
-        TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp));
+        TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp, true));
         if (n > h->n_valid)
           k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm);
       }
@@ -393,10 +395,12 @@ ta_status ta_run_sort_timeline(ta_window *h) {
         u64 *tk = cx.take<u64>(m), *tk2 = cx.take<u64>(m);
         u32 *alt = cx.take<u32>(m);
         u32 *cur = perm + h->n_valid, *nxt = alt;
-        for (int stage = 0; stage < 4; stage++) {
+        // packed keys: the first radix pass does not keep equal keys in input order, and all
+        // dropped records of a window share one key, so the tail is put in input order first
+        for (int stage = h->packed ? -1 : 0; stage < 4; stage++) {
           if (stage == 3 && h->W == 1) break;
           k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
-          int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : 64;
+          int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : stage < 0 ? 32 : 64;
           SortPlan tp = ta_make_plan(0, bits);
           TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
           u32 *t = cur; cur = nxt; nxt = t;
