@@ -46,3 +46,34 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
         assert "no CPU fallback" in str(e)
     else:
         raise AssertionError("loading a missing library must raise")
+
+
+def test_arguments_are_rejected_before_any_device_work():
+    """Argument checks of ta_load_window come before the first CUDA call, so they can be
+    exercised here: a record count of 2^31, a window of 2^40 ns, offsets that do not end at n,
+    a null handle pointer."""
+    import numpy as np
+    from paper_2609_40247_b200 import ta
+    L = ta.lib()
+    env = ta._Env()
+    env.device = 0
+    handle = ctypes.c_void_p()
+    ev = np.zeros(4, dtype=ta.EVENT_DTYPE)
+    summ = np.zeros(1, dtype=ta.LOAD_SUM)
+
+    def load(n, off, t0, t1, hp=ctypes.byref(handle)):
+        off = np.asarray(off, dtype=np.int64)
+        t0 = np.asarray(t0, dtype=np.int64)
+        t1 = np.asarray(t1, dtype=np.int64)
+        return L.ta_load_window(ctypes.byref(env), ev.ctypes.data, n, 0, off.ctypes.data, t0.ctypes.data,
+                                t1.ctypes.data, 1, summ.ctypes.data, hp)
+
+    assert load(2**31, [0, 2**31], [0], [1000]) == 5          # TA_ERR_TOO_LARGE
+    assert load(4, [0, 4], [0], [2**40]) == 5                 # window of 2^40 ns
+    assert load(4, [0, 3], [0], [1000]) == 1                  # TA_ERR_INVALID_ARG: offsets end before n
+    assert load(4, [0, 4], [10], [10]) == 1                   # empty window
+    assert load(-1, [0, 0], [0], [10]) == 1
+    assert load(4, [0, 4], [0], [1000], hp=None) == 1
+    assert not handle.value
+    L.ta_free(None)                                           # NULL-safe
+    assert L.ta_strerror(5) and L.ta_version() > 0
