@@ -14,7 +14,7 @@
 #include "ta_internal.cuh"
 
 #define RS_BINS 256
-// resident CTAs per SM the register budget is sized for (pairs, keys only)
+// resident CTAs per SM the register allocation is sized for (pairs, keys only)
 #ifndef RSP_MINB
 #define RSP_MINB 2
 #endif
