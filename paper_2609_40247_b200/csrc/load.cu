@@ -20,13 +20,17 @@ __device__ __forceinline__ i64 warp_max_i64(i64 v) {
 }
 
 // Pass 1 over the records: defect counters, the set of lane triples, the range
-// of name ids and the longest duration.
+// of name ids and the longest duration.  It also leaves one 64-bit word per record with
+// all the key pass needs - bit 63 for a dropped record, else the triple's slot in the hash
+// table (13 bits) and ts_start - t0 (40 bits) - so that the 40-byte records are read once.
+#define PRE_DROPPED (1ull << 63)
+#define PRE_TS_BITS 40
 __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n, const int64_t *off,
                                                   const int64_t *t0, const int64_t *t1, int W,
                                                   TripleTable *tt, CommTable *cm,
                                                   ta_load_summary *sum, int64_t *misc,
-                                                  int32_t *status) {
-  __shared__ u64 cache[256];
+                                                  int32_t *status, u64 *prekey) {
+  __shared__ u64 cache[256];  // (triple code << 13) | slot: one word, so a racing reader sees a pair
   __shared__ u64 ccache[64];
   cache[threadIdx.x] = TRIPLE_EMPTY;
   if (threadIdx.x < 64) ccache[threadIdx.x] = TRIPLE_EMPTY;
@@ -41,6 +45,7 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
       int64_t *f = def == 1 ? &sum[w].n_bad_kind
                             : def == 2 ? &sum[w].n_bad_interval : &sum[w].n_out_of_window;
       atomicAdd((u64 *)f, 1ull);
+      prekey[i] = PRE_DROPPED;
       continue;
     }
     mn = min(mn, (i64)r.name);
@@ -70,7 +75,12 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
     }
     u64 code = triple_code(r.pid, r.kind, r.stream);
     u32 hsh = hash_code(code);
-    if (cache[hsh & 255] == code) continue;  // a stale miss only costs a probe
+    const u64 ts_rel = (u64)(r.ts_start - t0[w]);
+    const u64 hit = cache[hsh & 255];
+    if ((hit >> 13) == code) {  // a stale miss only costs a probe
+      prekey[i] = ((hit & (TA_TRIPLE_SLOTS - 1)) << PRE_TS_BITS) | ts_rel;
+      continue;
+    }
     u32 slot = hsh & (TA_TRIPLE_SLOTS - 1);
     bool done = false;
     for (int probe = 0; probe < TA_TRIPLE_SLOTS; probe++) {
@@ -83,7 +93,8 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
       slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
     }
     if (!done) ta_set_err(status, TA_ERR_TOO_LARGE);
-    cache[hsh & 255] = code;
+    cache[hsh & 255] = (code << 13) | slot;
+    prekey[i] = ((u64)slot << PRE_TS_BITS) | ts_rel;
   }
   mn = warp_min_i64(mn);
   mx = warp_max_i64(mx);
@@ -277,6 +288,52 @@ __global__ void __launch_bounds__(256) k_load(LoadArgs a) {
     if (sh[i]) atomicAdd(&a.hist[i], sh[i]);
 }
 
+// The same from the words k_discover left in a.keys (rewritten in place): 8 B read + 8 B
+// written per record instead of another pass over the 40-byte records.
+__global__ void __launch_bounds__(256) k_load_pre(LoadArgs a) {
+  __shared__ u32 sh[10 * 256];
+  for (int i = threadIdx.x; i < a.plan.n_pass * 256; i += blockDim.x) sh[i] = 0;
+  __syncthreads();
+  const int tsb = a.sbits - a.dshift;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const int64_t n_round = ((a.n + 31) / 32) * 32;
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += stride) {
+    bool in = i < a.n;
+    u64 key = 0;
+    if (in) {
+      const u64 pk = a.keys[i];
+      int w = window_of(a.off, a.W, i);
+      u64 hi;
+      if (pk & PRE_DROPPED) {
+        hi = (1ull << (a.wbits + a.tbits + tsb)) | ((u64)w << (a.tbits + tsb));
+        if (!a.packed) hi = 1ull << (a.wbits + a.tbits + tsb);
+      } else {
+        const u32 slot = (u32)(pk >> PRE_TS_BITS) & (TA_TRIPLE_SLOTS - 1);
+        const u64 rank = (u64)__ldg(&a.tt->rank_of_slot[slot]);
+        hi = ((u64)w << (a.tbits + tsb)) | (rank << tsb) | ((pk & ((1ull << PRE_TS_BITS) - 1)) >> a.dshift);
+      }
+      key = a.packed ? (hi << a.ibits) | (u64)(i - a.off[w]) : hi;
+      a.keys[i] = key;
+    }
+    u32 active = __ballot_sync(0xffffffffu, in);
+    if (!in) continue;
+    const int lane = threadIdx.x & 31;
+    const int leader = __ffs(active) - 1;
+    for (int p = 0; p < a.plan.n_pass; p++) {
+      u32 d = (u32)(key >> a.plan.shift[p]) & ((1u << a.plan.bits[p]) - 1u);
+      u32 d0 = __shfl_sync(active, d, leader);
+      if (__all_sync(active, d == d0)) {
+        if (lane == leader) atomicAdd(&sh[p * 256 + d0], (u32)__popc(active));
+      } else {
+        atomicAdd(&sh[p * 256 + d], 1u);
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < a.plan.n_pass * 256; i += blockDim.x)
+    if (sh[i]) atomicAdd(&a.hist[i], sh[i]);
+}
+
 // ------------------------------------------------------------------ host
 static int bit_length(uint64_t v) {
   int b = 0;
@@ -294,7 +351,8 @@ ta_status ta_launch_discover(ta_window *h) {
   if (h->n > 0) {
     k_discover<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(
         h->events, h->n, h->d_off, h->d_t0, h->d_t1, h->W, h->d_triples, h->d_comms, h->d_load_sum,
-        h->d_misc, h->d_status);
+        h->d_misc, h->d_status, h->d_keys);
+    h->prekeys = 1;
   }
   k_rank_comms<<<TA_N 1, 1024, 0, h->stream>>>(h->d_comms, h->d_status);
   TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank_triples, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -352,7 +410,11 @@ ta_status ta_launch_load(ta_window *h, bool allow_packed) {
   a.tt = h->d_triples; a.keys = h->d_keys; a.hist = h->d_hist;
   a.sbits = h->sbits; a.tbits = h->tbits; a.wbits = h->wbits; a.plan = h->plan;
   a.packed = h->packed; a.dshift = h->dshift; a.ibits = h->ibits;
-  k_load<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
+  // the words of the discovery pass are there once; a later call (the fall back to full
+  // resolution keys) goes back to the records
+  if (h->prekeys) k_load_pre<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
+  else k_load<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);
+  h->prekeys = 0;
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }

@@ -247,6 +247,7 @@ ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
   h->events = nullptr;
   h->events_copy = nullptr;
   h->d_keys = nullptr;
+  h->prekeys = 0;
   h->attr_status = 0;
   h->d_op_gap_ns = nullptr;
   h->h_off.assign(win_off, win_off + W + 1);

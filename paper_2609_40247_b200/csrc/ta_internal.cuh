@@ -74,6 +74,7 @@ struct ta_window {
   int64_t min_seq, max_seq;
   ta_load_summary *d_load_sum;
   u64 *d_keys;
+  int prekeys;               // d_keys holds the words of the discovery pass, not keys yet
   u32 *d_hist;               // [pass][256]
   int64_t n_valid;
   int n_triples, n_pids;
