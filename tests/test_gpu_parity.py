@@ -122,8 +122,10 @@ def test_host_buffer_input_matches_device_input():
     assert_same(a, b)
 
 
+# c0 x 10: one process, one host thread, two streams - three lanes of 200 000 records each
+# (long look-back chains, a deep tree of tile stacks)
 CASES = [("c0", 1.0, 0), ("c0", 1.0, 1), ("c1", 0.1, 0), ("c1", 0.03, 1), ("c2", 0.02, 0),
-         ("c3", 0.01, 0), ("c4", 0.002, 0)]
+         ("c3", 0.01, 0), ("c4", 0.002, 0), ("c0", 10.0, 0)]
 
 
 @pytest.mark.parametrize("name,scale,shuffle", CASES)
