@@ -278,9 +278,10 @@ ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out);
  * output row per non-empty group in ascending signed key order with count,
  * sum, min, max and a histogram whose bin is min(39, floor(log2 v)) for
  * v >= 1 and 0 for v <= 0.
- * Limit: (#windows x #pids x (max name_id - min name_id + 1)) <= 2^27, else
- * TA_ERR_TOO_LARGE.  The result buffers of an earlier ta_aggregate_ops call on
- * the same handle stay valid.
+ * While (#windows x #pids x (max name_id - min name_id + 1)) <= 2^27 the rows are
+ * accumulated in a dense table; symbol ids spread wider than that are grouped
+ * by sorting instead (slower, same result).  The result buffers of an earlier
+ * ta_aggregate_ops call on the same handle stay valid.
  */
 typedef struct ta_agg_result {
   int64_t n_groups;

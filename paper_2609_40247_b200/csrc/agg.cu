@@ -249,6 +249,203 @@ struct AggRowOut {
   }
 };
 
+// ---- symbol ids too spread out for the dense table: aggregate by sorting ---------------
+// The selected records are compacted to (key, position) pairs with key = (window, pid) slot
+// << 32 | name_id (order-preserving code), sorted with the pair sorter, cut into groups where
+// the key changes, and reduced with atomics on the group rows - one per run of equal keys
+// inside a thread's eight consecutive elements, so a popular symbol costs an eighth of its
+// records in atomics.  Rows come out in key order, as from the dense path.
+struct AggSortCtx {
+  int64_t n_valid;
+  int n_lanes, n_pids;
+  uint32_t kind_mask;
+  int value_sel;
+  const int16_t *kind;
+  const int32_t *name;
+  const int64_t *ts, *te;
+  const int32_t *op_n;
+  const int64_t *op_first, *op_last, *op_gap;
+  const int32_t *lane_off, *lane_slot;
+  const TripleTable *tt;
+};
+__device__ __forceinline__ bool agg_selected(const AggSortCtx &c, int64_t p, i64 *v) {
+  const int k = c.kind[p];
+  if (k < 0 || k > 5 || !((c.kind_mask >> k) & 1u)) return false;
+  if (c.value_sel == 0) { *v = c.te[p] - c.ts[p]; return true; }
+  if (c.value_sel == 1) {
+    if (c.op_n[p] <= 0) return false;
+    *v = c.op_last[p] - c.op_first[p];
+    return true;
+  }
+  *v = c.op_gap[p];
+  return *v > 0;
+}
+struct AggSelIn {
+  AggSortCtx c;
+  __device__ u64 operator()(int64_t p) const {
+    i64 v;
+    return agg_selected(c, p, &v) ? 1ull : 0ull;
+  }
+};
+struct AggSelOut {
+  AggSortCtx c;
+  u64 *keys;
+  u32 *pos;
+  __device__ void operator()(int64_t p, u64 excl, u64 v) const {
+    if (!v) return;
+    const int lane = lane_of_pos(c.lane_off, c.n_lanes, p);
+    keys[excl] = ((u64)c.lane_slot[lane] << 32) | (u64)((u32)c.name[p] ^ 0x80000000u);
+    pos[excl] = (u32)p;
+  }
+};
+struct AggHeadIn {
+  const u64 *ks;
+  __device__ u64 operator()(int64_t j) const { return (j == 0 || ks[j] != ks[j - 1]) ? 1ull : 0ull; }
+};
+struct AggHeadOut {
+  int32_t *gid;     // per sorted element
+  int32_t *gstart;  // per group
+  __device__ void operator()(int64_t j, u64 excl, u64 v) const {
+    const int32_t g = (int32_t)(excl + v) - 1;
+    gid[j] = g;
+    if (v) gstart[g] = (int32_t)j;
+  }
+};
+struct AggSortedOut {
+  int32_t *g_window, *g_pid, *g_name;
+  int64_t *g_count, *g_sum, *g_min, *g_max;
+  u32 *g_hist;
+};
+__global__ void __launch_bounds__(256) k_agg_sorted_rows(AggSortCtx c, const u64 *ks, const int32_t *gstart,
+                                                        int64_t ng, AggSortedOut o) {
+  const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= ng) return;
+  const u64 key = ks[gstart[g]];
+  const int64_t slot = (int64_t)(key >> 32);
+  o.g_window[g] = (int32_t)(slot / c.n_pids);
+  o.g_pid[g] = c.tt->pid_value[slot % c.n_pids];
+  o.g_name[g] = (int32_t)((u32)key ^ 0x80000000u);
+  o.g_min[g] = INT64_MAX;
+  o.g_max[g] = INT64_MIN;
+}
+__global__ void __launch_bounds__(256) k_agg_sorted_reduce(AggSortCtx c, const u32 *pos, const int32_t *gid,
+                                                          int64_t m, AggSortedOut o) {
+  const int64_t j0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  if (j0 >= m) return;
+  int32_t cur = -1;
+  u64 cnt = 0, sum = 0;
+  i64 mn = INT64_MAX, mx = INT64_MIN;
+  for (int k = 0; k < 8 && j0 + k < m; k++) {
+    const int32_t g = gid[j0 + k];
+    i64 v = 0;
+    agg_selected(c, pos[j0 + k], &v);
+    if (g != cur) {
+      if (cur >= 0) {
+        atomicAdd((u64 *)&o.g_count[cur], cnt);
+        atomicAdd((u64 *)&o.g_sum[cur], sum);
+        atomicMin((i64 *)&o.g_min[cur], mn);
+        atomicMax((i64 *)&o.g_max[cur], mx);
+      }
+      cur = g; cnt = 0; sum = 0; mn = INT64_MAX; mx = INT64_MIN;
+    }
+    cnt++;
+    sum += (u64)v;
+    mn = v < mn ? v : mn;
+    mx = v > mx ? v : mx;
+    atomicAdd(&o.g_hist[(size_t)g * TA_NBINS + log2_bin(v)], 1u);
+  }
+  if (cur >= 0) {
+    atomicAdd((u64 *)&o.g_count[cur], cnt);
+    atomicAdd((u64 *)&o.g_sum[cur], sum);
+    atomicMin((i64 *)&o.g_min[cur], mn);
+    atomicMax((i64 *)&o.g_max[cur], mx);
+  }
+}
+
+static ta_status ta_run_aggregate_sorted(ta_window *h, uint32_t kind_mask, int value_sel,
+                                         ta_agg_result *out) {
+  cudaStream_t st = h->stream;
+  const int n_pids = h->n_pids > 0 ? h->n_pids : 1;
+  const int64_t nv = h->n_valid;
+  AggSortCtx c;
+  memset(&c, 0, sizeof(c));
+  c.n_valid = nv; c.n_lanes = h->sorted.n_lanes; c.n_pids = n_pids;
+  c.kind_mask = kind_mask & 63u; c.value_sel = value_sel;
+  c.kind = h->sorted.kind; c.name = h->sorted.name_id; c.ts = h->sorted.ts_start; c.te = h->sorted.ts_end;
+  c.op_n = h->attr.op_n_kernels; c.op_first = h->attr.op_first_start; c.op_last = h->attr.op_last_end;
+  c.op_gap = h->d_op_gap_ns; c.lane_off = h->sorted.lane_off; c.lane_slot = h->d_lane_slot;
+  c.tt = h->d_triples;
+
+  // 1. selection
+  size_t t1b = Carver::pad((size_t)nv * 8) + Carver::pad((size_t)nv * 4) + scan_temp_bytes(nv) + 256;
+  void *t1 = ta_dalloc(h, t1b);
+  if (!t1) return TA_ERR_OOM;
+  Carver c1(t1);
+  u64 *k_in = c1.take<u64>(nv);
+  u32 *v_in = c1.take<u32>(nv);
+  ScanTemp s1;
+  TA_TRY(scan_temp_init(h, c1.base + c1.off, nv, &s1));
+  AggSelIn si{c};
+  AggSelOut so{c, k_in, v_in};
+  TA_TRY((launch_scan<OpAdd, AggSelIn, AggSelOut>(h, nv, si, so, OpAdd(), s1)));
+  u64 m64 = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, s1.total, 8, cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  const int64_t m = (int64_t)m64;
+  if (m == 0) { ta_dfree(h, t1); return TA_OK; }
+
+  // 2. sort, 3. groups
+  int slot_bits = 1;
+  while (slot_bits < 31 && ((int64_t)h->W * n_pids - 1) >> slot_bits) slot_bits++;
+  size_t t2b = 2 * Carver::pad((size_t)m * 8) + 2 * Carver::pad((size_t)m * 4) + 2 * Carver::pad((size_t)(m + 1) * 4) +
+               ta_sort_temp_bytes(m) + scan_temp_bytes(m) + 256;
+  void *t2 = ta_dalloc(h, t2b);
+  if (!t2) return TA_ERR_OOM;
+  Carver c2(t2);
+  u64 *k_scr = c2.take<u64>(m), *ks = c2.take<u64>(m);
+  u32 *v_scr = c2.take<u32>(m), *vs = c2.take<u32>(m);
+  int32_t *gid = c2.take<int32_t>(m + 1), *gstart = c2.take<int32_t>(m + 1);
+  void *sort_tmp = c2.base + c2.off; c2.off += ta_sort_temp_bytes(m);
+  void *scan2 = c2.base + c2.off;
+  TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, ks, vs, m, ta_make_plan(0, 32 + slot_bits), nullptr,
+                             sort_tmp));
+  ScanTemp s2;
+  TA_TRY(scan_temp_init(h, scan2, m, &s2));
+  AggHeadIn hi{ks};
+  AggHeadOut ho{gid, gstart};
+  TA_TRY((launch_scan<OpAdd, AggHeadIn, AggHeadOut>(h, m, hi, ho, OpAdd(), s2)));
+  u64 ng64 = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng64, s2.total, 8, cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  const int64_t ng = (int64_t)ng64;
+
+  // 4. rows
+  size_t ob = 3 * Carver::pad((size_t)ng * 4) + 4 * Carver::pad((size_t)ng * 8) +
+              Carver::pad((size_t)ng * TA_NBINS * 4) + 256;
+  void *outb = ta_dalloc(h, ob);
+  if (!outb) return TA_ERR_OOM;
+  TA_CHECK_CUDA(h, cudaMemsetAsync(outb, 0, ob, st));
+  Carver co(outb);
+  AggSortedOut o;
+  o.g_window = co.take<int32_t>(ng); o.g_pid = co.take<int32_t>(ng); o.g_name = co.take<int32_t>(ng);
+  o.g_count = co.take<int64_t>(ng); o.g_sum = co.take<int64_t>(ng);
+  o.g_min = co.take<int64_t>(ng); o.g_max = co.take<int64_t>(ng);
+  o.g_hist = co.take<u32>((size_t)ng * TA_NBINS);
+  k_agg_sorted_rows<<<TA_N (unsigned)((ng + 255) / 256), 256, 0, st>>>(c, ks, gstart, ng, o);
+  k_agg_sorted_reduce<<<TA_N (unsigned)((m + 2047) / 2048), 256, 0, st>>>(c, vs, gid, m, o);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  int32_t words[ST_WORDS];
+  TA_TRY(ta_read_status(h, words));
+  ta_dfree(h, t1);
+  ta_dfree(h, t2);
+  if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+  out->n_groups = ng;
+  out->g_window = o.g_window; out->g_pid = o.g_pid; out->g_name = o.g_name;
+  out->g_count = o.g_count; out->g_sum = o.g_sum; out->g_min = o.g_min; out->g_max = o.g_max;
+  out->g_hist = o.g_hist;
+  return TA_OK;
+}
+
 ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_agg_result *out) {
   cudaStream_t st = h->stream;
   const int n_pids = h->n_pids > 0 ? h->n_pids : 1;
@@ -256,7 +453,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   if (h->n_valid == 0 || (kind_mask & 63u) == 0) return TA_OK;
   const unsigned __int128 R128 = (unsigned __int128)((uint64_t)h->max_name - (uint64_t)h->min_name) + 1;
   const unsigned __int128 G128 = R128 * (unsigned __int128)((uint64_t)h->W * (uint64_t)n_pids);
-  if (G128 > (unsigned __int128)TA_AGG_DENSE_LIMIT) return TA_ERR_TOO_LARGE;
+  if (G128 > (unsigned __int128)TA_AGG_DENSE_LIMIT) return ta_run_aggregate_sorted(h, kind_mask, value_sel, out);
   const int64_t R = (int64_t)R128, G = (int64_t)G128;
 
   size_t tb = 4 * Carver::pad((size_t)G * 8) + Carver::pad((size_t)G * TA_NBINS * 4) + Carver::pad(64) +

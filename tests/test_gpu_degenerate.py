@@ -1,0 +1,100 @@
+"""Degenerate and extreme inputs through the CUDA library and the oracle alike, run-to-run
+determinism, and two handles alive at once on different streams."""
+import numpy as np
+import pytest
+
+from helpers import make_events
+from paper_2609_40247_b200 import synth
+from runners import assert_same, run_gpu, run_oracle
+from tiny import random_window
+
+pytestmark = pytest.mark.gpu
+I32, I16 = 2**31, 2**15
+T0 = 1_700_000_000_000_000_000  # wall-clock nanoseconds: the full 64-bit range is in play
+
+
+def _both(rows, off=None, t0=(0,), t1=(10_000,), **kw):
+    ev = make_events(rows)
+    off = [0, len(ev)] if off is None else off
+    o = run_oracle(ev, off, list(t0), list(t1), **kw)
+    g = run_gpu(ev, off, list(t0), list(t1), **kw)
+    skip = ()
+    if o["attr_status"] != 0:
+        skip = tuple(k for k in o if k.startswith(("parent", "depth", "op_", "attr_sum", "aggT_", "incl_",
+                                                   "replay_", "roll_")))
+        assert g["attr_status"] == o["attr_status"]
+    assert_same(o, g, skip=skip)
+    return o
+
+
+CASES = {
+    "one kernel": [("KERNEL", 1, 0, 10, 20, 0, 0, 0)],
+    "one host record": [("OP", 1, 0, 10, 20, 0, 0, 0)],
+    "host records only": [("OP", 1, 0, 0, 100, 0, 0, 0), ("LAUNCH", 1, 0, 5, 6, 1, 0, 0), ("API", 1, 0, 7, 7, 0, 0, 0)],
+    "device records only": [("KERNEL", 1, s, 10 * s, 10 * s + 5, s, 0, 0) for s in range(7)],
+    "everything dropped": [("KERNEL", 1, 0, 20_000, 20_001, 0, 0, 0), (9, 1, 0, 1, 2, 0, 0, 0), ("OP", 1, 0, 9, 3, 0, 0, 0)],
+    "extreme ids": [("KERNEL", -I32, -I16, 10, 20, -2**63, -I32, 0), ("KERNEL", I32 - 1, I16 - 1, 10, 20, 2**63 - 1, I32 - 1, 0),
+                    ("LAUNCH", -I32, -I16, 1, 2, -2**63, 0, 0), ("LAUNCH", I32 - 1, I16 - 1, 1, 2, 2**63 - 1, 0, 0),
+                    ("OP", -I32, -I16, 0, 9000, 0, -I32, 0), ("OP", I32 - 1, I16 - 1, 0, 9000, 0, I32 - 1, 0),
+                    ("COLL", -I32, 3, 50, 60, 2**63 - 2, 0, -I32), ("COLL", I32 - 1, 3, 55, 60, 2**63 - 2, 0, -I32)],
+    "all zero length at one instant": [("KERNEL", 1, 0, 500, 500, i, 0, 0) for i in range(40)]
+    + [("OP", 1, 0, 500, 500, 0, i, 0) for i in range(6)] + [("LAUNCH", 1, 0, 500, 500, i, 0, 0) for i in range(40)],
+    "kernel that outlives the window": [("LAUNCH", 1, 0, 10, 11, 1, 0, 0), ("KERNEL", 1, 0, 20, 10**12, 1, 0, 0),
+                                        ("KERNEL", 1, 0, 30, 40, 2, 0, 0)],
+    "many kernels per launch": [("OP", 1, 0, 0, 5000, 0, 0, 0), ("LAUNCH", 1, 0, 10, 20, 7, 0, 0)]
+    + [("KERNEL", 1, i % 3, 100 + 10 * i, 105 + 10 * i, 7, 0, 0) for i in range(100)],
+}
+
+
+@pytest.mark.parametrize("name", sorted(CASES))
+def test_degenerate_windows(name):
+    _both(CASES[name], min_gap=3)
+
+
+def test_wall_clock_timestamps_and_empty_windows_between_full_ones():
+    rows, off, t0, t1 = [], [0], [], []
+    rng = np.random.default_rng(5)
+    for w in range(9):
+        a = T0 + w * 60_000_000_000
+        t0.append(a)
+        t1.append(a + 30_000_000_000)
+        if w % 3 != 1:  # every third window is empty
+            for i in range(50):
+                s = a + int(rng.integers(0, 29_000_000_000))
+                rows.append(("LAUNCH", 1 + w % 2, 0, s, s + 1000, i, 0, 0))
+                rows.append(("KERNEL", 1 + w % 2, i % 2, s + 5000, s + 5000 + int(rng.integers(0, 10**9)), i, i % 5, 0))
+        off.append(len(rows))
+    _both(rows, off=off, t0=t0, t1=t1, min_gap=10**6)
+
+
+def test_two_runs_give_identical_results():
+    wl = synth.make_workload("c3", 0.01, truth=False)
+    a = (wl.events, wl.win_off, wl.win_t0, wl.win_t1)
+    assert_same(run_gpu(*a, comm_sizes=wl.comm_sizes), run_gpu(*a, comm_sizes=wl.comm_sizes))
+
+
+def test_two_handles_on_two_streams_do_not_disturb_each_other():
+    import torch
+    from paper_2609_40247_b200 import ta
+    ev1, off1, a1, b1, _ = random_window(21)
+    wl = synth.make_workload("c1", 0.02, truth=False)
+    want1 = run_gpu(ev1, off1, a1, b1)
+    want2 = run_gpu(wl.events, wl.win_off, wl.win_t0, wl.win_t1)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    buf1 = torch.from_numpy(np.ascontiguousarray(ev1).view(np.uint8).reshape(-1)).cuda()
+    buf2 = torch.from_numpy(np.ascontiguousarray(wl.events).view(np.uint8).reshape(-1)).cuda()
+    torch.cuda.synchronize()
+    with ta.Window(buf1, off1, a1, b1, stream=s1) as w1, \
+            ta.Window(buf2, wl.win_off, wl.win_t0, wl.win_t1, stream=s2) as w2:
+        r2 = w2.sort_timeline()
+        r1 = w1.sort_timeline()
+        j1 = w1.correlate_launches()
+        j2 = w2.correlate_launches()
+        g2 = w2.stream_gaps(500_000)
+        g1 = w1.stream_gaps(500_000)
+        for k in ("perm", "ts_start", "kind", "lane_off"):
+            assert np.array_equal(r1.numpy(k), want1[k]) and np.array_equal(r2.numpy(k), want2[k])
+        for k in ("launch_of", "launch_latency"):
+            assert np.array_equal(j1.numpy(k), want1[k]) and np.array_equal(j2.numpy(k), want2[k])
+        assert np.array_equal(g1.numpy("gap_before"), want1["gap_before"])
+        assert np.array_equal(g2.numpy("gap_before"), want2["gap_before"])

@@ -63,6 +63,17 @@ def test_sparse_correlation_ids_take_the_sort_merge_join():
     assert int(o["join_sum"]["n_matched"].sum()) > 20_000
 
 
+def test_widely_spread_symbol_ids_are_grouped_by_sorting():
+    """name_id values a million apart: the dense aggregate table does not apply and the rows of
+    all three aggregate selectors come from the sort-based path."""
+    wl = synth.make_workload("c1", 0.05, truth=False)
+    ev = wl.events.copy()
+    ev["name_id"] = (ev["name_id"].astype(np.int64) * 1_048_573 - 2**30).astype(np.int32)
+    o, g = both(ev, wl.win_off, wl.win_t0, wl.win_t1, comm_sizes=wl.comm_sizes,
+                agg_masks=(DEVICE_MASK, 1 << 2, 63))
+    assert len(o["agg0_g_count"]) > 100 and len(o["aggT_g_count"]) > 10
+
+
 @pytest.mark.parametrize("run_len,ordinary", [(2, 300), (5, 300), (31, 300), (48, 300), (49, 300),
                                               (400, 300), (60, 12000)])
 def test_runs_of_equal_start_times(run_len, ordinary):
