@@ -180,33 +180,48 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
     for (int j = 0; j < GP_ITEMS; j++) {
       gap[j] = 0;
       const int l = ln[j];
-      if (l < 0) continue;
-      if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
-      const i64 Pi = ((pre >> 40) == (u64)(l + 1)) ? w0 + (i64)(pre & GP_LOW) : w0;
-      const i64 g = s[j] > Pi ? s[j] - Pi : 0;
-      const i64 from = s[j] > Pi ? s[j] : Pi;
-      const i64 bz = ce[j] > from ? ce[j] - from : 0;
-      const bool last = (p0 + j + 1 == (int64_t)a.lane_off[l + 1]);
-      i64 tl = 0;
-      if (last) tl = w1 - (Pi > ce[j] ? Pi : ce[j]);
-      gap[j] = g;
-      pre = max(pre, ((u64)(l + 1) << 40) | (u64)(ce[j] - w0));
-      // long-gap list (rare)
-      const bool lg = g > 0 && g >= a.min_gap, lt = last && tl > 0 && tl >= a.min_gap;
-      if (lg || lt) {
-        i64 o = (i64)atomicAdd(a.n_long, (u64)((lg ? 1 : 0) + (lt ? 1 : 0)));
-        if (lg) {
-          if (o < a.list_cap) {
-            a.list[o] = ta_long_gap{l, (int32_t)(p0 + j), Pi, g};
-            a.list_key[o] = ((u64)l << 32) | (u64)(u32)(p0 + j);
+      i64 Pi = 0, g = 0, bz = 0, tl = 0;
+      bool last = false, lg = false, lt = false;
+      if (l >= 0) {
+        if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
+        Pi = ((pre >> 40) == (u64)(l + 1)) ? w0 + (i64)(pre & GP_LOW) : w0;
+        g = s[j] > Pi ? s[j] - Pi : 0;
+        const i64 from = s[j] > Pi ? s[j] : Pi;
+        bz = ce[j] > from ? ce[j] - from : 0;
+        last = (p0 + j + 1 == (int64_t)a.lane_off[l + 1]);
+        if (last) tl = w1 - (Pi > ce[j] ? Pi : ce[j]);
+        gap[j] = g;
+        pre = max(pre, ((u64)(l + 1) << 40) | (u64)(ce[j] - w0));
+        lg = g > 0 && g >= a.min_gap;
+        lt = last && tl > 0 && tl >= a.min_gap;
+      }
+      // long-gap list: the warp reserves its entries with one add on the cursor (the order of
+      // the list does not matter, it is sorted afterwards)
+      {
+        const u32 m_g = __ballot_sync(0xffffffffu, lg), m_t = __ballot_sync(0xffffffffu, lt);
+        if (m_g | m_t) {
+          const int wlane = threadIdx.x & 31;
+          const u32 below = (1u << wlane) - 1u;
+          u64 base = 0;
+          if (wlane == 0) base = atomicAdd(a.n_long, (u64)(__popc(m_g) + __popc(m_t)));
+          base = __shfl_sync(0xffffffffu, base, 0);
+          if (lg) {
+            const i64 o = (i64)base + __popc(m_g & below);
+            if (o < a.list_cap) {
+              a.list[o] = ta_long_gap{l, (int32_t)(p0 + j), Pi, g};
+              a.list_key[o] = ((u64)l << 32) | (u64)(u32)(p0 + j);
+            }
           }
-          o++;
-        }
-        if (lt && o < a.list_cap) {
-          a.list[o] = ta_long_gap{l, -1, w1 - tl, tl};
-          a.list_key[o] = ((u64)l << 32) | 0xFFFFFFFFull;
+          if (lt) {
+            const i64 o = (i64)base + __popc(m_g) + __popc(m_t & below);
+            if (o < a.list_cap) {
+              a.list[o] = ta_long_gap{l, -1, w1 - tl, tl};
+              a.list_key[o] = ((u64)l << 32) | 0xFFFFFFFFull;
+            }
+          }
         }
       }
+      if (l < 0) continue;
       if (a.list_only) continue;
       if (lm < 0) lm = l;
       const int li = l - l0;
@@ -301,7 +316,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   cudaStream_t st = h->stream;
   if (L >= (1 << 22) - 1) return TA_ERR_TOO_LARGE;
   const int64_t tiles = (n + GP_TILE - 1) / GP_TILE;
-  int64_t cap = n / 16 > 65536 ? n / 16 : 65536;
+  int64_t cap = n / 8 > 65536 ? n / 8 : 65536;  // first guess; a longer list is rebuilt below
   size_t bytes = Carver::pad((size_t)(n > 0 ? n : 1) * 8) + Carver::pad((size_t)(L + 1) * sizeof(ta_lane_gaps)) +
                  Carver::pad((size_t)(L + 1) * TA_NBINS * 4) + Carver::pad((size_t)W * TA_NBINS * 4) +
                  Carver::pad((size_t)(tiles + 1) * 8) + Carver::pad(64) + 512;
