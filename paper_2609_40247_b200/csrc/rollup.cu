@@ -107,25 +107,42 @@ __global__ void __launch_bounds__(RO_THREADS) k_roll_finalize(RollArgs a) {
   if (!roll_tile(a, 0, &p0, &tile_end)) return;
   int16_t kd[RO_ITEMS];
   load8_i16(a.kind, p0, a.n, 9, kd);
+  // counts first (inclusive kernels of the OPs, kernels of the launches), then the coded times
+  // of the rows that were touched, all of a thread's loads of one kind issued together
+  int32_t cnt[RO_ITEMS];
+#pragma unroll
+  for (int j = 0; j < RO_ITEMS; j++) {
+    cnt[j] = 0;
+    if (p0 + j >= tile_end) continue;
+    if (kd[j] == TA_KIND_OP) cnt[j] = a.incl_n[p0 + j];
+    else if (kd[j] == TA_KIND_LAUNCH) cnt[j] = a.kol[p0 + j];
+  }
+  unsigned ops = 0, reps = 0;
+#pragma unroll
+  for (int j = 0; j < RO_ITEMS; j++) {
+    if (kd[j] == TA_KIND_OP && cnt[j] > 0) ops |= 1u << j;
+    if (kd[j] == TA_KIND_LAUNCH && cnt[j] >= 2) reps |= 1u << j;
+  }
+  if (!(ops | reps)) return;
+  u64 f[RO_ITEMS], l[RO_ITEMS];
+#pragma unroll
+  for (int j = 0; j < RO_ITEMS; j++) {
+    if (ops & (1u << j)) { f[j] = a.incl_first[p0 + j]; l[j] = a.incl_last[p0 + j]; }
+    else if (reps & (1u << j)) { f[j] = a.replay_first[p0 + j]; l[j] = a.replay_last[p0 + j]; }
+  }
 #pragma unroll
   for (int j = 0; j < RO_ITEMS; j++) {
     const int64_t p = p0 + j;
-    if (p >= tile_end) break;
-    if (kd[j] == TA_KIND_OP) {
-      if (a.incl_n[p] > 0) {
-        a.incl_first[p] = (~a.incl_first[p]) ^ (1ull << 63);
-        a.incl_last[p] = a.incl_last[p] ^ (1ull << 63);
-      }
-    } else if (kd[j] == TA_KIND_LAUNCH) {
-      const int32_t k = a.kol[p];
-      if (k >= 2) {
-        a.replay_first[p] = (~a.replay_first[p]) ^ (1ull << 63);
-        a.replay_last[p] = a.replay_last[p] ^ (1ull << 63);
-        const int w = a.lane_window[lane_of_pos(a.lane_off, a.n_lanes, p)];
-        atomicAdd(&a.win_sum[(size_t)w * 3], 1ull);
-        atomicAdd(&a.win_sum[(size_t)w * 3 + 1], (u64)k);
-        atomicMax(&a.win_sum[(size_t)w * 3 + 2], (u64)k);
-      }
+    if (ops & (1u << j)) {
+      a.incl_first[p] = (~f[j]) ^ (1ull << 63);
+      a.incl_last[p] = l[j] ^ (1ull << 63);
+    } else if (reps & (1u << j)) {
+      a.replay_first[p] = (~f[j]) ^ (1ull << 63);
+      a.replay_last[p] = l[j] ^ (1ull << 63);
+      const int w = a.lane_window[lane_of_pos(a.lane_off, a.n_lanes, p)];
+      atomicAdd(&a.win_sum[(size_t)w * 3], 1ull);
+      atomicAdd(&a.win_sum[(size_t)w * 3 + 1], (u64)cnt[j]);
+      atomicMax(&a.win_sum[(size_t)w * 3 + 2], (u64)cnt[j]);
     }
   }
 }
