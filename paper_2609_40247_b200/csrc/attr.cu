@@ -94,46 +94,7 @@ __device__ __forceinline__ void wstack_combine(const WStack &ear, WStack &acc, b
   acc.reset = ear.reset;
 }
 
-__device__ __forceinline__ int warp_lane_search_a(const int32_t *lane_off, int n_lanes, int64_t p) {
-  const int lane = threadIdx.x & 31;
-  int lo = 0, hi = n_lanes;
-  while (hi - lo > 1) {
-    int step = (hi - lo + 31) >> 5;
-    int idx = lo + lane * step;
-    bool ok = idx < hi && (int64_t)lane_off[idx] <= p;
-    u32 m = __ballot_sync(0xffffffffu, ok);
-    int k = 31 - __clz((int)m);
-    lo = lo + k * step;
-    hi = min(hi, lo + step);
-  }
-  return lo;
-}
 
-__device__ __forceinline__ void load_kinds8(const int16_t *kind, int64_t p0, int64_t n, int16_t *kd) {
-  if (p0 + AT_ITEMS <= n) {
-    uint4 q = *reinterpret_cast<const uint4 *>(kind + p0);
-    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
-#pragma unroll
-    for (int j = 0; j < AT_ITEMS; j++) kd[j] = hq[j];
-  } else {
-#pragma unroll
-    for (int j = 0; j < AT_ITEMS; j++) kd[j] = p0 + j < n ? kind[p0 + j] : (int16_t)9;
-  }
-}
-__device__ __forceinline__ void load_i64x8(const int64_t *col, int64_t p0, int64_t n, i64 *v) {
-  if (p0 + AT_ITEMS <= n) {
-    const longlong2 *ps = reinterpret_cast<const longlong2 *>(col + p0);
-#pragma unroll
-    for (int j = 0; j < AT_ITEMS / 2; j++) {
-      longlong2 x = ps[j];
-      v[2 * j] = x.x;
-      v[2 * j + 1] = x.y;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < AT_ITEMS; j++) v[j] = p0 + j < n ? col[p0 + j] : 0;
-  }
-}
 
 // ---- kernel 1: the stack each tile leaves behind --------------------------------
 __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
@@ -149,11 +110,11 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
   if (tid == 0) s_raw = 0;
   if (warp == 0) {
     int l = -1;
-    if (plast >= tile_start) l = warp_lane_search_a(a.lane_off, a.n_lanes, plast);
+    if (plast >= tile_start) l = tile_lane_search(a.lane_off, a.n_lanes, plast);
     if (lane == 0) s_lane1 = l;
   }
   int16_t kd[AT_ITEMS];
-  load_kinds8(a.kind, p0, a.n, kd);
+  load8_i16(a.kind, p0, a.n, 9, kd);
   __syncthreads();
   const int lane1 = s_lane1;
   if (lane1 < 0 || a.lane_domain[lane1] != 0) {
@@ -171,7 +132,7 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
   i64 m8 = INT64_MIN;
   if (opmask) {
     i64 t[AT_ITEMS];
-    load_i64x8(a.te, p0, a.n, t);
+    load8_i64(a.te, p0, a.n, t);
 #pragma unroll
     for (int j = 0; j < AT_ITEMS; j++)
       if (opmask & (1u << j)) { en[j] = t[j]; m8 = m8 > t[j] ? m8 : t[j]; }
@@ -366,7 +327,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
   if (tid == 0) { s.lane1 = -1; s.dmax = 0; s.lane0 = -1; }
   __syncthreads();
   if (warp == 0 && tile_start < a.n_valid && a.n_lanes > 0) {
-    int l = warp_lane_search_a(a.lane_off, a.n_lanes, tile_start);
+    int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (lane == 0) s.lane0 = l;
   }
   const int ccnt = a.carry_cnt[tile];
@@ -375,7 +336,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     s.carry_pos[tid] = a.carry_pos[(size_t)tile * AT_CAP + tid];
   }
   int16_t kd[AT_ITEMS];
-  load_kinds8(a.kind, p0, a.n, kd);
+  load8_i16(a.kind, p0, a.n, 9, kd);
   unsigned hostmask = 0;
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++)
@@ -396,8 +357,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) st[j] = en[j] = 0;
   if (hostmask) {
-    load_i64x8(a.ts, p0, a.n, st);
-    load_i64x8(a.te, p0, a.n, en);
+    load8_i64(a.ts, p0, a.n, st);
+    load8_i64(a.te, p0, a.n, en);
   }
   // lanes, leaves, the thread's maximum
   const int l0 = s.lane0;

@@ -12,6 +12,7 @@
 // HBM-bound: 18 B read + 8 B written per device record.
 #include <climits>
 
+#include "scan.cuh"
 #include "ta_internal.cuh"
 
 #define GP_THREADS 256
@@ -45,21 +46,6 @@ struct GapArgs {
   u64 *n_long;        // append cursor
 };
 
-// largest l with lane_off[l] <= p, found by the 32 lanes of one warp together
-__device__ __forceinline__ int warp_lane_search(const int32_t *lane_off, int n_lanes, int64_t p) {
-  const int lane = threadIdx.x & 31;
-  int lo = 0, hi = n_lanes;
-  while (hi - lo > 1) {
-    int step = (hi - lo + 31) >> 5;
-    int idx = lo + lane * step;
-    bool ok = idx < hi && (int64_t)lane_off[idx] <= p;
-    u32 m = __ballot_sync(0xffffffffu, ok);
-    int k = 31 - __clz((int)m);  // lane 0 always qualifies (lane_off[lo] <= p)
-    lo = lo + k * step;
-    hi = min(hi, lo + step);
-  }
-  return lo;
-}
 
 __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   __shared__ u64 tmp[33];
@@ -76,7 +62,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   const int64_t p0 = tile_start + (int64_t)tid * GP_ITEMS;
   if (tid < 32) {
     int l = -1;
-    if (tile_start < a.n_valid && a.n_lanes > 0) l = warp_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (tile_start < a.n_valid && a.n_lanes > 0) l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (tid == 0) s_lane0 = l;
   }
   __syncthreads();
