@@ -194,12 +194,6 @@ struct RankRowOut {
   }
 };
 
-static int bit_len(uint64_t v) {
-  int b = 0;
-  while (v) { b++; v >>= 1; }
-  return b;
-}
-
 ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_comms_given,
                              ta_coll_result *out) {
   const int64_t n = h->n, nn = n > 0 ? n : 1;
@@ -247,9 +241,9 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   cx.seq = h->sorted.seq; cx.pid = h->sorted.pid;
   cx.lane_off = h->sorted.lane_off; cx.lane_slot = h->d_lane_slot; cx.lane_window = h->sorted.lane_window;
   cx.n_lanes = h->sorted.n_lanes; cx.n_pids = n_pids; cx.cm = h->d_comms; cx.min_seq = h->min_seq;
-  cx.qbits = bit_len((uint64_t)(h->max_seq - h->min_seq));
-  cx.cbits = bit_len((uint64_t)(h->n_comms - 1));
-  const int wbits = bit_len((uint64_t)(h->W - 1));
+  cx.qbits = ta_bit_len((uint64_t)(h->max_seq - h->min_seq));
+  cx.cbits = ta_bit_len((uint64_t)(h->n_comms - 1));
+  const int wbits = ta_bit_len((uint64_t)(h->W - 1));
   if (cx.qbits < 1) cx.qbits = 1;
   if (cx.qbits + cx.cbits + wbits > 62) return TA_ERR_TOO_LARGE;
 

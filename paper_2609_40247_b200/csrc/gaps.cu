@@ -289,12 +289,6 @@ __global__ void __launch_bounds__(256) k_gap_list_gather(const ta_long_gap *src,
   if (i < m) dst[i] = src[order[i]];
 }
 
-static int bit_len_g(uint64_t v) {
-  int b = 0;
-  while (v) { b++; v >>= 1; }
-  return b;
-}
-
 ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   const int64_t n = h->n;
   const int L = h->sorted.n_lanes;
@@ -371,7 +365,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
     u64 *ks = cs.take<u64>(m), *kf = cs.take<u64>(m);
     u32 *vs = cs.take<u32>(m), *order = cs.take<u32>(m);
     TA_TRY(ta_radix_sort_pairs(h, ukeys, nullptr, ks, vs, kf, order, m,
-                               ta_make_plan(0, 32 + bit_len_g((uint64_t)(L > 1 ? L - 1 : 1))), nullptr,
+                               ta_make_plan(0, 32 + ta_bit_len((uint64_t)(L > 1 ? L - 1 : 1))), nullptr,
                                cs.base + cs.off));
     k_gap_list_gather<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(ulist, order, m, list);
     TA_CHECK_CUDA(h, cudaGetLastError());

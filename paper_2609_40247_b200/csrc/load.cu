@@ -335,12 +335,6 @@ __global__ void __launch_bounds__(256) k_load_pre(LoadArgs a) {
 }
 
 // ------------------------------------------------------------------ host
-static int bit_length(uint64_t v) {
-  int b = 0;
-  while (v) { b++; v >>= 1; }
-  return b;
-}
-
 static int grid_for(int64_t n, int threads, int per_sm) {
   int64_t g = (n + threads - 1) / threads;
   int64_t cap = 148ll * per_sm;
@@ -374,14 +368,14 @@ ta_status ta_launch_load(ta_window *h, bool allow_packed) {
     max_span = max_span > h->h_t1[w] - h->h_t0[w] ? max_span : h->h_t1[w] - h->h_t0[w];
     max_win = max_win > h->h_off[w + 1] - h->h_off[w] ? max_win : h->h_off[w + 1] - h->h_off[w];
   }
-  h->sbits = bit_length((uint64_t)(max_span - 1));
-  h->tbits = bit_length((uint64_t)(h->n_triples > 0 ? h->n_triples - 1 : 0));
-  h->wbits = bit_length((uint64_t)(h->W - 1));
+  h->sbits = ta_bit_len((uint64_t)(max_span - 1));
+  h->tbits = ta_bit_len((uint64_t)(h->n_triples > 0 ? h->n_triples - 1 : 0));
+  h->wbits = ta_bit_len((uint64_t)(h->W - 1));
   const int hd = h->has_dropped ? 1 : 0;
   int total = h->sbits + h->tbits + h->wbits + hd;
   if (total > 63) return TA_ERR_TOO_LARGE;
   if (((int64_t)h->W << h->tbits) > (1ll << 24)) return TA_ERR_TOO_LARGE;
-  h->ibits = bit_length((uint64_t)(max_win - 1));
+  h->ibits = ta_bit_len((uint64_t)(max_win - 1));
   if (h->ibits < 1) h->ibits = 1;
   int drop = total + h->ibits - 64;
   if (drop < 0) drop = 0;

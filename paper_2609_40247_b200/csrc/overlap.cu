@@ -243,12 +243,6 @@ struct OvRowOut {
   }
 };
 
-static int ov_bit_len(uint64_t v) {
-  int b = 0;
-  while (v) { b++; v >>= 1; }
-  return b;
-}
-
 ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   cudaStream_t st = h->stream;
   memset(out, 0, sizeof(*out));
@@ -258,12 +252,12 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   if (m <= 0 || h->n_valid <= 0) return TA_OK;
   int64_t max_span = 1;
   for (int w = 0; w < h->W; w++) max_span = h->h_t1[w] - h->h_t0[w] > max_span ? h->h_t1[w] - h->h_t0[w] : max_span;
-  const int tsbits = ov_bit_len((uint64_t)max_span);
-  const int slot_bits = ov_bit_len((uint64_t)(n_slots - 1));
+  const int tsbits = ta_bit_len((uint64_t)max_span);
+  const int slot_bits = ta_bit_len((uint64_t)(n_slots - 1));
   if (tsbits > 40 || tsbits + slot_bits > 63 || n_slots >= (1ll << 22)) return TA_ERR_TOO_LARGE;
   // when (slot, time, index) fit one 64-bit word the index travels inside the key and the
   // passes move keys only (8 B + 8 B per record instead of 12 B + 12 B)
-  int idxbits = ov_bit_len((uint64_t)(m - 1));
+  int idxbits = ta_bit_len((uint64_t)(m - 1));
   if (idxbits < 1) idxbits = 1;
   if (tsbits + slot_bits + idxbits > 64) idxbits = 0;
 

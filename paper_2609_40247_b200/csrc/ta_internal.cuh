@@ -101,6 +101,13 @@ struct ta_window {
   int attr_status;
 };
 
+// number of bits needed to write v (0 for 0)
+static inline int ta_bit_len(uint64_t v) {
+  int b = 0;
+  while (v) { b++; v >>= 1; }
+  return b;
+}
+
 // -------------------------------------------------------------- memory
 void *ta_dalloc(ta_window *h, size_t bytes);            // NULL on failure
 void ta_dfree(ta_window *h, void *p);                   // early release of one allocation
