@@ -1,8 +1,16 @@
 // ta_load_window kernels: validity (start-time filtering separates windows,
 // Sec. 5.2), discovery and dense ranking of the (pid, domain, stream) triples
-// that name a lane, and the 64-bit sort key (window | triple rank | ts_start -
-// t0) together with the digit histograms of every radix pass.
-// HBM-bound: each kernel streams the 40-byte records once.
+// that name a lane, and the 64-bit sort key together with the digit histograms
+// of every radix pass.
+//   k_discover      one pass over the 40-byte records: defect counters, the triple and
+//                   communicator sets, value ranges, and one 64-bit word per record
+//                   (dropped flag | triple slot | ts_start - t0);
+//   k_rank_*        one CTA each: sort and rank the few triples / communicator ids;
+//   k_load_pre      turns those words into keys in place - [dropped][window][triple
+//                   rank][(ts_start - t0) >> dshift]{[index in window]} - and takes the
+//                   histograms; k_load does the same from the records when the sort
+//                   falls back to full-resolution (key, index) pairs.
+// The records are streamed once here and gathered once by the sort.
 #include "ta_internal.cuh"
 #include "records.cuh"
 

@@ -1,21 +1,22 @@
 // ta_sort_timeline: canonical order of the timeline.
 //
-//   1. stable radix sort of (key, input index) by the key built at load time
-//      (window | lane triple rank | ts_start - t0); stability gives the input
-//      index tie-break for free;
-//   2. runs of equal keys are reordered by ts_end descending (short runs in
-//      place; if a longer run exists the sort is redone with the duration as a
-//      least-significant key);
-//   3. dropped records (tail) are ordered by the full tuple with a chain of
-//      stable sorts;
-//   4. whole 40-byte records are gathered once into eight sorted columns and
-//      lane boundaries are recorded.
+// Packed keys (the usual case): the key carries the record's index in its low bits and the
+// start time at a coarser resolution, so four keys-only radix passes settle the order down
+// to (lane, coarse time); k_gather, which brings every 40-byte record into registers once to
+// write the eight sorted columns, ranks the members of a run of equal coarse keys by
+// (ts_start, -ts_end, input index) on the way, and records the lane boundaries and the
+// correlation-id range of every (window, pid) for the join.
+// Fallback (a run longer than TA_TIE_RUN_MAX, or keys that do not fit): stable radix sort of
+// (key, input index) pairs at full time resolution; runs of equal keys are reordered by
+// ts_end descending in place (k_fix_ties), and if even such a run is too long the sort is
+// redone with the duration as a least-significant key.
+// Dropped records (the tail) are ordered by the full tuple with a chain of stable sorts.
 #include <climits>
 
 #include "records.cuh"
 #include "ta_internal.cuh"
 
-// ---- step 2: equal-key runs --------------------------------------------
+// ---- pair path: equal-key runs -------------------------------------------
 __global__ void __launch_bounds__(256) k_fix_ties(const u64 *keys, u32 *perm, int64_t n_valid,
                                                   const ta_event *ev, int32_t *status) {
   int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
