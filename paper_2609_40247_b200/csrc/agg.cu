@@ -1,5 +1,6 @@
 // ta_aggregate_ops: per (window, pid, name_id) count / sum / min / max and a log2
-// histogram of a value column (own duration, or T_op of operators with kernels).
+// histogram of a value column (own duration, T_op of operators with kernels, or the
+// idle time charged to an operator by the gap blame).
 // Per-symbol counts and duration statistics are what Sec. 8.1 compares.
 //
 // Symbol popularity is heavy-tailed (a few names carry most records), so global
@@ -8,7 +9,8 @@
 // hold a selected kind return at once) and folds its records into a
 // shared-memory hash table first; the table is flushed to a dense global table
 // indexed by (window, pid rank, name_id - min name) with one atomic per field.
-// A scan then compacts the non-empty rows in key order.
+// A scan then compacts the non-empty rows in key order.  Symbol ids spread too wide
+// for a dense table take the sort-based path at the end of this file instead.
 // HBM-bound on the column reads: 2 B (kind) for every record, 24 B more for the
 // selected ones.
 #include <climits>
