@@ -289,14 +289,17 @@ def main():
     ta.profile_enable(True)
     launches0 = ta.launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
     barrier()
     ev0.record()
-    for _ in range(args.steps):
+    for k in range(args.steps):
         n_valid, _ = run_pipeline(ta, dev_buf, wl)
+        marks[k].record()
     ev1.record()
     torch.cuda.synchronize()
     barrier()
     elapsed_ms = ev0.elapsed_time(ev1)
+    per_step = [(ev0 if k == 0 else marks[k - 1]).elapsed_time(marks[k]) for k in range(args.steps)]
     launches = ta.launch_count() - launches0
     n_pass, radix_ms, radix_bytes = ta.profile_radix()
     ta.profile_enable(False)
@@ -372,6 +375,7 @@ def main():
             "clocks": clocks, "gpu_launches": int(launches),
             "roofline": roof, "cpu_baseline": cpu,
             "per_call_ms": per_call_ms,
+            "step_ms": {"median": statistics.median(per_step), "best": min(per_step)} if per_step else None,
         }
         lsd_bytes, key_bits, passes, parts = lsd_model_bytes_per_event(wl)
         per_gpu = value / world
