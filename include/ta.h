@@ -27,6 +27,10 @@
  *   - Call order: load -> sort -> { correlate -> attribute ; gaps ;
  *     aggregate(value_sel 0) ; collectives }.  aggregate(value_sel 1) needs
  *     attribute.  A call made too early returns TA_ERR_ORDER.
+ *   - Threads: a handle is used by one thread at a time; different handles may
+ *     be used from different threads and on different streams at the same time
+ *     (the library keeps no state outside the handle except its memory pool, the
+ *     launch counter and the benchmark instrumentation at the end of this file).
  */
 #ifndef TA_H
 #define TA_H

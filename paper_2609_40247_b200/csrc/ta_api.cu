@@ -1,7 +1,9 @@
 // C-ABI entry points (include/ta.h): argument checks, the handle, memory
 // through the caller's allocator, call-order bookkeeping.  All arithmetic lives
 // in the kernels of the other translation units.
+#include <atomic>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "ta_internal.cuh"
@@ -11,7 +13,9 @@
 // memory back at every synchronisation, which makes each call pay for fresh gigabytes.
 static cudaMemPool_t own_pool(int device) {
   static cudaMemPool_t pools[64] = {};
+  static std::mutex guard;  // handles on different threads may arrive here together
   if (device < 0 || device >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(guard);
   if (!pools[device]) {
     cudaMemPoolProps props;
     memset(&props, 0, sizeof(props));
@@ -76,7 +80,7 @@ ta_status ta_read_status(ta_window *h, int32_t *w) {
 }
 
 // ---- instrumentation: launch counter and event pairs around the radix passes ----
-long long g_ta_launches = 0;
+std::atomic<long long> g_ta_launches{0};
 int g_ta_profile = 0;
 static std::vector<cudaEvent_t> g_prof_events;  // begin, end, begin, end, ...
 static size_t g_prof_used = 0;
@@ -118,7 +122,7 @@ int32_t ta_profile_radix(int64_t *n_passes, double *total_ms, double *total_byte
   if (total_bytes) *total_bytes = g_prof_bytes;
   return 0;
 }
-int64_t ta_launch_count(void) { return g_ta_launches; }
+int64_t ta_launch_count(void) { return g_ta_launches.load(); }
 
 const char *ta_strerror(ta_status s) {
   switch (s) {

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <vector>
 
 #include "../../include/ta.h"
@@ -180,7 +181,7 @@ ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result 
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 
 // ---- instrumentation (no work: a launch counter and optional event pairs) ----
-extern long long g_ta_launches;   // kernels launched by this library since load
+extern std::atomic<long long> g_ta_launches;  // kernels launched by this library since load
 extern int g_ta_profile;          // 1 = record a CUDA event pair around each radix pass
 static inline unsigned ta_one() { ++g_ta_launches; return 1u; }
 #define TA_N ta_one() *           // used as kernel<<<TA_N grid, ...>>>: counts the launch

@@ -98,3 +98,33 @@ def test_two_handles_on_two_streams_do_not_disturb_each_other():
             assert np.array_equal(j1.numpy(k), want1[k]) and np.array_equal(j2.numpy(k), want2[k])
         assert np.array_equal(g1.numpy("gap_before"), want1["gap_before"])
         assert np.array_equal(g2.numpy("gap_before"), want2["gap_before"])
+
+
+def test_two_threads_with_a_handle_each():
+    """ctypes releases the interpreter lock during a call, so two Python threads really are
+    inside the library at the same time, each with its own handle and stream."""
+    import threading
+    import torch
+    wl = [synth.make_workload("c1", 0.03, truth=False, seed_offset=k) for k in range(2)]
+    want = [run_gpu(w.events, w.win_off, w.win_t0, w.win_t1, comm_sizes=w.comm_sizes) for w in wl]
+    got = [None, None]
+    errors = []
+
+    def work(k):
+        try:
+            torch.cuda.set_device(0)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                for _ in range(3):
+                    got[k] = run_gpu(wl[k].events, wl[k].win_off, wl[k].win_t0, wl[k].win_t1,
+                                     comm_sizes=wl[k].comm_sizes)
+        except Exception as e:  # surfaced in the main thread below
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for k in range(2):
+        assert_same(want[k], got[k])
