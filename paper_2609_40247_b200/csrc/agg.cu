@@ -63,8 +63,8 @@ struct AggSmem {
 
 __device__ __forceinline__ void agg_global_add(const AggArgs &a, int64_t g, u64 cnt, u64 sum, u64 minc,
                                                u64 maxb) {
-  u64 old = atomicAdd(&a.d_cnt[g], cnt);
-  if (old == 0) atomicAdd(a.n_groups, 1ull);
+  // none of the results is used: the adds go out without the thread waiting for them
+  atomicAdd(&a.d_cnt[g], cnt);
   atomicAdd(&a.d_sum[g], sum);
   atomicMax(&a.d_minc[g], minc);
   atomicMax(&a.d_maxb[g], maxb);
@@ -213,6 +213,15 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
     }
   }
   agg_flush(a, s);
+}
+
+// number of non-empty rows (only needed up front when the output cannot be sized by a bound)
+__global__ void __launch_bounds__(256) k_agg_count_rows(const u64 *cnt, int64_t G, u64 *n_rows) {
+  u64 c = 0;
+  for (int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; g < G; g += (int64_t)gridDim.x * blockDim.x)
+    c += cnt[g] ? 1ull : 0ull;
+  c = warp_reduce(c, OpAdd());
+  if ((threadIdx.x & 31) == 0 && c) atomicAdd(n_rows, c);
 }
 
 // compaction of the non-empty rows in dense (= key) order
@@ -496,10 +505,13 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   u64 cap = (u64)G < (u64)h->n_valid ? (u64)G : (u64)h->n_valid;
   const bool bounded = cap * (28 + 32 + TA_NBINS * 4) <= (256ull << 20);
   if (!bounded) {
+    const int64_t want = (G + 255) / 256;
+    k_agg_count_rows<<<TA_N (unsigned)(want < 148 * 8 ? want : 148 * 8), 256, 0, st>>>(a.d_cnt, G, a.n_groups);
     TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
     cap = ng;
   }
+  u64 *scan_total = nullptr;
   if (cap > 0) {
     size_t ob = 3 * Carver::pad(cap * 4) + 4 * Carver::pad(cap * 8) + Carver::pad(cap * TA_NBINS * 4) + 256;
     void *outb = ta_dalloc(h, ob);
@@ -516,11 +528,13 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
     TA_TRY(scan_temp_init(h, scan_mem, G, &t));
     AggRowIn ri{a.d_cnt};
     TA_TRY((launch_scan<OpAdd, AggRowIn, AggRowOut>(h, G, ri, ro, OpAdd(), t)));
+    scan_total = t.total;
     out->g_window = ro.g_window; out->g_pid = ro.g_pid; out->g_name = ro.g_name;
     out->g_count = ro.g_count; out->g_sum = ro.g_sum; out->g_min = ro.g_min; out->g_max = ro.g_max;
     out->g_hist = ro.g_hist;
   }
-  if (bounded) TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
+  if (bounded && scan_total)  // the scan's total is the number of rows
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, scan_total, 8, cudaMemcpyDeviceToHost, st));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   out->n_groups = (int64_t)ng;
