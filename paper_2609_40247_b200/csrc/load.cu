@@ -44,10 +44,11 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
   if (threadIdx.x < 64) ccache[threadIdx.x] = TRIPLE_EMPTY;
   __syncthreads();
   i64 mn = INT64_MAX, mx = INT64_MIN, md = 0, qmn = INT64_MAX, qmx = INT64_MIN;
+  WindowWalker ww(off, W);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
        i += (int64_t)gridDim.x * blockDim.x) {
     Rec r = load_rec(ev, i);
-    int w = window_of(off, W, i);
+    int w = ww.at(i);
     int def = defect_of(r, t0[w], t1[w]);
     if (def) {
       int64_t *f = def == 1 ? &sum[w].n_bad_kind
@@ -305,12 +306,13 @@ __global__ void __launch_bounds__(256) k_load_pre(LoadArgs a) {
   const int tsb = a.sbits - a.dshift;
   const int64_t stride = (int64_t)gridDim.x * blockDim.x;
   const int64_t n_round = ((a.n + 31) / 32) * 32;
+  WindowWalker ww(a.off, a.W);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_round; i += stride) {
     bool in = i < a.n;
     u64 key = 0;
     if (in) {
       const u64 pk = a.keys[i];
-      int w = window_of(a.off, a.W, i);
+      int w = ww.at(i);
       u64 hi;
       if (pk & PRE_DROPPED) {
         hi = (1ull << (a.wbits + a.tbits + tsb)) | ((u64)w << (a.tbits + tsb));

@@ -53,6 +53,26 @@ __device__ __forceinline__ int window_of(const int64_t *off, int W, int64_t i) {
   return lo;
 }
 
+// Window of an input index for a thread whose indices only grow (grid-stride loops): one
+// binary search, then a forward walk over the window offsets.
+struct WindowWalker {
+  const int64_t *off;
+  int W, w;
+  int64_t hi;  // off[w + 1]
+  __device__ __forceinline__ WindowWalker(const int64_t *o, int nw) : off(o), W(nw), w(-1), hi(0) {}
+  __device__ __forceinline__ int at(int64_t i) {
+    if (w < 0) {
+      w = window_of(off, W, i);
+      hi = off[w + 1];
+    }
+    while (i >= hi) {  // also steps over empty windows
+      w++;
+      hi = off[w + 1];
+    }
+    return w;
+  }
+};
+
 // 0 = kept, 1 bad kind, 2 bad interval, 3 start outside the window
 __device__ __forceinline__ int defect_of(const Rec &r, i64 t0, i64 t1) {
   if (r.kind < 0 || r.kind > 5) return 1;
