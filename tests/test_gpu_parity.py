@@ -97,6 +97,22 @@ def test_runs_of_equal_start_times(run_len, ordinary):
     both(ev, [0, len(ev)], [0], [10000], min_gap=5)
 
 
+def test_defects_sprinkled_over_a_multi_window_batch():
+    """A few percent of the records of a nine-window batch are made defective (bad kind, negative
+    length, start outside the window): the dropped tail spans many tiles and every window."""
+    wl = synth.make_workload("c4", 0.002, truth=False, n_windows=9)
+    ev = wl.events.copy()
+    rng = np.random.default_rng(11)
+    n = len(ev)
+    bad = rng.choice(n, size=n // 25, replace=False)
+    third = len(bad) // 3
+    ev["kind"][bad[:third]] = 9
+    ev["ts_end"][bad[third:2 * third]] = ev["ts_start"][bad[third:2 * third]] - 1 - rng.integers(0, 1000, third)
+    ev["ts_start"][bad[2 * third:]] -= 10**12
+    o, g = both(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=500_000, comm_sizes=wl.comm_sizes)
+    assert o["n_valid"] < n - third and int(o["load_sum"]["n_bad_kind"].sum()) == third
+
+
 def test_deep_nesting_is_reported():
     rows = [("OP", 1, 0, 10 + i, 1000 - i, 0, i, 0) for i in range(12)]
     rows.append(("LAUNCH", 1, 0, 100, 110, 1, 0, 0))
