@@ -126,6 +126,12 @@ struct Oracle {
   std::vector<int32_t> d_window, d_pid;
   std::vector<int64_t> d_n_events, d_busy, d_idle, d_compute, d_comm, d_overlap, d_exposed;
 
+  // critical path
+  std::vector<uint8_t> on_path;                 // per sorted position
+  std::vector<int32_t> cp_window, cp_pid, cp_sink, cp_n_nodes, cp_reason;
+  std::vector<int64_t> cp_begin, cp_end, cp_ns;  // cp_ns: [row][8]
+  std::vector<int64_t> cp_sum;                  // [window][10]: paths, nodes, the eight classes
+
   bool is_kept(int64_t p) const { return p < n_valid; }
 
   // ---- step 1: validity.  Start-time filtering separates successive windows
@@ -552,6 +558,118 @@ struct Oracle {
     }
   }
 
+  // ---- critical path (needs correlate()).  Submission, execution-order and synchronisation
+  // dependencies identify the critical path; where a dependency is missing, the delay it would
+  // explain stays unresolved (Sec. 6.1, "Execution progress and state"; Fig. "Critical path":
+  // host work, the API call that submits kernel k1, k1, the end of the host's wait, host work
+  // again - kernel k2 of another stream and the wait itself are off the path).
+  // Readings.  One path per (window, process).  Nodes are the valid API and LAUNCH records
+  // (host) and the KERNEL, MEMCPY and COLL records (device); OP records are context.  A node
+  // has a START point (ts_start) and an END point (ts_end).  The walk starts at the END of the
+  // sink - the node with the greatest ts_end, the highest canonical position among equals -
+  // and always steps back to the dependency that was released last:
+  //   END(v), v an API record that waited: to END(d), where d is the device record of the
+  //     process with the greatest ts_end < ts_end(v) (highest position among equals) and
+  //     v waited iff ts_end(d) >= ts_start(v)                        [synchronisation edge]
+  //   END(v) otherwise: to START(v)                                  [v ran]
+  //   START(k), k a device record: stream order offers END(q), q the record just before k
+  //     in its lane, if ts_end(q) <= ts_start(k); submission offers START(l), l = launch_of[k],
+  //     if l >= 0 and ts_start(l) <= ts_start(k).  With both on offer stream order binds iff
+  //     ts_end(q) > ts_start(l) (the comparison of the gap blame); with neither the path
+  //     ends here, unresolved (reason 1).
+  //   START(h), h a host node: to the node u just before h in its lane (program order) -
+  //     END(u) if ts_end(u) <= ts_start(h), else START(u) (h ran inside u); without u the
+  //     path ends at the start of the thread (reason 0).
+  // Time never increases along the walk and strictly decreases on a synchronisation edge, and
+  // every cycle would need one, so the walk ends.  The time between the path's begin and the
+  // sink's end splits into eight classes that add up exactly:
+  //   0 KERNEL, 1 MEMCPY, 2 COLL execution; 3 launch latency (submission edges); 4 delay on a
+  //   stream-order edge (unresolved); 5 inside host API / LAUNCH calls; 6 host time between
+  //   calls; 7 tail of a wait after the device finished (synchronisation edges).
+  void critical_path() {
+    on_path.assign(n, 0);
+    cp_window.clear(); cp_pid.clear(); cp_sink.clear(); cp_n_nodes.clear(); cp_reason.clear();
+    cp_begin.clear(); cp_end.clear(); cp_ns.clear();
+    cp_sum.assign((size_t)W * 10, 0);
+    const int n_lanes = (int)lane_window.size();
+    std::vector<int32_t> lane_of(n, -1);
+    for (int l = 0; l < n_lanes; l++)
+      for (int64_t p = lane_off[l]; p < lane_off[l + 1]; p++) lane_of[p] = l;
+    auto is_host_node = [&](int64_t p) { return kind[p] == API || kind[p] == LAUNCH; };
+    auto is_node = [&](int64_t p) { return kind[p] != OP; };
+    // nodes of each (window, process); device records by (ts_end, position)
+    std::map<std::pair<int32_t, int32_t>, std::vector<int32_t>> nodes;
+    std::map<std::pair<int32_t, int32_t>, std::vector<std::pair<int64_t, int32_t>>> dev_by_end;
+    for (int64_t p = 0; p < n_valid; p++) {
+      if (!is_node(p)) continue;
+      const auto key = std::make_pair(win_sorted[p], pid[p]);
+      nodes[key].push_back((int32_t)p);
+      if (kind[p] >= KERNEL) dev_by_end[key].push_back(std::make_pair(ts_end[p], (int32_t)p));
+    }
+    for (auto& kv : dev_by_end) std::sort(kv.second.begin(), kv.second.end());
+    for (auto& kv : nodes) {
+      const auto& dv = dev_by_end[kv.first];
+      int32_t sink = -1;
+      for (int32_t p : kv.second)
+        if (sink < 0 || ts_end[p] >= ts_end[sink]) sink = p;  // positions ascend: the last equal wins
+      int64_t ns[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+      int32_t n_nodes = 0, reason = 0;
+      int64_t begin = 0;
+      auto visit = [&](int32_t v) { if (!on_path[v]) { on_path[v] = 1; n_nodes++; } };
+      int32_t v = sink;
+      bool at_end = true;
+      for (int64_t guard = 0; guard <= 2 * n_valid + 2; guard++) {
+        visit(v);
+        if (at_end) {
+          if (kind[v] == API) {
+            // the device record that finished last before the call returned
+            auto it = std::lower_bound(dv.begin(), dv.end(), std::make_pair(ts_end[v], (int32_t)-1));
+            if (it != dv.begin()) {
+              const int32_t d = (it - 1)->second;
+              if (ts_end[d] >= ts_start[v]) {
+                ns[7] += ts_end[v] - ts_end[d];
+                v = d;
+                continue;  // at END(d)
+              }
+            }
+          }
+          ns[kind[v] >= KERNEL ? kind[v] - KERNEL : 5] += ts_end[v] - ts_start[v];
+          at_end = false;
+          continue;
+        }
+        if (kind[v] >= KERNEL) {
+          const int32_t q = v > lane_off[lane_of[v]] ? v - 1 : -1;
+          const bool q_ok = q >= 0 && ts_end[q] <= ts_start[v];
+          const int32_t l = (kind[v] == KERNEL || kind[v] == MEMCPY) ? launch_of[v] : -1;
+          const bool l_ok = l >= 0 && ts_start[l] <= ts_start[v];
+          if (q_ok && (!l_ok || ts_end[q] > ts_start[l])) {
+            ns[4] += ts_start[v] - ts_end[q];
+            v = q; at_end = true;
+          } else if (l_ok) {
+            ns[3] += ts_start[v] - ts_start[l];
+            v = l;  // at START(l)
+          } else {
+            begin = ts_start[v]; reason = 1;
+            break;
+          }
+        } else {
+          int32_t u = -1;
+          for (int64_t p = (int64_t)v - 1; p >= lane_off[lane_of[v]]; p--)
+            if (is_host_node(p)) { u = (int32_t)p; break; }
+          if (u < 0) { begin = ts_start[v]; reason = 0; break; }
+          if (ts_end[u] <= ts_start[v]) { ns[6] += ts_start[v] - ts_end[u]; v = u; at_end = true; }
+          else { ns[5] += ts_start[v] - ts_start[u]; v = u; }
+        }
+      }
+      cp_window.push_back(kv.first.first); cp_pid.push_back(kv.first.second);
+      cp_sink.push_back(sink); cp_n_nodes.push_back(n_nodes); cp_reason.push_back(reason);
+      cp_begin.push_back(begin); cp_end.push_back(ts_end[sink]);
+      int64_t* ws = &cp_sum[(size_t)kv.first.first * 10];
+      ws[0]++; ws[1] += n_nodes;
+      for (int c = 0; c < 8; c++) { cp_ns.push_back(ns[c]); ws[2 + c] += ns[c]; }
+    }
+  }
+
   // ---- device-level coverage: from GPU activity, communication hidden by computation is
   // told apart from exposed time; exposed time is interval coverage (Sec. 6.1, "Execution
   // progress and state"; Fig. "Overlap and exposed work": a compute lane, a communication / IO
@@ -634,6 +752,7 @@ void orc_collectives(void* h, const void* sizes, int32_t n_comms) {
 void orc_device_overlap(void* h) { ((Oracle*)h)->device_overlap(); }
 void orc_blame(void* h) { ((Oracle*)h)->blame(); }
 void orc_rollup(void* h) { ((Oracle*)h)->rollup(); }
+void orc_critical_path(void* h) { ((Oracle*)h)->critical_path(); }
 int64_t orc_n_valid(void* h) { return ((Oracle*)h)->n_valid; }
 
 // Exposes a result array by name: pointer into the oracle's storage, element
@@ -655,6 +774,7 @@ int32_t orc_get(void* h, const char* name, const void** ptr, int64_t* count, int
   G(incl_n_kernels) G(incl_first_start) G(incl_last_end) G(incl_kernel_ns)
   G(replay_first_start) G(replay_last_end) G(replay_kernel_ns) G(roll_sum)
   G(b_class) G(b_launch) G(b_win_count) G(b_win_ns) G(op_gap_ns)
+  G(on_path) G(cp_window) G(cp_pid) G(cp_sink) G(cp_n_nodes) G(cp_reason) G(cp_begin) G(cp_end) G(cp_ns) G(cp_sum)
   G(d_window) G(d_pid) G(d_n_events) G(d_busy) G(d_idle) G(d_compute) G(d_comm) G(d_overlap) G(d_exposed)
 #undef G
   return -1;

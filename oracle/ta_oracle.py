@@ -58,6 +58,9 @@ _DTYPES = {
     "d_window": np.int32, "d_pid": np.int32, "d_n_events": np.int64, "d_busy": np.int64,
     "d_idle": np.int64, "d_compute": np.int64, "d_comm": np.int64, "d_overlap": np.int64,
     "d_exposed": np.int64,
+    "on_path": np.uint8, "cp_window": np.int32, "cp_pid": np.int32, "cp_sink": np.int32,
+    "cp_n_nodes": np.int32, "cp_reason": np.int32, "cp_begin": np.int64, "cp_end": np.int64,
+    "cp_ns": np.int64, "cp_sum": np.int64,
 }
 
 _lib = None
@@ -98,6 +101,8 @@ def _load():
         lib.orc_blame.restype = None
         lib.orc_rollup.argtypes = [ctypes.c_void_p]
         lib.orc_rollup.restype = None
+        lib.orc_critical_path.argtypes = [ctypes.c_void_p]
+        lib.orc_critical_path.restype = None
         lib.orc_n_valid.argtypes = [ctypes.c_void_p]
         lib.orc_n_valid.restype = ctypes.c_int64
         lib.orc_get.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_void_p),
@@ -199,6 +204,12 @@ class Oracle:
         """Per (window, process): busy / idle over all device streams, compute and
         communication coverage, their overlap and the exposed communication (needs sort())."""
         self._lib.orc_device_overlap(self._h)
+
+    def critical_path(self):
+        """Per (window, process): the chain of binding submission, stream-order, program-order
+        and synchronisation dependencies that ends at the last record to finish, and the split
+        of its length into eight classes (needs correlate())."""
+        self._lib.orc_critical_path(self._h)
 
     def run_all(self, min_gap_ns: int = 500_000, comm_sizes=()):
         """load, sort, correlate, attribute, gaps, collectives; returns attribute's status."""

@@ -295,3 +295,70 @@ def rollup(sv, n_valid, parent, op_n, op_first, op_last, op_ns, launch_of, kol):
         r = replays.setdefault(l, [s, e, 0])
         r[0], r[1], r[2] = min(r[0], s), max(r[1], e), r[2] + (e - s)
     return incl[0], incl[1], incl[2], incl[3], replays
+
+
+def critical_path(sv, wins, n_valid, launch_of):
+    """The backward walk over START / END points, with every predecessor found by scanning all
+    records for the one the definition names.  Returns {(window, pid): dict(sink, begin, end,
+    reason, nodes (set of positions), ns (eight classes))}."""
+    def slot(p):
+        return (int(wins[p]), int(sv[p]["pid"]))
+
+    def lane(p):
+        return slot(p) + (1 if sv[p]["kind"] >= 3 else 0, int(sv[p]["stream"]))
+
+    S = lambda p: int(sv[p]["ts_start"])
+    E = lambda p: int(sv[p]["ts_end"])
+    K = lambda p: int(sv[p]["kind"])
+    out = {}
+    for key in sorted({slot(p) for p in range(n_valid) if K(p) != 0}):
+        mine = [p for p in range(n_valid) if K(p) != 0 and slot(p) == key]
+        sink = max(mine, key=lambda p: (E(p), p))
+        point = ("END", sink)
+        ns = [0] * 8
+        seen = set()
+        reason = begin = None
+        for _ in range(4 * n_valid + 4):
+            what, v = point
+            seen.add(v)
+            if what == "END":
+                if K(v) == 1:
+                    cands = [d for d in mine if K(d) >= 3 and E(d) < E(v)]
+                    if cands:
+                        d = max(cands, key=lambda d: (E(d), d))
+                        if E(d) >= S(v):
+                            ns[7] += E(v) - E(d)
+                            point = ("END", d)
+                            continue
+                ns[K(v) - 3 if K(v) >= 3 else 5] += E(v) - S(v)
+                point = ("START", v)
+            elif K(v) >= 3:
+                before = [q for q in range(v) if lane(q) == lane(v)]
+                q = before[-1] if before and E(before[-1]) <= S(v) else None
+                l = int(launch_of[v]) if K(v) in (3, 4) else -1
+                if l < 0 or S(l) > S(v):
+                    l = None
+                if q is not None and (l is None or E(q) > S(l)):
+                    ns[4] += S(v) - E(q)
+                    point = ("END", q)
+                elif l is not None:
+                    ns[3] += S(v) - S(l)
+                    point = ("START", l)
+                else:
+                    reason, begin = 1, S(v)
+                    break
+            else:
+                before = [u for u in range(v) if lane(u) == lane(v) and K(u) in (1, 2)]
+                if not before:
+                    reason, begin = 0, S(v)
+                    break
+                u = before[-1]
+                if E(u) <= S(v):
+                    ns[6] += S(v) - E(u)
+                    point = ("END", u)
+                else:
+                    ns[5] += S(v) - S(u)
+                    point = ("START", u)
+        assert reason is not None, "the walk did not end"
+        out[key] = dict(sink=sink, begin=begin, end=E(sink), reason=reason, nodes=seen, ns=ns)
+    return out

@@ -159,4 +159,19 @@ def check_H8(run):
     assert r["roll_sum"][0].tolist() == ints(e["roll_sum"])
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8]
+def check_H9(run):
+    g = load_golden("H9_critical_path.txt")
+    r = run(g["events"], [0, len(g["events"])], [g["t0"]], [g["t1"]])
+    e = g["expect"]
+    assert r["cp_window"].tolist() == [0, 0] and r["cp_pid"].tolist() == ints(e["pids"])
+    assert r["cp_begin"].tolist() == ints(e["begin"]) and r["cp_end"].tolist() == ints(e["end"])
+    assert r["cp_reason"].tolist() == ints(e["reason"]) and r["cp_n_nodes"].tolist() == ints(e["n_nodes"])
+    want = [[int(x) for x in t.split(":")] for t in e["ns"]]
+    assert r["cp_ns"].reshape(-1, 8).tolist() == want
+    on = np.nonzero(r["on_path"])[0]
+    assert r["ts_start"][on].tolist() == ints(e["on_path"])
+    assert r["ts_start"][r["cp_sink"]].tolist() == ints(e["sinks"])
+    assert r["cp_sum"].reshape(-1, 10)[0].tolist() == [2, 10] + [a + b for a, b in zip(*want)]
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9]

@@ -20,6 +20,9 @@ BLAME_KEYS = ["b_class", "b_launch", "b_win_count", "b_win_ns", "op_gap_ns"]
 OVERLAP_KEYS = ["d_window", "d_pid", "d_n_events", "d_busy", "d_idle", "d_compute", "d_comm",
                 "d_overlap", "d_exposed"]
 
+CRITPATH_KEYS = ["on_path", "cp_window", "cp_pid", "cp_sink", "cp_n_nodes", "cp_reason", "cp_begin",
+                 "cp_end", "cp_ns", "cp_sum"]
+
 DEVICE_MASK = (1 << 3) | (1 << 4) | (1 << 5)
 OP_MASK = 1
 
@@ -64,6 +67,9 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
         r[f"aggG_{k}"] = o.get(k)
     o.device_overlap()
     for k in OVERLAP_KEYS:
+        r[k] = o.get(k)
+    o.critical_path()
+    for k in CRITPATH_KEYS:
         r[k] = o.get(k)
     o.close()
     return r

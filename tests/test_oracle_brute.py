@@ -5,7 +5,7 @@ import pytest
 
 import brute
 from runners import DEVICE_MASK, run_oracle
-from tiny import random_window
+from tiny import random_window, schedule_window
 
 SEEDS = list(range(12))
 
@@ -332,3 +332,69 @@ def test_rollup_against_parent_chains(seed):
     # roots of the forest hold everything that was attributed below them
     roots = (sv["kind"][:r["n_valid"]] == 0) & (r["parent"][:r["n_valid"]] < 0)
     assert int(r["incl_n_kernels"][:r["n_valid"]][roots].sum()) == int(r["attr_sum"]["n_attributed"].sum())
+
+
+def _critical_path_matches_brute(ev, off, t0, t1, sizes=()):
+    r = run_oracle(ev, off, t0, t1, min_gap=5, comm_sizes=sizes)
+    sv = _sorted_view(ev, r)
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    want = brute.critical_path(sv, wins, r["n_valid"], r["launch_of"])
+    keys = list(zip(r["cp_window"].tolist(), r["cp_pid"].tolist()))
+    assert keys == list(want)
+    on = np.zeros(len(sv), dtype=np.uint8)
+    tot = np.zeros((len(t0), 10), dtype=np.int64)
+    for i, key in enumerate(keys):
+        b = want[key]
+        assert int(r["cp_sink"][i]) == b["sink"] and int(r["cp_reason"][i]) == b["reason"]
+        assert int(r["cp_begin"][i]) == b["begin"] and int(r["cp_end"][i]) == b["end"]
+        assert int(r["cp_n_nodes"][i]) == len(b["nodes"])
+        assert r["cp_ns"].reshape(-1, 8)[i].tolist() == b["ns"]
+        assert sum(b["ns"]) == b["end"] - b["begin"]  # the classes telescope
+        on[list(b["nodes"])] = 1
+        tot[key[0], 0] += 1
+        tot[key[0], 1] += len(b["nodes"])
+        tot[key[0], 2:] += b["ns"]
+    assert np.array_equal(r["on_path"], on)
+    assert np.array_equal(r["cp_sum"].reshape(-1, 10), tot)
+    return r, want
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_critical_path_against_point_walk_random(seed):
+    ev, off, t0, t1, sizes = random_window(seed)
+    _critical_path_matches_brute(ev, off, t0, t1, sizes)
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_critical_path_against_point_walk_schedules(seed):
+    ev, off, t0, t1, _ = schedule_window(seed)
+    r, want = _critical_path_matches_brute(ev, off, t0, t1)
+    ns = r["cp_ns"].reshape(-1, 8).sum(0)
+    assert ns[7] > 0 and ns[3] > 0 and ns[6] > 0  # waits, submission edges and host time all occur
+
+
+@pytest.mark.parametrize("seed", SEEDS)
+def test_critical_path_of_a_tight_schedule_is_the_longest_path(seed):
+    """In a schedule without slack (a kernel starts the moment its launch call starts or its
+    stream frees up, a wait returns a fixed time after the last kernel) the chain of binding
+    dependencies is a longest path of the full dependency graph: it reaches the first call of the
+    thread, spans the makespan, and holds neither launch latency nor stream delay."""
+    ev, off, t0, t1, info = schedule_window(seed, tight=True)
+    r = run_oracle(ev, off, t0, t1)
+    for i, pid in enumerate(r["cp_pid"].tolist()):
+        g = info[pid]
+        # longest path over ALL dependencies: relax every edge until nothing changes
+        dist = {g["source"]: 0}
+        changed = True
+        while changed:
+            changed = False
+            for a, b, w in g["edges"]:
+                if a in dist and dist[a] + w > dist.get(b, -1):
+                    dist[b] = dist[a] + w
+                    changed = True
+        longest = max(dist.values())
+        assert longest == g["makespan"]
+        ns = r["cp_ns"].reshape(-1, 8)[i]
+        assert int(r["cp_reason"][i]) == 0 and int(r["cp_begin"][i]) == g["first"]
+        assert int(r["cp_end"][i]) - int(r["cp_begin"][i]) == longest == int(ns.sum())
+        assert ns[3] == 0 and ns[4] == 0
