@@ -457,6 +457,71 @@ ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result
 void ta_free(ta_window *h);
 
 /* ------------------------------------------------------------------------
+ * ta_critical_path - per (window, process), the chain of binding dependencies
+ * that ends at the last record to finish.  Submission, execution-order and
+ * synchronisation dependencies identify the critical path; where a dependency
+ * is missing, the delay it would explain stays unresolved (Sec. 6.1, "Execution
+ * progress and state"; Fig. "Critical path": host work, the call that submits
+ * k1, k1, the end of the host's wait, host work again - a kernel of another
+ * stream and the wait itself stay off the path).  Beyond the seven calls above.
+ * Needs ta_correlate_launches.
+ *
+ * Readings.  Nodes are the valid API and LAUNCH records (host) and the KERNEL,
+ * MEMCPY and COLL records (device); OP records are context, not nodes.  A node
+ * has a START point (ts_start) and an END point (ts_end).  The walk starts at the
+ * END of the sink - the node of the (window, process) with the greatest ts_end,
+ * the highest sorted position among equals - and always steps back to the
+ * dependency that was released last:
+ *   END(v), v an API record that waited: to END(d), d = the device record of the
+ *     process with the greatest ts_end < ts_end(v) (highest position among
+ *     equals); v waited iff ts_end(d) >= ts_start(v).        [synchronisation]
+ *   END(v) otherwise: to START(v).                            [v ran]
+ *   START(k), k a device record: stream order offers END(q), q the record just
+ *     before k in its lane, if ts_end(q) <= ts_start(k); submission offers
+ *     START(l), l = launch_of[k], if l >= 0 and ts_start(l) <= ts_start(k).  With
+ *     both on offer stream order binds iff ts_end(q) > ts_start(l) (the test of
+ *     ta_blame_gaps); with neither the path ends here, unresolved (reason 1).
+ *   START(h), h a host node: to the node u just before h in its lane (program
+ *     order): END(u) if ts_end(u) <= ts_start(h), else START(u) (h ran inside u);
+ *     without u the path ends at the start of the thread (reason 0).
+ * Time never increases along the walk and strictly decreases on a
+ * synchronisation edge, which every cycle would need, so the walk ends.
+ * The time between the path's begin and the sink's end splits into eight
+ * classes that add up exactly (p_ns, TA_CP_*): execution of KERNEL, MEMCPY and
+ * COLL records on the path; launch latency (ts_start(k) - ts_start(l) on
+ * submission edges); delay on stream-order edges (unresolved); time inside host
+ * calls; host time between calls; the tail of a wait after the device finished
+ * (ts_end(v) - ts_end(d) on synchronisation edges - the wait itself is context,
+ * not another copy of the device's time).
+ *
+ * Outputs (device memory owned by the handle): on_path[n], 1 for every node the
+ * walk passes through; one row per (window, process) that has a node, ordered by
+ * (window, pid): p_sink (sorted position), p_begin / p_end (time where the walk
+ * ended / ts_end of the sink), p_n_nodes, p_reason, p_ns[row * 8 + class].
+ * out_summary[w]: rows, nodes and class totals of window w.
+ * Limits: window span and the longest record < 2^40 ns each, windows x pids <
+ * 2^22, at most 2^22 changes of lane on one path (TA_ERR_TOO_LARGE).
+ * Errors: TA_ERR_ORDER before ta_correlate_launches; TA_ERR_OOM; TA_ERR_CUDA;
+ * TA_ERR_TIMEOUT.  One stream synchronisation at the end. */
+enum {
+  TA_CP_KERNEL = 0, TA_CP_MEMCPY = 1, TA_CP_COLL = 2, TA_CP_LAUNCH_LATENCY = 3,
+  TA_CP_STREAM_DELAY = 4, TA_CP_IN_CALL = 5, TA_CP_BETWEEN_CALLS = 6, TA_CP_WAIT_TAIL = 7
+};
+typedef struct ta_critpath_summary {
+  int64_t n_paths, n_nodes, ns[8];
+} ta_critpath_summary;
+
+typedef struct ta_critpath_result {
+  int64_t n_rows;
+  const uint8_t *on_path;
+  const int32_t *p_window, *p_pid, *p_sink, *p_n_nodes, *p_reason;
+  const int64_t *p_begin, *p_end, *p_ns;
+} ta_critpath_result;
+
+ta_status ta_critical_path(ta_window *h, ta_critpath_result *out,
+                           ta_critpath_summary *out_summary /* host, n_windows entries */);
+
+/* ------------------------------------------------------------------------
  * ta_lane_gaps_noalloc - the stream-gap scan of ONE device lane, for callers
  * that cannot allocate device memory.  (The paper has no counterpart for this
  * entry point; it exists for integration reasons only.)

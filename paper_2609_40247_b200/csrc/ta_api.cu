@@ -339,6 +339,16 @@ ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result
   return ta_run_blame(h, gaps, out, out_summary);
 }
 
+ta_status ta_critical_path(ta_window *h, ta_critpath_result *out, ta_critpath_summary *out_summary) {
+  if (!h || !out || !out_summary) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 4)) return TA_ERR_ORDER;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
+  return ta_run_critpath(h, out, out_summary);
+}
+
 ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;

@@ -178,6 +178,9 @@ ta_status ta_run_rollup(ta_window *h, ta_rollup_result *out, ta_rollup_summary *
 ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
                        ta_blame_summary *out_summary);
 
+// critpath.cu
+ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_summary *out_summary);
+
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 
 // ---- instrumentation (no work: a launch counter and optional event pairs) ----

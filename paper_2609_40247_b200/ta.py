@@ -91,11 +91,15 @@ _OverlapResult = _ptr_struct("_OverlapResult", [
     ("d_busy", _vp), ("d_idle", _vp), ("d_compute", _vp), ("d_comm", _vp), ("d_overlap", _vp),
     ("d_exposed", _vp)])
 
+_CritpathResult = _ptr_struct("_CritpathResult", [
+    ("n_rows", ctypes.c_int64), ("on_path", _vp), ("p_window", _vp), ("p_pid", _vp), ("p_sink", _vp),
+    ("p_n_nodes", _vp), ("p_reason", _vp), ("p_begin", _vp), ("p_end", _vp), ("p_ns", _vp)])
+
 EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_attribute_operators",
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
            "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps",
-           "ta_rollup_operators"]
+           "ta_rollup_operators", "ta_critical_path"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -134,6 +138,8 @@ def lib():
         L.ta_match_collectives.argtypes = [_vp, _vp, ctypes.c_int32, ctypes.POINTER(_CollResult)]
         L.ta_rollup_operators.restype = ctypes.c_int
         L.ta_rollup_operators.argtypes = [_vp, ctypes.POINTER(_RollupResult), _vp]
+        L.ta_critical_path.restype = ctypes.c_int
+        L.ta_critical_path.argtypes = [_vp, ctypes.POINTER(_CritpathResult), _vp]
         L.ta_blame_gaps.restype = ctypes.c_int
         L.ta_blame_gaps.argtypes = [_vp, _vp, ctypes.POINTER(_BlameResult), _vp]
         L.ta_device_overlap.restype = ctypes.c_int
@@ -339,6 +345,32 @@ class RollupResult(_Result):
         return super().numpy(name)
 
 
+CRITPATH_SUM = np.dtype([("n_paths", "<i8"), ("n_nodes", "<i8"), ("ns", "<i8", (8,))])
+
+
+class CritpathResult(_Result):
+    """on_path per sorted position; one row per (window, process): cp_window, cp_pid, cp_sink,
+    cp_n_nodes, cp_reason, cp_begin, cp_end, cp_ns[row][8]; cp_sum[window][10] = paths, nodes and
+    the eight class totals."""
+    _names = {"cp_window": "p_window", "cp_pid": "p_pid", "cp_sink": "p_sink", "cp_n_nodes": "p_n_nodes",
+              "cp_reason": "p_reason", "cp_begin": "p_begin", "cp_end": "p_end", "cp_ns": "p_ns"}
+    _layout = dict([("on_path", ("u1", lambda r: r.n))] +
+                   [(k, ("<i4", lambda r: r.n_rows)) for k in
+                    ("p_window", "p_pid", "p_sink", "p_n_nodes", "p_reason")] +
+                   [("p_begin", ("<i8", lambda r: r.n_rows)), ("p_end", ("<i8", lambda r: r.n_rows)),
+                    ("p_ns", ("<i8", lambda r: r.n_rows * 8))])
+
+    def numpy(self, name):
+        if name == "cp_sum":
+            s = self.critpath_sum
+            return np.concatenate([s["n_paths"][:, None], s["n_nodes"][:, None], s["ns"]],
+                                  axis=1).astype(np.int64).reshape(-1)
+        return super().numpy(self._names.get(name, name))
+
+    def tensor(self, name):
+        return super().tensor(self._names.get(name, name))
+
+
 BLAME_SUM = np.dtype([("count", "<i8", (4,)), ("ns", "<i8", (4,))])
 
 
@@ -500,6 +532,14 @@ class Window:
         if st != 0:
             raise TaError(st, "ta_rollup_operators")
         return RollupResult(self, raw, dict(self._dims(), rollup_sum=summ))
+
+    def critical_path(self) -> CritpathResult:
+        raw = _CritpathResult()
+        summ = np.zeros(self.W, dtype=CRITPATH_SUM)
+        st = self._lib.ta_critical_path(self._h, ctypes.byref(raw), summ.ctypes.data)
+        if st != 0:
+            raise TaError(st, "ta_critical_path")
+        return CritpathResult(self, raw, dict(self._dims(), n_rows=raw.n_rows, critpath_sum=summ))
 
     def blame_gaps(self, gaps) -> BlameResult:
         """gaps: the GapResult of an earlier stream_gaps() call on this window."""

@@ -125,6 +125,9 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
         d = w.device_overlap()
         for k in OVERLAP_KEYS:
             r[k] = d.numpy(k)
+        cp = w.critical_path()
+        for k in CRITPATH_KEYS:
+            r[k] = cp.numpy(k)
     return r
 
 

@@ -9,7 +9,7 @@ from helpers import make_events
 from paper_2609_40247_b200 import synth
 from runners import DEVICE_MASK, assert_same, run_gpu, run_oracle
 from test_oracle_truth import check_against_truth
-from tiny import random_window
+from tiny import random_window, schedule_window
 
 pytestmark = pytest.mark.gpu
 
@@ -45,6 +45,15 @@ def test_tiny_adversarial_windows(seed):
 def test_tiny_windows_with_partial_overlap(seed):
     ev, off, t0, t1, sizes = random_window(100 + seed, nested=False, defects=False)
     both(ev, off, t0, t1, min_gap=3, comm_sizes=sizes)
+
+
+@pytest.mark.parametrize("seed,tight", [(s, t) for s in range(6) for t in (False, True)])
+def test_simulated_schedules(seed, tight):
+    """Launches, kernels in stream order and waits of a simulated run: every kind of edge of the
+    critical path occurs (submission, stream order, program order, synchronisation)."""
+    ev, off, t0, t1, _ = schedule_window(seed, tight=tight, n_actions=300, n_streams=3, n_pid=3)
+    o, g = both(ev, off, t0, t1, min_gap=20)
+    assert int(o["cp_ns"].reshape(-1, 8)[:, 7].sum()) > 0
 
 
 def test_larger_random_window_spans_tiles():
