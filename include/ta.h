@@ -500,9 +500,9 @@ void ta_free(ta_window *h);
  * ended / ts_end of the sink), p_n_nodes, p_reason, p_ns[row * 8 + class].
  * out_summary[w]: rows, nodes and class totals of window w.
  * Limits: window span and the longest record < 2^40 ns each, windows x pids <
- * 2^22, at most 2^22 changes of lane on one path (TA_ERR_TOO_LARGE).
+ * 2^22 (TA_ERR_TOO_LARGE).
  * Errors: TA_ERR_ORDER before ta_correlate_launches; TA_ERR_OOM; TA_ERR_CUDA;
- * TA_ERR_TIMEOUT.  One stream synchronisation at the end. */
+ * TA_ERR_TIMEOUT.  Two stream synchronisations. */
 enum {
   TA_CP_KERNEL = 0, TA_CP_MEMCPY = 1, TA_CP_COLL = 2, TA_CP_LAUNCH_LATENCY = 3,
   TA_CP_STREAM_DELAY = 4, TA_CP_IN_CALL = 5, TA_CP_BETWEEN_CALLS = 6, TA_CP_WAIT_TAIL = 7

@@ -24,14 +24,19 @@
 //                  each host node, then the head of every run (device: last record whose
 //                  binding edge leaves the lane; host: last wait that was released by the
 //                  device and is entered from its END);
-//   k_cp_walk      one thread per slot hops run to run: device run -> launch of its head ->
-//                  host run -> the wait at its head -> the device record that released it;
-//                  it only records where each run was entered;
+//                  the waits that head a host run go to a list (they are few);
+//   k_cp_succ      per listed wait, the next wait down the path: wait -> the record that
+//                  released it -> head of that device run -> its launch -> head of that host run;
+//   k_cp_start     one thread per slot: the sink, and the hops from it to the first listed wait;
+//   k_cp_double    pointer doubling over the list: a wait reached from a marked wait is marked,
+//                  successors are squared; after log2(list) rounds exactly the waits on a path
+//                  are marked, whatever the length of the chain;
+//   k_cp_enter     every marked wait records where the walk enters the two runs that follow it;
 //   k_cp_mark      every record decides from its run's entry whether it is on the path and
 //                  adds its share of the eight time classes (folded per warp);
 //   a scan         compacts the slots that have a path into rows.
 // HBM traffic: the sort (8 B + 8 B per device record and pass) and three passes over the
-// columns; the walk is latency bound (a few dependent loads per wait on the path).
+// columns; the chain of lane changes costs a few short kernels over the list of waits.
 #include <climits>
 #include <cstring>
 #include <vector>
@@ -71,9 +76,14 @@ struct CpArgs {
   int32_t *slot_host_pos;  // per slot: highest position among the host nodes that end then
   u64 *st_a, *st_b;     // tile descriptors of the two scans
   u32 *counter;
+  u32 *n_eff;           // length of the list below
+  u32 *eff_pos;         // positions of the waits that head a host run, in no particular order
+  int32_t *id_of;       // [position] index in that list, or -1
+  int32_t *jump_in, *jump_out;  // per listed wait: the wait 2^round steps down the path, or -1
+  uint8_t *mark;        // per listed wait: on a path
+  int64_t n_list;
   u64 *acc;             // [slot][CP_ACC]
   uint8_t *on_path;
-  int64_t hop_cap;
   int32_t *status;
 };
 
@@ -207,10 +217,20 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_classify(CpArgs a) {
       }
     }
   }
-  if (run_slot >= 0) atomicMax(&a.slot_host_te[run_slot], run_max);
   if (p0 + CP_ITEMS <= a.n) *reinterpret_cast<u64 *>(a.link + p0) = links;
   else
     for (int j = 0; j < CP_ITEMS && p0 + j < a.n; j++) a.link[p0 + j] = (uint8_t)(links >> (8 * j));
+  // the thread's last slot: one atomic per warp when the whole warp is here and sits in that slot
+  const u32 act = __activemask();
+  const u32 has = __ballot_sync(act, run_slot >= 0);
+  if (!has) return;
+  const int s0 = __shfl_sync(act, run_slot, __ffs(has) - 1);
+  if (act == 0xffffffffu && __all_sync(act, run_slot < 0 || run_slot == s0)) {
+    const u64 v = warp_reduce(run_slot >= 0 ? run_max : 0ull, OpMax());
+    if ((threadIdx.x & 31) == 0) atomicMax(&a.slot_host_te[s0], v);
+  } else if (run_slot >= 0) {
+    atomicMax(&a.slot_host_te[run_slot], run_max);
+  }
 }
 
 // ---- runs: previous host node, then run heads ------------------------------------------
@@ -292,7 +312,12 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
     } else if (prev[j] >= 0) {
       const int32_t u = prev[j];
       // a wait that the device released, entered from its END (it ended before this node began)
-      if (a.kind[u] == TA_KIND_API && a.cross[u] >= 0 && a.te[u] <= s[j]) cand[j] = (u64)(u + 1);
+      if (a.kind[u] == TA_KIND_API && a.cross[u] >= 0 && a.te[u] <= s[j]) {
+        cand[j] = (u64)(u + 1);
+        const u32 id = atomicAdd(a.n_eff, 1u);  // each such wait is found once, by the node after it
+        a.eff_pos[id] = (u32)u;
+        a.id_of[u] = (int32_t)id;
+      }
     }
     run = max(run, cand[j]);
   }
@@ -319,8 +344,33 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
   store8_i32(a.head, p0, a.n, hd);
 }
 
-// ---- the walk: one thread per (window, process) ------------------------------------------
-__global__ void __launch_bounds__(64) k_cp_walk(CpArgs a) {
+// ---- the chain of lane changes ---------------------------------------------------------------
+// From the END of device record d: records where the walk enters d's run and, if the head of
+// that run was bound by its submission, the host run of its launch.  Returns the list index of
+// the wait that heads that host run, or -1 when the path ends first.
+__device__ __forceinline__ int32_t cp_follow(const CpArgs &a, int32_t d, bool record) {
+  const int32_t h = a.head[d];
+  if (h < 0) return -1;  // cannot happen: the first record of a device lane always heads a run
+  if (record) a.entry[h] = d;
+  if (a.link[h] != CP_LINK_SUBMIT) return -1;  // unresolved: the head records where the path begins
+  const int32_t l = a.launch_of[h];
+  const int32_t e = a.head[l];
+  if (e < 0) {
+    if (record) a.entry_lane[lane_of_pos(a.lane_off, a.n_lanes, l)] = l;
+    return -1;
+  }
+  if (record) a.entry[e] = l;
+  return a.id_of[e];
+}
+
+__global__ void __launch_bounds__(256) k_cp_succ(CpArgs a) {
+  const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= a.n_list) return;
+  a.jump_in[id] = cp_follow(a, a.cross[a.eff_pos[id]], false);
+}
+
+// one thread per (window, process): the sink and the hops from it to the first listed wait
+__global__ void __launch_bounds__(64) k_cp_start(CpArgs a) {
   const int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (slot >= a.n_slots) return;
   const int sh = a.tsbits + a.idxbits;
@@ -343,49 +393,46 @@ __global__ void __launch_bounds__(64) k_cp_walk(CpArgs a) {
   u64 *acc = a.acc + (size_t)slot * CP_ACC;
   acc[11] = (u64)(sink + 1);
 
-  int32_t v = sink;
-  bool on_device = cp_device(a.kind[sink]);
-  if (!on_device) {
+  int32_t first = -1;  // list index of the first wait on the path
+  if (cp_device(a.kind[sink])) {
+    first = cp_follow(a, sink, true);
+  } else {
     const int32_t d = a.kind[sink] == TA_KIND_API ? a.cross[sink] : -1;
     if (d >= 0) {  // the sink is a wait: its tail is on the path, then the record that released it
       atomicAdd(&acc[8], (u64)(a.te[sink] - a.te[d]));
       a.entry[sink] = sink;
-      v = d;
-      on_device = true;
-    } else {
+      first = cp_follow(a, d, true);
+    } else {       // the sink ran: the walk enters its host run at its START
       atomicAdd(&acc[6], (u64)(a.te[sink] - a.ts[sink]));
+      const int32_t e = a.head[sink];
+      if (e < 0) a.entry_lane[lane_of_pos(a.lane_off, a.n_lanes, sink)] = sink;
+      else {
+        a.entry[e] = sink;
+        first = a.id_of[e];
+      }
     }
   }
-  for (int64_t hop = 0;; hop++) {
-    if (hop > a.hop_cap) {
-      ta_set_err(a.status, TA_ERR_TOO_LARGE);
-      return;
-    }
-    if (on_device) {
-      const int32_t h = a.head[v];
-      if (h < 0) {  // cannot happen: the first record of a device lane always heads a run
-        ta_set_err(a.status, TA_ERR_OVERFLOW);
-        return;
-      }
-      a.entry[h] = v;
-      if (a.link[h] != CP_LINK_SUBMIT) return;  // unresolved: the head itself records where the path begins
-      v = a.launch_of[h];
-      on_device = false;
-    } else {
-      const int32_t e = a.head[v];
-      if (e < 0) {
-        a.entry_lane[lane_of_pos(a.lane_off, a.n_lanes, v)] = v;
-        return;
-      }
-      a.entry[e] = v;
-      v = a.cross[e];
-      if (v < 0) {  // cannot happen: only waits with a releasing record head a host run
-        ta_set_err(a.status, TA_ERR_OVERFLOW);
-        return;
-      }
-      on_device = true;
-    }
+  if (first >= 0) a.mark[first] = 1;
+}
+
+// one round: what a marked wait reaches is marked (a wait marked during the round may pass its
+// mark on at once - everything it reaches is on the path as well), successors are squared
+__global__ void __launch_bounds__(256) k_cp_double(CpArgs a) {
+  const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= a.n_list) return;
+  const int32_t j = a.jump_in[id];
+  if (j < 0) {
+    a.jump_out[id] = -1;
+    return;
   }
+  if (a.mark[id]) a.mark[j] = 1;
+  a.jump_out[id] = a.jump_in[j];
+}
+
+__global__ void __launch_bounds__(256) k_cp_enter(CpArgs a) {
+  const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= a.n_list || !a.mark[id]) return;
+  cp_follow(a, a.cross[a.eff_pos[id]], true);
 }
 
 // ---- membership and time classes ---------------------------------------------------------
@@ -559,7 +606,7 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   const int64_t tiles = (h->n_valid + CP_TILE - 1) / CP_TILE;
   const int64_t mm = m > 0 ? m : 1;
   size_t tb = 3 * Carver::pad((size_t)mm * 8) + 3 * Carver::pad((size_t)mm * 4) + ta_sort_temp_bytes(mm) +
-              Carver::pad((size_t)nn) + 4 * Carver::pad((size_t)nn * 4) + Carver::pad((size_t)(n_lanes + 1) * 4) +
+              Carver::pad((size_t)nn) + 6 * Carver::pad((size_t)nn * 4) + Carver::pad((size_t)(n_lanes + 1) * 4) +
               2 * Carver::pad((size_t)tiles * 8) + Carver::pad(64) + Carver::pad((size_t)n_slots * 8) +
               Carver::pad((size_t)n_slots * 4) + Carver::pad((size_t)n_slots * CP_ACC * 8) +
               scan_temp_bytes(n_slots) + 1024;
@@ -574,16 +621,19 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   a.cross = ct.take<int32_t>(nn);
   a.prev_node = ct.take<int32_t>(nn);
   a.head = ct.take<int32_t>(nn);
+  a.eff_pos = ct.take<u32>(nn);
   // zeroed block
   char *zb = ct.base + ct.off;
   a.st_a = ct.take<u64>(tiles); a.st_b = ct.take<u64>(tiles);
   a.counter = (u32 *)ct.take<u64>(8);
+  a.n_eff = a.counter + 2;
   a.slot_host_te = ct.take<u64>(n_slots);
   a.acc = ct.take<u64>(n_slots * CP_ACC);
   TA_CHECK_CUDA(h, cudaMemsetAsync(zb, 0, (ct.base + ct.off) - zb, st));
   // block filled with -1
   char *fb = ct.base + ct.off;
   a.entry = ct.take<int32_t>(nn);
+  a.id_of = ct.take<int32_t>(nn);
   a.entry_lane = ct.take<int32_t>(n_lanes + 1);
   a.slot_host_pos = ct.take<int32_t>(n_slots);
   TA_CHECK_CUDA(h, cudaMemsetAsync(fb, 0xff, (ct.base + ct.off) - fb, st));
@@ -599,7 +649,6 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   a.tsbits = tsbits; a.idxbits = idxbits;
   a.keys = k_in; a.pos = v_in;
   a.on_path = on_path; a.status = h->d_status;
-  a.hop_cap = h->n_valid + 2 < (1ll << 22) ? h->n_valid + 2 : (1ll << 22);
 
   if (m > 0) {
     k_cp_keys<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
@@ -617,7 +666,30 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   a.skeys = k_fin;
   k_cp_classify<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
   k_cp_runs<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
-  k_cp_walk<<<TA_N (unsigned)((n_slots + 63) / 64), 64, 0, st>>>(a);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  // the waits that head a host run: a list whose length decides the number of doubling rounds
+  u32 n_list = 0;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_list, a.n_eff, 4, cudaMemcpyDeviceToHost, st));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  a.n_list = (int64_t)n_list;
+  const int64_t nl = n_list > 0 ? n_list : 1;
+  void *lb = ta_dalloc(h, 2 * Carver::pad((size_t)nl * 4) + Carver::pad((size_t)nl) + 256);
+  if (!lb) return TA_ERR_OOM;
+  Carver cl(lb);
+  a.jump_in = cl.take<int32_t>(nl);
+  a.jump_out = cl.take<int32_t>(nl);
+  a.mark = cl.take<uint8_t>(nl);
+  TA_CHECK_CUDA(h, cudaMemsetAsync(a.mark, 0, (size_t)nl, st));
+  const unsigned lblocks = (unsigned)((nl + 255) / 256);
+  if (n_list) k_cp_succ<<<TA_N lblocks, 256, 0, st>>>(a);
+  k_cp_start<<<TA_N (unsigned)((n_slots + 63) / 64), 64, 0, st>>>(a);
+  if (n_list) {
+    for (int r = ta_bit_len((uint64_t)n_list); r > 0; r--) {
+      k_cp_double<<<TA_N lblocks, 256, 0, st>>>(a);
+      int32_t *t = a.jump_in; a.jump_in = a.jump_out; a.jump_out = t;
+    }
+    k_cp_enter<<<TA_N lblocks, 256, 0, st>>>(a);
+  }
   k_cp_mark<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
 
@@ -632,6 +704,7 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   TA_CHECK_CUDA(h, cudaMemcpyAsync(hacc.data(), a.acc, hacc.size() * 8, cudaMemcpyDeviceToHost, st));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
+  ta_dfree(h, lb);
   ta_dfree(h, tmpb);
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
   for (int64_t s = 0; s < n_slots; s++) {

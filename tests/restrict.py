@@ -12,8 +12,8 @@ host, where they are compared with the oracle run on the subset.
 import numpy as np
 
 from paper_2609_40247_b200.ta import NBINS
-from runners import (AGG_KEYS, ATTR_KEYS, BLAME_KEYS, COLL_KEYS, DEVICE_MASK, GAP_KEYS, JOIN_KEYS,
-                     OP_MASK, OVERLAP_KEYS, ROLLUP_KEYS)
+from runners import (AGG_KEYS, ATTR_KEYS, BLAME_KEYS, COLL_KEYS, CRITPATH_KEYS, DEVICE_MASK, GAP_KEYS,
+                     JOIN_KEYS, OP_MASK, OVERLAP_KEYS, ROLLUP_KEYS)
 
 _POSITIONAL = {"launch_of", "parent", "op_of"}  # values are sorted positions (or -1)
 _PER_RECORD_SORT = ["ts_start", "ts_end", "corr_id", "pid", "name_id", "seq", "stream", "kind"]
@@ -70,10 +70,11 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
         ru = w.rollup_operators() if a.status == 0 else None
         bl = w.blame_gaps(g)
         ag_gap = w.aggregate_ops(OP_MASK, 2)
+        cp = w.critical_path()
         del buf
         if checks is not None:
             checks(dict(window=w, sort=s, join=j, attr=a, gaps=g, agg_dev=ag_dev, agg_op=ag_op,
-                        coll=c, overlap=ov, blame=bl))
+                        coll=c, overlap=ov, blame=bl, critpath=cp))
         n, n_valid = s.n, s.n_valid
         perm = _typed(s, "perm")[0].long()
         lane_off = _typed(s, "lane_off")[0].long()
@@ -216,6 +217,24 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
                     if k == "d_window":
                         v = wmap[v.long()]
                     r[k] = _host(v, dt)
+            if "critpath" in sub.groups:
+                r["on_path"] = per_record(cp, "on_path")
+                rows = wmap[_typed(cp, "cp_window")[0].long()] >= 0
+                if sub.pid is not None:
+                    rows &= _typed(cp, "cp_pid")[0] == sub.pid
+                for k in CRITPATH_KEYS[1:-1]:
+                    t, dt = _typed(cp, k)
+                    if k == "cp_ns":
+                        r[k] = _host(t.reshape(-1, 8)[rows].reshape(-1), dt)
+                        continue
+                    v = t[rows]
+                    if k == "cp_window":
+                        v = wmap[v.long()]
+                    elif k == "cp_sink":
+                        v = pos_map[v.long()]
+                    r[k] = _host(v, dt)
+                if sub.windows is not None:
+                    r["cp_sum"] = cp.numpy("cp_sum").reshape(-1, 10)[wkeep].reshape(-1)
             out[sub.name] = r
             del sel, pos_sel, pos_idx, pos_map, inv, csum
     return out

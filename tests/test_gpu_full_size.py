@@ -65,6 +65,16 @@ def _properties(t0, t1, full):
     assert np.array_equal(ov["d_busy"], ov["d_compute"] + ov["d_comm"] - ov["d_overlap"])
     assert (ov["d_overlap"] >= 0).all() and (ov["d_exposed"] >= 0).all()
     assert int(ov["d_n_events"].sum()) == int((kind[:nv] >= 3).sum())
+    # critical paths: the classes telescope, the flags count the nodes, every sink is on its path
+    cp = full["critpath"]
+    ns = cp.numpy("cp_ns").reshape(-1, 8)
+    assert np.array_equal(ns.sum(1), cp.numpy("cp_end") - cp.numpy("cp_begin")) and (ns >= 0).all()
+    on = _typed(cp, "on_path")[0]
+    assert int(on.sum()) == int(cp.numpy("cp_n_nodes").sum())
+    assert bool((on[torch.from_numpy(cp.numpy("cp_sink")).long().to(on.device)] == 1).all())
+    assert bool((kind[:nv][on[:nv] == 1] > 0).all()) and int(on[nv:].sum()) == 0
+    csum = cp.numpy("cp_sum").reshape(-1, 10)
+    assert int(csum[:, 0].sum()) == len(ns) and np.array_equal(csum[:, 2:].sum(0), ns.sum(0))
     # aggregates count every kept device record once
     n_dev = int((kind[:nv] >= 3).sum())
     assert int(full["agg_dev"].numpy("g_count").sum()) == n_dev
@@ -90,7 +100,7 @@ def test_c3_full_size_one_process_and_collectives():
     ev = wl.events
     assert len(ev) > 2**25
     pids = np.unique(ev["pid"])
-    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap", "blame", "rollup")
+    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap", "blame", "rollup", "critpath")
     subsets = [Subset(f"pid{p}", ev["pid"] == p, per_pid, pid=int(p)) for p in (pids[0], pids[-1])]
     subsets.append(Subset("coll", ev["kind"] == 5, ("sort", "coll")))
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
@@ -109,7 +119,7 @@ def test_c4_full_size_whole_windows():
     sel = np.zeros(len(ev), dtype=bool)
     for w in keep:
         sel[off[w]:off[w + 1]] = True
-    every = ("sort", "join", "attr", "gaps", "agg", "coll", "overlap", "blame", "rollup")
+    every = ("sort", "join", "attr", "gaps", "agg", "coll", "overlap", "blame", "rollup", "critpath")
     subsets = [Subset("windows", sel, every, windows=keep)]
     r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
                            comm_sizes=wl.comm_sizes,
