@@ -148,6 +148,8 @@ def run_pipeline(ta, buf, wl, read_back=False, per_call=None):
             mark("blame_gaps + aggregate_ops(OP, idle charged) (outside the timed step)")
             w.rollup_operators()
             mark("rollup_operators (outside the timed step)")
+            w.critical_path()
+            mark("critical_path (outside the timed step)")
         nbytes = w.load_summary.nbytes + j.join_sum.nbytes + a.attr_sum.nbytes
         if read_back:
             for res, names in ((g, ("lane_gaps", "win_hist", "long_gaps")),

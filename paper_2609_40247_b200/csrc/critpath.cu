@@ -58,6 +58,7 @@ struct CpArgs {
   const int16_t *kind;
   const int64_t *ts, *te;
   const int32_t *launch_of;
+  const int64_t *latency;  // ts_start - ts_start of the launch, for records with a launch
   const int32_t *lane_off, *lane_slot, *lane_window, *lane_dom_end, *lane_dev_base;
   const int16_t *lane_domain;
   const int64_t *t0;
@@ -165,13 +166,33 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_classify(CpArgs a) {
   load8_i64(a.ts, p0, a.n, s);
   load8_i64(a.te, p0, a.n, e);
   const i64 e_before = p0 > 0 ? a.te[p0 - 1] : 0;
+  // start of the launch = own start - launch latency: two sequential columns, no gather
   int32_t lo[CP_ITEMS];
   i64 sl[CP_ITEMS];
+  bool any_dev = false;
 #pragma unroll
-  for (int j = 0; j < CP_ITEMS; j++)
-    lo[j] = (p0 + j < tile_end && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) ? a.launch_of[p0 + j] : -1;
+  for (int j = 0; j < CP_ITEMS; j++) {
+    lo[j] = -1;
+    sl[j] = 0;
+    any_dev |= p0 + j < tile_end && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY);
+  }
+  if (any_dev) {
+    if (p0 + CP_ITEMS <= a.n) {
+      const int4 x = *reinterpret_cast<const int4 *>(a.launch_of + p0), y = *reinterpret_cast<const int4 *>(a.launch_of + p0 + 4);
+      lo[0] = x.x; lo[1] = x.y; lo[2] = x.z; lo[3] = x.w;
+      lo[4] = y.x; lo[5] = y.y; lo[6] = y.z; lo[7] = y.w;
+    } else {
 #pragma unroll
-  for (int j = 0; j < CP_ITEMS; j++) sl[j] = lo[j] >= 0 ? a.ts[lo[j]] : 0;
+      for (int j = 0; j < CP_ITEMS; j++)
+        if (p0 + j < a.n) lo[j] = a.launch_of[p0 + j];
+    }
+    load8_i64(a.latency, p0, a.n, sl);
+#pragma unroll
+    for (int j = 0; j < CP_ITEMS; j++) {
+      if (!(kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) lo[j] = -1;
+      sl[j] = s[j] - sl[j];
+    }
+  }
 
   CpLane ln(a, l0);
   const int sh = a.tsbits + a.idxbits;
@@ -252,25 +273,30 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
   for (int j = 0; j < CP_ITEMS; j++)
     if (p0 + j >= tile_end) kd[j] = -1;
 
-  // scan A: position + 1 of the last host node before each position
-  u64 run = 0;
-#pragma unroll
-  for (int j = 0; j < CP_ITEMS; j++)
-    if (cp_host_node(kd[j])) run = (u64)(p0 + j + 1);
-  u64 total;
-  u64 pre = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &total);
-  if (tid < 32) {
-    const u64 ex = tile_lookback<OpMax>(a.st_a, tile, total, OpMax(), a.status);
-    if (tid == 0) s_excl = ex;
-  }
-  __syncthreads();
-  pre = max(pre, s_excl);
+  // scan A: position + 1 of the last host node before each position.  A tile without host
+  // lanes has nothing to add and nobody after it in its lanes to tell: it publishes an empty
+  // prefix (values of earlier lanes are ignored anyway) and leaves prev_node untouched.
+  const bool no_host = span_outside_domain(a.lane_domain, a.lane_dom_end, l0, tile_end, 0);
+  u64 run = 0, total, pre;
   int32_t prev[CP_ITEMS];
-  {
+#pragma unroll
+  for (int j = 0; j < CP_ITEMS; j++) prev[j] = -1;
+  if (no_host) {
+    if (tid == 0) st_relaxed(&a.st_a[tile], td_pack(TD_PREFIX, 0));
+  } else {
+#pragma unroll
+    for (int j = 0; j < CP_ITEMS; j++)
+      if (cp_host_node(kd[j])) run = (u64)(p0 + j + 1);
+    pre = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &total);
+    if (tid < 32) {
+      const u64 ex = tile_lookback<OpMax>(a.st_a, tile, total, OpMax(), a.status);
+      if (tid == 0) s_excl = ex;
+    }
+    __syncthreads();
+    pre = max(pre, s_excl);
     CpLane ln(a, l0);
 #pragma unroll
     for (int j = 0; j < CP_ITEMS; j++) {
-      prev[j] = -1;
       if (kd[j] < 0) continue;
       if (!cp_host_node(kd[j])) continue;
       const int64_t p = p0 + j;
@@ -281,8 +307,9 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
       const int slot = a.lane_slot[ln.l];
       if (cp_code(a.te[p]) == a.slot_host_te[slot]) atomicMax(&a.slot_host_pos[slot], (int32_t)p);
     }
+    store8_i32(a.prev_node, p0, a.n, prev);
+    __syncthreads();  // s_excl is written again below
   }
-  store8_i32(a.prev_node, p0, a.n, prev);
 
   // scan B: position + 1 of the last run head at or before each position
   i64 s[CP_ITEMS];
@@ -488,7 +515,7 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_mark(CpArgs a) {
           add[3] = kd[j] == TA_KIND_COLL ? dur : 0;
           const int lk = a.link[p];
           if (lk == CP_LINK_STREAM) add[5] = (u64)(s - a.te[p - 1]);
-          else if (lk == CP_LINK_SUBMIT) add[4] = (u64)(s - a.ts[a.launch_of[p]]);
+          else if (lk == CP_LINK_SUBMIT) add[4] = (u64)a.latency[p];
           else { acc[9] = (u64)s; acc[10] = 1; }
         } else {
           const int32_t u = a.prev_node[p];
@@ -642,7 +669,7 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
 
   a.n = n; a.n_valid = h->n_valid; a.m = m; a.n_lanes = n_lanes; a.n_pids = n_pids; a.n_slots = n_slots;
   a.kind = h->sorted.kind; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
-  a.launch_of = h->join.launch_of;
+  a.launch_of = h->join.launch_of; a.latency = h->join.launch_latency;
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot; a.lane_window = h->sorted.lane_window;
   a.lane_dom_end = h->d_lane_dom_end; a.lane_dev_base = h->d_lane_dev_base;
   a.lane_domain = h->sorted.lane_domain; a.t0 = h->d_t0;
