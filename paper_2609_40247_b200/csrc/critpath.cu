@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_keys(CpArgs a) {
 }
 
 // ---- binding dependency of device records, waits of API records ------------------------
-__global__ void __launch_bounds__(CP_THREADS) k_cp_classify(CpArgs a) {
+__global__ void __launch_bounds__(CP_THREADS, 3) k_cp_classify(CpArgs a) {
   __shared__ int s_lane0;
   const int64_t tile_start = (int64_t)blockIdx.x * CP_TILE;
   if (tile_start >= a.n_valid) return;
