@@ -66,6 +66,25 @@ int main(void) {
   CHECK(cudaMemcpy(&comm, ov.d_comm, 8, cudaMemcpyDeviceToHost) == cudaSuccess);
   CHECK(busy == 450 && comm == 0);
 
+  /* the critical path of a stream without launches: from the kernel that ends last (1200) back
+   * along the stream - [520,540) ended before it began, a delay of 360 - and unresolved at 520,
+   * because the kernel before that one was still running when it began */
+  ta_critpath_result cp;
+  ta_critpath_summary cps;
+  CHECK(ta_critical_path(h, &cp, &cps) == TA_ERR_ORDER); /* the join comes first */
+  ta_join_result join;
+  ta_join_summary js;
+  CHECK(ta_correlate_launches(h, &join, &js) == TA_OK);
+  CHECK(ta_critical_path(h, &cp, &cps) == TA_OK && cp.n_rows == 1);
+  CHECK(cps.n_paths == 1 && cps.n_nodes == 2);
+  CHECK(cps.ns[TA_CP_KERNEL] == 320 && cps.ns[TA_CP_STREAM_DELAY] == 360);
+  int64_t begin = 0, end = 0;
+  int32_t reason = -1;
+  CHECK(cudaMemcpy(&begin, cp.p_begin, 8, cudaMemcpyDeviceToHost) == cudaSuccess);
+  CHECK(cudaMemcpy(&end, cp.p_end, 8, cudaMemcpyDeviceToHost) == cudaSuccess);
+  CHECK(cudaMemcpy(&reason, cp.p_reason, 4, cudaMemcpyDeviceToHost) == cudaSuccess);
+  CHECK(begin == 520 && end == 1200 && reason == 1);
+
   ta_free(h);
   ta_free(NULL);
   printf("c abi ok (library version %d, %lld kernel launches)\n", (int)ta_version(), (long long)ta_launch_count());

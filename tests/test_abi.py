@@ -77,3 +77,10 @@ def test_arguments_are_rejected_before_any_device_work():
     assert not handle.value
     L.ta_free(None)                                           # NULL-safe
     assert L.ta_strerror(5) and L.ta_version() > 0
+    # the analyses on top of the seven calls reject a missing handle or output before any CUDA call
+    out = ctypes.create_string_buffer(256)
+    vp = ctypes.c_void_p
+    for fn, nargs in ((L.ta_critical_path, 3), (L.ta_device_overlap, 2), (L.ta_rollup_operators, 3),
+                      (L.ta_blame_gaps, 4)):
+        raw = ctypes.CFUNCTYPE(ctypes.c_int, *([vp] * nargs))(ctypes.cast(fn, vp).value)
+        assert raw(None, *([ctypes.addressof(out)] * (nargs - 1))) == 1

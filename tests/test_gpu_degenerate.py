@@ -41,6 +41,17 @@ CASES = {
     + [("OP", 1, 0, 500, 500, 0, i, 0) for i in range(6)] + [("LAUNCH", 1, 0, 500, 500, i, 0, 0) for i in range(40)],
     "kernel that outlives the window": [("LAUNCH", 1, 0, 10, 11, 1, 0, 0), ("KERNEL", 1, 0, 20, 10**12, 1, 0, 0),
                                         ("KERNEL", 1, 0, 30, 40, 2, 0, 0)],
+    # a kernel that ends exactly when the wait returns did not release it (strictly before), one that
+    # ends exactly when the wait begins did; calls nested in a call; zero-length waits; equal last ends
+    "waits, ties and nested calls": [
+        ("LAUNCH", 1, 0, 10, 12, 1, 0, 0), ("LAUNCH", 1, 0, 13, 14, 2, 0, 0), ("KERNEL", 1, 0, 15, 50, 1, 0, 0),
+        ("KERNEL", 1, 1, 16, 20, 2, 0, 0), ("API", 1, 0, 20, 50, 0, 0, 0),
+        ("API", 1, 0, 60, 100, 0, 1, 0), ("LAUNCH", 1, 0, 70, 72, 3, 0, 0), ("API", 1, 0, 95, 98, 0, 2, 0),
+        ("KERNEL", 1, 0, 75, 96, 3, 0, 0), ("API", 1, 0, 200, 200, 0, 3, 0), ("KERNEL", 1, 1, 150, 199, 9, 0, 0),
+        ("LAUNCH", 1, 0, 250, 260, 4, 0, 0), ("KERNEL", 1, 0, 255, 300, 4, 0, 0), ("API", 1, 0, 270, 300, 0, 4, 0),
+        ("API", 2, 0, 10, 300, 0, 0, 0), ("COLL", 2, 7, 20, 40, 5, 0, 0), ("COLL", 2, 7, 40, 290, 5, 0, 1),
+        ("KERNEL", 2, 7, 100, 120, 6, 0, 0), ("LAUNCH", 2, 0, 5, 6, 6, 0, 0),
+        ("LAUNCH", 3, 0, 500, 510, 8, 0, 0), ("KERNEL", 3, 0, 400, 450, 8, 0, 0)],  # launch after its kernel
     "many kernels per launch": [("OP", 1, 0, 0, 5000, 0, 0, 0), ("LAUNCH", 1, 0, 10, 20, 7, 0, 0)]
     + [("KERNEL", 1, i % 3, 100 + 10 * i, 105 + 10 * i, 7, 0, 0) for i in range(100)],
 }

@@ -38,7 +38,9 @@ def test_call_order_is_enforced():
         g = w.stream_gaps(1000)
         assert _status(lambda: w.blame_gaps(g)) == TA_ERR_ORDER  # before the join
         assert _status(w.rollup_operators) == TA_ERR_ORDER
+        assert _status(w.critical_path) == TA_ERR_ORDER          # before the join
         w.correlate_launches()
+        assert w.critical_path().n_rows > 0
         assert _status(lambda: w.aggregate_ops(1, 2)) == TA_ERR_ORDER  # idle charged before the blame
         w.attribute_operators()
         w.blame_gaps(g)
