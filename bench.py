@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--cpu-sample-events", type=int, default=6_000_000)
+    ap.add_argument("--cpu-sample-events", type=int, default=24_000_000)
     return ap.parse_args()
 
 
