@@ -101,12 +101,15 @@ __device__ __forceinline__ int32_t winner_of(const JoinArgs &a, int64_t p, int s
 }
 
 // ---- pass 2: probes ----------------------------------------------------------
-// 256 threads x 8 consecutive positions; every output column is written once.
+// 256 threads x JP_ITEMS consecutive positions; every output column is written once.
 #define JP_THREADS 256
 #ifndef JP_MINB
 #define JP_MINB 3
 #endif
-#define JP_TILE (JP_THREADS * 8)
+#ifndef JP_ITEMS
+#define JP_ITEMS 8
+#endif
+#define JP_TILE (JP_THREADS * JP_ITEMS)
 
 template <bool DIRECT>
 __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) {
@@ -114,36 +117,37 @@ __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) 
   __shared__ int s_lane0, s_lane1;
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t tile_start = (int64_t)blockIdx.x * JP_TILE;
-  const int64_t p0 = tile_start + (int64_t)tid * 8;
+  constexpr int IT = JP_ITEMS;
+  const int64_t p0 = tile_start + (int64_t)tid * IT;
   if (tid == 0) { s_lane0 = -1; s_lane1 = -1; }
   __syncthreads();
   if (tid < 32 && tile_start < a.n_valid && a.n_lanes > 0) {
     int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (lane == 0) s_lane0 = l;
   }
-  int16_t kd[8];
-  load8_i16(a.kind, p0, a.n, 0, kd);
+  int16_t kd[IT];
+  loadn_i16<IT>(a.kind, p0, a.n, 0, kd);
   unsigned pm = 0;  // probes among the thread's records
 #pragma unroll
-  for (int j = 0; j < 8; j++)
+  for (int j = 0; j < IT; j++)
     if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
-  i64 c[8], s[8];
+  i64 c[IT], s[IT];
 #pragma unroll
-  for (int j = 0; j < 8; j++) c[j] = s[j] = 0;
+  for (int j = 0; j < IT; j++) c[j] = s[j] = 0;
   if (pm) {
-    load8_i64(a.corr, p0, a.n, c);
-    load8_i64(a.ts, p0, a.n, s);
+    loadn_i64<IT>(a.corr, p0, a.n, c);
+    loadn_i64<IT>(a.ts, p0, a.n, s);
   }
   __syncthreads();
   const int l0 = s_lane0;
-  int32_t lo[8];
-  int ln[8];
+  int32_t lo[IT];
+  int ln[IT];
   {
     int l = l0;
     int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
     int slot = l >= 0 ? a.lane_slot[l] : 0;
 #pragma unroll
-    for (int j = 0; j < 8; j++) {
+    for (int j = 0; j < IT; j++) {
       lo[j] = -1;
       ln[j] = -1;
       if (pm & (1u << j)) {
@@ -162,23 +166,23 @@ __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) 
       }
     }
     const int64_t plast = min(tile_start + JP_TILE, a.n_valid) - 1;
-    if (plast >= p0 && plast < p0 + 8) {
+    if (plast >= p0 && plast < p0 + IT) {
       while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
       s_lane1 = l;
     }
   }
   // launch times of the matched probes (independent gathers, issued together)
-  i64 ls[8], le[8];
+  i64 ls[IT], le[IT];
 #pragma unroll
-  for (int j = 0; j < 8; j++) {
+  for (int j = 0; j < IT; j++) {
     ls[j] = le[j] = 0;
     if (lo[j] >= 0) { ls[j] = a.ts[lo[j]]; le[j] = a.te[lo[j]]; }
   }
-  i64 lat[8], q[8];
+  i64 lat[IT], q[IT];
   u64 np = 0, nm = 0, sl = 0, sq = 0, mxl = 0, mnl_inv = 0, mxq = 0;
   int lm = -1;
 #pragma unroll
-  for (int j = 0; j < 8; j++) {
+  for (int j = 0; j < IT; j++) {
     lat[j] = q[j] = 0;
     if (!(pm & (1u << j))) continue;
     const bool matched = lo[j] >= 0;
@@ -212,9 +216,9 @@ __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) 
       }
     }
   }
-  store8_i32(a.launch_of, p0, a.n, lo);
-  store8_i64(a.latency, p0, a.n, lat);
-  store8_i64(a.qdelay, p0, a.n, q);
+  storen_i32<IT>(a.launch_of, p0, a.n, lo);
+  storen_i64<IT>(a.latency, p0, a.n, lat);
+  storen_i64<IT>(a.qdelay, p0, a.n, q);
   __syncthreads();
   const int l1 = s_lane1;
   for (int li = 0; li < 2; li++) {
@@ -256,12 +260,13 @@ __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) 
 }
 
 // ---- pass 3: launch statistics (duplicates, orphans) ---------------------------
+#define JS_TILE (JP_THREADS * 8)
 template <bool DIRECT>
 __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
   __shared__ u64 red[JP_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
   const int tid = threadIdx.x, lane = tid & 31;
-  const int64_t tile_start = (int64_t)blockIdx.x * JP_TILE;
+  const int64_t tile_start = (int64_t)blockIdx.x * JS_TILE;
   const int64_t p0 = tile_start + (int64_t)tid * 8;
   if (tid == 0) { s_lane0 = -1; s_lane1 = -1; }
   __syncthreads();
@@ -300,7 +305,7 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
         if (orphan) atomicAdd((u64 *)&sm->n_orphan_launch, 1ull);
       }
     }
-    const int64_t plast = min(tile_start + JP_TILE, a.n_valid) - 1;
+    const int64_t plast = min(tile_start + JS_TILE, a.n_valid) - 1;
     if (plast >= p0 && plast < p0 + 8) {
       while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
       s_lane1 = l;
@@ -403,7 +408,8 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   a.slot_min = slot_min; a.slot_max = slot_max; a.slot_base = slot_base;
   a.launch_of = launch_of; a.kol = kol; a.latency = latency; a.qdelay = qdelay; a.sum = d_sum;
   const unsigned grid = (unsigned)((n + JN_TILE - 1) / JN_TILE);
-  const unsigned grid8 = (unsigned)((n + JP_TILE - 1) / JP_TILE);
+  const unsigned grid8 = (unsigned)((n + JS_TILE - 1) / JS_TILE);
+  const unsigned grid_probe = (unsigned)((n + JP_TILE - 1) / JP_TILE);
   void *tmp_alloc = nullptr;
   bool direct = true;
   if (n > 0) {
@@ -424,7 +430,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       TA_CHECK_CUDA(h, cudaMemsetAsync(a.table, 0xFF, (size_t)(M > 0 ? M : 1) * 4, st));
       TA_CHECK_CUDA(h, cudaMemcpyAsync(slot_base, hbase.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
       k_join_build<<<TA_N grid, JN_THREADS, 0, st>>>(a);
-      k_join_probe<true><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
+      k_join_probe<true><<<TA_N grid_probe, JP_THREADS, 0, st>>>(a);
       k_join_launch_stats<true><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
     } else {
       // general path: compact, sort by (slot, corr) with sorted position as the stable tie-break
@@ -467,7 +473,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
         TA_TRY((launch_scan<OpMax, JoinHeadIn, JoinHeadOut>(h, m, hin, hout, OpMax(), t2)));
       }
       a.found = found;
-      k_join_probe<false><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
+      k_join_probe<false><<<TA_N grid_probe, JP_THREADS, 0, st>>>(a);
       k_join_launch_stats<false><<<TA_N grid8, JP_THREADS, 0, st>>>(a);
     }
     TA_CHECK_CUDA(h, cudaGetLastError());

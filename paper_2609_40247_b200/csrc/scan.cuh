@@ -142,6 +142,60 @@ __device__ __forceinline__ void store8_i32(int32_t *col, int64_t p0, int64_t n, 
   }
 }
 
+// the same for IT = 4 or 8 consecutive positions (p0 a multiple of IT)
+template <int IT>
+__device__ __forceinline__ void loadn_i16(const int16_t *col, int64_t p0, int64_t n, int16_t fill, int16_t *v) {
+  if (IT == 8) { load8_i16(col, p0, n, fill, v); return; }
+  if (p0 + IT <= n) {
+    const uint2 q = *reinterpret_cast<const uint2 *>(col + p0);
+    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+#pragma unroll
+    for (int j = 0; j < IT; j++) v[j] = hq[j];
+  } else {
+#pragma unroll
+    for (int j = 0; j < IT; j++) v[j] = p0 + j < n ? col[p0 + j] : fill;
+  }
+}
+template <int IT>
+__device__ __forceinline__ void loadn_i64(const int64_t *col, int64_t p0, int64_t n, i64 *v) {
+  if (p0 + IT <= n) {
+    const longlong2 *ps = reinterpret_cast<const longlong2 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < IT / 2; j++) {
+      const longlong2 x = ps[j];
+      v[2 * j] = x.x;
+      v[2 * j + 1] = x.y;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < IT; j++) v[j] = p0 + j < n ? col[p0 + j] : 0;
+  }
+}
+template <int IT>
+__device__ __forceinline__ void storen_i64(int64_t *col, int64_t p0, int64_t n, const i64 *v) {
+  if (p0 + IT <= n) {
+    longlong2 *ps = reinterpret_cast<longlong2 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < IT / 2; j++) ps[j] = make_longlong2(v[2 * j], v[2 * j + 1]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < IT; j++)
+      if (p0 + j < n) col[p0 + j] = v[j];
+  }
+}
+template <int IT>
+__device__ __forceinline__ void storen_i32(int32_t *col, int64_t p0, int64_t n, const int32_t *v) {
+  if (p0 + IT <= n) {
+    int4 *ps = reinterpret_cast<int4 *>(col + p0);
+#pragma unroll
+    for (int j = 0; j < IT / 4; j++) ps[j] = make_int4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+  } else {
+#pragma unroll
+    for (int j = 0; j < IT; j++)
+      if (p0 + j < n) col[p0 + j] = v[j];
+  }
+}
+
 // Ordered compaction of the sorted positions whose kind is in `kind_mask`: 256 threads x 16
 // positions per tile, vector loads of the kind column, one tile scan.
 #define CK_THREADS 256
