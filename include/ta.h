@@ -278,7 +278,10 @@ ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out);
  * (else INVALID_ARG); the population is further restricted to OPs with
  * op_n_kernels > 0 and value = T_op.  value_sel 2 (after ta_blame_gaps, else
  * TA_ERR_ORDER; kind_mask again exactly 1 << TA_KIND_OP): OPs with
- * op_gap_ns > 0, value = op_gap_ns.  Group key (window, pid, name_id); one
+ * op_gap_ns > 0, value = op_gap_ns.  value_sel 3 (after ta_critical_path, else
+ * TA_ERR_ORDER; any kind_mask): records with on_path = 1, value = ts_end -
+ * ts_start - which symbols the critical paths run through, and for how long.
+ * Group key (window, pid, name_id); one
  * output row per non-empty group in ascending signed key order with count,
  * sum, min, max and a histogram whose bin is min(39, floor(log2 v)) for
  * v >= 1 and 0 for v <= 0.

@@ -369,8 +369,8 @@ struct Oracle {
   // ---- step 6: per-symbol counts and duration statistics (Sec. 8.1 compares
   // per-symbol call counts and kernel durations).
   int aggregate(uint32_t kind_mask, int value_sel) {
-    if (value_sel < 0 || value_sel > 2) return 1;
-    if (value_sel != 0 && kind_mask != (1u << OP)) return 1;
+    if (value_sel < 0 || value_sel > 3) return 1;
+    if ((value_sel == 1 || value_sel == 2) && kind_mask != (1u << OP)) return 1;
     struct Row { int64_t count, sum, mn, mx; uint32_t hist[NBINS]; };
     std::map<std::tuple<int32_t, int32_t, int32_t>, Row> rows;
     for (int64_t p = 0; p < n_valid; p++) {
@@ -380,9 +380,12 @@ struct Oracle {
       else if (value_sel == 1) {
         if (op_n_kernels[p] <= 0) continue;
         v = op_last_end[p] - op_first_start[p];
-      } else {  // idle time of the process's device streams that coincides with the operator
+      } else if (value_sel == 2) {  // idle time of the process's device streams that coincides with the operator
         if (op_gap_ns[p] <= 0) continue;
         v = op_gap_ns[p];
+      } else {  // records a critical path passes through, by their own duration
+        if (!on_path[p]) continue;
+        v = ts_end[p] - ts_start[p];
       }
       auto key = std::make_tuple(win_sorted[p], pid[p], name_id[p]);
       auto it = rows.find(key);

@@ -38,6 +38,7 @@ struct AggArgs {
   const int32_t *op_n;
   const int64_t *op_first, *op_last;
   const int64_t *op_gap;  // value_sel 2
+  const uint8_t *on_path; // value_sel 3
   uint32_t kind_mask;
   int value_sel;
   int64_t min_name, R;
@@ -158,13 +159,20 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
-      } else {
+      } else if (a.value_sel == 2) {
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) { v[j] = a.op_gap[p0 + j]; sel[j] = v[j] > 0; }
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) nm[j] = a.name[p0 + j];
+      } else {
+#pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) sel[j] = a.on_path[p0 + j] != 0;
+#pragma unroll
+        for (int j = 0; j < AG_ITEMS; j++)
+          if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
       }
 #pragma unroll
       for (int j = 0; j < AG_ITEMS; j++) {
@@ -276,6 +284,7 @@ struct AggSortCtx {
   const int64_t *ts, *te;
   const int32_t *op_n;
   const int64_t *op_first, *op_last, *op_gap;
+  const uint8_t *on_path;
   const int32_t *lane_off, *lane_slot;
   const TripleTable *tt;
 };
@@ -288,8 +297,13 @@ __device__ __forceinline__ bool agg_selected(const AggSortCtx &c, int64_t p, i64
     *v = c.op_last[p] - c.op_first[p];
     return true;
   }
-  *v = c.op_gap[p];
-  return *v > 0;
+  if (c.value_sel == 2) {
+    *v = c.op_gap[p];
+    return *v > 0;
+  }
+  if (!c.on_path[p]) return false;
+  *v = c.te[p] - c.ts[p];
+  return true;
 }
 struct AggSelIn {
   AggSortCtx c;
@@ -384,7 +398,7 @@ static ta_status ta_run_aggregate_sorted(ta_window *h, uint32_t kind_mask, int v
   c.kind_mask = kind_mask & 63u; c.value_sel = value_sel;
   c.kind = h->sorted.kind; c.name = h->sorted.name_id; c.ts = h->sorted.ts_start; c.te = h->sorted.ts_end;
   c.op_n = h->attr.op_n_kernels; c.op_first = h->attr.op_first_start; c.op_last = h->attr.op_last_end;
-  c.op_gap = h->d_op_gap_ns; c.lane_off = h->sorted.lane_off; c.lane_slot = h->d_lane_slot;
+  c.op_gap = h->d_op_gap_ns; c.on_path = h->d_on_path; c.lane_off = h->sorted.lane_off; c.lane_slot = h->d_lane_slot;
   c.tt = h->d_triples;
 
   // 1. selection
@@ -487,7 +501,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.kind = h->sorted.kind; a.name = h->sorted.name_id; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot;
   a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
-  a.op_gap = h->d_op_gap_ns;
+  a.op_gap = h->d_op_gap_ns; a.on_path = h->d_on_path;
   a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
   a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   const bool host_kinds = (a.kind_mask & 7u) != 0, dev_kinds = (a.kind_mask & 56u) != 0;

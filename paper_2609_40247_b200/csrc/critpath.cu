@@ -628,7 +628,10 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   ro.p_ns = ck.take<int64_t>(n_slots * 8);
   TA_CHECK_CUDA(h, cudaMemsetAsync(on_path, 0, (size_t)nn, st));
   out->on_path = on_path;
-  if (h->n_valid <= 0) return TA_OK;
+  if (h->n_valid <= 0) {
+    h->d_on_path = on_path;
+    return TA_OK;
+  }
 
   const int64_t tiles = (h->n_valid + CP_TILE - 1) / CP_TILE;
   const int64_t mm = m > 0 ? m : 1;
@@ -743,6 +746,7 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
     for (int c = 0; c < 8; c++) ws->ns[c] += (int64_t)r[1 + c];
   }
   out->n_rows = (int64_t)rows;
+  h->d_on_path = on_path;
   out->p_window = ro.p_window; out->p_pid = ro.p_pid; out->p_sink = ro.p_sink;
   out->p_n_nodes = ro.p_n_nodes; out->p_reason = ro.p_reason;
   out->p_begin = ro.p_begin; out->p_end = ro.p_end; out->p_ns = ro.p_ns;

@@ -254,6 +254,7 @@ ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
   h->prekeys = 0;
   h->attr_status = 0;
   h->d_op_gap_ns = nullptr;
+  h->d_on_path = nullptr;
   h->h_off.assign(win_off, win_off + W + 1);
   h->h_t0.assign(win_t0, win_t0 + W);
   h->h_t1.assign(win_t1, win_t1 + W);
@@ -302,11 +303,12 @@ ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out) {
 
 ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel, ta_agg_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
-  if (value_sel < 0 || value_sel > 2) return TA_ERR_INVALID_ARG;
-  if (value_sel != 0 && kind_mask != (1u << TA_KIND_OP)) return TA_ERR_INVALID_ARG;
+  if (value_sel < 0 || value_sel > 3) return TA_ERR_INVALID_ARG;
+  if ((value_sel == 1 || value_sel == 2) && kind_mask != (1u << TA_KIND_OP)) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
   if (value_sel == 1 && (!(h->stage & 8) || h->attr_status != 0)) return TA_ERR_ORDER;
   if (value_sel == 2 && !h->d_op_gap_ns) return TA_ERR_ORDER;
+  if (value_sel == 3 && !h->d_on_path) return TA_ERR_ORDER;
   return ta_run_aggregate(h, kind_mask, value_sel, out);
 }
 

@@ -99,6 +99,7 @@ struct ta_window {
   ta_join_result join;
   ta_attr_result attr;
   const int64_t *d_op_gap_ns;  // per sorted position, set by the gap blame (null before)
+  const uint8_t *d_on_path;    // per sorted position, set by the critical path (null before)
   int attr_status;
 };
 

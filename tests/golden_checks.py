@@ -172,6 +172,9 @@ def check_H9(run):
     assert r["ts_start"][on].tolist() == ints(e["on_path"])
     assert r["ts_start"][r["cp_sink"]].tolist() == ints(e["sinks"])
     assert r["cp_sum"].reshape(-1, 10)[0].tolist() == [2, 10] + [a + b for a, b in zip(*want)]
+    sym = [tuple(int(x) for x in t.split(":")) for t in e["on_path_symbols"]]
+    assert list(zip(r["aggP_g_pid"].tolist(), r["aggP_g_name"].tolist(), r["aggP_g_count"].tolist(),
+                    r["aggP_g_sum"].tolist())) == sym
 
 
 ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9]

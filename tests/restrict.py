@@ -71,6 +71,7 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
         bl = w.blame_gaps(g)
         ag_gap = w.aggregate_ops(OP_MASK, 2)
         cp = w.critical_path()
+        ag_path = w.aggregate_ops(62, 3)
         del buf
         if checks is not None:
             checks(dict(window=w, sort=s, join=j, attr=a, gaps=g, agg_dev=ag_dev, agg_op=ag_op,
@@ -174,8 +175,10 @@ def run_gpu_restricted(events, win_off, t0, t1, subsets, min_gap=500_000, comm_s
                     r["b_win_count"] = bl.numpy("b_win_count")[wkeep]
                     r["b_win_ns"] = bl.numpy("b_win_ns")[wkeep]
             if "agg" in sub.groups:
-                for tag, res in (("agg0", ag_dev), ("aggT", ag_op), ("aggG", ag_gap)):
+                for tag, res in (("agg0", ag_dev), ("aggT", ag_op), ("aggG", ag_gap), ("aggP", ag_path)):
                     if tag == "aggG" and "blame" not in sub.groups:
+                        continue
+                    if tag == "aggP" and "critpath" not in sub.groups:
                         continue
                     if res is None:
                         continue

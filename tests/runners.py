@@ -25,6 +25,7 @@ CRITPATH_KEYS = ["on_path", "cp_window", "cp_pid", "cp_sink", "cp_n_nodes", "cp_
 
 DEVICE_MASK = (1 << 3) | (1 << 4) | (1 << 5)
 OP_MASK = 1
+NODE_MASK = 62  # API, LAUNCH and the device kinds: what a critical path is made of
 
 
 def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(DEVICE_MASK,)):
@@ -71,6 +72,9 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
     o.critical_path()
     for k in CRITPATH_KEYS:
         r[k] = o.get(k)
+    assert o.aggregate(NODE_MASK, 3) == 0
+    for k in AGG_KEYS:
+        r[f"aggP_{k}"] = o.get(k)
     o.close()
     return r
 
@@ -128,6 +132,9 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
         cp = w.critical_path()
         for k in CRITPATH_KEYS:
             r[k] = cp.numpy(k)
+        ag = w.aggregate_ops(NODE_MASK, 3)
+        for k in AGG_KEYS:
+            r[f"aggP_{k}"] = ag.numpy(k)
     return r
 
 

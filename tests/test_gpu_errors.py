@@ -40,7 +40,9 @@ def test_call_order_is_enforced():
         assert _status(w.rollup_operators) == TA_ERR_ORDER
         assert _status(w.critical_path) == TA_ERR_ORDER          # before the join
         w.correlate_launches()
+        assert _status(lambda: w.aggregate_ops(62, 3)) == TA_ERR_ORDER  # on-path table before the path
         assert w.critical_path().n_rows > 0
+        assert w.aggregate_ops(62, 3).n_groups > 0
         assert _status(lambda: w.aggregate_ops(1, 2)) == TA_ERR_ORDER  # idle charged before the blame
         w.attribute_operators()
         w.blame_gaps(g)
@@ -52,7 +54,7 @@ def test_invalid_arguments():
     wl, buf = _small()
     with ta.Window(buf, wl.win_off, wl.win_t0, wl.win_t1) as w:
         w.sort_timeline()
-        assert _status(lambda: w.aggregate_ops(1, 3)) == TA_ERR_INVALID_ARG
+        assert _status(lambda: w.aggregate_ops(1, 4)) == TA_ERR_INVALID_ARG
         assert _status(lambda: w.aggregate_ops(1 << 3, 1)) == TA_ERR_INVALID_ARG  # T_op needs the OP mask
     with pytest.raises((ta.TaError, ValueError)):
         ta.Window(buf, [0, len(wl.events)], [10], [10])  # empty window span

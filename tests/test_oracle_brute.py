@@ -356,6 +356,17 @@ def _critical_path_matches_brute(ev, off, t0, t1, sizes=()):
         tot[key[0], 2:] += b["ns"]
     assert np.array_equal(r["on_path"], on)
     assert np.array_equal(r["cp_sum"].reshape(-1, 10), tot)
+    # the per-symbol table of the records on a path is the plain aggregate of their durations
+    rows = brute.aggregate(sv, wins, r["n_valid"], 62,
+                           [int(sv[p]["ts_end"]) - int(sv[p]["ts_start"]) if on[p] else None
+                            for p in range(len(sv))])
+    assert len(rows) == len(r["aggP_g_count"])
+    for i, (key, row) in enumerate(rows):
+        assert (int(r["aggP_g_window"][i]), int(r["aggP_g_pid"][i]), int(r["aggP_g_name"][i])) == key
+        assert int(r["aggP_g_count"][i]) == row["count"] and int(r["aggP_g_sum"][i]) == row["sum"]
+        assert int(r["aggP_g_min"][i]) == row["min"] and int(r["aggP_g_max"][i]) == row["max"]
+        assert r["aggP_g_hist"][i].tolist() == row["hist"]
+    assert int(r["aggP_g_count"].sum()) == int(on.sum())
     return r, want
 
 
