@@ -374,8 +374,14 @@ def main():
         if world == 1 and not args.no_cpu_baseline:
             full = synth.CONFIG_EVENTS[args.workload] * args.scale
             sc = min(1.0, args.cpu_sample_events / full) * args.scale
-            swl = synth.make_workload(args.workload, sc, truth=False,
-                                      n_windows=12 if args.workload == "c4" else None)
+            if args.workload == "c4":  # whole windows of the batch's own size, as many as the sample allows
+                per_window = full / synth.C4_WINDOWS
+                sc = args.scale
+                swl = synth.make_workload("c4", sc, truth=False,
+                                          n_windows=max(1, min(synth.C4_WINDOWS,
+                                                               int(args.cpu_sample_events / per_window))))
+            else:
+                swl = synth.make_workload(args.workload, sc, truth=False)
             dt = time_oracle(swl)
             cpu = {"value": len(swl.events) / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": f"{len(swl.events)} records of workload {args.workload} "
