@@ -30,11 +30,15 @@
 #include "ta_internal.cuh"
 
 #define AT_THREADS 256
-#define AT_ITEMS 8
+// 4 or 8 records per thread in the stack and resolve kernels: with four the resolve kernel fits
+// 64 registers and 16 KB of shared memory, four CTAs per SM (eight and three: 0.12 ms slower)
+#ifndef AT_ITEMS
+#define AT_ITEMS 4
+#endif
 #define AT_TILE (AT_THREADS * AT_ITEMS)
 #define AT_CAP 16
 #ifndef AT_RES_MINB
-#define AT_RES_MINB 3
+#define AT_RES_MINB 4
 #endif
 // k_attr_ops: four records per thread keep it at 64 registers, four CTAs per SM (eight records and
 // three CTAs measured 0.12 ms slower on the 66.8 M record window: the kernel waits on gathers)
@@ -116,7 +120,7 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
     if (lane == 0) s_lane1 = l;
   }
   int16_t kd[AT_ITEMS];
-  load8_i16(a.kind, p0, a.n, 9, kd);
+  loadn_i16<AT_ITEMS>(a.kind, p0, a.n, 9, kd);
   __syncthreads();
   const int lane1 = s_lane1;
   if (lane1 < 0 || a.lane_domain[lane1] != 0) {
@@ -134,7 +138,7 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
   i64 m8 = INT64_MIN;
   if (opmask) {
     i64 t[AT_ITEMS];
-    load8_i64(a.te, p0, a.n, t);
+    loadn_i64<AT_ITEMS>(a.te, p0, a.n, t);
 #pragma unroll
     for (int j = 0; j < AT_ITEMS; j++)
       if (opmask & (1u << j)) { en[j] = t[j]; m8 = m8 > t[j] ? m8 : t[j]; }
@@ -338,7 +342,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     s.carry_pos[tid] = a.carry_pos[(size_t)tile * AT_CAP + tid];
   }
   int16_t kd[AT_ITEMS];
-  load8_i16(a.kind, p0, a.n, 9, kd);
+  loadn_i16<AT_ITEMS>(a.kind, p0, a.n, 9, kd);
   unsigned hostmask = 0;
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++)
@@ -346,9 +350,11 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
   const int any_host = __syncthreads_or(hostmask != 0);
   if (!any_host) {
     if (full) {
-      *reinterpret_cast<int4 *>(a.parent + p0) = make_int4(-1, -1, -1, -1);
-      *reinterpret_cast<int4 *>(a.parent + p0 + 4) = make_int4(-1, -1, -1, -1);
-      *reinterpret_cast<uint2 *>(a.depth + p0) = make_uint2(0, 0);
+#pragma unroll
+      for (int q = 0; q < AT_ITEMS / 4; q++) {
+        *reinterpret_cast<int4 *>(a.parent + p0 + 4 * q) = make_int4(-1, -1, -1, -1);
+        *reinterpret_cast<u32 *>(a.depth + p0 + 4 * q) = 0u;
+      }
     } else {
       for (int j = 0; j < AT_ITEMS; j++)
         if (p0 + j < a.n) { a.parent[p0 + j] = -1; a.depth[p0 + j] = 0; }
@@ -359,8 +365,8 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++) st[j] = en[j] = 0;
   if (hostmask) {
-    load8_i64(a.ts, p0, a.n, st);
-    load8_i64(a.te, p0, a.n, en);
+    loadn_i64<AT_ITEMS>(a.ts, p0, a.n, st);
+    loadn_i64<AT_ITEMS>(a.te, p0, a.n, en);
   }
   // lanes, leaves, the thread's maximum
   const int l0 = s.lane0;
@@ -492,14 +498,10 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     }
     plv[j] = (int16_t)pl;
   }
-  {
-    uint4 q;
-    q.x = (u32)(uint16_t)plv[0] | ((u32)(uint16_t)plv[1] << 16);
-    q.y = (u32)(uint16_t)plv[2] | ((u32)(uint16_t)plv[3] << 16);
-    q.z = (u32)(uint16_t)plv[4] | ((u32)(uint16_t)plv[5] << 16);
-    q.w = (u32)(uint16_t)plv[6] | ((u32)(uint16_t)plv[7] << 16);
-    *reinterpret_cast<uint4 *>(&s.parent_local[x0]) = q;
-  }
+#pragma unroll
+  for (int q = 0; q < AT_ITEMS / 2; q++)
+    *reinterpret_cast<u32 *>(&s.parent_local[x0 + 2 * q]) =
+        (u32)(uint16_t)plv[2 * q] | ((u32)(uint16_t)plv[2 * q + 1] << 16);
   __syncthreads();
   // depth = level in the parent forest; the chain is only followed through shared memory when
   // the parent is another thread's record and differs from the previous record's parent
@@ -538,12 +540,13 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     dep[j] = (uint8_t)d;
   }
   if (full) {
-    *reinterpret_cast<int4 *>(a.parent + p0) = make_int4(par_abs[0], par_abs[1], par_abs[2], par_abs[3]);
-    *reinterpret_cast<int4 *>(a.parent + p0 + 4) = make_int4(par_abs[4], par_abs[5], par_abs[6], par_abs[7]);
-    uint2 dq;
-    dq.x = dep[0] | (dep[1] << 8) | (dep[2] << 16) | ((u32)dep[3] << 24);
-    dq.y = dep[4] | (dep[5] << 8) | (dep[6] << 16) | ((u32)dep[7] << 24);
-    *reinterpret_cast<uint2 *>(a.depth + p0) = dq;
+#pragma unroll
+    for (int q = 0; q < AT_ITEMS / 4; q++) {
+      *reinterpret_cast<int4 *>(a.parent + p0 + 4 * q) =
+          make_int4(par_abs[4 * q], par_abs[4 * q + 1], par_abs[4 * q + 2], par_abs[4 * q + 3]);
+      *reinterpret_cast<u32 *>(a.depth + p0 + 4 * q) =
+          dep[4 * q] | (dep[4 * q + 1] << 8) | (dep[4 * q + 2] << 16) | ((u32)dep[4 * q + 3] << 24);
+    }
   } else {
 #pragma unroll
     for (int j = 0; j < AT_ITEMS; j++)

@@ -16,7 +16,9 @@
 #include "ta_internal.cuh"
 
 #define GP_THREADS 256
+#ifndef GP_ITEMS
 #define GP_ITEMS 8
+#endif
 #ifndef GP_MINB
 #define GP_MINB 4
 #endif
@@ -85,15 +87,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   }
   // kinds of the thread's eight records (0 = not a device record of the window)
   int16_t kd[GP_ITEMS];
-  if (full) {
-    uint4 q = *reinterpret_cast<const uint4 *>(a.kind + p0);
-    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
-#pragma unroll
-    for (int j = 0; j < GP_ITEMS; j++) kd[j] = hq[j];
-  } else {
-#pragma unroll
-    for (int j = 0; j < GP_ITEMS; j++) kd[j] = p0 + j < a.n ? a.kind[p0 + j] : (int16_t)0;
-  }
+  loadn_i16<GP_ITEMS>(a.kind, p0, a.n, 0, kd);
   bool any_dev = false;
 #pragma unroll
   for (int j = 0; j < GP_ITEMS; j++) {
