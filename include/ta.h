@@ -86,7 +86,9 @@ typedef enum ta_status {
  * `device` aligned to at least 256 bytes, or NULL; release takes it back.  If
  * alloc is NULL the library allocates stream-ordered from a pool of its own (one
  * per device, created on first use) that keeps freed memory for later calls
- * until the process ends. */
+ * until the process ends; released blocks are handed out again to requests of
+ * the same size on the same stream, and those that no handle has asked for
+ * during the lifetime of the last two handles return to the pool. */
 typedef struct ta_env {
   void *(*alloc)(size_t bytes, void *ctx);
   void (*release)(void *ptr, void *ctx);

@@ -64,7 +64,8 @@ struct ta_window {
   std::vector<int64_t> h_off, h_t0, h_t1;
   int64_t *d_off, *d_t0, *d_t1;
 
-  std::vector<void *> allocs;  // everything obtained from env.alloc
+  std::vector<void *> allocs;  // everything obtained from env.alloc (or the library's own pool)
+  std::vector<size_t> alloc_bytes;  // their sizes, same order
 
   // load products
   int32_t *d_status;

@@ -80,7 +80,7 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
 
 
 def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(DEVICE_MASK,),
-            on_device=True):
+            on_device=True, use_torch_allocator=True):
     """Same analysis through the C ABI of the CUDA library (torch supplies memory + stream)."""
     import torch
     from paper_2609_40247_b200 import ta
@@ -89,7 +89,7 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
     else:
         buf = np.ascontiguousarray(events)
     r = {}
-    with ta.Window(buf, win_off, t0, t1) as w:
+    with ta.Window(buf, win_off, t0, t1, use_torch_allocator=use_torch_allocator) as w:
         r["load_sum"] = w.load_summary
         s = w.sort_timeline()
         r["n_valid"] = s.n_valid

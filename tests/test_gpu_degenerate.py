@@ -139,3 +139,21 @@ def test_two_threads_with_a_handle_each():
     assert not errors, errors
     for k in range(2):
         assert_same(want[k], got[k])
+
+
+def test_library_pool_serves_windows_of_changing_sizes():
+    """Without allocator callbacks the library keeps released blocks by size and hands them out
+    again; windows of alternating sizes must not disturb each other's results, and blocks that
+    nobody asks for any more are given back (device memory in use stays bounded)."""
+    import torch
+    wls = [synth.make_workload("c1", s, truth=False) for s in (0.05, 0.02, 0.05, 0.01, 0.03, 0.05)]
+    want = [run_gpu(w.events, w.win_off, w.win_t0, w.win_t1, comm_sizes=w.comm_sizes) for w in wls]
+    used = []
+    for rep in range(3):
+        for w, ref in zip(wls, want):
+            got = run_gpu(w.events, w.win_off, w.win_t0, w.win_t1, comm_sizes=w.comm_sizes,
+                          use_torch_allocator=False)
+            assert_same(ref, got)
+        free, total = torch.cuda.mem_get_info()
+        used.append(total - free)
+    assert used[2] <= used[0] + (64 << 20)  # no growth from round to round
