@@ -331,12 +331,16 @@ __global__ void __launch_bounds__(256) k_load_pre(LoadArgs a) {
     const int leader = __ffs(active) - 1;
     for (int p = 0; p < a.plan.n_pass; p++) {
       u32 d = (u32)(key >> a.plan.shift[p]) & ((1u << a.plan.bits[p]) - 1u);
-      u32 d0 = __shfl_sync(active, d, leader);
-      if (__all_sync(active, d == d0)) {
-        if (lane == leader) atomicAdd(&sh[p * 256 + d0], (u32)__popc(active));
-      } else {
-        atomicAdd(&sh[p * 256 + d], 1u);
+      // only the two most significant digits (window, lane, top time bits) are ever the same for
+      // a whole warp: the test is not worth its instructions on the others
+      if (p >= a.plan.n_pass - 2) {
+        u32 d0 = __shfl_sync(active, d, leader);
+        if (__all_sync(active, d == d0)) {
+          if (lane == leader) atomicAdd(&sh[p * 256 + d0], (u32)__popc(active));
+          continue;
+        }
       }
+      atomicAdd(&sh[p * 256 + d], 1u);
     }
   }
   __syncthreads();
