@@ -85,7 +85,8 @@ __device__ __forceinline__ void wstack_combine(const WStack &ear, WStack &acc, b
   int keep = ear.cnt;
   if (acc.cnt > 0) {
     const i64 e0 = __shfl_sync(0xffffffffu, acc.e, 0);
-    keep = __popc(__ballot_sync(0xffffffffu, lane < ear.cnt && ear.e > e0));
+    // an earlier OP that ends exactly when the outermost later one does still encloses it
+    keep = __popc(__ballot_sync(0xffffffffu, lane < ear.cnt && ear.e >= e0));
   }
   if (keep + acc.cnt > AT_CAP) {
     *overflow = true;
@@ -162,7 +163,7 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
 #pragma unroll
   for (int j = AT_ITEMS - 1; j >= 0; j--) {
     if (opmask & (1u << j)) {
-      if (en[j] > sfx) {
+      if (en[j] >= sfx) {  // equal ends nest: the earlier OP encloses the later one
         int o = atomicAdd(&s_raw, 1);
         if (o < AT_CAP) { s_e[o] = en[j]; s_pos[o] = (int32_t)(p0 + j); }
       }

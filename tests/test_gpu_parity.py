@@ -56,6 +56,18 @@ def test_simulated_schedules(seed, tight):
     assert int(o["cp_ns"].reshape(-1, 8)[:, 7].sum()) > 0
 
 
+@pytest.mark.parametrize("seed", [5598, 6030, 6746, 7166, 7226, 8514])
+def test_equal_operator_ends_across_tile_boundaries(seed):
+    """Windows found by differential fuzzing: an operator and one nested in it end at the same
+    instant, and the records they enclose continue in the next tile of the attribution kernels
+    (the stack carried from tile to tile has to keep both)."""
+    rng = np.random.default_rng(seed)
+    ev, off, t0, t1, sizes = random_window(seed, span=int(rng.integers(200, 20000)),
+                                           n_dev=int(rng.integers(10, 6000)),
+                                           max_depth=int(rng.integers(1, 8)), n_pid=int(rng.integers(1, 5)))
+    both(ev, off, t0, t1, min_gap=1, comm_sizes=sizes)
+
+
 def test_larger_random_window_spans_tiles():
     ev, off, t0, t1, sizes = random_window(50, span=6000, n_dev=9000, max_depth=7, n_pid=3)
     both(ev, off, t0, t1, min_gap=1, comm_sizes=sizes)
