@@ -507,7 +507,9 @@ void ta_free(ta_window *h);
  * Limits: window span and the longest record < 2^40 ns each, windows x pids <
  * 2^22 (TA_ERR_TOO_LARGE).
  * Errors: TA_ERR_ORDER before ta_correlate_launches; TA_ERR_OOM; TA_ERR_CUDA;
- * TA_ERR_TIMEOUT.  Two stream synchronisations. */
+ * TA_ERR_TIMEOUT.  Two stream synchronisations (three when some stream lane
+ * does not end its records in ascending order and the device records have to
+ * be sorted by end time). */
 enum {
   TA_CP_KERNEL = 0, TA_CP_MEMCPY = 1, TA_CP_COLL = 2, TA_CP_LAUNCH_LATENCY = 3,
   TA_CP_STREAM_DELAY = 4, TA_CP_IN_CALL = 5, TA_CP_BETWEEN_CALLS = 6, TA_CP_WAIT_TAIL = 7

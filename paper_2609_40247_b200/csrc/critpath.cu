@@ -14,9 +14,12 @@
 //   - edges that change lane (submission: device -> host; synchronisation: host -> device)
 //     are the only ones the walk itself has to follow.
 // Kernels:
-//   k_cp_keys      (slot, ts_end) keys of the device records, then a stable radix sort:
-//                  "the device record of the process that finished last before t" becomes a
-//                  binary search (needed per API record, and for the sink);
+//   (in-order streams end their records in ascending order: then "the device record of the
+//   process that finished last before t" - needed per API record and for the sink - is one
+//   binary search per stream lane; k_cp_classify checks the order on the way, and only if some
+//   record ends before the one in front of it the step starts over with)
+//   k_cp_keys      (slot, ts_end) keys of the device records and a stable radix sort, after
+//                  which the same question is one binary search in the sorted keys;
 //   k_cp_classify  device records: which dependency binds (stream order / submission /
 //                  none); API records: the record whose end released the wait; per slot the
 //                  latest end among host nodes;
@@ -35,8 +38,8 @@
 //   k_cp_mark      every record decides from its run's entry whether it is on the path and
 //                  adds its share of the eight time classes (folded per warp);
 //   a scan         compacts the slots that have a path into rows.
-// HBM traffic: the sort (8 B + 8 B per device record and pass) and three passes over the
-// columns; the chain of lane changes costs a few short kernels over the list of waits.
+// HBM traffic: three passes over the columns (plus the sort, 8 B + 8 B per device record and
+// pass, when it is needed); the chain of lane changes costs a few short kernels over the list of waits.
 #include <climits>
 #include <cstring>
 #include <vector>
@@ -59,10 +62,12 @@ struct CpArgs {
   const int64_t *ts, *te;
   const int32_t *launch_of;
   const int64_t *latency;  // ts_start - ts_start of the launch, for records with a launch
-  const int32_t *lane_off, *lane_slot, *lane_window, *lane_dom_end, *lane_dev_base;
+  const int32_t *lane_off, *lane_slot, *lane_window, *lane_dom_end, *lane_dev_base, *lane_dom_next;
   const int16_t *lane_domain;
   const int64_t *t0;
   int tsbits, idxbits;
+  int use_sort;         // 0: every device lane is taken to end in ascending order (checked), no sort
+  u32 *not_ascending;   // set when some device record ends before the one in front of it in its lane
   u64 *keys;            // [device record index] ((slot << tsbits) | ts_end - t0) << idxbits | index
   u32 *pos;             // [device record index] sorted position
   const u64 *skeys;     // sorted keys
@@ -96,6 +101,31 @@ __device__ __forceinline__ bool cp_device(int k) { return k >= TA_KIND_KERNEL; }
 __device__ __forceinline__ int32_t cp_pos_of(const CpArgs &a, int64_t i) {
   if (a.idxbits) return (int32_t)a.pos[a.skeys[i] & ((1ull << a.idxbits) - 1)];
   return (int32_t)a.spos[i];
+}
+
+// Device lanes of one (window, process) are neighbours in the lane table.  When the ends of every
+// lane ascend, the record of the process that ended last before `limit` (or at all, limit =
+// INT64_MAX and `inclusive`) is the best of one binary search per lane: greatest ts_end, then
+// the highest position.
+__device__ __forceinline__ int32_t cp_last_ended(const CpArgs &a, int first_dev_lane, int slot, i64 limit,
+                                                 bool inclusive) {
+  int32_t best = -1;
+  i64 best_e = 0;
+  for (int dl = first_dev_lane; dl >= 0 && dl < a.n_lanes && a.lane_slot[dl] == slot && a.lane_domain[dl] == 1; dl++) {
+    int64_t lo = a.lane_off[dl], hi = a.lane_off[dl + 1];  // first position of the lane that ends at / after the limit
+    const int64_t begin = lo;
+    while (lo < hi) {
+      const int64_t mid = (lo + hi) >> 1;
+      const i64 e = a.te[mid];
+      if (inclusive ? e <= limit : e < limit) lo = mid + 1;
+      else hi = mid;
+    }
+    if (lo > begin) {
+      const i64 e = a.te[lo - 1];
+      if (best < 0 || e >= best_e) { best = (int32_t)(lo - 1); best_e = e; }
+    }
+  }
+  return best;
 }
 
 // lane bookkeeping of a thread that visits ascending positions
@@ -206,6 +236,7 @@ __global__ void __launch_bounds__(CP_THREADS, 3) k_cp_classify(CpArgs a) {
     ln.to(p);
     if (cp_device(kd[j])) {
       const i64 eq = j ? e[j - 1] : e_before;
+      if (!a.use_sort && p > ln.cur_off && e[j] < eq) *a.not_ascending = 1u;
       const bool q_ok = p > ln.cur_off && eq <= s[j];
       const bool l_ok = lo[j] >= 0 && sl[j] <= s[j];
       const u64 lk = (q_ok && (!l_ok || eq > sl[j])) ? CP_LINK_STREAM : (l_ok ? CP_LINK_SUBMIT : CP_LINK_END);
@@ -221,7 +252,10 @@ __global__ void __launch_bounds__(CP_THREADS, 3) k_cp_classify(CpArgs a) {
       if (kd[j] == TA_KIND_API) {
         // last element of the sorted (slot, ts_end) keys below (slot, this call's ts_end)
         int32_t d = -1;
-        if (a.m > 0) {
+        if (!a.use_sort) {
+          d = cp_last_ended(a, a.lane_dom_next[ln.l], slot, e[j], false);
+          if (d >= 0 && a.te[d] < s[j]) d = -1;
+        } else if (a.m > 0) {
           const u64 want = ((u64)slot << a.tsbits) | (u64)(e[j] - a.t0[a.lane_window[ln.l]]);
           int64_t lo_i = 0, hi_i = a.m;
           while (lo_i < hi_i) {
@@ -403,7 +437,16 @@ __global__ void __launch_bounds__(64) k_cp_start(CpArgs a) {
   const int sh = a.tsbits + a.idxbits;
   // last device record of the slot in (ts_end, position) order
   int32_t dsink = -1;
-  if (a.m > 0) {
+  if (!a.use_sort) {
+    int lo = 0, hi = a.n_lanes;  // first lane of the slot (lane_slot ascends with the lane index)
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if ((int64_t)a.lane_slot[mid] < slot) lo = mid + 1;
+      else hi = mid;
+    }
+    while (lo < a.n_lanes && (int64_t)a.lane_slot[lo] == slot && a.lane_domain[lo] != 1) lo++;
+    dsink = cp_last_ended(a, lo, (int)slot, LLONG_MAX, true);
+  } else if (a.m > 0) {
     int64_t lo = 0, hi = a.m;
     while (lo < hi) {
       const int64_t mid = (lo + hi) >> 1;
@@ -635,16 +678,13 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
 
   const int64_t tiles = (h->n_valid + CP_TILE - 1) / CP_TILE;
   const int64_t mm = m > 0 ? m : 1;
-  size_t tb = 3 * Carver::pad((size_t)mm * 8) + 3 * Carver::pad((size_t)mm * 4) + ta_sort_temp_bytes(mm) +
-              Carver::pad((size_t)nn) + 6 * Carver::pad((size_t)nn * 4) + Carver::pad((size_t)(n_lanes + 1) * 4) +
+  size_t tb = Carver::pad((size_t)nn) + 6 * Carver::pad((size_t)nn * 4) + Carver::pad((size_t)(n_lanes + 1) * 4) +
               2 * Carver::pad((size_t)tiles * 8) + Carver::pad(64) + Carver::pad((size_t)n_slots * 8) +
               Carver::pad((size_t)n_slots * 4) + Carver::pad((size_t)n_slots * CP_ACC * 8) +
               scan_temp_bytes(n_slots) + 1024;
   void *tmpb = ta_dalloc(h, tb);
   if (!tmpb) return TA_ERR_OOM;
   Carver ct(tmpb);
-  u64 *k_in = ct.take<u64>(mm), *k_scr = ct.take<u64>(mm), *k_fin = ct.take<u64>(mm);
-  u32 *v_in = ct.take<u32>(mm), *v_scr = ct.take<u32>(mm), *v_fin = ct.take<u32>(mm);
   CpArgs a;
   memset(&a, 0, sizeof(a));
   a.link = ct.take<uint8_t>(nn);
@@ -657,17 +697,17 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   a.st_a = ct.take<u64>(tiles); a.st_b = ct.take<u64>(tiles);
   a.counter = (u32 *)ct.take<u64>(8);
   a.n_eff = a.counter + 2;
+  a.not_ascending = a.counter + 3;
   a.slot_host_te = ct.take<u64>(n_slots);
   a.acc = ct.take<u64>(n_slots * CP_ACC);
-  TA_CHECK_CUDA(h, cudaMemsetAsync(zb, 0, (ct.base + ct.off) - zb, st));
+  const size_t zbytes = (ct.base + ct.off) - zb;
   // block filled with -1
   char *fb = ct.base + ct.off;
   a.entry = ct.take<int32_t>(nn);
   a.id_of = ct.take<int32_t>(nn);
   a.entry_lane = ct.take<int32_t>(n_lanes + 1);
   a.slot_host_pos = ct.take<int32_t>(n_slots);
-  TA_CHECK_CUDA(h, cudaMemsetAsync(fb, 0xff, (ct.base + ct.off) - fb, st));
-  void *sort_tmp = ct.base + ct.off; ct.off += ta_sort_temp_bytes(mm);
+  const size_t fbytes = (ct.base + ct.off) - fb;
   void *scan_mem = ct.base + ct.off;
 
   a.n = n; a.n_valid = h->n_valid; a.m = m; a.n_lanes = n_lanes; a.n_pids = n_pids; a.n_slots = n_slots;
@@ -675,32 +715,53 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   a.launch_of = h->join.launch_of; a.latency = h->join.launch_latency;
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot; a.lane_window = h->sorted.lane_window;
   a.lane_dom_end = h->d_lane_dom_end; a.lane_dev_base = h->d_lane_dev_base;
+  a.lane_dom_next = h->d_lane_dom_next;
   a.lane_domain = h->sorted.lane_domain; a.t0 = h->d_t0;
   a.tsbits = tsbits; a.idxbits = idxbits;
-  a.keys = k_in; a.pos = v_in;
   a.on_path = on_path; a.status = h->d_status;
 
-  if (m > 0) {
-    k_cp_keys<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
-    TA_CHECK_CUDA(h, cudaGetLastError());
-    if (idxbits) {
-      TA_TRY(ta_radix_sort_keys(h, k_in, k_scr, k_fin, m, ta_make_plan(idxbits, idxbits + tsbits + slot_bits),
-                                nullptr, sort_tmp, false));
-      a.spos = v_in;
-    } else {
-      TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, k_fin, v_fin, m,
-                                 ta_make_plan(0, tsbits + slot_bits), nullptr, sort_tmp));
-      a.spos = v_fin;
-    }
-  }
-  a.skeys = k_fin;
-  k_cp_classify<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
-  k_cp_runs<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
-  TA_CHECK_CUDA(h, cudaGetLastError());
-  // the waits that head a host run: a list whose length decides the number of doubling rounds
+  // In-order streams end their records in ascending order; then "the record of the process that
+  // ended last before t" is a binary search per device lane and nothing has to be sorted.  The
+  // first attempt assumes that and checks it; if some record ends before its predecessor, the
+  // second attempt sorts the device records by (process slot, ts_end) and searches there.
+  void *sortb = nullptr;
   u32 n_list = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_list, a.n_eff, 4, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  for (int attempt = 0; attempt < 2; attempt++) {
+    a.use_sort = attempt;
+    TA_CHECK_CUDA(h, cudaMemsetAsync(zb, 0, zbytes, st));
+    TA_CHECK_CUDA(h, cudaMemsetAsync(fb, 0xff, fbytes, st));
+    if (a.use_sort && m > 0) {
+      sortb = ta_dalloc(h, 3 * Carver::pad((size_t)mm * 8) + 3 * Carver::pad((size_t)mm * 4) + ta_sort_temp_bytes(mm) + 256);
+      if (!sortb) return TA_ERR_OOM;
+      Carver cs(sortb);
+      u64 *k_in = cs.take<u64>(mm), *k_scr = cs.take<u64>(mm), *k_fin = cs.take<u64>(mm);
+      u32 *v_in = cs.take<u32>(mm), *v_scr = cs.take<u32>(mm), *v_fin = cs.take<u32>(mm);
+      void *sort_tmp = cs.base + cs.off;
+      a.keys = k_in; a.pos = v_in;
+      k_cp_keys<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
+      TA_CHECK_CUDA(h, cudaGetLastError());
+      if (idxbits) {
+        TA_TRY(ta_radix_sort_keys(h, k_in, k_scr, k_fin, m, ta_make_plan(idxbits, idxbits + tsbits + slot_bits),
+                                  nullptr, sort_tmp, false));
+        a.spos = v_in;
+      } else {
+        TA_TRY(ta_radix_sort_pairs(h, k_in, v_in, k_scr, v_scr, k_fin, v_fin, m,
+                                   ta_make_plan(0, tsbits + slot_bits), nullptr, sort_tmp));
+        a.spos = v_fin;
+      }
+      a.skeys = k_fin;
+    }
+    k_cp_classify<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
+    k_cp_runs<<<TA_N (unsigned)tiles, CP_THREADS, 0, st>>>(a);
+    TA_CHECK_CUDA(h, cudaGetLastError());
+    // the waits that head a host run: a list whose length decides the number of doubling rounds
+    u32 words2[2] = {0, 0};
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(words2, a.n_eff, 8, cudaMemcpyDeviceToHost, st));
+    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    n_list = words2[0];
+    if (!a.use_sort && words2[1]) continue;
+    break;
+  }
   a.n_list = (int64_t)n_list;
   const int64_t nl = n_list > 0 ? n_list : 1;
   void *lb = ta_dalloc(h, 2 * Carver::pad((size_t)nl * 4) + Carver::pad((size_t)nl) + 256);
@@ -735,6 +796,7 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, lb);
+  if (sortb) ta_dfree(h, sortb);
   ta_dfree(h, tmpb);
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
   for (int64_t s = 0; s < n_slots; s++) {

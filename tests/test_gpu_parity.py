@@ -134,6 +134,18 @@ def test_defects_sprinkled_over_a_multi_window_batch():
     assert o["n_valid"] < n - third and int(o["load_sum"]["n_bad_kind"].sum()) == third
 
 
+def test_one_overlong_kernel_sends_the_critical_path_to_its_sorted_search():
+    """In-order streams end their records in ascending order and the critical path searches
+    each stream lane directly; a single kernel that outlives its successors makes it sort the
+    device records by end time instead (several tiles, sixteen processes)."""
+    wl = synth.make_workload("c3", 0.01, truth=False)
+    ev = wl.events.copy()
+    k = np.nonzero(ev["kind"] == 3)[0]
+    ev["ts_end"][k[len(k) // 2]] += 10_000_000
+    o, g = both(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=500_000, comm_sizes=wl.comm_sizes)
+    assert int(o["cp_n_nodes"].sum()) > 10_000
+
+
 def test_deep_nesting_is_reported():
     rows = [("OP", 1, 0, 10 + i, 1000 - i, 0, i, 0) for i in range(12)]
     rows.append(("LAUNCH", 1, 0, 100, 110, 1, 0, 0))
