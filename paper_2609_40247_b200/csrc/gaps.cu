@@ -36,6 +36,8 @@ struct GapArgs {
   const int64_t *t0, *t1;
   i64 min_gap;
   int list_only;  // second run: only (re)write the long-gap list
+  int local;      // 1: take the end of the record in front as the running maximum (and check that it is)
+  u32 *not_ascending;  // set in local mode when some lane does not end its records in ascending order
   int64_t *gap_before;
   ta_lane_gaps *lane_gaps;
   u32 *lane_hist, *win_hist;
@@ -140,14 +142,28 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
       s_lane1 = l;
     }
   }
-  u64 tile_max;
-  u64 thread_excl = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &tile_max);
-  if (tid < 32) {
-    u64 ex = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status);
-    if (tid == 0) s_excl_max = ex;
+  u64 pre = 0;
+  if (a.local) {
+    // in-order streams end their records in ascending order: the running maximum in front of a
+    // record is the (clipped) end of its neighbour, no scan and no look-back; the loop below
+    // checks the order and reports the first lane that breaks it
+    const int l = ln[0];
+    if (l >= 0 && p0 > (int64_t)a.lane_off[l]) {
+      const int w = a.lane_window[l];
+      const i64 w0 = a.t0[w], w1 = a.t1[w], e = a.te[p0 - 1];
+      pre = ((u64)(l + 1) << 40) | (u64)((e < w1 ? e : w1) - w0);
+    }
+    __syncthreads();  // s_lane1 and the zeroed histograms are read below
+  } else {
+    u64 tile_max;
+    u64 thread_excl = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &tile_max);
+    if (tid < 32) {
+      u64 ex = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status);
+      if (tid == 0) s_excl_max = ex;
+    }
+    __syncthreads();
+    pre = s_excl_max > thread_excl ? s_excl_max : thread_excl;
   }
-  __syncthreads();
-  u64 pre = s_excl_max > thread_excl ? s_excl_max : thread_excl;
 
   // gaps; statistics of the thread's first lane stay in registers, anything else is rare
   i64 gap[GP_ITEMS];
@@ -165,6 +181,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
       if (l >= 0) {
         if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
         Pi = ((pre >> 40) == (u64)(l + 1)) ? w0 + (i64)(pre & GP_LOW) : w0;
+        if (a.local && (pre >> 40) == (u64)(l + 1) && ce[j] < Pi) *a.not_ascending = 1u;
         g = s[j] > Pi ? s[j] - Pi : 0;
         const i64 from = s[j] > Pi ? s[j] : Pi;
         bz = ce[j] > from ? ce[j] - from : 0;
@@ -323,13 +340,22 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
   a.gap_before = gap_before; a.lane_gaps = lane_gaps; a.lane_hist = lane_hist; a.win_hist = win_hist;
   a.list = ulist; a.list_key = ukeys; a.list_cap = cap; a.st_max = st_max;
   a.counter = (u32 *)(scal + 1); a.status = h->d_status; a.n_long = scal;
-  if (tiles > 0) k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
-  TA_CHECK_CUDA(h, cudaGetLastError());
+  a.not_ascending = (u32 *)(scal + 2);
   u64 n_long = 0;
   int32_t words[ST_WORDS];
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&n_long, scal, 8, cudaMemcpyDeviceToHost, st));
-  TA_TRY(ta_read_status(h, words));
-  if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+  // first without the scan (every lane is taken to end its records in ascending order, which the
+  // kernel checks); if a lane does not, once more with the chained maximum scan
+  for (a.local = 1; a.local >= 0; a.local--) {
+    if (tiles > 0) k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
+    TA_CHECK_CUDA(h, cudaGetLastError());
+    u64 two[3] = {0, 0, 0};
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(two, scal, 24, cudaMemcpyDeviceToHost, st));
+    TA_TRY(ta_read_status(h, words));
+    if (words[ST_ERR]) return (ta_status)words[ST_ERR];
+    n_long = two[0];
+    if (!a.local || !(u32)two[2]) break;
+    TA_CHECK_CUDA(h, cudaMemsetAsync(zero_begin, 0, zero_end - zero_begin, st));
+  }
   if ((int64_t)n_long > cap) {
     // rare: a tiny min_gap made the list longer than the first guess; rebuild it
     ta_dfree(h, lt);
