@@ -45,3 +45,59 @@ def test_random_windows_match_the_oracle(block):
             assert_same(o, g, skip=skip)
         except AssertionError as e:
             raise AssertionError(f"seed {seed}: {e}") from None
+
+
+def _workload_case(seed):
+    """A scaled copy of one benchmark workload with a random seed and delivery order, timestamps
+    quantised (ties, long runs of equal keys) and, sometimes, sparse correlation ids, spread
+    symbol ids, sprinkled defects or duplicate launch ids."""
+    from paper_2609_40247_b200 import synth
+    rng = np.random.default_rng(seed)
+    name = ["c0", "c1", "c2", "c3", "c4"][seed % 5]
+    n_target = int(rng.integers(3000, 150000))
+    nw = int(rng.integers(2, 12)) if name == "c4" else None
+    scale = n_target / synth.CONFIG_EVENTS[name] * ((512 / nw) if nw else 1)
+    q = int(rng.choice([1, 10, 1000, 100000, 10_000_000, 1_000_000_000]))
+    wl = synth.make_workload(name, scale, shuffle_mode=int(rng.integers(0, 3)), truth=False, n_windows=nw,
+                             seed_offset=seed)
+    ev = wl.events.copy()
+    if q > 1:
+        base = int(min(wl.win_t0))
+        ev["ts_start"] = (ev["ts_start"] - base) // q * q + base
+        ev["ts_end"] = (ev["ts_end"] - base) // q * q + base
+    if rng.random() < 0.25:
+        m = ev["kind"] != 5
+        ev["corr_id"][m] = ev["corr_id"][m] * 1_000_003 - 2**45
+    if rng.random() < 0.25:
+        ev["name_id"] = (ev["name_id"].astype(np.int64) * 1_048_573 - 2**30).astype(np.int32)
+    if rng.random() < 0.3:
+        n = len(ev)
+        bad = rng.choice(n, size=max(3, n // int(rng.integers(5, 200))), replace=False)
+        third = len(bad) // 3
+        ev["kind"][bad[:third]] = 9
+        ev["ts_end"][bad[third:2 * third]] = ev["ts_start"][bad[third:2 * third]] - 1
+        ev["ts_start"][bad[2 * third:]] -= 10**12
+    if rng.random() < 0.2:
+        ev["corr_id"][ev["kind"] == 2] //= 2
+    return ev, wl.win_off, wl.win_t0, wl.win_t1, dict(min_gap=int(rng.choice([1, 1000, 500000])),
+                                                      comm_sizes=wl.comm_sizes)
+
+
+@pytest.mark.parametrize("block", range(4))
+def test_perturbed_workloads_match_the_oracle(block):
+    for seed in range(30_000 + 10 * block, 30_000 + 10 * (block + 1)):
+        try:
+            ev, off, t0, t1, kw = _workload_case(seed)
+        except RuntimeError:  # the generator could not fit this draw into its window
+            continue
+        o = run_oracle(ev, off, t0, t1, **kw)
+        g = run_gpu(ev, off, t0, t1, **kw)
+        skip = ()
+        if o["attr_status"] != 0:
+            assert g["attr_status"] == o["attr_status"], seed
+            skip = tuple(k for k in o if k.startswith(("parent", "depth", "op_", "attr_sum", "aggT_", "incl_",
+                                                       "replay_", "roll_")))
+        try:
+            assert_same(o, g, skip=skip)
+        except AssertionError as e:
+            raise AssertionError(f"seed {seed}: {e}") from None
