@@ -125,3 +125,19 @@ def test_c4_full_size_whole_windows():
                            comm_sizes=wl.comm_sizes,
                            checks=partial(_properties, wl.win_t0, wl.win_t1))
     _compare(ev, wl.win_off, wl.win_t0, wl.win_t1, wl.comm_sizes, subsets, r)
+
+
+def test_c3_quarter_size_with_one_overlong_kernel():
+    """One kernel that outlives its successors switches the gap kernel to its chained scan and
+    the critical path to its sorted search: both fallbacks at 16.7 M records, compared by process."""
+    wl = synth.make_workload("c3", 0.25, truth=False)
+    ev = wl.events.copy()
+    pids = np.unique(ev["pid"])
+    k = np.nonzero((ev["kind"] == 3) & (ev["pid"] == pids[0]))[0]
+    ev["ts_end"][k[len(k) // 3]] += 50_000_000
+    per_pid = ("sort", "join", "attr", "gaps", "agg", "overlap", "blame", "rollup", "critpath")
+    subsets = [Subset(f"pid{p}", ev["pid"] == p, per_pid, pid=int(p)) for p in (pids[0], pids[5])]
+    r = run_gpu_restricted(ev, wl.win_off, wl.win_t0, wl.win_t1, subsets, min_gap=MIN_GAP,
+                           comm_sizes=wl.comm_sizes,
+                           checks=partial(_properties, wl.win_t0, wl.win_t1))
+    _compare(ev, wl.win_off, wl.win_t0, wl.win_t1, wl.comm_sizes, subsets, r)
