@@ -78,7 +78,9 @@ typedef enum ta_status {
   TA_ERR_TOO_LARGE = 5,  /* a documented size limit was exceeded             */
   TA_ERR_OVERFLOW = 6,   /* an internal bounded table filled up              */
   TA_ERR_TIMEOUT = 7,    /* a bounded device-side wait gave up               */
-  TA_ERR_DEPTH = 8,      /* some host event has more than TA_MAX_DEPTH enclosing OPs */
+  TA_ERR_DEPTH = 8,      /* some host record's depth (its level in the parent
+                            forest, see ta_attribute_operators) exceeds
+                            TA_MAX_DEPTH                                     */
   TA_ERR_BAD_NESTING = 9 /* two ranges of one host thread overlap partially  */
 } ta_status;
 

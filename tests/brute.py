@@ -82,11 +82,13 @@ def join(sv, wins, n_valid):
 
 
 def attribution(sv, wins, n_valid, lane_list):
-    """O(n^2) scan of the enclosure definition.  Returns parent, depth, bad_nesting."""
+    """O(n^2) scan of the enclosure definition.  Returns parent, depth, bad_nesting, the
+    number of enclosers and the enclosers themselves."""
     n = len(sv)
     parent = [-1] * n
     depth = [0] * n
     n_enc = [0] * n
+    enc_of = [()] * n
     bad = False
     for (w, pid, dom, st, b, e) in lane_list:
         if dom != 0:
@@ -103,6 +105,7 @@ def attribution(sv, wins, n_valid, lane_list):
                 if sj <= si and ei <= ej and ((sj, ej) != (si, ei) or j < i):
                     enc.append(j)
             n_enc[i] = len(enc)
+            enc_of[i] = tuple(enc)
             if enc:
                 parent[i] = max(enc, key=lambda j: (int(sv[j]["ts_start"]), -int(sv[j]["ts_end"]), j))
     # depth = level in the forest the parents define
@@ -112,7 +115,7 @@ def attribution(sv, wins, n_valid, lane_list):
             d += 1
             c = parent[c]
         depth[i] = min(d, 255)
-    return parent, depth, bad, n_enc
+    return parent, depth, bad, n_enc, enc_of
 
 
 def gaps_bitmap(sv, lane, W0, W1):

@@ -177,4 +177,36 @@ def check_H9(run):
                     r["aggP_g_sum"].tolist())) == sym
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9]
+def check_H10(run):
+    g = load_golden("H10_depth_boundary.txt")
+    ev = g["events"]
+    n = len(ev)
+    r = run(ev, [0, n], [g["t0"]], [g["t1"]])
+    e = g["expect"]
+    assert r["perm"].tolist() == list(range(n))
+    assert r["parent"].tolist() == ints(e["parent"])
+    assert r["depth"].tolist() == ints(e["depth"])
+    assert r["op_of"].tolist() == ints(e["op_of"])
+    assert r["attr_status"] == 0
+    for k, v in kv(e["attr"]).items():
+        assert int(r["attr_sum"][0][k]) == v, k
+    # the fixture's encloser counts, from the enclosure rule itself (records are in canonical
+    # order, one host lane); the surplus over the depth = enclosers that are no ancestors
+    want_enc = ints(e["enclosers"])
+    for i in range(n):
+        if ev[i]["kind"] > 2:
+            assert want_enc[i] == 0
+            continue
+        enc = [j for j in range(n) if j != i and ev[j]["kind"] == 0
+               and ev[j]["ts_start"] <= ev[i]["ts_start"] and ev[i]["ts_end"] <= ev[j]["ts_end"]
+               and ((ev[j]["ts_start"], ev[j]["ts_end"]) != (ev[i]["ts_start"], ev[i]["ts_end"]) or j < i)]
+        assert len(enc) == want_enc[i], i
+        chain, c = [], int(r["parent"][i])
+        while c >= 0:
+            chain.append(c)
+            c = int(r["parent"][c])
+        assert set(chain) <= set(enc)
+        assert want_enc[i] - int(r["depth"][i]) == len(set(enc) - set(chain)), i
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9, check_H10]

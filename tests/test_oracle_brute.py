@@ -80,10 +80,25 @@ def test_attribution_against_quadratic_scan(seed):
     sv = _sorted_view(ev, r)
     wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
     ll = brute.lanes(sv, wins, r["n_valid"])
-    parent, depth, bad, n_enc = brute.attribution(sv, wins, r["n_valid"], ll)
+    parent, depth, bad, n_enc, enc_of = brute.attribution(sv, wins, r["n_valid"], ll)
     assert not bad and r["attr_status"] in (0, 8)
     assert r["parent"].tolist() == parent
     assert r["depth"].tolist() == depth
+    # what the depth is, said through the enclosure rule alone: every ancestor of a record
+    # encloses it, and the enclosers the depth leaves out are exactly those that are no
+    # ancestors (ranges that end at the very instant a zero-length record sits on)
+    for i in range(r["n_valid"]):
+        if sv[i]["kind"] > 2:
+            continue
+        chain, c = set(), int(r["parent"][i])
+        while c >= 0:
+            chain.add(c)
+            c = int(r["parent"][c])
+        assert chain <= set(enc_of[i])
+        off_chain = set(enc_of[i]) - chain
+        assert n_enc[i] - min(int(r["depth"][i]), n_enc[i]) == len(off_chain) or r["depth"][i] == 255
+        for j in off_chain:
+            assert sv[i]["ts_start"] == sv[i]["ts_end"] == sv[j]["ts_end"]
     # the forest level equals the number of enclosers for every record of non-zero length
     for i in range(r["n_valid"]):
         if sv[i]["kind"] <= 2 and sv[i]["ts_end"] > sv[i]["ts_start"]:
@@ -129,7 +144,7 @@ def test_bad_nesting_flag(seed):
     sv = _sorted_view(ev, r)
     wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
     ll = brute.lanes(sv, wins, r["n_valid"])
-    parent, depth, bad, _ = brute.attribution(sv, wins, r["n_valid"], ll)
+    parent, depth, bad, _, _ = brute.attribution(sv, wins, r["n_valid"], ll)
     assert (r["attr_status"] == 9) == bad
     assert bool(r["attr_sum"]["bad_nesting"].any()) == bad
     # the oracle evaluates the definition even then
