@@ -117,7 +117,8 @@ typedef struct ta_window ta_window; /* opaque handle; owns every result buffer *
  *   ts_start < t0 or >= t1        -> n_out_of_window
  * (ts_end > t1 is legal.)  Dropped records take part in nothing but `perm`.
  * Limits: n < 2^31; at most 4096 distinct (pid, domain, stream) triples; the
- * sort key (window, triple, ts_start - t0) must fit 63 bits.
+ * sort key (window, triple, ts_start - t0) must fit 63 bits; W x 2^ceil(log2(number of
+ * triples)) <= 2^24.
  * out_summary: host, W entries, caller-owned.
  * Errors: INVALID_ARG (null pointers, bad offsets, t0 >= t1), TOO_LARGE, OOM, CUDA.
  */
@@ -584,6 +585,29 @@ int32_t ta_version(void);
 int64_t ta_launch_count(void);
 void ta_profile_enable(int32_t on);
 int32_t ta_profile_radix(int64_t *n_passes, double *total_ms, double *total_bytes);
+
+/* Test hooks for the failure path (process-wide; meant for tests).
+ * Kernels that wait for another thread block (the chained scans, the radix
+ * passes) poll a descriptor a bounded number of times - 2^22 unless changed
+ * here - and then record TA_ERR_TIMEOUT in the handle's device status word and
+ * finish without writing output; every kernel launched on the handle afterwards
+ * sees the word and returns at once, and the entry point returns TA_ERR_TIMEOUT
+ * (as does every later call on that handle except ta_free).
+ * ta_set_spin_limit: poll limit of handles created from now on (<= 0 restores
+ * the default).  ta_selftest_wait_timeout: launches one warp on cuda_stream that
+ * waits, with a limit of `polls` polls (1 .. 2^20), for a descriptor that nothing
+ * ever publishes, waits for the kernel and returns what the wait recorded:
+ * TA_ERR_TIMEOUT when the bounded wait works as intended.  Uses 512 bytes from
+ * cudaMallocAsync.  Other returns: TA_ERR_INVALID_ARG, TA_ERR_OOM, TA_ERR_CUDA. */
+void ta_set_spin_limit(int32_t polls);
+ta_status ta_selftest_wait_timeout(void *cuda_stream, int32_t polls);
+/* ta_inject_device_error: writes `code` (an error status) into the handle's
+ * device status word from the host, as a device-side wait that gave up would,
+ * so that a test can check what follows such a failure without causing one:
+ * every later call on the handle except ta_free returns `code`, and its kernels
+ * return without touching their inputs.  Returns TA_OK, TA_ERR_INVALID_ARG or
+ * TA_ERR_CUDA. */
+ta_status ta_inject_device_error(ta_window *h, ta_status code);
 
 #ifdef __cplusplus
 }

@@ -511,6 +511,44 @@ struct Oracle {
     }
   }
 
+  // ---- operator efficiency (needs attribute() == 0).  An invocation's theoretical operation
+  // count and logical data volume, normalised by T_op and the device peaks, give model FLOPs
+  // utilisation and model bandwidth utilisation; speed-of-light attainment is the larger of
+  // the two (Sec. 6.1, "Operator execution and efficiency").  The counts come from outside
+  // the trace (shapes, data types, sharding): one pair of doubles per INPUT record, read for
+  // OP records only; a negative or NaN count means "not known".  Missing composition or
+  // inputs leave the measurement unresolved:
+  //   state 0  not a kept OP record            state 2  no kernels, or T_op == 0
+  //   state 1  resolved                        state 3  kernels, but a count is missing
+  //   MFU = flops / (T_op * 1e-9 s * peak_flops),  MBU = bytes / (T_op * 1e-9 s * peak_bw),
+  //   SOL_op = max(MFU, MBU); all three 0 unless resolved.
+  // Per window: the three state counts, the sums of flops, bytes and T_op over resolved
+  // invocations, and the largest SOL_op.  The only floating-point step of the analyzer.
+  struct SolSummary { int64_t n_resolved, n_no_kernels, n_no_counts, sum_top_ns; double sum_flops, sum_bytes, max_sol; };
+  std::vector<double> sol_mfu, sol_mbu, sol_op;
+  std::vector<uint8_t> sol_state;
+  std::vector<SolSummary> sol_sum;
+  void sol(const double* flops, const double* bytes, double peak_flops, double peak_bw) {
+    sol_mfu.assign(n, 0.0); sol_mbu.assign(n, 0.0); sol_op.assign(n, 0.0);
+    sol_state.assign(n, 0);
+    sol_sum.assign(W, SolSummary{0, 0, 0, 0, 0.0, 0.0, 0.0});
+    for (int64_t p = 0; p < n_valid; p++) {
+      if (kind[p] != OP) continue;
+      SolSummary& s = sol_sum[win_sorted[p]];
+      const int64_t top = op_last_end[p] - op_first_start[p];
+      if (op_n_kernels[p] <= 0 || top <= 0) { sol_state[p] = 2; s.n_no_kernels++; continue; }
+      const double f = flops[perm[p]], b = bytes[perm[p]];
+      if (!(f >= 0.0) || !(b >= 0.0)) { sol_state[p] = 3; s.n_no_counts++; continue; }
+      const double seconds = (double)top * 1e-9;
+      sol_mfu[p] = f / (seconds * peak_flops);
+      sol_mbu[p] = b / (seconds * peak_bw);
+      sol_op[p] = std::max(sol_mfu[p], sol_mbu[p]);
+      sol_state[p] = 1;
+      s.n_resolved++; s.sum_top_ns += top; s.sum_flops += f; s.sum_bytes += b;
+      s.max_sol = std::max(s.max_sol, sol_op[p]);
+    }
+  }
+
   // ---- gap blame (needs correlate() and gaps()).  For waits, readiness, dispatch and first
   // use are compared: ready work dispatched late implicates submission (Sec. 6.2, engine
   // patterns; "submission gaps", Sec. 8.2), and waits in a host call are matched with the
@@ -756,6 +794,9 @@ void orc_device_overlap(void* h) { ((Oracle*)h)->device_overlap(); }
 void orc_blame(void* h) { ((Oracle*)h)->blame(); }
 void orc_rollup(void* h) { ((Oracle*)h)->rollup(); }
 void orc_critical_path(void* h) { ((Oracle*)h)->critical_path(); }
+void orc_sol(void* h, const double* flops, const double* bytes, double peak_flops, double peak_bw) {
+  ((Oracle*)h)->sol(flops, bytes, peak_flops, peak_bw);
+}
 int64_t orc_n_valid(void* h) { return ((Oracle*)h)->n_valid; }
 
 // Exposes a result array by name: pointer into the oracle's storage, element
@@ -778,6 +819,7 @@ int32_t orc_get(void* h, const char* name, const void** ptr, int64_t* count, int
   G(replay_first_start) G(replay_last_end) G(replay_kernel_ns) G(roll_sum)
   G(b_class) G(b_launch) G(b_win_count) G(b_win_ns) G(op_gap_ns)
   G(on_path) G(cp_window) G(cp_pid) G(cp_sink) G(cp_n_nodes) G(cp_reason) G(cp_begin) G(cp_end) G(cp_ns) G(cp_sum)
+  G(sol_mfu) G(sol_mbu) G(sol_op) G(sol_state) G(sol_sum)
   G(d_window) G(d_pid) G(d_n_events) G(d_busy) G(d_idle) G(d_compute) G(d_comm) G(d_overlap) G(d_exposed)
 #undef G
   return -1;

@@ -28,6 +28,9 @@ LANE_GAPS = np.dtype([(k, "<i8") for k in
                       ("busy", "idle", "n_events", "n_gaps", "max_gap", "first_start", "last_end")])
 LONG_GAP = np.dtype([("lane", "<i4"), ("next_event", "<i4"), ("gap_start", "<i8"), ("gap_len", "<i8")])
 COMM_SIZE = np.dtype([("comm_id", "<i8"), ("n_ranks", "<i4"), ("reserved", "<i4")])
+SOL_SUM = np.dtype([("n_resolved", "<i8"), ("n_no_kernels", "<i8"), ("n_no_counts", "<i8"),
+                    ("sum_top_ns", "<i8"), ("sum_flops", "<f8"), ("sum_bytes", "<f8"),
+                    ("max_sol", "<f8")])
 
 _DTYPES = {
     "load_sum": LOAD_SUM, "dropped": np.uint8, "win_of": np.int32,
@@ -61,6 +64,8 @@ _DTYPES = {
     "on_path": np.uint8, "cp_window": np.int32, "cp_pid": np.int32, "cp_sink": np.int32,
     "cp_n_nodes": np.int32, "cp_reason": np.int32, "cp_begin": np.int64, "cp_end": np.int64,
     "cp_ns": np.int64, "cp_sum": np.int64,
+    "sol_mfu": np.float64, "sol_mbu": np.float64, "sol_op": np.float64, "sol_state": np.uint8,
+    "sol_sum": SOL_SUM,
 }
 
 _lib = None
@@ -103,6 +108,9 @@ def _load():
         lib.orc_rollup.restype = None
         lib.orc_critical_path.argtypes = [ctypes.c_void_p]
         lib.orc_critical_path.restype = None
+        lib.orc_sol.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_double,
+                                ctypes.c_double]
+        lib.orc_sol.restype = None
         lib.orc_n_valid.argtypes = [ctypes.c_void_p]
         lib.orc_n_valid.restype = ctypes.c_int64
         lib.orc_get.argtypes = [ctypes.c_void_p, ctypes.c_char_p, ctypes.POINTER(ctypes.c_void_p),
@@ -210,6 +218,15 @@ class Oracle:
         and synchronisation dependencies that ends at the last record to finish, and the split
         of its length into eight classes (needs correlate())."""
         self._lib.orc_critical_path(self._h)
+
+    def sol(self, flops, bytes_, peak_flops: float, peak_bw: float):
+        """MFU, MBU and SOL_op = max(MFU, MBU) of every operator invocation from its T_op, the
+        operation count and data volume given per INPUT record (float64, negative or NaN =
+        not known) and the device peaks in FLOP/s and B/s (needs attribute() == 0)."""
+        f = np.ascontiguousarray(flops, dtype=np.float64)
+        b = np.ascontiguousarray(bytes_, dtype=np.float64)
+        assert len(f) == self.n and len(b) == self.n
+        self._lib.orc_sol(self._h, f.ctypes.data, b.ctypes.data, float(peak_flops), float(peak_bw))
 
     def run_all(self, min_gap_ns: int = 500_000, comm_sizes=()):
         """load, sort, correlate, attribute, gaps, collectives; returns attribute's status."""

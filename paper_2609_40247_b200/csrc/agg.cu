@@ -51,6 +51,7 @@ struct AggArgs {
   u64 *d_cnt, *d_sum, *d_minc, *d_maxb;
   u32 *d_hist;
   u64 *n_groups;
+  const int32_t *status;
 };
 
 struct AggSmem {
@@ -105,6 +106,7 @@ __device__ __forceinline__ void agg_flush(const AggArgs &a, AggSmem &s) {
 
 __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
   __shared__ AggSmem s;
+  if (ta_failed(a.status)) return;
   int since_flush = 0;
   LaneWalker lw(a.lane_off, a.n_lanes, a.n_valid, a.n_valid);
   {
@@ -287,6 +289,7 @@ struct AggSortCtx {
   const uint8_t *on_path;
   const int32_t *lane_off, *lane_slot;
   const TripleTable *tt;
+  const int32_t *status;
 };
 __device__ __forceinline__ bool agg_selected(const AggSortCtx &c, int64_t p, i64 *v) {
   const int k = c.kind[p];
@@ -343,6 +346,7 @@ struct AggSortedOut {
 };
 __global__ void __launch_bounds__(256) k_agg_sorted_rows(AggSortCtx c, const u64 *ks, const int32_t *gstart,
                                                         int64_t ng, AggSortedOut o) {
+  if (ta_failed(c.status)) return;
   const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= ng) return;
   const u64 key = ks[gstart[g]];
@@ -355,6 +359,7 @@ __global__ void __launch_bounds__(256) k_agg_sorted_rows(AggSortCtx c, const u64
 }
 __global__ void __launch_bounds__(256) k_agg_sorted_reduce(AggSortCtx c, const u32 *pos, const int32_t *gid,
                                                           int64_t m, AggSortedOut o) {
+  if (ta_failed(c.status)) return;
   const int64_t j0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (j0 >= m) return;
   int32_t cur = -1;
@@ -399,7 +404,7 @@ static ta_status ta_run_aggregate_sorted(ta_window *h, uint32_t kind_mask, int v
   c.kind = h->sorted.kind; c.name = h->sorted.name_id; c.ts = h->sorted.ts_start; c.te = h->sorted.ts_end;
   c.op_n = h->attr.op_n_kernels; c.op_first = h->attr.op_first_start; c.op_last = h->attr.op_last_end;
   c.op_gap = h->d_op_gap_ns; c.on_path = h->d_on_path; c.lane_off = h->sorted.lane_off; c.lane_slot = h->d_lane_slot;
-  c.tt = h->d_triples;
+  c.tt = h->d_triples; c.status = h->d_status;
 
   // 1. selection
   size_t t1b = Carver::pad((size_t)nv * 8) + Carver::pad((size_t)nv * 4) + scan_temp_bytes(nv) + 256;
@@ -503,7 +508,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   a.op_n = h->attr.op_n_kernels; a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
   a.op_gap = h->d_op_gap_ns; a.on_path = h->d_on_path;
   a.kind_mask = kind_mask & 63u; a.value_sel = value_sel; a.min_name = h->min_name; a.R = R;
-  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end; a.status = h->d_status;
   const bool host_kinds = (a.kind_mask & 7u) != 0, dev_kinds = (a.kind_mask & 56u) != 0;
   a.want_domain = host_kinds && dev_kinds ? -1 : (dev_kinds ? 1 : 0);
   a.chunk = AG_ITEM;

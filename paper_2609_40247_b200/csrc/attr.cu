@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(AT_THREADS) k_attr_agg(AttrArgs a) {
   __shared__ i64 s_e[AT_CAP];
   __shared__ int32_t s_pos[AT_CAP];
   __shared__ int s_raw, s_lane1;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x;
   const int64_t tile_start = (int64_t)tile * AT_TILE;
@@ -255,6 +256,7 @@ __device__ __forceinline__ void stack_store(const StackArr &dst, int64_t t, cons
 __global__ void __launch_bounds__(128) k_attr_fold_up(StackArr child, int64_t n_child, StackArr parent,
                                                       int64_t n_parent, int32_t *status) {
   __shared__ StackStage st;
+  if (ta_failed(status)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t j = (int64_t)blockIdx.x * 4 + warp;
   if (j >= n_parent) return;
@@ -275,6 +277,7 @@ __global__ void __launch_bounds__(128) k_attr_fold_up(StackArr child, int64_t n_
 // one warp: start[i] = node[0] (+) ... (+) node[i - 1] for the few nodes of the top level
 __global__ void __launch_bounds__(32) k_attr_fold_top(StackArr node, int64_t n, StackArr start,
                                                       int leaf, int32_t *status) {
+  if (ta_failed(status)) return;
   const int lane = threadIdx.x & 31;
   bool overflow = false;
   WStack acc;
@@ -293,6 +296,7 @@ __global__ void __launch_bounds__(128) k_attr_fold_down(StackArr child, int64_t 
                                                         StackArr parent_start, int64_t n_parent,
                                                         StackArr child_start, int leaf, int32_t *status) {
   __shared__ StackStage st;
+  if (ta_failed(status)) return;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int64_t j = (int64_t)blockIdx.x * 4 + warp;
   if (j >= n_parent) return;
@@ -325,6 +329,7 @@ struct __align__(16) AttrSmem {
 
 __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrArgs a) {
   __shared__ AttrSmem s;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int tile = blockIdx.x;
   const int64_t tile_start = (int64_t)tile * AT_TILE;
@@ -578,6 +583,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a
   constexpr int IT = AT_OPS_ITEMS;
   __shared__ u64 red[AT_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t tile_start = (int64_t)blockIdx.x * AT_OPS_TILE;
   const int64_t p0 = tile_start + (int64_t)tid * IT;
@@ -708,6 +714,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a
 
 // first/last were accumulated in an order-preserving unsigned encoding (0 = untouched)
 __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
   if (p0 >= a.n_valid) return;
   int16_t kd[8];

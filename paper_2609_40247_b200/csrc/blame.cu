@@ -40,9 +40,11 @@ struct BlameArgs {
   u64 *pre;                 // exclusive running total of gap_len along the list
   int32_t *lane_first;      // [n_lanes + 1] first list entry of every lane
   int64_t *op_gap_ns;
+  const int32_t *status;
 };
 
 __global__ void __launch_bounds__(256) k_blame_classify(BlameArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const int lane = threadIdx.x & 31;
   int cls = -1, w = -1;
@@ -91,6 +93,7 @@ struct GapLenOut {
 
 // lane_first[l] = number of list entries whose lane is < l
 __global__ void __launch_bounds__(256) k_blame_lanes(BlameArgs a) {
+  if (ta_failed(a.status)) return;
   const int l = blockIdx.x * blockDim.x + threadIdx.x;
   if (l > a.n_lanes) return;
   int64_t lo = 0, hi = a.m;
@@ -133,6 +136,7 @@ __device__ __forceinline__ i64 gap_time_within(const BlameArgs &a, int64_t first
 
 __global__ void __launch_bounds__(BL_THREADS) k_blame_ops(BlameArgs a) {
   __shared__ int s_lane0;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x;
   const int64_t tile_start = (int64_t)blockIdx.x * BL_TILE;
   if (tile_start >= a.n_valid) return;
@@ -222,7 +226,7 @@ ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result 
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window; a.lane_slot = h->d_lane_slot;
   a.lane_dom_end = h->d_lane_dom_end; a.lane_dom_next = h->d_lane_dom_next;
   a.lane_domain = h->sorted.lane_domain;
-  a.g_class = g_class; a.g_launch = g_launch; a.op_gap_ns = op_gap;
+  a.g_class = g_class; a.g_launch = g_launch; a.op_gap_ns = op_gap; a.status = h->d_status;
 
   k_blame_classify<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(a);
   ScanTemp s1;

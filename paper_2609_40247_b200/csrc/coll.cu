@@ -37,15 +37,20 @@ __device__ __forceinline__ u32 coll_hash(u64 c) {
   return (u32)c;
 }
 
-__global__ void __launch_bounds__(256) k_coll_keys(CollCtx c, u64 *keys, int32_t *slot_of) {
+__global__ void __launch_bounds__(256) k_coll_keys(CollCtx c, u64 *keys, int32_t *slot_of, int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= c.m) return;
   u32 p = c.posc[j];
   int lane = lane_of_pos(c.lane_off, c.n_lanes, p);
   u64 cc = (u64)c.corr[p] ^ (1ull << 63);
+  // every communicator id was inserted while the records were loaded: a bounded probe all the same
   u32 s = coll_hash(cc) & (TA_COMM_SLOTS - 1);
-  while (c.cm->slots[s] != cc) s = (s + 1) & (TA_COMM_SLOTS - 1);
-  u64 rank = (u64)c.cm->rank_of_slot[s];
+  int probes = 0;
+  while (c.cm->slots[s] != cc && ++probes < TA_COMM_SLOTS) s = (s + 1) & (TA_COMM_SLOTS - 1);
+  u64 rank = 0;
+  if (probes < TA_COMM_SLOTS) rank = (u64)c.cm->rank_of_slot[s];
+  else ta_set_err(status, TA_ERR_OVERFLOW);
   u64 w = (u64)c.lane_window[lane];
   keys[j] = (w << (c.cbits + c.qbits)) | (rank << c.qbits) | (u64)((int64_t)c.seq[p] - c.min_seq);
   slot_of[j] = c.lane_slot[lane];
@@ -77,9 +82,11 @@ struct CollGroupArgs {
   int32_t *g_window, *g_seq, *g_n, *g_strag, *g_flags;
   int64_t *g_comm, *g_min, *g_max, *g_skew, *g_end;
   u64 *r_nstrag;                 // per (window, pid) slot
+  const int32_t *status;
 };
 
 __global__ void __launch_bounds__(256) k_coll_groups(CollGroupArgs a) {
+  if (ta_failed(a.status)) return;
   int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (g >= a.n_groups) return;
   const int64_t b = a.gstart[g], e = g + 1 < a.n_groups ? (int64_t)a.gstart[g + 1] : a.c.m;
@@ -123,12 +130,14 @@ struct CollMemberArgs {
   const int32_t *g_flags;
   int64_t *wait_ns;
   u64 *r_seen, *r_ncoll, *r_sum, *r_maxw;  // per (window, pid) slot
+  const int32_t *status;
 };
 
 // members in compacted (= pid-major) order: a CTA almost always sees one slot
 __global__ void __launch_bounds__(256) k_coll_members(CollMemberArgs a) {
   __shared__ int s_same;
   __shared__ u64 red[4][8];
+  if (ta_failed(a.status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   const bool in = j < a.c.m;
   int slot = -1;
@@ -269,7 +278,7 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   TA_CHECK_CUDA(h, cudaMemcpyAsync(d_expected, expected.data(), h->n_comms * 4, cudaMemcpyHostToDevice, st));
 
   const int gb = (int)((m + 255) / 256);
-  k_coll_keys<<<TA_N gb, 256, 0, st>>>(cx, k_in, slot_of);
+  k_coll_keys<<<TA_N gb, 256, 0, st>>>(cx, k_in, slot_of, h->d_status);
   TA_TRY(ta_radix_sort_pairs(h, k_in, nullptr, k_s, v_s, ks, cs, m,
                              ta_make_plan(0, cx.qbits + cx.cbits + wbits), nullptr, sort_tmp));
   ScanTemp s2;
@@ -294,12 +303,13 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   ga.g_strag = co.take<int32_t>(ng); ga.g_flags = co.take<int32_t>(ng);
   ga.g_comm = co.take<int64_t>(ng); ga.g_min = co.take<int64_t>(ng); ga.g_max = co.take<int64_t>(ng);
   ga.g_skew = co.take<int64_t>(ng); ga.g_end = co.take<int64_t>(ng);
-  ga.r_nstrag = r_nstrag;
+  ga.r_nstrag = r_nstrag; ga.status = h->d_status;
   k_coll_groups<<<TA_N (unsigned)((ng + 255) / 256), 256, 0, st>>>(ga);
 
   // 5. members
   CollMemberArgs ma;
   ma.c = cx; ma.gid_of_c = gid_of_c; ma.slot_of = slot_of; ma.g_max = ga.g_max; ma.g_flags = ga.g_flags;
+  ma.status = h->d_status;
   ma.wait_ns = wait_ns; ma.r_seen = r_seen; ma.r_ncoll = r_ncoll; ma.r_sum = r_sum; ma.r_maxw = r_maxw;
   k_coll_members<<<TA_N gb, 256, 0, st>>>(ma);
   TA_CHECK_CUDA(h, cudaGetLastError());

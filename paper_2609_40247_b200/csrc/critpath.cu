@@ -157,6 +157,7 @@ __device__ __forceinline__ int cp_tile_lane(const CpArgs &a, int64_t tile_start,
 
 // ---- keys of the device records ------------------------------------------------------
 __global__ void __launch_bounds__(CP_THREADS) k_cp_keys(CpArgs a) {
+  if (ta_failed(a.status)) return;
   __shared__ int s_lane0;
   const int64_t tile_start = (int64_t)blockIdx.x * CP_TILE;
   if (tile_start >= a.n_valid) return;
@@ -183,6 +184,7 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_keys(CpArgs a) {
 
 // ---- binding dependency of device records, waits of API records ------------------------
 __global__ void __launch_bounds__(CP_THREADS, 3) k_cp_classify(CpArgs a) {
+  if (ta_failed(a.status)) return;
   __shared__ int s_lane0;
   const int64_t tile_start = (int64_t)blockIdx.x * CP_TILE;
   if (tile_start >= a.n_valid) return;
@@ -292,10 +294,14 @@ __global__ void __launch_bounds__(CP_THREADS, 3) k_cp_classify(CpArgs a) {
 __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
   __shared__ u64 tmp[33];
   __shared__ u64 s_excl;
-  __shared__ int s_tile, s_lane0;
+  __shared__ int s_tile, s_lane0, s_fail;
   const int tid = threadIdx.x;
-  if (tid == 0) s_tile = (int)atomicAdd(a.counter, 1u);
+  if (tid == 0) {
+    s_tile = (int)atomicAdd(a.counter, 1u);
+    s_fail = ta_failed(a.status) ? 1 : 0;
+  }
   __syncthreads();
+  if (s_fail) return;
   const int tile = s_tile;
   const int64_t tile_start = (int64_t)tile * CP_TILE;
   const int64_t tile_end = min(tile_start + CP_TILE, a.n_valid);
@@ -323,10 +329,12 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
       if (cp_host_node(kd[j])) run = (u64)(p0 + j + 1);
     pre = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &total);
     if (tid < 32) {
-      const u64 ex = tile_lookback<OpMax>(a.st_a, tile, total, OpMax(), a.status);
-      if (tid == 0) s_excl = ex;
+      bool failed;
+      const u64 ex = tile_lookback<OpMax>(a.st_a, tile, total, OpMax(), a.status, &failed);
+      if (tid == 0) { s_excl = ex; s_fail = failed ? 1 : 0; }
     }
     __syncthreads();
+    if (s_fail) return;
     pre = max(pre, s_excl);
     CpLane ln(a, l0);
 #pragma unroll
@@ -384,10 +392,12 @@ __global__ void __launch_bounds__(CP_THREADS) k_cp_runs(CpArgs a) {
   }
   pre = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &total);
   if (tid < 32) {
-    const u64 ex = tile_lookback<OpMax>(a.st_b, tile, total, OpMax(), a.status);
-    if (tid == 0) s_excl = ex;
+    bool failed;
+    const u64 ex = tile_lookback<OpMax>(a.st_b, tile, total, OpMax(), a.status, &failed);
+    if (tid == 0) { s_excl = ex; s_fail = failed ? 1 : 0; }
   }
   __syncthreads();
+  if (s_fail) return;
   pre = max(pre, s_excl);
   int32_t hd[CP_ITEMS];
   {
@@ -425,6 +435,7 @@ __device__ __forceinline__ int32_t cp_follow(const CpArgs &a, int32_t d, bool re
 }
 
 __global__ void __launch_bounds__(256) k_cp_succ(CpArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (id >= a.n_list) return;
   a.jump_in[id] = cp_follow(a, a.cross[a.eff_pos[id]], false);
@@ -432,6 +443,7 @@ __global__ void __launch_bounds__(256) k_cp_succ(CpArgs a) {
 
 // one thread per (window, process): the sink and the hops from it to the first listed wait
 __global__ void __launch_bounds__(64) k_cp_start(CpArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t slot = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (slot >= a.n_slots) return;
   const int sh = a.tsbits + a.idxbits;
@@ -488,6 +500,7 @@ __global__ void __launch_bounds__(64) k_cp_start(CpArgs a) {
 // one round: what a marked wait reaches is marked (a wait marked during the round may pass its
 // mark on at once - everything it reaches is on the path as well), successors are squared
 __global__ void __launch_bounds__(256) k_cp_double(CpArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (id >= a.n_list) return;
   const int32_t j = a.jump_in[id];
@@ -500,6 +513,7 @@ __global__ void __launch_bounds__(256) k_cp_double(CpArgs a) {
 }
 
 __global__ void __launch_bounds__(256) k_cp_enter(CpArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t id = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (id >= a.n_list || !a.mark[id]) return;
   cp_follow(a, a.cross[a.eff_pos[id]], true);
@@ -507,6 +521,7 @@ __global__ void __launch_bounds__(256) k_cp_enter(CpArgs a) {
 
 // ---- membership and time classes ---------------------------------------------------------
 __global__ void __launch_bounds__(CP_THREADS) k_cp_mark(CpArgs a) {
+  if (ta_failed(a.status)) return;
   __shared__ int s_lane0;
   const int lane = threadIdx.x & 31;
   const int64_t tile_start = (int64_t)blockIdx.x * CP_TILE;

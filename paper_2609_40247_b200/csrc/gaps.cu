@@ -56,11 +56,16 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   __shared__ u64 red[4][GP_THREADS / 32];
   __shared__ u64 s_excl_max;
   __shared__ u32 s_hist[2][TA_NBINS];  // the tile's first two lanes; further lanes go straight to global
-  __shared__ int s_tile, s_lane0, s_lane1;
+  __shared__ int s_tile, s_lane0, s_lane1, s_fail;
   const int tid = threadIdx.x;
-  if (tid == 0) { s_tile = (int)atomicAdd(a.counter, 1u); s_lane1 = -1; }
+  if (tid == 0) {
+    s_tile = (int)atomicAdd(a.counter, 1u);
+    s_lane1 = -1;
+    s_fail = ta_failed(a.status) ? 1 : 0;
+  }
   if (tid < 2 * TA_NBINS) (&s_hist[0][0])[tid] = 0;
   __syncthreads();
+  if (s_fail) return;
   const int tile = s_tile;
   const int64_t tile_start = (int64_t)tile * GP_TILE;
   const int64_t p0 = tile_start + (int64_t)tid * GP_ITEMS;
@@ -158,10 +163,12 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
     u64 tile_max;
     u64 thread_excl = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &tile_max);
     if (tid < 32) {
-      u64 ex = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status);
-      if (tid == 0) s_excl_max = ex;
+      bool failed;
+      u64 ex = tile_lookback<OpMax>(a.st_max, tile, tile_max, OpMax(), a.status, &failed);
+      if (tid == 0) { s_excl_max = ex; s_fail = failed ? 1 : 0; }
     }
     __syncthreads();
+    if (s_fail) return;
     pre = s_excl_max > thread_excl ? s_excl_max : thread_excl;
   }
 
@@ -295,7 +302,9 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
 }
 
 __global__ void __launch_bounds__(256) k_gap_list_gather(const ta_long_gap *src, const u32 *order,
-                                                         int64_t m, ta_long_gap *dst) {
+                                                         int64_t m, ta_long_gap *dst,
+                                                         const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < m) dst[i] = src[order[i]];
 }
@@ -387,7 +396,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
     TA_TRY(ta_radix_sort_pairs(h, ukeys, nullptr, ks, vs, kf, order, m,
                                ta_make_plan(0, 32 + ta_bit_len((uint64_t)(L > 1 ? L - 1 : 1))), nullptr,
                                cs.base + cs.off));
-    k_gap_list_gather<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(ulist, order, m, list);
+    k_gap_list_gather<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(ulist, order, m, list, h->d_status);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
     ta_dfree(h, stb);

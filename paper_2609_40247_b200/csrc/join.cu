@@ -40,6 +40,7 @@ struct JoinArgs {
   int32_t *launch_of, *kol;
   int64_t *latency, *qdelay;
   ta_join_summary *sum;           // device, per window
+  const int32_t *status;
 };
 
 __device__ __forceinline__ u64 bias64(i64 v) { return (u64)v ^ (1ull << 63); }
@@ -76,6 +77,7 @@ __device__ __forceinline__ void tile_lane_range(int my_lo, int my_hi, int *s_lo,
 
 // ---- direct path: fill the table -------------------------------------------
 __global__ void __launch_bounds__(JN_THREADS) k_join_build(JoinArgs a) {
+  if (ta_failed(a.status)) return;
   const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
   LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
 #pragma unroll
@@ -115,6 +117,7 @@ template <bool DIRECT>
 __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) {
   __shared__ u64 red[7][JP_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t tile_start = (int64_t)blockIdx.x * JP_TILE;
   constexpr int IT = JP_ITEMS;
@@ -265,6 +268,7 @@ template <bool DIRECT>
 __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
   __shared__ u64 red[JP_THREADS / 32];
   __shared__ int s_lane0, s_lane1;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x, lane = tid & 31;
   const int64_t tile_start = (int64_t)blockIdx.x * JS_TILE;
   const int64_t p0 = tile_start + (int64_t)tid * 8;
@@ -335,13 +339,16 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
 
 // ---- general path helpers -----------------------------------------------------
 __global__ void __launch_bounds__(256) k_join_key_corr(const u32 *pos, int64_t m, const int64_t *corr,
-                                                       u64 *out) {
+                                                       u64 *out, const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j < m) out[j] = bias64(corr[pos[j]]);
 }
 __global__ void __launch_bounds__(256) k_join_key_slot(const u32 *pos, int64_t m,
                                                        const int32_t *lane_off, int n_lanes,
-                                                       const int32_t *lane_slot, u64 *out) {
+                                                       const int32_t *lane_slot, u64 *out,
+                                                       const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j < m) out[j] = (u64)lane_slot[lane_of_pos(lane_off, n_lanes, pos[j])];
 }
@@ -407,6 +414,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   a.lane_domain = h->sorted.lane_domain;
   a.slot_min = slot_min; a.slot_max = slot_max; a.slot_base = slot_base;
   a.launch_of = launch_of; a.kol = kol; a.latency = latency; a.qdelay = qdelay; a.sum = d_sum;
+  a.status = h->d_status;
   const unsigned grid = (unsigned)((n + JN_TILE - 1) / JN_TILE);
   const unsigned grid8 = (unsigned)((n + JS_TILE - 1) / JS_TILE);
   const unsigned grid_probe = (unsigned)((n + JP_TILE - 1) / JP_TILE);
@@ -458,10 +466,11 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
       if (m > 0) {
         const int gb = (int)((m + 255) / 256);
         u32 *vscr = (u32 *)found;  // found is not needed before the sorts are done
-        k_join_key_corr<<<TA_N gb, 256, 0, st>>>(pos, m, a.corr, k_in);
+        k_join_key_corr<<<TA_N gb, 256, 0, st>>>(pos, m, a.corr, k_in, h->d_status);
         TA_TRY(ta_radix_sort_pairs(h, k_in, pos, k_s, vscr, k_f, pos_s, m, ta_make_plan(0, 64), nullptr,
                                    sort_tmp));
-        k_join_key_slot<<<TA_N gb, 256, 0, st>>>(pos_s, m, a.lane_off, a.n_lanes, a.lane_slot, k_in);
+        k_join_key_slot<<<TA_N gb, 256, 0, st>>>(pos_s, m, a.lane_off, a.n_lanes, a.lane_slot, k_in,
+                                                 h->d_status);
         int sb = bit_length64((uint64_t)(n_slots > 1 ? n_slots - 1 : 1));
         TA_TRY(ta_radix_sort_pairs(h, k_in, pos_s, k_s, vscr, k_f, pos, m, ta_make_plan(0, sb), nullptr,
                                    sort_tmp));

@@ -247,6 +247,7 @@ struct LoadArgs {
   int sbits, tbits, wbits;
   int packed, dshift, ibits;  // packed: key also carries the index inside the window (low ibits)
   SortPlan plan;
+  int32_t *status;
 };
 
 // Pass 2 over the records: sort key and the digit histograms of all passes.
@@ -269,9 +270,15 @@ __global__ void __launch_bounds__(256) k_load(LoadArgs a) {
         if (!a.packed) hi = 1ull << (a.wbits + a.tbits + tsb);
       } else {
         u64 code = triple_code(r.pid, r.kind, r.stream);
+        // the discovery pass inserted every triple; a record that is not found was changed
+        // behind the library's back (the records are borrowed): bounded probe, error, rank 0
         u32 slot = hash_code(code) & (TA_TRIPLE_SLOTS - 1);
-        while (__ldg(&a.tt->slots[slot]) != code) slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
-        u64 rank = (u64)__ldg(&a.tt->rank_of_slot[slot]);
+        int probes = 0;
+        while (__ldg(&a.tt->slots[slot]) != code && ++probes < TA_TRIPLE_SLOTS)
+          slot = (slot + 1) & (TA_TRIPLE_SLOTS - 1);
+        u64 rank = 0;
+        if (probes < TA_TRIPLE_SLOTS) rank = (u64)__ldg(&a.tt->rank_of_slot[slot]);
+        else ta_set_err(a.status, TA_ERR_OVERFLOW);
         hi = ((u64)w << (a.tbits + tsb)) | (rank << tsb) | ((u64)(r.ts_start - a.t0[w]) >> a.dshift);
       }
       key = a.packed ? (hi << a.ibits) | (u64)(i - a.off[w]) : hi;
@@ -417,7 +424,7 @@ ta_status ta_launch_load(ta_window *h, bool allow_packed) {
   a.ev = h->events; a.n = h->n; a.off = h->d_off; a.t0 = h->d_t0; a.t1 = h->d_t1; a.W = h->W;
   a.tt = h->d_triples; a.keys = h->d_keys; a.hist = h->d_hist;
   a.sbits = h->sbits; a.tbits = h->tbits; a.wbits = h->wbits; a.plan = h->plan;
-  a.packed = h->packed; a.dshift = h->dshift; a.ibits = h->ibits;
+  a.packed = h->packed; a.dshift = h->dshift; a.ibits = h->ibits; a.status = h->d_status;
   // the words of the discovery pass are there once; a later call (the fall back to full
   // resolution keys) goes back to the records
   if (h->prekeys) k_load_pre<<<TA_N grid_for(h->n, 256, 8), 256, 0, h->stream>>>(a);

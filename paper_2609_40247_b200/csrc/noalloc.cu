@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(NA_THREADS) k_lane_gaps_noalloc(const int64_t 
   __shared__ u64 tmp[33];
   __shared__ u64 red[5][8];
   __shared__ u64 s_excl;
-  __shared__ int s_tile;
+  __shared__ int s_tile, s_fail;
   const int tid = threadIdx.x;
   if (tid == 0) s_tile = (int)atomicAdd(&sc->counter, 1u);
   __syncthreads();
@@ -56,10 +56,12 @@ __global__ void __launch_bounds__(NA_THREADS) k_lane_gaps_noalloc(const int64_t 
   u64 tile_max;
   u64 thread_excl = block_scan_exclusive<OpMax>(run, OpMax(), tmp, &tile_max);
   if (tid < 32) {
-    u64 e = tile_lookback<OpMax>(sc->state, tile, tile_max, OpMax(), sc->status);
-    if (tid == 0) s_excl = e;
+    bool failed;
+    u64 e = tile_lookback<OpMax>(sc->state, tile, tile_max, OpMax(), sc->status, &failed);
+    if (tid == 0) { s_excl = e; s_fail = failed ? 1 : 0; }
   }
   __syncthreads();
+  if (s_fail) return;  // a bounded wait gave up: the status word says so, nothing is written
   u64 pre = s_excl > thread_excl ? s_excl : thread_excl;
   u64 sb = 0, si = 0, ng = 0, mg = 0;
 #pragma unroll

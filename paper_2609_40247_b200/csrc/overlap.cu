@@ -36,11 +36,13 @@ struct OvKeyArgs {
   int tsbits, idxbits;
   u64 *keys;  // [device record index] ((slot << tsbits) | (ts_start - t0)) << idxbits | index
   u32 *pos;   // [device record index] sorted position
+  const int32_t *status;
 };
 
 // one tile of 2048 sorted positions per CTA; tiles that hold host lanes only leave at once
 __global__ void __launch_bounds__(OV_THREADS) k_ov_keys(OvKeyArgs a) {
   __shared__ int s_lane0;
+  if (ta_failed(a.status)) return;
   const int tid = threadIdx.x;
   const int64_t tile_start = (int64_t)blockIdx.x * OV_TILE;
   if (tile_start >= a.n_valid) return;
@@ -101,10 +103,14 @@ struct OvScanArgs {
 __global__ void __launch_bounds__(OV_THREADS, 3) k_ov_scan(OvScanArgs a) {
   __shared__ u64 tmp[3][33];
   __shared__ u64 s_excl[3];
-  __shared__ int s_tile;
+  __shared__ int s_tile, s_fail;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_tile = (int)atomicAdd(a.counter, 1u);
+  if (tid == 0) {
+    s_tile = (int)atomicAdd(a.counter, 1u);
+    s_fail = ta_failed(a.status) ? 1 : 0;
+  }
   __syncthreads();
+  if (s_fail) return;  // the sort gave up: the keys name no records
   const int tile = s_tile;
   const int64_t i0 = (int64_t)tile * OV_TILE + (int64_t)tid * OV_ITEMS;
   // keys and positions of the thread's eight records, then the gathers, all issued together
@@ -161,11 +167,14 @@ __global__ void __launch_bounds__(OV_THREADS, 3) k_ov_scan(OvScanArgs a) {
     u64 total;
     pre[ch] = block_scan_exclusive<OpMax>(run[ch], OpMax(), tmp[ch], &total);
     if (warp == ch) {  // three warps look back at the same time, one channel each
-      const u64 ex = tile_lookback<OpMax>(a.st[ch], tile, total, OpMax(), a.status);
+      bool failed;
+      const u64 ex = tile_lookback<OpMax>(a.st[ch], tile, total, OpMax(), a.status, &failed);
       if (lane == 0) s_excl[ch] = ex;
+      if (lane == 0 && failed) s_fail = 1;
     }
   }
   __syncthreads();
+  if (s_fail) return;
 #pragma unroll
   for (int ch = 0; ch < 3; ch++) pre[ch] = max(pre[ch], s_excl[ch]);
 
@@ -297,7 +306,7 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   ka.lane_off = h->sorted.lane_off; ka.lane_slot = h->d_lane_slot; ka.lane_window = h->sorted.lane_window;
   ka.lane_dom_end = h->d_lane_dom_end; ka.lane_dev_base = h->d_lane_dev_base;
   ka.lane_domain = h->sorted.lane_domain; ka.t0 = h->d_t0; ka.tsbits = tsbits; ka.idxbits = idxbits;
-  ka.keys = k_in; ka.pos = v_in;
+  ka.keys = k_in; ka.pos = v_in; ka.status = h->d_status;
   const int64_t key_tiles = (h->n_valid + OV_TILE - 1) / OV_TILE;
   k_ov_keys<<<TA_N (unsigned)key_tiles, OV_THREADS, 0, st>>>(ka);
   TA_CHECK_CUDA(h, cudaGetLastError());

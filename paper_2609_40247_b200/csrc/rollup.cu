@@ -36,6 +36,7 @@ struct RollArgs {
   u64 *incl_first, *incl_last, *replay_first, *replay_last;  // coded until the finalize kernel
   int64_t *incl_ns, *replay_ns;
   u64 *win_sum;  // [window][3]
+  const int32_t *status;
 };
 
 __device__ __forceinline__ u64 roll_code(i64 v) { return (u64)v ^ (1ull << 63); }
@@ -43,6 +44,7 @@ __device__ __forceinline__ u64 roll_code(i64 v) { return (u64)v ^ (1ull << 63); 
 // lane of the tile's first position; false if the tile holds no lane of `domain`
 __device__ __forceinline__ bool roll_tile(const RollArgs &a, int domain, int64_t *p0, int64_t *tile_end) {
   __shared__ int s_lane0;
+  if (ta_failed(a.status)) return false;
   const int64_t tile_start = (int64_t)blockIdx.x * RO_TILE;
   if (tile_start >= a.n_valid) return false;
   if (threadIdx.x < 32) {
@@ -178,7 +180,7 @@ ta_status ta_run_rollup(ta_window *h, ta_rollup_result *out, ta_rollup_summary *
   a.kol = h->join.kernels_of_launch;
   a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end; a.op_ns = h->attr.op_kernel_ns;
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window;
-  a.lane_dom_end = h->d_lane_dom_end; a.lane_domain = h->sorted.lane_domain;
+  a.lane_dom_end = h->d_lane_dom_end; a.lane_domain = h->sorted.lane_domain; a.status = h->d_status;
   const unsigned tiles = (unsigned)((h->n_valid + RO_TILE - 1) / RO_TILE);
   k_roll_ops<<<TA_N tiles, RO_THREADS, 0, st>>>(a);
   k_roll_replays<<<TA_N tiles, RO_THREADS, 0, st>>>(a);

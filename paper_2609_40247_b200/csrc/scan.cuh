@@ -37,10 +37,14 @@ __global__ void __launch_bounds__(SC_THREADS) k_scan(int64_t n, In in, Out out, 
                                                      int32_t *status) {
   __shared__ u64 tmp[33];
   __shared__ u64 s_excl;
-  __shared__ int s_tile;
+  __shared__ int s_tile, s_fail;
   const int tid = threadIdx.x;
-  if (tid == 0) s_tile = (int)atomicAdd(t.counter, 1u);
+  if (tid == 0) {
+    s_tile = (int)atomicAdd(t.counter, 1u);
+    s_fail = ta_failed(status) ? 1 : 0;
+  }
   __syncthreads();
+  if (s_fail) return;
   const int tile = s_tile;
   const int64_t i0 = (int64_t)tile * SC_TILE + (int64_t)tid * SC_ITEMS;
   u64 v[SC_ITEMS];
@@ -53,13 +57,16 @@ __global__ void __launch_bounds__(SC_THREADS) k_scan(int64_t n, In in, Out out, 
   u64 tile_total;
   u64 ex = block_scan_exclusive<Op>(run, op, tmp, &tile_total);
   if (tid < 32) {
-    u64 e = tile_lookback<Op>(t.state, tile, tile_total, op, status);
+    bool failed;
+    u64 e = tile_lookback<Op>(t.state, tile, tile_total, op, status, &failed);
     if (tid == 0) {
       s_excl = e;
-      if ((int64_t)(tile + 1) * SC_TILE >= n) *t.total = op(e, tile_total);
+      s_fail = failed ? 1 : 0;
+      if (!failed && (int64_t)(tile + 1) * SC_TILE >= n) *t.total = op(e, tile_total);
     }
   }
   __syncthreads();
+  if (s_fail) return;
   u64 pre = op(s_excl, ex);
 #pragma unroll
   for (int j = 0; j < SC_ITEMS; j++) {
@@ -206,10 +213,14 @@ static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_
                                                              int32_t *status) {
   __shared__ u64 tmp[33];
   __shared__ u64 s_excl;
-  __shared__ int s_tile;
+  __shared__ int s_tile, s_fail;
   const int tid = threadIdx.x;
-  if (tid == 0) s_tile = (int)atomicAdd(t.counter, 1u);
+  if (tid == 0) {
+    s_tile = (int)atomicAdd(t.counter, 1u);
+    s_fail = ta_failed(status) ? 1 : 0;
+  }
   __syncthreads();
+  if (s_fail) return;
   const int tile = s_tile;
   const int64_t p0 = (int64_t)tile * CK_TILE + (int64_t)tid * CK_ITEMS;
   int16_t kd[CK_ITEMS];
@@ -222,13 +233,16 @@ static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_
   u64 total;
   u64 ex = block_scan_exclusive<OpAdd>((u64)__popc(sel), OpAdd(), tmp, &total);
   if (tid < 32) {
-    u64 e = tile_lookback<OpAdd>(t.state, tile, total, OpAdd(), status);
+    bool failed;
+    u64 e = tile_lookback<OpAdd>(t.state, tile, total, OpAdd(), status, &failed);
     if (tid == 0) {
       s_excl = e;
-      if ((int64_t)(tile + 1) * CK_TILE >= n_valid) *t.total = e + total;
+      s_fail = failed ? 1 : 0;
+      if (!failed && (int64_t)(tile + 1) * CK_TILE >= n_valid) *t.total = e + total;
     }
   }
   __syncthreads();
+  if (s_fail) return;
   u64 o = s_excl + ex;
 #pragma unroll
   for (int j = 0; j < CK_ITEMS; j++)

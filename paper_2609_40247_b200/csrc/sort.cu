@@ -146,8 +146,10 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
         excl += w & TD_MASK;
         if ((w >> 62) == TD_PREFIX) break;
       }
-      st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
+      // a wait that gave up leaves the descriptor at its aggregate: the tiles behind this one
+      // look past it, meet the same unpublished tile (or the error word) and give up as well
       if (timed_out) s.fail = 1;
+      else st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
     }
     s.adj[tid] = (u32)excl - (u32)ex;
   }
@@ -189,10 +191,11 @@ __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_p
   const int tid = threadIdx.x;
   if (tid == 0) {
     s.tile = (int)atomicAdd(a.tile_counter, 1u);
-    s.fail = 0;
+    s.fail = ta_failed(a.status) ? 1 : 0;
   }
   for (int i = tid; i < (THREADS / 32) * RS_BINS; i += THREADS) (&s.warp_hist[0][0])[i] = 0;
   __syncthreads();
+  if (s.fail) return;  // an earlier kernel failed: the keys may be incomplete
   const int tile = s.tile;
   const int count = (int)min((int64_t)TILE, a.n - (int64_t)tile * TILE);
   if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true, STABLE>(a, s, tile, count);
@@ -212,6 +215,7 @@ __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_p
 // digit histograms of every pass (used when the caller has none)
 __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, int64_t n, SortPlan plan,
                                                     u32 *hist) {
+  // no failure check: reads keys by position only, and the passes that use the histogram check
   __shared__ u32 sh[10 * RS_BINS];
   for (int i = threadIdx.x; i < plan.n_pass * RS_BINS; i += blockDim.x) sh[i] = 0;
   __syncthreads();

@@ -136,6 +136,16 @@ ta_status ta_read_status(ta_window *h, int32_t *w) {
   return TA_OK;
 }
 
+// ---- test hooks: the poll limit of device-side waits, and a wait that nothing ends ----
+static std::atomic<int> g_ta_spin_limit{0};  // 0 = TA_SPIN_LIMIT; copied into each new handle's status word
+
+// One warp looks back from tile 1 at a tile-0 descriptor that nothing publishes.
+__global__ void k_selftest_wait(u64 *state, int32_t *status) {
+  bool failed;
+  tile_lookback<OpAdd>(state, 1, 1ull, OpAdd(), status, &failed);
+  if (threadIdx.x == 0) status[ST_LONG_RUN] = failed ? 1 : 0;
+}
+
 // ---- instrumentation: launch counter and event pairs around the radix passes ----
 std::atomic<long long> g_ta_launches{0};
 int g_ta_profile = 0;
@@ -180,6 +190,45 @@ int32_t ta_profile_radix(int64_t *n_passes, double *total_ms, double *total_byte
   return 0;
 }
 int64_t ta_launch_count(void) { return g_ta_launches.load(); }
+
+void ta_set_spin_limit(int32_t polls) { g_ta_spin_limit.store(polls > 0 ? polls : 0); }
+
+ta_status ta_inject_device_error(ta_window *h, ta_status code) {
+  if (!h || !h->d_status || code <= TA_OK || code > TA_ERR_BAD_NESTING) return TA_ERR_INVALID_ARG;
+  if (cudaSetDevice(h->device) != cudaSuccess) return TA_ERR_CUDA;
+  const int32_t c = (int32_t)code;
+  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_status + ST_ERR, &c, sizeof(c), cudaMemcpyHostToDevice, h->stream));
+  TA_CHECK_CUDA(h, cudaStreamSynchronize(h->stream));
+  return TA_OK;
+}
+
+ta_status ta_selftest_wait_timeout(void *cuda_stream, int32_t polls) {
+  if (polls < 1 || polls > (1 << 20)) return TA_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  unsigned char *buf = nullptr;
+  if (cudaMallocAsync((void **)&buf, 512, st) != cudaSuccess) {
+    cudaGetLastError();
+    return TA_ERR_OOM;
+  }
+  u64 *state = (u64 *)buf;                    // two descriptors, both EMPTY
+  int32_t *status = (int32_t *)(buf + 256);   // ST_WORDS words
+  int32_t words[ST_WORDS];
+  memset(words, 0, sizeof(words));
+  words[ST_SPIN] = polls;
+  cudaError_t e = cudaMemsetAsync(buf, 0, 512, st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(status, words, sizeof(words), cudaMemcpyHostToDevice, st);
+  if (e == cudaSuccess) {
+    k_selftest_wait<<<TA_N 1, 32, 0, st>>>(state, status);
+    e = cudaGetLastError();
+  }
+  if (e == cudaSuccess) e = cudaMemcpyAsync(words, status, sizeof(words), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  cudaFreeAsync(buf, st);
+  if (e != cudaSuccess) return TA_ERR_CUDA;
+  // the kernel must have come back by itself, with the error recorded and nothing published
+  if (words[ST_LONG_RUN] != 1) return TA_ERR_CUDA;
+  return (ta_status)words[ST_ERR];
+}
 
 const char *ta_strerror(ta_status s) {
   switch (s) {
@@ -236,6 +285,9 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t0, h->h_t0.data(), W * 8, cudaMemcpyHostToDevice, st));
   TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t1, h->h_t1.data(), W * 8, cudaMemcpyHostToDevice, st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status, 0, ST_WORDS * 4, st));
+  const int32_t spin = g_ta_spin_limit.load();
+  if (spin > 0)  // staged by the runtime before the call returns (pageable source)
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_status + ST_SPIN, &spin, sizeof(spin), cudaMemcpyHostToDevice, st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_triples->slots, 0xFF, sizeof(h->d_triples->slots), st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_comms->slots, 0xFF, sizeof(h->d_comms->slots), st));
   TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_load_sum, 0, W * sizeof(ta_load_summary), st));

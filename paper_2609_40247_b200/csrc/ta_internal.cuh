@@ -27,7 +27,9 @@ typedef unsigned int u32;
 #define TA_AGG_DENSE_LIMIT (1ll << 27)
 
 // device status word indices (h->d_status)
-enum { ST_ERR = 0, ST_LONG_RUN = 1, ST_N_TRIPLES = 2, ST_N_PIDS = 3, ST_N_COMMS = 4, ST_WORDS = 16 };
+// ST_SPIN: polls a device-side wait may make before it gives up (0 = TA_SPIN_LIMIT)
+enum { ST_ERR = 0, ST_LONG_RUN = 1, ST_N_TRIPLES = 2, ST_N_PIDS = 3, ST_N_COMMS = 4, ST_SPIN = 5,
+       ST_WORDS = 16 };
 
 struct TripleTable {       // device-resident, filled by the discovery kernel
   u64 slots[TA_TRIPLE_SLOTS];          // biased code or EMPTY
@@ -212,6 +214,14 @@ __device__ __forceinline__ int32_t ld_relaxed_i32(const int32_t *p) {
 __device__ __forceinline__ void ta_set_err(int32_t *status, int code) {
   atomicCAS(&status[ST_ERR], 0, code);
 }
+// Failure rule of the library: once the status word holds an error other than the data error
+// TA_ERR_DEPTH (a bounded wait gave up, a bounded table filled), intermediate buffers may be
+// incomplete, so every kernel launched afterwards returns before it indexes with anything an
+// earlier kernel produced.  ta_peek_err issues the load (kernels call it first and test the
+// value after their first position-only loads, so that the load costs no latency of its own).
+__device__ __forceinline__ int ta_peek_err(const int32_t *status) { return __ldcg(&status[ST_ERR]); }
+__device__ __forceinline__ bool ta_is_failure(int err) { return err != 0 && err != TA_ERR_DEPTH; }
+__device__ __forceinline__ bool ta_failed(const int32_t *status) { return ta_is_failure(ta_peek_err(status)); }
 
 // Tile descriptor: bits 63..62 = flag, low 62 bits = value.
 #define TD_EMPTY 0ull
@@ -220,13 +230,19 @@ __device__ __forceinline__ void ta_set_err(int32_t *status, int code) {
 #define TD_MASK ((1ull << 62) - 1)
 __device__ __forceinline__ u64 td_pack(u64 flag, u64 v) { return (flag << 62) | (v & TD_MASK); }
 
-// Polls a descriptor until it is published; gives up after TA_SPIN_LIMIT polls
-// (sets *timed_out and returns a PREFIX of 0 so that the caller terminates).
+// Polls a descriptor until it is published; gives up after status[ST_SPIN] polls (TA_SPIN_LIMIT
+// when that word is 0), or as soon as another wait has given up: sets *timed_out, records
+// TA_ERR_TIMEOUT and returns a PREFIX of 0 so that the caller's loop terminates.  A caller whose
+// wait timed out publishes no inclusive prefix and writes no output.
 __device__ __forceinline__ u64 td_wait(const u64 *p, int32_t *status, bool *timed_out) {
   u64 w = ld_relaxed(p);
-  int spins = 0;
+  int spins = 0, limit = 0;
   while ((w >> 62) == TD_EMPTY) {
-    if (++spins > TA_SPIN_LIMIT || ld_relaxed_i32(&status[ST_ERR]) != 0) {
+    if (limit == 0) {
+      limit = ld_relaxed_i32(&status[ST_SPIN]);
+      if (limit <= 0) limit = TA_SPIN_LIMIT;
+    }
+    if (++spins > limit || ta_is_failure(ld_relaxed_i32(&status[ST_ERR]))) {
       *timed_out = true;
       ta_set_err(status, TA_ERR_TIMEOUT);
       return td_pack(TD_PREFIX, 0);
@@ -266,11 +282,15 @@ __device__ __forceinline__ u64 warp_scan_inclusive(u64 v, Op op) {
 // Decoupled look-back for one value per tile; called by all 32 lanes of ONE
 // warp.  Publishes this tile's aggregate, combines the predecessors' values
 // (commutative op) and publishes the inclusive prefix.  Returns the exclusive
-// prefix in every lane.
+// prefix in every lane.  *failed (the same in every lane) is set when a wait
+// gave up: the prefix is then incomplete, nothing more is published (tiles
+// behind this one run into the same unpublished descriptor, or into the error
+// word, and fail too) and the caller must not write any output.
 template <class Op>
 __device__ __forceinline__ u64 tile_lookback(u64 *state, int tile, u64 aggregate, Op op,
-                                             int32_t *status) {
+                                             int32_t *status, bool *failed) {
   const int lane = threadIdx.x & 31;
+  *failed = false;
   if (tile == 0) {
     if (lane == 0) st_relaxed(&state[0], td_pack(TD_PREFIX, aggregate));
     return op.identity();
@@ -286,6 +306,10 @@ __device__ __forceinline__ u64 tile_lookback(u64 *state, int tile, u64 aggregate
     u64 c = lane <= first ? (w & TD_MASK) : op.identity();
     c = warp_reduce(c, op);
     excl = op(c, excl);
+    if (__any_sync(0xffffffffu, timed_out)) {
+      *failed = true;
+      return excl;
+    }
     if (pm) break;
   }
   if (lane == 0) st_relaxed(&state[tile], td_pack(TD_PREFIX, op(excl, aggregate)));

@@ -19,6 +19,7 @@
 // ---- pair path: equal-key runs -------------------------------------------
 __global__ void __launch_bounds__(256) k_fix_ties(const u64 *keys, u32 *perm, int64_t n_valid,
                                                   const ta_event *ev, int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p >= n_valid || p + 1 >= n_valid) return;
   u64 k = keys[p];
@@ -60,7 +61,9 @@ __global__ void __launch_bounds__(256) k_duration_key(const ta_event *ev, int64_
   const i64 *p = reinterpret_cast<const i64 *>(ev) + i * 5;
   out[i] = (u64)(max_dur - (p[1] - p[0]));  // longer first
 }
-__global__ void __launch_bounds__(256) k_gather_u64(const u64 *src, const u32 *idx, int64_t n, u64 *dst) {
+__global__ void __launch_bounds__(256) k_gather_u64(const u64 *src, const u32 *idx, int64_t n, u64 *dst,
+                                                    const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[idx[i]];
 }
@@ -68,7 +71,9 @@ __global__ void __launch_bounds__(256) k_gather_u64(const u64 *src, const u32 *i
 // ---- step 3: full-tuple keys for the dropped tail -------------------------
 // stage 0: ~ts_end, 1: ts_start, 2: (pid, domain, stream), 3: window
 __global__ void __launch_bounds__(256) k_tail_key(const ta_event *ev, const u32 *idx, int64_t m,
-                                                  int stage, const int64_t *off, int W, u64 *out) {
+                                                  int stage, const int64_t *off, int W, u64 *out,
+                                                  const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= m) return;
   Rec r = load_rec(ev, idx[j]);
@@ -107,6 +112,7 @@ __device__ __forceinline__ u32 gather_index(u64 k, const GatherArgs &a) {
 __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   __shared__ int s_slot[8];
   __shared__ u64 s_mx[8], s_mn[8];
+  if (ta_failed(a.status)) return;  // the sort gave up: the keys name no records
   const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   int slot = -1;
   u64 mx = 0, mn_inv = 0;
@@ -215,9 +221,13 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
                                                      int32_t *lane_code, int32_t *lane_slot,
                                                      int32_t *lane_dom_end, int32_t *lane_dom_next,
                                                      int32_t *lane_dev_base, int32_t *n_lanes_out,
-                                                     int64_t cap) {
+                                                     int64_t cap, const int32_t *status) {
   __shared__ u64 tmp[33];
   __shared__ u64 base;
+  if (ta_failed(status)) {  // no lanes: every later call then finds nothing to index
+    if (threadIdx.x == 0) { n_lanes_out[0] = 0; n_lanes_out[1] = 0; }
+    return;
+  }
   if (threadIdx.x == 0) base = 0;
   __syncthreads();
   for (int64_t c0 = 0; c0 < n_codes; c0 += blockDim.x) {
@@ -286,7 +296,8 @@ __device__ __forceinline__ u32 packed_index(u64 k, const PackInfo &pi) {
   return (u32)(pi.off[w] + (int64_t)(k & ((1ull << pi.ibits) - 1)));
 }
 __global__ void __launch_bounds__(256) k_unpack_tail(const u64 *keys, int64_t n_valid, int64_t n,
-                                                     PackInfo pi, u32 *perm) {
+                                                     PackInfo pi, u32 *perm, const int32_t *status) {
+  if (ta_failed(status)) return;
   int64_t p = n_valid + (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (p < n) perm[p] = packed_index(keys[p], pi);
 }
@@ -350,7 +361,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
         PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
         TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp, true));
         if (n > h->n_valid)
-          k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm);
+          k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm,
+                                                                            h->d_status);
       }
       if (!h->packed) {
         // step 1: (key, input index) pairs; the last pass writes (skeys, perm)
@@ -379,7 +391,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
           SortPlan dplan = ta_make_plan(0, dbits);
           TA_TRY(ta_radix_sort_pairs(h, dkeys, nullptr, kscr, vscr, skeys, dorder, n, dplan, nullptr,
                                      sort_tmp));
-          k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys);
+          k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys, h->d_status);
           TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
                                      sort_tmp));
           TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
@@ -400,7 +412,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
         // dropped records of a window share one key, so the tail is put in input order first
         for (int stage = h->packed ? -1 : 0; stage < 4; stage++) {
           if (stage == 3 && h->W == 1) break;
-          k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk);
+          k_tail_key<<<TA_N nblk(m, 256), 256, 0, st>>>(h->events, cur, m, stage, h->d_off, h->W, tk,
+                                                        h->d_status);
           int bits = stage == 2 ? 49 : stage == 3 ? (h->wbits > 0 ? h->wbits : 1) : stage < 0 ? 32 : 64;
           SortPlan tp = ta_make_plan(0, bits);
           TA_TRY(ta_radix_sort_pairs(h, tk, cur, kscr, vscr, tk2, nxt, m, tp, nullptr, sort_tmp));
@@ -428,7 +441,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
                                      h->n_pids > 0 ? h->n_pids : 1, h->d_triples, h->n_valid,
                                      lane_window, lane_pid, lane_stream, lane_domain, lane_off,
                                      lane_code, lane_slot, lane_dom_end, lane_dom_next, lane_dev_base, n_lanes_dev,
-                                     lane_cap);
+                                     lane_cap, h->d_status);
     TA_CHECK_CUDA(h, cudaGetLastError());
     TA_CHECK_CUDA(h, cudaMemcpyAsync(n_lanes_host, n_lanes_dev, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));

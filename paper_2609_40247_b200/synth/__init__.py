@@ -286,3 +286,33 @@ def make_workload(name: str, scale: float = 1.0, shuffle_mode: int = 0, truth: b
         win_t1=np.array([r[2] for r in results], dtype=np.int64),
         truth=[r[3] for r in results] if truth else None,
         comm_sizes=sorted(sizes.items()), params=plist)
+
+
+# Device peaks used with the synthetic operation counts (nominal dense bf16 and HBM3e figures
+# of one B200; inputs of the efficiency step, not measurements).
+PEAK_FLOPS = 2.25e15
+PEAK_BW = 7.7e12
+
+
+def op_work(events: np.ndarray, seed: int = 0, unknown_frac: float = 0.03):
+    """Synthetic side table for the operator-efficiency step: per INPUT record a theoretical
+    operation count (FLOP) and a logical data volume (bytes), float64, the stand-in for what
+    an analyzer derives from shapes, data types and sharding.  Only OP records get counts
+    (every other record holds -1 = not known); the counts depend on the symbol (a GEMM-like
+    or a bandwidth-bound operator per name_id) and vary per invocation like a batch size; a
+    fraction `unknown_frac` of the OP records has no counts."""
+    n = len(events)
+    rng = np.random.default_rng(seed)
+    flops = np.full(n, -1.0)
+    nbytes = np.full(n, -1.0)
+    ops = np.nonzero(events["kind"] == 0)[0]
+    name = events["name_id"][ops].astype(np.int64)
+    batch = rng.integers(1, 65, size=len(ops)).astype(np.float64)
+    hidden = 1024.0 * (1 + name % 8)
+    gemm_like = (name % 3) != 0
+    f = np.where(gemm_like, 2.0 * batch * hidden * hidden, 4.0 * batch * hidden)
+    b = np.where(gemm_like, 2.0 * (hidden * hidden + 2.0 * batch * hidden), 6.0 * batch * hidden)
+    known = rng.random(len(ops)) >= unknown_frac
+    flops[ops] = np.where(known, f, -1.0)
+    nbytes[ops] = np.where(known, b, -1.0)
+    return flops, nbytes

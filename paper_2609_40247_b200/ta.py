@@ -99,7 +99,8 @@ EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_at
            "ta_stream_gaps", "ta_aggregate_ops", "ta_match_collectives", "ta_free", "ta_strerror",
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
            "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps",
-           "ta_rollup_operators", "ta_critical_path"]
+           "ta_rollup_operators", "ta_critical_path", "ta_set_spin_limit",
+           "ta_selftest_wait_timeout", "ta_inject_device_error"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -153,6 +154,12 @@ def lib():
         L.ta_lane_gaps_noalloc.argtypes = [_vp, _vp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                            _vp, _vp, _vp]
         L.ta_launch_count.restype = ctypes.c_int64
+        L.ta_set_spin_limit.restype = None
+        L.ta_set_spin_limit.argtypes = [ctypes.c_int32]
+        L.ta_inject_device_error.restype = ctypes.c_int
+        L.ta_inject_device_error.argtypes = [_vp, ctypes.c_int]
+        L.ta_selftest_wait_timeout.restype = ctypes.c_int
+        L.ta_selftest_wait_timeout.argtypes = [_vp, ctypes.c_int32]
         L.ta_profile_enable.restype = None
         L.ta_profile_enable.argtypes = [ctypes.c_int32]
         L.ta_profile_radix.restype = ctypes.c_int32
@@ -197,6 +204,19 @@ def lane_gaps_noalloc(ts_start, ts_end, win_t0: int, win_t1: int, gap_before=Non
 def launch_count() -> int:
     """Kernels launched by the library since it was loaded."""
     return int(lib().ta_launch_count())
+
+
+def set_spin_limit(polls: int) -> None:
+    """Poll limit of the device-side waits of windows created from now on (0 = default)."""
+    lib().ta_set_spin_limit(int(polls))
+
+
+def selftest_wait_timeout(polls: int, stream=None) -> int:
+    """Runs a wait that nothing ever ends, limited to `polls` polls; returns the status the
+    kernel recorded (7 = TA_ERR_TIMEOUT when the bounded wait works)."""
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(lib().ta_selftest_wait_timeout(s.cuda_stream, int(polls)))
 
 
 def profile_enable(on: bool) -> None:
@@ -402,7 +422,9 @@ class Window:
     host numpy array of EVENT_DTYPE (copied to the device by the library)."""
 
     def __init__(self, events, win_off, win_t0, win_t1, device=None, stream=None,
-                 use_torch_allocator=True):
+                 use_torch_allocator=True, alloc_fn=None, release_fn=None):
+        """alloc_fn(nbytes) -> device address or None, release_fn(address): replace torch's
+        caching allocator behind the ta_env callbacks (both or neither)."""
         import torch
         L = lib()
         self._lib = L
@@ -435,12 +457,17 @@ class Window:
 
         def _alloc(size, ctx):
             try:
+                if alloc_fn is not None:
+                    return alloc_fn(int(size))
                 return torch.cuda.caching_allocator_alloc(int(size), dev, sptr)
             except Exception:
                 return None
 
         def _release(ptr, ctx):
-            torch.cuda.caching_allocator_delete(ptr)
+            if release_fn is not None:
+                release_fn(ptr)
+            else:
+                torch.cuda.caching_allocator_delete(ptr)
 
         self._alloc_cb = _ALLOC_T(_alloc)
         self._release_cb = _RELEASE_T(_release)
@@ -459,6 +486,12 @@ class Window:
             self.close()
             raise TaError(st, "ta_load_window")
         self._sorted = None
+
+    def inject_device_error(self, code: int) -> None:
+        """Test hook: marks the handle as failed, as a device-side wait that gave up would."""
+        st = self._lib.ta_inject_device_error(self._h, int(code))
+        if st != 0:
+            raise TaError(st, "ta_inject_device_error")
 
     # -- context manager / lifetime
     def close(self):

@@ -365,3 +365,31 @@ def critical_path(sv, wins, n_valid, launch_of):
         assert reason is not None, "the walk did not end"
         out[key] = dict(sink=sink, begin=begin, end=E(sink), reason=reason, nodes=seen, ns=ns)
     return out
+
+
+def operator_sol(kind, perm, op_n, op_first, op_last, flops, nbytes, peak_flops, peak_bw):
+    """MFU, MBU and SOL_op of every OP record as EXACT rationals (fractions.Fraction), from the
+    definition: count / (T_op seconds x peak).  Returns (state, mfu, mbu, sol) lists."""
+    from fractions import Fraction
+    n = len(kind)
+    state = [0] * n
+    mfu = [Fraction(0)] * n
+    mbu = [Fraction(0)] * n
+    sol = [Fraction(0)] * n
+    for p in range(n):
+        if kind[p] != 0:
+            continue
+        top = int(op_last[p]) - int(op_first[p])
+        if op_n[p] <= 0 or top <= 0:
+            state[p] = 2
+            continue
+        f, b = float(flops[perm[p]]), float(nbytes[perm[p]])
+        if not (f >= 0) or not (b >= 0):
+            state[p] = 3
+            continue
+        seconds = Fraction(top, 10**9)
+        mfu[p] = Fraction(f) / (seconds * Fraction(peak_flops))
+        mbu[p] = Fraction(b) / (seconds * Fraction(peak_bw))
+        sol[p] = max(mfu[p], mbu[p])
+        state[p] = 1
+    return state, mfu, mbu, sol

@@ -209,4 +209,22 @@ def check_H10(run):
         assert want_enc[i] - int(r["depth"][i]) == len(set(enc) - set(chain)), i
 
 
-ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9, check_H10]
+def check_H11(run):
+    g = load_golden("H11_operator_sol.txt")
+    n = len(g["events"])
+    r = run(g["events"], [0, n], [g["t0"]], [g["t1"]], op_work=g["op_work"])
+    e = g["expect"]
+    assert r["perm"].tolist() == list(range(n)) and r["attr_status"] == 0
+    assert r["sol_state"].tolist() == ints(e["sol_state"])
+    for k in ("sol_mfu", "sol_mbu", "sol_op"):
+        want = np.array([float(t) for t in e[k]])
+        # T_op * 1e-9 s is rounded (1e-9 is no binary fraction): a few units in the last place
+        assert np.allclose(r[k], want, rtol=1e-12, atol=0), k
+        assert np.array_equal(r[k] == 0, want == 0), k
+    s = r["sol_sum"][0]
+    for t in e["sol_sum"]:
+        k, v = t.split("=")
+        assert abs(float(s[k]) - float(v)) <= 1e-12 * abs(float(v)), k
+
+
+ALL = [check_H1, check_H2, check_H3, check_H4, check_H5, check_H6, check_H7, check_H8, check_H9, check_H10, check_H11]

@@ -19,9 +19,11 @@ def make_events(rows):
 
 
 def load_golden(name):
-    """Parses tests/golden/<name>: returns dict(events, t0, t1, min_gap, comm_sizes, expect)."""
-    rows, expect, comm = [], {}, []
+    """Parses tests/golden/<name>: returns dict(events, t0, t1, min_gap, comm_sizes, expect
+    [, op_work = (flops, bytes, peak_flops, peak_bw)])."""
+    rows, expect, comm, work = [], {}, [], []
     t0 = t1 = None
+    peaks = None
     min_gap = 1
     with open(os.path.join(GOLDEN, name)) as f:
         for line in f:
@@ -40,14 +42,25 @@ def load_golden(name):
                     rows.append(("KERNEL", 1, 0, t0 + i * dur, t0 + (i + 1) * dur, 0, 0, 0))
             elif tok[0] == "min_gap":
                 min_gap = int(tok[1])
+            elif tok[0] == "peaks":
+                peaks = (float(tok[1]), float(tok[2]))
+            elif tok[0] == "work":
+                work.append((int(tok[1]), float(tok[2]), float(tok[3])))
             elif tok[0] == "comm_size":
                 comm.append((int(tok[1]), int(tok[2])))
             elif tok[0] == "expect":
                 expect[tok[1]] = tok[2:]
             else:
                 raise ValueError(line)
-    return dict(events=make_events(rows), t0=t0, t1=t1, min_gap=min_gap, comm_sizes=comm,
-                expect=expect)
+    g = dict(events=make_events(rows), t0=t0, t1=t1, min_gap=min_gap, comm_sizes=comm,
+             expect=expect)
+    if peaks is not None:  # per input record: operation count and data volume, -1 = not known
+        flops = np.full(len(rows), -1.0)
+        nbytes = np.full(len(rows), -1.0)
+        for k, f, b in work:
+            flops[k], nbytes[k] = f, b
+        g["op_work"] = (flops, nbytes, peaks[0], peaks[1])
+    return g
 
 
 def ints(tokens):

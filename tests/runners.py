@@ -20,6 +20,7 @@ BLAME_KEYS = ["b_class", "b_launch", "b_win_count", "b_win_ns", "op_gap_ns"]
 OVERLAP_KEYS = ["d_window", "d_pid", "d_n_events", "d_busy", "d_idle", "d_compute", "d_comm",
                 "d_overlap", "d_exposed"]
 
+SOL_KEYS = ["sol_mfu", "sol_mbu", "sol_op", "sol_state", "sol_sum"]
 CRITPATH_KEYS = ["on_path", "cp_window", "cp_pid", "cp_sink", "cp_n_nodes", "cp_reason", "cp_begin",
                  "cp_end", "cp_ns", "cp_sum"]
 
@@ -28,7 +29,9 @@ OP_MASK = 1
 NODE_MASK = 62  # API, LAUNCH and the device kinds: what a critical path is made of
 
 
-def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(DEVICE_MASK,)):
+def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(DEVICE_MASK,),
+               op_work=None):
+    """op_work = (flops, bytes, peak_flops, peak_bw): also the operator efficiency step."""
     from oracle.ta_oracle import Oracle
     o = Oracle(events, win_off, t0, t1)
     r = {}
@@ -60,6 +63,10 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
         o.rollup()
         for k in ROLLUP_KEYS:
             r[k] = o.get(k)
+        if op_work is not None:
+            o.sol(*op_work)
+            for k in SOL_KEYS:
+                r[k] = o.get(k)
     o.blame()
     for k in BLAME_KEYS:
         r[k] = o.get(k)
@@ -80,7 +87,7 @@ def run_oracle(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_mask
 
 
 def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(DEVICE_MASK,),
-            on_device=True, use_torch_allocator=True):
+            on_device=True, use_torch_allocator=True, op_work=None):
     """Same analysis through the C ABI of the CUDA library (torch supplies memory + stream)."""
     import torch
     from paper_2609_40247_b200 import ta
@@ -120,6 +127,10 @@ def run_gpu(events, win_off, t0, t1, min_gap=500_000, comm_sizes=(), agg_masks=(
             ru = w.rollup_operators()
             for k in ROLLUP_KEYS:
                 r[k] = ru.numpy(k)
+            if op_work is not None:
+                so = w.operator_sol(*op_work)
+                for k in SOL_KEYS:
+                    r[k] = so.numpy(k)
         b = w.blame_gaps(g)
         for k in BLAME_KEYS:
             r[k] = b.numpy(k)

@@ -1,5 +1,7 @@
 """Pins the CPU oracle to brute-force twins of the definitions (tests/brute.py)
 on random tiny adversarial windows: quadratic scans and tick bitmaps."""
+from fractions import Fraction
+
 import numpy as np
 import pytest
 
@@ -424,3 +426,47 @@ def test_critical_path_of_a_tight_schedule_is_the_longest_path(seed):
         assert int(r["cp_reason"][i]) == 0 and int(r["cp_begin"][i]) == g["first"]
         assert int(r["cp_end"][i]) - int(r["cp_begin"][i]) == longest == int(ns.sum())
         assert ns[3] == 0 and ns[4] == 0
+
+
+@pytest.mark.parametrize("seed", SEEDS[:6])
+def test_operator_sol_against_exact_rationals(seed):
+    """The efficiency step against the definition evaluated in exact rational arithmetic: each
+    double must lie within a few units in the last place of the exact quotient (two roundings
+    in the denominator, one in the division); plus the identities the definition implies."""
+    ev, off, t0, t1, sizes = random_window(seed)
+    rng = np.random.default_rng(seed)
+    flops = rng.integers(0, 10**12, size=len(ev)).astype(np.float64)
+    nbytes = rng.integers(0, 10**9, size=len(ev)).astype(np.float64)
+    flops[rng.random(len(ev)) < 0.1] = -1.0
+    nbytes[rng.random(len(ev)) < 0.05] = np.nan
+    pf, pb = 2.25e15, 7.7e12
+    r = run_oracle(ev, off, t0, t1, op_work=(flops, nbytes, pf, pb))
+    if r["attr_status"] != 0:
+        pytest.skip("window without a legal operator nesting")
+    nv = r["n_valid"]
+    state, mfu, mbu, sol = brute.operator_sol(r["kind"][:nv], r["perm"], r["op_n_kernels"],
+                                              r["op_first_start"], r["op_last_end"], flops, nbytes, pf, pb)
+    assert r["sol_state"][:nv].tolist() == state and not r["sol_state"][nv:].any()
+    for got, want in ((r["sol_mfu"], mfu), (r["sol_mbu"], mbu), (r["sol_op"], sol)):
+        for p in range(nv):
+            assert abs(Fraction(float(got[p])) - want[p]) <= abs(want[p]) * Fraction(4, 2**53), p
+    res = r["sol_state"] == 1
+    assert (r["sol_op"] >= r["sol_mfu"]).all() and (r["sol_op"] >= r["sol_mbu"]).all()
+    assert ((r["sol_op"] == r["sol_mfu"]) | (r["sol_op"] == r["sol_mbu"])).all()
+    assert not r["sol_op"][~res].any() and not r["sol_mfu"][~res].any()
+    wins = np.searchsorted(np.asarray(off), r["perm"], side="right") - 1
+    for w in range(len(t0)):
+        s = r["sol_sum"][w]
+        m = res & (wins == w)
+        assert (s["n_resolved"], s["n_no_kernels"], s["n_no_counts"]) == \
+            (int(m.sum()), int(((r["sol_state"] == 2) & (wins == w)).sum()),
+             int(((r["sol_state"] == 3) & (wins == w)).sum()))
+        top = (r["op_last_end"] - r["op_first_start"])[m]
+        assert s["sum_top_ns"] == int(top.sum())
+        assert s["max_sol"] == (r["sol_op"][m].max() if m.any() else 0.0)
+        assert np.isclose(s["sum_flops"], flops[r["perm"][m]].sum(), rtol=1e-12)
+        assert np.isclose(s["sum_bytes"], nbytes[r["perm"][m]].sum(), rtol=1e-12)
+    # scaling laws that hold exactly in binary floating point: twice the work doubles the
+    # utilisation, twice the peak halves it
+    r2 = run_oracle(ev, off, t0, t1, op_work=(flops * 2, nbytes * 2, pf, pb * 2))
+    assert np.array_equal(r2["sol_mfu"], r["sol_mfu"] * 2) and np.array_equal(r2["sol_mbu"], r["sol_mbu"])
