@@ -20,7 +20,9 @@
  *     OWNED BY THE HANDLE (valid until ta_free) and host scalars.  Host-side
  *     per-window summary arrays are CALLER-OWNED, W entries, and are filled
  *     after one stream synchronisation at the end of the call.
- *   - Every kernel is enqueued on env.cuda_stream.
+ *   - Every kernel is enqueued on env.cuda_stream.  Every call that takes a
+ *     handle (and ta_load_window) makes env.device the current device of the
+ *     calling thread and leaves it current when it returns.
  *   - "Sorted position" p in [0, n) always means a position in the canonical
  *     order produced by ta_sort_timeline; every per-event output of the later
  *     calls is indexed by sorted position.
@@ -399,7 +401,7 @@ ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out);
  * out_summary[w]: number of such launches in window w, the device records they
  * own, and the most owned by one launch.
  * MFU, MBU and SOL_op of the same section need per-invocation operation counts
- * and device peaks that a 40-byte record does not carry; they are not computed.
+ * and device peaks that a 40-byte record does not carry: see ta_operator_sol.
  * All arrays are device memory owned by the handle, n entries each.
  * Errors: TA_ERR_ORDER unless ta_attribute_operators returned TA_OK;
  * TA_ERR_OOM; TA_ERR_CUDA.  One stream synchronisation at the end. */
@@ -415,6 +417,52 @@ typedef struct ta_rollup_result {
 
 ta_status ta_rollup_operators(ta_window *h, ta_rollup_result *out,
                               ta_rollup_summary *out_summary /* host, n_windows entries */);
+
+/* ------------------------------------------------------------------------
+ * ta_operator_sol - efficiency of every operator invocation (Sec. 6.1, "Operator
+ * execution and efficiency"): its theoretical operation count and its logical
+ * data volume, each normalised by T_op and by the device peak, are the model
+ * FLOPs utilisation and the model bandwidth utilisation; speed-of-light
+ * attainment is SOL_op = max(MFU, MBU).  Beyond the seven calls above.  Needs
+ * ta_attribute_operators to have returned TA_OK.  The only floating-point step
+ * of the library.
+ *
+ * The counts are the caller's: they follow from shapes, data types and sharding,
+ * which no trace record carries.  flops / bytes: n float64 each, indexed by INPUT
+ * record index (the order of `events`), in device memory if counts_on_device else
+ * in host memory (then copied first); read for OP records only; a negative value
+ * or a NaN means "not known".  Borrowed for the duration of the call.
+ * peak_flops in FLOP/s, peak_bw in bytes/s, both > 0 (else TA_ERR_INVALID_ARG).
+ * Per kept OP record at sorted position r with T_op = op_last_end - op_first_start:
+ *   state[r] = 2  op_n_kernels[r] == 0 or T_op == 0: no kernel composition, unresolved
+ *              3  kernels, but flops or bytes of the record is not known: unresolved
+ *              1  resolved:  mfu[r] = flops / (T_op * 1e-9 * peak_flops)
+ *                            mbu[r] = bytes / (T_op * 1e-9 * peak_bw)
+ *                            sol[r] = max(mfu[r], mbu[r])
+ * state = 0 at every other position; mfu = mbu = sol = 0 unless state = 1.
+ * out_summary[w]: the three state counts of window w; over its resolved
+ * invocations the sums of T_op (exact), flops and bytes, and the largest sol.
+ * Precision: IEEE double, the operations exactly as written above (two
+ * multiplications and one division per figure), so the per-record figures equal
+ * a plain CPU evaluation bit for bit; sum_flops and sum_bytes are accumulated in
+ * no particular order and agree with a sequential sum to a relative 1e-9 (the
+ * worst case of adding 10^7 positive doubles in another order).
+ * All arrays are device memory owned by the handle, n entries each.
+ * Errors: TA_ERR_ORDER unless ta_attribute_operators returned TA_OK;
+ * TA_ERR_INVALID_ARG; TA_ERR_OOM; TA_ERR_CUDA.  One stream synchronisation. */
+typedef struct ta_sol_summary {
+  int64_t n_resolved, n_no_kernels, n_no_counts, sum_top_ns;
+  double sum_flops, sum_bytes, max_sol;
+} ta_sol_summary;
+
+typedef struct ta_sol_result {
+  const double *mfu, *mbu, *sol; /* device, n each */
+  const uint8_t *state;          /* device, n      */
+} ta_sol_result;
+
+ta_status ta_operator_sol(ta_window *h, const double *flops, const double *bytes,
+                          int32_t counts_on_device, double peak_flops, double peak_bw,
+                          ta_sol_result *out, ta_sol_summary *out_summary /* host, n_windows entries */);
 
 /* ------------------------------------------------------------------------
  * ta_blame_gaps - why a device stream sat idle, and which host calls the idle

@@ -419,8 +419,8 @@ static ta_status ta_run_aggregate_sorted(ta_window *h, uint32_t kind_mask, int v
   AggSelOut so{c, k_in, v_in};
   TA_TRY((launch_scan<OpAdd, AggSelIn, AggSelOut>(h, nv, si, so, OpAdd(), s1)));
   u64 m64 = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, s1.total, 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  TA_TRY(ta_queue_d2h(h, &m64, s1.total, 8));
+  TA_TRY(ta_sync_fetch(h));
   const int64_t m = (int64_t)m64;
   if (m == 0) { ta_dfree(h, t1); return TA_OK; }
 
@@ -445,8 +445,8 @@ static ta_status ta_run_aggregate_sorted(ta_window *h, uint32_t kind_mask, int v
   AggHeadOut ho{gid, gstart};
   TA_TRY((launch_scan<OpAdd, AggHeadIn, AggHeadOut>(h, m, hi, ho, OpAdd(), s2)));
   u64 ng64 = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng64, s2.total, 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+  TA_TRY(ta_queue_d2h(h, &ng64, s2.total, 8));
+  TA_TRY(ta_sync_fetch(h));
   const int64_t ng = (int64_t)ng64;
 
   // 4. rows
@@ -526,8 +526,8 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
   if (!bounded) {
     const int64_t want = (G + 255) / 256;
     k_agg_count_rows<<<TA_N (unsigned)(want < 148 * 8 ? want : 148 * 8), 256, 0, st>>>(a.d_cnt, G, a.n_groups);
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, a.n_groups, 8, cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    TA_TRY(ta_queue_d2h(h, &ng, a.n_groups, 8));
+    TA_TRY(ta_sync_fetch(h));
     cap = ng;
   }
   u64 *scan_total = nullptr;
@@ -553,7 +553,7 @@ ta_status ta_run_aggregate(ta_window *h, uint32_t kind_mask, int value_sel, ta_a
     out->g_hist = ro.g_hist;
   }
   if (bounded && scan_total)  // the scan's total is the number of rows
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng, scan_total, 8, cudaMemcpyDeviceToHost, st));
+    TA_TRY(ta_queue_d2h(h, &ng, scan_total, 8));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   out->n_groups = (int64_t)ng;

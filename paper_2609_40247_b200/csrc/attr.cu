@@ -832,7 +832,7 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
     TA_CHECK_CUDA(h, cudaGetLastError());
   }
   std::vector<ta_attr_summary> hs(W);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hs.data(), d_sum, W * sizeof(ta_attr_summary), cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, hs.data(), d_sum, W * sizeof(ta_attr_summary)));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, tmpb);

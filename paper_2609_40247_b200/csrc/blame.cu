@@ -240,8 +240,8 @@ ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result 
   TA_CHECK_CUDA(h, cudaGetLastError());
 
   std::vector<u64> hc((size_t)W * 4), hn((size_t)W * 4);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hc.data(), a.win_count, (size_t)W * 32, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hn.data(), a.win_ns, (size_t)W * 32, cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, hc.data(), a.win_count, (size_t)W * 32));
+  TA_TRY(ta_queue_d2h(h, hn.data(), a.win_ns, (size_t)W * 32));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, tmpb);

@@ -73,7 +73,8 @@ struct CollHeadOut {
 
 struct CollGroupArgs {
   CollCtx c;
-  int64_t n_groups;
+  int64_t n_groups;          // rows allocated; the number of groups unless n_groups_dev is set
+  const u64 *n_groups_dev;   // device: the number of groups (the total of the head scan), or null
   const u64 *ks;
   const u32 *cs;
   const int32_t *gstart;
@@ -88,8 +89,9 @@ struct CollGroupArgs {
 __global__ void __launch_bounds__(256) k_coll_groups(CollGroupArgs a) {
   if (ta_failed(a.status)) return;
   int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= a.n_groups) return;
-  const int64_t b = a.gstart[g], e = g + 1 < a.n_groups ? (int64_t)a.gstart[g + 1] : a.c.m;
+  const int64_t n_groups = a.n_groups_dev ? (int64_t)*a.n_groups_dev : a.n_groups;
+  if (g >= n_groups) return;
+  const int64_t b = a.gstart[g], e = g + 1 < n_groups ? (int64_t)a.gstart[g + 1] : a.c.m;
   i64 mn = INT64_MAX, mx = INT64_MIN, me = INT64_MIN;
   int32_t strag = 0, strag_slot = 0, prev_pid = 0;
   int flags = 0;
@@ -218,23 +220,18 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   out->wait_ns = wait_ns;
   if (h->n_valid == 0 || h->n_comms == 0) return TA_OK;
 
-  // 1. compaction
-  size_t t1b = Carver::pad((size_t)nn * 4) + scan_temp_bytes(n) + 256;
+  // 1. compaction; the number of kept COLL records was counted while the records were loaded
+  const int64_t m = h->n_coll;
+  if (m == 0) return TA_OK;
+  size_t t1b = Carver::pad((size_t)m * 4) + scan_temp_bytes(n) + 256;
   void *t1 = ta_dalloc(h, t1b);
   if (!t1) return TA_ERR_OOM;
   Carver c1(t1);
-  u32 *pos_all = c1.take<u32>(nn);
+  u32 *pos_all = c1.take<u32>(m);
   ScanTemp s1;
   TA_TRY(scan_temp_init(h, c1.base + c1.off, n, &s1));
   TA_TRY(launch_compact_kind(h, h->sorted.kind, h->n_valid, 1u << TA_KIND_COLL, pos_all, s1));
-  u64 m64 = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, s1.total, 8, cudaMemcpyDeviceToHost, st));
-  std::vector<u64> comm_sorted(h->n_comms);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(comm_sorted.data(), h->d_comms->sorted_id, h->n_comms * 8,
-                                   cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-  const int64_t m = (int64_t)m64;
-  if (m == 0) { ta_dfree(h, t1); return TA_OK; }
+  const std::vector<u64> &comm_sorted = h->h_comm_sorted;
 
   // expected communicator sizes by rank
   std::vector<int32_t> expected(h->n_comms, -1);
@@ -286,10 +283,16 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   CollHeadIn hin{ks};
   CollHeadOut hout{cs, gid_of_c, gstart};
   TA_TRY((launch_scan<OpAdd, CollHeadIn, CollHeadOut>(h, m, hin, hout, OpAdd(), s2)));
+  // The group tables are sized by the number of groups when that is worth a round trip; while
+  // the bound "one group per COLL record" keeps them under 1 GiB they are sized by the bound
+  // and the count comes back with the call's one synchronisation.
   u64 ng64 = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&ng64, s2.total, 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-  const int64_t ng = (int64_t)ng64;
+  const bool bounded = (u64)m * 60 <= (1ull << 30);
+  if (!bounded) {
+    TA_TRY(ta_queue_d2h(h, &ng64, s2.total, 8));
+    TA_TRY(ta_sync_fetch(h));
+  }
+  const int64_t ng = bounded ? m : (int64_t)ng64;  // rows allocated (an upper bound when bounded)
 
   // 4. groups
   size_t ob = 5 * Carver::pad((size_t)ng * 4) + 5 * Carver::pad((size_t)ng * 8) + 256;
@@ -297,7 +300,7 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   if (!outb) return TA_ERR_OOM;
   Carver co(outb);
   CollGroupArgs ga;
-  ga.c = cx; ga.n_groups = ng; ga.ks = ks; ga.cs = cs; ga.gstart = gstart; ga.slot_of = slot_of;
+  ga.c = cx; ga.n_groups = ng; ga.n_groups_dev = bounded ? s2.total : nullptr; ga.ks = ks; ga.cs = cs; ga.gstart = gstart; ga.slot_of = slot_of;
   ga.expected = d_expected;
   ga.g_window = co.take<int32_t>(ng); ga.g_seq = co.take<int32_t>(ng); ga.g_n = co.take<int32_t>(ng);
   ga.g_strag = co.take<int32_t>(ng); ga.g_flags = co.take<int32_t>(ng);
@@ -330,14 +333,15 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   RankRowIn ri{r_seen};
   TA_TRY((launch_scan<OpAdd, RankRowIn, RankRowOut>(h, n_slots, ri, ro, OpAdd(), s3)));
   u64 nr64 = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&nr64, s3.total, 8, cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, &nr64, s3.total, 8));
+  if (bounded) TA_TRY(ta_queue_d2h(h, &ng64, s2.total, 8));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, t1);
   ta_dfree(h, t2);
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
 
-  out->n_groups = ng;
+  out->n_groups = (int64_t)ng64;
   out->n_ranks = (int64_t)nr64;
   out->g_window = ga.g_window; out->g_comm = ga.g_comm; out->g_seq = ga.g_seq; out->g_n_members = ga.g_n;
   out->g_min_start = ga.g_min; out->g_max_start = ga.g_max; out->g_skew = ga.g_skew;

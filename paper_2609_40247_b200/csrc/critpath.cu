@@ -771,8 +771,8 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
     TA_CHECK_CUDA(h, cudaGetLastError());
     // the waits that head a host run: a list whose length decides the number of doubling rounds
     u32 words2[2] = {0, 0};
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(words2, a.n_eff, 8, cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+    TA_TRY(ta_queue_d2h(h, words2, a.n_eff, 8));
+    TA_TRY(ta_sync_fetch(h));
     n_list = words2[0];
     if (!a.use_sort && words2[1]) continue;
     break;
@@ -806,8 +806,8 @@ ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_sum
   TA_TRY((launch_scan<OpAdd, CpRowIn, CpRowOut>(h, n_slots, ri, ro, OpAdd(), s3)));
   u64 rows = 0;
   std::vector<u64> hacc((size_t)n_slots * CP_ACC);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&rows, s3.total, 8, cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hacc.data(), a.acc, hacc.size() * 8, cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, &rows, s3.total, 8));
+  TA_TRY(ta_queue_d2h(h, hacc.data(), a.acc, hacc.size() * 8));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, lb);

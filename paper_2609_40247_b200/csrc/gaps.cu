@@ -358,7 +358,7 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
     if (tiles > 0) k_gaps<<<TA_N (unsigned)tiles, GP_THREADS, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
     u64 two[3] = {0, 0, 0};
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(two, scal, 24, cudaMemcpyDeviceToHost, st));
+    TA_TRY(ta_queue_d2h(h, two, scal, 24));
     TA_TRY(ta_read_status(h, words));
     if (words[ST_ERR]) return (ta_status)words[ST_ERR];
     n_long = two[0];
@@ -398,10 +398,13 @@ ta_status ta_run_gaps(ta_window *h, int64_t min_gap, ta_gap_result *out) {
                                cs.base + cs.off));
     k_gap_list_gather<<<TA_N (unsigned)((m + 255) / 256), 256, 0, st>>>(ulist, order, m, list, h->d_status);
     TA_CHECK_CUDA(h, cudaGetLastError());
-    TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
-    ta_dfree(h, stb);
+    // the sort and the gather are still queued: their temporaries go back after the handle's
+    // next synchronisation (the list itself is used in stream order like every other result)
+    ta_dfree_later(h, stb);
+    ta_dfree_later(h, lt);
+    lt = nullptr;
   }
-  ta_dfree(h, lt);
+  if (lt) ta_dfree(h, lt);
   out->gap_before = gap_before;
   out->lane_gaps = lane_gaps;
   out->lane_hist = lane_hist;

@@ -459,8 +459,8 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
                                  (1u << TA_KIND_LAUNCH) | (1u << TA_KIND_KERNEL) | (1u << TA_KIND_MEMCPY),
                                  pos, t1));
       u64 m64 = 0;
-      TA_CHECK_CUDA(h, cudaMemcpyAsync(&m64, t1.total, 8, cudaMemcpyDeviceToHost, st));
-      TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+      TA_TRY(ta_queue_d2h(h, &m64, t1.total, 8));
+      TA_TRY(ta_sync_fetch(h));
       const int64_t m = (int64_t)m64;
       TA_CHECK_CUDA(h, cudaMemsetAsync(found, 0xFF, nn * 4, st));
       if (m > 0) {
@@ -487,7 +487,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
     }
     TA_CHECK_CUDA(h, cudaGetLastError());
   }
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hs.data(), d_sum, W * sizeof(ta_join_summary), cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, hs.data(), d_sum, W * sizeof(ta_join_summary)));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   if (tmp_alloc) ta_dfree(h, tmp_alloc);

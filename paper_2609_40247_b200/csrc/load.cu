@@ -44,6 +44,7 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
   if (threadIdx.x < 64) ccache[threadIdx.x] = TRIPLE_EMPTY;
   __syncthreads();
   i64 mn = INT64_MAX, mx = INT64_MIN, md = 0, qmn = INT64_MAX, qmx = INT64_MIN;
+  u64 n_coll = 0;  // kept COLL records: sizes the collective matching without a count round trip
   WindowWalker ww(off, W);
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n;
        i += (int64_t)gridDim.x * blockDim.x) {
@@ -61,6 +62,7 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
     mx = max(mx, (i64)r.name);
     md = max(md, r.ts_end - r.ts_start);
     if (r.kind == TA_KIND_COLL) {  // communicator set and sequence range
+      n_coll++;
       qmn = min(qmn, (i64)r.seq);
       qmx = max(qmx, (i64)r.seq);
       u64 cc = (u64)r.corr ^ (1ull << 63);
@@ -110,9 +112,11 @@ __global__ void __launch_bounds__(256) k_discover(const ta_event *ev, int64_t n,
   md = warp_max_i64(md);
   qmn = warp_min_i64(qmn);
   qmx = warp_max_i64(qmx);
+  n_coll = warp_reduce(n_coll, OpAdd());
   if ((threadIdx.x & 31) == 0 && qmn != INT64_MAX) {
     atomicMin((i64 *)&misc[3], qmn);
     atomicMax((i64 *)&misc[4], qmx);
+    atomicAdd((u64 *)&misc[5], n_coll);
   }
   if ((threadIdx.x & 31) == 0) {
     if (mn != INT64_MAX) {

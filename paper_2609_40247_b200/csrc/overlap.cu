@@ -332,7 +332,7 @@ ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out) {
   OvRowIn ri{sa.acc};
   TA_TRY((launch_scan<OpAdd, OvRowIn, OvRowOut>(h, n_slots, ri, ro, OpAdd(), s3)));
   u64 rows = 0;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(&rows, s3.total, 8, cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, &rows, s3.total, 8));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   ta_dfree(h, tmpb);

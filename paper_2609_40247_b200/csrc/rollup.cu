@@ -187,7 +187,7 @@ ta_status ta_run_rollup(ta_window *h, ta_rollup_result *out, ta_rollup_summary *
   k_roll_finalize<<<TA_N tiles, RO_THREADS, 0, st>>>(a);
   TA_CHECK_CUDA(h, cudaGetLastError());
   std::vector<u64> hs((size_t)W * 3);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(hs.data(), a.win_sum, (size_t)W * 24, cudaMemcpyDeviceToHost, st));
+  TA_TRY(ta_queue_d2h(h, hs.data(), a.win_sum, (size_t)W * 24));
   int32_t words[ST_WORDS];
   TA_TRY(ta_read_status(h, words));
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];

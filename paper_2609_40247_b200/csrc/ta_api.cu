@@ -129,10 +129,82 @@ void ta_dfree(ta_window *h, void *p) {
     }
 }
 
+// Page-locked staging blocks are expensive to create (a system call and a page-table update
+// each), so they are kept for the life of the process and handed from handle to handle.
+#define TA_PIN_BYTES (512u << 10)
+static std::mutex g_pin_guard;
+static std::vector<unsigned char *> g_pin_free;
+static unsigned char *pin_take() {
+  {
+    std::lock_guard<std::mutex> lock(g_pin_guard);
+    if (!g_pin_free.empty()) {
+      unsigned char *p = g_pin_free.back();
+      g_pin_free.pop_back();
+      return p;
+    }
+  }
+  void *p = nullptr;
+  if (cudaHostAlloc(&p, TA_PIN_BYTES, cudaHostAllocPortable) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;  // the copies then go straight to their (pageable) destinations
+  }
+  return (unsigned char *)p;
+}
+static void pin_put(unsigned char *p) {
+  if (!p) return;
+  std::lock_guard<std::mutex> lock(g_pin_guard);
+  g_pin_free.push_back(p);
+}
+
+ta_status ta_queue_d2h(ta_window *h, void *dst, const void *dev_src, size_t bytes) {
+  if (bytes == 0) return TA_OK;
+  const size_t need = (bytes + 15) & ~(size_t)15;
+  if (h->pin && h->pin_used + need <= h->pin_bytes) {
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->pin + h->pin_used, dev_src, bytes, cudaMemcpyDeviceToHost, h->stream));
+    h->pending.push_back(ta_window::Pending{dst, h->pin_used, bytes});
+    h->pin_used += need;
+  } else {
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(dst, dev_src, bytes, cudaMemcpyDeviceToHost, h->stream));
+  }
+  return TA_OK;
+}
+
+static void release_one(ta_window *h, void *p, size_t bytes);
+
+ta_status ta_sync_fetch(ta_window *h) {
+  const cudaError_t e = cudaStreamSynchronize(h->stream);
+  if (e == cudaSuccess)
+    for (const ta_window::Pending &q : h->pending) memcpy(q.dst, h->pin + q.off, q.bytes);
+  h->pending.clear();
+  h->pin_used = 0;
+  if (e != cudaSuccess) {
+    h->last_cuda = e;
+    return TA_ERR_CUDA;
+  }
+  for (void *p : h->deferred) ta_dfree(h, p);
+  h->deferred.clear();
+  return TA_OK;
+}
+
 ta_status ta_read_status(ta_window *h, int32_t *w) {
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(w, h->d_status, ST_WORDS * sizeof(int32_t),
-                                   cudaMemcpyDeviceToHost, h->stream));
-  TA_CHECK_CUDA(h, cudaStreamSynchronize(h->stream));
+  TA_TRY(ta_queue_d2h(h, w, h->d_status, ST_WORDS * sizeof(int32_t)));
+  return ta_sync_fetch(h);
+}
+
+void ta_dfree_later(ta_window *h, void *p) {
+  if (p) h->deferred.push_back(p);
+}
+
+// Start of every entry point: copies an earlier call queued and never collected (it returned
+// early with an error) must not be delivered to destinations that no longer exist.
+// Also makes the handle's device current (it stays current when the call returns).
+static ta_status begin_call(ta_window *h) {
+  h->pending.clear();
+  h->pin_used = 0;
+  if (cudaSetDevice(h->device) != cudaSuccess) {
+    h->last_cuda = cudaGetLastError();
+    return TA_ERR_CUDA;
+  }
   return TA_OK;
 }
 
@@ -253,21 +325,29 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   const int64_t n = h->n;
   const int W = h->W;
   cudaStream_t st = h->stream;
-  size_t bytes = 3 * Carver::pad((W + 1) * 8) + Carver::pad(ST_WORDS * 4) +
-                 Carver::pad(sizeof(TripleTable)) + Carver::pad(sizeof(CommTable)) + Carver::pad(16 * 8) +
+  // one device block: [off | t0 | t1 | misc] filled by one copy, [status | load summaries |
+  // digit histograms] zeroed by one fill, [triple table | communicator table] emptied (all
+  // ones) by one fill
+  const size_t up_words = (size_t)(W + 1) + 2 * (size_t)W + 16;
+  size_t bytes = Carver::pad(up_words * 8) + Carver::pad(ST_WORDS * 4) +
+                 Carver::pad(sizeof(TripleTable)) + Carver::pad(sizeof(CommTable)) +
                  Carver::pad(W * sizeof(ta_load_summary)) + Carver::pad(10 * 256 * 4) + 256;
   void *b = ta_dalloc(h, bytes);
   if (!b) return TA_ERR_OOM;
   Carver c(b);
-  h->d_off = c.take<int64_t>(W + 1);
-  h->d_t0 = c.take<int64_t>(W + 1);
-  h->d_t1 = c.take<int64_t>(W + 1);
+  int64_t *up = c.take<int64_t>(up_words);
+  h->d_off = up;
+  h->d_t0 = up + (W + 1);
+  h->d_t1 = h->d_t0 + W;
+  h->d_misc = h->d_t1 + W;
+  char *zero_begin = c.base + c.off;
   h->d_status = c.take<int32_t>(ST_WORDS);
-  h->d_triples = c.take<TripleTable>(1);
-  h->d_comms = c.take<CommTable>(1);
-  h->d_misc = c.take<int64_t>(16);
   h->d_load_sum = c.take<ta_load_summary>(W);
   h->d_hist = c.take<u32>(10 * 256);
+  char *zero_end = c.base + c.off;
+  h->d_triples = c.take<TripleTable>(1);
+  h->d_comms = c.take<CommTable>(1);
+  char *ones_end = c.base + c.off;
   h->d_keys = (u64 *)ta_dalloc(h, (size_t)(n > 0 ? n : 1) * 8);
   if (!h->d_keys) return TA_ERR_OOM;
 
@@ -281,33 +361,34 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   } else {
     h->events = events;
   }
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_off, h->h_off.data(), (W + 1) * 8, cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t0, h->h_t0.data(), W * 8, cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_t1, h->h_t1.data(), W * 8, cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_status, 0, ST_WORDS * 4, st));
+  {
+    std::vector<int64_t> host(up_words, 0);
+    memcpy(host.data(), h->h_off.data(), (size_t)(W + 1) * 8);
+    memcpy(host.data() + (W + 1), h->h_t0.data(), (size_t)W * 8);
+    memcpy(host.data() + (W + 1) + W, h->h_t1.data(), (size_t)W * 8);
+    int64_t *misc_init = host.data() + (W + 1) + 2 * (size_t)W;
+    misc_init[0] = INT64_MAX;  // min name
+    misc_init[1] = INT64_MIN;  // max name
+    misc_init[3] = INT64_MAX;  // min seq
+    misc_init[4] = INT64_MIN;  // max seq
+    // a pageable source is staged by the runtime before the call returns
+    TA_CHECK_CUDA(h, cudaMemcpyAsync(up, host.data(), up_words * 8, cudaMemcpyHostToDevice, st));
+  }
+  TA_CHECK_CUDA(h, cudaMemsetAsync(zero_begin, 0, zero_end - zero_begin, st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(zero_end, 0xFF, ones_end - zero_end, st));
   const int32_t spin = g_ta_spin_limit.load();
-  if (spin > 0)  // staged by the runtime before the call returns (pageable source)
+  if (spin > 0)
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_status + ST_SPIN, &spin, sizeof(spin), cudaMemcpyHostToDevice, st));
-  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_triples->slots, 0xFF, sizeof(h->d_triples->slots), st));
-  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_comms->slots, 0xFF, sizeof(h->d_comms->slots), st));
-  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_load_sum, 0, W * sizeof(ta_load_summary), st));
-  TA_CHECK_CUDA(h, cudaMemsetAsync(h->d_hist, 0, 10 * 256 * 4, st));
-  int64_t misc_init[16] = {0};
-  misc_init[0] = INT64_MAX;
-  misc_init[1] = INT64_MIN;
-  misc_init[2] = 0;
-  misc_init[3] = INT64_MAX;
-  misc_init[4] = INT64_MIN;
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_misc, misc_init, sizeof(misc_init), cudaMemcpyHostToDevice, st));
 
   TA_TRY(ta_launch_discover(h));
 
   int32_t words[ST_WORDS];
   int64_t misc[16];
   std::vector<ta_load_summary> sums(W);
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(misc, h->d_misc, sizeof(misc), cudaMemcpyDeviceToHost, st));
-  TA_CHECK_CUDA(h, cudaMemcpyAsync(sums.data(), h->d_load_sum, W * sizeof(ta_load_summary),
-                                   cudaMemcpyDeviceToHost, st));
+  h->h_comm_sorted.assign(TA_MAX_COMMS, 0);
+  TA_TRY(ta_queue_d2h(h, misc, h->d_misc, sizeof(misc)));
+  TA_TRY(ta_queue_d2h(h, sums.data(), h->d_load_sum, W * sizeof(ta_load_summary)));
+  TA_TRY(ta_queue_d2h(h, h->h_comm_sorted.data(), h->d_comms->sorted_id, TA_MAX_COMMS * sizeof(u64)));
   TA_TRY(ta_read_status(h, words));
   if (words[ST_ERR]) return (ta_status)words[ST_ERR];
   h->n_triples = words[ST_N_TRIPLES];
@@ -317,7 +398,9 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   h->max_dur = misc[2];
   h->min_seq = misc[3];
   h->max_seq = misc[4];
+  h->n_coll = misc[5];
   h->n_comms = words[ST_N_COMMS];
+  h->h_comm_sorted.resize((size_t)h->n_comms);
   h->n_valid = 0;
   for (int w = 0; w < W; w++) {
     ta_load_summary &s = sums[w];
@@ -364,20 +447,22 @@ ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
   h->attr_status = 0;
   h->d_op_gap_ns = nullptr;
   h->d_on_path = nullptr;
+  h->d_status = nullptr;
+  h->pin = pin_take();
+  h->pin_bytes = h->pin ? TA_PIN_BYTES : 0;
+  h->pin_used = 0;
   h->h_off.assign(win_off, win_off + W + 1);
   h->h_t0.assign(win_t0, win_t0 + W);
   h->h_t1.assign(win_t1, win_t1 + W);
   *handle = h;
-  if (cudaSetDevice(h->device) != cudaSuccess) {
-    h->last_cuda = cudaGetLastError();
-    return TA_ERR_CUDA;
-  }
+  TA_TRY(begin_call(h));
   return load_impl(h, events, events_on_device, out_summary);
 }
 
 ta_status ta_sort_timeline(ta_window *h, ta_sort_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 1) || (h->stage & 2)) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   TA_TRY(ta_run_sort_timeline(h));
   h->stage |= 2;
   *out = h->sorted;
@@ -387,6 +472,7 @@ ta_status ta_sort_timeline(ta_window *h, ta_sort_result *out) {
 ta_status ta_correlate_launches(ta_window *h, ta_join_result *out, ta_join_summary *out_summary) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2) || (h->stage & 4)) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   TA_TRY(ta_run_correlate(h, out_summary));
   h->stage |= 4;
   *out = h->join;
@@ -396,6 +482,7 @@ ta_status ta_correlate_launches(ta_window *h, ta_join_result *out, ta_join_summa
 ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out, ta_attr_summary *out_summary) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 4) || (h->stage & 8)) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   ta_status s = ta_run_attribute(h, out_summary);
   if (s != TA_OK && s != TA_ERR_DEPTH && s != TA_ERR_BAD_NESTING) return s;
   h->stage |= 8;
@@ -407,6 +494,7 @@ ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out, ta_attr_summ
 ta_status ta_stream_gaps(ta_window *h, int64_t min_gap_ns, ta_gap_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   return ta_run_gaps(h, min_gap_ns, out);
 }
 
@@ -418,6 +506,7 @@ ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel, 
   if (value_sel == 1 && (!(h->stage & 8) || h->attr_status != 0)) return TA_ERR_ORDER;
   if (value_sel == 2 && !h->d_op_gap_ns) return TA_ERR_ORDER;
   if (value_sel == 3 && !h->d_on_path) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   return ta_run_aggregate(h, kind_mask, value_sel, out);
 }
 
@@ -425,17 +514,25 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes, int32_t 
                                ta_coll_result *out) {
   if (!h || !out || n_comms < 0 || (n_comms > 0 && !sizes)) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
   return ta_run_collectives(h, sizes, n_comms, out);
 }
 
 ta_status ta_rollup_operators(ta_window *h, ta_rollup_result *out, ta_rollup_summary *out_summary) {
   if (!h || !out || !out_summary) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 8) || h->attr_status != 0) return TA_ERR_ORDER;
-  if (cudaSetDevice(h->device) != cudaSuccess) {
-    h->last_cuda = cudaGetLastError();
-    return TA_ERR_CUDA;
-  }
+  TA_TRY(begin_call(h));
   return ta_run_rollup(h, out, out_summary);
+}
+
+ta_status ta_operator_sol(ta_window *h, const double *flops, const double *bytes,
+                          int32_t counts_on_device, double peak_flops, double peak_bw,
+                          ta_sol_result *out, ta_sol_summary *out_summary) {
+  if (!h || !out || !out_summary || (h->n > 0 && (!flops || !bytes))) return TA_ERR_INVALID_ARG;
+  if (!(peak_flops > 0.0) || !(peak_bw > 0.0)) return TA_ERR_INVALID_ARG;
+  if (!(h->stage & 8) || h->attr_status != 0) return TA_ERR_ORDER;
+  TA_TRY(begin_call(h));
+  return ta_run_sol(h, flops, bytes, counts_on_device, peak_flops, peak_bw, out, out_summary);
 }
 
 ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
@@ -443,30 +540,21 @@ ta_status ta_blame_gaps(ta_window *h, const ta_gap_result *gaps, ta_blame_result
   if (!h || !gaps || !out || !out_summary) return TA_ERR_INVALID_ARG;
   if (gaps->n_long_gaps < 0 || (gaps->n_long_gaps > 0 && !gaps->long_gaps)) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 4)) return TA_ERR_ORDER;
-  if (cudaSetDevice(h->device) != cudaSuccess) {
-    h->last_cuda = cudaGetLastError();
-    return TA_ERR_CUDA;
-  }
+  TA_TRY(begin_call(h));
   return ta_run_blame(h, gaps, out, out_summary);
 }
 
 ta_status ta_critical_path(ta_window *h, ta_critpath_result *out, ta_critpath_summary *out_summary) {
   if (!h || !out || !out_summary) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 4)) return TA_ERR_ORDER;
-  if (cudaSetDevice(h->device) != cudaSuccess) {
-    h->last_cuda = cudaGetLastError();
-    return TA_ERR_CUDA;
-  }
+  TA_TRY(begin_call(h));
   return ta_run_critpath(h, out, out_summary);
 }
 
 ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out) {
   if (!h || !out) return TA_ERR_INVALID_ARG;
   if (!(h->stage & 2)) return TA_ERR_ORDER;
-  if (cudaSetDevice(h->device) != cudaSuccess) {
-    h->last_cuda = cudaGetLastError();
-    return TA_ERR_CUDA;
-  }
+  TA_TRY(begin_call(h));
   return ta_run_overlap(h, out);
 }
 
@@ -477,6 +565,7 @@ void ta_free(ta_window *h) {
   for (size_t i = 0; i < h->allocs.size(); i++) release_one(h, h->allocs[i], h->alloc_bytes[i]);
   h->allocs.clear();
   h->alloc_bytes.clear();
+  pin_put(h->pin);
   const bool own = !h->env.alloc;
   delete h;
   if (own) cache_age();

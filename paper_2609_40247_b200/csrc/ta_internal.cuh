@@ -68,14 +68,25 @@ struct ta_window {
 
   std::vector<void *> allocs;  // everything obtained from env.alloc (or the library's own pool)
   std::vector<size_t> alloc_bytes;  // their sizes, same order
+  std::vector<void *> deferred;  // temporaries to release after the next synchronisation
+
+  // device -> host results of the call in progress: copies are queued into one page-locked
+  // staging block (truly asynchronous, unlike a copy into pageable memory, which blocks until
+  // it is done) and handed to their destinations after the call's one synchronisation
+  unsigned char *pin;
+  size_t pin_bytes, pin_used;
+  struct Pending { void *dst; size_t off, bytes; };
+  std::vector<Pending> pending;
 
   // load products
   int32_t *d_status;
   TripleTable *d_triples;
-  int64_t *d_misc;           // [0]=min name,[1]=max name,[2]=max duration,[3]=min seq,[4]=max seq
+  int64_t *d_misc;           // [0]=min name,[1]=max name,[2]=max duration,[3]=min seq,[4]=max seq,
+                             // [5]=kept COLL records
   CommTable *d_comms;
   int n_comms;
-  int64_t min_seq, max_seq;
+  std::vector<u64> h_comm_sorted;  // host copy of the ranked communicator ids (biased)
+  int64_t min_seq, max_seq, n_coll;
   ta_load_summary *d_load_sum;
   u64 *d_keys;
   int prekeys;               // d_keys holds the words of the discovery pass, not keys yet
@@ -178,6 +189,9 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
 ta_status ta_run_overlap(ta_window *h, ta_overlap_result *out);
 // rollup.cu
 ta_status ta_run_rollup(ta_window *h, ta_rollup_result *out, ta_rollup_summary *out_summary);
+// sol.cu
+ta_status ta_run_sol(ta_window *h, const double *flops, const double *bytes, int on_device,
+                     double peak_flops, double peak_bw, ta_sol_result *out, ta_sol_summary *out_summary);
 // blame.cu
 ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result *out,
                        ta_blame_summary *out_summary);
@@ -185,7 +199,15 @@ ta_status ta_run_blame(ta_window *h, const ta_gap_result *gaps, ta_blame_result 
 // critpath.cu
 ta_status ta_run_critpath(ta_window *h, ta_critpath_result *out, ta_critpath_summary *out_summary);
 
+// Queues a device -> host copy of the call in progress; *dst is valid after the next
+// ta_read_status / ta_sync_fetch.
+ta_status ta_queue_d2h(ta_window *h, void *dst, const void *dev_src, size_t bytes);
+// One stream synchronisation: delivers the queued copies and releases deferred temporaries.
+ta_status ta_sync_fetch(ta_window *h);
+// The same, with the device status words.
 ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
+// Releases a temporary that queued work may still use: after the next synchronisation.
+void ta_dfree_later(ta_window *h, void *p);
 
 // ---- instrumentation (no work: a launch counter and optional event pairs) ----
 extern std::atomic<long long> g_ta_launches;  // kernels launched by this library since load

@@ -314,7 +314,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   // result buffers (kept until ta_free)
   size_t keep = Carver::pad(n * 4) + 3 * Carver::pad(n * 8) + 3 * Carver::pad(n * 4) +
                 2 * Carver::pad(n * 2) + 7 * Carver::pad(lane_cap * 4) + 2 * Carver::pad(lane_cap * 2) +
-                Carver::pad((lane_cap + 1) * 4) + 2 * Carver::pad((size_t)n_slots * 8) + 512;
+                Carver::pad((lane_cap + 1) * 4) + Carver::pad((size_t)n_slots * 16) + 512;
   void *kb = ta_dalloc(h, keep);
   if (!kb) return TA_ERR_OOM;
   Carver ck(kb);
@@ -330,8 +330,8 @@ ta_status ta_run_sort_timeline(ta_window *h) {
   int32_t *lane_dev_base = ck.take<int32_t>(lane_cap);
   int32_t *lane_dom_next = ck.take<int32_t>(lane_cap);
   int32_t *n_lanes_dev = ck.take<int32_t>(2);  // [0] lanes, [1] device records
-  h->d_slot_min = ck.take<i64>(n_slots);
-  h->d_slot_max = ck.take<i64>(n_slots);
+  h->d_slot_min = ck.take<i64>(2 * n_slots);  // minima, then maxima, contiguous
+  h->d_slot_max = h->d_slot_min + n_slots;
 
   // temporaries (released at the end of the call)
   size_t tmp_bytes = 2 * Carver::pad(n * 8) + Carver::pad(n * 4) + ta_sort_temp_bytes(n) +
@@ -352,8 +352,11 @@ ta_status ta_run_sort_timeline(ta_window *h) {
     int32_t words[ST_WORDS];
     h->h_slot_min.assign((size_t)n_slots, INT64_MAX);
     h->h_slot_max.assign((size_t)n_slots, INT64_MIN);
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_min, h->h_slot_min.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_max, h->h_slot_max.data(), n_slots * 8, cudaMemcpyHostToDevice, st));
+    {  // the two ranges sit side by side on the device: one copy
+      std::vector<int64_t> init(h->h_slot_min);
+      init.insert(init.end(), h->h_slot_max.begin(), h->h_slot_max.end());
+      TA_CHECK_CUDA(h, cudaMemcpyAsync(h->d_slot_min, init.data(), 2 * n_slots * 8, cudaMemcpyHostToDevice, st));
+    }
     TA_CHECK_CUDA(h, cudaMemsetAsync(lane_start, 0xFF, n_codes * sizeof(int32_t), st));
     if (n > 0) {
       if (h->packed) {
@@ -394,7 +397,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
           k_gather_u64<<<TA_N nblk(n, 256), 256, 0, st>>>(h->d_keys, dorder, n, dkeys, h->d_status);
           TA_TRY(ta_radix_sort_pairs(h, dkeys, dorder, kscr, vscr, skeys, perm, n, h->plan, nullptr,
                                      sort_tmp));
-          TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+          TA_TRY(ta_sync_fetch(h));
           ta_dfree(h, xb);
         }
       }
@@ -422,7 +425,7 @@ ta_status ta_run_sort_timeline(ta_window *h) {
         if (cur != perm + h->n_valid)
           TA_CHECK_CUDA(h, cudaMemcpyAsync(perm + h->n_valid, cur, m * sizeof(u32),
                                            cudaMemcpyDeviceToDevice, st));
-        TA_CHECK_CUDA(h, cudaStreamSynchronize(st));
+        TA_TRY(ta_sync_fetch(h));
         ta_dfree(h, xb);
       }
       // step 4
@@ -443,9 +446,9 @@ ta_status ta_run_sort_timeline(ta_window *h) {
                                      lane_code, lane_slot, lane_dom_end, lane_dom_next, lane_dev_base, n_lanes_dev,
                                      lane_cap, h->d_status);
     TA_CHECK_CUDA(h, cudaGetLastError());
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(n_lanes_host, n_lanes_dev, 2 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_min.data(), h->d_slot_min, n_slots * 8, cudaMemcpyDeviceToHost, st));
-    TA_CHECK_CUDA(h, cudaMemcpyAsync(h->h_slot_max.data(), h->d_slot_max, n_slots * 8, cudaMemcpyDeviceToHost, st));
+    TA_TRY(ta_queue_d2h(h, n_lanes_host, n_lanes_dev, 2 * sizeof(int32_t)));
+    TA_TRY(ta_queue_d2h(h, h->h_slot_min.data(), h->d_slot_min, n_slots * 8));
+    TA_TRY(ta_queue_d2h(h, h->h_slot_max.data(), h->d_slot_max, n_slots * 8));
     TA_TRY(ta_read_status(h, words));
     if (words[ST_ERR]) return (ta_status)words[ST_ERR];
     if (!words[ST_LONG_RUN]) break;

@@ -86,6 +86,7 @@ _RollupResult = _ptr_struct("_RollupResult", [
     ("replay_first_start", _vp), ("replay_last_end", _vp), ("replay_kernel_ns", _vp)])
 _BlameResult = _ptr_struct("_BlameResult", [
     ("n_long_gaps", ctypes.c_int64), ("g_class", _vp), ("g_launch", _vp), ("op_gap_ns", _vp)])
+_SolResult = _ptr_struct("_SolResult", [("mfu", _vp), ("mbu", _vp), ("sol", _vp), ("state", _vp)])
 _OverlapResult = _ptr_struct("_OverlapResult", [
     ("n_rows", ctypes.c_int64), ("d_window", _vp), ("d_pid", _vp), ("d_n_events", _vp),
     ("d_busy", _vp), ("d_idle", _vp), ("d_compute", _vp), ("d_comm", _vp), ("d_overlap", _vp),
@@ -100,7 +101,7 @@ EXPORTS = ["ta_load_window", "ta_sort_timeline", "ta_correlate_launches", "ta_at
            "ta_version", "ta_launch_count", "ta_profile_enable", "ta_profile_radix",
            "ta_lane_gaps_noalloc", "ta_device_overlap", "ta_blame_gaps",
            "ta_rollup_operators", "ta_critical_path", "ta_set_spin_limit",
-           "ta_selftest_wait_timeout", "ta_inject_device_error"]
+           "ta_selftest_wait_timeout", "ta_inject_device_error", "ta_operator_sol"]
 NOALLOC_MAX_RECORDS = 1 << 22
 
 _lib = None
@@ -143,6 +144,9 @@ def lib():
         L.ta_critical_path.argtypes = [_vp, ctypes.POINTER(_CritpathResult), _vp]
         L.ta_blame_gaps.restype = ctypes.c_int
         L.ta_blame_gaps.argtypes = [_vp, _vp, ctypes.POINTER(_BlameResult), _vp]
+        L.ta_operator_sol.restype = ctypes.c_int
+        L.ta_operator_sol.argtypes = [_vp, _vp, _vp, ctypes.c_int32, ctypes.c_double, ctypes.c_double,
+                                      ctypes.POINTER(_SolResult), _vp]
         L.ta_device_overlap.restype = ctypes.c_int
         L.ta_device_overlap.argtypes = [_vp, ctypes.POINTER(_OverlapResult)]
         L.ta_free.restype = None
@@ -410,6 +414,27 @@ class BlameResult(_Result):
         return super().tensor(self._names.get(name, name))
 
 
+SOL_SUM = np.dtype([("n_resolved", "<i8"), ("n_no_kernels", "<i8"), ("n_no_counts", "<i8"),
+                    ("sum_top_ns", "<i8"), ("sum_flops", "<f8"), ("sum_bytes", "<f8"),
+                    ("max_sol", "<f8")])
+
+
+class SolResult(_Result):
+    """Per sorted position: sol_mfu, sol_mbu, sol_op (float64), sol_state (uint8); sol_sum per
+    window (SOL_SUM)."""
+    _names = {"sol_mfu": "mfu", "sol_mbu": "mbu", "sol_op": "sol", "sol_state": "state"}
+    _layout = {"mfu": ("<f8", lambda r: r.n), "mbu": ("<f8", lambda r: r.n),
+               "sol": ("<f8", lambda r: r.n), "state": ("|u1", lambda r: r.n)}
+
+    def numpy(self, name):
+        if name == "sol_sum":
+            return self.sol_sum
+        return super().numpy(self._names.get(name, name))
+
+    def tensor(self, name):
+        return super().tensor(self._names.get(name, name))
+
+
 class OverlapResult(_Result):
     _layout = dict([("d_window", ("<i4", lambda r: r.n_rows)), ("d_pid", ("<i4", lambda r: r.n_rows))] +
                    [(k, ("<i8", lambda r: r.n_rows)) for k in
@@ -582,6 +607,30 @@ class Window:
         if st != 0:
             raise TaError(st, "ta_blame_gaps")
         return BlameResult(self, raw, dict(self._dims(), n_long_gaps=raw.n_long_gaps, blame_sum=summ))
+
+    def operator_sol(self, flops, nbytes, peak_flops: float, peak_bw: float) -> SolResult:
+        """flops / nbytes: float64 per INPUT record (numpy arrays, or CUDA tensors on this
+        window's device); negative or NaN = not known."""
+        raw = _SolResult()
+        summ = np.zeros(self.W, dtype=SOL_SUM)
+        on_device = hasattr(flops, "is_cuda")
+        if on_device:
+            import torch
+            if not (flops.is_cuda and nbytes.is_cuda and flops.dtype == torch.float64
+                    and nbytes.dtype == torch.float64 and flops.is_contiguous() and nbytes.is_contiguous()):
+                raise ValueError("counts must be contiguous float64 CUDA tensors")
+            fp, bp, cnt = flops.data_ptr(), nbytes.data_ptr(), (flops.numel(), nbytes.numel())
+        else:
+            flops = np.ascontiguousarray(flops, dtype=np.float64)
+            nbytes = np.ascontiguousarray(nbytes, dtype=np.float64)
+            fp, bp, cnt = flops.ctypes.data, nbytes.ctypes.data, (len(flops), len(nbytes))
+        if cnt != (self.n, self.n):
+            raise ValueError("one operation count and one data volume per input record")
+        st = self._lib.ta_operator_sol(self._h, fp, bp, 1 if on_device else 0, float(peak_flops),
+                                       float(peak_bw), ctypes.byref(raw), summ.ctypes.data)
+        if st != 0:
+            raise TaError(st, "ta_operator_sol")
+        return SolResult(self, raw, dict(self._dims(), sol_sum=summ))
 
     def device_overlap(self) -> OverlapResult:
         raw = _OverlapResult()

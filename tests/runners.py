@@ -155,6 +155,16 @@ def assert_same(a, b, skip=()):
         if k in skip or k not in b:
             continue
         x, y = a[k], b[k]
+        if k == "sol_sum":
+            # the two float sums are accumulated in no particular order on the GPU; everything
+            # else in the row (counts, the exact T_op sum, the maximum) is compared exactly
+            assert x.dtype == y.dtype and x.shape == y.shape
+            for f in x.dtype.names:
+                if f in ("sum_flops", "sum_bytes"):
+                    assert np.allclose(x[f], y[f], rtol=1e-9, atol=0), (k, f)
+                else:
+                    assert np.array_equal(x[f], y[f]), (k, f)
+            continue
         if isinstance(x, np.ndarray):
             assert x.dtype == y.dtype, (k, x.dtype, y.dtype)
             assert x.shape == y.shape, (k, x.shape, y.shape)

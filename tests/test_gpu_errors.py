@@ -153,7 +153,7 @@ def test_a_failed_handle_fails_every_later_call_and_frees():
                 calls.append(lambda: w.blame_gaps(g))
             got = [_status(c) for c in calls]
             assert set(got) <= {TA_ERR_TIMEOUT, TA_ERR_ORDER}, got
-            assert got.count(TA_ERR_TIMEOUT) >= 2
+            assert got.count(TA_ERR_TIMEOUT) >= (1 if after == 0 else 3), got
     torch.cuda.synchronize()
     a = (wl.events, wl.win_off, wl.win_t0, wl.win_t1)
     assert_same(run_oracle(*a, comm_sizes=wl.comm_sizes), run_gpu(*a, comm_sizes=wl.comm_sizes))

@@ -111,8 +111,16 @@ def test_c1_c2_full_size_whole(cfg):
     wl = synth.make_workload(cfg, 1.0, truth=False)
     ev = wl.events
     assert len(ev) > (2**22 - 2**18 if cfg == "c1" else 2**24 - 2**20)
-    o = run_oracle(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=MIN_GAP, comm_sizes=wl.comm_sizes)
-    g = run_gpu(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=MIN_GAP, comm_sizes=wl.comm_sizes)
+    # c2 holds a million stalls of 0.5 to 5 ms; the oracle's gap blame intersects every operator
+    # with every long gap of its process, so only the longest one percent go on the list here
+    # (every gap still enters gap_before, the lane figures and the histograms)
+    min_gap = MIN_GAP if cfg == "c1" else 4_950_000
+    work = synth.op_work(ev, seed=11) + (synth.PEAK_FLOPS, synth.PEAK_BW)
+    o = run_oracle(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=min_gap, comm_sizes=wl.comm_sizes,
+                   op_work=work)
+    g = run_gpu(ev, wl.win_off, wl.win_t0, wl.win_t1, min_gap=min_gap, comm_sizes=wl.comm_sizes,
+                op_work=work)
+    assert len(o["long_gaps"]) > 1000
     assert o["attr_status"] == 0 and int(o["attr_sum"]["max_depth"].max()) == (8 if cfg == "c2" else 3)
     assert_same(o, g)
 

@@ -191,6 +191,23 @@ CASES = [("c0", 1.0, 0), ("c0", 1.0, 1), ("c1", 0.1, 0), ("c1", 0.03, 1), ("c2",
 @pytest.mark.parametrize("name,scale,shuffle", CASES)
 def test_scaled_workloads(name, scale, shuffle):
     wl = synth.make_workload(name, scale, shuffle_mode=shuffle, n_windows=9 if name == "c4" else None)
+    flops, nbytes = synth.op_work(wl.events, seed=7)
     o, g = both(wl.events, wl.win_off, wl.win_t0, wl.win_t1, min_gap=500_000,
-                comm_sizes=wl.comm_sizes)
+                comm_sizes=wl.comm_sizes, op_work=(flops, nbytes, synth.PEAK_FLOPS, synth.PEAK_BW))
+    assert int((o["sol_state"] == 1).sum()) > 100 and int((o["sol_state"] == 3).sum()) > 0
     check_against_truth(wl, g)
+
+
+def test_operator_sol_counts_on_the_device_and_unknown_counts():
+    """The side table as CUDA tensors (no copy inside the call), NaN and negative counts, a
+    window batch (the warp fold meets window boundaries)."""
+    import torch
+    wl = synth.make_workload("c4", 0.002, truth=False, n_windows=9)
+    flops, nbytes = synth.op_work(wl.events, seed=3, unknown_frac=0.2)
+    nbytes[::7] = np.nan
+    args = (wl.events, wl.win_off, wl.win_t0, wl.win_t1)
+    o = run_oracle(*args, comm_sizes=wl.comm_sizes, op_work=(flops, nbytes, 1e15, 5e12))
+    g = run_gpu(*args, comm_sizes=wl.comm_sizes,
+                op_work=(torch.from_numpy(flops).cuda(), torch.from_numpy(nbytes).cuda(), 1e15, 5e12))
+    assert_same(o, g)
+    assert int(o["sol_sum"]["n_no_counts"].sum()) > 100
