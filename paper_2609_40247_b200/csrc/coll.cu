@@ -30,13 +30,6 @@ struct CollCtx {
   int qbits, cbits;
 };
 
-__device__ __forceinline__ u32 coll_hash(u64 c) {
-  c ^= c >> 29;
-  c *= 0xBF58476D1CE4E5B9ull;
-  c ^= c >> 32;
-  return (u32)c;
-}
-
 __global__ void __launch_bounds__(256) k_coll_keys(CollCtx c, u64 *keys, int32_t *slot_of, int32_t *status) {
   if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -45,7 +38,7 @@ __global__ void __launch_bounds__(256) k_coll_keys(CollCtx c, u64 *keys, int32_t
   int lane = lane_of_pos(c.lane_off, c.n_lanes, p);
   u64 cc = (u64)c.corr[p] ^ (1ull << 63);
   // every communicator id was inserted while the records were loaded: a bounded probe all the same
-  u32 s = coll_hash(cc) & (TA_COMM_SLOTS - 1);
+  u32 s = hash_code(cc) & (TA_COMM_SLOTS - 1);
   int probes = 0;
   while (c.cm->slots[s] != cc && ++probes < TA_COMM_SLOTS) s = (s + 1) & (TA_COMM_SLOTS - 1);
   u64 rank = 0;

@@ -35,13 +35,6 @@ __device__ __forceinline__ int32_t code_pid(u64 c) { return (int32_t)((u32)(c >>
 __device__ __forceinline__ int16_t code_domain(u64 c) { return (int16_t)((c >> 16) & 1); }
 __device__ __forceinline__ int16_t code_stream(u64 c) { return (int16_t)((uint16_t)(c & 0xFFFF) ^ 0x8000u); }
 
-__device__ __forceinline__ u32 hash_code(u64 c) {
-  c ^= c >> 29;
-  c *= 0xBF58476D1CE4E5B9ull;
-  c ^= c >> 32;
-  return (u32)c;
-}
-
 __device__ __forceinline__ int window_of(const int64_t *off, int W, int64_t i) {
   if (W == 1) return 0;
   int lo = 0, hi = W - 1;

@@ -33,7 +33,25 @@ struct RadixArgs {
   u64 *tile_state;        // [tile][RS_BINS]
   u32 *tile_counter;
   int32_t *status;
+  PrekeyInfo pk;          // PREKEY passes only
 };
+
+// Discovery word of input record i ([dropped][triple slot, 13 bits][ts_start - t0, 40 bits]) ->
+// packed key [dropped][window][triple rank][(ts_start - t0) >> dshift][index inside the window].
+#define RS_PRE_DROPPED (1ull << 63)
+#define RS_PRE_TS_BITS 40
+__device__ __forceinline__ u64 prekey_to_key(const PrekeyInfo &k, u64 w64, int w, int64_t i) {
+  u64 hi;
+  if (w64 & RS_PRE_DROPPED) {
+    hi = (1ull << (k.wbits + k.tbits + k.tsb)) | ((u64)w << (k.tbits + k.tsb));
+  } else {
+    const u32 slot = (u32)(w64 >> RS_PRE_TS_BITS) & (TA_TRIPLE_SLOTS - 1);
+    const u64 rank = (u64)__ldg(&k.rank_of_slot[slot]);
+    hi = ((u64)w << (k.tbits + k.tsb)) | (rank << k.tsb) |
+         ((w64 & ((1ull << RS_PRE_TS_BITS) - 1)) >> k.dshift);
+  }
+  return (hi << k.ibits) | (u64)(i - k.off[w]);
+}
 
 template <int THREADS, int ITEMS>
 struct RadixSmem {
@@ -43,12 +61,13 @@ struct RadixSmem {
   u64 scan_tmp[33];
   int tile;
   int fail;
+  int win0;  // PREKEY passes: window of the tile's first record
 };
 
 // STABLE = false: equal digits may leave the pass in any order (one shared-memory atomic per
 // key instead of the vote ranking).  Only legal for the FIRST pass of a sort whose caller
 // does not rely on the input order of keys that are equal in all sorted bits.
-template <int THREADS, int ITEMS, bool VALS, int BITS, bool FULL, bool STABLE>
+template <int THREADS, int ITEMS, bool VALS, int BITS, bool FULL, bool STABLE, bool PREKEY>
 __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS, ITEMS> &s, int tile,
                                            int count) {
   constexpr int TILE = THREADS * ITEMS;
@@ -65,6 +84,24 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   for (int j = 0; j < ITEMS; j++) {
     const int li = wbase + j * 32 + lane;
     key[j] = (FULL || li < count) ? a.keys_in[base + li] : ~0ull;
+  }
+  if (PREKEY) {
+    // the words are in input order: the tile's window range is short (usually one window); the
+    // window of the tile's first record comes from one search per CTA, each thread walks on
+    int w = s.win0;
+    int64_t next = a.pk.off[w + 1];
+#pragma unroll
+    for (int j = 0; j < ITEMS; j++) {
+      const int li = wbase + j * 32 + lane;  // grows with j: the walk only moves forward
+      if (FULL || li < count) {
+        const int64_t i = base + li;
+        while (i >= next) {  // also steps over empty windows; off[W] = n > i
+          w++;
+          next = a.pk.off[w + 1];
+        }
+        key[j] = prekey_to_key(a.pk, key[j], w, i);
+      }
+    }
   }
   // rank inside the warp, item row by item row (stable: row-major, then lane)
   u32 *wh = s.warp_hist[warp];
@@ -183,7 +220,7 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   }
 }
 
-template <int THREADS, int ITEMS, bool VALS, int BITS, bool STABLE>
+template <int THREADS, int ITEMS, bool VALS, int BITS, bool STABLE, bool PREKEY>
 __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_pass(RadixArgs a) {
   constexpr int TILE = THREADS * ITEMS;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -197,9 +234,22 @@ __global__ void __launch_bounds__(THREADS, VALS ? RSP_MINB : RSK_MINB) k_radix_p
   __syncthreads();
   if (s.fail) return;  // an earlier kernel failed: the keys may be incomplete
   const int tile = s.tile;
+  if (PREKEY) {
+    if (tid == 0) {
+      const int64_t first = (int64_t)tile * TILE;
+      int lo = 0, hi = a.pk.W - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (a.pk.off[mid] <= first) lo = mid;
+        else hi = mid - 1;
+      }
+      s.win0 = lo;
+    }
+    __syncthreads();
+  }
   const int count = (int)min((int64_t)TILE, a.n - (int64_t)tile * TILE);
-  if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true, STABLE>(a, s, tile, count);
-  else radix_tile<THREADS, ITEMS, VALS, BITS, false, STABLE>(a, s, tile, count);
+  if (count == TILE) radix_tile<THREADS, ITEMS, VALS, BITS, true, STABLE, PREKEY>(a, s, tile, count);
+  else radix_tile<THREADS, ITEMS, VALS, BITS, false, STABLE, PREKEY>(a, s, tile, count);
 }
 
 // tile shapes
@@ -239,20 +289,7 @@ __global__ void __launch_bounds__(256) k_radix_scan_hist(const u32 *hist, u32 *b
   bin_offset[blockIdx.x * RS_BINS + threadIdx.x] = (u32)ex;
 }
 
-SortPlan ta_make_plan(int lo_bit, int hi_bit) {
-  SortPlan p;
-  int total = hi_bit - lo_bit;
-  if (total < 1) total = 1;
-  p.n_pass = (total + 7) / 8;
-  int b = lo_bit;
-  for (int i = 0; i < p.n_pass; i++) {
-    int w = (total - (b - lo_bit) + (p.n_pass - i) - 1) / (p.n_pass - i);  // spread bits evenly
-    p.shift[i] = b;
-    p.bits[i] = w;
-    b += w;
-  }
-  return p;
-}
+SortPlan ta_make_plan(int lo_bit, int hi_bit) { return ta_plan_bits(lo_bit, hi_bit); }
 
 static size_t min_tile() {
   size_t a = (size_t)RSP_THREADS * RSP_ITEMS, b = (size_t)RSK_THREADS * RSK_ITEMS;
@@ -266,12 +303,12 @@ size_t ta_sort_temp_bytes(int64_t n) {
          2 * Carver::pad(10 * RS_BINS * sizeof(u32));
 }
 
-template <int THREADS, int ITEMS, bool VALS, bool STABLE>
+template <int THREADS, int ITEMS, bool VALS, bool STABLE, bool PREKEY = false>
 static cudaError_t launch_pass(const RadixArgs &a, int bits, unsigned tiles, cudaStream_t st) {
   typedef RadixSmem<THREADS, ITEMS> Smem;
 #define RS_CASE(B)                                                                                  \
   case B: {                                                                                         \
-    auto kern = k_radix_pass<THREADS, ITEMS, VALS, B, STABLE>;                                      \
+    auto kern = k_radix_pass<THREADS, ITEMS, VALS, B, STABLE, PREKEY>;                                     \
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
                                          (int)sizeof(Smem));                                        \
     if (e != cudaSuccess) return e;                                                                 \
@@ -294,7 +331,7 @@ template <bool VALS>
 static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in, u64 *keys_scratch,
                             u32 *vals_scratch, u64 *keys_final, u32 *vals_final, int64_t n,
                             const SortPlan &plan, const u32 *hist, void *temp,
-                            bool first_pass_unstable) {
+                            bool first_pass_unstable, const PrekeyInfo *prekey) {
   if (n <= 0) return TA_OK;
   constexpr int THREADS = VALS ? RSP_THREADS : RSK_THREADS;
   constexpr int ITEMS = VALS ? RSP_ITEMS : RSK_ITEMS;
@@ -321,7 +358,7 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     bool to_final = ((plan.n_pass - 1 - p) & 1) == 0;
     TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * RS_BINS * sizeof(u64), st));
     TA_CHECK_CUDA(h, cudaMemsetAsync(counter, 0, sizeof(u32), st));
-    RadixArgs a;
+    RadixArgs a = RadixArgs();
     a.keys_in = kin; a.keys_out = to_final ? keys_final : keys_scratch;
     a.vals_in = vin; a.vals_out = to_final ? vals_final : vals_scratch;
     a.n = n; a.shift = plan.shift[p];
@@ -329,9 +366,19 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
     if (timed) ta_profile_mark(st, 1, (VALS ? 24.0 : 16.0) * (double)n);
-    if (!VALS && p == 0 && first_pass_unstable)
-      TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, false, false>(a, plan.bits[p], (unsigned)tiles, st)));
-    else
+    bool launched = false;
+    if constexpr (!VALS) {
+      if (p == 0 && first_pass_unstable) {
+        if (prekey) {
+          a.pk = *prekey;
+          TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, false, false, true>(a, plan.bits[p], (unsigned)tiles, st)));
+        } else {
+          TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, false, false>(a, plan.bits[p], (unsigned)tiles, st)));
+        }
+        launched = true;
+      }
+    }
+    if (!launched)
       TA_CHECK_CUDA(h, (launch_pass<THREADS, ITEMS, VALS, true>(a, plan.bits[p], (unsigned)tiles, st)));
     if (timed) ta_profile_mark(st, 0, 0.0);
     kin = a.keys_out;
@@ -346,12 +393,12 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
                               u32 *vals_final, int64_t n, const SortPlan &plan, const u32 *hist,
                               void *temp) {
   return radix_sort<true>(h, keys_in, vals_in, keys_scratch, vals_scratch, keys_final, vals_final, n,
-                          plan, hist, temp, false);
+                          plan, hist, temp, false, nullptr);
 }
 
 ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
                              int64_t n, const SortPlan &plan, const u32 *hist, void *temp,
-                             bool first_pass_unstable) {
+                             bool first_pass_unstable, const PrekeyInfo *prekey) {
   return radix_sort<false>(h, keys_in, nullptr, keys_scratch, nullptr, keys_final, nullptr, n, plan,
-                           hist, temp, first_pass_unstable);
+                           hist, temp, first_pass_unstable, prekey);
 }

@@ -331,7 +331,8 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   const size_t up_words = (size_t)(W + 1) + 2 * (size_t)W + 16;
   size_t bytes = Carver::pad(up_words * 8) + Carver::pad(ST_WORDS * 4) +
                  Carver::pad(sizeof(TripleTable)) + Carver::pad(sizeof(CommTable)) +
-                 Carver::pad(W * sizeof(ta_load_summary)) + Carver::pad(10 * 256 * 4) + 256;
+                 Carver::pad(W * sizeof(ta_load_summary)) + Carver::pad(10 * 256 * 4) +
+                 Carver::pad(TA_TRIPLE_SLOTS * 4) + 256;
   void *b = ta_dalloc(h, bytes);
   if (!b) return TA_ERR_OOM;
   Carver c(b);
@@ -344,6 +345,7 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   h->d_status = c.take<int32_t>(ST_WORDS);
   h->d_load_sum = c.take<ta_load_summary>(W);
   h->d_hist = c.take<u32>(10 * 256);
+  h->d_slot_cnt = c.take<u32>(TA_TRIPLE_SLOTS);
   char *zero_end = c.base + c.off;
   h->d_triples = c.take<TripleTable>(1);
   h->d_comms = c.take<CommTable>(1);
@@ -399,6 +401,7 @@ static ta_status load_impl(ta_window *h, const ta_event *events, int32_t on_devi
   h->min_seq = misc[3];
   h->max_seq = misc[4];
   h->n_coll = misc[5];
+  if (h->tkeep < 0) h->tkeep = (int)misc[6];
   h->n_comms = words[ST_N_COMMS];
   h->h_comm_sorted.resize((size_t)h->n_comms);
   h->n_valid = 0;

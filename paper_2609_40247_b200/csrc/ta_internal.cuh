@@ -50,6 +50,26 @@ struct SortPlan {
   int shift[10];
   int bits[10];
 };
+// Passes over key bits [lo_bit, hi_bit): as few digits of at most 8 bits as cover them, the
+// bits spread evenly.  Host and device build the same plan from the same two numbers.
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+static inline SortPlan ta_plan_bits(int lo_bit, int hi_bit) {
+  SortPlan p;
+  int total = hi_bit - lo_bit;
+  if (total < 1) total = 1;
+  p.n_pass = (total + 7) / 8;
+  int b = lo_bit;
+  for (int i = 0; i < 10; i++) { p.shift[i] = 0; p.bits[i] = 0; }
+  for (int i = 0; i < p.n_pass; i++) {
+    const int w = (total - (b - lo_bit) + (p.n_pass - i) - 1) / (p.n_pass - i);
+    p.shift[i] = b;
+    p.bits[i] = w;
+    b += w;
+  }
+  return p;
+}
 
 // --------------------------------------------------------------- handle
 struct ta_window {
@@ -95,6 +115,9 @@ struct ta_window {
   int n_triples, n_pids;
   int sbits, tbits, wbits, has_dropped;
   int packed, dshift, ibits;   // packed keys: low ibits = index inside the window, dshift low time bits dropped
+  int tkeep;                   // time bits the planning kernel decided to keep (0 = it did not run)
+  int fast_keys;               // the first radix pass builds the keys from the discovery words itself
+  u32 *d_slot_cnt;             // kept records per triple slot (one window only), or null
   int64_t min_name, max_name, max_dur;
   SortPlan plan;
 
@@ -162,10 +185,17 @@ ta_status ta_radix_sort_pairs(ta_window *h, const u64 *keys_in, const u32 *vals_
                               u64 *keys_scratch, u32 *vals_scratch, u64 *keys_final,
                               u32 *vals_final, int64_t n, const SortPlan &plan,
                               const u32 *hist /*nullable*/, void *temp);
+// How the first pass of the timeline sort turns a discovery word into a key on the fly.
+struct PrekeyInfo {
+  const int64_t *off;          // window offsets (device), W + 1
+  int W;
+  const int32_t *rank_of_slot; // triple slot -> rank
+  int tbits, wbits, tsb, dshift, ibits;  // tsb = time bits kept
+};
 ta_status ta_radix_sort_keys(ta_window *h, const u64 *keys_in, u64 *keys_scratch, u64 *keys_final,
                              int64_t n, const SortPlan &plan, const u32 *hist /*nullable*/,
                              void *temp,
-                             bool first_pass_unstable);
+                             bool first_pass_unstable, const PrekeyInfo *prekey = nullptr);
 SortPlan ta_make_plan(int lo_bit, int hi_bit);
 // load.cu
 ta_status ta_launch_discover(ta_window *h);
@@ -377,6 +407,16 @@ __device__ __forceinline__ int lane_of_pos(const int32_t *lane_off, int n_lanes,
     else hi = mid - 1;
   }
   return lo;
+}
+
+// Hash of a triple code or a biased communicator id: 32-bit mixing of the two halves (the
+// tables it indexes hold a few dozen entries; a 64-bit multiply per record is not worth it).
+__device__ __forceinline__ u32 hash_code(u64 c) {
+  u32 h = (u32)c * 0x9E3779B1u ^ (u32)(c >> 32) * 0x85EBCA77u;
+  h ^= h >> 15;
+  h *= 0x2C1B3C6Du;
+  h ^= h >> 13;
+  return h;
 }
 
 __device__ __forceinline__ int log2_bin(int64_t v) {

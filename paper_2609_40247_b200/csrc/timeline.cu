@@ -362,7 +362,10 @@ ta_status ta_run_sort_timeline(ta_window *h) {
       if (h->packed) {
         // keys carry the index: 8-byte elements, fewer bytes per pass
         PackInfo pi{h->ibits, h->ibits + h->tbits + (h->sbits - h->dshift), h->wbits, h->d_off};
-        TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp, true));
+        PrekeyInfo pre{h->d_off, h->W, h->d_triples->rank_of_slot, h->tbits, h->wbits,
+                       h->sbits - h->dshift, h->dshift, h->ibits};
+        TA_TRY(ta_radix_sort_keys(h, h->d_keys, kscr, skeys, n, h->plan, h->d_hist, sort_tmp, true,
+                                  h->fast_keys ? &pre : nullptr));
         if (n > h->n_valid)
           k_unpack_tail<<<TA_N nblk(n - h->n_valid, 256), 256, 0, st>>>(skeys, h->n_valid, n, pi, perm,
                                                                             h->d_status);
