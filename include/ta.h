@@ -602,9 +602,13 @@ ta_status ta_critical_path(ta_window *h, ta_critpath_result *out,
  * first_start, last_end).  No histogram and no long-gap list.
  *
  * Limits and rules: n <= TA_NOALLOC_MAX_RECORDS, else TA_ERR_TOO_LARGE (the
- * fixed scratch covers no more).  The first call on a device looks up the
- * address of the scratch array (with that device current) and should therefore
- * be made before any stream capture begins.  All calls on a device share the
+ * fixed scratch covers no more).  gap_before and lane_out must be 8-byte aligned
+ * (lane_out receives 64-bit atomic updates).  The first call on a device looks
+ * up the address of the scratch array (with that device current) and should
+ * therefore be made before any stream capture begins; it is also the call at
+ * which the CUDA runtime may load the library's code and the scratch array onto
+ * the device (lazy module loading), which does take device memory: make it once
+ * at start-up, before the heap is reserved, not at the first moment of need.  All calls on a device share the
  * one scratch array, which keeps the previous call's contents; each call clears
  * it first, so two calls that overlap on the GPU (different streams or threads)
  * race and must be serialised by the caller.  The call enqueues its work on

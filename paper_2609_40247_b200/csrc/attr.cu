@@ -769,9 +769,10 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   int32_t *op_n = ck.take<int32_t>(nn);
   u64 *op_first = ck.take<u64>(nn), *op_last = ck.take<u64>(nn);
   int64_t *op_ns = ck.take<int64_t>(nn);
-  ta_attr_summary *d_sum = ck.take<ta_attr_summary>(W);
   char *zero_end = ck.base + ck.off;
+  ta_attr_summary *d_sum = ck.take<ta_attr_summary>(W);
   TA_CHECK_CUDA(h, cudaMemsetAsync(zero_begin, 0, zero_end - zero_begin, st));
+  TA_CHECK_CUDA(h, cudaMemsetAsync(d_sum, 0, (size_t)W * sizeof(ta_attr_summary), st));
 
   const int64_t tt = tiles > 0 ? tiles : 1;
   size_t tb = 2 * Carver::pad(tt * 4) + 2 * Carver::pad(tt * AT_CAP * 8) + 2 * Carver::pad(tt * AT_CAP * 4) + 256;

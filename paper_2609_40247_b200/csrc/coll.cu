@@ -211,11 +211,10 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   if (!wait_ns) return TA_ERR_OOM;
   TA_CHECK_CUDA(h, cudaMemsetAsync(wait_ns, 0, (size_t)nn * 8, st));
   out->wait_ns = wait_ns;
-  if (h->n_valid == 0 || h->n_comms == 0) return TA_OK;
+  const int64_t m = h->n_coll;  // kept COLL records, counted while the records were loaded
+  if (h->n_valid == 0 || h->n_comms == 0 || m == 0) return TA_OK;
 
-  // 1. compaction; the number of kept COLL records was counted while the records were loaded
-  const int64_t m = h->n_coll;
-  if (m == 0) return TA_OK;
+  // 1. compaction
   size_t t1b = Carver::pad((size_t)m * 4) + scan_temp_bytes(n) + 256;
   void *t1 = ta_dalloc(h, t1b);
   if (!t1) return TA_ERR_OOM;

@@ -239,6 +239,7 @@ ta_status ta_read_status(ta_window *h, int32_t *host_words /*ST_WORDS*/);
 // Releases a temporary that queued work may still use: after the next synchronisation.
 void ta_dfree_later(ta_window *h, void *p);
 
+
 // ---- instrumentation (no work: a launch counter and optional event pairs) ----
 extern std::atomic<long long> g_ta_launches;  // kernels launched by this library since load
 extern int g_ta_profile;          // 1 = record a CUDA event pair around each radix pass
