@@ -104,8 +104,9 @@ typedef struct ta_env {
 typedef struct ta_window ta_window; /* opaque handle; owns every result buffer */
 
 /* ------------------------------------------------------------------------
- * ta_load_window - ingest and validate (start-time filtering separates
- * successive windows, Sec. 5.2 "Session transitions").
+ * ta_load_window - ingest and validate.  A record belongs to a window by the time
+ * it starts (the rule the collection side uses when one recording session
+ * follows another, Sec. 5.2 "Session transitions").
  *
  * events   n records, device memory if events_on_device else host memory
  *          (then copied to the device first).  BORROWED: must stay alive and
@@ -163,8 +164,9 @@ typedef struct ta_sort_result {
 ta_status ta_sort_timeline(ta_window *h, ta_sort_result *out);
 
 /* ------------------------------------------------------------------------
- * ta_correlate_launches - correlation id associates submissions with device
- * activity (Sec. 5.2; Fig. "Key performance observations" (a)).
+ * ta_correlate_launches - joins every device record to the host call that
+ * submitted it, through the correlation id both carry (Sec. 5.2; Fig. "Key
+ * performance observations" (a)).
  *
  * Build side: kept LAUNCH records.  Probe side: kept KERNEL and MEMCPY
  * records.  Key = (window, pid, corr_id), all 64 bits of corr_id significant.
@@ -196,10 +198,12 @@ ta_status ta_correlate_launches(ta_window *h, ta_join_result *out,
                                 ta_join_summary *out_summary);
 
 /* ------------------------------------------------------------------------
- * ta_attribute_operators - thread id plus call intervals link host API calls
- * to the enclosing calls (Sec. 9.1); T_op spans the first kernel start to the
- * last completion (Sec. 6.1).  Device work can outlive the enclosing call
- * (Sec. 5.2), so containment is tested on the LAUNCH interval.
+ * ta_attribute_operators - finds, for every host record, the operator range of
+ * the same thread that contains it (the linkage of Sec. 9.1: same thread,
+ * nested intervals) and gives every device record the operator of its launch;
+ * per operator, T_op runs from the start of its first kernel to the end of its
+ * last (Sec. 6.1).  A kernel may still run after the call that launched it has
+ * returned (Sec. 5.2), so containment is tested on the LAUNCH interval.
  *
  * Inside one host lane, OP j ENCLOSES host record i (i != j) iff
  * ts_start[j] <= ts_start[i] and ts_end[i] <= ts_end[j] and, when both
@@ -239,7 +243,8 @@ ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out,
                                  ta_attr_summary *out_summary);
 
 /* ------------------------------------------------------------------------
- * ta_stream_gaps - device activity records reveal idle intervals (Sec. 9.1).
+ * ta_stream_gaps - where each device stream sat idle: the time not covered by
+ * any of its activity records (the idle-time observation of Sec. 9.1).
  *
  * For a device lane of a window [W0, W1) with records 0..m-1 in canonical
  * order and clipped ends c_i = min(ts_end_i, W1):
@@ -253,6 +258,7 @@ ta_status ta_attribute_operators(ta_window *h, ta_attr_result *out,
  * lanes are zero.  win_hist[w] sums the window's lanes.  The long-gap list
  * holds every gap with g > 0 and g >= min_gap_ns, ordered by lane, then time,
  * a lane's tail gap last.
+ * Limits: fewer than 2^22 - 1 lanes (TA_ERR_TOO_LARGE).
  */
 typedef struct ta_lane_gaps {
   int64_t busy, idle, n_events, n_gaps, max_gap, first_start, last_end;
@@ -308,9 +314,10 @@ ta_status ta_aggregate_ops(ta_window *h, uint32_t kind_mask, int32_t value_sel,
                            ta_agg_result *out);
 
 /* ------------------------------------------------------------------------
- * ta_match_collectives - cross-process links by shared identifiers; ranks
- * meet in collectives and a late rank leaves the others waiting (Sec. 6.1
- * "Execution progress and state", Sec. 9.2).
+ * ta_match_collectives - links the records of different processes that name the
+ * same collective (same communicator, same sequence number) and measures how
+ * long each rank waited for the last one to arrive (cross-process links:
+ * Sec. 6.1 "Execution progress and state"; ranks held up by a late one: Sec. 9.2).
  *
  * Population: kept COLL records; comm_id = corr_id.  Group key
  * (window, comm_id, seq), groups output in ascending signed key order.
@@ -351,10 +358,10 @@ ta_status ta_match_collectives(ta_window *h, const ta_comm_size *sizes,
                                int32_t n_comms, ta_coll_result *out);
 
 /* ------------------------------------------------------------------------
- * ta_device_overlap - device-level coverage per (window, process): from GPU
- * activity, communication hidden by computation is told apart from exposed
- * time, and exposed time is interval coverage (Sec. 6.1, "Execution progress
- * and state"; Fig. "Overlap and exposed work").  Beyond the seven calls above:
+ * ta_device_overlap - device-level coverage per (window, process): how much of
+ * the communication time ran while kernels were running too, and how much was
+ * left uncovered, both as measures of unions of intervals (Sec. 6.1, "Execution
+ * progress and state"; Fig. "Overlap and exposed work").  Beyond the seven calls above:
  * the first of the analyses that build on them.  Needs ta_sort_timeline only.
  *
  * For every (window, pid) that has at least one kept device record, over ALL of
@@ -383,10 +390,10 @@ ta_status ta_device_overlap(ta_window *h, ta_overlap_result *out);
 
 /* ------------------------------------------------------------------------
  * ta_rollup_operators - inclusive per-operator kernel figures and graph
- * replays.  An invocation's kernel composition comes from the call-to-kernel
- * links and T_op spans the first kernel start to the last completion; CUDA
- * Graph replay hides the operator calls and launch correlations separate the
- * replays (Sec. 6.1, "Operator execution and efficiency").  Beyond the seven
+ * replays.  Which kernels make up an operator invocation follows from the join
+ * and the attribution above; under CUDA Graph replay no operator call is
+ * recorded and the kernels of one replay are told apart only by the launch they
+ * share (Sec. 6.1, "Operator execution and efficiency").  Beyond the seven
  * calls above.  Needs ta_attribute_operators to have returned TA_OK.
  *
  * Readings.  For an OP at sorted position r, over r itself and every OP below it
@@ -465,11 +472,12 @@ ta_status ta_operator_sol(ta_window *h, const double *flops, const double *bytes
                           ta_sol_result *out, ta_sol_summary *out_summary /* host, n_windows entries */);
 
 /* ------------------------------------------------------------------------
- * ta_blame_gaps - why a device stream sat idle, and which host calls the idle
- * time coincides with.  For waits, readiness, dispatch and first use are
- * compared: ready work dispatched late implicates submission (Sec. 6.2, engine
- * patterns; "submission gaps", Sec. 8.2); waits in one host call are found to
- * coincide with the GPU idle time (Sec. 9.1).  Beyond the seven calls above.
+ * ta_blame_gaps - why a device stream sat idle, and which host calls were
+ * running meanwhile.  A gap is laid at the door of the host when the work that
+ * ended it had not even been submitted while the stream was already idle (the
+ * late-dispatch test of Sec. 6.2, engine patterns; "submission gaps", Sec. 8.2);
+ * idle time is charged to the operators it overlaps (the case of Sec. 9.1, where
+ * one waiting call accounts for most of the idle time).  Beyond the seven calls above.
  * Needs ta_correlate_launches and the result of a ta_stream_gaps call on the
  * same handle (`gaps`, borrowed for the duration of the call).
  *
@@ -514,9 +522,11 @@ void ta_free(ta_window *h);
 
 /* ------------------------------------------------------------------------
  * ta_critical_path - per (window, process), the chain of binding dependencies
- * that ends at the last record to finish.  Submission, execution-order and
- * synchronisation dependencies identify the critical path; where a dependency
- * is missing, the delay it would explain stays unresolved (Sec. 6.1, "Execution
+ * that ends at the last record to finish.  Three kinds of dependency are
+ * followed - a kernel on its launch, a record on the one before it in its
+ * stream or thread, a waiting host call on the device record that released it -
+ * and a delay for which the trace holds no such dependency is reported as
+ * unresolved rather than guessed (Sec. 6.1, "Execution
  * progress and state"; Fig. "Critical path": host work, the call that submits
  * k1, k1, the end of the host's wait, host work again - a kernel of another
  * stream and the wait itself stay off the path).  Beyond the seven calls above.

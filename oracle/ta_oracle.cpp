@@ -134,7 +134,7 @@ struct Oracle {
 
   bool is_kept(int64_t p) const { return p < n_valid; }
 
-  // ---- step 1: validity.  Start-time filtering separates successive windows
+  // ---- step 1: validity.  A record belongs to the window in which it starts
   // (Sec. 5.2).  Reading: the first failing rule counts; ts_end > t1 is legal.
   void load() {
     win_of.assign(n, 0);
@@ -198,8 +198,8 @@ struct Oracle {
     lane_off.push_back((int32_t)n_valid);
   }
 
-  // ---- step 3: correlation id associates submissions with device activity
-  // (Sec. 5.2; Fig. "Key performance observations" (a)).  Readings: the key is
+  // ---- step 3: a device record and the host call that submitted it carry the same
+  // correlation id (Sec. 5.2; Fig. "Key performance observations" (a)).  Readings: the key is
   // (window, pid, corr_id); the first LAUNCH in canonical order wins a key;
   // latency = kernel start - launch start; queue delay = the part of it after
   // the launch call returned; COLL records do not join.
@@ -252,9 +252,9 @@ struct Oracle {
         join_sum[win_sorted[p]].n_orphan_launch++;
   }
 
-  // ---- step 4: thread id plus call intervals link host API calls to the
-  // enclosing calls (Sec. 9.1); T_op spans the first kernel start to the last
-  // completion (Sec. 6.1); device work may outlive the enclosing call (Sec.
+  // ---- step 4: a host record lies in the operator ranges of its own thread whose
+  // intervals contain it (Sec. 9.1); T_op runs from the start of an operator's first
+  // kernel to the end of its last (Sec. 6.1); a kernel may outlive the call (Sec.
   // 5.2) so containment is tested on the launch interval.  The definition is
   // evaluated against every earlier OP of the lane that has not ended before
   // the record starts (an OP that ended earlier can enclose nothing later).
@@ -324,7 +324,7 @@ struct Oracle {
     return 0;
   }
 
-  // ---- step 5: device activity records reveal idle intervals (Sec. 9.1).
+  // ---- step 5: a stream is idle where none of its activity records covers (Sec. 9.1).
   // Readings: all three device kinds occupy the stream; ends are clipped to the
   // window; head and tail gaps are idle time and enter the histogram.
   void gaps(int64_t min_gap) {
@@ -409,8 +409,8 @@ struct Oracle {
     return 0;
   }
 
-  // ---- step 7: cross-process links by shared identifiers; ranks meet in
-  // collectives and a late rank leaves the others waiting (Sec. 6.1, Sec. 9.2).
+  // ---- step 7: records of different processes that name the same collective are
+  // linked; each rank waits for the last one to arrive (Sec. 6.1, Sec. 9.2).
   // Readings: arrival = the rank's ts_start; wait = time until the last arrival;
   // all pids share one clock; corr_id carries the communicator id.
   void collectives(const CommSize* sizes, int32_t n_comms) {
@@ -468,7 +468,8 @@ struct Oracle {
   // Readings: the inclusive figures of an OP are those of the OP itself plus those of every OP
   // below it in the parent forest (count and nanoseconds add; first start is the minimum and
   // last end the maximum over the OPs that own kernels; all zero when the subtree owns none).
-  // CUDA Graph replay hides the operator calls and launch correlations separate the replays:
+  // Under CUDA Graph replay no operator call is recorded; the launch they share tells the
+  // kernels of one replay apart (Sec. 6.1):
   // a LAUNCH that owns two or more device records is one replay, spanning the first start to
   // the last end of those records, with the sum of their durations; all zero for other launches.
   void rollup() {
@@ -549,10 +550,10 @@ struct Oracle {
     }
   }
 
-  // ---- gap blame (needs correlate() and gaps()).  For waits, readiness, dispatch and first
-  // use are compared: ready work dispatched late implicates submission (Sec. 6.2, engine
-  // patterns; "submission gaps", Sec. 8.2), and waits in a host call are matched with the
-  // device idle time they coincide with (Sec. 9.1: waits in one call coincide with 13.8 s of
+  // ---- gap blame (needs correlate() and gaps()).  A gap counts against the host when the
+  // work that ended it was submitted only after the stream had gone idle (the late-dispatch
+  // test of Sec. 6.2, engine patterns; "submission gaps", Sec. 8.2), and idle time is charged
+  // to the host calls that were running meanwhile (Sec. 9.1: one waiting call overlaps 13.8 s of
   // GPU idle).  Readings, per long gap of the list gaps() made:
   //   class 3 TAIL        the gap runs to the end of the window (no next record);
   //   class 0 NO_LAUNCH   the next record has no launch (a COLL record, or launch_of = -1);
@@ -599,9 +600,10 @@ struct Oracle {
     }
   }
 
-  // ---- critical path (needs correlate()).  Submission, execution-order and synchronisation
-  // dependencies identify the critical path; where a dependency is missing, the delay it would
-  // explain stays unresolved (Sec. 6.1, "Execution progress and state"; Fig. "Critical path":
+  // ---- critical path (needs correlate()).  Three kinds of dependency are followed (a kernel on
+  // its launch, a record on its predecessor in stream or thread, a waiting call on the device
+  // record that released it); a delay that none of them explains is reported as unresolved
+  // (Sec. 6.1, "Execution progress and state"; Fig. "Critical path":
   // host work, the API call that submits kernel k1, k1, the end of the host's wait, host work
   // again - kernel k2 of another stream and the wait itself are off the path).
   // Readings.  One path per (window, process).  Nodes are the valid API and LAUNCH records
@@ -711,8 +713,8 @@ struct Oracle {
     }
   }
 
-  // ---- device-level coverage: from GPU activity, communication hidden by computation is
-  // told apart from exposed time; exposed time is interval coverage (Sec. 6.1, "Execution
+  // ---- device-level coverage: how much communication time ran while kernels ran too and
+  // how much was left uncovered, as measures of unions of intervals (Sec. 6.1, "Execution
   // progress and state"; Fig. "Overlap and exposed work": a compute lane, a communication / IO
   // lane, their overlap, the exposed remainder).  Readings: per (window, process), over all
   // device streams; compute = KERNEL records, communication / IO = MEMCPY and COLL records;

@@ -1,6 +1,7 @@
-// ta_attribute_operators: thread id plus call intervals link host API calls to
-// the enclosing calls (Sec. 9.1); device records inherit the operator of their
-// launch; T_op spans the first kernel start to the last completion (Sec. 6.1).
+// ta_attribute_operators: every host record gets the operator range of its own
+// thread that contains it (same thread, nested intervals: the linkage of Sec. 9.1);
+// device records inherit the operator of their launch; per operator, T_op runs from
+// the start of its first kernel to the end of its last (Sec. 6.1).
 //
 // In canonical order (ts_start ascending, ts_end descending) a properly nested
 // host lane has a simple structure: the innermost encloser of record i is the

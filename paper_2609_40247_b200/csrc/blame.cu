@@ -1,7 +1,7 @@
 // ta_blame_gaps: why was a device stream idle, and which host calls did the idle
-// time coincide with.  For waits, readiness, dispatch and first use are compared:
-// ready work dispatched late implicates submission (Sec. 6.2); waits inside a
-// host call are matched with the GPU idle time they coincide with (Sec. 9.1).
+// time overlap.  A gap counts against the host when the work that ended it was
+// submitted only after the stream had gone idle (the late-dispatch test of Sec. 6.2);
+// idle time is charged to the operators that were running meanwhile (Sec. 9.1).
 //
 // Input: the long-gap list of ta_stream_gaps (ordered by lane, then time) and the
 // launch of every device record (ta_correlate_launches).

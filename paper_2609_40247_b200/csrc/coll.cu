@@ -1,6 +1,6 @@
-// ta_match_collectives: cross-process links by shared identifiers; ranks meet in
-// collectives and a late rank leaves the others waiting (Sec. 6.1 "Execution
-// progress and state", Sec. 9.2).  Group key (window, comm_id, seq).
+// ta_match_collectives: records of different processes that name the same collective
+// are linked, and every rank's wait for the last arrival is measured (cross-process
+// links: Sec. 6.1 "Execution progress and state"; ranks held up by a late one: Sec. 9.2).  Group key (window, comm_id, seq).
 //
 //   1. compact the COLL records (a few percent of the window), in sorted-
 //      position order, which is pid-major;

@@ -1,7 +1,8 @@
 // ta_critical_path: per (window, process) the chain of binding dependencies that ends
-// at the last record to finish.  Submission, execution-order and synchronisation
-// dependencies identify the critical path; where a dependency is missing the delay
-// stays unresolved (Sec. 6.1, "Execution progress and state"; Fig. "Critical path").
+// at the last record to finish.  Three kinds of dependency are followed (a kernel on
+// its launch, a record on its predecessor in the same stream or thread, a waiting call
+// on the device record that released it); a delay the trace explains by none of them
+// is reported as unresolved (Sec. 6.1, "Execution progress and state"; Fig. "Critical path").
 //
 // Nodes are the API / LAUNCH records of the host lanes and the records of the device
 // lanes; each has a START and an END point.  The path is the backward walk from the END

@@ -1,7 +1,7 @@
 // ta_stream_gaps: per device lane, the running maximum of the clipped end times
 // (an exclusive max-scan in canonical order) gives the gap before every record,
 // the busy union, idle time, a log2 gap histogram and the list of long gaps.
-// Device activity records reveal idle intervals (Sec. 9.1).
+// Idle time of a stream = what none of its activity records covers (Sec. 9.1).
 //
 // One pass over the sorted ts_start / ts_end / kind columns.  The scan is made
 // lane-aware without segment flags: the scanned value is (lane + 1) << 40 |

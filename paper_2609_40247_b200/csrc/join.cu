@@ -1,5 +1,6 @@
-// ta_correlate_launches: correlation id associates submissions with device
-// activity (Sec. 5.2; Fig. "Key performance observations" (a)).  Key =
+// ta_correlate_launches: every device record is joined to the host call that
+// submitted it through the correlation id both carry (Sec. 5.2; Fig. "Key
+// performance observations" (a)).  Key =
 // (window, pid, corr_id); the smallest sorted position among equal LAUNCH keys
 // wins.
 //

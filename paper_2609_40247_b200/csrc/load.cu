@@ -1,5 +1,5 @@
-// ta_load_window kernels: validity (start-time filtering separates windows,
-// Sec. 5.2), discovery and dense ranking of the (pid, domain, stream) triples
+// ta_load_window kernels: validity (a record belongs to the window in which it
+// starts, Sec. 5.2), discovery and dense ranking of the (pid, domain, stream) triples
 // that name a lane, and the 64-bit sort key together with the digit histograms
 // of every radix pass.
 //   k_plan          one CTA samples the records and decides how many time bits the packed

@@ -1,7 +1,7 @@
 // ta_device_overlap: per (window, process), over ALL device streams, the time the
 // device was busy, the time covered by computation (KERNEL) and by communication /
 // IO (MEMCPY, COLL), how much of the communication was hidden under computation and
-// how much stayed exposed.  Exposed time is interval coverage (Sec. 6.1, "Execution
+// how much stayed exposed, all as measures of unions of intervals (Sec. 6.1, "Execution
 // progress and state"; Fig. "Overlap and exposed work").
 //
 // The measure of a union of intervals taken in start order is

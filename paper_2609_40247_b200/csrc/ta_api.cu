@@ -67,7 +67,10 @@ static void cache_put(int device, cudaStream_t stream, void *p, size_t bytes) {
   std::lock_guard<std::mutex> lock(g_cache_guard);
   g_cache.push_back(CachedBlock{p, bytes, device, stream, g_cache_gen});
 }
-// called when a handle goes away (its stream is idle): ages the cache
+// Called when a handle goes away, after its stream has been synchronised.  Invariant: a block
+// enters the cache only once the stream it was used on is idle (ta_dfree and ta_free are only
+// reached behind a synchronisation), so handing it back to the pool below cannot race with work
+// still queued on that stream - cudaFree itself does not wait for a stream-ordered allocation.
 static void cache_age() {
   std::vector<void *> out;
   {
@@ -83,7 +86,7 @@ static void cache_age() {
       }
     }
   }
-  for (void *p : out) cudaFree(p);  // synchronising free: the stream of the block may be gone
+  for (void *p : out) cudaFree(p);  // the stream the block was used on may no longer exist
 }
 
 void *ta_dalloc(ta_window *h, size_t bytes) {

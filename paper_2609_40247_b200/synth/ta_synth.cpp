@@ -9,7 +9,7 @@
 // Shapes and magnitudes follow the paper's reported ranges: kernel durations
 // from half a microsecond to several milliseconds (Sec. 8.1), tens to
 // hundreds of inference steps per 30 s window (Sec. 5.3), ranks that meet in
-// collectives where a late rank leaves the others waiting (Sec. 9.2).
+// collectives, where the other ranks wait for the last one to arrive (Sec. 9.2).
 //
 // Build: g++ -O2 -std=c++17 -shared -fPIC ta_synth.cpp -o libta_synth.so
 #include <algorithm>

@@ -80,6 +80,27 @@ def test_documented_limits_return_too_large():
         with ta.Window(buf, [0, 1], [0], [2**41]) as w:
             w.sort_timeline()
     assert _status(too_long) == TA_ERR_TOO_LARGE
+    # windows x 2^ceil(log2(triples)) beyond 2^24: 2^21 windows and 16 streams
+    W = 1 << 21
+    rows = [("KERNEL", 1, s, 10, 20, 0, 0, 0) for s in range(16)]
+    ev = make_events(rows)
+    buf = torch.from_numpy(ev.view(np.uint8).reshape(-1)).cuda()
+    off = np.full(W + 1, len(ev), dtype=np.int64)
+    off[0] = 0
+    assert _status(lambda: ta.Window(buf, off, np.zeros(W, dtype=np.int64),
+                                     np.full(W, 1000, dtype=np.int64))) == TA_ERR_TOO_LARGE
+    # 2^22 lanes (one record in each of 2^22 windows): the gap scan's lane limit
+    W = 1 << 22
+    ev = np.zeros(W, dtype=ta.EVENT_DTYPE)
+    ev["ts_start"], ev["ts_end"], ev["pid"], ev["kind"] = 10, 20, 1, 3
+    buf = torch.from_numpy(ev.view(np.uint8).reshape(-1)).cuda()
+
+    def too_many_lanes():
+        with ta.Window(buf, np.arange(W + 1, dtype=np.int64), np.zeros(W, dtype=np.int64),
+                       np.full(W, 1000, dtype=np.int64)) as w:
+            assert w.sort_timeline().n_lanes == W
+            w.stream_gaps(1)
+    assert _status(too_many_lanes) == TA_ERR_TOO_LARGE
 
 
 def test_device_is_fine_after_errors():
