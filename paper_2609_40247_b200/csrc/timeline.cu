@@ -259,14 +259,32 @@ __global__ void __launch_bounds__(1024) k_lane_table(const int32_t *lane_start, 
     *n_lanes_out = (int32_t)L;
   }
   __syncthreads();
-  // per lane: the first position behind the run of lanes of its domain (host and device lanes
-  // alternate per (window, pid), so the runs are a few lanes long)
+  // per lane: the first later lane of the other domain, and the position where it begins (host
+  // and device lanes alternate per (window, pid), so the runs are a few lanes long - but a batch
+  // of device-only windows is one long run, hence a scan and no walk).  Going backwards over
+  // the lanes, the nearest boundary at or behind lane l is a running maximum of
+  // L - (index of the lane behind a boundary); chunks of blockDim.x lanes, carried in `base`.
   const int64_t L = (int64_t)base < cap ? (int64_t)base : cap;
-  for (int64_t l = threadIdx.x; l < L; l += blockDim.x) {
-    int64_t m = l + 1;
-    while (m < L && lane_domain[m] == lane_domain[l]) m++;
-    lane_dom_end[l] = m < L ? lane_off[m] : (int32_t)n_valid;
-    lane_dom_next[l] = (int32_t)m;  // index of the first later lane of the other domain (L if none)
+  __syncthreads();  // every thread has read the lane count before `base` is reused
+  if (threadIdx.x == 0) base = 0;
+  __syncthreads();
+  for (int64_t r0 = 0; r0 < L; r0 += blockDim.x) {
+    const int64_t r = r0 + threadIdx.x;  // reversed lane index
+    const int64_t l = L - 1 - r;
+    u64 v = 0;
+    if (r < L && l + 1 < L && lane_domain[l + 1] != lane_domain[l]) v = (u64)(L - (l + 1));
+    u64 total;
+    const u64 ex = block_scan_exclusive<OpMax>(v, OpMax(), tmp, &total);
+    if (r < L) {
+      u64 best = ex > v ? ex : v;
+      best = best > base ? best : base;
+      const int64_t m = best ? L - (int64_t)best : L;
+      lane_dom_end[l] = m < L ? lane_off[m] : (int32_t)n_valid;
+      lane_dom_next[l] = (int32_t)m;  // index of the first later lane of the other domain (L if none)
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) base = base > total ? base : total;
+    __syncthreads();
   }
   // per device lane: how many device records sit in earlier lanes (their index once the device
   // records are taken out in order); n_lanes_out[1] = the number of device records
