@@ -714,40 +714,46 @@ __global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a
 }
 
 // first/last were accumulated in an order-preserving unsigned encoding (0 = untouched)
+#ifndef AT_FIN_ITEMS
+#define AT_FIN_ITEMS 4
+#endif
 __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
-  if (ta_failed(a.status)) return;
-  const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+  constexpr int IT = AT_FIN_ITEMS;
+  const int err = ta_peek_err(a.status);
+  const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * IT;
   if (p0 >= a.n_valid) return;
-  int16_t kd[8];
-  load8_i16(a.kind, p0, a.n, 9, kd);
+  int16_t kd[IT];
+  loadn_i16<IT>(a.kind, p0, a.n, 9, kd);
+  if (ta_is_failure(err)) return;
   unsigned ops = 0;
 #pragma unroll
-  for (int j = 0; j < 8; j++)
+  for (int j = 0; j < IT; j++)
     if (p0 + j < a.n_valid && kd[j] == TA_KIND_OP) ops |= 1u << j;
   if (!ops) return;
-  // counts of all eight positions in two vector loads, then both times of the operators that
-  // own kernels: the thread's misses overlap instead of following one another
-  int32_t cnt[8];
-  if (p0 + 8 <= a.n) {
-    const int4 x = *reinterpret_cast<const int4 *>(a.op_n + p0);
-    const int4 y = *reinterpret_cast<const int4 *>(a.op_n + p0 + 4);
-    cnt[0] = x.x; cnt[1] = x.y; cnt[2] = x.z; cnt[3] = x.w;
-    cnt[4] = y.x; cnt[5] = y.y; cnt[6] = y.z; cnt[7] = y.w;
+  // counts of all the thread's positions in vector loads, then both times of the operators
+  // that own kernels: the thread's misses overlap instead of following one another
+  int32_t cnt[IT];
+  if (p0 + IT <= a.n) {
+#pragma unroll
+    for (int q = 0; q < IT / 4; q++) {
+      const int4 x = *reinterpret_cast<const int4 *>(a.op_n + p0 + 4 * q);
+      cnt[4 * q] = x.x; cnt[4 * q + 1] = x.y; cnt[4 * q + 2] = x.z; cnt[4 * q + 3] = x.w;
+    }
   } else {
 #pragma unroll
-    for (int j = 0; j < 8; j++) cnt[j] = p0 + j < a.n ? a.op_n[p0 + j] : 0;
+    for (int j = 0; j < IT; j++) cnt[j] = p0 + j < a.n ? a.op_n[p0 + j] : 0;
   }
   unsigned m = 0;
 #pragma unroll
-  for (int j = 0; j < 8; j++)
+  for (int j = 0; j < IT; j++)
     if ((ops & (1u << j)) && cnt[j] > 0) m |= 1u << j;
   if (!m) return;
-  u64 f[8], l[8];
+  u64 f[IT], l[IT];
 #pragma unroll
-  for (int j = 0; j < 8; j++)
+  for (int j = 0; j < IT; j++)
     if (m & (1u << j)) { f[j] = a.op_first[p0 + j]; l[j] = a.op_last[p0 + j]; }
 #pragma unroll
-  for (int j = 0; j < 8; j++)
+  for (int j = 0; j < IT; j++)
     if (m & (1u << j)) {
       a.op_first[p0 + j] = (~f[j]) ^ (1ull << 63);
       a.op_last[p0 + j] = l[j] ^ (1ull << 63);
@@ -829,7 +835,7 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
     }
     k_attr_resolve<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
     k_attr_ops<<<TA_N (unsigned)((n + AT_OPS_TILE - 1) / AT_OPS_TILE), AT_THREADS, 0, st>>>(a);
-    const int64_t fb = (h->n_valid + 2047) / 2048;
+    const int64_t fb = (h->n_valid + 256 * AT_FIN_ITEMS - 1) / (256 * AT_FIN_ITEMS);
     k_attr_finalize<<<TA_N (unsigned)(fb > 0 ? fb : 1), 256, 0, st>>>(a);
     TA_CHECK_CUDA(h, cudaGetLastError());
   }

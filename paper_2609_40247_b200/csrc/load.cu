@@ -202,8 +202,12 @@ __global__ void __launch_bounds__(PL_THREADS) k_plan(const ta_event *ev, int64_t
 }
 
 // ---- discovery with staged tiles -----------------------------------------------------------
+#ifndef DS_THREADS
 #define DS_THREADS 256
+#endif
+#ifndef DS_RPT
 #define DS_RPT 2                          // records per thread and tile
+#endif
 #define DS_TILE (DS_THREADS * DS_RPT)     // 512 records = 20480 bytes
 #define DS_TILE_BYTES (DS_TILE * 40)
 #define DS_WAIT_POLLS (1 << 18)  // a tile arrives within microseconds; each poll may itself wait a little
@@ -266,7 +270,7 @@ __global__ void __launch_bounds__(DS_THREADS) k_discover_staged(DiscoverArgs a) 
   extern __shared__ __align__(128) unsigned char ds_raw[];
   DiscoverSmem &s = *reinterpret_cast<DiscoverSmem *>(ds_raw);
   const int tid = threadIdx.x, lane = tid & 31;
-  s.cache[tid] = TRIPLE_EMPTY;
+  for (int i = tid; i < 256; i += DS_THREADS) s.cache[i] = TRIPLE_EMPTY;
   if (tid < 64) s.ccache[tid] = TRIPLE_EMPTY;
   for (int i = tid; i < 5 * 256; i += DS_THREADS) (&s.hist[0][0])[i] = 0;
   if (tid == 0) {
@@ -803,7 +807,10 @@ ta_status ta_launch_discover(ta_window *h) {
       TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_discover_staged, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             (int)sizeof(DiscoverSmem)));
       const int64_t tiles = (h->n + DS_TILE - 1) / DS_TILE;
-      const int grid = (int)(tiles < 148 * 4 ? tiles : 148 * 4);
+#ifndef DS_CTAS_PER_SM
+#define DS_CTAS_PER_SM 4
+#endif
+      const int grid = (int)(tiles < 148 * DS_CTAS_PER_SM ? tiles : 148 * DS_CTAS_PER_SM);
       k_discover_staged<<<TA_N grid, DS_THREADS, sizeof(DiscoverSmem), h->stream>>>(a);
       h->tkeep = -1;  // read back with the other results of the pass
     } else {

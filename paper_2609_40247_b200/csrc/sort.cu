@@ -124,6 +124,19 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
       m &= bal ^ (bit - 1u);  // bit set: keep bal; bit clear: keep ~bal
     }
     if (!FULL && !valid) m = 0;
+#ifndef RS_RANK_READBACK
+    // The lowest peer adds the group size to the warp's digit counter and hands the counter's
+    // old value to its peers by a shuffle; a peer's rank is that value plus the number of peers
+    // below it.  No read-back of the counter and no warp barrier: the rows of a thread are
+    // independent up to the order of the warp's own atomics on one address, which is program
+    // order, so the votes of later rows overlap the atomics of earlier ones.
+    const int leader = __ffs((int)m) - 1;  // -1 for an invalid lane (m = 0)
+    u32 old = 0;
+    if (valid && lane == leader) old = atomicAdd(&wh[d], (u32)__popc(m));
+    old = __shfl_sync(0xffffffffu, old, leader < 0 ? lane : leader);
+    rd[j] = (int)(((old + (u32)__popc(m & lt)) << 8) | d);
+  }
+#else
     // one population count per key: the number of peers at or above the lane.  The lowest
     // peer adds the group size to the warp's digit counter; every peer then reads the counter
     // back and steps down from its new value.
@@ -134,6 +147,7 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
     rd[j] = (int)(((after - above1) << 8) | d);
     __syncwarp();
   }
+#endif
   __syncthreads();
   // per digit: the CTA's count, exclusive starts of the digits, and per warp the tile-local
   // start of its run (so the scatter needs one shared load per key)
