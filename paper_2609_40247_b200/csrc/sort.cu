@@ -14,6 +14,11 @@
 #include "ta_internal.cuh"
 
 #define RS_BINS 256
+// descriptors of earlier tiles fetched together in the look back (1 = one at a time)
+#ifndef RS_LOOKBACK_BATCH
+#define RS_LOOKBACK_BATCH 4
+#endif
+
 // resident CTAs per SM the register allocation is sized for (pairs, keys only)
 #ifndef RSP_MINB
 #define RSP_MINB 2
@@ -192,10 +197,27 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
     } else {
       excl = 0;
       bool timed_out = false;
-      for (int t = tile - 1;; --t) {
-        const u64 w = td_wait(a.tile_state + (size_t)t * RS_BINS + tid, a.status, &timed_out);
-        excl += w & TD_MASK;
-        if ((w >> 62) == TD_PREFIX) break;
+      // The walk over earlier tiles is a chain of dependent L2 reads (each some hundred
+      // cycles): the descriptors of the next few tiles back are fetched together and consumed
+      // in order, which divides the latency of a long walk by the batch size.  An unpublished
+      // descriptor among them is waited for with the bounded wait.
+      for (int lb_t = tile - 1;; lb_t -= RS_LOOKBACK_BATCH) {
+        u64 lb[RS_LOOKBACK_BATCH];
+#pragma unroll
+        for (int i = 0; i < RS_LOOKBACK_BATCH; i++)
+          lb[i] = lb_t - i >= 0 ? ld_relaxed(a.tile_state + (size_t)(lb_t - i) * RS_BINS + tid)
+                                : td_pack(TD_PREFIX, 0);
+        bool done = false;
+#pragma unroll
+        for (int i = 0; i < RS_LOOKBACK_BATCH; i++) {
+          if (done) continue;
+          u64 x = lb[i];
+          if ((x >> 62) == TD_EMPTY)
+            x = td_wait(a.tile_state + (size_t)(lb_t - i) * RS_BINS + tid, a.status, &timed_out);
+          excl += x & TD_MASK;
+          if ((x >> 62) == TD_PREFIX) done = true;
+        }
+        if (done) break;
       }
       // a wait that gave up leaves the descriptor at its aggregate: the tiles behind this one
       // look past it, meet the same unpublished tile (or the error word) and give up as well
