@@ -55,7 +55,7 @@ struct AttrArgs {
   int64_t n_tiles;
   const int16_t *kind;
   const int64_t *ts, *te;
-  const int32_t *lane_off, *lane_window;
+  const int32_t *lane_off, *lane_window, *lane_dom_end;
   const int16_t *lane_domain;
   int32_t *parent;
   uint8_t *depth;
@@ -594,58 +594,55 @@ __global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a
     int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (lane == 0) s_lane0 = l;
   }
-  int16_t kd[IT];
-  if (IT == 8) load8_i16(a.kind, p0, a.n, 0, kd);
-  else if (p0 + IT <= a.n) {
-    const uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
-    const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
+  __syncthreads();
+  const int l0 = s_lane0;
+  // A tile of host lanes holds no device record: nothing to read, op_of = -1 throughout.
+  if (l0 >= 0 && span_outside_domain(a.lane_domain, a.lane_dom_end, l0,
+                                     min(tile_start + AT_OPS_TILE, a.n_valid), 1)) {
+    if (p0 + IT <= a.n) {
 #pragma unroll
-    for (int j = 0; j < IT; j++) kd[j] = hq[j];
-  } else {
-#pragma unroll
-    for (int j = 0; j < IT; j++) kd[j] = p0 + j < a.n ? a.kind[p0 + j] : (int16_t)0;
+      for (int q = 0; q < IT / 4; q++) *reinterpret_cast<int4 *>(a.op_of + p0 + 4 * q) = make_int4(-1, -1, -1, -1);
+    } else {
+      for (int j = 0; j < IT; j++)
+        if (p0 + j < a.n) a.op_of[p0 + j] = -1;
+    }
+    return;
   }
-  unsigned pm = 0;
-#pragma unroll
-  for (int j = 0; j < IT; j++)
-    if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
+  // kinds, launches and times of the thread's records are requested together (launch_of is -1
+  // wherever the record is no matched kernel or copy, so the gather below needs no kind), then
+  // the parents of the launches: two rounds of memory latency instead of three
+  int16_t kd[IT];
+  loadn_i16<IT>(a.kind, p0, a.n, 0, kd);
   int32_t lo[IT], op[IT];
   i64 st[IT], en[IT];
 #pragma unroll
   for (int j = 0; j < IT; j++) { lo[j] = -1; op[j] = -1; st[j] = en[j] = 0; }
-  if (pm) {
-    if (p0 + IT <= a.n) {
+  if (p0 + IT <= a.n) {
 #pragma unroll
-      for (int q = 0; q < IT / 4; q++) {
-        const int4 x = *reinterpret_cast<const int4 *>(a.launch_of + p0 + 4 * q);
-        lo[4 * q] = x.x; lo[4 * q + 1] = x.y; lo[4 * q + 2] = x.z; lo[4 * q + 3] = x.w;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < IT; j++)
-        if (p0 + j < a.n) lo[j] = a.launch_of[p0 + j];
+    for (int q = 0; q < IT / 4; q++) {
+      const int4 x = *reinterpret_cast<const int4 *>(a.launch_of + p0 + 4 * q);
+      lo[4 * q] = x.x; lo[4 * q + 1] = x.y; lo[4 * q + 2] = x.z; lo[4 * q + 3] = x.w;
     }
-    if (p0 + IT <= a.n) {
-      const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
-      const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
+    const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
+    const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
 #pragma unroll
-      for (int q = 0; q < IT / 2; q++) {
-        const longlong2 x = ps[q], y = pe[q];
-        st[2 * q] = x.x; st[2 * q + 1] = x.y;
-        en[2 * q] = y.x; en[2 * q + 1] = y.y;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < IT; j++)
-        if (p0 + j < a.n) { st[j] = a.ts[p0 + j]; en[j] = a.te[p0 + j]; }
+    for (int q = 0; q < IT / 2; q++) {
+      const longlong2 x = ps[q], y = pe[q];
+      st[2 * q] = x.x; st[2 * q + 1] = x.y;
+      en[2 * q] = y.x; en[2 * q + 1] = y.y;
     }
-    // parents of the launches: independent gathers, issued together
+  } else {
 #pragma unroll
     for (int j = 0; j < IT; j++)
-      if ((pm & (1u << j)) && lo[j] >= 0) op[j] = a.parent[lo[j]];
+      if (p0 + j < a.n) { lo[j] = a.launch_of[p0 + j]; st[j] = a.ts[p0 + j]; en[j] = a.te[p0 + j]; }
   }
-  __syncthreads();
-  const int l0 = s_lane0;
+#pragma unroll
+  for (int j = 0; j < IT; j++)
+    if (lo[j] >= 0) op[j] = a.parent[lo[j]];
+  unsigned pm = 0;
+#pragma unroll
+  for (int j = 0; j < IT; j++)
+    if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
   u64 packed = 0;  // attributed | no launch << 20 | no op << 40, for the thread's first lane
   int lm = -1;
   {
@@ -806,7 +803,7 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   a.n = n; a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes; a.n_tiles = tiles;
   a.kind = h->sorted.kind; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window;
-  a.lane_domain = h->sorted.lane_domain;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   a.parent = parent; a.depth = depth; a.sum = d_sum; a.status = h->d_status;
   a.launch_of = h->join.launch_of; a.op_of = op_of; a.op_n = op_n; a.op_first = op_first;
   a.op_last = op_last; a.op_ns = op_ns;

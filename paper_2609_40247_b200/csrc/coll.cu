@@ -88,16 +88,32 @@ __global__ void __launch_bounds__(256) k_coll_groups(CollGroupArgs a) {
   i64 mn = INT64_MAX, mx = INT64_MIN, me = INT64_MIN;
   int32_t strag = 0, strag_slot = 0, prev_pid = 0;
   int flags = 0;
-  for (int64_t j = b; j < e; j++) {
-    u32 ci = a.cs[j];
-    u32 p = a.c.posc[ci];
-    i64 s = a.c.ts[p], en = a.c.te[p];
-    int32_t pd = a.c.pid[p];
-    mn = min(mn, s);
-    me = max(me, en);
-    if (s > mx || (s == mx && pd < strag)) { mx = s; strag = pd; strag_slot = a.slot_of[ci]; }
-    if (j > b && pd == prev_pid) flags |= TA_COLL_DUP_PID;
-    prev_pid = pd;
+  // members four at a time: each is reached through two index levels (sorted rank -> compacted
+  // index -> sorted position), and one member after the other would make the group a chain of
+  // forty-odd dependent loads; the order of the updates stays the members' order
+  for (int64_t j0 = b; j0 < e; j0 += 4) {
+    u32 ci[4], p[4];
+    i64 s[4], en[4];
+    int32_t pd[4], sl[4];
+#pragma unroll
+    for (int k = 0; k < 4; k++) ci[k] = j0 + k < e ? a.cs[j0 + k] : 0u;
+#pragma unroll
+    for (int k = 0; k < 4; k++) p[k] = j0 + k < e ? a.c.posc[ci[k]] : 0u;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      s[k] = en[k] = 0;
+      pd[k] = sl[k] = 0;
+      if (j0 + k < e) { s[k] = a.c.ts[p[k]]; en[k] = a.c.te[p[k]]; pd[k] = a.c.pid[p[k]]; sl[k] = a.slot_of[ci[k]]; }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      if (j0 + k >= e) break;
+      mn = min(mn, s[k]);
+      me = max(me, en[k]);
+      if (s[k] > mx || (s[k] == mx && pd[k] < strag)) { mx = s[k]; strag = pd[k]; strag_slot = sl[k]; }
+      if (j0 + k > b && pd[k] == prev_pid) flags |= TA_COLL_DUP_PID;
+      prev_pid = pd[k];
+    }
   }
   const u64 key = a.ks[b];
   const int rank = (int)((key >> a.c.qbits) & ((1ull << a.c.cbits) - 1));

@@ -31,7 +31,7 @@ struct JoinArgs {
   int n_lanes;
   const int16_t *kind;
   const int64_t *corr, *ts, *te;
-  const int32_t *lane_off, *lane_slot, *lane_window;
+  const int32_t *lane_off, *lane_slot, *lane_window, *lane_dom_end;
   const int16_t *lane_domain;
   // per slot (window * n_pids + pid rank)
   i64 *slot_min, *slot_max;       // corr range of LAUNCH records
@@ -129,21 +129,30 @@ __global__ void __launch_bounds__(JP_THREADS, JP_MINB) k_join_probe(JoinArgs a) 
     int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (lane == 0) s_lane0 = l;
   }
+  __syncthreads();
+  const int l0 = s_lane0;
+  // A tile of host lanes holds no probe: nothing to read, the three outputs are -1 / 0 / 0.
+  if (l0 >= 0 && span_outside_domain(a.lane_domain, a.lane_dom_end, l0, min(tile_start + JP_TILE, a.n_valid), 1)) {
+    int32_t lo0[IT];
+    i64 z[IT];
+#pragma unroll
+    for (int j = 0; j < IT; j++) { lo0[j] = -1; z[j] = 0; }
+    storen_i32<IT>(a.launch_of, p0, a.n, lo0);
+    storen_i64<IT>(a.latency, p0, a.n, z);
+    storen_i64<IT>(a.qdelay, p0, a.n, z);
+    return;
+  }
+  // kinds, correlation ids and start times are requested together: one round of memory
+  // latency less than loading the ids only where the kinds ask for them
   int16_t kd[IT];
+  i64 c[IT], s[IT];
   loadn_i16<IT>(a.kind, p0, a.n, 0, kd);
+  loadn_i64<IT>(a.corr, p0, a.n, c);
+  loadn_i64<IT>(a.ts, p0, a.n, s);
   unsigned pm = 0;  // probes among the thread's records
 #pragma unroll
   for (int j = 0; j < IT; j++)
     if (p0 + j < a.n_valid && (kd[j] == TA_KIND_KERNEL || kd[j] == TA_KIND_MEMCPY)) pm |= 1u << j;
-  i64 c[IT], s[IT];
-#pragma unroll
-  for (int j = 0; j < IT; j++) c[j] = s[j] = 0;
-  if (pm) {
-    loadn_i64<IT>(a.corr, p0, a.n, c);
-    loadn_i64<IT>(a.ts, p0, a.n, s);
-  }
-  __syncthreads();
-  const int l0 = s_lane0;
   int32_t lo[IT];
   int ln[IT];
   {
@@ -412,7 +421,7 @@ ta_status ta_run_correlate(ta_window *h, ta_join_summary *out_summary) {
   a.n = n; a.n_valid = h->n_valid; a.n_lanes = h->sorted.n_lanes;
   a.kind = h->sorted.kind; a.corr = h->sorted.corr_id; a.ts = h->sorted.ts_start; a.te = h->sorted.ts_end;
   a.lane_off = h->sorted.lane_off; a.lane_slot = h->d_lane_slot; a.lane_window = h->sorted.lane_window;
-  a.lane_domain = h->sorted.lane_domain;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   a.slot_min = slot_min; a.slot_max = slot_max; a.slot_base = slot_base;
   a.launch_of = launch_of; a.kol = kol; a.latency = latency; a.qdelay = qdelay; a.sum = d_sum;
   a.status = h->d_status;
