@@ -78,15 +78,33 @@ __device__ __forceinline__ void tile_lane_range(int my_lo, int my_hi, int *s_lo,
 
 // ---- direct path: fill the table -------------------------------------------
 __global__ void __launch_bounds__(JN_THREADS) k_join_build(JoinArgs a) {
+  __shared__ int s_lane0;
   if (ta_failed(a.status)) return;
-  const int64_t p0 = ((int64_t)blockIdx.x * JN_THREADS + threadIdx.x) * JN_ITEMS;
-  LaneWalker lw(a.lane_off, a.n_lanes, p0, a.n_valid);
+  const int tid = threadIdx.x;
+  const int64_t tile_start = (int64_t)blockIdx.x * JN_TILE;
+  if (tile_start >= a.n_valid) return;
+  if (tid < 32) {
+    const int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
+    if (tid == 0) s_lane0 = l;
+  }
+  __syncthreads();
+  const int l0 = s_lane0;
+  // launches live in host lanes: a tile of device lanes has none
+  if (span_outside_domain(a.lane_domain, a.lane_dom_end, l0, min(tile_start + JN_TILE, a.n_valid), 0)) return;
+  const int64_t p0 = tile_start + (int64_t)tid * JN_ITEMS;
+  int16_t kd[JN_ITEMS];
+  i64 c[JN_ITEMS];
+  loadn_i16<JN_ITEMS>(a.kind, p0, a.n, 9, kd);
+  loadn_i64<JN_ITEMS>(a.corr, p0, a.n, c);
+  int l = l0;
+  int64_t next_off = a.lane_off[l + 1];
+  int slot = a.lane_slot[l];
 #pragma unroll
   for (int j = 0; j < JN_ITEMS; j++) {
-    int64_t p = p0 + j;
-    if (p < a.n_valid && a.kind[p] == TA_KIND_LAUNCH) {
-      int slot = a.lane_slot[lw.at(p)];
-      i64 idx = a.slot_base[slot] + (a.corr[p] - a.slot_min[slot]);
+    const int64_t p = p0 + j;
+    if (p < a.n_valid && kd[j] == TA_KIND_LAUNCH) {
+      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; slot = a.lane_slot[l]; }
+      const i64 idx = a.slot_base[slot] + (c[j] - a.slot_min[slot]);
       atomicMin(&a.table[idx], (u32)p);
     }
   }
@@ -288,14 +306,17 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
     int l = tile_lane_search(a.lane_off, a.n_lanes, tile_start);
     if (lane == 0) s_lane0 = l;
   }
+  __syncthreads();
+  const int l0 = s_lane0;
+  // launches live in host lanes: a tile of device lanes has none
+  if (l0 < 0 || span_outside_domain(a.lane_domain, a.lane_dom_end, l0, min(tile_start + JS_TILE, a.n_valid), 0))
+    return;
   int16_t kd[8];
   load8_i16(a.kind, p0, a.n, 0, kd);
   unsigned lmask = 0;
 #pragma unroll
   for (int j = 0; j < 8; j++)
     if (p0 + j < a.n_valid && kd[j] == TA_KIND_LAUNCH) lmask |= 1u << j;
-  __syncthreads();
-  const int l0 = s_lane0;
   u64 packed = 0;  // n_launch | n_dup << 20 | n_orphan << 40 for the thread's first lane
   int lm = -1;
   {
