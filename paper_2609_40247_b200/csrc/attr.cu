@@ -719,16 +719,10 @@ __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
   const int err = ta_peek_err(a.status);
   const int64_t p0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * IT;
   if (p0 >= a.n_valid) return;
-  int16_t kd[IT];
-  loadn_i16<IT>(a.kind, p0, a.n, 9, kd);
-  if (ta_is_failure(err)) return;
-  unsigned ops = 0;
-#pragma unroll
-  for (int j = 0; j < IT; j++)
-    if (p0 + j < a.n_valid && kd[j] == TA_KIND_OP) ops |= 1u << j;
-  if (!ops) return;
-  // counts of all the thread's positions in vector loads, then both times of the operators
-  // that own kernels: the thread's misses overlap instead of following one another
+  // A kernel count above zero only ever sits at the position of an operator that owns kernels
+  // (the counts are accumulated on operator rows alone), so the kinds need not be read: the
+  // counts of all the thread's positions in vector loads, then both times of those operators -
+  // two rounds of memory latency, the thread's misses overlapping
   int32_t cnt[IT];
   if (p0 + IT <= a.n) {
 #pragma unroll
@@ -740,10 +734,11 @@ __global__ void __launch_bounds__(256) k_attr_finalize(AttrArgs a) {
 #pragma unroll
     for (int j = 0; j < IT; j++) cnt[j] = p0 + j < a.n ? a.op_n[p0 + j] : 0;
   }
+  if (ta_is_failure(err)) return;
   unsigned m = 0;
 #pragma unroll
   for (int j = 0; j < IT; j++)
-    if ((ops & (1u << j)) && cnt[j] > 0) m |= 1u << j;
+    if (p0 + j < a.n_valid && cnt[j] > 0) m |= 1u << j;
   if (!m) return;
   u64 f[IT], l[IT];
 #pragma unroll

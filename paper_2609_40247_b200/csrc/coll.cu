@@ -31,11 +31,20 @@ struct CollCtx {
 };
 
 __global__ void __launch_bounds__(256) k_coll_keys(CollCtx c, u64 *keys, int32_t *slot_of, int32_t *status) {
+  __shared__ int s_lane0;
   if (ta_failed(status)) return;
   int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // the compacted positions ascend: the lane of the CTA's first record is searched once, the
+  // others walk on from it (a few lanes at most as a rule; a full search after eight steps)
+  if (threadIdx.x == 0) s_lane0 = lane_of_pos(c.lane_off, c.n_lanes, c.posc[min(j, c.m - 1)]);
+  __syncthreads();
   if (j >= c.m) return;
   u32 p = c.posc[j];
-  int lane = lane_of_pos(c.lane_off, c.n_lanes, p);
+  int lane = s_lane0;
+  for (int step = 0; lane + 1 < c.n_lanes && (int64_t)c.lane_off[lane + 1] <= (int64_t)p; step++) {
+    if (step == 8) { lane = lane_of_pos(c.lane_off, c.n_lanes, p); break; }
+    lane++;
+  }
   u64 cc = (u64)c.corr[p] ^ (1ull << 63);
   // every communicator id was inserted while the records were loaded: a bounded probe all the same
   u32 s = hash_code(cc) & (TA_COMM_SLOTS - 1);

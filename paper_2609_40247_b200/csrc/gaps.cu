@@ -92,34 +92,32 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
     }
     return;
   }
-  // kinds of the thread's eight records (0 = not a device record of the window)
+  // kinds, start and end times of the thread's records and, for the scan-free mode, the end of
+  // the record in front of the thread's first one: all requested together (the tile holds a
+  // device lane, so nearly every record needs its times anyway)
   int16_t kd[GP_ITEMS];
   loadn_i16<GP_ITEMS>(a.kind, p0, a.n, 0, kd);
-  bool any_dev = false;
-#pragma unroll
-  for (int j = 0; j < GP_ITEMS; j++) {
-    if (p0 + j >= a.n_valid) kd[j] = 0;
-    any_dev |= kd[j] >= 3;
-  }
   i64 s[GP_ITEMS], ce[GP_ITEMS];  // ce: ts_end, clipped below
 #pragma unroll
   for (int j = 0; j < GP_ITEMS; j++) s[j] = ce[j] = 0;
-  if (any_dev) {
-    if (full) {
-      const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
-      const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
+  if (full) {
+    const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
+    const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
 #pragma unroll
-      for (int j = 0; j < GP_ITEMS / 2; j++) {
-        longlong2 x = ps[j], y = pe[j];
-        s[2 * j] = x.x; s[2 * j + 1] = x.y;
-        ce[2 * j] = y.x; ce[2 * j + 1] = y.y;
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < GP_ITEMS; j++)
-        if (p0 + j < a.n) { s[j] = a.ts[p0 + j]; ce[j] = a.te[p0 + j]; }
+    for (int j = 0; j < GP_ITEMS / 2; j++) {
+      longlong2 x = ps[j], y = pe[j];
+      s[2 * j] = x.x; s[2 * j + 1] = x.y;
+      ce[2 * j] = y.x; ce[2 * j + 1] = y.y;
     }
+  } else {
+#pragma unroll
+    for (int j = 0; j < GP_ITEMS; j++)
+      if (p0 + j < a.n) { s[j] = a.ts[p0 + j]; ce[j] = a.te[p0 + j]; }
   }
+  const i64 e_before = (a.local && p0 > 0 && p0 <= a.n) ? a.te[p0 - 1] : 0;
+#pragma unroll
+  for (int j = 0; j < GP_ITEMS; j++)
+    if (p0 + j >= a.n_valid) kd[j] = 0;
   // lanes of the items: walk forward from the tile's first lane
   int ln[GP_ITEMS];
   u64 run = 0;
@@ -155,7 +153,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
     const int l = ln[0];
     if (l >= 0 && p0 > (int64_t)a.lane_off[l]) {
       const int w = a.lane_window[l];
-      const i64 w0 = a.t0[w], w1 = a.t1[w], e = a.te[p0 - 1];
+      const i64 w0 = a.t0[w], w1 = a.t1[w], e = e_before;
       pre = ((u64)(l + 1) << 40) | (u64)((e < w1 ? e : w1) - w0);
     }
     __syncthreads();  // s_lane1 and the zeroed histograms are read below
