@@ -130,16 +130,41 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
         continue;
       lw.lane = bl;
       const int64_t p0 = base + (int64_t)threadIdx.x * AG_ITEMS;
-      // all loads of the thread's four records are issued before any of them is used
+      // all loads of the thread's four records are issued before any of them is used; for the
+      // plain duration the times and names are requested with the kinds, not after them (the
+      // step holds lanes of the wanted domain, so most records are selected anyway)
       int16_t kd[AG_ITEMS];
+      i64 pre_v[AG_ITEMS];
+      int32_t pre_nm[AG_ITEMS];
+#pragma unroll
+      for (int j = 0; j < AG_ITEMS; j++) { pre_v[j] = 0; pre_nm[j] = 0; }
       if (p0 + AG_ITEMS <= end) {
         uint2 q = *reinterpret_cast<const uint2 *>(a.kind + p0);
+        if (a.value_sel == 0) {
+          const longlong2 *ps = reinterpret_cast<const longlong2 *>(a.ts + p0);
+          const longlong2 *pe = reinterpret_cast<const longlong2 *>(a.te + p0);
+          const int4 nq = *reinterpret_cast<const int4 *>(a.name + p0);
+#pragma unroll
+          for (int h2 = 0; h2 < AG_ITEMS / 2; h2++) {
+            const longlong2 x = ps[h2], y = pe[h2];
+            pre_v[2 * h2] = y.x - x.x;
+            pre_v[2 * h2 + 1] = y.y - x.y;
+          }
+          pre_nm[0] = nq.x; pre_nm[1] = nq.y; pre_nm[2] = nq.z; pre_nm[3] = nq.w;
+        } else if (a.value_sel == 1) {  // the kernel counts with the kinds (pre_nm holds them)
+          const int4 cq = *reinterpret_cast<const int4 *>(a.op_n + p0);
+          pre_nm[0] = cq.x; pre_nm[1] = cq.y; pre_nm[2] = cq.z; pre_nm[3] = cq.w;
+        }
         const int16_t *hq = reinterpret_cast<const int16_t *>(&q);
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++) kd[j] = hq[j];
       } else {
 #pragma unroll
-        for (int j = 0; j < AG_ITEMS; j++) kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
+        for (int j = 0; j < AG_ITEMS; j++) {
+          kd[j] = p0 + j < end ? a.kind[p0 + j] : (int16_t)-1;
+          if (a.value_sel == 0 && p0 + j < end) { pre_v[j] = a.te[p0 + j] - a.ts[p0 + j]; pre_nm[j] = a.name[p0 + j]; }
+          if (a.value_sel == 1 && p0 + j < end) pre_nm[j] = a.op_n[p0 + j];
+        }
       }
       bool sel[AG_ITEMS];
       i64 v[AG_ITEMS];
@@ -153,11 +178,11 @@ __global__ void __launch_bounds__(AG_THREADS, 6) k_agg(AggArgs a) {
       if (a.value_sel == 0) {
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
-          if (sel[j]) { v[j] = a.te[p0 + j] - a.ts[p0 + j]; nm[j] = a.name[p0 + j]; }
+          if (sel[j]) { v[j] = pre_v[j]; nm[j] = pre_nm[j]; }
       } else if (a.value_sel == 1) {
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
-          if (sel[j]) sel[j] = a.op_n[p0 + j] > 0;
+          if (sel[j]) sel[j] = pre_nm[j] > 0;
 #pragma unroll
         for (int j = 0; j < AG_ITEMS; j++)
           if (sel[j]) { v[j] = a.op_last[p0 + j] - a.op_first[p0 + j]; nm[j] = a.name[p0 + j]; }
