@@ -348,14 +348,10 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     s.carry_e[tid] = a.carry_e[(size_t)tile * AT_CAP + tid];
     s.carry_pos[tid] = a.carry_pos[(size_t)tile * AT_CAP + tid];
   }
-  int16_t kd[AT_ITEMS];
-  loadn_i16<AT_ITEMS>(a.kind, p0, a.n, 9, kd);
-  unsigned hostmask = 0;
-#pragma unroll
-  for (int j = 0; j < AT_ITEMS; j++)
-    if (p0 + j < a.n_valid && kd[j] <= TA_KIND_LAUNCH) hostmask |= 1u << j;
-  const int any_host = __syncthreads_or(hostmask != 0);
-  if (!any_host) {
+  __syncthreads();
+  const int l0 = s.lane0;
+  // A tile of device lanes holds no host record: parent -1, depth 0 throughout, nothing read.
+  if (l0 < 0 || span_outside_domain(a.lane_domain, a.lane_dom_end, l0, min(tile_start + AT_TILE, a.n_valid), 0)) {
     if (full) {
 #pragma unroll
       for (int q = 0; q < AT_ITEMS / 4; q++) {
@@ -368,15 +364,18 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
     }
     return;
   }
+  // kinds and both times of the thread's records are requested together (the tile holds a host
+  // lane, so nearly every record needs its times)
+  int16_t kd[AT_ITEMS];
   i64 st[AT_ITEMS], en[AT_ITEMS];
+  loadn_i16<AT_ITEMS>(a.kind, p0, a.n, 9, kd);
+  loadn_i64<AT_ITEMS>(a.ts, p0, a.n, st);
+  loadn_i64<AT_ITEMS>(a.te, p0, a.n, en);
+  unsigned hostmask = 0;
 #pragma unroll
-  for (int j = 0; j < AT_ITEMS; j++) st[j] = en[j] = 0;
-  if (hostmask) {
-    loadn_i64<AT_ITEMS>(a.ts, p0, a.n, st);
-    loadn_i64<AT_ITEMS>(a.te, p0, a.n, en);
-  }
+  for (int j = 0; j < AT_ITEMS; j++)
+    if (p0 + j < a.n_valid && kd[j] <= TA_KIND_LAUNCH) hostmask |= 1u << j;
   // lanes, leaves, the thread's maximum
-  const int l0 = s.lane0;
   int ln[AT_ITEMS];
   int lo_local[AT_ITEMS];  // first tile-local index of the record's lane (-1: the lane began earlier)
   i64 m8 = INT64_MIN;
