@@ -65,6 +65,7 @@ struct AttrArgs {
   i64 *agg_e, *carry_e;           // [tile][AT_CAP]
   int32_t *agg_pos, *carry_pos;
   int32_t *status;
+  const int32_t *kol;  // kernels of each launch (from the join)
   // k_attr_ops
   const int32_t *launch_of;
   int32_t *op_of, *op_n;
@@ -371,6 +372,17 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
   loadn_i16<AT_ITEMS>(a.kind, p0, a.n, 9, kd);
   loadn_i64<AT_ITEMS>(a.ts, p0, a.n, st);
   loadn_i64<AT_ITEMS>(a.te, p0, a.n, en);
+  int32_t nk[AT_ITEMS];  // kernels of the thread's launches (0 elsewhere)
+  if (full) {
+#pragma unroll
+    for (int q = 0; q < AT_ITEMS / 4; q++) {
+      const int4 x = *reinterpret_cast<const int4 *>(a.kol + p0 + 4 * q);
+      nk[4 * q] = x.x; nk[4 * q + 1] = x.y; nk[4 * q + 2] = x.z; nk[4 * q + 3] = x.w;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++) nk[j] = p0 + j < a.n ? a.kol[p0 + j] : 0;
+  }
   unsigned hostmask = 0;
 #pragma unroll
   for (int j = 0; j < AT_ITEMS; j++)
@@ -503,6 +515,24 @@ __global__ void __launch_bounds__(AT_THREADS, AT_RES_MINB) k_attr_resolve(AttrAr
       }
     }
     plv[j] = (int16_t)pl;
+  }
+  // Kernels per operator: an operator owns the kernels of the launches directly inside it, and
+  // the join has counted the kernels of every launch, so the counts are added up here, from
+  // the launch side - consecutive launches mostly share their operator, and one add serves a
+  // run of them - instead of one atomic per kernel from the device side.
+  {
+    int32_t run_par = -1, run_cnt = 0;
+#pragma unroll
+    for (int j = 0; j < AT_ITEMS; j++) {
+      if (!(hostmask & (1u << j)) || kd[j] != TA_KIND_LAUNCH || par_abs[j] < 0 || nk[j] <= 0) continue;
+      if (par_abs[j] != run_par) {
+        if (run_cnt) atomicAdd(&a.op_n[run_par], run_cnt);
+        run_par = par_abs[j];
+        run_cnt = 0;
+      }
+      run_cnt += nk[j];
+    }
+    if (run_cnt) atomicAdd(&a.op_n[run_par], run_cnt);
   }
 #pragma unroll
   for (int q = 0; q < AT_ITEMS / 2; q++)
@@ -658,7 +688,7 @@ __global__ void __launch_bounds__(AT_THREADS, AT_OPS_MINB) k_attr_ops(AttrArgs a
       else {
         add = 1ull;
         const int32_t r = op[j];
-        atomicAdd(&a.op_n[r], 1);
+        // (the kernel count of the operator is accumulated from the launch side, in k_attr_resolve)
         atomicAdd((u64 *)&a.op_ns[r], (u64)(en[j] - st[j]));
         atomicMax(&a.op_first[r], ~((u64)st[j] ^ (1ull << 63)));
         atomicMax(&a.op_last[r], (u64)en[j] ^ (1ull << 63));
@@ -799,7 +829,7 @@ ta_status ta_run_attribute(ta_window *h, ta_attr_summary *out_summary) {
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window;
   a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   a.parent = parent; a.depth = depth; a.sum = d_sum; a.status = h->d_status;
-  a.launch_of = h->join.launch_of; a.op_of = op_of; a.op_n = op_n; a.op_first = op_first;
+  a.launch_of = h->join.launch_of; a.kol = h->join.kernels_of_launch; a.op_of = op_of; a.op_n = op_n; a.op_first = op_first;
   a.op_last = op_last; a.op_ns = op_ns;
   if (n > 0) {
     k_attr_agg<<<TA_N (unsigned)tiles, AT_THREADS, 0, st>>>(a);
