@@ -311,8 +311,20 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
   // launches live in host lanes: a tile of device lanes has none
   if (l0 < 0 || span_outside_domain(a.lane_domain, a.lane_dom_end, l0, min(tile_start + JS_TILE, a.n_valid), 0))
     return;
+  // kinds, correlation ids and kernel counts of the thread's records together, then the table
+  // entries of its launches together: two rounds of memory latency
   int16_t kd[8];
+  i64 cr[8];
+  int32_t nk[8];
   load8_i16(a.kind, p0, a.n, 0, kd);
+  load8_i64(a.corr, p0, a.n, cr);
+  if (p0 + 8 <= a.n) {
+    const int4 x = *reinterpret_cast<const int4 *>(a.kol + p0), y = *reinterpret_cast<const int4 *>(a.kol + p0 + 4);
+    nk[0] = x.x; nk[1] = x.y; nk[2] = x.z; nk[3] = x.w; nk[4] = y.x; nk[5] = y.y; nk[6] = y.z; nk[7] = y.w;
+  } else {
+#pragma unroll
+    for (int j = 0; j < 8; j++) nk[j] = p0 + j < a.n ? a.kol[p0 + j] : 0;
+  }
   unsigned lmask = 0;
 #pragma unroll
   for (int j = 0; j < 8; j++)
@@ -322,14 +334,36 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
   {
     int l = l0;
     int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+    int ln[8];
+    int32_t win[8];
+#pragma unroll
+    for (int j = 0; j < 8; j++) {
+      ln[j] = -1;
+      win[j] = -1;
+      if (!(lmask & (1u << j))) continue;
+      const int64_t p = p0 + j;
+      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+      ln[j] = l;
+      if (DIRECT) {
+        const int slot = a.lane_slot[l];
+        const i64 base = a.slot_base[slot];
+        if (base >= 0 && cr[j] >= a.slot_min[slot] && cr[j] <= a.slot_max[slot]) {
+          const u32 v = a.table[base + (cr[j] - a.slot_min[slot])];
+          win[j] = v == EMPTY_U32 ? -1 : (int32_t)v;
+        }
+      } else {
+        win[j] = a.found[p];
+      }
+    }
+    const int l_end = l;
+    int64_t next_end = next_off;
 #pragma unroll
     for (int j = 0; j < 8; j++) {
       if (!(lmask & (1u << j))) continue;
       const int64_t p = p0 + j;
-      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
-      const int32_t w = winner_of<DIRECT>(a, p, a.lane_slot[l]);
-      const bool dup = w != (int32_t)p;
-      const bool orphan = !dup && a.kol[p] == 0;
+      const int l = ln[j];
+      const bool dup = win[j] != (int32_t)p;
+      const bool orphan = !dup && nk[j] == 0;
       if (lm < 0) lm = l;
       if (l == lm && l - l0 <= 1) {
         packed += 1ull + ((u64)dup << 20) + ((u64)orphan << 40);
@@ -342,8 +376,9 @@ __global__ void __launch_bounds__(JP_THREADS) k_join_launch_stats(JoinArgs a) {
     }
     const int64_t plast = min(tile_start + JS_TILE, a.n_valid) - 1;
     if (plast >= p0 && plast < p0 + 8) {
-      while (plast >= next_off) { l++; next_off = a.lane_off[l + 1]; }
-      s_lane1 = l;
+      int le = l_end;
+      while (plast >= next_end) { le++; next_end = a.lane_off[le + 1]; }
+      s_lane1 = le;
     }
   }
   __syncthreads();

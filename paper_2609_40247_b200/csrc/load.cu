@@ -545,8 +545,7 @@ __global__ void __launch_bounds__(256) k_top_hist_words(TopHistArgs a) {
 }
 
 // One CTA: sorts the discovered triples, ranks them and the pids they contain.
-__global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t *status) {
-  extern __shared__ u64 buf[];  // TA_TRIPLE_SLOTS
+__device__ __forceinline__ void rank_triples(TripleTable *tt, int32_t *status, u64 *buf /* TA_TRIPLE_SLOTS */) {
   __shared__ u64 tmp[33];
   __shared__ int n_tr;
   const int tid = threadIdx.x;
@@ -612,8 +611,7 @@ __global__ void __launch_bounds__(1024) k_rank_triples(TripleTable *tt, int32_t 
 }
 
 // One CTA: sorts and ranks the communicator ids.
-__global__ void __launch_bounds__(1024) k_rank_comms(CommTable *cm, int32_t *status) {
-  __shared__ u64 buf[TA_COMM_SLOTS];
+__device__ __forceinline__ void rank_comms(CommTable *cm, int32_t *status, u64 *buf /* TA_COMM_SLOTS */) {
   __shared__ int n_c;
   const int tid = threadIdx.x;
   for (int i = tid; i < TA_COMM_SLOTS; i += blockDim.x) buf[i] = cm->slots[i];
@@ -655,6 +653,14 @@ __global__ void __launch_bounds__(1024) k_rank_comms(CommTable *cm, int32_t *sta
     }
     cm->rank_of_slot[s] = r;
   }
+}
+
+// Both rankings in one launch: CTA 0 the triples, CTA 1 the communicator ids (they are
+// independent, and two single-CTA kernels one after the other cost a launch latency more).
+__global__ void __launch_bounds__(1024) k_rank(TripleTable *tt, CommTable *cm, int32_t *status) {
+  extern __shared__ u64 rank_buf[];  // TA_TRIPLE_SLOTS
+  if (blockIdx.x == 0) rank_triples(tt, status, rank_buf);
+  else rank_comms(cm, status, rank_buf);
 }
 
 struct LoadArgs {
@@ -820,10 +826,9 @@ ta_status ta_launch_discover(ta_window *h) {
     }
     h->prekeys = 1;
   }
-  k_rank_comms<<<TA_N 1, 1024, 0, h->stream>>>(h->d_comms, h->d_status);
-  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank_triples, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  TA_CHECK_CUDA(h, cudaFuncSetAttribute(k_rank, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         TA_TRIPLE_SLOTS * (int)sizeof(u64)));
-  k_rank_triples<<<TA_N 1, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_status);
+  k_rank<<<TA_N 2, 1024, TA_TRIPLE_SLOTS * sizeof(u64), h->stream>>>(h->d_triples, h->d_comms, h->d_status);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }
