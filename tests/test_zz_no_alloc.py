@@ -53,7 +53,7 @@ def test_no_alloc_entry_matches_stream_gaps_on_two_calls_in_a_row():
 
 
 def test_no_alloc_entry_on_lanes_of_many_tiles():
-    """Two device lanes of 250 000 records, 123 scan tiles each (a tile is 2048 records), one
+    """Two device lanes of 150 000 records, 74 scan tiles each (a tile is 2048 records), one
     after the other and twice over, so that the chained scan really looks back through
     descriptors in the fixed scratch and every call starts from what the one before left there.  Each call is compared
     element by element with ta_stream_gaps on the same lane; the calls are given buffers the
@@ -62,7 +62,7 @@ def test_no_alloc_entry_on_lanes_of_many_tiles():
     import torch
     from paper_2609_40247_b200 import synth, ta
 
-    wl = synth.make_workload("c0", 25.0, truth=False)
+    wl = synth.make_workload("c0", 15.0, truth=False)
     buf = torch.from_numpy(np.ascontiguousarray(wl.events).view(np.uint8).reshape(-1)).cuda()
     with ta.Window(buf, wl.win_off, wl.win_t0, wl.win_t1) as w:
         s = w.sort_timeline()
