@@ -120,6 +120,7 @@ class ClockSampler:
 
 
 ALLOCATOR = "library"
+SOL_WORK = None  # (flops, bytes) CUDA tensors per input record, for the per-call timing of ta_operator_sol
 
 
 def run_pipeline(ta, buf, wl, read_back=False, per_call=None, stream=None):
@@ -158,6 +159,10 @@ def run_pipeline(ta, buf, wl, read_back=False, per_call=None, stream=None):
             mark("blame_gaps + aggregate_ops(OP, idle charged) (outside the timed step)")
             w.rollup_operators()
             mark("rollup_operators (outside the timed step)")
+            if SOL_WORK is not None:
+                from paper_2609_40247_b200 import synth as _synth
+                w.operator_sol(SOL_WORK[0], SOL_WORK[1], _synth.PEAK_FLOPS, _synth.PEAK_BW)
+                mark("operator_sol (outside the timed step)")
             w.critical_path()
             mark("critical_path (outside the timed step)")
         nbytes = w.load_summary.nbytes + j.join_sum.nbytes + a.attr_sum.nbytes
@@ -372,10 +377,14 @@ def main():
     ta.profile_enable(False)
 
     # ---- per-call breakdown (outside the timed region) ----
+    global SOL_WORK
+    fl, nb = synth.op_work(wl.events, seed=1)
+    SOL_WORK = (torch.from_numpy(fl).to(dev), torch.from_numpy(nb).to(dev))
     per_call = {}
     for _ in range(3):
         run_pipeline(ta, dev_buf, wl, per_call=per_call)
     per_call_ms = {k: round(min(v), 4) for k, v in per_call.items()}
+    SOL_WORK = None
 
     # ---- end to end: pinned host input, host<->device copies inside the timed region ----
     e2e = None
