@@ -226,9 +226,9 @@ def built_path_bytes_per_event(wl, radix_bytes_per_event):
                 + (2.0 + f_K * 36.0 + 20.0 + f_K * 4.0)   # probe: kind, corr, ts, slot, launch ts/te; 3 outputs; kol
                 + (2.0 + f_l * 8.0),                  # launch statistics: kind, slot, kol
         "attribute": 28.0 + (2.0 + f_h * 8.0)         # per-operator fill; tile stacks: kind, ts_end
-                     + (2.0 + f_h * 16.0 + 5.0)       # resolve: kind, ts pair; parent, depth
-                     + (2.0 + f_K * (4.0 + 16.0 + 4.0 + 32.0) + 4.0)   # inherit: launch_of, ts pair, parent, 4 atomics; op_of
-                     + (2.0 + f_o * 36.0),            # finalize: kind, count, first/last rewritten
+                     + (2.0 + f_h * 16.0 + 5.0 + f_l * 12.0)   # resolve: kind, ts pair; parent, depth; kernels of the launch, count added to its operator
+                     + (2.0 + f_K * (4.0 + 16.0 + 4.0 + 24.0) + 4.0)   # inherit: launch_of, ts pair, parent, 3 atomics; op_of
+                     + (4.0 + f_o * 32.0),            # finalize: count; first/last read and rewritten
         "gaps": 2.0 + f_d * 16.0 + 8.0,
         "aggregate": (2.0 + f_d * 20.0) + (2.0 + f_o * 24.0),
         "collectives": 8.0 + 2.0 + f_c * 100.0,       # wait fill, kind, compaction + pair sort + groups
