@@ -25,7 +25,8 @@ struct SolArgs {
   const int64_t *op_first, *op_last;
   const double *flops, *bytes;  // per input record
   double peak_flops, peak_bw;
-  const int32_t *lane_off, *lane_window;
+  const int32_t *lane_off, *lane_window, *lane_dom_end;
+  const int16_t *lane_domain;
   double *mfu, *mbu, *sol;
   uint8_t *state;
   ta_sol_summary *sum;  // device, per window
@@ -46,26 +47,110 @@ __device__ __forceinline__ void sol_add(ta_sol_summary *s, u64 n1, u64 n2, u64 n
   if (n3) atomicAdd((u64 *)&s->n_no_counts, n3);
 }
 
-__global__ void __launch_bounds__(SO_THREADS) k_operator_sol(SolArgs a) {
-  const int err = ta_peek_err(a.status);
-  const int64_t p0 = ((int64_t)blockIdx.x * SO_THREADS + threadIdx.x) * SO_ITEMS;
-  int16_t kd[SO_ITEMS];
-  loadn_i16<SO_ITEMS>(a.kind, p0, a.n, 9, kd);
-  if (ta_is_failure(err)) return;
-  unsigned ops = 0;
+__device__ __forceinline__ void sol_store_zero(const SolArgs &a, int64_t p0) {
+  if (p0 + SO_ITEMS <= a.n) {
+    double2 *pm = reinterpret_cast<double2 *>(a.mfu + p0), *pb = reinterpret_cast<double2 *>(a.mbu + p0);
+    double2 *ps = reinterpret_cast<double2 *>(a.sol + p0);
 #pragma unroll
-  for (int j = 0; j < SO_ITEMS; j++)
-    if (p0 + j < a.n_valid && kd[j] == TA_KIND_OP) ops |= 1u << j;
-  double mfu[SO_ITEMS], mbu[SO_ITEMS], sol[SO_ITEMS];
-  uint8_t st[SO_ITEMS];
+    for (int q = 0; q < SO_ITEMS / 2; q++) pm[q] = pb[q] = ps[q] = make_double2(0.0, 0.0);
+    *reinterpret_cast<u32 *>(a.state + p0) = 0u;
+  } else {
+    for (int j = 0; j < SO_ITEMS; j++)
+      if (p0 + j < a.n) { a.mfu[p0 + j] = a.mbu[p0 + j] = a.sol[p0 + j] = 0.0; a.state[p0 + j] = 0; }
+  }
+}
+
+// Per-window sums of one CTA: every thread keeps its share in registers while the CTA stays inside
+// one window; the CTA folds and adds them to the window's row when it moves on (a row takes seven
+// atomics on the same addresses, so adding per warp would serialise the whole grid on them).
+struct SolAcc {
+  u64 n1, n2, n3, top;
+  double f, b, mx;
+  __device__ __forceinline__ void clear() { n1 = n2 = n3 = top = 0; f = b = mx = 0.0; }
+};
+
+__device__ __forceinline__ void sol_flush(SolAcc &acc, ta_sol_summary *row, u64 (*red)[SO_THREADS / 32]) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const u64 n1 = warp_reduce(acc.n1, OpAdd()), n2 = warp_reduce(acc.n2, OpAdd());
+  const u64 n3 = warp_reduce(acc.n3, OpAdd()), top = warp_reduce(acc.top, OpAdd());
+  double f = acc.f, b = acc.b, mx = acc.mx;
 #pragma unroll
-  for (int j = 0; j < SO_ITEMS; j++) { mfu[j] = mbu[j] = sol[j] = 0.0; st[j] = 0; }
-  u64 n1 = 0, n2 = 0, n3 = 0, top_sum = 0;
-  double fs = 0.0, bs = 0.0, mx = 0.0;
-  int win = -1;
-  if (ops) {
-    int l = lane_of_pos(a.lane_off, a.n_lanes, p0);
-    int64_t next_off = a.lane_off[l + 1];
+  for (int o = 16; o > 0; o >>= 1) {
+    f += __shfl_xor_sync(0xffffffffu, f, o);
+    b += __shfl_xor_sync(0xffffffffu, b, o);
+    const double t = __shfl_xor_sync(0xffffffffu, mx, o);
+    mx = t > mx ? t : mx;
+  }
+  __syncthreads();  // red may still be read by the flush before
+  if (lane == 0) {
+    red[0][warp] = n1; red[1][warp] = n2; red[2][warp] = n3; red[3][warp] = top;
+    red[4][warp] = (u64)__double_as_longlong(f); red[5][warp] = (u64)__double_as_longlong(b);
+    red[6][warp] = (u64)__double_as_longlong(mx);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u64 t1 = 0, t2 = 0, t3 = 0, tt = 0;
+    double tf = 0.0, tb = 0.0, tm = 0.0;
+    for (int w = 0; w < SO_THREADS / 32; w++) {
+      t1 += red[0][w]; t2 += red[1][w]; t3 += red[2][w]; tt += red[3][w];
+      tf += __longlong_as_double((i64)red[4][w]);
+      tb += __longlong_as_double((i64)red[5][w]);
+      const double m = __longlong_as_double((i64)red[6][w]);
+      tm = m > tm ? m : tm;
+    }
+    sol_add(row, t1, t2, t3, tt, tf, tb, tm);
+  }
+  acc.clear();
+}
+
+// Persistent CTAs, each over a contiguous range of tiles.
+__global__ void __launch_bounds__(SO_THREADS) k_operator_sol(SolArgs a, int64_t n_tiles, int64_t tiles_per_cta) {
+  __shared__ int s_lane0, s_lane1;
+  __shared__ u64 red[7][SO_THREADS / 32];
+  if (ta_failed(a.status)) return;
+  const int tid = threadIdx.x;
+  SolAcc acc;
+  acc.clear();
+  int cw = -1;  // window the registers hold sums of (the same in every thread)
+  const int64_t t_begin = (int64_t)blockIdx.x * tiles_per_cta;
+  const int64_t t_end = min(t_begin + tiles_per_cta, n_tiles);
+  for (int64_t tile = t_begin; tile < t_end; tile++) {
+    const int64_t tile_start = tile * SO_TILE;
+    const int64_t p0 = tile_start + (int64_t)tid * SO_ITEMS;
+    const int64_t valid_end = min(tile_start + SO_TILE, a.n_valid);
+    __syncthreads();  // the lanes of the tile before have been read
+    if (tid < 64) {
+      // warp 0: lane of the tile's first record; warp 1: lane of its last kept record
+      int l = -1;
+      if (tile_start < a.n_valid && a.n_lanes > 0)
+        l = tile_lane_search(a.lane_off, a.n_lanes, tid < 32 ? tile_start : valid_end - 1);
+      if (tid == 0) s_lane0 = l;
+      if (tid == 32) s_lane1 = l;
+    }
+    __syncthreads();
+    const int l0 = s_lane0, l1 = s_lane1;
+    // Operators sit in host lanes: a tile of device lanes (or of dropped records) is all zeros
+    // and reads nothing.
+    if (l0 < 0 || span_outside_domain(a.lane_domain, a.lane_dom_end, l0, valid_end, 0)) {
+      sol_store_zero(a, p0);
+      continue;
+    }
+    // one window per tile, almost always: its sums stay in registers.  A tile that spans windows
+    // (at most one per window boundary) adds record by record.
+    const int w_first = a.lane_window[l0];
+    const bool one_window = w_first == a.lane_window[l1];
+    if (cw >= 0 && (!one_window || w_first != cw)) { sol_flush(acc, &a.sum[cw], red); cw = -1; }
+    if (one_window) cw = w_first;
+    int16_t kd[SO_ITEMS];
+    loadn_i16<SO_ITEMS>(a.kind, p0, a.n, 9, kd);
+    unsigned ops = 0;
+#pragma unroll
+    for (int j = 0; j < SO_ITEMS; j++)
+      if (p0 + j < a.n_valid && kd[j] == TA_KIND_OP) ops |= 1u << j;
+    if (!ops) {
+      sol_store_zero(a, p0);
+      continue;
+    }
     // counts and times of the thread's OP records first, then the two gathers of those that
     // own kernels, so that the misses overlap
     i64 top[SO_ITEMS];
@@ -85,67 +170,59 @@ __global__ void __launch_bounds__(SO_THREADS) k_operator_sol(SolArgs a) {
       f[j] = b[j] = -1.0;
       if (src[j] >= 0) { f[j] = a.flops[src[j]]; b[j] = a.bytes[src[j]]; }
     }
-#pragma unroll
-    for (int j = 0; j < SO_ITEMS; j++) {
-      if (!(ops & (1u << j))) continue;
-      const int64_t p = p0 + j;
-      while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
-      const int w = a.lane_window[l];
-      u64 c1 = 0, c2 = 0, c3 = 0;
-      if (top[j] <= 0) { st[j] = 2; c2 = 1; }
-      else if (!(f[j] >= 0.0) || !(b[j] >= 0.0)) { st[j] = 3; c3 = 1; }
-      else {
-        // the same operations in the same order as the definition: no sum, so nothing fuses
-        const double seconds = (double)top[j] * 1e-9;
-        mfu[j] = f[j] / (seconds * a.peak_flops);
-        mbu[j] = b[j] / (seconds * a.peak_bw);
-        sol[j] = mfu[j] > mbu[j] ? mfu[j] : mbu[j];
-        st[j] = 1;
-        c1 = 1;
-      }
-      if (win < 0) win = w;
-      if (w == win) {
-        n1 += c1; n2 += c2; n3 += c3;
-        if (c1) { top_sum += (u64)top[j]; fs += f[j]; bs += b[j]; mx = sol[j] > mx ? sol[j] : mx; }
-      } else {  // a thread that straddles two windows
-        sol_add(&a.sum[w], c1, c2, c3, c1 ? (u64)top[j] : 0, c1 ? f[j] : 0.0, c1 ? b[j] : 0.0, sol[j]);
-      }
-    }
-  }
-  if (p0 + SO_ITEMS <= a.n) {
-    double2 *pm = reinterpret_cast<double2 *>(a.mfu + p0), *pb = reinterpret_cast<double2 *>(a.mbu + p0);
-    double2 *ps = reinterpret_cast<double2 *>(a.sol + p0);
+    int l = l0;
+    int64_t next_off = a.lane_off[l + 1];
+    u32 st_word = 0;
+    const bool whole = p0 + SO_ITEMS <= a.n;
 #pragma unroll
     for (int q = 0; q < SO_ITEMS / 2; q++) {
-      pm[q] = make_double2(mfu[2 * q], mfu[2 * q + 1]);
-      pb[q] = make_double2(mbu[2 * q], mbu[2 * q + 1]);
-      ps[q] = make_double2(sol[2 * q], sol[2 * q + 1]);
-    }
-    *reinterpret_cast<u32 *>(a.state + p0) = st[0] | (st[1] << 8) | (st[2] << 16) | ((u32)st[3] << 24);
-  } else {
+      double mfu[2] = {0.0, 0.0}, mbu[2] = {0.0, 0.0}, sol[2] = {0.0, 0.0};
 #pragma unroll
-    for (int j = 0; j < SO_ITEMS; j++)
-      if (p0 + j < a.n) { a.mfu[p0 + j] = mfu[j]; a.mbu[p0 + j] = mbu[j]; a.sol[p0 + j] = sol[j]; a.state[p0 + j] = st[j]; }
-  }
-  // fold per warp when the warp sits in one window (almost always)
-  const int lane = threadIdx.x & 31;
-  const u32 has = __ballot_sync(0xffffffffu, win >= 0);
-  if (!has) return;
-  const int w0 = __shfl_sync(0xffffffffu, win, __ffs(has) - 1);
-  if (__all_sync(0xffffffffu, win < 0 || win == w0)) {
-    n1 = warp_reduce(n1, OpAdd()); n2 = warp_reduce(n2, OpAdd()); n3 = warp_reduce(n3, OpAdd());
-    top_sum = warp_reduce(top_sum, OpAdd());
+      for (int h = 0; h < 2; h++) {
+        const int j = 2 * q + h;
+        if (!(ops & (1u << j))) continue;
+        u64 c1 = 0, c2 = 0, c3 = 0;
+        u32 st = 0;
+        if (top[j] <= 0) { st = 2; c2 = 1; }
+        else if (!(f[j] >= 0.0) || !(b[j] >= 0.0)) { st = 3; c3 = 1; }
+        else {
+          // the same operations in the same order as the definition: no sum, so nothing fuses
+          const double seconds = (double)top[j] * 1e-9;
+          mfu[h] = f[j] / (seconds * a.peak_flops);
+          mbu[h] = b[j] / (seconds * a.peak_bw);
+          sol[h] = mfu[h] > mbu[h] ? mfu[h] : mbu[h];
+          st = 1;
+          c1 = 1;
+        }
+        st_word |= st << (8 * j);
+        if (one_window) {
+          acc.n1 += c1; acc.n2 += c2; acc.n3 += c3;
+          if (c1) { acc.top += (u64)top[j]; acc.f += f[j]; acc.b += b[j]; acc.mx = sol[h] > acc.mx ? sol[h] : acc.mx; }
+        } else {
+          const int64_t p = p0 + j;
+          while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+          sol_add(&a.sum[a.lane_window[l]], c1, c2, c3, c1 ? (u64)top[j] : 0, c1 ? f[j] : 0.0,
+                  c1 ? b[j] : 0.0, sol[h]);
+        }
+      }
+      if (whole) {
+        reinterpret_cast<double2 *>(a.mfu + p0)[q] = make_double2(mfu[0], mfu[1]);
+        reinterpret_cast<double2 *>(a.mbu + p0)[q] = make_double2(mbu[0], mbu[1]);
+        reinterpret_cast<double2 *>(a.sol + p0)[q] = make_double2(sol[0], sol[1]);
+      } else {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      fs += __shfl_xor_sync(0xffffffffu, fs, o);
-      bs += __shfl_xor_sync(0xffffffffu, bs, o);
-      const double t = __shfl_xor_sync(0xffffffffu, mx, o);
-      mx = t > mx ? t : mx;
+        for (int h = 0; h < 2; h++)
+          if (p0 + 2 * q + h < a.n) {
+            a.mfu[p0 + 2 * q + h] = mfu[h]; a.mbu[p0 + 2 * q + h] = mbu[h]; a.sol[p0 + 2 * q + h] = sol[h];
+          }
+      }
     }
-    if (lane == 0) sol_add(&a.sum[w0], n1, n2, n3, top_sum, fs, bs, mx);
-  } else if (win >= 0) {
-    sol_add(&a.sum[win], n1, n2, n3, top_sum, fs, bs, mx);
+    if (whole) *reinterpret_cast<u32 *>(a.state + p0) = st_word;
+    else
+      for (int j = 0; j < SO_ITEMS; j++)
+        if (p0 + j < a.n) a.state[p0 + j] = (uint8_t)(st_word >> (8 * j));
   }
+  if (cw >= 0) sol_flush(acc, &a.sum[cw], red);
 }
 
 ta_status ta_run_sol(ta_window *h, const double *flops, const double *bytes, int on_device,
@@ -180,8 +257,12 @@ ta_status ta_run_sol(ta_window *h, const double *flops, const double *bytes, int
   a.op_first = h->attr.op_first_start; a.op_last = h->attr.op_last_end;
   a.flops = flops; a.bytes = bytes; a.peak_flops = peak_flops; a.peak_bw = peak_bw;
   a.lane_off = h->sorted.lane_off; a.lane_window = h->sorted.lane_window; a.status = h->d_status;
+  a.lane_domain = h->sorted.lane_domain; a.lane_dom_end = h->d_lane_dom_end;
   if (n > 0) {
-    k_operator_sol<<<TA_N (unsigned)((n + SO_TILE - 1) / SO_TILE), SO_THREADS, 0, st>>>(a);
+    const int64_t n_tiles = (n + SO_TILE - 1) / SO_TILE;
+    const int64_t ctas = n_tiles < 148 * 8 ? n_tiles : 148 * 8;
+    const int64_t per = (n_tiles + ctas - 1) / ctas;
+    k_operator_sol<<<TA_N (unsigned)((n_tiles + per - 1) / per), SO_THREADS, 0, st>>>(a, n_tiles, per);
     TA_CHECK_CUDA(h, cudaGetLastError());
   }
   std::vector<ta_sol_summary> hs(W);

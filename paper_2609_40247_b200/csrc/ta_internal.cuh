@@ -321,6 +321,22 @@ __device__ __forceinline__ u64 warp_reduce(u64 v, Op op) {
   for (int o = 16; o > 0; o >>= 1) v = op(v, __shfl_xor_sync(0xffffffffu, v, o));
   return v;
 }
+// Maximum over the warp in two hardware reductions (high words, then the low words of the lanes
+// that hold the largest high word) instead of five shuffle rounds on 64-bit values.
+__device__ __forceinline__ u64 warp_reduce(u64 v, OpMax) {
+  const u32 hi = (u32)(v >> 32);
+  const u32 mh = __reduce_max_sync(0xffffffffu, hi);
+  const u32 ml = __reduce_max_sync(0xffffffffu, hi == mh ? (u32)v : 0u);
+  return ((u64)mh << 32) | ml;
+}
+// Sum over the warp (mod 2^64) in three hardware reductions: limbs of 22 bits, so that 32 of
+// them cannot overflow a 32-bit sum.
+__device__ __forceinline__ u64 warp_reduce(u64 v, OpAdd) {
+  const u32 s0 = __reduce_add_sync(0xffffffffu, (u32)v & 0x3FFFFFu);
+  const u32 s1 = __reduce_add_sync(0xffffffffu, (u32)(v >> 22) & 0x3FFFFFu);
+  const u32 s2 = __reduce_add_sync(0xffffffffu, (u32)(v >> 44));
+  return (u64)s0 + ((u64)s1 << 22) + ((u64)s2 << 44);
+}
 template <class Op>
 __device__ __forceinline__ u64 warp_scan_inclusive(u64 v, Op op) {
   const int lane = threadIdx.x & 31;
