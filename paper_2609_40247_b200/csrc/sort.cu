@@ -38,6 +38,7 @@ struct RadixArgs {
   u64 *tile_state;        // [tile][RS_BINS]
   u32 *tile_counter;
   int32_t *status;
+  u32 gen;                // 1 + pass index: tags this pass's tile descriptors
   PrekeyInfo pk;          // PREKEY passes only
 };
 
@@ -56,6 +57,43 @@ __device__ __forceinline__ u64 prekey_to_key(const PrekeyInfo &k, u64 w64, int w
          ((w64 & ((1ull << RS_PRE_TS_BITS) - 1)) >> k.dshift);
   }
   return (hi << k.ibits) | (u64)(i - k.off[w]);
+}
+
+// Tile descriptors of the pair passes (the small sorts: long-gap list, collective keys) carry the
+// pass they belong to, so that one clearing of the descriptor array serves every pass of a sort:
+// [status, 2 bits][pass tag, 6 bits][count, 56 bits]; a descriptor whose tag is not the running
+// pass's is as good as empty.  The keys-only passes (the timeline sort: 16 k tiles) keep plain
+// descriptors and a clearing per pass: the tag test cost them 11 us per pass, more than the
+// clearings it saves.
+#define RS_GEN_SHIFT 56
+#define RS_VMASK ((1ull << RS_GEN_SHIFT) - 1)
+template <bool GEN>
+__device__ __forceinline__ u64 rs_pack(u64 flag, u32 gen, u64 v) {
+  return GEN ? (flag << 62) | ((u64)gen << RS_GEN_SHIFT) | (v & RS_VMASK) : td_pack(flag, v);
+}
+template <bool GEN>
+__device__ __forceinline__ bool rs_ready(u64 x, u32 gen) {
+  return GEN ? (u32)(x >> RS_GEN_SHIFT & 0x3Fu) == gen : (x >> 62) != TD_EMPTY;
+}
+// bounded wait for a descriptor of this pass, as td_wait
+template <bool GEN>
+__device__ __forceinline__ u64 rs_wait(const u64 *p, u32 gen, int32_t *status, bool *timed_out) {
+  u64 w = ld_relaxed(p);
+  int spins = 0, limit = 0;
+  while (!rs_ready<GEN>(w, gen)) {
+    if (limit == 0) {
+      limit = ld_relaxed_i32(&status[ST_SPIN]);
+      if (limit <= 0) limit = TA_SPIN_LIMIT;
+    }
+    if (++spins > limit || ta_is_failure(ld_relaxed_i32(&status[ST_ERR]))) {
+      *timed_out = true;
+      ta_set_err(status, TA_ERR_TIMEOUT);
+      return rs_pack<GEN>(TD_PREFIX, gen, 0);
+    }
+    __nanosleep(40);
+    w = ld_relaxed(p);
+  }
+  return w;
 }
 
 template <int THREADS, int ITEMS>
@@ -177,8 +215,8 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
   // and the look back over the earlier tiles comes last, when they have had time to publish
   u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
   if (tid < (1 << BITS)) {
-    if (tile == 0) st_relaxed(st, td_pack(TD_PREFIX, (u64)a.bin_offset[tid] + cnt));
-    else st_relaxed(st, td_pack(TD_AGG, cnt));
+    if (tile == 0) st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, (u64)a.bin_offset[tid] + cnt));
+    else st_relaxed(st, rs_pack<VALS>(TD_AGG, a.gen, cnt));
   }
   __syncthreads();
 #pragma unroll
@@ -206,15 +244,15 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
 #pragma unroll
         for (int i = 0; i < RS_LOOKBACK_BATCH; i++)
           lb[i] = lb_t - i >= 0 ? ld_relaxed(a.tile_state + (size_t)(lb_t - i) * RS_BINS + tid)
-                                : td_pack(TD_PREFIX, 0);
+                                : rs_pack<VALS>(TD_PREFIX, a.gen, 0);
         bool done = false;
 #pragma unroll
         for (int i = 0; i < RS_LOOKBACK_BATCH; i++) {
           if (done) continue;
           u64 x = lb[i];
-          if ((x >> 62) == TD_EMPTY)
-            x = td_wait(a.tile_state + (size_t)(lb_t - i) * RS_BINS + tid, a.status, &timed_out);
-          excl += x & TD_MASK;
+          if (!rs_ready<VALS>(x, a.gen))
+            x = rs_wait<VALS>(a.tile_state + (size_t)(lb_t - i) * RS_BINS + tid, a.gen, a.status, &timed_out);
+          excl += x & (VALS ? RS_VMASK : TD_MASK);
           if ((x >> 62) == TD_PREFIX) done = true;
         }
         if (done) break;
@@ -222,7 +260,7 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
       // a wait that gave up leaves the descriptor at its aggregate: the tiles behind this one
       // look past it, meet the same unpublished tile (or the error word) and give up as well
       if (timed_out) s.fail = 1;
-      else st_relaxed(st, td_pack(TD_PREFIX, excl + cnt));
+      else st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, excl + cnt));
     }
     s.adj[tid] = (u32)excl - (u32)ex;
   }
@@ -388,18 +426,22 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     hist = own_hist;
   }
   k_radix_scan_hist<<<TA_N plan.n_pass, 256, 0, st>>>(hist, bin_offset);
+  // one clearing for all passes of a pair sort (descriptors tagged with their pass); every pass
+  // draws its tile tickets from a counter of its own (state and counters are neighbours)
+  TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, (size_t)((char *)(counter + 16) - (char *)state), st));
   const u64 *kin = keys_in;
   const u32 *vin = vals_in;
   for (int p = 0; p < plan.n_pass; p++) {
     bool to_final = ((plan.n_pass - 1 - p) & 1) == 0;
-    TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * RS_BINS * sizeof(u64), st));
-    TA_CHECK_CUDA(h, cudaMemsetAsync(counter, 0, sizeof(u32), st));
     RadixArgs a = RadixArgs();
     a.keys_in = kin; a.keys_out = to_final ? keys_final : keys_scratch;
     a.vals_in = vin; a.vals_out = to_final ? vals_final : vals_scratch;
     a.n = n; a.shift = plan.shift[p];
     a.bin_offset = bin_offset + p * RS_BINS;
-    a.tile_state = state; a.tile_counter = counter; a.status = h->d_status;
+    if (!VALS && p > 0)  // untagged descriptors: cleared in front of every pass
+      TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * RS_BINS * sizeof(u64), st));
+    a.tile_state = state; a.tile_counter = counter + p; a.status = h->d_status;
+    a.gen = VALS ? (u32)(p + 1) : 0u;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
     if (timed) ta_profile_mark(st, 1, (VALS ? 24.0 : 16.0) * (double)n);
     bool launched = false;

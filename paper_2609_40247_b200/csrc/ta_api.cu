@@ -147,7 +147,7 @@ static unsigned char *pin_take() {
     }
   }
   void *p = nullptr;
-  if (cudaHostAlloc(&p, TA_PIN_BYTES, cudaHostAllocPortable) != cudaSuccess) {
+  if (cudaHostAlloc(&p, TA_PIN_BYTES, cudaHostAllocPortable | cudaHostAllocMapped) != cudaSuccess) {
     cudaGetLastError();
     return nullptr;  // the copies then go straight to their (pageable) destinations
   }
@@ -159,10 +159,46 @@ static void pin_put(unsigned char *p) {
   g_pin_free.push_back(p);
 }
 
+// Writes up to TA_FETCH_MAX small device regions into the mapped staging block: one launch in
+// place of one copy each (a copy costs some six microseconds of stream time, however small).
+#define TA_FETCH_MAX 8
+#define TA_FETCH_BYTES (16u << 10)
+struct FetchList {
+  const void *src[TA_FETCH_MAX];
+  unsigned off[TA_FETCH_MAX], bytes[TA_FETCH_MAX];
+};
+__global__ void __launch_bounds__(256) k_collect(FetchList f, unsigned char *pin_dev) {
+  const unsigned char *s = (const unsigned char *)f.src[blockIdx.x];
+  unsigned char *d = pin_dev + f.off[blockIdx.x];
+  const unsigned b = f.bytes[blockIdx.x];
+  if ((((uintptr_t)s | (uintptr_t)b) & 7u) == 0) {
+    for (unsigned i = threadIdx.x; i < b / 8; i += blockDim.x)
+      reinterpret_cast<u64 *>(d)[i] = reinterpret_cast<const u64 *>(s)[i];
+  } else {
+    for (unsigned i = threadIdx.x; i < b; i += blockDim.x) d[i] = s[i];
+  }
+}
+static ta_status flush_fetch(ta_window *h) {
+  if (h->fetch.empty()) return TA_OK;
+  FetchList f;
+  memset(&f, 0, sizeof(f));
+  const unsigned m = (unsigned)h->fetch.size();
+  for (unsigned i = 0; i < m; i++) { f.src[i] = h->fetch[i].src; f.off[i] = h->fetch[i].off; f.bytes[i] = h->fetch[i].bytes; }
+  h->fetch.clear();
+  k_collect<<<TA_N m, 256, 0, h->stream>>>(f, h->pin_dev);
+  TA_CHECK_CUDA(h, cudaGetLastError());
+  return TA_OK;
+}
+
 ta_status ta_queue_d2h(ta_window *h, void *dst, const void *dev_src, size_t bytes) {
   if (bytes == 0) return TA_OK;
   const size_t need = (bytes + 15) & ~(size_t)15;
-  if (h->pin && h->pin_used + need <= h->pin_bytes) {
+  if (h->pin_dev && bytes <= TA_FETCH_BYTES && h->pin_used + need <= h->pin_bytes) {
+    if (h->fetch.size() == TA_FETCH_MAX) TA_TRY(flush_fetch(h));
+    h->fetch.push_back(ta_window::Fetch{dev_src, (unsigned)h->pin_used, (unsigned)bytes});
+    h->pending.push_back(ta_window::Pending{dst, h->pin_used, bytes});
+    h->pin_used += need;
+  } else if (h->pin && h->pin_used + need <= h->pin_bytes) {
     TA_CHECK_CUDA(h, cudaMemcpyAsync(h->pin + h->pin_used, dev_src, bytes, cudaMemcpyDeviceToHost, h->stream));
     h->pending.push_back(ta_window::Pending{dst, h->pin_used, bytes});
     h->pin_used += need;
@@ -175,6 +211,8 @@ ta_status ta_queue_d2h(ta_window *h, void *dst, const void *dev_src, size_t byte
 static void release_one(ta_window *h, void *p, size_t bytes);
 
 ta_status ta_sync_fetch(ta_window *h) {
+  const ta_status fs = flush_fetch(h);
+  if (fs != TA_OK) { h->pending.clear(); h->pin_used = 0; return fs; }
   const cudaError_t e = cudaStreamSynchronize(h->stream);
   if (e == cudaSuccess)
     for (const ta_window::Pending &q : h->pending) memcpy(q.dst, h->pin + q.off, q.bytes);
@@ -203,6 +241,7 @@ void ta_dfree_later(ta_window *h, void *p) {
 // Also makes the handle's device current (it stays current when the call returns).
 static ta_status begin_call(ta_window *h) {
   h->pending.clear();
+  h->fetch.clear();
   h->pin_used = 0;
   if (cudaSetDevice(h->device) != cudaSuccess) {
     h->last_cuda = cudaGetLastError();
@@ -456,6 +495,12 @@ ta_status ta_load_window(const ta_env *env, const ta_event *events, int64_t n,
   h->d_status = nullptr;
   h->pin = pin_take();
   h->pin_bytes = h->pin ? TA_PIN_BYTES : 0;
+  h->pin_dev = nullptr;
+  if (h->pin) {
+    void *dp = nullptr;
+    if (cudaHostGetDevicePointer(&dp, h->pin, 0) == cudaSuccess) h->pin_dev = (unsigned char *)dp;
+    else cudaGetLastError();
+  }
   h->pin_used = 0;
   h->h_off.assign(win_off, win_off + W + 1);
   h->h_t0.assign(win_t0, win_t0 + W);

@@ -97,6 +97,11 @@ struct ta_window {
   size_t pin_bytes, pin_used;
   struct Pending { void *dst; size_t off, bytes; };
   std::vector<Pending> pending;
+  // small results (status words, per-window summaries) are not copied one by one: one kernel
+  // at the end of the call writes them all into the staging block through its device alias
+  unsigned char *pin_dev;  // device address of `pin`, null when the block is not mapped
+  struct Fetch { const void *src; unsigned off, bytes; };
+  std::vector<Fetch> fetch;
 
   // load products
   int32_t *d_status;
