@@ -497,14 +497,14 @@ def main():
         radix_per_event = (radix_bytes / radix_steps / n) if (n_pass > 0 and n > 0) else 0.0
         built_bytes, built_parts = built_path_bytes_per_event(wl, radix_per_event)
         line["hbm_model"] = {
-            # headline: the bytes the path as built touches (kernel-by-kernel table of the design doc)
+            # headline: the bytes the path as built touches (kernel by kernel, built_path_bytes_per_event)
             "built_bytes_per_event": round(built_bytes, 2),
             "built_parts": {k: round(v, 2) for k, v in built_parts.items()},
             "radix_passes_per_step": (n_pass / radix_steps) if n_pass else 0,
             "frac_of_measured_peak": per_gpu * built_bytes / (peak * 1e9),
             "frac_of_nominal_8TBs": per_gpu * built_bytes / 8.0e12,
             "target_ms_for_half_of_measured_peak": 2e3 * n * built_bytes / (peak * 1e9),
-            # secondary: the survey's model of an LSD sort of (key, index) pairs, one pass per key
+            # secondary: the byte model of an LSD sort of (key, index) pairs, one pass per key
             # byte - a different algorithm's bytes - and the compulsory bytes alone
             "lsd_bytes_per_event": round(lsd_bytes, 2), "lsd_key_bits": key_bits, "lsd_passes": passes,
             "lsd_parts": {k: round(v, 2) for k, v in parts.items()},

@@ -217,7 +217,7 @@ __device__ __forceinline__ void mbar_init(u64 *bar, u32 count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
 }
 // one tile of whole records from this GPU's memory into shared memory: a 1-D bulk copy (no
-// tensor map, no multicast) that reports its bytes to the barrier
+// tensor map; the copy goes to this CTA alone) that reports its bytes to the barrier
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, u32 bytes, u64 *bar) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                : "memory");
