@@ -101,6 +101,7 @@ struct RadixSmem {
   u64 keys[THREADS * ITEMS];  // aliased by u32 values after the keys are written out
   u32 warp_hist[THREADS / 32][RS_BINS];  // per warp: digit counts, later tile-local start of the warp's run
   u32 adj[RS_BINS];           // global position of a digit's run minus its tile-local start (mod 2^32)
+  u32 pcnt[RS_BINS];          // keys-only passes: the digit counts, for the thread that publishes two digits
   u64 scan_tmp[33];
   int tile;
   int fail;
@@ -206,9 +207,11 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
 #pragma unroll
     for (int w = 0; w < WARPS; w++) cnt += s.warp_hist[w][tid];
   }
+  if (!VALS && tid < RS_BINS) s.pcnt[tid] = cnt;  // visible after the scan's barriers
   u64 total;
   const u64 ex = block_scan_exclusive<OpAdd>((u64)cnt, OpAdd(), s.scan_tmp, &total);
   if (tid < RS_BINS) {
+    if (!VALS) s.adj[tid] = (u32)ex;  // read by the digit's publisher after the next barrier
     u32 run = (u32)ex;
 #pragma unroll
     for (int w = 0; w < WARPS; w++) {
@@ -217,13 +220,29 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
       run += t;
     }
   }
-  // chained scan over tiles, one digit per thread: the tile's own count is published first,
-  // the keys are staged in shared memory in digit order (which needs tile-local offsets only),
-  // and the look back over the earlier tiles comes last, when they have had time to publish
-  u64 *st = a.tile_state + (size_t)tile * RS_BINS + tid;
-  if (tid < (1 << BITS)) {
-    if (tile == 0) st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, (u64)a.bin_offset[tid] + cnt));
-    else st_relaxed(st, rs_pack<VALS>(TD_AGG, a.gen, cnt));
+  // chained scan over tiles: the tile's own counts are published first, the keys are staged in
+  // shared memory in digit order (which needs tile-local offsets only), and the look back over
+  // the earlier tiles comes last, when they have had time to publish.
+  // Pair passes: one digit per thread and descriptor.  Keys-only passes: TWO digits per thread
+  // and descriptor, [status, 2 bits][digit d + NB/2, 31 bits][digit d, 31 bits] - counts and
+  // prefixes stay below 2^31 (n < 2^31), so one 64-bit add sums both without a carry between
+  // them, and half as many threads walk half as many descriptors.
+  constexpr int NB = 1 << BITS, HB = NB / 2;
+  constexpr int PER_TILE = VALS ? RS_BINS : RS_BINS / 2;
+  constexpr int WALKERS = VALS ? NB : HB;
+  u64 *st = a.tile_state + (size_t)tile * PER_TILE + tid;
+  u32 cnt_hi = 0;  // keys-only: count of digit tid + HB
+  if (tid < WALKERS) {
+    if (VALS) {
+      if (tile == 0) st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, (u64)a.bin_offset[tid] + cnt));
+      else st_relaxed(st, rs_pack<VALS>(TD_AGG, a.gen, cnt));
+    } else {
+      cnt_hi = s.pcnt[tid + HB];
+      if (tile == 0)
+        st_relaxed(st, td_pack(TD_PREFIX, ((u64)(a.bin_offset[tid + HB] + cnt_hi) << 31) | (a.bin_offset[tid] + cnt)));
+      else
+        st_relaxed(st, td_pack(TD_AGG, ((u64)cnt_hi << 31) | cnt));
+    }
   }
   __syncthreads();
 #pragma unroll
@@ -235,44 +254,49 @@ __device__ __forceinline__ void radix_tile(const RadixArgs &a, RadixSmem<THREADS
       s.keys[r] = key[j];
     }
   }
-  if (tid < (1 << BITS)) {
-    u64 excl;
+  if (tid < WALKERS) {
+    u64 sum = 0;  // pair passes: the exclusive prefix; keys-only passes: both of them, packed
     if (tile == 0) {
-      excl = a.bin_offset[tid];
+      sum = VALS ? (u64)a.bin_offset[tid] : ((u64)a.bin_offset[tid + HB] << 31) | a.bin_offset[tid];
     } else {
       bool timed_out = false;
       // The walk over earlier tiles is a chain of dependent L2 reads (each some hundred
       // cycles): the descriptors of the next few tiles back are fetched together and consumed
       // in order, which divides the latency of a long walk by the batch size.  An unpublished
-      // descriptor among them is waited for with the bounded wait.  Counts fit 32 bits (n < 2^31),
-      // so the running sum is a 32-bit register; an index below tile 0 is clamped to tile 0, whose
-      // descriptor is an inclusive prefix from the start and ends the walk before it is met twice.
-      u32 sum = 0;
+      // descriptor among them is waited for with the bounded wait.  An index below tile 0 is
+      // clamped to tile 0, whose descriptor is an inclusive prefix from the start and ends the
+      // walk before it is met twice.
       const u64 *sp = a.tile_state + tid;
       for (int lb_t = tile - 1;; lb_t -= RS_LOOKBACK_BATCH) {
         u64 lb[RS_LOOKBACK_BATCH];
 #pragma unroll
         for (int i = 0; i < RS_LOOKBACK_BATCH; i++)
-          lb[i] = ld_relaxed(sp + (size_t)max(lb_t - i, 0) * RS_BINS);
+          lb[i] = ld_relaxed(sp + (size_t)max(lb_t - i, 0) * PER_TILE);
         bool done = false;
 #pragma unroll
         for (int i = 0; i < RS_LOOKBACK_BATCH; i++) {
           if (done) continue;
           u64 x = lb[i];
           if (!rs_ready<VALS>(x, a.gen))
-            x = rs_wait<VALS>(sp + (size_t)max(lb_t - i, 0) * RS_BINS, a.gen, a.status, &timed_out);
-          sum += (u32)x;
+            x = rs_wait<VALS>(sp + (size_t)max(lb_t - i, 0) * PER_TILE, a.gen, a.status, &timed_out);
+          sum += x & (VALS ? RS_VMASK : TD_MASK);
           done = (x >> 62) == TD_PREFIX;
         }
         if (done) break;
       }
-      excl = sum;
       // a wait that gave up leaves the descriptor at its aggregate: the tiles behind this one
       // look past it, meet the same unpublished tile (or the error word) and give up as well
       if (timed_out) s.fail = 1;
-      else st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, excl + cnt));
+      else if (VALS) st_relaxed(st, rs_pack<VALS>(TD_PREFIX, a.gen, sum + cnt));
+      else st_relaxed(st, td_pack(TD_PREFIX, sum + (((u64)cnt_hi << 31) | cnt)));
     }
-    s.adj[tid] = (u32)excl - (u32)ex;
+    if (VALS) {
+      s.adj[tid] = (u32)sum - (u32)ex;
+    } else {
+      const u32 ex_hi = s.adj[tid + HB];
+      s.adj[tid] = ((u32)sum & 0x7FFFFFFFu) - (u32)ex;
+      s.adj[tid + HB] = ((u32)(sum >> 31) & 0x7FFFFFFFu) - ex_hi;
+    }
   }
   __syncthreads();
   if (s.fail) return;
@@ -449,7 +473,7 @@ static ta_status radix_sort(ta_window *h, const u64 *keys_in, const u32 *vals_in
     a.n = n; a.shift = plan.shift[p];
     a.bin_offset = bin_offset + p * RS_BINS;
     if (!VALS && p > 0)  // untagged descriptors: cleared in front of every pass
-      TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * RS_BINS * sizeof(u64), st));
+      TA_CHECK_CUDA(h, cudaMemsetAsync(state, 0, tiles * (RS_BINS / 2) * sizeof(u64), st));
     a.tile_state = state; a.tile_counter = counter + p; a.status = h->d_status;
     a.gen = VALS ? (u32)(p + 1) : 0u;
     const bool timed = g_ta_profile && n == h->n;  // only the timeline sort (all records)
