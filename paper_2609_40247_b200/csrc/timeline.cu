@@ -113,24 +113,34 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   __shared__ int s_slot[8];
   __shared__ u64 s_mx[8], s_mn[8];
   if (ta_failed(a.status)) return;  // the sort gave up: the keys name no records
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  // positions fit 32 bits (n < 2^31): 32-bit indices keep the address arithmetic of the nine
+  // column stores and of the neighbour reads short
+  const u32 p = blockIdx.x * blockDim.x + threadIdx.x;
+  const u32 n = (u32)a.n, nv = (u32)a.n_valid;
   int slot = -1;
   u64 mx = 0, mn_inv = 0;
-  if (p < a.n) {
+  if (p < n) {
   u32 idx;
-  int64_t dst = p;  // where the record goes: p, or its place inside a run of equal coarse keys
+  u32 dst = p;  // where the record goes: p, or its place inside a run of equal coarse keys
   int before = 0, after = 0;
-  if (a.packed && p < a.n_valid) {
-    const u64 k = a.keys[p];
+  // the record's key and the key in front of it: both are needed twice below
+  u64 k = 0, kprev = 0;
+  if (p < nv) {
+    k = a.keys[p];
+    if (p > 0) kprev = a.keys[p - 1];
+  }
+  if (a.packed && p < nv) {
     idx = gather_index(k, a);
     // packed keys order the records down to a coarse time only: members of a run of equal
     // (lane, coarse time) sit in no particular order (the first radix pass is not stable) and
     // are ranked here by (ts_start, -ts_end, input index)
     const u64 hk = k >> a.ibits;
-    while (before <= TA_TIE_RUN_MAX && p - before > 0 && (a.keys[p - before - 1] >> a.ibits) == hk)
-      before++;
-    while (after <= TA_TIE_RUN_MAX && p + after + 1 < a.n_valid &&
-           (a.keys[p + after + 1] >> a.ibits) == hk)
+    if (p > 0 && (kprev >> a.ibits) == hk) {
+      before = 1;
+      while (before <= TA_TIE_RUN_MAX && p - before > 0 && (a.keys[p - before - 1] >> a.ibits) == hk)
+        before++;
+    }
+    while (after <= TA_TIE_RUN_MAX && p + after + 1 < nv && (a.keys[p + after + 1] >> a.ibits) == hk)
       after++;
     if (before + after + 1 > TA_TIE_RUN_MAX) {
       a.status[ST_LONG_RUN] = 1;  // the caller starts over with full-resolution keys
@@ -145,14 +155,14 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
     for (int q = -before; q <= after; q++) {
       if (q == 0) continue;
       const u32 oi = gather_index(a.keys[p + q], a);
-      const i64 *o = reinterpret_cast<const i64 *>(a.ev) + (int64_t)oi * 5;
+      const i64 *o = reinterpret_cast<const i64 *>(a.ev) + (u64)oi * 5;
       const i64 os = o[0], oe = o[1];
       const bool first = os < r.ts_start || (os == r.ts_start && (oe > r.ts_end || (oe == r.ts_end && oi < idx)));
       rank += first ? 1 : 0;
     }
     dst = p - before + rank;
   }
-  if (a.packed && p < a.n_valid) a.perm[dst] = idx;
+  if (a.packed && p < nv) a.perm[dst] = idx;
   a.ts_start[dst] = r.ts_start;
   a.ts_end[dst] = r.ts_end;
   a.corr[dst] = r.corr;
@@ -161,9 +171,9 @@ __global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
   a.seq[dst] = r.seq;
   a.stream[dst] = r.stream;
   a.kind[dst] = r.kind;
-  if (p < a.n_valid) {
-    u64 code = a.keys[p] >> a.sbits;
-    if (p == 0 || (a.keys[p - 1] >> a.sbits) != code) a.lane_start[code] = (int32_t)p;
+  if (p < nv) {
+    const u64 code = k >> a.sbits;
+    if (p == 0 || (kprev >> a.sbits) != code) a.lane_start[code] = (int32_t)p;
     if (r.kind == TA_KIND_LAUNCH) {
       slot = (int)(code >> a.tbits) * a.n_pids + a.tt->pid_rank[code & ((1ull << a.tbits) - 1)];
       mx = (u64)r.corr ^ (1ull << 63);
