@@ -37,7 +37,7 @@ WORKLOAD_TEXT = {
 }
 # ncu: dram__bytes_read.sum + dram__bytes_write.sum of one k_radix_pass launch divided by the
 # records it sorted, on the quarter-size case (profiles/radix_pass_c3_quarter.txt)
-RADIX_TRAFFIC_BYTES_PER_RECORD = 14.1
+RADIX_TRAFFIC_BYTES_PER_RECORD = 13.8
 
 
 def parse_args():
