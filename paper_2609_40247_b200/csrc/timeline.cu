@@ -109,7 +109,11 @@ __device__ __forceinline__ u32 gather_index(u64 k, const GatherArgs &a) {
   return (u32)(a.off[w] + (int64_t)(k & ((1ull << a.ibits) - 1)));
 }
 
-__global__ void __launch_bounds__(256) k_gather(GatherArgs a) {
+// eight CTAs per SM (32 registers): the kernel lives on occupancy, 42 or 51 registers measured slower
+#ifndef GT_MINB
+#define GT_MINB 8
+#endif
+__global__ void __launch_bounds__(256, GT_MINB) k_gather(GatherArgs a) {
   __shared__ int s_slot[8];
   __shared__ u64 s_mx[8], s_mn[8];
   if (ta_failed(a.status)) return;  // the sort gave up: the keys name no records
