@@ -234,10 +234,12 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   // kept: wait_ns; everything else is sized once the counts are known
   int64_t *wait_ns = (int64_t *)ta_dalloc(h, (size_t)nn * 8);
   if (!wait_ns) return TA_ERR_OOM;
-  TA_CHECK_CUDA(h, cudaMemsetAsync(wait_ns, 0, (size_t)nn * 8, st));
   out->wait_ns = wait_ns;
   const int64_t m = h->n_coll;  // kept COLL records, counted while the records were loaded
-  if (h->n_valid == 0 || h->n_comms == 0 || m == 0) return TA_OK;
+  if (h->n_valid == 0 || h->n_comms == 0 || m == 0) {
+    TA_CHECK_CUDA(h, cudaMemsetAsync(wait_ns, 0, (size_t)nn * 8, st));
+    return TA_OK;
+  }
 
   // 1. compaction
   size_t t1b = Carver::pad((size_t)m * 4) + scan_temp_bytes(n) + 256;
@@ -247,7 +249,8 @@ ta_status ta_run_collectives(ta_window *h, const ta_comm_size *sizes, int32_t n_
   u32 *pos_all = c1.take<u32>(m);
   ScanTemp s1;
   TA_TRY(scan_temp_init(h, c1.base + c1.off, n, &s1));
-  TA_TRY(launch_compact_kind(h, h->sorted.kind, h->n_valid, 1u << TA_KIND_COLL, pos_all, s1));
+  // the compaction pass clears the wait column on its way (one 0.5 GB memset less on c3)
+  TA_TRY(launch_compact_kind(h, h->sorted.kind, h->n_valid, 1u << TA_KIND_COLL, pos_all, s1, reinterpret_cast<i64 *>(wait_ns), nn));
   const std::vector<u64> &comm_sorted = h->h_comm_sorted;
 
   // expected communicator sizes by rank

@@ -208,9 +208,13 @@ __device__ __forceinline__ void storen_i32(int32_t *col, int64_t p0, int64_t n, 
 #define CK_THREADS 256
 #define CK_ITEMS 16
 #define CK_TILE (CK_THREADS * CK_ITEMS)
+// zero_col (may be null): an n-sized 64-bit column the caller needs cleared; the kernel reads two
+// bytes per record and has the bandwidth to write it on the way (positions below zero_n that its
+// tiles cover; the caller clears the rest).
 static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_t *kind, int64_t n_valid,
                                                              u32 kind_mask, u32 *pos_out, ScanTemp t,
-                                                             int32_t *status) {
+                                                             int32_t *status, i64 *zero_col,
+                                                             int64_t zero_n) {
   __shared__ u64 tmp[33];
   __shared__ u64 s_excl;
   __shared__ int s_tile, s_fail;
@@ -223,6 +227,14 @@ static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_
   if (s_fail) return;
   const int tile = s_tile;
   const int64_t p0 = (int64_t)tile * CK_TILE + (int64_t)tid * CK_ITEMS;
+  if (zero_col) {
+#pragma unroll
+    for (int k = 0; k < CK_ITEMS / 2; k++) {
+      const int64_t z = (int64_t)tile * CK_TILE + (int64_t)k * (2 * CK_THREADS) + 2 * tid;
+      if (z + 2 <= zero_n) *reinterpret_cast<longlong2 *>(zero_col + z) = make_longlong2(0, 0);
+      else if (z < zero_n) zero_col[z] = 0;
+    }
+  }
   int16_t kd[CK_ITEMS];
   load8_i16(kind, p0, n_valid, -1, kd);
   load8_i16(kind, p0 + 8, n_valid, -1, kd + 8);
@@ -249,11 +261,15 @@ static __global__ void __launch_bounds__(CK_THREADS) k_compact_kind(const int16_
     if (sel & (1u << j)) pos_out[o++] = (u32)(p0 + j);
 }
 static inline ta_status launch_compact_kind(ta_window *h, const int16_t *kind, int64_t n_valid,
-                                            u32 kind_mask, u32 *pos_out, ScanTemp t) {
+                                            u32 kind_mask, u32 *pos_out, ScanTemp t,
+                                            i64 *zero_col = nullptr, int64_t zero_n = 0) {
+  int64_t tiles = n_valid > 0 ? (n_valid + CK_TILE - 1) / CK_TILE : 0;
+  if (zero_col && tiles * CK_TILE < zero_n)  // what the tiles do not reach (the dropped tail)
+    TA_CHECK_CUDA(h, cudaMemsetAsync(zero_col + tiles * CK_TILE, 0, (size_t)(zero_n - tiles * CK_TILE) * 8,
+                                     h->stream));
   if (n_valid <= 0) return TA_OK;
-  int64_t tiles = (n_valid + CK_TILE - 1) / CK_TILE;
   k_compact_kind<<<TA_N (unsigned)tiles, CK_THREADS, 0, h->stream>>>(kind, n_valid, kind_mask, pos_out, t,
-                                                                   h->d_status);
+                                                                   h->d_status, zero_col, zero_n);
   TA_CHECK_CUDA(h, cudaGetLastError());
   return TA_OK;
 }
