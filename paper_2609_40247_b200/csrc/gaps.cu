@@ -121,9 +121,11 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
   // lanes of the items: walk forward from the tile's first lane
   int ln[GP_ITEMS];
   u64 run = 0;
+  unsigned lastmask = 0, firstmask = 0;  // items that end / begin their lane
   {
     int l = l0;
     int64_t next_off = l >= 0 ? (int64_t)a.lane_off[l + 1] : LLONG_MAX;
+    int64_t cur_off = l >= 0 ? (int64_t)a.lane_off[l] : 0;
     i64 w0 = 0, w1 = 0;
     int wl = -1;
 #pragma unroll
@@ -131,9 +133,11 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
       const int64_t p = p0 + j;
       ln[j] = -1;
       if (kd[j] >= 3) {
-        while (p >= next_off) { l++; next_off = a.lane_off[l + 1]; }
+        while (p >= next_off) { l++; cur_off = next_off; next_off = a.lane_off[l + 1]; }
         if (wl != l) { int w = a.lane_window[l]; w0 = a.t0[w]; w1 = a.t1[w]; wl = l; }
         ln[j] = l;
+        if (p + 1 == next_off) lastmask |= 1u << j;
+        if (p == cur_off) firstmask |= 1u << j;
         ce[j] = ce[j] < w1 ? ce[j] : w1;
         u64 v = ((u64)(l + 1) << 40) | (u64)(ce[j] - w0);
         run = run > v ? run : v;
@@ -190,7 +194,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
         g = s[j] > Pi ? s[j] - Pi : 0;
         const i64 from = s[j] > Pi ? s[j] : Pi;
         bz = ce[j] > from ? ce[j] - from : 0;
-        last = (p0 + j + 1 == (int64_t)a.lane_off[l + 1]);
+        last = (lastmask >> j) & 1u;
         if (last) tl = w1 - (Pi > ce[j] ? Pi : ce[j]);
         gap[j] = g;
         pre = max(pre, ((u64)(l + 1) << 40) | (u64)(ce[j] - w0));
@@ -199,9 +203,9 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
       }
       // long-gap list: the warp reserves its entries with one add on the cursor (the order of
       // the list does not matter, it is sorted afterwards)
-      {
+      if (__any_sync(0xffffffffu, lg || lt)) {  // rare: one vote decides for the warp
         const u32 m_g = __ballot_sync(0xffffffffu, lg), m_t = __ballot_sync(0xffffffffu, lt);
-        if (m_g | m_t) {
+        {
           const int wlane = threadIdx.x & 31;
           const u32 below = (1u << wlane) - 1u;
           u64 base = 0;
@@ -254,7 +258,7 @@ __global__ void __launch_bounds__(GP_THREADS, GP_MINB) k_gaps(GapArgs a) {
         a.lane_gaps[l].last_end = w1 - tl;
         a.lane_gaps[l].n_events = (i64)a.lane_off[l + 1] - (i64)a.lane_off[l];
       }
-      if (p0 + j == (int64_t)a.lane_off[l]) a.lane_gaps[l].first_start = s[j];
+      if ((firstmask >> j) & 1u) a.lane_gaps[l].first_start = s[j];
     }
   }
   if (a.list_only) return;
